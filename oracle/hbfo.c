@@ -1,0 +1,514 @@
+/*
+ * hbfo.c -- sequential CPU oracle of the HBF service model.  TEST INFRASTRUCTURE ONLY; see hbfo.h.
+ *
+ * Every step is the plain definition: ranges are found by linear scan, addresses are decoded with
+ * '/' and '%', each queue is a list sorted by (issue time, batch index) and served one access at a
+ * time, the thermal field is advanced cell by cell in double precision.  No blocking, no fusion.
+ */
+#include "hbfo.h"
+
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+
+typedef struct { uint64_t base, length, media_offset; uint32_t perms, kind, stream_tag, id; } range_t;
+
+struct hbfo_ctx {
+    hbfo_config_t cfg;
+    uint32_t n_queues, n_dies;
+    size_t n_cells;
+    range_t ranges[HBFO_MAX_RANGES];
+    uint32_t n_ranges, next_range_id;
+    int64_t *busy_until;       /* [n_queues] */
+    int64_t *pending_pj;       /* [n_dies]   */
+    int32_t mode; int64_t q_ppm;
+    hbfo_batch_result_t last;
+    uint32_t *order; uint64_t order_count, order_cap;
+    /* thermal */
+    int thermal;
+    double *C, *Gx, *Gy, *Gs, *T, *Tn, *P;
+    int32_t *cell_region, *die_region, *region_kind;
+    double *region_idle_w, *region_cells;
+    double euler_limit_s;
+};
+
+/* ---- small helpers ---------------------------------------------------------------------- */
+
+static int is_pow2_u32(uint32_t v) { return v != 0 && (v & (v - 1)) == 0; }
+
+static int64_t ceil_div_i64(int64_t a, int64_t b) { return (a + b - 1) / b; }   /* a >= 0, b > 0 */
+
+static double *dup_f32_as_f64(const float *src, size_t n) {
+    double *d = (double *)malloc(n * sizeof(double));
+    if (d) for (size_t i = 0; i < n; ++i) d[i] = (double)src[i];
+    return d;
+}
+static int32_t *dup_i32(const int32_t *src, size_t n) {
+    int32_t *d = (int32_t *)malloc(n * sizeof(int32_t));
+    if (d) memcpy(d, src, n * sizeof(int32_t));
+    return d;
+}
+
+const char *hbfo_strerror(int code) {
+    switch (code) {
+    case HBFO_OK: return "ok";
+    case HBFO_E_INVAL: return "invalid argument";
+    case HBFO_E_RANGE_OVERLAP: return "range overlaps a registered range";
+    case HBFO_E_RANGE_FULL: return "range table full";
+    case HBFO_E_CAPACITY: return "range exceeds media capacity";
+    case HBFO_E_WORKSPACE: return "workspace too small";
+    case HBFO_E_CUDA: return "device error";
+    case HBFO_E_ACCESS_FAULT: return "batch refused: fail-closed access";
+    case HBFO_E_THROTTLED: return "throttled: new reservations withheld";
+    case HBFO_E_LINK_SHUTDOWN: return "link shutdown";
+    case HBFO_E_TIMEOUT: return "bounded wait expired";
+    case HBFO_E_NOMEM: return "out of memory";
+    default: return "unknown";
+    }
+}
+
+/* ---- create / destroy --------------------------------------------------------------------- */
+
+static void free_ctx(hbfo_ctx *c) {
+    if (!c) return;
+    free(c->busy_until); free(c->pending_pj); free(c->order);
+    free(c->C); free(c->Gx); free(c->Gy); free(c->Gs); free(c->T); free(c->Tn); free(c->P);
+    free(c->cell_region); free(c->die_region); free(c->region_kind);
+    free(c->region_idle_w); free(c->region_cells);
+    free(c);
+}
+
+int hbfo_create(const hbfo_config_t *cfg, hbfo_ctx **out) {
+    if (!cfg || !out) return HBFO_E_INVAL;
+    if (cfg->channels == 0 || cfg->dies == 0 || cfg->planes == 0) return HBFO_E_INVAL;
+    if (!is_pow2_u32(cfg->page_bytes) || !is_pow2_u32(cfg->stripe_bytes)) return HBFO_E_INVAL;
+    if (cfg->stripe_bytes < cfg->page_bytes) return HBFO_E_INVAL;
+    if (!is_pow2_u32(cfg->read_granule) || !is_pow2_u32(cfg->prog_granule)) return HBFO_E_INVAL;
+    if (cfg->queue_level > 1) return HBFO_E_INVAL;
+    if (cfg->t_read_ns <= 0 || cfg->t_prog_ns <= 0 || cfg->chan_bytes_per_us == 0) return HBFO_E_INVAL;
+    if (cfg->e_cmd_read_pj < 0 || cfg->e_byte_read_pj < 0 || cfg->e_cmd_prog_pj < 0 || cfg->e_byte_prog_pj < 0)
+        return HBFO_E_INVAL;
+    if (cfg->q_light_ppm < 1 || cfg->q_light_ppm > 1000000) return HBFO_E_INVAL;
+    uint64_t nd = (uint64_t)cfg->channels * cfg->dies;
+    uint64_t nq = cfg->queue_level == 0 ? nd * cfg->planes : nd;
+    if (nq > 65536 || nd > 65536) return HBFO_E_INVAL;
+
+    hbfo_ctx *c = (hbfo_ctx *)calloc(1, sizeof(*c));
+    if (!c) return HBFO_E_NOMEM;
+    c->cfg = *cfg;
+    c->n_queues = (uint32_t)nq; c->n_dies = (uint32_t)nd;
+    c->busy_until = (int64_t *)calloc(nq, sizeof(int64_t));
+    c->pending_pj = (int64_t *)calloc(nd, sizeof(int64_t));
+    if (!c->busy_until || !c->pending_pj) { free_ctx(c); return HBFO_E_NOMEM; }
+    c->mode = HBFO_MODE_NORMAL; c->q_ppm = 1000000;
+
+    c->thermal = cfg->cell_C != NULL;
+    if (c->thermal) {
+        if (cfg->grid_h == 0 || cfg->grid_w == 0 || cfg->n_sub == 0 || cfg->n_regions == 0 ||
+            !cfg->cell_Gx || !cfg->cell_Gy || !cfg->cell_Gsink || !cfg->cell_region || !cfg->die_region ||
+            !cfg->region_kind || !cfg->region_idle_w) { free_ctx(c); return HBFO_E_INVAL; }
+        if (!(cfg->rtt_c < cfg->ltt_c && cfg->ltt_c < cfg->stt_c && cfg->stt_c < cfg->shutdown_c)) {
+            free_ctx(c); return HBFO_E_INVAL;
+        }
+        size_t nc = (size_t)cfg->grid_h * cfg->grid_w;
+        c->n_cells = nc;
+        c->C = dup_f32_as_f64(cfg->cell_C, nc);  c->Gx = dup_f32_as_f64(cfg->cell_Gx, nc);
+        c->Gy = dup_f32_as_f64(cfg->cell_Gy, nc); c->Gs = dup_f32_as_f64(cfg->cell_Gsink, nc);
+        c->T = (double *)malloc(nc * sizeof(double)); c->Tn = (double *)malloc(nc * sizeof(double));
+        c->P = (double *)calloc(nc, sizeof(double));
+        c->cell_region = dup_i32(cfg->cell_region, nc);
+        c->die_region = dup_i32(cfg->die_region, nd);
+        c->region_kind = dup_i32(cfg->region_kind, cfg->n_regions);
+        c->region_idle_w = dup_f32_as_f64(cfg->region_idle_w, cfg->n_regions);
+        c->region_cells = (double *)calloc(cfg->n_regions, sizeof(double));
+        if (!c->C || !c->Gx || !c->Gy || !c->Gs || !c->T || !c->Tn || !c->P || !c->cell_region ||
+            !c->die_region || !c->region_kind || !c->region_idle_w || !c->region_cells) {
+            free_ctx(c); return HBFO_E_NOMEM;
+        }
+        for (size_t i = 0; i < nc; ++i) {
+            if (!(c->C[i] > 0.0) || c->Gx[i] < 0.0 || c->Gy[i] < 0.0 || c->Gs[i] < 0.0) { free_ctx(c); return HBFO_E_INVAL; }
+            int32_t g = c->cell_region[i];
+            if (g >= (int32_t)cfg->n_regions) { free_ctx(c); return HBFO_E_INVAL; }
+            if (g >= 0) c->region_cells[g] += 1.0;
+            c->T[i] = (double)cfg->ambient_c;          /* the field starts at ambient everywhere */
+        }
+        for (uint64_t d = 0; d < nd; ++d) {
+            int32_t g = c->die_region[d];
+            if (g < 0 || g >= (int32_t)cfg->n_regions || c->region_cells[g] == 0.0) { free_ctx(c); return HBFO_E_INVAL; }
+        }
+        /* largest stable explicit step: min over cells of C / (sum of conductances on the cell) */
+        uint32_t H = cfg->grid_h, W = cfg->grid_w;
+        double lim = INFINITY;
+        for (uint32_t y = 0; y < H; ++y) for (uint32_t x = 0; x < W; ++x) {
+            size_t i = (size_t)y * W + x;
+            double g = c->Gs[i];
+            if (x + 1 < W) g += c->Gx[i];
+            if (x > 0)     g += c->Gx[i - 1];
+            if (y + 1 < H) g += c->Gy[i];
+            if (y > 0)     g += c->Gy[i - W];
+            if (g > 0.0 && c->C[i] / g < lim) lim = c->C[i] / g;
+        }
+        c->euler_limit_s = lim;
+    }
+    *out = c;
+    return HBFO_OK;
+}
+
+int hbfo_destroy(hbfo_ctx *ctx) { free_ctx(ctx); return HBFO_OK; }
+
+double hbfo_euler_limit_ns(hbfo_ctx *ctx) { return ctx && ctx->thermal ? ctx->euler_limit_s * 1e9 : 0.0; }
+
+int hbfo_reset(hbfo_ctx *c) {
+    if (!c) return HBFO_E_INVAL;
+    memset(c->busy_until, 0, c->n_queues * sizeof(int64_t));
+    memset(c->pending_pj, 0, c->n_dies * sizeof(int64_t));
+    c->mode = HBFO_MODE_NORMAL; c->q_ppm = 1000000;
+    memset(&c->last, 0, sizeof(c->last));
+    c->order_count = 0;
+    if (c->thermal) for (size_t i = 0; i < c->n_cells; ++i) c->T[i] = (double)c->cfg.ambient_c;
+    return HBFO_OK;
+}
+
+int hbfo_force_mode(hbfo_ctx *c, int32_t mode, int64_t q_ppm) {
+    if (!c || mode < 0 || mode > 3 || q_ppm < 1 || q_ppm > 1000000) return HBFO_E_INVAL;
+    c->mode = mode; c->q_ppm = q_ppm;
+    return HBFO_OK;
+}
+
+int hbfo_get_mode(hbfo_ctx *c, int32_t *mode, int64_t *q_ppm) {
+    if (!c) return HBFO_E_INVAL;
+    if (mode) *mode = c->mode;
+    if (q_ppm) *q_ppm = c->q_ppm;
+    return HBFO_OK;
+}
+
+/* ---- ranges (Design D1) -------------------------------------------------------------------- */
+
+int hbfo_register_range(hbfo_ctx *c, uint64_t base, uint64_t length, uint32_t perms, uint32_t kind,
+                        uint32_t stream_tag, uint64_t media_offset, uint32_t *out_id) {
+    if (!c || length == 0 || (perms & ~3u) || perms == 0 || kind > 1) return HBFO_E_INVAL;
+    if (base + length < base) return HBFO_E_INVAL;                       /* wraps the address space */
+    if (media_offset + length < media_offset) return HBFO_E_INVAL;
+    if (c->cfg.capacity_bytes && media_offset + length > c->cfg.capacity_bytes) return HBFO_E_CAPACITY;
+    if (c->n_ranges == HBFO_MAX_RANGES) return HBFO_E_RANGE_FULL;
+    for (uint32_t g = 0; g < c->n_ranges; ++g) {
+        const range_t *r = &c->ranges[g];
+        if (base < r->base + r->length && r->base < base + length) return HBFO_E_RANGE_OVERLAP;
+    }
+    range_t *r = &c->ranges[c->n_ranges++];
+    r->base = base; r->length = length; r->media_offset = media_offset;
+    r->perms = perms; r->kind = kind; r->stream_tag = stream_tag; r->id = c->next_range_id++;
+    if (out_id) *out_id = r->id;
+    return HBFO_OK;
+}
+
+int hbfo_clear_ranges(hbfo_ctx *c) { if (!c) return HBFO_E_INVAL; c->n_ranges = 0; return HBFO_OK; }
+
+/* Classification of one access.  Outside every range: native path.  Inside a range: modeled only
+ * if the whole byte span lies in that one range and the operation is permitted; otherwise it fails. */
+int hbfo_classify(hbfo_ctx *c, const hbfo_access_t *a, int32_t *range_id) {
+    if (range_id) *range_id = -1;
+    if (a->bytes == 0 || (a->flags & ~1u) || a->issue_ns < 0 || a->issue_ns >= HBFO_ISSUE_LIMIT)
+        return HBFO_ST_UNSUPPORTED;
+    for (uint32_t g = 0; g < c->n_ranges; ++g) {                         /* linear scan, on purpose */
+        const range_t *r = &c->ranges[g];
+        if (a->addr >= r->base && a->addr - r->base < r->length) {
+            uint64_t rel = a->addr - r->base;
+            if (range_id) *range_id = (int32_t)g;
+            if ((uint64_t)a->bytes > r->length - rel) return HBFO_ST_FAULT_PARTIAL;   /* leaves the range (or wraps) */
+            uint32_t need = (a->flags & 1u) ? 2u : 1u;                   /* bit0 read, bit1 program */
+            if (!(r->perms & need)) return HBFO_ST_FAULT_PERM;
+            return HBFO_ST_READY;
+        }
+    }
+    return HBFO_ST_NATIVE;
+}
+
+/* ---- decode and service terms --------------------------------------------------------------- */
+
+int hbfo_decode(hbfo_ctx *c, uint64_t off, uint32_t bytes, uint32_t *channel, uint32_t *die,
+                uint32_t *plane, uint64_t *row, uint64_t *page, uint64_t *npages, uint32_t *queue) {
+    if (!c) return HBFO_E_INVAL;
+    const uint64_t Cn = c->cfg.channels, Dn = c->cfg.dies, Pn = c->cfg.planes;
+    const uint64_t stripe = c->cfg.stripe_bytes, pg = c->cfg.page_bytes;
+    uint64_t u  = off / stripe;                     /* stripe unit: channel first, then die, then plane */
+    uint64_t ch = u % Cn;
+    uint64_t di = (u / Cn) % Dn;
+    uint64_t pl = (u / (Cn * Dn)) % Pn;
+    uint64_t rw = u / (Cn * Dn * Pn);
+    uint64_t pa = rw * (stripe / pg) + (off % stripe) / pg;
+    uint64_t np = ((off % pg) + (uint64_t)bytes + pg - 1) / pg;
+    uint64_t q  = c->cfg.queue_level == 0 ? (ch * Dn + di) * Pn + pl : ch * Dn + di;
+    if (channel) *channel = (uint32_t)ch;
+    if (die) *die = (uint32_t)di;
+    if (plane) *plane = (uint32_t)pl;
+    if (row) *row = rw;
+    if (page) *page = pa;
+    if (npages) *npages = np;
+    if (queue) *queue = (uint32_t)q;
+    return HBFO_OK;
+}
+
+int hbfo_service_terms(hbfo_ctx *c, uint32_t bytes, uint64_t npages, uint32_t op, int64_t q_ppm,
+                       int64_t *charged_bytes, int64_t *xfer_ns, int64_t *s_ns, int64_t *energy_pj) {
+    if (!c || q_ppm < 1 || op > 1) return HBFO_E_INVAL;
+    int64_t gran = op ? (int64_t)c->cfg.prog_granule : (int64_t)c->cfg.read_granule;
+    int64_t cb   = ceil_div_i64((int64_t)bytes, gran) * gran;           /* bytes charged: whole granules */
+    int64_t xfer = ceil_div_i64(cb * 1000, (int64_t)c->cfg.chan_bytes_per_us);
+    int64_t s0   = (int64_t)npages * (op ? c->cfg.t_prog_ns : c->cfg.t_read_ns);
+    int64_t s    = ceil_div_i64(s0 * 1000000, q_ppm);                   /* Eq. 3 */
+    int64_t e    = op ? c->cfg.e_cmd_prog_pj + c->cfg.e_byte_prog_pj * cb
+                      : c->cfg.e_cmd_read_pj + c->cfg.e_byte_read_pj * cb;
+    if (charged_bytes) *charged_bytes = cb;
+    if (xfer_ns) *xfer_ns = xfer;
+    if (s_ns) *s_ns = s;
+    if (energy_pj) *energy_pj = e;
+    return HBFO_OK;
+}
+
+/* ---- submit --------------------------------------------------------------------------------- */
+
+typedef struct { int64_t issue_ns; uint32_t idx; } qent_t;
+
+static int cmp_qent(const void *pa, const void *pb) {
+    const qent_t *a = (const qent_t *)pa, *b = (const qent_t *)pb;
+    if (a->issue_ns != b->issue_ns) return a->issue_ns < b->issue_ns ? -1 : 1;
+    if (a->idx != b->idx) return a->idx < b->idx ? -1 : 1;
+    return 0;
+}
+
+int hbfo_submit_batch(hbfo_ctx *c, const hbfo_access_t *acc, uint64_t n, int64_t *completion_ns,
+                      int64_t *stall_ns, uint8_t *status, hbfo_die_stats_t *die_stats) {
+    if (!c || (n && (!acc || !completion_ns || !stall_ns)) || n > 0xffffffffull) return HBFO_E_INVAL;
+    hbfo_batch_result_t res; memset(&res, 0, sizeof(res));
+    const int64_t q = c->q_ppm;                               /* snapshot before any reservation */
+    res.mode = c->mode; res.q_ppm = q;
+    if (c->mode == HBFO_MODE_SHUTDOWN) { res.code = HBFO_E_LINK_SHUTDOWN; c->last = res; return res.code; }
+    if (c->mode == HBFO_MODE_SEVERE)   { res.code = HBFO_E_THROTTLED;     c->last = res; return res.code; }
+
+    uint8_t *st = (uint8_t *)malloc(n ? n : 1);
+    int32_t *rg = (int32_t *)malloc((n ? n : 1) * sizeof(int32_t));
+    if (!st || !rg) { free(st); free(rg); return HBFO_E_NOMEM; }
+
+    /* validate pass: nothing changes if any access fails */
+    uint64_t n_fault = 0, n_native = 0, n_ready = 0;
+    for (uint64_t i = 0; i < n; ++i) {
+        st[i] = (uint8_t)hbfo_classify(c, &acc[i], &rg[i]);
+        if (st[i] == HBFO_ST_NATIVE) ++n_native; else if (st[i] == HBFO_ST_READY) ++n_ready; else ++n_fault;
+    }
+    if (status) memcpy(status, st, n);
+    if (die_stats) memset(die_stats, 0, c->n_dies * sizeof(hbfo_die_stats_t));
+    if (n_fault) {
+        memset(completion_ns, 0, n * sizeof(int64_t)); memset(stall_ns, 0, n * sizeof(int64_t));
+        res.code = HBFO_E_ACCESS_FAULT; res.n_fault = n_fault; res.n_native = n_native;
+        c->last = res; free(st); free(rg);
+        return res.code;
+    }
+
+    /* decode + terms */
+    uint32_t *queue = (uint32_t *)malloc((n ? n : 1) * sizeof(uint32_t));
+    uint32_t *die   = (uint32_t *)malloc((n ? n : 1) * sizeof(uint32_t));
+    int64_t *a_ns = (int64_t *)malloc((n ? n : 1) * sizeof(int64_t));
+    int64_t *s_ns = (int64_t *)malloc((n ? n : 1) * sizeof(int64_t));
+    int64_t *post = (int64_t *)malloc((n ? n : 1) * sizeof(int64_t));
+    int64_t *cbs  = (int64_t *)malloc((n ? n : 1) * sizeof(int64_t));
+    int64_t *eng  = (int64_t *)malloc((n ? n : 1) * sizeof(int64_t));
+    uint64_t *cnt = (uint64_t *)calloc((size_t)c->n_queues + 1, sizeof(uint64_t));
+    qent_t *ent = (qent_t *)malloc((n_ready ? n_ready : 1) * sizeof(qent_t));
+    int rc = HBFO_OK;
+    if (!queue || !die || !a_ns || !s_ns || !post || !cbs || !eng || !cnt || !ent) { rc = HBFO_E_NOMEM; goto done; }
+    if (c->order_cap < n_ready) {
+        free(c->order); c->order = (uint32_t *)malloc((n_ready ? n_ready : 1) * sizeof(uint32_t));
+        if (!c->order) { c->order_cap = 0; rc = HBFO_E_NOMEM; goto done; }
+        c->order_cap = n_ready;
+    }
+
+    for (uint64_t i = 0; i < n; ++i) {
+        if (st[i] != HBFO_ST_READY) continue;
+        const range_t *r = &c->ranges[rg[i]];
+        uint64_t off = r->media_offset + (acc[i].addr - r->base);
+        uint32_t ch, di, pl, qu; uint64_t np;
+        hbfo_decode(c, off, acc[i].bytes, &ch, &di, &pl, NULL, NULL, &np, &qu);
+        uint32_t op = acc[i].flags & 1u;
+        int64_t cb, xfer, s, e;
+        hbfo_service_terms(c, acc[i].bytes, np, op, q, &cb, &xfer, &s, &e);
+        queue[i] = qu; die[i] = ch * c->cfg.dies + di;
+        s_ns[i] = s; cbs[i] = cb; eng[i] = e;
+        if (op) { a_ns[i] = acc[i].issue_ns + xfer; post[i] = 0; }       /* program: data moves in first */
+        else    { a_ns[i] = acc[i].issue_ns;        post[i] = xfer; }    /* read: data moves out after  */
+        cnt[qu + 1]++;
+    }
+
+    /* per-queue lists in index order, then each sorted by (issue, index) */
+    for (uint32_t r = 0; r < c->n_queues; ++r) cnt[r + 1] += cnt[r];
+    {
+        uint64_t *fill = (uint64_t *)malloc((size_t)c->n_queues * sizeof(uint64_t));
+        if (!fill) { rc = HBFO_E_NOMEM; goto done; }
+        memcpy(fill, cnt, (size_t)c->n_queues * sizeof(uint64_t));
+        for (uint64_t i = 0; i < n; ++i) {
+            if (st[i] != HBFO_ST_READY) continue;
+            qent_t *e = &ent[fill[queue[i]]++];
+            e->issue_ns = acc[i].issue_ns; e->idx = (uint32_t)i;
+        }
+        free(fill);
+    }
+    for (uint32_t r = 0; r < c->n_queues; ++r)
+        qsort(ent + cnt[r], (size_t)(cnt[r + 1] - cnt[r]), sizeof(qent_t), cmp_qent);
+
+    /* serve each queue, one access at a time */
+    hbfo_die_stats_t *ds = (hbfo_die_stats_t *)calloc(c->n_dies, sizeof(hbfo_die_stats_t));
+    if (!ds) { rc = HBFO_E_NOMEM; goto done; }
+    for (uint64_t i = 0; i < n; ++i)
+        if (st[i] == HBFO_ST_NATIVE) { completion_ns[i] = acc[i].issue_ns; stall_ns[i] = 0; }
+    for (uint32_t r = 0; r < c->n_queues; ++r) {
+        int64_t B = c->busy_until[r];
+        for (uint64_t k = cnt[r]; k < cnt[r + 1]; ++k) {
+            uint32_t i = ent[k].idx;
+            int64_t start = a_ns[i] > B ? a_ns[i] : B;
+            B = start + s_ns[i];
+            int64_t done_ns = B + post[i];
+            completion_ns[i] = done_ns;
+            stall_ns[i] = done_ns - acc[i].issue_ns;
+            hbfo_die_stats_t *d = &ds[die[i]];
+            d->busy_ns += s_ns[i]; d->energy_pj += eng[i];
+            if (acc[i].flags & 1u) { d->bytes_prog += cbs[i]; d->n_prog += 1; }
+            else                   { d->bytes_read += cbs[i]; d->n_read += 1; }
+            res.modeled_ns += stall_ns[i]; res.service_ns += s_ns[i];
+            if (done_ns > res.max_completion_ns) res.max_completion_ns = done_ns;
+            c->order[k] = i;
+        }
+        c->busy_until[r] = B;
+    }
+    c->order_count = n_ready;
+    for (uint32_t d = 0; d < c->n_dies; ++d) c->pending_pj[d] += ds[d].energy_pj;
+    if (die_stats) memcpy(die_stats, ds, c->n_dies * sizeof(hbfo_die_stats_t));
+    free(ds);
+    res.code = HBFO_OK; res.n_native = n_native; res.n_modeled = n_ready;
+    c->last = res;
+
+done:
+    free(st); free(rg); free(queue); free(die); free(a_ns); free(s_ns); free(post); free(cbs); free(eng);
+    free(cnt); free(ent);
+    return rc;
+}
+
+int hbfo_last_result(hbfo_ctx *c, hbfo_batch_result_t *out) {
+    if (!c || !out) return HBFO_E_INVAL;
+    *out = c->last;
+    return c->last.code;
+}
+
+int hbfo_last_order(hbfo_ctx *c, uint32_t *order, uint64_t cap, uint64_t *count) {
+    if (!c || !count) return HBFO_E_INVAL;
+    *count = c->order_count;
+    if (order) {
+        if (cap < c->order_count) return HBFO_E_INVAL;
+        memcpy(order, c->order, c->order_count * sizeof(uint32_t));
+    }
+    return HBFO_OK;
+}
+
+int hbfo_get_busy_until(hbfo_ctx *c, int64_t *out, uint64_t cap) {
+    if (!c || !out || cap < c->n_queues) return HBFO_E_INVAL;
+    memcpy(out, c->busy_until, c->n_queues * sizeof(int64_t));
+    return HBFO_OK;
+}
+int hbfo_get_pending_energy(hbfo_ctx *c, int64_t *out, uint64_t cap) {
+    if (!c || !out || cap < c->n_dies) return HBFO_E_INVAL;
+    memcpy(out, c->pending_pj, c->n_dies * sizeof(int64_t));
+    return HBFO_OK;
+}
+int hbfo_get_temps(hbfo_ctx *c, double *out, uint64_t cap) {
+    if (!c || !c->thermal || !out || cap < c->n_cells) return HBFO_E_INVAL;
+    memcpy(out, c->T, c->n_cells * sizeof(double));
+    return HBFO_OK;
+}
+int hbfo_set_temps(hbfo_ctx *c, const double *in, uint64_t count) {
+    if (!c || !c->thermal || !in || count != c->n_cells) return HBFO_E_INVAL;
+    memcpy(c->T, in, c->n_cells * sizeof(double));
+    return HBFO_OK;
+}
+
+/* ---- thermal step (Design D3, Eq. 1) ------------------------------------------------------- */
+
+int64_t hbfo_quantise_mk(double t_c) { return (int64_t)floor(t_c * 1000.0 + 0.5); }   /* round half up */
+
+int32_t hbfo_next_mode(hbfo_ctx *c, int32_t mode, int64_t t) {
+    const int64_t rtt = hbfo_quantise_mk((double)c->cfg.rtt_c), ltt = hbfo_quantise_mk((double)c->cfg.ltt_c);
+    const int64_t stt = hbfo_quantise_mk((double)c->cfg.stt_c), shut = hbfo_quantise_mk((double)c->cfg.shutdown_c);
+    if (mode == HBFO_MODE_SHUTDOWN) return HBFO_MODE_SHUTDOWN;            /* absorbing */
+    if (t >= shut) return HBFO_MODE_SHUTDOWN;
+    switch (mode) {
+    case HBFO_MODE_NORMAL:
+        if (t >= stt) return HBFO_MODE_SEVERE;
+        if (t >= ltt) return HBFO_MODE_LIGHT;
+        return HBFO_MODE_NORMAL;
+    case HBFO_MODE_LIGHT:
+        if (t >= stt) return HBFO_MODE_SEVERE;
+        if (t <= rtt) return HBFO_MODE_NORMAL;
+        return HBFO_MODE_LIGHT;
+    case HBFO_MODE_SEVERE:
+        if (t <= rtt) return HBFO_MODE_NORMAL;
+        if (t <= ltt) return HBFO_MODE_LIGHT;
+        return HBFO_MODE_SEVERE;
+    default: return mode;
+    }
+}
+
+int hbfo_thermal_step(hbfo_ctx *c, int64_t dt_ns, const float *ext_power_w, uint32_t n_ext,
+                      double *temps_out, double hot_c_out[3]) {
+    if (!c || !c->thermal || dt_ns <= 0) return HBFO_E_INVAL;
+    if (n_ext != 0 && (n_ext != c->cfg.n_regions || !ext_power_w)) return HBFO_E_INVAL;
+    const uint32_t H = c->cfg.grid_h, W = c->cfg.grid_w, NR = c->cfg.n_regions;
+    const double dt_s = (double)dt_ns * 1e-9;
+    const double dt_sub = dt_s / (double)c->cfg.n_sub;
+    if (dt_sub > c->euler_limit_s) return HBFO_E_INVAL;                    /* explicit step would be unstable */
+    const double amb = (double)c->cfg.ambient_c;
+
+    /* power map: energy of the window / window length + idle + external, spread over the region */
+    double *Pr = (double *)calloc(NR, sizeof(double));
+    if (!Pr) return HBFO_E_NOMEM;
+    for (uint32_t d = 0; d < c->n_dies; ++d)
+        Pr[c->die_region[d]] += ((double)c->pending_pj[d] * 1e-12) / dt_s;
+    for (uint32_t g = 0; g < NR; ++g) {
+        Pr[g] += c->region_idle_w[g];
+        if (n_ext) Pr[g] += (double)ext_power_w[g];
+    }
+    for (size_t i = 0; i < c->n_cells; ++i) {
+        int32_t g = c->cell_region[i];
+        c->P[i] = g >= 0 ? Pr[g] / c->region_cells[g] : 0.0;
+    }
+    free(Pr);
+    memset(c->pending_pj, 0, c->n_dies * sizeof(int64_t));
+
+    /* explicit Euler, every cell from the previous substep's field */
+    for (uint32_t k = 0; k < c->cfg.n_sub; ++k) {
+        for (uint32_t y = 0; y < H; ++y) for (uint32_t x = 0; x < W; ++x) {
+            size_t i = (size_t)y * W + x;
+            double Ti = c->T[i], flow = 0.0;
+            if (x + 1 < W) flow += c->Gx[i]     * (Ti - c->T[i + 1]);
+            if (x > 0)     flow += c->Gx[i - 1] * (Ti - c->T[i - 1]);
+            if (y + 1 < H) flow += c->Gy[i]     * (Ti - c->T[i + W]);
+            if (y > 0)     flow += c->Gy[i - W] * (Ti - c->T[i - W]);
+            c->Tn[i] = Ti + dt_sub / c->C[i] * (c->P[i] - flow - c->Gs[i] * (Ti - amb));
+        }
+        double *t = c->T; c->T = c->Tn; c->Tn = t;
+    }
+
+    /* hotspots per medium; the HBF one drives the controller */
+    double hot[3] = { -INFINITY, -INFINITY, -INFINITY };
+    for (size_t i = 0; i < c->n_cells; ++i) {
+        int32_t g = c->cell_region[i];
+        if (g < 0) continue;
+        int32_t k = c->region_kind[g];
+        int slot = k == HBFO_KIND_HBF ? 0 : k == HBFO_KIND_HBM ? 1 : k == HBFO_KIND_GPU ? 2 : -1;
+        if (slot >= 0 && c->T[i] > hot[slot]) hot[slot] = c->T[i];
+    }
+    for (int k = 0; k < 3; ++k) if (hot[k] == -INFINITY) hot[k] = amb;
+    c->mode = hbfo_next_mode(c, c->mode, hbfo_quantise_mk(hot[0]));
+    if (c->mode == HBFO_MODE_NORMAL) c->q_ppm = 1000000;
+    else if (c->mode == HBFO_MODE_LIGHT) c->q_ppm = c->cfg.q_light_ppm;
+    if (temps_out) memcpy(temps_out, c->T, c->n_cells * sizeof(double));
+    if (hot_c_out) { hot_c_out[0] = hot[0]; hot_c_out[1] = hot[1]; hot_c_out[2] = hot[2]; }
+    return HBFO_OK;
+}

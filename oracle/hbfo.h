@@ -1,0 +1,107 @@
+/*
+ * hbfo -- sequential CPU oracle of the HBF service model.  TEST INFRASTRUCTURE ONLY.
+ *
+ * This is the plain definition of what the GPU library computes, one access at a time, written
+ * from the paper (HBFSim) and from the stated readings of what the paper leaves open.  It shares
+ * no code, header, table or helper with the CUDA path.  Only tests, the smoke check and the
+ * benchmark's CPU-baseline leg may call it; the product path never does.
+ *
+ * What follows the paper directly:
+ *   - range classification, fail-closed            (Design D1, "An Explicit and Fail-Closed Boundary")
+ *   - ticket = slot index, result lands at the same index   (Implementation, control region)
+ *   - thermal service scaling s_T = ceil(s*10^6/q)  (Eq. 3)
+ *   - throttle modes Normal/Light/Severe/Shutdown   (Design D3)
+ *   - event energy E = E_command + e_byte*bytes, P = E/dt + P_idle   (Design D3)
+ *   - RC node equation                              (Eq. 1)
+ * What is a reading (the paper gives no equations for the queue itself, no plane/die timing and
+ * no threshold values): the FIFO recurrence start = max(arrival, busy_until), the address
+ * interleave, data transfer as pure latency, granule rounding, the threshold numbers.
+ *
+ * Pins: hand-worked single-queue examples, the closed form n*tR + transfer, queue invariants,
+ * an independent event-driven brute force on tiny inputs, the M/D/1 mean wait, the printed power
+ * figure 37.256 W at 384 GB/s, thermal steady state against a direct linear solve and the lumped
+ * closed form.  Parity unpinned (no value in the paper, fixed by the committed profile only):
+ * program energy per byte, the threshold temperatures, q_light, the floorplan constants.
+ *
+ * All times int64 ns on one shared origin; energies int64 pJ; temperatures double, deg C.
+ */
+#ifndef HBFO_H
+#define HBFO_H
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum { HBFO_OK = 0, HBFO_E_INVAL = -1, HBFO_E_RANGE_OVERLAP = -2, HBFO_E_RANGE_FULL = -3,
+       HBFO_E_CAPACITY = -4, HBFO_E_WORKSPACE = -5, HBFO_E_CUDA = -6, HBFO_E_ACCESS_FAULT = -7,
+       HBFO_E_THROTTLED = -8, HBFO_E_LINK_SHUTDOWN = -9, HBFO_E_TIMEOUT = -10, HBFO_E_NOMEM = -11 };
+enum { HBFO_ST_NATIVE = 0, HBFO_ST_READY = 1, HBFO_ST_FAULT_PARTIAL = 2, HBFO_ST_FAULT_PERM = 3,
+       HBFO_ST_UNSUPPORTED = 4 };
+enum { HBFO_MODE_NORMAL = 0, HBFO_MODE_LIGHT = 1, HBFO_MODE_SEVERE = 2, HBFO_MODE_SHUTDOWN = 3 };
+enum { HBFO_KIND_NONE = 0, HBFO_KIND_GPU = 1, HBFO_KIND_HBM = 2, HBFO_KIND_HBF = 3 };
+#define HBFO_MAX_RANGES 64
+#define HBFO_ISSUE_LIMIT (((int64_t)1) << 47)   /* issue_ns must lie in [0, 2^47) */
+
+typedef struct { uint64_t addr; int64_t issue_ns; uint32_t bytes; uint32_t flags; } hbfo_access_t;
+typedef struct { int64_t busy_ns, bytes_read, bytes_prog, energy_pj, n_read, n_prog; } hbfo_die_stats_t;
+typedef struct {
+    int32_t code, mode; int64_t q_ppm; uint64_t n_native, n_modeled, n_fault;
+    int64_t modeled_ns, service_ns, max_completion_ns;
+} hbfo_batch_result_t;
+
+typedef struct {
+    uint32_t channels, dies, planes, page_bytes, stripe_bytes, queue_level;
+    uint64_t capacity_bytes;
+    int64_t  t_read_ns, t_prog_ns;
+    uint64_t chan_bytes_per_us;
+    uint32_t read_granule, prog_granule;
+    int64_t  e_cmd_read_pj, e_byte_read_pj, e_cmd_prog_pj, e_byte_prog_pj;
+    uint32_t grid_h, grid_w, n_sub, n_regions;
+    float    ambient_c, rtt_c, ltt_c, stt_c, shutdown_c;
+    int64_t  q_light_ppm;
+    const float *cell_C, *cell_Gx, *cell_Gy, *cell_Gsink;      /* [grid_h*grid_w]; NULL cell_C => no thermal */
+    const int32_t *cell_region;                                /* [grid_h*grid_w], -1 = no region */
+    const int32_t *die_region;                                 /* [channels*dies] */
+    const int32_t *region_kind;                                /* [n_regions] */
+    const float *region_idle_w;                                /* [n_regions] */
+} hbfo_config_t;
+
+typedef struct hbfo_ctx hbfo_ctx;
+
+int  hbfo_create(const hbfo_config_t *cfg, hbfo_ctx **out);
+int  hbfo_destroy(hbfo_ctx *ctx);
+int  hbfo_register_range(hbfo_ctx *ctx, uint64_t base, uint64_t length, uint32_t perms, uint32_t kind,
+                         uint32_t stream_tag, uint64_t media_offset, uint32_t *out_id);
+int  hbfo_clear_ranges(hbfo_ctx *ctx);
+int  hbfo_submit_batch(hbfo_ctx *ctx, const hbfo_access_t *acc, uint64_t n, int64_t *completion_ns,
+                       int64_t *stall_ns, uint8_t *status, hbfo_die_stats_t *die_stats);
+int  hbfo_last_result(hbfo_ctx *ctx, hbfo_batch_result_t *out);
+/* The order in which the last accepted batch was served: indices, queue-major. */
+int  hbfo_last_order(hbfo_ctx *ctx, uint32_t *order, uint64_t cap, uint64_t *count);
+int  hbfo_thermal_step(hbfo_ctx *ctx, int64_t dt_ns, const float *ext_power_w, uint32_t n_ext,
+                       double *temps_out, double hot_c_out[3]);
+int  hbfo_force_mode(hbfo_ctx *ctx, int32_t mode, int64_t q_ppm);
+int  hbfo_reset(hbfo_ctx *ctx);
+/* State readers/writers used by tests. */
+int  hbfo_get_busy_until(hbfo_ctx *ctx, int64_t *out, uint64_t cap);
+int  hbfo_get_pending_energy(hbfo_ctx *ctx, int64_t *out, uint64_t cap);
+int  hbfo_get_temps(hbfo_ctx *ctx, double *out, uint64_t cap);
+int  hbfo_set_temps(hbfo_ctx *ctx, const double *in, uint64_t count);
+int  hbfo_get_mode(hbfo_ctx *ctx, int32_t *mode, int64_t *q_ppm);
+double hbfo_euler_limit_ns(hbfo_ctx *ctx);
+/* Single steps of the definition, exposed so that each can be pinned on its own. */
+int  hbfo_classify(hbfo_ctx *ctx, const hbfo_access_t *a, int32_t *range_id);
+int  hbfo_decode(hbfo_ctx *ctx, uint64_t off, uint32_t bytes, uint32_t *channel, uint32_t *die,
+                 uint32_t *plane, uint64_t *row, uint64_t *page, uint64_t *npages, uint32_t *queue);
+int  hbfo_service_terms(hbfo_ctx *ctx, uint32_t bytes, uint64_t npages, uint32_t op, int64_t q_ppm,
+                        int64_t *charged_bytes, int64_t *xfer_ns, int64_t *s_ns, int64_t *energy_pj);
+int32_t hbfo_next_mode(hbfo_ctx *ctx, int32_t mode, int64_t t_hot_mk);
+int64_t hbfo_quantise_mk(double t_c);
+const char *hbfo_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif
