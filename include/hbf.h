@@ -1,0 +1,174 @@
+/*
+ * hbf.h -- C ABI of the B200 HBF service-model library (libhbf.so).
+ *
+ * The library applies an online High-Bandwidth-Flash service model to batches of memory accesses:
+ * range check, address decode to channel/die/plane/page, per-queue FIFO service, completion time
+ * and injected stall per access, per-die busy/byte/energy totals, and the coupled package thermal
+ * step with its throttle controller.  Every step runs in CUDA kernels (sm_100a); there is no CPU
+ * path.  "device" pointers are CUDA device memory owned by the caller; "host" pointers are plain
+ * host memory.  All times are int64 ns on one caller-chosen origin (the paper forbids mixing clock
+ * origins, Design D3); energies are int64 pJ; temperatures are float degrees C.
+ *
+ * Return values: 0 = HBF_OK, negative = error.  Nothing is downgraded silently (Implementation,
+ * "Every failure ends the run").  Calls on one context must come from one thread at a time.
+ */
+#ifndef HBF_H
+#define HBF_H
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define HBF_API __attribute__((visibility("default")))
+#else
+#define HBF_API
+#endif
+
+enum {
+    HBF_OK = 0,
+    HBF_E_INVAL = -1,          /* null pointer, zero size, non-power-of-two page/stripe/granule, bad mode ... */
+    HBF_E_RANGE_OVERLAP = -2,  /* overlapping registration would make classification ambiguous (Design D1) */
+    HBF_E_RANGE_FULL = -3,     /* more than HBF_MAX_RANGES ranges */
+    HBF_E_CAPACITY = -4,       /* media_offset + length beyond capacity_bytes */
+    HBF_E_WORKSPACE = -5,      /* workspace smaller than hbf_workspace_bytes(n) or misaligned */
+    HBF_E_CUDA = -6,           /* a CUDA runtime call failed */
+    HBF_E_ACCESS_FAULT = -7,   /* >= 1 fail-closed access: batch refused, status[] filled, outputs zeroed, no state change */
+    HBF_E_THROTTLED = -8,      /* mode Severe: new reservations withheld, no state change (Design D3) */
+    HBF_E_LINK_SHUTDOWN = -9,  /* mode Shutdown: terminal, every later batch returns it (Design D3) */
+    HBF_E_TIMEOUT = -10,       /* a bounded device-side wait expired; the context is poisoned */
+    HBF_E_NOMEM = -11
+};
+
+/* Per-access status: the batch analogue of the paper's per-request terminal states (Implementation). */
+enum { HBF_ST_NATIVE = 0,        /* address outside every range: native HBM path, not modeled */
+       HBF_ST_READY = 1,         /* whole span inside one range and permitted: modeled */
+       HBF_ST_FAULT_PARTIAL = 2, /* starts inside a range but leaves it (or wraps) */
+       HBF_ST_FAULT_PERM = 3,    /* operation not permitted by the range */
+       HBF_ST_UNSUPPORTED = 4 }; /* bytes == 0, unknown flag bits, issue_ns outside [0, 2^47) */
+
+enum { HBF_MODE_NORMAL = 0, HBF_MODE_LIGHT = 1, HBF_MODE_SEVERE = 2, HBF_MODE_SHUTDOWN = 3 };
+enum { HBF_KIND_NONE = 0, HBF_KIND_GPU = 1, HBF_KIND_HBM = 2, HBF_KIND_HBF = 3 };     /* region kinds */
+enum { HBF_PERM_READ = 1, HBF_PERM_PROGRAM = 2 };
+enum { HBF_RANGE_TIMING = 0, HBF_RANGE_CAPACITY = 1 };
+enum { HBF_PATH_AUTO = 0, HBF_PATH_SORT = 1, HBF_PATH_INORDER = 2, HBF_PATH_SORT_FULL = 3 };
+
+#define HBF_MAX_RANGES 64
+#define HBF_MAX_BATCH ((uint64_t)((1u << 30) - 1))      /* accesses per batch */
+#define HBF_ISSUE_LIMIT (((int64_t)1) << 47)            /* issue_ns in [0, 2^47): 39 h, above the paper's longest run (86,400 s) */
+
+/* One access record, 24 bytes.  flags bit 0: 0 = read, 1 = program; all other bits must be 0. */
+typedef struct { uint64_t addr; int64_t issue_ns; uint32_t bytes; uint32_t flags; } hbf_access_t;
+
+/* Per-die totals of one batch ([channels*dies], index channel*dies + die). */
+typedef struct { int64_t busy_ns, bytes_read, bytes_prog, energy_pj, n_read, n_prog; } hbf_die_stats_t;
+
+/* Batch summary.  modeled_ns = sum of stalls, service_ns = sum of queue service: two of the paper's
+ * four time counters (Implementation); the other two are wall-clock quantities of the caller. */
+typedef struct {
+    int32_t code, mode; int64_t q_ppm; uint64_t n_native, n_modeled, n_fault;
+    int64_t modeled_ns, service_ns, max_completion_ns;
+} hbf_batch_result_t;
+
+typedef struct {
+    /* geometry: a media offset is striped channel first, then die, then plane, in units of stripe_bytes */
+    uint32_t channels, dies, planes, page_bytes, stripe_bytes;
+    uint32_t queue_level;                 /* 0: one queue per plane, 1: one queue per die */
+    uint64_t capacity_bytes;              /* 0 = unbounded */
+    /* timing */
+    int64_t  t_read_ns, t_prog_ns;        /* array time per page */
+    uint64_t chan_bytes_per_us;           /* data transfer rate of one channel */
+    uint32_t read_granule, prog_granule;  /* charged bytes are rounded up to these (powers of two) */
+    /* energy: E = e_cmd + e_byte * charged bytes (Design D3) */
+    int64_t  e_cmd_read_pj, e_byte_read_pj, e_cmd_prog_pj, e_byte_prog_pj;
+    /* thermal (ignored when cell_C is NULL) */
+    uint32_t grid_h, grid_w, n_sub, n_regions;
+    float    ambient_c, rtt_c, ltt_c, stt_c, shutdown_c;   /* rtt < ltt < stt < shutdown */
+    int64_t  q_light_ppm;                 /* service fraction published in Light mode, 1..10^6 */
+    const float *cell_C, *cell_Gx, *cell_Gy, *cell_Gsink;  /* host [grid_h*grid_w]; Gx[y][x] joins (y,x),(y,x+1); Gy[y][x] joins (y,x),(y+1,x) */
+    const int32_t *cell_region;           /* host [grid_h*grid_w], -1 = cell belongs to no region */
+    const int32_t *die_region;            /* host [channels*dies] -> region */
+    const int32_t *region_kind;           /* host [n_regions], HBF_KIND_* */
+    const float *region_idle_w;           /* host [n_regions] */
+} hbf_config_t;
+
+typedef struct hbf_ctx hbf_ctx;           /* opaque, library-owned */
+
+/* Validates the configuration, copies every host array, allocates the context's device state on the
+ * current CUDA device.  cuda_stream is a cudaStream_t (NULL = default stream); all work of the
+ * context is ordered on it.  Queue state starts idle, the thermal field at ambient, mode Normal. */
+HBF_API int hbf_create(const hbf_config_t *cfg, void *cuda_stream, hbf_ctx **out);
+HBF_API int hbf_destroy(hbf_ctx *ctx);
+
+/* Registers the address interval [base, base+length) as an HBF range (Design D1: base, length,
+ * permissions, stream tag, backing offset) and publishes a new sorted snapshot for later batches.
+ * media_offset is the range's first byte on the media.  out_id (nullable) receives the range id. */
+HBF_API int hbf_register_range(hbf_ctx *ctx, uint64_t base, uint64_t length, uint32_t perms, uint32_t kind,
+                       uint32_t stream_tag, uint64_t media_offset, uint32_t *out_id);
+HBF_API int hbf_clear_ranges(hbf_ctx *ctx);
+
+/* Bytes of device scratch hbf_submit_batch needs for a batch of n accesses (256-byte aligned). */
+HBF_API size_t hbf_workspace_bytes(const hbf_ctx *ctx, uint64_t n);
+
+/* Serves one batch, asynchronously on the context's stream.  For access i (its index plays the role
+ * of the paper's ring ticket: results land at the same index):
+ *   classify (Design D1) -> decode -> service terms (Eq. 3 with the batch's snapshot of q) ->
+ *   FIFO per queue in (issue_ns, index) order after everything earlier batches left on the queue ->
+ *   d_completion_ns[i], d_stall_ns[i] = completion - issue.  NATIVE rows: completion = issue, stall 0.
+ * d_acc [n] device, read only, 8-byte aligned.  d_completion_ns, d_stall_ns [n] device.  d_status [n]
+ * device, nullable.  d_die_stats [channels*dies] device, nullable, overwritten with this batch's totals.
+ * d_workspace: device scratch of at least hbf_workspace_bytes(n), 256-byte aligned, must stay valid
+ * until the batch has run.  The return value covers argument checks and launches only; the batch's
+ * own outcome (access fault, throttled, shutdown, timeout) is read with hbf_last_result. */
+HBF_API int hbf_submit_batch(hbf_ctx *ctx, const hbf_access_t *d_acc, uint64_t n, int64_t *d_completion_ns,
+                     int64_t *d_stall_ns, uint8_t *d_status, hbf_die_stats_t *d_die_stats,
+                     void *d_workspace, size_t workspace_bytes);
+
+/* Waits for the last submitted batch and copies its summary to host_out; returns its code. */
+HBF_API int hbf_last_result(hbf_ctx *ctx, hbf_batch_result_t *host_out);
+
+/* Advances the package thermal model by dt_ns (Eq. 1, explicit Euler in n_sub substeps): the energy
+ * the batches since the last step charged to each die becomes power over this window (P = E/dt +
+ * idle, Design D3), ext_power_w (host, [n_regions], nullable with n_ext = 0) adds the external power
+ * of each region; then the HBF hotspot drives the four-state throttle controller, whose mode and
+ * service fraction the next batch snapshots.  d_temps_out (device [grid_h*grid_w], nullable) receives
+ * the field in degrees C.  hot_c_out (host [3], nullable): hottest HBF, HBM and GPU cell; passing it
+ * makes the call wait for the step.  Refuses (HBF_E_INVAL) a substep longer than the stability limit. */
+HBF_API int hbf_thermal_step(hbf_ctx *ctx, int64_t dt_ns, const float *ext_power_w, uint32_t n_ext,
+                     float *d_temps_out, float *hot_c_out);
+
+/* Sets the mode and service fraction directly: the paper's "declared constant" source for
+ * deterministic experiments (Design D3). */
+HBF_API int hbf_force_mode(hbf_ctx *ctx, int32_t mode, int64_t q_ppm);
+HBF_API int hbf_get_mode(hbf_ctx *ctx, int32_t *mode, int64_t *q_ppm);           /* waits for pending work */
+HBF_API int hbf_reset(hbf_ctx *ctx);                                             /* queues idle, field at ambient, mode Normal */
+
+/* Chooses how batches are ordered: HBF_PATH_AUTO (default) serves a batch whose records arrive in
+ * non-decreasing issue order without a global sort and falls back to the radix sort otherwise;
+ * HBF_PATH_SORT always sorts (a batch already in issue order is sorted on its queue bits only, which a
+ * stable sort allows); HBF_PATH_SORT_FULL sorts on every key bit regardless.  All give identical results. */
+HBF_API int hbf_set_path(hbf_ctx *ctx, int32_t path);
+
+/* State snapshot (host blob): header, busy_until[queues], pending energy[dies], thermal field and
+ * its compensation term.  Call with host_buf NULL to get the size. */
+HBF_API int hbf_get_state(hbf_ctx *ctx, void *host_buf, size_t *bytes);
+HBF_API int hbf_set_state(hbf_ctx *ctx, const void *host_buf, size_t bytes);
+/* Individual state arrays, host outputs; each waits for pending work. */
+HBF_API int hbf_get_busy_until(hbf_ctx *ctx, int64_t *host_out, uint64_t cap);
+HBF_API int hbf_get_pending_energy(hbf_ctx *ctx, int64_t *host_out, uint64_t cap);
+HBF_API int hbf_get_temps(hbf_ctx *ctx, float *host_out, uint64_t cap);
+HBF_API double hbf_euler_limit_ns(const hbf_ctx *ctx);
+
+/* The order in which the last batch was served when it went through the sort path: batch indices,
+ * queue-major, read back from the workspace of that batch into d_order (device [n]); *count (host)
+ * receives the number of modeled accesses. */
+HBF_API int hbf_queue_order(hbf_ctx *ctx, const void *d_workspace, uint64_t n, uint32_t *d_order, uint64_t *count);
+
+HBF_API const char *hbf_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

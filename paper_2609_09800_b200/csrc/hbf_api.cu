@@ -1,0 +1,436 @@
+// Host shell of libhbf.so: argument validation, context and range bookkeeping, launches.
+// No step of the service model runs here; the host only checks arguments and enqueues kernels.
+#include <algorithm>
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "hbf_dev.cuh"
+
+using namespace hbf;
+
+namespace {
+
+struct HostRange { uint64_t base, length, media_offset; uint32_t perms, kind, stream_tag, id; };
+
+struct StateHeader {            // hbf_get_state / hbf_set_state blob header
+    uint32_t magic, version, n_queues, n_dies, n_cells; int32_t mode; int64_t q_ppm; int32_t poisoned, cur;
+};
+constexpr uint32_t kStateMagic = 0x48424631u;   // "HBF1"
+
+}  // namespace
+
+struct hbf_ctx {
+    hbf_config_t cfg{};
+    cudaStream_t stream = nullptr;
+    int device = 0, sm_count = 148;
+    ModelParams mp{};
+    std::vector<HostRange> ranges;
+    uint32_t next_range_id = 0;
+    int32_t path = HBF_PATH_AUTO;
+    bool terminal = false;           // a shutdown result has been observed
+    // device state
+    RangeSnap *d_ranges = nullptr; ModelParams *d_mp = nullptr; DevState *d_state = nullptr;
+    BatchCtrl *d_ctrl = nullptr; hbf_batch_result_t *d_result = nullptr;
+    int64_t *d_busy = nullptr, *d_busy_stage = nullptr, *d_pending = nullptr; hbf_die_stats_t *d_stats_stage = nullptr;
+    hbf_batch_result_t *h_result = nullptr;      // pinned
+    float *h_hot = nullptr;                      // pinned [3]
+    float *h_ext = nullptr;                      // pinned [n_regions]
+    bool submitted = false;
+    // thermal
+    bool thermal = false; ThermalDev td{}; int cur = 0; double euler_limit_s = 0.0;
+    std::vector<void *> owned;
+};
+
+#define CK(expr) do { cudaError_t e_ = (expr); if (e_ != cudaSuccess) return HBF_E_CUDA; } while (0)
+
+static bool is_pow2(uint64_t v) { return v && !(v & (v - 1)); }
+static uint32_t log2u(uint64_t v) { uint32_t s = 0; while ((1ull << s) < v) ++s; return s; }
+
+template <typename T>
+static int dev_copy(hbf_ctx *c, T **dst, const void *src, size_t count) {
+    void *p = nullptr;
+    if (cudaMalloc(&p, std::max<size_t>(count, 1) * sizeof(T)) != cudaSuccess) return HBF_E_NOMEM;
+    c->owned.push_back(p);
+    if (src) { if (cudaMemcpy(p, src, count * sizeof(T), cudaMemcpyHostToDevice) != cudaSuccess) return HBF_E_CUDA; }
+    else if (cudaMemset(p, 0, std::max<size_t>(count, 1) * sizeof(T)) != cudaSuccess) return HBF_E_CUDA;
+    *dst = static_cast<T *>(p);
+    return HBF_OK;
+}
+
+static int publish_ranges(hbf_ctx *c) {
+    RangeSnap snap; memset(&snap, 0, sizeof(snap));
+    std::vector<HostRange> sorted = c->ranges;
+    std::sort(sorted.begin(), sorted.end(), [](const HostRange &a, const HostRange &b) { return a.base < b.base; });
+    snap.count = (uint32_t)sorted.size();
+    for (size_t i = 0; i < sorted.size(); ++i) {
+        snap.base[i] = sorted[i].base; snap.length[i] = sorted[i].length;
+        snap.media_offset[i] = sorted[i].media_offset; snap.perms[i] = sorted[i].perms;
+    }
+    // ordered after every batch already enqueued, before every later one
+    CK(cudaMemcpyAsync(c->d_ranges, &snap, sizeof(snap), cudaMemcpyHostToDevice, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    return HBF_OK;
+}
+
+extern "C" {
+
+const char *hbf_strerror(int code) {
+    switch (code) {
+    case HBF_OK: return "ok";
+    case HBF_E_INVAL: return "invalid argument";
+    case HBF_E_RANGE_OVERLAP: return "range overlaps a registered range";
+    case HBF_E_RANGE_FULL: return "range table full";
+    case HBF_E_CAPACITY: return "range exceeds media capacity";
+    case HBF_E_WORKSPACE: return "workspace too small or misaligned";
+    case HBF_E_CUDA: return "CUDA runtime error";
+    case HBF_E_ACCESS_FAULT: return "batch refused: fail-closed access";
+    case HBF_E_THROTTLED: return "throttled: new reservations withheld";
+    case HBF_E_LINK_SHUTDOWN: return "link shutdown";
+    case HBF_E_TIMEOUT: return "bounded device wait expired";
+    case HBF_E_NOMEM: return "out of memory";
+    default: return "unknown";
+    }
+}
+
+int hbf_destroy(hbf_ctx *c) {
+    if (!c) return HBF_E_INVAL;
+    cudaStreamSynchronize(c->stream);
+    for (void *p : c->owned) cudaFree(p);
+    if (c->h_result) cudaFreeHost(c->h_result);
+    if (c->h_hot) cudaFreeHost(c->h_hot);
+    if (c->h_ext) cudaFreeHost(c->h_ext);
+    delete c;
+    return HBF_OK;
+}
+
+int hbf_create(const hbf_config_t *cfg, void *cuda_stream, hbf_ctx **out) {
+    if (!cfg || !out) return HBF_E_INVAL;
+    if (!cfg->channels || !cfg->dies || !cfg->planes) return HBF_E_INVAL;
+    if (!is_pow2(cfg->page_bytes) || !is_pow2(cfg->stripe_bytes) || cfg->stripe_bytes < cfg->page_bytes) return HBF_E_INVAL;
+    if (!is_pow2(cfg->read_granule) || !is_pow2(cfg->prog_granule) || cfg->queue_level > 1) return HBF_E_INVAL;
+    if (cfg->t_read_ns <= 0 || cfg->t_prog_ns <= 0 || !cfg->chan_bytes_per_us) return HBF_E_INVAL;
+    if (cfg->e_cmd_read_pj < 0 || cfg->e_byte_read_pj < 0 || cfg->e_cmd_prog_pj < 0 || cfg->e_byte_prog_pj < 0) return HBF_E_INVAL;
+    if (cfg->q_light_ppm < 1 || cfg->q_light_ppm > 1000000) return HBF_E_INVAL;
+    const uint64_t nd = (uint64_t)cfg->channels * cfg->dies;
+    const uint64_t nq = cfg->queue_level == 0 ? nd * cfg->planes : nd;
+    if (nq > 65536 || nd > 65536) return HBF_E_INVAL;
+
+    hbf_ctx *c = new (std::nothrow) hbf_ctx();
+    if (!c) return HBF_E_NOMEM;
+    c->cfg = *cfg; c->stream = static_cast<cudaStream_t>(cuda_stream);
+    int rc = HBF_OK;
+    auto fail = [&](int code) { hbf_destroy(c); return code; };
+    if (cudaGetDevice(&c->device) != cudaSuccess) return fail(HBF_E_CUDA);
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, c->device) != cudaSuccess) return fail(HBF_E_CUDA);
+    c->sm_count = prop.multiProcessorCount;
+
+    ModelParams &mp = c->mp;
+    mp.channels = cfg->channels; mp.dies = cfg->dies; mp.planes = cfg->planes;
+    mp.n_queues = (uint32_t)nq; mp.n_dies = (uint32_t)nd;
+    mp.page_shift = log2u(cfg->page_bytes); mp.stripe_shift = log2u(cfg->stripe_bytes);
+    mp.pages_per_stripe_shift = mp.stripe_shift - mp.page_shift;
+    mp.queue_level = cfg->queue_level;
+    mp.pow2_geom = is_pow2(cfg->channels) && is_pow2(cfg->dies) && is_pow2(cfg->planes);
+    mp.ch_shift = log2u(cfg->channels); mp.die_shift = log2u(cfg->dies); mp.plane_shift = log2u(cfg->planes);
+    mp.read_gran_shift = log2u(cfg->read_granule); mp.prog_gran_shift = log2u(cfg->prog_granule);
+    mp.t_read_ns = cfg->t_read_ns; mp.t_prog_ns = cfg->t_prog_ns; mp.chan_bytes_per_us = cfg->chan_bytes_per_us;
+    mp.e_cmd_read_pj = cfg->e_cmd_read_pj; mp.e_byte_read_pj = cfg->e_byte_read_pj;
+    mp.e_cmd_prog_pj = cfg->e_cmd_prog_pj; mp.e_byte_prog_pj = cfg->e_byte_prog_pj;
+
+    DevState st0; st0.mode = HBF_MODE_NORMAL; st0.poisoned = 0; st0.q_ppm = 1000000;
+    if ((rc = dev_copy(c, &c->d_ranges, nullptr, 1))) return fail(rc);
+    if ((rc = dev_copy(c, &c->d_mp, &mp, 1))) return fail(rc);
+    if ((rc = dev_copy(c, &c->d_state, &st0, 1))) return fail(rc);
+    if ((rc = dev_copy(c, &c->d_ctrl, nullptr, 1))) return fail(rc);
+    if ((rc = dev_copy(c, &c->d_result, nullptr, 1))) return fail(rc);
+    if ((rc = dev_copy(c, &c->d_busy, nullptr, nq))) return fail(rc);
+    if ((rc = dev_copy(c, &c->d_busy_stage, nullptr, nq))) return fail(rc);
+    if ((rc = dev_copy(c, &c->d_pending, nullptr, nd))) return fail(rc);
+    if ((rc = dev_copy(c, &c->d_stats_stage, nullptr, nd))) return fail(rc);
+    if (cudaMallocHost(&c->h_result, sizeof(hbf_batch_result_t)) != cudaSuccess) return fail(HBF_E_NOMEM);
+    memset(c->h_result, 0, sizeof(hbf_batch_result_t));
+    if (cudaMallocHost(&c->h_hot, 3 * sizeof(float)) != cudaSuccess) return fail(HBF_E_NOMEM);
+
+    c->thermal = cfg->cell_C != nullptr;
+    if (c->thermal) {
+        if (!cfg->grid_h || !cfg->grid_w || !cfg->n_sub || !cfg->n_regions || !cfg->cell_Gx || !cfg->cell_Gy ||
+            !cfg->cell_Gsink || !cfg->cell_region || !cfg->die_region || !cfg->region_kind || !cfg->region_idle_w)
+            return fail(HBF_E_INVAL);
+        if (!(cfg->rtt_c < cfg->ltt_c && cfg->ltt_c < cfg->stt_c && cfg->stt_c < cfg->shutdown_c)) return fail(HBF_E_INVAL);
+        const uint32_t H = cfg->grid_h, W = cfg->grid_w, NR = cfg->n_regions;
+        const size_t nc = (size_t)H * W;
+        if (nc > (1u << 30)) return fail(HBF_E_INVAL);
+        std::vector<float> inv_cells(NR, 0.0f); std::vector<double> cells(NR, 0.0);
+        double lim = INFINITY;
+        for (uint32_t y = 0; y < H; ++y) for (uint32_t x = 0; x < W; ++x) {
+            const size_t i = (size_t)y * W + x;
+            if (!(cfg->cell_C[i] > 0.0f) || cfg->cell_Gx[i] < 0.0f || cfg->cell_Gy[i] < 0.0f || cfg->cell_Gsink[i] < 0.0f) return fail(HBF_E_INVAL);
+            const int32_t g = cfg->cell_region[i];
+            if (g >= (int32_t)NR) return fail(HBF_E_INVAL);
+            if (g >= 0) cells[g] += 1.0;
+            double gs = cfg->cell_Gsink[i];
+            if (x + 1 < W) gs += cfg->cell_Gx[i];
+            if (x > 0) gs += cfg->cell_Gx[i - 1];
+            if (y + 1 < H) gs += cfg->cell_Gy[i];
+            if (y > 0) gs += cfg->cell_Gy[i - W];
+            if (gs > 0.0) lim = std::min(lim, (double)cfg->cell_C[i] / gs);
+        }
+        c->euler_limit_s = lim;
+        std::vector<int32_t> ptr(NR + 1, 0), list(nd);
+        for (uint64_t d = 0; d < nd; ++d) {
+            const int32_t g = cfg->die_region[d];
+            if (g < 0 || g >= (int32_t)NR || cells[g] == 0.0) return fail(HBF_E_INVAL);
+            ptr[g + 1]++;
+        }
+        for (uint32_t g = 0; g < NR; ++g) { ptr[g + 1] += ptr[g]; inv_cells[g] = cells[g] > 0.0 ? (float)(1.0 / cells[g]) : 0.0f; }
+        { std::vector<int32_t> fill(ptr.begin(), ptr.end() - 1);
+          for (uint64_t d = 0; d < nd; ++d) list[fill[cfg->die_region[d]]++] = (int32_t)d; }
+        ThermalDev &t = c->td;
+        t.H = H; t.W = W; t.n_regions = NR; t.n_dies = (uint32_t)nd; t.n_sub = cfg->n_sub; t.ambient_c = cfg->ambient_c;
+        auto mk = [](float v) { return (int64_t)std::floor((double)v * 1000.0 + 0.5); };
+        t.rtt_mk = mk(cfg->rtt_c); t.ltt_mk = mk(cfg->ltt_c); t.stt_mk = mk(cfg->stt_c); t.shut_mk = mk(cfg->shutdown_c);
+        t.q_light_ppm = cfg->q_light_ppm;
+        float *p;
+        int32_t *q;
+        double *dp;
+        if ((rc = dev_copy(c, &p, cfg->cell_C, nc))) return fail(rc); t.C = p;
+        if ((rc = dev_copy(c, &p, cfg->cell_Gx, nc))) return fail(rc); t.Gx = p;
+        if ((rc = dev_copy(c, &p, cfg->cell_Gy, nc))) return fail(rc); t.Gy = p;
+        if ((rc = dev_copy(c, &p, cfg->cell_Gsink, nc))) return fail(rc); t.Gs = p;
+        if ((rc = dev_copy(c, &q, cfg->cell_region, nc))) return fail(rc); t.cell_region = q;
+        if ((rc = dev_copy(c, &q, cfg->die_region, nd))) return fail(rc); t.die_region = q;
+        if ((rc = dev_copy(c, &q, cfg->region_kind, NR))) return fail(rc); t.region_kind = q;
+        if ((rc = dev_copy(c, &p, cfg->region_idle_w, NR))) return fail(rc); t.region_idle_w = p;
+        if ((rc = dev_copy(c, &p, inv_cells.data(), NR))) return fail(rc); t.region_inv_cells = p;
+        if ((rc = dev_copy(c, &q, ptr.data(), NR + 1))) return fail(rc); t.region_die_ptr = q;
+        if ((rc = dev_copy(c, &q, list.data(), nd))) return fail(rc); t.region_die_list = q;
+        if ((rc = dev_copy(c, &t.theta[0], nullptr, nc))) return fail(rc);
+        if ((rc = dev_copy(c, &t.theta[1], nullptr, nc))) return fail(rc);
+        if ((rc = dev_copy(c, &t.comp, nullptr, nc))) return fail(rc);
+        if ((rc = dev_copy(c, &t.P, nullptr, nc))) return fail(rc);
+        if ((rc = dev_copy(c, &dp, nullptr, NR))) return fail(rc); t.region_power = dp;
+        if ((rc = dev_copy(c, &t.ext_power, nullptr, NR))) return fail(rc);
+        if ((rc = dev_copy(c, &t.hot, nullptr, 3))) return fail(rc);
+        if (cudaMallocHost(&c->h_ext, NR * sizeof(float)) != cudaSuccess) return fail(HBF_E_NOMEM);
+        // the descriptor keeps no pointer into the caller's arrays
+        c->cfg.cell_C = c->cfg.cell_Gx = c->cfg.cell_Gy = c->cfg.cell_Gsink = c->cfg.region_idle_w = nullptr;
+        c->cfg.cell_region = c->cfg.die_region = c->cfg.region_kind = nullptr;
+    }
+    if (cudaDeviceSynchronize() != cudaSuccess) return fail(HBF_E_CUDA);
+    *out = c;
+    return HBF_OK;
+}
+
+int hbf_register_range(hbf_ctx *c, uint64_t base, uint64_t length, uint32_t perms, uint32_t kind,
+                       uint32_t stream_tag, uint64_t media_offset, uint32_t *out_id) {
+    if (!c || length == 0 || (perms & ~3u) || perms == 0 || kind > 1) return HBF_E_INVAL;
+    if (base + length < base || media_offset + length < media_offset) return HBF_E_INVAL;
+    if (c->cfg.capacity_bytes && media_offset + length > c->cfg.capacity_bytes) return HBF_E_CAPACITY;
+    if (c->ranges.size() >= HBF_MAX_RANGES) return HBF_E_RANGE_FULL;
+    for (const HostRange &r : c->ranges)
+        if (base < r.base + r.length && r.base < base + length) return HBF_E_RANGE_OVERLAP;
+    HostRange r{base, length, media_offset, perms, kind, stream_tag, c->next_range_id++};
+    c->ranges.push_back(r);
+    if (out_id) *out_id = r.id;
+    return publish_ranges(c);
+}
+
+int hbf_clear_ranges(hbf_ctx *c) {
+    if (!c) return HBF_E_INVAL;
+    c->ranges.clear();
+    return publish_ranges(c);
+}
+
+size_t hbf_workspace_bytes(const hbf_ctx *c, uint64_t n) {
+    if (!c) return 0;
+    return workspace_layout(n, c->mp.n_queues, nullptr, nullptr);
+}
+
+int hbf_set_path(hbf_ctx *c, int32_t path) {
+    if (!c || path < 0 || path > 3) return HBF_E_INVAL;
+    c->path = path;
+    return HBF_OK;
+}
+
+int hbf_submit_batch(hbf_ctx *c, const hbf_access_t *d_acc, uint64_t n, int64_t *d_completion_ns,
+                     int64_t *d_stall_ns, uint8_t *d_status, hbf_die_stats_t *d_die_stats,
+                     void *d_workspace, size_t workspace_bytes) {
+    if (!c) return HBF_E_INVAL;
+    if (c->terminal) return HBF_E_LINK_SHUTDOWN;
+    if (n > HBF_MAX_BATCH) return HBF_E_INVAL;
+    if (n && (!d_acc || !d_completion_ns || !d_stall_ns)) return HBF_E_INVAL;
+    if ((reinterpret_cast<uintptr_t>(d_acc) & 7u) || (reinterpret_cast<uintptr_t>(d_completion_ns) & 7u) ||
+        (reinterpret_cast<uintptr_t>(d_stall_ns) & 7u) || (reinterpret_cast<uintptr_t>(d_die_stats) & 7u)) return HBF_E_INVAL;
+    SubmitArgs a{};
+    const size_t need = workspace_layout(n, c->mp.n_queues, &a.ws, d_workspace);
+    if (!d_workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(d_workspace) & 255u)) return HBF_E_WORKSPACE;
+    a.acc = d_acc; a.n = n; a.completion = d_completion_ns; a.stall = d_stall_ns; a.status = d_status; a.die_stats = d_die_stats;
+    a.ranges = c->d_ranges; a.mp_dev = c->d_mp; a.mp = c->mp; a.state = c->d_state; a.ctrl = c->d_ctrl; a.result = c->d_result;
+    a.busy = c->d_busy; a.busy_stage = c->d_busy_stage; a.pending = c->d_pending; a.stats_stage = c->d_stats_stage;
+    a.path = c->path; a.sm_count = c->sm_count;
+    CK(launch_submit(a, c->stream));
+    c->submitted = true;
+    return HBF_OK;
+}
+
+int hbf_last_result(hbf_ctx *c, hbf_batch_result_t *host_out) {
+    if (!c || !host_out) return HBF_E_INVAL;
+    if (!c->submitted) { memset(host_out, 0, sizeof(*host_out)); return HBF_OK; }
+    CK(cudaMemcpyAsync(c->h_result, c->d_result, sizeof(hbf_batch_result_t), cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    *host_out = *c->h_result;
+    if (host_out->code == HBF_E_LINK_SHUTDOWN) c->terminal = true;
+    return host_out->code;
+}
+
+int hbf_queue_order(hbf_ctx *c, const void *d_workspace, uint64_t n, uint32_t *d_order, uint64_t *count) {
+    if (!c || !d_workspace || !d_order || !count) return HBF_E_INVAL;
+    Workspace ws;
+    workspace_layout(n, c->mp.n_queues, &ws, const_cast<void *>(d_workspace));
+    CK(launch_queue_order(c->d_ctrl, ws, d_order, n, c->stream));
+    BatchCtrl hc;
+    CK(cudaMemcpyAsync(&hc, c->d_ctrl, sizeof(hc), cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    if (hc.code != HBF_OK || hc.inorder_used) return HBF_E_INVAL;
+    *count = hc.n_ready;
+    return HBF_OK;
+}
+
+int hbf_thermal_step(hbf_ctx *c, int64_t dt_ns, const float *ext_power_w, uint32_t n_ext, float *d_temps_out, float *hot_c_out) {
+    if (!c || !c->thermal || dt_ns <= 0) return HBF_E_INVAL;
+    if (n_ext != 0 && (n_ext != c->td.n_regions || !ext_power_w)) return HBF_E_INVAL;
+    const double dt_sub = (double)dt_ns * 1e-9 / (double)c->td.n_sub;
+    if (dt_sub > c->euler_limit_s) return HBF_E_INVAL;
+    if (n_ext) {
+        CK(cudaStreamSynchronize(c->stream));          // the pinned staging buffer may still feed an earlier step
+        memcpy(c->h_ext, ext_power_w, n_ext * sizeof(float));
+        CK(cudaMemcpyAsync(c->td.ext_power, c->h_ext, n_ext * sizeof(float), cudaMemcpyHostToDevice, c->stream));
+    }
+    CK(launch_thermal_step(c->td, c->d_state, c->d_pending, dt_ns, n_ext != 0, d_temps_out, &c->cur, c->stream));
+    if (hot_c_out) {
+        CK(cudaMemcpyAsync(c->h_hot, c->td.hot, 3 * sizeof(float), cudaMemcpyDeviceToHost, c->stream));
+        CK(cudaStreamSynchronize(c->stream));
+        memcpy(hot_c_out, c->h_hot, 3 * sizeof(float));
+    }
+    return HBF_OK;
+}
+
+int hbf_force_mode(hbf_ctx *c, int32_t mode, int64_t q_ppm) {
+    if (!c || mode < 0 || mode > 3 || q_ppm < 1 || q_ppm > 1000000) return HBF_E_INVAL;
+    DevState s;
+    CK(cudaMemcpyAsync(&s, c->d_state, sizeof(s), cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    s.mode = mode; s.q_ppm = q_ppm;
+    CK(cudaMemcpyAsync(c->d_state, &s, sizeof(s), cudaMemcpyHostToDevice, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    if (mode != HBF_MODE_SHUTDOWN) c->terminal = false;
+    return HBF_OK;
+}
+
+int hbf_get_mode(hbf_ctx *c, int32_t *mode, int64_t *q_ppm) {
+    if (!c) return HBF_E_INVAL;
+    DevState s;
+    CK(cudaMemcpyAsync(&s, c->d_state, sizeof(s), cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    if (mode) *mode = s.mode;
+    if (q_ppm) *q_ppm = s.q_ppm;
+    return HBF_OK;
+}
+
+int hbf_reset(hbf_ctx *c) {
+    if (!c) return HBF_E_INVAL;
+    DevState s; s.mode = HBF_MODE_NORMAL; s.poisoned = 0; s.q_ppm = 1000000;
+    CK(cudaStreamSynchronize(c->stream));
+    CK(cudaMemcpyAsync(c->d_state, &s, sizeof(s), cudaMemcpyHostToDevice, c->stream));
+    CK(cudaMemsetAsync(c->d_busy, 0, c->mp.n_queues * sizeof(int64_t), c->stream));
+    CK(cudaMemsetAsync(c->d_pending, 0, c->mp.n_dies * sizeof(int64_t), c->stream));
+    CK(cudaMemsetAsync(c->d_result, 0, sizeof(hbf_batch_result_t), c->stream));
+    if (c->thermal) {
+        const size_t nc = (size_t)c->td.H * c->td.W;
+        CK(cudaMemsetAsync(c->td.theta[0], 0, nc * sizeof(float), c->stream));
+        CK(cudaMemsetAsync(c->td.theta[1], 0, nc * sizeof(float), c->stream));
+        CK(cudaMemsetAsync(c->td.comp, 0, nc * sizeof(float), c->stream));
+        c->cur = 0;
+    }
+    CK(cudaStreamSynchronize(c->stream));
+    c->terminal = false;
+    return HBF_OK;
+}
+
+int hbf_get_busy_until(hbf_ctx *c, int64_t *host_out, uint64_t cap) {
+    if (!c || !host_out || cap < c->mp.n_queues) return HBF_E_INVAL;
+    CK(cudaMemcpyAsync(host_out, c->d_busy, c->mp.n_queues * sizeof(int64_t), cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    return HBF_OK;
+}
+
+int hbf_get_pending_energy(hbf_ctx *c, int64_t *host_out, uint64_t cap) {
+    if (!c || !host_out || cap < c->mp.n_dies) return HBF_E_INVAL;
+    CK(cudaMemcpyAsync(host_out, c->d_pending, c->mp.n_dies * sizeof(int64_t), cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    return HBF_OK;
+}
+
+int hbf_get_temps(hbf_ctx *c, float *host_out, uint64_t cap) {
+    if (!c || !c->thermal || !host_out) return HBF_E_INVAL;
+    const size_t nc = (size_t)c->td.H * c->td.W;
+    if (cap < nc) return HBF_E_INVAL;
+    CK(cudaMemcpyAsync(host_out, c->td.theta[c->cur], nc * sizeof(float), cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    for (size_t i = 0; i < nc; ++i) host_out[i] += c->td.ambient_c;
+    return HBF_OK;
+}
+
+double hbf_euler_limit_ns(const hbf_ctx *c) { return c && c->thermal ? c->euler_limit_s * 1e9 : 0.0; }
+
+int hbf_get_state(hbf_ctx *c, void *host_buf, size_t *bytes) {
+    if (!c || !bytes) return HBF_E_INVAL;
+    const size_t nc = c->thermal ? (size_t)c->td.H * c->td.W : 0;
+    const size_t need = sizeof(StateHeader) + (size_t)c->mp.n_queues * 8 + (size_t)c->mp.n_dies * 8 + nc * 8;
+    if (!host_buf) { *bytes = need; return HBF_OK; }
+    if (*bytes < need) return HBF_E_INVAL;
+    *bytes = need;
+    char *p = static_cast<char *>(host_buf);
+    DevState s;
+    CK(cudaMemcpyAsync(&s, c->d_state, sizeof(s), cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    StateHeader h{kStateMagic, 1u, c->mp.n_queues, c->mp.n_dies, (uint32_t)nc, s.mode, s.q_ppm, s.poisoned, 0};
+    memcpy(p, &h, sizeof(h)); p += sizeof(h);
+    CK(cudaMemcpyAsync(p, c->d_busy, (size_t)c->mp.n_queues * 8, cudaMemcpyDeviceToHost, c->stream)); p += (size_t)c->mp.n_queues * 8;
+    CK(cudaMemcpyAsync(p, c->d_pending, (size_t)c->mp.n_dies * 8, cudaMemcpyDeviceToHost, c->stream)); p += (size_t)c->mp.n_dies * 8;
+    if (nc) {
+        CK(cudaMemcpyAsync(p, c->td.theta[c->cur], nc * 4, cudaMemcpyDeviceToHost, c->stream)); p += nc * 4;
+        CK(cudaMemcpyAsync(p, c->td.comp, nc * 4, cudaMemcpyDeviceToHost, c->stream));
+    }
+    CK(cudaStreamSynchronize(c->stream));
+    return HBF_OK;
+}
+
+int hbf_set_state(hbf_ctx *c, const void *host_buf, size_t bytes) {
+    if (!c || !host_buf) return HBF_E_INVAL;
+    const size_t nc = c->thermal ? (size_t)c->td.H * c->td.W : 0;
+    const size_t need = sizeof(StateHeader) + (size_t)c->mp.n_queues * 8 + (size_t)c->mp.n_dies * 8 + nc * 8;
+    if (bytes < need) return HBF_E_INVAL;
+    const char *p = static_cast<const char *>(host_buf);
+    StateHeader h; memcpy(&h, p, sizeof(h)); p += sizeof(h);
+    if (h.magic != kStateMagic || h.version != 1u || h.n_queues != c->mp.n_queues || h.n_dies != c->mp.n_dies ||
+        h.n_cells != (uint32_t)nc || h.mode < 0 || h.mode > 3 || h.q_ppm < 1 || h.q_ppm > 1000000) return HBF_E_INVAL;
+    DevState s; s.mode = h.mode; s.q_ppm = h.q_ppm; s.poisoned = h.poisoned;
+    CK(cudaStreamSynchronize(c->stream));
+    CK(cudaMemcpyAsync(c->d_state, &s, sizeof(s), cudaMemcpyHostToDevice, c->stream));
+    CK(cudaMemcpyAsync(c->d_busy, p, (size_t)c->mp.n_queues * 8, cudaMemcpyHostToDevice, c->stream)); p += (size_t)c->mp.n_queues * 8;
+    CK(cudaMemcpyAsync(c->d_pending, p, (size_t)c->mp.n_dies * 8, cudaMemcpyHostToDevice, c->stream)); p += (size_t)c->mp.n_dies * 8;
+    if (nc) {
+        CK(cudaMemcpyAsync(c->td.theta[c->cur], p, nc * 4, cudaMemcpyHostToDevice, c->stream)); p += nc * 4;
+        CK(cudaMemcpyAsync(c->td.comp, p, nc * 4, cudaMemcpyHostToDevice, c->stream));
+    }
+    CK(cudaStreamSynchronize(c->stream));
+    c->terminal = (h.mode == HBF_MODE_SHUTDOWN) ? c->terminal : false;
+    return HBF_OK;
+}
+
+}  // extern "C"

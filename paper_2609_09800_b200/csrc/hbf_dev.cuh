@@ -1,0 +1,110 @@
+// Internal declarations shared by the translation units of libhbf.so: device-side parameter blocks,
+// the per-batch control block, and the host launchers of each kernel group.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/hbf.h"
+
+namespace hbf {
+
+constexpr int kMaxPasses = 8;            // 63 key bits / 8-bit digits
+constexpr int kRadix = 256;
+constexpr int kIssueBits = 47;           // key = queue << 47 | issue_ns
+constexpr uint64_t kIssueMask = (1ull << kIssueBits) - 1;
+constexpr int64_t kNegInf = INT64_MIN / 4;
+constexpr uint32_t kSpinLimit = 1u << 24;  // polls of one look-back slot before giving up
+
+// Sorted snapshot of the registered ranges (Design D1).
+struct RangeSnap {
+    uint64_t base[HBF_MAX_RANGES];
+    uint64_t length[HBF_MAX_RANGES];
+    uint64_t media_offset[HBF_MAX_RANGES];
+    uint32_t perms[HBF_MAX_RANGES];
+    uint32_t count;
+    uint32_t pad;
+};
+
+// Geometry and timing, fixed at create.
+struct ModelParams {
+    uint32_t channels, dies, planes;
+    uint32_t n_queues, n_dies;
+    uint32_t page_shift, stripe_shift, pages_per_stripe_shift;
+    uint32_t queue_level;
+    uint32_t pow2_geom;                  // channels, dies, planes all powers of two
+    uint32_t ch_shift, die_shift, plane_shift;
+    uint32_t read_gran_shift, prog_gran_shift;
+    int64_t t_read_ns, t_prog_ns;
+    uint64_t chan_bytes_per_us;
+    int64_t e_cmd_read_pj, e_byte_read_pj, e_cmd_prog_pj, e_byte_prog_pj;
+};
+
+// Radix plan of one batch, written by the plan kernel.
+struct SortPlan {
+    uint32_t n_passes;
+    uint32_t lo_bits, hi_bits;           // participating bits of the issue field and of the queue field
+    uint32_t shift[kMaxPasses];
+    uint32_t bits[kMaxPasses];
+};
+
+// Per-batch control block in device memory, cleared by the begin kernel.
+struct BatchCtrl {
+    int32_t code;                        // HBF_OK or the batch's refusal / failure code
+    int32_t skip;                        // later kernels do nothing when set
+    int32_t mode; int32_t pad0;
+    int64_t q_ppm;
+    unsigned long long n_native, n_ready, n_fault;
+    unsigned long long key_or, key_and;
+    uint32_t unsorted;                   // some record has a smaller issue time than its predecessor
+    uint32_t inorder_used;               // the in-order path served this batch
+    uint32_t tile_counter[kMaxPasses + 2];
+    long long modeled_ns, service_ns, max_completion_ns;
+    SortPlan plan;
+};
+
+// Long-lived device state of a context.
+struct DevState {
+    int32_t mode; int32_t poisoned;
+    int64_t q_ppm;
+};
+
+// Workspace carve-up for a batch of n records.
+struct Workspace {
+    uint64_t *keys[2];
+    uint32_t *idx[2];
+    uint32_t *hist;                      // [kMaxPasses][kRadix]
+    uint32_t *sort_desc[2];              // [tiles][kRadix] look-back words, ping-pong between passes
+    void *scan_desc;                     // [scan tiles] ScanDesc
+    void *inorder_desc;                  // in-order path tile state
+    size_t bytes;
+};
+
+struct SubmitArgs {
+    const hbf_access_t *acc; uint64_t n;
+    int64_t *completion, *stall; uint8_t *status; hbf_die_stats_t *die_stats;
+    const RangeSnap *ranges; const ModelParams *mp_dev; ModelParams mp;
+    DevState *state; BatchCtrl *ctrl; hbf_batch_result_t *result;
+    int64_t *busy, *busy_stage, *pending; hbf_die_stats_t *stats_stage;
+    Workspace ws; int32_t path; int sm_count;
+};
+
+size_t workspace_layout(uint64_t n, uint32_t n_queues, Workspace *ws, void *base);
+cudaError_t launch_submit(const SubmitArgs &a, cudaStream_t st);
+cudaError_t launch_queue_order(const BatchCtrl *ctrl, const Workspace &ws, uint32_t *out, uint64_t n, cudaStream_t st);
+
+// ---- thermal -------------------------------------------------------------------------------------
+struct ThermalDev {
+    uint32_t H, W, n_regions, n_dies, n_sub;
+    float ambient_c;
+    int64_t rtt_mk, ltt_mk, stt_mk, shut_mk, q_light_ppm;
+    const float *C, *Gx, *Gy, *Gs;
+    const int32_t *cell_region, *die_region, *region_kind;
+    const float *region_idle_w; const float *region_inv_cells;
+    const int32_t *region_die_ptr, *region_die_list;   // dies of each region, CSR
+    float *theta[2]; float *comp; float *P; double *region_power; float *ext_power;
+    float *hot;                          // [3] device
+};
+cudaError_t launch_thermal_step(const ThermalDev &t, DevState *state, int64_t *pending, int64_t dt_ns,
+                                int has_ext, float *d_temps_out, int *cur, cudaStream_t st);
+
+}  // namespace hbf

@@ -1,0 +1,684 @@
+// Kernels of hbf_submit_batch, sort path:
+//   begin -> classify (load, range filter, decode, key) -> plan -> histogram -> onesweep radix passes ->
+//   scan (segmented max-plus scan with decoupled look-back, fused with the scatter back to batch order
+//   and the per-die reductions) -> finish (commit or refuse).
+// Every kernel reads the batch control block first and does nothing once the batch is refused, so the
+// whole sequence can be enqueued without a host round trip.
+#include <algorithm>
+
+#include "device_utils.cuh"
+
+namespace hbf {
+
+// =====================================================================================================
+// begin: snapshot mode and q (before any reservation, Eq. 3), stage the queue state, clear the block
+// =====================================================================================================
+__global__ void k_begin(BatchCtrl *ctrl, const DevState *state, const int64_t *busy, int64_t *busy_stage,
+                        hbf_die_stats_t *stats_stage, uint32_t *hist, uint32_t n_queues, uint32_t n_dies) {
+    const int tid = threadIdx.x;
+    uint32_t *w = reinterpret_cast<uint32_t *>(ctrl);
+    for (int i = tid; i < (int)(sizeof(BatchCtrl) / 4); i += blockDim.x) w[i] = 0u;
+    __syncthreads();
+    if (tid == 0) {
+        int32_t mode = state->mode;
+        ctrl->mode = mode; ctrl->q_ppm = state->q_ppm;
+        ctrl->key_and = ~0ull;
+        if (state->poisoned) { ctrl->code = HBF_E_TIMEOUT; ctrl->skip = 1; }
+        else if (mode == HBF_MODE_SHUTDOWN) { ctrl->code = HBF_E_LINK_SHUTDOWN; ctrl->skip = 1; }
+        else if (mode == HBF_MODE_SEVERE) { ctrl->code = HBF_E_THROTTLED; ctrl->skip = 1; }
+    }
+    for (uint32_t r = tid; r < n_queues; r += blockDim.x) busy_stage[r] = busy[r];
+    int64_t *s = reinterpret_cast<int64_t *>(stats_stage);
+    for (uint32_t i = tid; i < n_dies * 6u; i += blockDim.x) s[i] = 0;
+    for (int i = tid; i < kMaxPasses * kRadix; i += blockDim.x) hist[i] = 0u;
+}
+
+// =====================================================================================================
+// classify: 16-byte coalesced loads of the 24-byte records into shared memory, then per record the
+// range filter, the decode and the sort key (queue << 47 | issue).  NATIVE rows are answered here.
+// =====================================================================================================
+constexpr int kClsThreads = 256;
+constexpr int kClsItems = 4;
+constexpr int kClsTile = kClsThreads * kClsItems;       // 1024 records = 24 KiB
+
+__global__ void __launch_bounds__(kClsThreads)
+k_classify(const hbf_access_t *__restrict__ acc, uint64_t n, const RangeSnap *__restrict__ ranges_g,
+           const ModelParams *__restrict__ mp_g, BatchCtrl *ctrl, uint64_t *__restrict__ keys,
+           uint8_t *__restrict__ status, int64_t *__restrict__ completion, int64_t *__restrict__ stall) {
+    __shared__ RangeSnap rs;
+    __shared__ ModelParams mp;
+    __shared__ __align__(16) uint64_t rec[kClsTile * 3];
+    if (ctrl->skip) return;
+    const int tid = threadIdx.x;
+    for (int i = tid; i < (int)(sizeof(RangeSnap) / 4); i += kClsThreads)
+        reinterpret_cast<uint32_t *>(&rs)[i] = reinterpret_cast<const uint32_t *>(ranges_g)[i];
+    for (int i = tid; i < (int)(sizeof(ModelParams) / 4); i += kClsThreads)
+        reinterpret_cast<uint32_t *>(&mp)[i] = reinterpret_cast<const uint32_t *>(mp_g)[i];
+    const bool aligned16 = (reinterpret_cast<uintptr_t>(acc) & 15u) == 0;
+    const uint64_t sentinel = (uint64_t)mp_g->n_queues << kIssueBits;
+
+    unsigned long long n_native = 0, n_ready = 0, n_fault = 0, k_or = 0, k_and = ~0ull;
+    unsigned unsorted = 0;
+    const uint64_t n_tiles = (n + kClsTile - 1) / kClsTile;
+    for (uint64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+        const uint64_t base = tile * kClsTile;
+        const int cnt = (int)min((uint64_t)kClsTile, n - base);
+        __syncthreads();
+        const uint64_t *src = reinterpret_cast<const uint64_t *>(acc + base);
+        if (cnt == kClsTile && aligned16) {
+            const uint4 *s4 = reinterpret_cast<const uint4 *>(src);
+            uint4 *d4 = reinterpret_cast<uint4 *>(rec);
+#pragma unroll
+            for (int k = 0; k < kClsTile * 24 / 16 / kClsThreads; ++k) d4[tid + k * kClsThreads] = __ldg(s4 + tid + k * kClsThreads);
+        } else {
+            for (int i = tid; i < cnt * 3; i += kClsThreads) rec[i] = __ldg(src + i);
+        }
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < kClsItems; ++k) {
+            const int li = tid + k * kClsThreads;
+            if (li >= cnt) break;
+            const uint64_t i = base + li;
+            const uint64_t addr = rec[li * 3];
+            const int64_t issue = (int64_t)rec[li * 3 + 1];
+            const uint64_t bf = rec[li * 3 + 2];
+            const uint32_t bytes = (uint32_t)bf, flags = (uint32_t)(bf >> 32);
+            int64_t prev;
+            if (li > 0) prev = (int64_t)rec[li * 3 - 2];
+            else prev = i > 0 ? acc[i - 1].issue_ns : INT64_MIN;
+            unsorted |= (issue < prev) ? 1u : 0u;
+            int g = 0;
+            const int st = classify(rs, addr, issue, bytes, flags, &g);
+            uint64_t key = sentinel;
+            if (st == HBF_ST_READY) {
+                const uint64_t off = rs.media_offset[g] + (addr - rs.base[g]);
+                const Decoded d = decode(mp, off, bytes);
+                key = ((uint64_t)d.queue << kIssueBits) | (uint64_t)issue;
+                ++n_ready;
+            } else if (st == HBF_ST_NATIVE) {
+                ++n_native;
+                completion[i] = issue; stall[i] = 0;
+            } else {
+                ++n_fault;
+            }
+            keys[i] = key;
+            k_or |= key; k_and &= key;
+            if (status) status[i] = (uint8_t)st;
+        }
+    }
+    n_native = (unsigned long long)warp_sum((long long)n_native);
+    n_ready = (unsigned long long)warp_sum((long long)n_ready);
+    n_fault = (unsigned long long)warp_sum((long long)n_fault);
+    k_or = warp_or(k_or); k_and = warp_and(k_and);
+    unsorted = __any_sync(0xffffffffu, unsorted);
+    if (lane_id() == 0) {
+        if (n_native) atomicAdd(&ctrl->n_native, n_native);
+        if (n_ready) atomicAdd(&ctrl->n_ready, n_ready);
+        if (n_fault) atomicAdd(&ctrl->n_fault, n_fault);
+        atomicOr(&ctrl->key_or, k_or); atomicAnd(&ctrl->key_and, k_and);
+        if (unsorted) atomicOr(&ctrl->unsorted, 1u);
+    }
+}
+
+// =====================================================================================================
+// plan: refuse the batch on any fail-closed access; otherwise choose the radix passes.  Only bits that
+// differ between keys take part; a batch already in issue order needs the queue bits only (the sort is
+// stable, so issue order and then batch index survive as the minor keys).
+// =====================================================================================================
+__device__ __forceinline__ uint64_t compact_key(uint64_t key, uint32_t lo_bits, uint32_t hi_bits) {
+    const uint64_t lo = lo_bits ? (key & ((1ull << lo_bits) - 1ull)) : 0ull;
+    const uint64_t hi = (key >> kIssueBits) & ((1ull << hi_bits) - 1ull);
+    return lo | (hi << lo_bits);
+}
+
+__global__ void k_plan(BatchCtrl *ctrl, int force_full) {
+    if (threadIdx.x != 0 || ctrl->skip) return;
+    if (ctrl->n_fault) { ctrl->code = HBF_E_ACCESS_FAULT; ctrl->skip = 1; return; }
+    const uint64_t diff = ctrl->key_or ^ ctrl->key_and;
+    const uint64_t dlo = diff & kIssueMask, dhi = diff >> kIssueBits;
+    uint32_t lo = (ctrl->unsorted || force_full) ? (dlo ? 64u - (uint32_t)__clzll((long long)dlo) : 0u) : 0u;
+    uint32_t hi = dhi ? 64u - (uint32_t)__clzll((long long)dhi) : 0u;
+    const uint32_t total = lo + hi;
+    const uint32_t np = (total + 7u) / 8u;
+    SortPlan p; p.n_passes = np; p.lo_bits = lo; p.hi_bits = hi;
+    uint32_t shift = 0;
+    for (uint32_t i = 0; i < (uint32_t)kMaxPasses; ++i) {
+        uint32_t b = 0;
+        if (i < np) b = total / np + (i < total % np ? 1u : 0u);
+        p.shift[i] = shift; p.bits[i] = b; shift += b;
+    }
+    ctrl->plan = p;
+}
+
+// =====================================================================================================
+// histogram of every planned digit (shared-memory bins, warp-aggregated with match_any)
+// =====================================================================================================
+constexpr int kHistThreads = 512;
+
+__global__ void __launch_bounds__(kHistThreads)
+k_hist(const uint64_t *__restrict__ keys, uint64_t n, const BatchCtrl *ctrl, uint32_t *hist) {
+    __shared__ uint32_t sh[kMaxPasses * kRadix];
+    if (ctrl->skip) return;
+    const SortPlan p = ctrl->plan;
+    if (p.n_passes == 0) return;
+    for (int i = threadIdx.x; i < kMaxPasses * kRadix; i += kHistThreads) sh[i] = 0u;
+    __syncthreads();
+    const uint64_t stride = (uint64_t)gridDim.x * kHistThreads;
+    const uint64_t n_round = (n + 31ull) & ~31ull;         // whole warps stay in the loop together
+    for (uint64_t i = (uint64_t)blockIdx.x * kHistThreads + threadIdx.x; i < n_round; i += stride) {
+        const bool valid = i < n;
+        const uint64_t ck = valid ? compact_key(keys[i], p.lo_bits, p.hi_bits) : 0ull;
+        for (uint32_t k = 0; k < p.n_passes; ++k) {
+            const uint32_t d = valid ? (uint32_t)(ck >> p.shift[k]) & ((1u << p.bits[k]) - 1u) : 0xffffffffu;
+            const unsigned peers = __match_any_sync(0xffffffffu, d);
+            if (valid && (peers & lanemask_lt()) == 0u) atomicAdd(&sh[k * kRadix + d], (uint32_t)__popc(peers));
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < (int)p.n_passes * kRadix; i += kHistThreads)
+        if (sh[i]) atomicAdd(&hist[i], sh[i]);
+}
+
+// =====================================================================================================
+// one onesweep pass: stable partition of (key, index) by one digit, in a single sweep.  Tiles take
+// their number from a counter (so every predecessor of a running tile has started), rank their keys
+// per warp with match_any, publish the tile's digit counts and look back over earlier tiles for the
+// running totals.  Look-back words carry flag and count in one 32-bit word.
+// =====================================================================================================
+constexpr int kSortThreads = 512;
+constexpr int kSortItems = 8;
+constexpr int kSortTile = kSortThreads * kSortItems;     // 4096
+constexpr int kSortWarps = kSortThreads / 32;
+constexpr size_t kSortSmem = (size_t)kSortTile * 12 + (size_t)kSortWarps * kRadix * 4;
+constexpr uint32_t kFlagAgg = 1u << 30, kFlagPrefix = 2u << 30, kCountMask = (1u << 30) - 1u;
+
+__global__ void __launch_bounds__(kSortThreads)
+k_sort_pass(int pass, uint64_t n, BatchCtrl *ctrl, DevState *state, const uint32_t *__restrict__ hist,
+            uint64_t *keys0, uint64_t *keys1, uint32_t *idx0, uint32_t *idx1, uint32_t *desc0, uint32_t *desc1) {
+    extern __shared__ __align__(16) unsigned char sort_smem[];
+    uint64_t *s_keys = reinterpret_cast<uint64_t *>(sort_smem);                       // [kSortTile]
+    uint32_t *s_idx = reinterpret_cast<uint32_t *>(s_keys + kSortTile);               // [kSortTile]
+    uint32_t *s_cnt = s_idx + kSortTile;                                              // [kSortWarps][kRadix]
+    __shared__ uint32_t s_local_start[kRadix];
+    __shared__ uint32_t s_delta[kRadix];
+    __shared__ uint32_t s_warp_tot[kRadix / 32], s_hist_tot[kRadix / 32];
+    __shared__ uint32_t s_tile;
+    if (ctrl->skip) return;
+    const SortPlan &pl = ctrl->plan;
+    if (pass >= (int)pl.n_passes) return;
+    const uint32_t lo_bits = pl.lo_bits, hi_bits = pl.hi_bits, shift = pl.shift[pass];
+    const uint32_t dmask = (1u << pl.bits[pass]) - 1u;
+    const uint64_t *kin = (pass & 1) ? keys1 : keys0;
+    uint64_t *kout = (pass & 1) ? keys0 : keys1;
+    const uint32_t *iin = (pass & 1) ? idx1 : idx0;
+    uint32_t *iout = (pass & 1) ? idx0 : idx1;
+    uint32_t *desc = (pass & 1) ? desc1 : desc0;
+    uint32_t *desc_next = (pass & 1) ? desc0 : desc1;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    if (tid == 0) s_tile = atomicAdd(&ctrl->tile_counter[pass], 1u);
+    for (int i = tid; i < kSortWarps * kRadix; i += kSortThreads) s_cnt[i] = 0u;
+    __syncthreads();
+    const uint32_t tile = s_tile;
+    const uint64_t base = (uint64_t)tile * kSortTile;
+    if (tid < kRadix) desc_next[(uint64_t)tile * kRadix + tid] = 0u;     // ready for the pass after this one
+
+    // load, warp-striped: the warp's chunk is contiguous and item j of lane l sits at j*32 + l
+    uint64_t key[kSortItems]; uint32_t val[kSortItems]; uint32_t dig[kSortItems]; uint32_t rank[kSortItems];
+    const uint64_t wbase = base + (uint64_t)warp * (32 * kSortItems);
+#pragma unroll
+    for (int j = 0; j < kSortItems; ++j) {
+        const uint64_t i = wbase + j * 32 + lane;
+        if (i < n) {
+            key[j] = kin[i];
+            val[j] = pass == 0 ? (uint32_t)i : iin[i];
+            dig[j] = (uint32_t)(compact_key(key[j], lo_bits, hi_bits) >> shift) & dmask;
+        } else {
+            key[j] = ~0ull; val[j] = 0u; dig[j] = kRadix - 1;       // padding ranks behind every real key
+        }
+    }
+    // rank inside the warp, in memory order
+    uint32_t *wcnt = s_cnt + warp * kRadix;
+#pragma unroll
+    for (int j = 0; j < kSortItems; ++j) {
+        const unsigned peers = __match_any_sync(0xffffffffu, dig[j]);
+        const uint32_t before = wcnt[dig[j]];
+        rank[j] = before + (uint32_t)__popc(peers & lanemask_lt());
+        __syncwarp();
+        if ((peers >> lane) <= 1u) wcnt[dig[j]] = before + (uint32_t)__popc(peers);    // highest peer lane writes
+        __syncwarp();
+    }
+    __syncthreads();
+
+    // per digit: exclusive prefix over warps and the tile total; publish it; block-wide exclusive scans of
+    // the tile's digit counts (positions inside the tile) and of the pass histogram (global digit starts)
+    uint32_t tile_count = 0, local_incl = 0, hist_incl = 0, hist_mine = 0;
+    if (tid < kRadix) {
+#pragma unroll
+        for (int w = 0; w < kSortWarps; ++w) { const uint32_t c = s_cnt[w * kRadix + tid]; s_cnt[w * kRadix + tid] = tile_count; tile_count += c; }
+        st_relaxed_u32(desc + (uint64_t)tile * kRadix + tid, (tile == 0 ? kFlagPrefix : kFlagAgg) | tile_count);
+        hist_mine = hist[pass * kRadix + tid];
+        local_incl = tile_count; hist_incl = hist_mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t t = __shfl_up_sync(0xffffffffu, local_incl, o), u = __shfl_up_sync(0xffffffffu, hist_incl, o);
+            if (lane >= o) { local_incl += t; hist_incl += u; }
+        }
+        if (lane == 31) { s_warp_tot[warp] = local_incl; s_hist_tot[warp] = hist_incl; }
+    }
+    __syncthreads();
+    if (tid < kRadix) {
+        uint32_t woff = 0, hoff = 0;
+        for (int w = 0; w < warp; ++w) { woff += s_warp_tot[w]; hoff += s_hist_tot[w]; }
+        const uint32_t local_start = local_incl - tile_count + woff;
+        const uint32_t gstart = hist_incl - hist_mine + hoff;
+        // look back over earlier tiles for the number of keys with this digit before this tile
+        uint32_t excl = 0;
+        bool failed = false;
+        for (int64_t t = (int64_t)tile - 1; t >= 0; --t) {
+            const uint32_t *p = desc + (uint64_t)t * kRadix + tid;
+            uint32_t v = ld_relaxed_u32(p), spins = 0;
+            while ((v >> 30) == 0u) {
+                if (++spins > kSpinLimit) { failed = true; break; }
+                __nanosleep(20);
+                v = ld_relaxed_u32(p);
+            }
+            if (failed) break;
+            excl += v & kCountMask;
+            if ((v >> 30) == 2u) break;
+        }
+        if (failed) { atomicExch(&ctrl->code, (int)HBF_E_TIMEOUT); state->poisoned = 1; }
+        if (tile != 0) st_relaxed_u32(desc + (uint64_t)tile * kRadix + tid, kFlagPrefix | ((excl + tile_count) & kCountMask));
+        s_local_start[tid] = local_start;
+        s_delta[tid] = gstart + excl - local_start;
+    }
+    __syncthreads();
+
+    // place keys at their position inside the tile, then write runs out
+#pragma unroll
+    for (int j = 0; j < kSortItems; ++j) {
+        const uint32_t pos = s_local_start[dig[j]] + wcnt[dig[j]] + rank[j];
+        s_keys[pos] = key[j]; s_idx[pos] = val[j];
+    }
+    __syncthreads();
+    const int cnt = (int)min((uint64_t)kSortTile, n - base);
+    for (int i = tid; i < cnt; i += kSortThreads) {
+        const uint64_t k = s_keys[i];
+        const uint32_t d = (uint32_t)(compact_key(k, lo_bits, hi_bits) >> shift) & dmask;
+        const uint32_t g = (uint32_t)i + s_delta[d];
+        kout[g] = k; iout[g] = s_idx[i];
+    }
+}
+
+// =====================================================================================================
+// scan + scatter: in sorted order every access is the max-plus map B -> max(B + s, a + s); queues are
+// segments.  A single-pass segmented scan with decoupled look-back gives each access the busy-until
+// value it leaves behind; completion and stall go straight back to the access's own index, per-die
+// totals are reduced with warp shuffles before they touch memory.
+// =====================================================================================================
+constexpr int kScanThreads = 256;
+constexpr int kScanItems = 8;
+constexpr int kScanTile = kScanThreads * kScanItems;     // 2048
+constexpr int kScanWarps = kScanThreads / 32;
+
+struct __align__(32) ScanDesc { int64_t S, M, value; uint32_t status; uint32_t pad; };
+struct Map { int64_t S, M; int f; };
+
+__device__ __forceinline__ Map compose(const Map &x, const Map &y) {      // x earlier, y later
+    if (y.f) return y;
+    Map r; r.f = x.f; r.S = x.S + y.S; r.M = max(x.M + y.S, y.M); return r;
+}
+__device__ __forceinline__ Map shfl_up_map(const Map &m, int o) {
+    Map r; r.S = __shfl_up_sync(0xffffffffu, m.S, o); r.M = __shfl_up_sync(0xffffffffu, m.M, o);
+    r.f = __shfl_up_sync(0xffffffffu, m.f, o); return r;
+}
+
+__global__ void __launch_bounds__(kScanThreads)
+k_scan(const hbf_access_t *__restrict__ acc, uint64_t n, const RangeSnap *__restrict__ ranges_g,
+       const ModelParams *__restrict__ mp_g, BatchCtrl *ctrl, DevState *state,
+       const uint64_t *keys0, const uint64_t *keys1, const uint32_t *idx0, const uint32_t *idx1,
+       ScanDesc *desc, const int64_t *__restrict__ busy, int64_t *busy_stage, hbf_die_stats_t *stats_stage,
+       int64_t *__restrict__ completion, int64_t *__restrict__ stall) {
+    __shared__ RangeSnap rs;
+    __shared__ ModelParams mp;
+    __shared__ uint32_t s_first_q[kScanThreads], s_last_q[kScanThreads];
+    __shared__ Map s_warp_map[kScanWarps];
+    __shared__ int64_t s_tile_in;
+    __shared__ uint32_t s_tile;
+    __shared__ long long s_die_acc[6];
+    __shared__ long long s_res[3];
+    if (ctrl->skip) return;
+    const uint64_t m = ctrl->n_ready;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) s_tile = atomicAdd(&ctrl->tile_counter[kMaxPasses], 1u);
+    for (int i = tid; i < (int)(sizeof(RangeSnap) / 4); i += kScanThreads)
+        reinterpret_cast<uint32_t *>(&rs)[i] = reinterpret_cast<const uint32_t *>(ranges_g)[i];
+    for (int i = tid; i < (int)(sizeof(ModelParams) / 4); i += kScanThreads)
+        reinterpret_cast<uint32_t *>(&mp)[i] = reinterpret_cast<const uint32_t *>(mp_g)[i];
+    if (tid < 6) s_die_acc[tid] = 0;
+    if (tid < 3) s_res[tid] = tid == 2 ? INT64_MIN : 0;
+    __syncthreads();
+    const uint32_t tile = s_tile;
+    const uint64_t base = (uint64_t)tile * kScanTile;
+    if (base >= m) return;
+    const uint32_t np = ctrl->plan.n_passes;
+    const uint64_t *keys = (np & 1u) ? keys1 : keys0;
+    const uint32_t *idxs = np == 0u ? nullptr : ((np & 1u) ? idx1 : idx0);
+    const int64_t q_ppm = ctrl->q_ppm;
+    const int cnt = (int)min((uint64_t)kScanTile, m - base);
+
+    // this thread's consecutive items
+    uint32_t queue[kScanItems], idx[kScanItems], post[kScanItems];
+    int64_t a[kScanItems], s[kScanItems], issue[kScanItems];
+    const int t0 = tid * kScanItems;
+    const int mine = max(0, min(kScanItems, cnt - t0));
+    {
+        uint64_t k[kScanItems];
+        if (mine == kScanItems) {
+            const ulonglong2 *k2 = reinterpret_cast<const ulonglong2 *>(keys + base + t0);
+#pragma unroll
+            for (int j = 0; j < kScanItems / 2; ++j) { const ulonglong2 v = k2[j]; k[2 * j] = v.x; k[2 * j + 1] = v.y; }
+            if (idxs) {
+                const uint4 *i4 = reinterpret_cast<const uint4 *>(idxs + base + t0);
+#pragma unroll
+                for (int j = 0; j < kScanItems / 4; ++j) { const uint4 v = i4[j]; idx[4 * j] = v.x; idx[4 * j + 1] = v.y; idx[4 * j + 2] = v.z; idx[4 * j + 3] = v.w; }
+            } else {
+#pragma unroll
+                for (int j = 0; j < kScanItems; ++j) idx[j] = (uint32_t)(base + t0 + j);
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < kScanItems; ++j) {
+                k[j] = j < mine ? keys[base + t0 + j] : 0ull;
+                idx[j] = j < mine ? (idxs ? idxs[base + t0 + j] : (uint32_t)(base + t0 + j)) : 0u;
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < kScanItems; ++j) { queue[j] = (uint32_t)(k[j] >> kIssueBits); issue[j] = (int64_t)(k[j] & kIssueMask); }
+    }
+    // gather the records and rebuild their service terms
+    long long acc_busy = 0, acc_br = 0, acc_bp = 0, acc_e = 0, acc_nr = 0, acc_np = 0;
+    uint32_t run_die = 0xffffffffu;
+    auto flush_run = [&](uint32_t die) {
+        long long *d = reinterpret_cast<long long *>(stats_stage + die);
+        if (acc_busy) atomicAdd((unsigned long long *)&d[0], (unsigned long long)acc_busy);
+        if (acc_br) atomicAdd((unsigned long long *)&d[1], (unsigned long long)acc_br);
+        if (acc_bp) atomicAdd((unsigned long long *)&d[2], (unsigned long long)acc_bp);
+        if (acc_e) atomicAdd((unsigned long long *)&d[3], (unsigned long long)acc_e);
+        if (acc_nr) atomicAdd((unsigned long long *)&d[4], (unsigned long long)acc_nr);
+        if (acc_np) atomicAdd((unsigned long long *)&d[5], (unsigned long long)acc_np);
+        acc_busy = acc_br = acc_bp = acc_e = acc_nr = acc_np = 0;
+    };
+    uint64_t r_addr[kScanItems], r_bf[kScanItems];
+#pragma unroll
+    for (int j = 0; j < kScanItems; ++j) {
+        if (j < mine) {
+            const uint64_t *p = reinterpret_cast<const uint64_t *>(acc + idx[j]);
+            r_addr[j] = ld_nc_u64(p); r_bf[j] = ld_nc_u64(p + 2);
+        }
+    }
+    long long sum_s = 0;
+#pragma unroll
+    for (int j = 0; j < kScanItems; ++j) {
+        if (j < mine) {
+            const uint32_t bytes = (uint32_t)r_bf[j], op = (uint32_t)(r_bf[j] >> 32) & 1u;
+            int g = 0;
+            classify(rs, r_addr[j], issue[j], bytes, op, &g);
+            const uint64_t off = rs.media_offset[g] + (r_addr[j] - rs.base[g]);
+            const Decoded d = decode(mp, off, bytes);
+            const Terms t = service_terms(mp, bytes, d.npages, op, q_ppm);
+            s[j] = t.s;
+            if (op) { a[j] = issue[j] + t.xfer; post[j] = 0u; } else { a[j] = issue[j]; post[j] = (uint32_t)t.xfer; }
+            if (d.die != run_die) { if (run_die != 0xffffffffu) flush_run(run_die); run_die = d.die; }
+            acc_busy += t.s; acc_e += t.energy; sum_s += t.s;
+            if (op) { acc_bp += t.cb; acc_np += 1; } else { acc_br += t.cb; acc_nr += 1; }
+        }
+    }
+    // segment heads: a queue change against the previous sorted element
+    s_first_q[tid] = mine > 0 ? queue[0] : 0xffffffffu;
+    s_last_q[tid] = mine > 0 ? queue[mine - 1] : 0xffffffffu;
+    __syncthreads();
+    uint32_t prev_q, next_q;
+    if (tid > 0) prev_q = s_last_q[tid - 1];
+    else prev_q = base > 0 ? (uint32_t)(keys[base - 1] >> kIssueBits) : 0xffffffffu;
+    if (t0 + mine < cnt) next_q = s_first_q[tid + 1];
+    else next_q = (base + cnt < m) ? (uint32_t)(keys[base + cnt] >> kIssueBits) : 0xffffffffu;
+
+    // thread-local fold, then block scan of the thread maps
+    Map tm; tm.f = 0; tm.S = 0; tm.M = kNegInf;
+    {
+        uint32_t pq = prev_q;
+#pragma unroll
+        for (int j = 0; j < kScanItems; ++j) {
+            if (j < mine) {
+                Map e; e.S = s[j]; e.f = queue[j] != pq;
+                e.M = e.f ? max(busy[queue[j]], a[j]) + s[j] : a[j] + s[j];
+                tm = compose(tm, e);
+                pq = queue[j];
+            }
+        }
+    }
+    Map incl = tm;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const Map up = shfl_up_map(incl, o); if (lane >= o) incl = compose(up, incl); }
+    if (lane == 31) s_warp_map[warp] = incl;
+    __syncthreads();
+    Map wprefix; wprefix.f = 0; wprefix.S = 0; wprefix.M = kNegInf;
+    for (int w = 0; w < warp; ++w) wprefix = compose(wprefix, s_warp_map[w]);
+    Map excl = shfl_up_map(incl, 1);
+    if (lane == 0) { excl.f = 0; excl.S = 0; excl.M = kNegInf; }
+    excl = compose(wprefix, excl);
+
+    // tile aggregate, publish, look back
+    if (tid == kScanThreads - 1) {
+        const Map agg = compose(excl, tm);
+        ScanDesc *my = desc + tile;
+        int64_t tile_in = 0;
+        if (agg.f) {
+            st_relaxed_s64(&my->value, agg.M);
+            st_release_u32(&my->status, 2u);
+            // the tile's own first segment may still continue the previous tile's queue
+        } else {
+            st_relaxed_s64(&my->S, agg.S); st_relaxed_s64(&my->M, agg.M);
+            st_release_u32(&my->status, 1u);
+        }
+        // incoming busy-until for the tile's first element (unused when that element is a segment head)
+        if (tile > 0) {
+            int64_t S_acc = 0, M_acc = kNegInf;
+            bool failed = false;
+            for (int64_t t = (int64_t)tile - 1; t >= 0; --t) {
+                const ScanDesc *p = desc + t;
+                uint32_t stt = ld_acquire_u32(&p->status), spins = 0;
+                while (stt == 0u) {
+                    if (++spins > kSpinLimit) { failed = true; break; }
+                    __nanosleep(20);
+                    stt = ld_acquire_u32(&p->status);
+                }
+                if (failed) break;
+                if (stt == 2u) {
+                    // a later upgrade from 1 to 2 is also fine: value is complete once status reads 2
+                    const int64_t v = ld_relaxed_s64(&p->value);
+                    tile_in = max(v + S_acc, M_acc);
+                    break;
+                }
+                const int64_t St = ld_relaxed_s64(&p->S), Mt = ld_relaxed_s64(&p->M);
+                M_acc = max(Mt + S_acc, M_acc); S_acc += St;
+            }
+            if (failed) { atomicExch(&ctrl->code, (int)HBF_E_TIMEOUT); state->poisoned = 1; }
+        }
+        if (!agg.f) {
+            st_relaxed_s64(&my->value, max(tile_in + agg.S, agg.M));
+            st_release_u32(&my->status, 2u);
+        }
+        s_tile_in = tile_in;
+    }
+    __syncthreads();
+    int64_t B = excl.f ? excl.M : max(s_tile_in + excl.S, excl.M);
+
+    // apply: serve this thread's items in order
+    long long sum_stall = 0, max_c = INT64_MIN;
+    {
+        uint32_t pq = prev_q;
+#pragma unroll
+        for (int j = 0; j < kScanItems; ++j) {
+            if (j < mine) {
+                if (queue[j] != pq) B = busy[queue[j]];
+                const int64_t start = max(a[j], B);
+                B = start + s[j];
+                const int64_t c = B + (int64_t)post[j];
+                completion[idx[j]] = c;
+                stall[idx[j]] = c - issue[j];
+                sum_stall += c - issue[j];
+                max_c = max(max_c, (long long)c);
+                const uint32_t nq = j + 1 < mine ? queue[j + 1] : next_q;
+                if (nq != queue[j]) busy_stage[queue[j]] = B;       // last access of its queue in this batch
+                pq = queue[j];
+            }
+        }
+    }
+    // per-die totals: whole warps on one die reduce by shuffle into the tile's slot
+    {
+        const uint32_t tile_die = __shfl_sync(0xffffffffu, run_die, 0);
+        const bool uniform = __all_sync(0xffffffffu, run_die == tile_die || run_die == 0xffffffffu) && tile_die != 0xffffffffu;
+        __shared__ uint32_t s_tile_die;
+        if (tid == 0) s_tile_die = run_die;
+        __syncthreads();
+        if (uniform && tile_die == s_tile_die) {
+            acc_busy = warp_sum(acc_busy); acc_br = warp_sum(acc_br); acc_bp = warp_sum(acc_bp);
+            acc_e = warp_sum(acc_e); acc_nr = warp_sum(acc_nr); acc_np = warp_sum(acc_np);
+            if (lane == 0) {
+                atomicAdd((unsigned long long *)&s_die_acc[0], (unsigned long long)acc_busy);
+                atomicAdd((unsigned long long *)&s_die_acc[1], (unsigned long long)acc_br);
+                atomicAdd((unsigned long long *)&s_die_acc[2], (unsigned long long)acc_bp);
+                atomicAdd((unsigned long long *)&s_die_acc[3], (unsigned long long)acc_e);
+                atomicAdd((unsigned long long *)&s_die_acc[4], (unsigned long long)acc_nr);
+                atomicAdd((unsigned long long *)&s_die_acc[5], (unsigned long long)acc_np);
+            }
+        } else if (run_die != 0xffffffffu) {
+            flush_run(run_die);
+        }
+        sum_stall = warp_sum(sum_stall); sum_s = warp_sum(sum_s); max_c = warp_max(max_c);
+        if (lane == 0) {
+            atomicAdd((unsigned long long *)&s_res[0], (unsigned long long)sum_stall);
+            atomicAdd((unsigned long long *)&s_res[1], (unsigned long long)sum_s);
+            atomicMax(&s_res[2], max_c);
+        }
+        __syncthreads();
+        if (tid == 0) {
+            long long *d = reinterpret_cast<long long *>(stats_stage + s_tile_die);
+            for (int k = 0; k < 6; ++k) if (s_die_acc[k]) atomicAdd((unsigned long long *)&d[k], (unsigned long long)s_die_acc[k]);
+            atomicAdd((unsigned long long *)&ctrl->modeled_ns, (unsigned long long)s_res[0]);
+            atomicAdd((unsigned long long *)&ctrl->service_ns, (unsigned long long)s_res[1]);
+            atomicMax(&ctrl->max_completion_ns, s_res[2]);
+        }
+    }
+}
+
+// =====================================================================================================
+// finish: commit the staged state, or zero the outputs of a refused batch; write the batch summary
+// =====================================================================================================
+__global__ void k_finish(uint64_t n, BatchCtrl *ctrl, DevState *state, int64_t *busy, const int64_t *busy_stage,
+                         int64_t *pending, const hbf_die_stats_t *stats_stage, hbf_die_stats_t *die_stats,
+                         int64_t *completion, int64_t *stall, hbf_batch_result_t *result,
+                         uint32_t n_queues, uint32_t n_dies) {
+    const int code = ctrl->code;
+    const uint64_t gtid = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const uint64_t gsz = (uint64_t)gridDim.x * blockDim.x;
+    if (code == HBF_E_ACCESS_FAULT || code == HBF_E_TIMEOUT) {
+        for (uint64_t i = gtid; i < n; i += gsz) { completion[i] = 0; stall[i] = 0; }
+        if (die_stats) for (uint64_t i = gtid; i < (uint64_t)n_dies * 6u; i += gsz) reinterpret_cast<int64_t *>(die_stats)[i] = 0;
+    } else if (code == HBF_OK) {
+        for (uint64_t r = gtid; r < n_queues; r += gsz) busy[r] = busy_stage[r];
+        for (uint64_t d = gtid; d < n_dies; d += gsz) {
+            pending[d] += stats_stage[d].energy_pj;
+            if (die_stats) die_stats[d] = stats_stage[d];
+        }
+    }
+    if (gtid == 0) {
+        hbf_batch_result_t r;
+        r.code = code; r.mode = ctrl->mode; r.q_ppm = ctrl->q_ppm;
+        r.n_native = code == HBF_OK || code == HBF_E_ACCESS_FAULT ? ctrl->n_native : 0;
+        r.n_modeled = code == HBF_OK ? ctrl->n_ready : 0;
+        r.n_fault = ctrl->n_fault;
+        r.modeled_ns = code == HBF_OK ? ctrl->modeled_ns : 0;
+        r.service_ns = code == HBF_OK ? ctrl->service_ns : 0;
+        r.max_completion_ns = code == HBF_OK && ctrl->n_ready ? ctrl->max_completion_ns : 0;
+        *result = r;
+    }
+}
+
+// copy of the served order out of the workspace (sort path only)
+__global__ void k_queue_order(const BatchCtrl *ctrl, const uint32_t *idx0, const uint32_t *idx1, uint32_t *out, uint64_t n) {
+    const uint64_t m = ctrl->n_ready;
+    const uint32_t np = ctrl->plan.n_passes;
+    const uint32_t *src = np == 0u ? nullptr : ((np & 1u) ? idx1 : idx0);
+    for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < m && i < n; i += (uint64_t)gridDim.x * blockDim.x)
+        out[i] = src ? src[i] : (uint32_t)i;
+}
+
+// =====================================================================================================
+// host side
+// =====================================================================================================
+static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+size_t workspace_layout(uint64_t n, uint32_t n_queues, Workspace *ws, void *base_ptr) {
+    (void)n_queues;
+    const uint64_t nn = n ? n : 1;
+    const uint64_t sort_tiles = (nn + kSortTile - 1) / kSortTile, scan_tiles = (nn + kScanTile - 1) / kScanTile;
+    size_t off = 0;
+    char *b = static_cast<char *>(base_ptr);
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return b ? b + o : nullptr; };
+    void *k0 = take(nn * 8), *k1 = take(nn * 8), *i0 = take(nn * 4), *i1 = take(nn * 4);
+    void *h = take((size_t)kMaxPasses * kRadix * 4);
+    void *d0 = take(sort_tiles * kRadix * 4), *d1 = take(sort_tiles * kRadix * 4);
+    void *sd = take(scan_tiles * sizeof(ScanDesc));
+    if (ws) {
+        ws->keys[0] = (uint64_t *)k0; ws->keys[1] = (uint64_t *)k1; ws->idx[0] = (uint32_t *)i0; ws->idx[1] = (uint32_t *)i1;
+        ws->hist = (uint32_t *)h; ws->sort_desc[0] = (uint32_t *)d0; ws->sort_desc[1] = (uint32_t *)d1;
+        ws->scan_desc = sd; ws->inorder_desc = nullptr; ws->bytes = off;
+    }
+    return off;
+}
+
+cudaError_t launch_submit(const SubmitArgs &a, cudaStream_t st) {
+    const uint64_t n = a.n;
+    k_begin<<<1, 256, 0, st>>>(a.ctrl, a.state, a.busy, a.busy_stage, a.stats_stage, a.ws.hist, a.mp.n_queues, a.mp.n_dies);
+    if (n > 0) {
+        const uint64_t sort_tiles = (n + kSortTile - 1) / kSortTile, scan_tiles = (n + kScanTile - 1) / kScanTile;
+        cudaError_t e = cudaMemsetAsync(a.ws.sort_desc[0], 0, sort_tiles * kRadix * 4, st);
+        if (e != cudaSuccess) return e;
+        e = cudaMemsetAsync(a.ws.scan_desc, 0, scan_tiles * sizeof(ScanDesc), st);
+        if (e != cudaSuccess) return e;
+        const uint64_t cls_tiles = (n + kClsTile - 1) / kClsTile;
+        const unsigned cls_grid = (unsigned)std::min<uint64_t>(cls_tiles, (uint64_t)a.sm_count * 8);
+        k_classify<<<cls_grid, kClsThreads, 0, st>>>(a.acc, n, a.ranges, a.mp_dev, a.ctrl, a.ws.keys[0], a.status,
+                                                     a.completion, a.stall);
+        k_plan<<<1, 32, 0, st>>>(a.ctrl, a.path == HBF_PATH_SORT_FULL ? 1 : 0);
+        const unsigned hist_grid = (unsigned)std::min<uint64_t>((n + kHistThreads * 8 - 1) / (kHistThreads * 8), (uint64_t)a.sm_count * 4);
+        k_hist<<<hist_grid, kHistThreads, 0, st>>>(a.ws.keys[0], n, a.ctrl, a.ws.hist);
+        static bool attr_set = false;
+        if (!attr_set) {
+            e = cudaFuncSetAttribute(k_sort_pass, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSortSmem);
+            if (e != cudaSuccess) return e;
+            attr_set = true;
+        }
+        for (int p = 0; p < kMaxPasses; ++p)
+            k_sort_pass<<<(unsigned)sort_tiles, kSortThreads, kSortSmem, st>>>(p, n, a.ctrl, a.state, a.ws.hist, a.ws.keys[0], a.ws.keys[1],
+                                                                       a.ws.idx[0], a.ws.idx[1], a.ws.sort_desc[0], a.ws.sort_desc[1]);
+        k_scan<<<(unsigned)scan_tiles, kScanThreads, 0, st>>>(a.acc, n, a.ranges, a.mp_dev, a.ctrl, a.state, a.ws.keys[0], a.ws.keys[1],
+                                                             a.ws.idx[0], a.ws.idx[1], (ScanDesc *)a.ws.scan_desc, a.busy,
+                                                             a.busy_stage, a.stats_stage, a.completion, a.stall);
+    }
+    const unsigned fin_grid = (unsigned)std::max<uint64_t>(1, std::min<uint64_t>((n + 1023) / 1024, (uint64_t)a.sm_count * 4));
+    k_finish<<<fin_grid, 256, 0, st>>>(n, a.ctrl, a.state, a.busy, a.busy_stage, a.pending, a.stats_stage, a.die_stats,
+                                       a.completion, a.stall, a.result, a.mp.n_queues, a.mp.n_dies);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_queue_order(const BatchCtrl *ctrl, const Workspace &ws, uint32_t *out, uint64_t n, cudaStream_t st) {
+    if (n == 0) return cudaSuccess;
+    k_queue_order<<<(unsigned)std::min<uint64_t>((n + 255) / 256, 1184), 256, 0, st>>>(ctrl, ws.idx[0], ws.idx[1], out, n);
+    return cudaGetLastError();
+}
+
+}  // namespace hbf

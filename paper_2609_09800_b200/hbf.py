@@ -1,0 +1,311 @@
+"""Thin ctypes binding of ``libhbf.so`` (``include/hbf.h``): argument marshalling only.
+
+Every step of the service model runs in the library's CUDA kernels.  PyTorch is used for device
+memory and streams.  There is no CPU fallback: if the library has not been built, or no CUDA device
+is present, the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SO = os.path.join(_HERE, "libhbf.so")
+
+OK, E_INVAL, E_RANGE_OVERLAP, E_RANGE_FULL, E_CAPACITY, E_WORKSPACE, E_CUDA = 0, -1, -2, -3, -4, -5, -6
+E_ACCESS_FAULT, E_THROTTLED, E_LINK_SHUTDOWN, E_TIMEOUT, E_NOMEM = -7, -8, -9, -10, -11
+ST_NATIVE, ST_READY, ST_FAULT_PARTIAL, ST_FAULT_PERM, ST_UNSUPPORTED = range(5)
+MODE_NORMAL, MODE_LIGHT, MODE_SEVERE, MODE_SHUTDOWN = range(4)
+PATH_AUTO, PATH_SORT, PATH_INORDER, PATH_SORT_FULL = range(4)
+
+ACCESS_DTYPE = np.dtype([("addr", "<u8"), ("issue_ns", "<i8"), ("bytes", "<u4"), ("flags", "<u4")])
+DIE_STATS_DTYPE = np.dtype([(k, "<i8") for k in
+                            ("busy_ns", "bytes_read", "bytes_prog", "energy_pj", "n_read", "n_prog")])
+
+EXPORTS = ("hbf_create", "hbf_destroy", "hbf_register_range", "hbf_clear_ranges", "hbf_workspace_bytes",
+           "hbf_submit_batch", "hbf_last_result", "hbf_thermal_step", "hbf_force_mode", "hbf_get_mode",
+           "hbf_reset", "hbf_set_path", "hbf_get_state", "hbf_set_state", "hbf_get_busy_until",
+           "hbf_get_pending_energy", "hbf_get_temps", "hbf_euler_limit_ns", "hbf_queue_order", "hbf_strerror")
+
+
+class hbf_config_t(C.Structure):
+    _fields_ = [
+        ("channels", C.c_uint32), ("dies", C.c_uint32), ("planes", C.c_uint32),
+        ("page_bytes", C.c_uint32), ("stripe_bytes", C.c_uint32), ("queue_level", C.c_uint32),
+        ("capacity_bytes", C.c_uint64),
+        ("t_read_ns", C.c_int64), ("t_prog_ns", C.c_int64), ("chan_bytes_per_us", C.c_uint64),
+        ("read_granule", C.c_uint32), ("prog_granule", C.c_uint32),
+        ("e_cmd_read_pj", C.c_int64), ("e_byte_read_pj", C.c_int64),
+        ("e_cmd_prog_pj", C.c_int64), ("e_byte_prog_pj", C.c_int64),
+        ("grid_h", C.c_uint32), ("grid_w", C.c_uint32), ("n_sub", C.c_uint32), ("n_regions", C.c_uint32),
+        ("ambient_c", C.c_float), ("rtt_c", C.c_float), ("ltt_c", C.c_float), ("stt_c", C.c_float),
+        ("shutdown_c", C.c_float),
+        ("q_light_ppm", C.c_int64),
+        ("cell_C", C.c_void_p), ("cell_Gx", C.c_void_p), ("cell_Gy", C.c_void_p), ("cell_Gsink", C.c_void_p),
+        ("cell_region", C.c_void_p), ("die_region", C.c_void_p), ("region_kind", C.c_void_p),
+        ("region_idle_w", C.c_void_p),
+    ]
+
+
+class hbf_batch_result_t(C.Structure):
+    _fields_ = [("code", C.c_int32), ("mode", C.c_int32), ("q_ppm", C.c_int64),
+                ("n_native", C.c_uint64), ("n_modeled", C.c_uint64), ("n_fault", C.c_uint64),
+                ("modeled_ns", C.c_int64), ("service_ns", C.c_int64), ("max_completion_ns", C.c_int64)]
+
+    def as_dict(self):
+        return {k: getattr(self, k) for k, _ in self._fields_}
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _SO
+
+
+def lib():
+    """The loaded CUDA library.  Raises if it has not been built (python -m paper_2609_09800_b200.build)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_SO):
+            raise RuntimeError("libhbf.so is missing: build it with `python -m paper_2609_09800_b200.build` "
+                               "(nvcc, sm_100a); there is no CPU fallback")
+        L = C.CDLL(_SO)
+        vp, u64, u32, i64, i32 = C.c_void_p, C.c_uint64, C.c_uint32, C.c_int64, C.c_int32
+        L.hbf_create.argtypes = [C.POINTER(hbf_config_t), vp, C.POINTER(vp)]
+        L.hbf_destroy.argtypes = [vp]
+        L.hbf_register_range.argtypes = [vp, u64, u64, u32, u32, u32, u64, C.POINTER(u32)]
+        L.hbf_clear_ranges.argtypes = [vp]
+        L.hbf_workspace_bytes.argtypes = [vp, u64]
+        L.hbf_workspace_bytes.restype = C.c_size_t
+        L.hbf_submit_batch.argtypes = [vp, vp, u64, vp, vp, vp, vp, vp, C.c_size_t]
+        L.hbf_last_result.argtypes = [vp, C.POINTER(hbf_batch_result_t)]
+        L.hbf_thermal_step.argtypes = [vp, i64, vp, u32, vp, vp]
+        L.hbf_force_mode.argtypes = [vp, i32, i64]
+        L.hbf_get_mode.argtypes = [vp, C.POINTER(i32), C.POINTER(i64)]
+        L.hbf_reset.argtypes = [vp]
+        L.hbf_set_path.argtypes = [vp, i32]
+        L.hbf_get_state.argtypes = [vp, vp, C.POINTER(C.c_size_t)]
+        L.hbf_set_state.argtypes = [vp, vp, C.c_size_t]
+        L.hbf_get_busy_until.argtypes = [vp, vp, u64]
+        L.hbf_get_pending_energy.argtypes = [vp, vp, u64]
+        L.hbf_get_temps.argtypes = [vp, vp, u64]
+        L.hbf_euler_limit_ns.argtypes = [vp]
+        L.hbf_euler_limit_ns.restype = C.c_double
+        L.hbf_queue_order.argtypes = [vp, vp, u64, vp, C.POINTER(u64)]
+        L.hbf_strerror.argtypes = [C.c_int]
+        L.hbf_strerror.restype = C.c_char_p
+        _lib = L
+    return _lib
+
+
+class HbfError(RuntimeError):
+    def __init__(self, code, what=""):
+        super().__init__("%s: %s (%d)" % (what or "hbf", lib().hbf_strerror(code).decode(), code))
+        self.code = code
+
+
+_SCALARS = ("channels", "dies", "planes", "page_bytes", "stripe_bytes", "queue_level", "capacity_bytes",
+            "t_read_ns", "t_prog_ns", "chan_bytes_per_us", "read_granule", "prog_granule",
+            "e_cmd_read_pj", "e_byte_read_pj", "e_cmd_prog_pj", "e_byte_prog_pj",
+            "grid_h", "grid_w", "n_sub", "n_regions", "ambient_c", "rtt_c", "ltt_c", "stt_c", "shutdown_c",
+            "q_light_ppm")
+_ARRAYS = (("cell_C", np.float32), ("cell_Gx", np.float32), ("cell_Gy", np.float32), ("cell_Gsink", np.float32),
+           ("cell_region", np.int32), ("die_region", np.int32), ("region_kind", np.int32),
+           ("region_idle_w", np.float32))
+
+
+def make_config(profile: dict, floorplan: dict | None = None):
+    """Fills an ``hbf_config_t`` from a profile dict (scalars) and a floorplan dict (host arrays).
+    Returns (config, keepalive list)."""
+    cfg = hbf_config_t()
+    for k in _SCALARS:
+        if k in profile:
+            setattr(cfg, k, profile[k])
+    keep = []
+    if floorplan is not None:
+        for k, dt in _ARRAYS:
+            arr = np.ascontiguousarray(floorplan[k], dtype=dt)
+            keep.append(arr)
+            setattr(cfg, k, arr.ctypes.data)
+        cfg.grid_h, cfg.grid_w = floorplan["grid_h"], floorplan["grid_w"]
+        cfg.n_regions = len(floorplan["region_kind"])
+    return cfg, keep
+
+
+def _ptr(t):
+    return None if t is None else t.data_ptr()
+
+
+class Context:
+    """One ``hbf_ctx``.  Methods carry the C function's name without the ``hbf_`` prefix and take torch
+    CUDA tensors where the C function takes device pointers."""
+
+    def __init__(self, profile: dict, floorplan: dict | None = None, stream=None):
+        import torch
+        if not torch.cuda.is_available():
+            raise RuntimeError("hbf needs a CUDA device; there is no CPU fallback")
+        self._torch = torch
+        cfg, keep = make_config(profile, floorplan)
+        self.n_dies = cfg.channels * cfg.dies
+        self.n_queues = self.n_dies * (cfg.planes if cfg.queue_level == 0 else 1)
+        self.n_cells = cfg.grid_h * cfg.grid_w if floorplan is not None else 0
+        self.stream = stream if stream is not None else torch.cuda.current_stream()
+        h = C.c_void_p()
+        rc = lib().hbf_create(C.byref(cfg), C.c_void_p(self.stream.cuda_stream), C.byref(h))
+        if rc != 0:
+            raise HbfError(rc, "hbf_create")
+        self._h = h
+        self._ws = None
+
+    def destroy(self):
+        if getattr(self, "_h", None):
+            lib().hbf_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+    # ---- ranges -------------------------------------------------------------------------------
+    def register_range(self, base, length, perms=3, kind=0, stream_tag=0, media_offset=0, check=True):
+        rid = C.c_uint32()
+        rc = lib().hbf_register_range(self._h, base, length, perms, kind, stream_tag, media_offset, C.byref(rid))
+        if rc != 0:
+            if check:
+                raise HbfError(rc, "hbf_register_range")
+            return rc
+        return rid.value
+
+    def clear_ranges(self):
+        return lib().hbf_clear_ranges(self._h)
+
+    # ---- batches ------------------------------------------------------------------------------
+    def workspace_bytes(self, n: int) -> int:
+        return lib().hbf_workspace_bytes(self._h, n)
+
+    def workspace(self, n: int):
+        """A cached device scratch tensor large enough for a batch of n."""
+        need = self.workspace_bytes(n)
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = self._torch.empty(need, dtype=self._torch.uint8, device="cuda")
+        return self._ws
+
+    def submit_batch(self, d_acc, n, d_completion, d_stall, d_status=None, d_die_stats=None, d_workspace=None):
+        ws = d_workspace if d_workspace is not None else self.workspace(n)
+        return lib().hbf_submit_batch(self._h, _ptr(d_acc), n, _ptr(d_completion), _ptr(d_stall), _ptr(d_status),
+                                      _ptr(d_die_stats), _ptr(ws), ws.numel() * ws.element_size())
+
+    def last_result(self) -> dict:
+        r = hbf_batch_result_t()
+        lib().hbf_last_result(self._h, C.byref(r))
+        return r.as_dict()
+
+    def queue_order(self, n, d_workspace=None):
+        ws = d_workspace if d_workspace is not None else self.workspace(n)
+        out = self._torch.empty(max(n, 1), dtype=self._torch.int32, device="cuda")
+        cnt = C.c_uint64()
+        rc = lib().hbf_queue_order(self._h, _ptr(ws), n, _ptr(out), C.byref(cnt))
+        if rc != 0:
+            raise HbfError(rc, "hbf_queue_order")
+        return out[:cnt.value].cpu().numpy().view(np.uint32)
+
+    def set_path(self, path: int):
+        rc = lib().hbf_set_path(self._h, path)
+        if rc != 0:
+            raise HbfError(rc, "hbf_set_path")
+
+    # ---- thermal ------------------------------------------------------------------------------
+    def thermal_step(self, dt_ns, ext_power_w=None, d_temps_out=None, want_hot=True):
+        hot = np.empty(3, np.float32) if want_hot else None
+        if ext_power_w is None:
+            p, n = None, 0
+        else:
+            ext = np.ascontiguousarray(ext_power_w, np.float32)
+            p, n = ext.ctypes.data, ext.shape[0]
+        rc = lib().hbf_thermal_step(self._h, dt_ns, p, n, _ptr(d_temps_out), hot.ctypes.data if want_hot else None)
+        if rc != 0:
+            raise HbfError(rc, "hbf_thermal_step")
+        return hot
+
+    def force_mode(self, mode, q_ppm):
+        rc = lib().hbf_force_mode(self._h, mode, q_ppm)
+        if rc != 0:
+            raise HbfError(rc, "hbf_force_mode")
+
+    def get_mode(self):
+        m, q = C.c_int32(), C.c_int64()
+        lib().hbf_get_mode(self._h, C.byref(m), C.byref(q))
+        return m.value, q.value
+
+    def reset(self):
+        rc = lib().hbf_reset(self._h)
+        if rc != 0:
+            raise HbfError(rc, "hbf_reset")
+
+    # ---- state --------------------------------------------------------------------------------
+    def get_busy_until(self):
+        out = np.empty(self.n_queues, np.int64)
+        rc = lib().hbf_get_busy_until(self._h, out.ctypes.data, out.shape[0])
+        if rc != 0:
+            raise HbfError(rc, "hbf_get_busy_until")
+        return out
+
+    def get_pending_energy(self):
+        out = np.empty(self.n_dies, np.int64)
+        rc = lib().hbf_get_pending_energy(self._h, out.ctypes.data, out.shape[0])
+        if rc != 0:
+            raise HbfError(rc, "hbf_get_pending_energy")
+        return out
+
+    def get_temps(self):
+        out = np.empty(self.n_cells, np.float32)
+        rc = lib().hbf_get_temps(self._h, out.ctypes.data, out.shape[0])
+        if rc != 0:
+            raise HbfError(rc, "hbf_get_temps")
+        return out
+
+    def euler_limit_ns(self):
+        return lib().hbf_euler_limit_ns(self._h)
+
+    def get_state(self) -> bytes:
+        sz = C.c_size_t()
+        lib().hbf_get_state(self._h, None, C.byref(sz))
+        buf = C.create_string_buffer(sz.value)
+        rc = lib().hbf_get_state(self._h, buf, C.byref(sz))
+        if rc != 0:
+            raise HbfError(rc, "hbf_get_state")
+        return buf.raw[:sz.value]
+
+    def set_state(self, blob: bytes):
+        rc = lib().hbf_set_state(self._h, blob, len(blob))
+        if rc != 0:
+            raise HbfError(rc, "hbf_set_state")
+
+    # ---- host-buffer convenience: copies in, one submit, copies out ---------------------------------
+    def submit_host(self, acc: np.ndarray, want_status=True, check=True):
+        """Marshals a host batch through the device: H2D of the records, ``hbf_submit_batch``, D2H of
+        completions, stalls, status and per-die stats.  Returns (code, completion, stall, status, die_stats)."""
+        torch = self._torch
+        acc = np.ascontiguousarray(acc, dtype=ACCESS_DTYPE)
+        n = acc.shape[0]
+        with torch.cuda.stream(self.stream):
+            d_acc = torch.from_numpy(acc.view(np.int64).reshape(-1)).cuda() if n else torch.empty(0, dtype=torch.int64, device="cuda")
+            d_comp = torch.empty(n, dtype=torch.int64, device="cuda")
+            d_stall = torch.empty(n, dtype=torch.int64, device="cuda")
+            d_status = torch.empty(n, dtype=torch.uint8, device="cuda") if want_status else None
+            d_ds = torch.empty(self.n_dies * 6, dtype=torch.int64, device="cuda")
+            rc = self.submit_batch(d_acc, n, d_comp, d_stall, d_status, d_ds)
+            if rc != 0:
+                raise HbfError(rc, "hbf_submit_batch")
+            res = self.last_result()
+            if check and res["code"] != 0:
+                raise HbfError(res["code"], "batch")
+            comp, stall = d_comp.cpu().numpy(), d_stall.cpu().numpy()
+            status = d_status.cpu().numpy() if want_status else None
+            ds = d_ds.cpu().numpy().view(DIE_STATS_DTYPE)
+        return res["code"], comp, stall, status, ds

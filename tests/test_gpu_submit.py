@@ -1,0 +1,205 @@
+"""Parity of the CUDA submit path with the CPU oracle, through the C ABI, element by element.
+
+Integer outputs (completions, stalls, status, per-die stats, queue state, batch summary, served
+order) must be bit-exact."""
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+from oracle import hbfo
+from paper_2609_09800_b200 import workloads as wl
+
+
+@pytest.fixture(scope="module")
+def hbf():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2609_09800_b200 import build, hbf as mod
+    build.build()
+    return mod
+
+
+def contexts(hbf, profile, ranges, path=None):
+    g = hbf.Context(profile)
+    o = hbfo.Oracle(profile)
+    for r in ranges:
+        g.register_range(*r)
+        o.register_range(*r)
+    if path is not None:
+        g.set_path(path)
+    return g, o
+
+
+def compare_batch(g, o, acc, check_order=False):
+    rc_o, c_o, s_o, st_o, ds_o = o.submit(acc, check=False)
+    rc_g, c_g, s_g, st_g, ds_g = g.submit_host(acc, check=False)
+    assert rc_g == rc_o
+    assert np.array_equal(st_g, st_o)
+    bad = np.flatnonzero(c_g != c_o)
+    assert bad.size == 0, "first mismatch at %d: gpu %d oracle %d (%d mismatches)" % (
+        bad[0], c_g[bad[0]], c_o[bad[0]], bad.size)
+    assert np.array_equal(s_g, s_o)
+    for k in hbfo.DIE_STATS_DTYPE.names:
+        assert np.array_equal(ds_g[k], ds_o[k]), k
+    assert np.array_equal(g.get_busy_until(), o.busy_until())
+    assert np.array_equal(g.get_pending_energy(), o.pending_energy())
+    rg, ro = g.last_result(), o.last_result()
+    assert rg == ro, (rg, ro)
+    if check_order and rc_o == 0:
+        assert np.array_equal(g.queue_order(acc.shape[0]), o.last_order())
+    return rc_g
+
+
+PATHS = ["auto", "sort", "sort_full"]
+
+
+def path_id(hbf, name):
+    return {"auto": hbf.PATH_AUTO, "sort": hbf.PATH_SORT, "sort_full": hbf.PATH_SORT_FULL}[name]
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_tiny_uniform_reads(hbf, path):
+    w = wl.tiny_uniform()
+    g, o = contexts(hbf, w.profile, w.ranges, path_id(hbf, path))
+    compare_batch(g, o, w.acc, check_order=path != "auto")
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_mixed_status_shuffled(hbf, path):
+    w = wl.mixed_status(10_000, seed=0)
+    g, o = contexts(hbf, w.profile, w.ranges, path_id(hbf, path))
+    compare_batch(g, o, w.acc[:6000], check_order=path != "auto")
+    compare_batch(g, o, w.acc[6000:], check_order=path != "auto")          # queue state carries over
+
+
+def test_faulting_batch_is_refused(hbf):
+    w = wl.mixed_status(10_000, seed=0)
+    wf = wl.mixed_status(10_000, seed=0, faults=True)
+    g, o = contexts(hbf, w.profile, w.ranges)
+    compare_batch(g, o, w.acc[:3000])
+    assert compare_batch(g, o, wf.acc) == hbfo.E_ACCESS_FAULT
+    compare_batch(g, o, w.acc[3000:])                    # the context stays usable, state untouched by the refusal
+
+
+@pytest.mark.parametrize("n", [0, 1, 2, 31, 32, 33, 1023, 1024, 1025, 2047, 2048, 2049, 4095, 4096, 4097, 12289])
+def test_ragged_sizes(hbf, n):
+    w = wl.mixed_status(max(n, 1), seed=n)
+    for path in (hbf.PATH_AUTO, hbf.PATH_SORT_FULL):
+        g, o = contexts(hbf, w.profile, w.ranges, path)
+        compare_batch(g, o, w.acc[:n], check_order=(path != hbf.PATH_AUTO and n > 0))
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_decode_weight_streaming(hbf, path):
+    w = wl.decode_weights(tokens=4)
+    g, o = contexts(hbf, w.profile, w.ranges, path_id(hbf, path))
+    compare_batch(g, o, w.acc)
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_prefix_kv_programs_and_reads(hbf, path):
+    w = wl.prefix_kv(epochs=2, steps=1, batch=16, kv_tokens=2048, layers=6)
+    assert 0.005 < w.meta["frac_program"] < 0.2
+    g, o = contexts(hbf, w.profile, w.ranges, path_id(hbf, path))
+    cut = w.n // 3
+    compare_batch(g, o, w.acc[:cut])
+    compare_batch(g, o, w.acc[cut:])
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_capacity_mode_sizes(hbf, path):
+    w = wl.capacity_mode(n=700_001)
+    g, o = contexts(hbf, w.profile, w.ranges, path_id(hbf, path))
+    compare_batch(g, o, w.acc)
+
+
+def test_light_mode_scales_service(hbf):
+    w = wl.prefix_kv(epochs=1, steps=1, batch=4, kv_tokens=1024, layers=3)
+    g, o = contexts(hbf, w.profile, w.ranges)
+    for q in (800_000, 999_999, 123_457, 1):
+        g.force_mode(hbf.MODE_LIGHT, q); o.force_mode(hbfo.MODE_LIGHT, q)
+        compare_batch(g, o, w.acc[:20_000])
+
+
+def test_severe_and_shutdown_refuse(hbf):
+    w = wl.tiny_uniform(3000)
+    g, o = contexts(hbf, w.profile, w.ranges)
+    compare_batch(g, o, w.acc[:1000])
+    g.force_mode(hbf.MODE_SEVERE, 1_000_000); o.force_mode(hbfo.MODE_SEVERE, 1_000_000)
+    rc_g = g.submit_host(w.acc[1000:2000], check=False)[0]
+    rc_o = o.submit(w.acc[1000:2000], check=False)[0]
+    assert rc_g == rc_o == hbfo.E_THROTTLED
+    assert np.array_equal(g.get_busy_until(), o.busy_until())
+    g.force_mode(hbf.MODE_NORMAL, 1_000_000); o.force_mode(hbfo.MODE_NORMAL, 1_000_000)
+    compare_batch(g, o, w.acc[1000:2000])
+    g.force_mode(hbf.MODE_SHUTDOWN, 1_000_000); o.force_mode(hbfo.MODE_SHUTDOWN, 1_000_000)
+    assert g.submit_host(w.acc[2000:], check=False)[0] == o.submit(w.acc[2000:], check=False)[0] == hbfo.E_LINK_SHUTDOWN
+    # terminal: the host side now refuses without launching
+    assert g.submit_batch(None, 0, None, None) == hbf.E_LINK_SHUTDOWN
+
+
+@pytest.mark.parametrize("geo", [dict(channels=3, dies=5, planes=2, page_bytes=4096, stripe_bytes=16384),
+                                 dict(channels=8, dies=4, planes=2, page_bytes=16384, stripe_bytes=16384, queue_level=1),
+                                 dict(channels=256, dies=16, planes=16, page_bytes=16384, stripe_bytes=16384),
+                                 dict(channels=1, dies=1, planes=1, page_bytes=16384, stripe_bytes=16384)])
+def test_other_geometries(hbf, geo):
+    w = wl.mixed_status(30_000, seed=5)
+    prof = dict(w.profile); prof.update(geo)
+    for path in (hbf.PATH_AUTO, hbf.PATH_SORT_FULL):
+        g, o = contexts(hbf, prof, w.ranges, path)
+        compare_batch(g, o, w.acc, check_order=path != hbf.PATH_AUTO)
+
+
+def test_equal_issue_times_and_hot_queue(hbf):
+    # every access on one plane with many equal issue times: index order must decide
+    rng = np.random.default_rng(3)
+    n = 50_000
+    acc = np.zeros(n, hbfo.ACCESS_DTYPE)
+    acc["addr"] = wl.RANGE_BASE + rng.integers(0, 4, n).astype(np.uint64) * np.uint64(4096)
+    acc["issue_ns"] = rng.integers(0, 50, n)
+    acc["bytes"] = rng.choice([64, 4096, 16384], n)
+    acc["flags"] = rng.random(n) < 0.3
+    prof = wl.load_profile("nominal", **wl.GEOMETRY["tiny"])
+    for path in (hbf.PATH_AUTO, hbf.PATH_SORT_FULL):
+        g, o = contexts(hbf, prof, [(wl.RANGE_BASE, wl.GIB, 3, 0, 0, 0)], path)
+        compare_batch(g, o, acc, check_order=path != hbf.PATH_AUTO)
+        compare_batch(g, o, np.sort(acc, order="issue_ns", kind="stable"))
+
+
+def test_large_issue_times_near_the_limit(hbf):
+    w = wl.mixed_status(5000, seed=9)
+    acc = w.acc.copy()
+    acc["issue_ns"] += (1 << 47) - 1 - int(acc["issue_ns"].max())
+    g, o = contexts(hbf, w.profile, w.ranges)
+    compare_batch(g, o, acc)
+    acc["issue_ns"][17] = 1 << 47                           # one past the limit: unsupported, batch refused
+    assert compare_batch(g, o, acc) == hbfo.E_ACCESS_FAULT
+
+
+def test_argument_errors(hbf):
+    import torch
+    w = wl.tiny_uniform(100)
+    g, _ = contexts(hbf, w.profile, w.ranges)
+    d = torch.zeros(300, dtype=torch.int64, device="cuda")
+    out = torch.zeros(100, dtype=torch.int64, device="cuda")
+    small = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    assert g.submit_batch(d, 100, out, out, d_workspace=small) == hbf.E_WORKSPACE
+    assert g.submit_batch(None, 100, out, out) == hbf.E_INVAL
+    assert g.submit_batch(d, 1 << 30, out, out) == hbf.E_INVAL
+    assert g.register_range(wl.RANGE_BASE + 5, 10, check=False) == hbf.E_RANGE_OVERLAP
+    assert g.workspace_bytes(1000) >= 1000 * 24
+
+
+def test_state_blob_round_trip(hbf):
+    w = wl.mixed_status(8000, seed=4)
+    g, o = contexts(hbf, w.profile, w.ranges)
+    compare_batch(g, o, w.acc[:4000])
+    blob = g.get_state()
+    g2, _ = contexts(hbf, w.profile, w.ranges)
+    g2.set_state(blob)
+    assert np.array_equal(g2.get_busy_until(), o.busy_until())
+    compare_batch(g2, o, w.acc[4000:])
+    with pytest.raises(hbf.HbfError):
+        g2.set_state(blob[:-8])
