@@ -1,0 +1,306 @@
+#!/usr/bin/env python
+"""Benchmark of the HBF service-model hot path on B200.
+
+One step = one pass of the whole hot path over one batch: ``hbf_submit_batch`` (classify, decode,
+queue order, max-plus scan, scatter, per-die stats) followed by ``hbf_thermal_step`` (power map, RC
+stencil, throttle controller).  The workload is the capacity-mode stream (200 M accesses in one batch,
+64 channels x 8 dies x 4 planes); with N > 1 every rank runs an independent replica on its own stream
+(replicas only: the path needs no exchange at one GPU per model instance).
+
+Prints ONE JSON line.  ``--impl reference`` times the CPU oracle instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2609_09800_b200 import workloads as wl  # noqa: E402
+
+METRIC = "simulated HBF accesses/s"
+UNIT = "accesses/s"
+ALGO_BYTES_PER_ACCESS = 41            # 24 B record in, 8 B completion + 8 B stall + 1 B status out
+# algorithmic bytes per access of each kernel group (what the kernel itself must move)
+STAGE_BYTES = {"classify": 24 + 8 + 1, "plan_hist": 8, "scan": 8 + 4 + 24 + 16, "inorder": 24 + 16 + 1}
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--n", type=int, default=200_000_000, help="accesses per batch (default: the capacity-mode config)")
+    ap.add_argument("--path", default="auto", choices=["auto", "sort", "sort_full"])
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--cpu-sample", type=int, default=20_000_000)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            with open(p) as f:
+                return float(json.load(f)["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons, sampled every 200 ms while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu, self.proc = gpu_index, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill(); out = ""
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def make_stream(n: int, seed: int):
+    t = time.time()
+    w = wl.capacity_mode(n=n, seed=seed)
+    return w, time.time() - t
+
+
+def cpu_oracle_rate(w, sample: int, repeats: int = 1):
+    """The oracle as it stands, on one host core, on the first ``sample`` accesses of the stream."""
+    from oracle import hbfo
+    acc = w.acc[:sample]
+    o = hbfo.Oracle(w.profile, wl.package_floorplan(channels=w.profile["channels"], dies=w.profile["dies"]))
+    for r in w.ranges:
+        o.register_range(*r)
+    times = []
+    for _ in range(repeats):
+        o.reset()
+        t = time.perf_counter()
+        o.submit(acc)
+        o.thermal_step(1_000_000, None)
+        times.append(time.perf_counter() - t)
+    return acc.shape[0] / min(times), times
+
+
+def run_reference(args, rank: int):
+    """The CPU oracle on this machine's host cores: each step is a bounded sample of the workload."""
+    if rank != 0:
+        return
+    sample = min(args.n, 4_000_000)
+    w, _ = make_stream(sample, 0)
+    from oracle import hbfo
+    fp = wl.package_floorplan(channels=w.profile["channels"], dies=w.profile["dies"])
+    o = hbfo.Oracle(w.profile, fp)
+    for r in w.ranges:
+        o.register_range(*r)
+    for _ in range(args.warmup):
+        o.submit(w.acc); o.thermal_step(1_000_000, fp["ext_power_w"])
+    t = time.perf_counter()
+    for _ in range(args.steps):
+        o.submit(w.acc); o.thermal_step(1_000_000, fp["ext_power_w"])
+    dt = time.perf_counter() - t
+    value = args.steps * sample / dt
+    sample_txt = "first %d accesses of the capacity-mode stream per step, 1 thermal step per batch" % sample
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+            "config": {"workload": "capacity_mode", "accesses_per_step": sample, "geometry": "64x8x4"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample_txt},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    args = parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2609_09800_b200 import build as hbf_build, hbf
+
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (no CPU fallback)"
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if local_rank == 0:
+        hbf_build.build()
+    if world > 1:
+        dist.barrier()
+
+    n = args.n
+    w, gen_s = make_stream(n, seed=rank)               # every rank: an independent replica on its own stream
+    fp = wl.package_floorplan(channels=w.profile["channels"], dies=w.profile["dies"])
+    ctx = hbf.Context(w.profile, fp)
+    for r in w.ranges:
+        ctx.register_range(*r)
+    ctx.set_path({"auto": hbf.PATH_AUTO, "sort": hbf.PATH_SORT, "sort_full": hbf.PATH_SORT_FULL}[args.path])
+
+    # inputs resident in HBM before the timed region
+    h_acc = torch.from_numpy(w.acc.view(np.int64).reshape(-1))
+    d_acc = h_acc.cuda()
+    d_comp = torch.empty(n, dtype=torch.int64, device="cuda")
+    d_stall = torch.empty(n, dtype=torch.int64, device="cuda")
+    d_status = torch.empty(n, dtype=torch.uint8, device="cuda")
+    d_stats = torch.empty(ctx.n_dies * 6, dtype=torch.int64, device="cuda")
+    ws = ctx.workspace(n)
+    ext = fp["ext_power_w"]
+    stream = torch.cuda.current_stream()
+
+    def step():
+        rc = ctx.submit_batch(d_acc, n, d_comp, d_stall, d_status, d_stats, ws)
+        assert rc == 0, rc
+        ctx.thermal_step(1_000_000, ext, None, want_hot=False)
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    ctx.set_profiling(True)
+    for _ in range(args.warmup):
+        step()
+    sync_all()
+    res = ctx.last_result()
+    assert res["code"] == 0, res
+    launches0 = hbf.kernel_launches()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    stage_ms = {k: [] for k in hbf.PROF_STAGES}
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sync_all()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    sync_all()
+    total_ms = e0.elapsed_time(e1)
+    clocks = sampler.stop()
+    launches = hbf.kernel_launches() - launches0
+    # per-stage device times of a few more steps (events recorded between kernel groups on the same stream)
+    for _ in range(min(3, args.steps)):
+        step()
+        prof = ctx.get_profile()
+        for k, v in prof.items():
+            stage_ms[k].append(v)
+    if world > 1:
+        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    value = world * n * args.steps / (total_ms * 1e-3)
+
+    # end to end through the C ABI with host buffers: H2D of the records, submit + thermal step, D2H of results
+    e2e = None
+    if not args.no_e2e:
+        h_in = h_acc.pin_memory()
+        h_comp = torch.empty(n, dtype=torch.int64).pin_memory()
+        h_stall = torch.empty(n, dtype=torch.int64).pin_memory()
+        h_stats = torch.empty(ctx.n_dies * 6, dtype=torch.int64).pin_memory()
+
+        def e2e_step():
+            d_acc.copy_(h_in, non_blocking=True)
+            step()
+            h_comp.copy_(d_comp, non_blocking=True); h_stall.copy_(d_stall, non_blocking=True)
+            h_stats.copy_(d_stats, non_blocking=True)
+        e2e_step(); sync_all()
+        e0.record(stream)
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        e1.record(stream)
+        sync_all()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        e2e = {"value": world * n * args.e2e_steps / (ms * 1e-3), "unit": UNIT, "steps": args.e2e_steps,
+               "h2d_bytes_per_step": n * 24, "d2h_bytes_per_step": n * 16 + ctx.n_dies * 48}
+
+    if rank == 0:
+        peak, peak_kind = measured_peak()
+        med = {k: (statistics.median(v) if v else 0.0) for k, v in stage_ms.items()}
+        timed = {k: v for k, v in med.items() if k in STAGE_BYTES or k == "sort"}
+        dom = max(timed, key=lambda k: timed[k])
+        if dom == "sort":
+            n_pass = 2 if args.path != "sort_full" else 6
+            dom_bytes = (8 + 12) + (n_pass - 1) * 24            # first pass reads keys only
+            per_launch_ms = med["sort"]
+        else:
+            dom_bytes = STAGE_BYTES[dom]; per_launch_ms = med[dom]
+        achieved = dom_bytes * n / (per_launch_ms * 1e-3) / 1e9 if per_launch_ms > 0 else 0.0
+        roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+                    "frac": achieved / peak, "traffic": None, "algorithmic_bytes_per_access": dom_bytes,
+                    "ms_per_launch": per_launch_ms}
+        path_gbs = ALGO_BYTES_PER_ACCESS * value / world / 1e9
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+                "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "int64", "data": "synthetic",
+                "config": {"workload": "capacity_mode", "accesses_per_step": n, "geometry": "64x8x4", "queues": 2048,
+                           "path": args.path, "thermal_grid": "128x128", "l2": "inputs (%.1f GB) larger than L2" % (n * 24 / 1e9),
+                           "multi_gpu": "replicas only", "gen_seconds": round(gen_s, 1)},
+                "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
+                "path_algorithmic": {"bytes_per_access": ALGO_BYTES_PER_ACCESS, "achieved": path_gbs, "unit": "GB/s",
+                                     "frac": path_gbs / peak, "frac_of_8tbs_nominal": path_gbs / 8000.0},
+                "stage_ms": {k: round(v, 4) for k, v in med.items()},
+                "batch_result": {k: res[k] for k in ("n_modeled", "n_native", "max_completion_ns")}}
+        if world == 1 and not args.no_cpu_baseline:
+            sample = min(n, args.cpu_sample)
+            rate, times = cpu_oracle_rate(w, sample)
+            line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": 1, "kind": "oracle",
+                                    "sample": "first %d accesses of the same stream, one pass (%.1f s)" % (sample, min(times))}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

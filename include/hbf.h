@@ -166,6 +166,17 @@ HBF_API double hbf_euler_limit_ns(const hbf_ctx *ctx);
  * receives the number of modeled accesses. */
 HBF_API int hbf_queue_order(hbf_ctx *ctx, const void *d_workspace, uint64_t n, uint32_t *d_order, uint64_t *count);
 
+/* Stage timing.  With profiling on, every submit and thermal step records CUDA events between its
+ * kernel groups on the context's stream (no synchronisation).  hbf_get_profile waits for the stream
+ * and writes the milliseconds of the last batch's stages to ms_out (host, [HBF_PROF_STAGES]):
+ * begin, classify, plan+histogram, sort passes, scan+scatter, finish, in-order path, thermal step.
+ * A stage that did not run reads 0. */
+#define HBF_PROF_STAGES 8
+HBF_API int hbf_set_profiling(hbf_ctx *ctx, int on);
+HBF_API int hbf_get_profile(hbf_ctx *ctx, float *ms_out, uint32_t cap);
+/* Number of kernels this library has launched in the calling process so far. */
+HBF_API uint64_t hbf_kernel_launches(void);
+
 HBF_API const char *hbf_strerror(int code);
 
 #ifdef __cplusplus

@@ -39,6 +39,8 @@ struct hbf_ctx {
     float *h_hot = nullptr;                      // pinned [3]
     float *h_ext = nullptr;                      // pinned [n_regions]
     bool submitted = false;
+    bool profiling = false; cudaEvent_t ev[kProfEvents] = {}; cudaEvent_t ev_th[2] = {}; bool ev_made = false;
+    bool prof_submit = false, prof_thermal = false;
     // thermal
     bool thermal = false; ThermalDev td{}; int cur = 0; double euler_limit_s = 0.0;
     std::vector<void *> owned;
@@ -99,6 +101,7 @@ int hbf_destroy(hbf_ctx *c) {
     if (!c) return HBF_E_INVAL;
     cudaStreamSynchronize(c->stream);
     for (void *p : c->owned) cudaFree(p);
+    if (c->ev_made) { for (auto &e : c->ev) cudaEventDestroy(e); for (auto &e : c->ev_th) cudaEventDestroy(e); }
     if (c->h_result) cudaFreeHost(c->h_result);
     if (c->h_hot) cudaFreeHost(c->h_hot);
     if (c->h_ext) cudaFreeHost(c->h_ext);
@@ -272,6 +275,8 @@ int hbf_submit_batch(hbf_ctx *c, const hbf_access_t *d_acc, uint64_t n, int64_t 
     a.ranges = c->d_ranges; a.mp_dev = c->d_mp; a.mp = c->mp; a.state = c->d_state; a.ctrl = c->d_ctrl; a.result = c->d_result;
     a.busy = c->d_busy; a.busy_stage = c->d_busy_stage; a.pending = c->d_pending; a.stats_stage = c->d_stats_stage;
     a.path = c->path; a.sm_count = c->sm_count;
+    a.ev = c->profiling ? c->ev : nullptr;
+    c->prof_submit = c->profiling;
     CK(launch_submit(a, c->stream));
     c->submitted = true;
     return HBF_OK;
@@ -305,12 +310,11 @@ int hbf_thermal_step(hbf_ctx *c, int64_t dt_ns, const float *ext_power_w, uint32
     if (n_ext != 0 && (n_ext != c->td.n_regions || !ext_power_w)) return HBF_E_INVAL;
     const double dt_sub = (double)dt_ns * 1e-9 / (double)c->td.n_sub;
     if (dt_sub > c->euler_limit_s) return HBF_E_INVAL;
-    if (n_ext) {
-        CK(cudaStreamSynchronize(c->stream));          // the pinned staging buffer may still feed an earlier step
-        memcpy(c->h_ext, ext_power_w, n_ext * sizeof(float));
-        CK(cudaMemcpyAsync(c->td.ext_power, c->h_ext, n_ext * sizeof(float), cudaMemcpyHostToDevice, c->stream));
-    }
+    if (n_ext)      // pageable source: the runtime stages the bytes before returning, so the caller's array is free at once
+        CK(cudaMemcpyAsync(c->td.ext_power, ext_power_w, n_ext * sizeof(float), cudaMemcpyHostToDevice, c->stream));
+    if (c->profiling) CK(cudaEventRecord(c->ev_th[0], c->stream));
     CK(launch_thermal_step(c->td, c->d_state, c->d_pending, dt_ns, n_ext != 0, d_temps_out, &c->cur, c->stream));
+    if (c->profiling) { CK(cudaEventRecord(c->ev_th[1], c->stream)); c->prof_thermal = true; }
     if (hot_c_out) {
         CK(cudaMemcpyAsync(c->h_hot, c->td.hot, 3 * sizeof(float), cudaMemcpyDeviceToHost, c->stream));
         CK(cudaStreamSynchronize(c->stream));
@@ -384,6 +388,30 @@ int hbf_get_temps(hbf_ctx *c, float *host_out, uint64_t cap) {
     for (size_t i = 0; i < nc; ++i) host_out[i] += c->td.ambient_c;
     return HBF_OK;
 }
+
+int hbf_set_profiling(hbf_ctx *c, int on) {
+    if (!c) return HBF_E_INVAL;
+    if (on && !c->ev_made) {
+        for (auto &e : c->ev) CK(cudaEventCreate(&e));
+        for (auto &e : c->ev_th) CK(cudaEventCreate(&e));
+        c->ev_made = true;
+    }
+    c->profiling = on != 0;
+    if (!on) c->prof_submit = c->prof_thermal = false;
+    return HBF_OK;
+}
+
+int hbf_get_profile(hbf_ctx *c, float *ms_out, uint32_t cap) {
+    if (!c || !ms_out || cap < HBF_PROF_STAGES) return HBF_E_INVAL;
+    for (int k = 0; k < HBF_PROF_STAGES; ++k) ms_out[k] = 0.0f;
+    CK(cudaStreamSynchronize(c->stream));
+    if (c->prof_submit)
+        for (int k = 0; k < 6; ++k) CK(cudaEventElapsedTime(&ms_out[k], c->ev[k], c->ev[k + 1]));
+    if (c->prof_thermal) CK(cudaEventElapsedTime(&ms_out[7], c->ev_th[0], c->ev_th[1]));
+    return HBF_OK;
+}
+
+uint64_t hbf_kernel_launches(void) { return g_kernel_launches; }
 
 double hbf_euler_limit_ns(const hbf_ctx *c) { return c && c->thermal ? c->euler_limit_s * 1e9 : 0.0; }
 

@@ -86,7 +86,10 @@ struct SubmitArgs {
     DevState *state; BatchCtrl *ctrl; hbf_batch_result_t *result;
     int64_t *busy, *busy_stage, *pending; hbf_die_stats_t *stats_stage;
     Workspace ws; int32_t path; int sm_count;
+    cudaEvent_t *ev;                     // [kProfEvents] or null: recorded between kernel groups
 };
+constexpr int kProfEvents = 8;
+extern unsigned long long g_kernel_launches;
 
 size_t workspace_layout(uint64_t n, uint32_t n_queues, Workspace *ws, void *base);
 cudaError_t launch_submit(const SubmitArgs &a, cudaStream_t st);

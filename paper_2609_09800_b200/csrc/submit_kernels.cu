@@ -640,22 +640,30 @@ size_t workspace_layout(uint64_t n, uint32_t n_queues, Workspace *ws, void *base
     return off;
 }
 
+unsigned long long g_kernel_launches = 0;
+
 cudaError_t launch_submit(const SubmitArgs &a, cudaStream_t st) {
     const uint64_t n = a.n;
+    auto mark = [&](int k) { if (a.ev) cudaEventRecord(a.ev[k], st); };
+    mark(0);
     k_begin<<<1, 256, 0, st>>>(a.ctrl, a.state, a.busy, a.busy_stage, a.stats_stage, a.ws.hist, a.mp.n_queues, a.mp.n_dies);
+    g_kernel_launches += 1;
     if (n > 0) {
         const uint64_t sort_tiles = (n + kSortTile - 1) / kSortTile, scan_tiles = (n + kScanTile - 1) / kScanTile;
         cudaError_t e = cudaMemsetAsync(a.ws.sort_desc[0], 0, sort_tiles * kRadix * 4, st);
         if (e != cudaSuccess) return e;
         e = cudaMemsetAsync(a.ws.scan_desc, 0, scan_tiles * sizeof(ScanDesc), st);
         if (e != cudaSuccess) return e;
+        mark(1);
         const uint64_t cls_tiles = (n + kClsTile - 1) / kClsTile;
         const unsigned cls_grid = (unsigned)std::min<uint64_t>(cls_tiles, (uint64_t)a.sm_count * 8);
         k_classify<<<cls_grid, kClsThreads, 0, st>>>(a.acc, n, a.ranges, a.mp_dev, a.ctrl, a.ws.keys[0], a.status,
                                                      a.completion, a.stall);
+        mark(2);
         k_plan<<<1, 32, 0, st>>>(a.ctrl, a.path == HBF_PATH_SORT_FULL ? 1 : 0);
         const unsigned hist_grid = (unsigned)std::min<uint64_t>((n + kHistThreads * 8 - 1) / (kHistThreads * 8), (uint64_t)a.sm_count * 4);
         k_hist<<<hist_grid, kHistThreads, 0, st>>>(a.ws.keys[0], n, a.ctrl, a.ws.hist);
+        mark(3);
         static bool attr_set = false;
         if (!attr_set) {
             e = cudaFuncSetAttribute(k_sort_pass, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSortSmem);
@@ -664,14 +672,21 @@ cudaError_t launch_submit(const SubmitArgs &a, cudaStream_t st) {
         }
         for (int p = 0; p < kMaxPasses; ++p)
             k_sort_pass<<<(unsigned)sort_tiles, kSortThreads, kSortSmem, st>>>(p, n, a.ctrl, a.state, a.ws.hist, a.ws.keys[0], a.ws.keys[1],
-                                                                       a.ws.idx[0], a.ws.idx[1], a.ws.sort_desc[0], a.ws.sort_desc[1]);
+                                                                               a.ws.idx[0], a.ws.idx[1], a.ws.sort_desc[0], a.ws.sort_desc[1]);
+        mark(4);
         k_scan<<<(unsigned)scan_tiles, kScanThreads, 0, st>>>(a.acc, n, a.ranges, a.mp_dev, a.ctrl, a.state, a.ws.keys[0], a.ws.keys[1],
                                                              a.ws.idx[0], a.ws.idx[1], (ScanDesc *)a.ws.scan_desc, a.busy,
                                                              a.busy_stage, a.stats_stage, a.completion, a.stall);
+        g_kernel_launches += 4 + kMaxPasses;
+    } else {
+        mark(1); mark(2); mark(3); mark(4);
     }
+    mark(5);
     const unsigned fin_grid = (unsigned)std::max<uint64_t>(1, std::min<uint64_t>((n + 1023) / 1024, (uint64_t)a.sm_count * 4));
     k_finish<<<fin_grid, 256, 0, st>>>(n, a.ctrl, a.state, a.busy, a.busy_stage, a.pending, a.stats_stage, a.die_stats,
                                        a.completion, a.stall, a.result, a.mp.n_queues, a.mp.n_dies);
+    g_kernel_launches += 1;
+    mark(6);
     return cudaGetLastError();
 }
 

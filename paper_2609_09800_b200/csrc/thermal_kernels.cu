@@ -111,6 +111,7 @@ cudaError_t launch_thermal_step(const ThermalDev &t, DevState *state, int64_t *p
         c ^= 1;
     }
     *cur = c;
+    g_kernel_launches += 2ull + t.n_sub;
     k_controller<<<1, 1024, 0, st>>>(t, t.theta[c], state, d_temps_out);
     return cudaGetLastError();
 }

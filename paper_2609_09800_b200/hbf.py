@@ -27,7 +27,9 @@ DIE_STATS_DTYPE = np.dtype([(k, "<i8") for k in
 EXPORTS = ("hbf_create", "hbf_destroy", "hbf_register_range", "hbf_clear_ranges", "hbf_workspace_bytes",
            "hbf_submit_batch", "hbf_last_result", "hbf_thermal_step", "hbf_force_mode", "hbf_get_mode",
            "hbf_reset", "hbf_set_path", "hbf_get_state", "hbf_set_state", "hbf_get_busy_until",
-           "hbf_get_pending_energy", "hbf_get_temps", "hbf_euler_limit_ns", "hbf_queue_order", "hbf_strerror")
+           "hbf_get_pending_energy", "hbf_get_temps", "hbf_euler_limit_ns", "hbf_queue_order", "hbf_strerror",
+           "hbf_set_profiling", "hbf_get_profile", "hbf_kernel_launches")
+PROF_STAGES = ("begin", "classify", "plan_hist", "sort", "scan", "finish", "inorder", "thermal")
 
 
 class hbf_config_t(C.Structure):
@@ -95,10 +97,18 @@ def lib():
         L.hbf_euler_limit_ns.argtypes = [vp]
         L.hbf_euler_limit_ns.restype = C.c_double
         L.hbf_queue_order.argtypes = [vp, vp, u64, vp, C.POINTER(u64)]
+        L.hbf_set_profiling.argtypes = [vp, C.c_int]
+        L.hbf_get_profile.argtypes = [vp, vp, u32]
+        L.hbf_kernel_launches.argtypes = []
+        L.hbf_kernel_launches.restype = u64
         L.hbf_strerror.argtypes = [C.c_int]
         L.hbf_strerror.restype = C.c_char_p
         _lib = L
     return _lib
+
+
+def kernel_launches() -> int:
+    return lib().hbf_kernel_launches()
 
 
 class HbfError(RuntimeError):
@@ -271,6 +281,18 @@ class Context:
 
     def euler_limit_ns(self):
         return lib().hbf_euler_limit_ns(self._h)
+
+    def set_profiling(self, on: bool):
+        rc = lib().hbf_set_profiling(self._h, 1 if on else 0)
+        if rc != 0:
+            raise HbfError(rc, "hbf_set_profiling")
+
+    def get_profile(self) -> dict:
+        ms = np.zeros(len(PROF_STAGES), np.float32)
+        rc = lib().hbf_get_profile(self._h, ms.ctypes.data, ms.shape[0])
+        if rc != 0:
+            raise HbfError(rc, "hbf_get_profile")
+        return dict(zip(PROF_STAGES, ms.tolist()))
 
     def get_state(self) -> bytes:
         sz = C.c_size_t()

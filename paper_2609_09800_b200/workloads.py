@@ -181,26 +181,48 @@ CAPACITY_REPLICAS, CAPACITY_SLOT = 16, 96 * GIB
 CAPACITY_RANGE = CAPACITY_REPLICAS * CAPACITY_SLOT                       # 1.5 TiB
 
 
+def _capacity_chunk(seed: int, k: int, m: int, mean_gap: float):
+    """Chunk k of the capacity stream: records with issue times relative to the chunk's start."""
+    rng = np.random.Generator(np.random.PCG64([seed, 4, k]))
+    replica = rng.integers(0, CAPACITY_REPLICAS, m, dtype=np.uint64)
+    lg = rng.integers(7, 17, m, dtype=np.uint64)                     # 128 B ... 64 KiB
+    slots = np.uint64(WEIGHT_BYTES) >> lg
+    slot = (rng.random(m) * slots.astype(np.float64)).astype(np.uint64)
+    slot = np.minimum(slot, slots - np.uint64(1))
+    out = np.empty(m, ACCESS_DTYPE)
+    out["addr"] = np.uint64(RANGE_BASE) + replica * np.uint64(CAPACITY_SLOT) + (slot << lg)
+    out["bytes"] = (np.uint64(1) << lg).astype(np.uint32)
+    out["flags"] = 0
+    rel = np.cumsum(rng.exponential(mean_gap, m))
+    return out, rel
+
+
 def capacity_chunks(n: int = 200_000_000, seed: int = 0, rho: float = 0.5, profile: str = "nominal",
-                    chunk: int = 8_000_000):
-    """Yields the capacity-mode stream in issue order, ``chunk`` records at a time."""
+                    chunk: int = 4_000_000, workers: int | None = None):
+    """Yields the capacity-mode stream in issue order, ``chunk`` records at a time.  Chunks are drawn
+    from independent substreams (in a thread pool); issue times are chained across chunks."""
+    from concurrent.futures import ThreadPoolExecutor
     prof = load_profile(profile, **GEOMETRY["capacity"])
     R = 64 * 8 * 4
-    mean_gap = 1.4 * prof["t_read_ns"] / (rho * R)                      # E[pages per read] = 1.4
-    t0, done, k = 0.0, 0, 0
-    while done < n:
-        m = min(chunk, n - done)
-        rng = np.random.Generator(np.random.PCG64([seed, 4, k]))
-        replica = rng.integers(0, CAPACITY_REPLICAS, m, dtype=np.uint64)
-        lg = rng.integers(7, 17, m, dtype=np.uint64)                     # 128 B ... 64 KiB
-        size = np.uint64(1) << lg
-        slots = np.uint64(WEIGHT_BYTES) >> lg
-        slot = (rng.random(m) * slots.astype(np.float64)).astype(np.uint64)
-        slot = np.minimum(slot, slots - np.uint64(1))
-        addr = np.uint64(RANGE_BASE) + replica * np.uint64(CAPACITY_SLOT) + (slot << lg)
-        issue, t0 = _poisson_issue(rng, m, mean_gap, t0)
-        yield _records(addr, issue, size.astype(np.uint32), 0)
-        done += m; k += 1
+    mean_gap = 1.4 * prof["t_read_ns"] / (rho * R)                  # E[pages per read] = 1.4
+    sizes = [min(chunk, n - s) for s in range(0, n, chunk)]
+    workers = workers or min(32, os.cpu_count() or 1)
+    t0 = 0.0
+    with ThreadPoolExecutor(workers) as pool:
+        pending = []
+        it = iter(enumerate(sizes))
+        for _ in range(workers + 1):
+            nxt = next(it, None)
+            if nxt is not None:
+                pending.append(pool.submit(_capacity_chunk, seed, nxt[0], nxt[1], mean_gap))
+        while pending:
+            out, rel = pending.pop(0).result()
+            nxt = next(it, None)
+            if nxt is not None:
+                pending.append(pool.submit(_capacity_chunk, seed, nxt[0], nxt[1], mean_gap))
+            out["issue_ns"] = np.floor(rel + t0).astype(np.int64)
+            t0 += float(rel[-1])
+            yield out
 
 
 def capacity_mode(n: int = 200_000_000, seed: int = 0, rho: float = 0.5, profile: str = "nominal",
@@ -301,7 +323,7 @@ def package_floorplan(channels: int = 32, dies: int = 8) -> dict:
     16 channel blocks each (the paper's three-HBM / two-HBF layout).  All dies of a channel map to
     that channel's block.  External power: 86.6 W over the GPU tiles (the paper's compute-limit
     load), 8 W per HBM stack; HBF idle 5 W per stack."""
-    assert channels == 32, "the package floorplan has 2 HBF stacks x 16 channel blocks"
+    assert channels % 32 == 0, "the package floorplan has 2 HBF stacks x 16 channel blocks"
     H = W = 128
     kind = np.zeros((H, W), np.int64); region = -np.ones((H, W), np.int64)
     region_kind, idle, ext = [], [], []
@@ -319,7 +341,7 @@ def package_floorplan(channels: int = 32, dies: int = 8) -> dict:
             by, bx = y0 + 12 * (b // 4), 100 + 6 * (b % 4)
             kind[by:by + 12, bx:bx + 6] = KIND_HBF; region[by:by + 12, bx:bx + 6] = len(region_kind)
             region_kind.append(KIND_HBF); idle.append(5.0 / 16); ext.append(0.0)
-    die_region = [first_hbf + c for c in range(channels) for _ in range(dies)]
+    die_region = [first_hbf + c % 32 for c in range(channels) for _ in range(dies)]     # channels beyond 32 share blocks
     return _finish_floorplan(kind, region, region_kind, idle, die_region, ext)
 
 

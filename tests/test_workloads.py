@@ -48,7 +48,7 @@ def test_prefix_kv_small():
 
 def test_capacity_chunks_are_deterministic_and_sorted():
     w = wl.capacity_mode(n=300_000)
-    parts = np.concatenate(list(wl.capacity_chunks(n=300_000, chunk=8_000_000)))
+    parts = np.concatenate(list(wl.capacity_chunks(n=300_000, workers=1)))
     assert np.array_equal(w.acc, parts)
     assert in_ranges(w).all() and (np.diff(w.acc["issue_ns"]) >= 0).all()
     sz = w.acc["bytes"].astype(np.int64)
