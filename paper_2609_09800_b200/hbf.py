@@ -323,7 +323,9 @@ class Context:
             d_ds = torch.empty(self.n_dies * 6, dtype=torch.int64, device="cuda")
             rc = self.submit_batch(d_acc, n, d_comp, d_stall, d_status, d_ds)
             if rc != 0:
-                raise HbfError(rc, "hbf_submit_batch")
+                if check:
+                    raise HbfError(rc, "hbf_submit_batch")
+                return rc, None, None, None, None
             res = self.last_result()
             if check and res["code"] != 0:
                 raise HbfError(res["code"], "batch")
