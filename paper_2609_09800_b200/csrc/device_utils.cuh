@@ -27,6 +27,21 @@ __device__ __forceinline__ uint64_t ld_nc_u64(const uint64_t *p) {
     uint64_t v; asm volatile("ld.global.nc.u64 %0, [%1];" : "=l"(v) : "l"(p)); return v;
 }
 
+// ---- division by a run-time constant ----------------------------------------------------------------
+// For d not a power of two, l = ceil(log2 d), magic = floor(2^(63+l) / d) + 1: floor(n / d) =
+// mulhi(n, magic) >> (l - 1) for every n < 2^63 (the error term n * (magic*d - 2^(63+l)) stays below 2^(63+l)).
+__host__ __device__ inline Div64 make_div64(uint64_t d) {
+    Div64 r; r.magic = 0; r.shift = 0; r.pow2 = 0;
+    if ((d & (d - 1)) == 0) { r.pow2 = 1; while ((1ull << r.shift) < d) ++r.shift; return r; }
+    uint32_t l = 0; while (l < 64 && (1ull << l) < d) ++l;
+    const unsigned __int128 num = (unsigned __int128)1 << (63 + l);
+    r.magic = (uint64_t)(num / d) + 1ull; r.shift = l - 1;
+    return r;
+}
+__device__ __forceinline__ uint64_t div64(uint64_t n, const Div64 &d) {
+    return d.pow2 ? (n >> d.shift) : (__umul64hi(n, d.magic) >> d.shift);
+}
+
 __device__ __forceinline__ unsigned lane_id() { return threadIdx.x & 31u; }
 __device__ __forceinline__ unsigned lanemask_lt() { unsigned m; asm("mov.u32 %0, %%lanemask_lt;" : "=r"(m)); return m; }
 
@@ -100,14 +115,14 @@ __device__ __forceinline__ Decoded decode(const ModelParams &mp, uint64_t off, u
 struct Terms { int64_t s, xfer, energy, cb; };
 
 __device__ __forceinline__ Terms service_terms(const ModelParams &mp, uint32_t bytes, uint32_t npages, uint32_t op,
-                                               int64_t q_ppm) {
+                                               int64_t q_ppm, const Div64 &div_q) {
     Terms t;
     uint32_t gs = op ? mp.prog_gran_shift : mp.read_gran_shift;
     uint64_t cb = (((uint64_t)bytes + (1ull << gs) - 1ull) >> gs) << gs;
     t.cb = (int64_t)cb;
-    t.xfer = (int64_t)((cb * 1000ull + mp.chan_bytes_per_us - 1ull) / mp.chan_bytes_per_us);
+    t.xfer = (int64_t)div64(cb * 1000ull + mp.chan_bytes_per_us - 1ull, mp.div_chan);
     int64_t s0 = (int64_t)npages * (op ? mp.t_prog_ns : mp.t_read_ns);
-    t.s = q_ppm == 1000000 ? s0 : (int64_t)(((uint64_t)s0 * 1000000ull + (uint64_t)q_ppm - 1ull) / (uint64_t)q_ppm);
+    t.s = q_ppm == 1000000 ? s0 : (int64_t)div64((uint64_t)s0 * 1000000ull + (uint64_t)q_ppm - 1ull, div_q);
     t.energy = op ? mp.e_cmd_prog_pj + mp.e_byte_prog_pj * (int64_t)cb : mp.e_cmd_read_pj + mp.e_byte_read_pj * (int64_t)cb;
     return t;
 }

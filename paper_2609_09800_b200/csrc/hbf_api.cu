@@ -40,13 +40,21 @@ struct hbf_ctx {
     float *h_ext = nullptr;                      // pinned [n_regions]
     bool submitted = false;
     bool profiling = false; cudaEvent_t ev[kProfEvents] = {}; cudaEvent_t ev_th[2] = {}; bool ev_made = false;
-    bool prof_submit = false, prof_thermal = false;
+    bool prof_submit = false, prof_thermal = false, prof_inorder = false, inorder_ok = false;
     // thermal
     bool thermal = false; ThermalDev td{}; int cur = 0; double euler_limit_s = 0.0;
     std::vector<void *> owned;
 };
 
 #define CK(expr) do { cudaError_t e_ = (expr); if (e_ != cudaSuccess) return HBF_E_CUDA; } while (0)
+
+static Div64 make_div64_host(uint64_t d) {       // same construction as the device helper
+    Div64 r; r.magic = 0; r.shift = 0; r.pow2 = 0;
+    if ((d & (d - 1)) == 0) { r.pow2 = 1; while ((1ull << r.shift) < d) ++r.shift; return r; }
+    uint32_t l = 0; while (l < 64 && (1ull << l) < d) ++l;
+    r.magic = (uint64_t)(((unsigned __int128)1 << (63 + l)) / d) + 1ull; r.shift = l - 1;
+    return r;
+}
 
 static bool is_pow2(uint64_t v) { return v && !(v & (v - 1)); }
 static uint32_t log2u(uint64_t v) { uint32_t s = 0; while ((1ull << s) < v) ++s; return s; }
@@ -144,6 +152,12 @@ int hbf_create(const hbf_config_t *cfg, void *cuda_stream, hbf_ctx **out) {
     mp.e_cmd_read_pj = cfg->e_cmd_read_pj; mp.e_byte_read_pj = cfg->e_byte_read_pj;
     mp.e_cmd_prog_pj = cfg->e_cmd_prog_pj; mp.e_byte_prog_pj = cfg->e_byte_prog_pj;
 
+    mp.div_chan = make_div64_host(cfg->chan_bytes_per_us);
+    {   // the in-order path packs the transfer time of an access into 31 bits and keeps per-queue state in shared memory
+        const unsigned __int128 worst = ((unsigned __int128)0xffffffffull + std::max(cfg->read_granule, cfg->prog_granule)) * 1000u;
+        c->inorder_ok = nq <= kInMaxQueues && worst / cfg->chan_bytes_per_us < ((unsigned __int128)1 << 31) &&
+                        57344u + nq * 16u + nd * 24u <= 200u * 1024u;
+    }
     DevState st0; st0.mode = HBF_MODE_NORMAL; st0.poisoned = 0; st0.q_ppm = 1000000;
     if ((rc = dev_copy(c, &c->d_ranges, nullptr, 1))) return fail(rc);
     if ((rc = dev_copy(c, &c->d_mp, &mp, 1))) return fail(rc);
@@ -274,7 +288,8 @@ int hbf_submit_batch(hbf_ctx *c, const hbf_access_t *d_acc, uint64_t n, int64_t 
     a.acc = d_acc; a.n = n; a.completion = d_completion_ns; a.stall = d_stall_ns; a.status = d_status; a.die_stats = d_die_stats;
     a.ranges = c->d_ranges; a.mp_dev = c->d_mp; a.mp = c->mp; a.state = c->d_state; a.ctrl = c->d_ctrl; a.result = c->d_result;
     a.busy = c->d_busy; a.busy_stage = c->d_busy_stage; a.pending = c->d_pending; a.stats_stage = c->d_stats_stage;
-    a.path = c->path; a.sm_count = c->sm_count;
+    a.path = c->path; a.sm_count = c->sm_count; a.inorder_ok = c->inorder_ok ? 1 : 0;
+    c->prof_inorder = c->profiling && n > 0 && c->inorder_ok && (c->path == HBF_PATH_AUTO || c->path == HBF_PATH_INORDER);
     a.ev = c->profiling ? c->ev : nullptr;
     c->prof_submit = c->profiling;
     CK(launch_submit(a, c->stream));
@@ -405,8 +420,15 @@ int hbf_get_profile(hbf_ctx *c, float *ms_out, uint32_t cap) {
     if (!c || !ms_out || cap < HBF_PROF_STAGES) return HBF_E_INVAL;
     for (int k = 0; k < HBF_PROF_STAGES; ++k) ms_out[k] = 0.0f;
     CK(cudaStreamSynchronize(c->stream));
-    if (c->prof_submit)
-        for (int k = 0; k < 6; ++k) CK(cudaEventElapsedTime(&ms_out[k], c->ev[k], c->ev[k + 1]));
+    if (c->prof_submit) {
+        for (int k = 1; k < 6; ++k) CK(cudaEventElapsedTime(&ms_out[k], c->ev[k], c->ev[k + 1]));
+        if (c->prof_inorder) {                      // begin | in-order kernels | (second begin +) sort path ...
+            CK(cudaEventElapsedTime(&ms_out[0], c->ev[0], c->ev[7]));
+            CK(cudaEventElapsedTime(&ms_out[6], c->ev[7], c->ev[8]));
+        } else {
+            CK(cudaEventElapsedTime(&ms_out[0], c->ev[0], c->ev[1]));
+        }
+    }
     if (c->prof_thermal) CK(cudaEventElapsedTime(&ms_out[7], c->ev_th[0], c->ev_th[1]));
     return HBF_OK;
 }

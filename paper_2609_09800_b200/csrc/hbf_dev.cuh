@@ -25,6 +25,9 @@ struct RangeSnap {
     uint32_t pad;
 };
 
+// Exact unsigned division of n < 2^63 by a run-time constant: one multiply-high and a shift.
+struct Div64 { uint64_t magic; uint32_t shift; uint32_t pow2; };
+
 // Geometry and timing, fixed at create.
 struct ModelParams {
     uint32_t channels, dies, planes;
@@ -36,6 +39,7 @@ struct ModelParams {
     uint32_t read_gran_shift, prog_gran_shift;
     int64_t t_read_ns, t_prog_ns;
     uint64_t chan_bytes_per_us;
+    Div64 div_chan;                      // division by chan_bytes_per_us
     int64_t e_cmd_read_pj, e_byte_read_pj, e_cmd_prog_pj, e_byte_prog_pj;
 };
 
@@ -53,10 +57,13 @@ struct BatchCtrl {
     int32_t skip;                        // later kernels do nothing when set
     int32_t mode; int32_t pad0;
     int64_t q_ppm;
+    Div64 div_q;                         // division by the batch's snapshot of q
     unsigned long long n_native, n_ready, n_fault;
     unsigned long long key_or, key_and;
     uint32_t unsorted;                   // some record has a smaller issue time than its predecessor
     uint32_t inorder_used;               // the in-order path served this batch
+    uint32_t run_sort;                   // the sort path has to serve this batch
+    uint32_t pad1;
     uint32_t tile_counter[kMaxPasses + 2];
     long long modeled_ns, service_ns, max_completion_ns;
     SortPlan plan;
@@ -75,7 +82,8 @@ struct Workspace {
     uint32_t *hist;                      // [kMaxPasses][kRadix]
     uint32_t *sort_desc[2];              // [tiles][kRadix] look-back words, ping-pong between passes
     void *scan_desc;                     // [scan tiles] ScanDesc
-    void *inorder_desc;                  // in-order path tile state
+    int64_t *in_agg;                     // [tiles][queues][2]: per-tile, per-queue max-plus aggregate (S, M)
+    int64_t *in_bin;                     // [tiles][queues]: busy-until entering each tile
     size_t bytes;
 };
 
@@ -85,13 +93,18 @@ struct SubmitArgs {
     const RangeSnap *ranges; const ModelParams *mp_dev; ModelParams mp;
     DevState *state; BatchCtrl *ctrl; hbf_batch_result_t *result;
     int64_t *busy, *busy_stage, *pending; hbf_die_stats_t *stats_stage;
-    Workspace ws; int32_t path; int sm_count;
+    Workspace ws; int32_t path; int sm_count; int inorder_ok;
     cudaEvent_t *ev;                     // [kProfEvents] or null: recorded between kernel groups
 };
-constexpr int kProfEvents = 8;
+constexpr int kProfEvents = 10;
 extern unsigned long long g_kernel_launches;
 
+constexpr uint32_t kInMaxQueues = 2048;  // the in-order path keeps per-queue state in shared memory
+constexpr uint32_t kInMaxTiles = 1024;
 size_t workspace_layout(uint64_t n, uint32_t n_queues, Workspace *ws, void *base);
+// tile size (records) of the in-order path for a batch of n on a device with sm_count SMs
+uint64_t inorder_tile_records(uint64_t n, int sm_count);
+cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st);
 cudaError_t launch_submit(const SubmitArgs &a, cudaStream_t st);
 cudaError_t launch_queue_order(const BatchCtrl *ctrl, const Workspace &ws, uint32_t *out, uint64_t n, cudaStream_t st);
 

@@ -13,16 +13,27 @@ namespace hbf {
 // =====================================================================================================
 // begin: snapshot mode and q (before any reservation, Eq. 3), stage the queue state, clear the block
 // =====================================================================================================
+// role 0: first kernel of a batch; run_sort tells whether the sort path serves it.
+// role 1: placed between the in-order attempt and the sort kernels; it starts the batch over for the
+//         sort path when the in-order attempt found the records out of issue order, else does nothing.
 __global__ void k_begin(BatchCtrl *ctrl, const DevState *state, const int64_t *busy, int64_t *busy_stage,
-                        hbf_die_stats_t *stats_stage, uint32_t *hist, uint32_t n_queues, uint32_t n_dies) {
+                        hbf_die_stats_t *stats_stage, uint32_t *hist, uint32_t n_queues, uint32_t n_dies,
+                        int role, int run_sort) {
     const int tid = threadIdx.x;
+    if (role == 1) {
+        if (ctrl->skip || !ctrl->run_sort) return;
+        run_sort = 1;
+    }
+    __syncthreads();
     uint32_t *w = reinterpret_cast<uint32_t *>(ctrl);
     for (int i = tid; i < (int)(sizeof(BatchCtrl) / 4); i += blockDim.x) w[i] = 0u;
     __syncthreads();
     if (tid == 0) {
         int32_t mode = state->mode;
         ctrl->mode = mode; ctrl->q_ppm = state->q_ppm;
+        ctrl->div_q = make_div64((uint64_t)state->q_ppm);
         ctrl->key_and = ~0ull;
+        ctrl->run_sort = (uint32_t)run_sort;
         if (state->poisoned) { ctrl->code = HBF_E_TIMEOUT; ctrl->skip = 1; }
         else if (mode == HBF_MODE_SHUTDOWN) { ctrl->code = HBF_E_LINK_SHUTDOWN; ctrl->skip = 1; }
         else if (mode == HBF_MODE_SEVERE) { ctrl->code = HBF_E_THROTTLED; ctrl->skip = 1; }
@@ -48,7 +59,7 @@ k_classify(const hbf_access_t *__restrict__ acc, uint64_t n, const RangeSnap *__
     __shared__ RangeSnap rs;
     __shared__ ModelParams mp;
     __shared__ __align__(16) uint64_t rec[kClsTile * 3];
-    if (ctrl->skip) return;
+    if (ctrl->skip || !ctrl->run_sort) return;
     const int tid = threadIdx.x;
     for (int i = tid; i < (int)(sizeof(RangeSnap) / 4); i += kClsThreads)
         reinterpret_cast<uint32_t *>(&rs)[i] = reinterpret_cast<const uint32_t *>(ranges_g)[i];
@@ -132,7 +143,7 @@ __device__ __forceinline__ uint64_t compact_key(uint64_t key, uint32_t lo_bits, 
 }
 
 __global__ void k_plan(BatchCtrl *ctrl, int force_full) {
-    if (threadIdx.x != 0 || ctrl->skip) return;
+    if (threadIdx.x != 0 || ctrl->skip || !ctrl->run_sort) return;
     if (ctrl->n_fault) { ctrl->code = HBF_E_ACCESS_FAULT; ctrl->skip = 1; return; }
     const uint64_t diff = ctrl->key_or ^ ctrl->key_and;
     const uint64_t dlo = diff & kIssueMask, dhi = diff >> kIssueBits;
@@ -158,7 +169,7 @@ constexpr int kHistThreads = 512;
 __global__ void __launch_bounds__(kHistThreads)
 k_hist(const uint64_t *__restrict__ keys, uint64_t n, const BatchCtrl *ctrl, uint32_t *hist) {
     __shared__ uint32_t sh[kMaxPasses * kRadix];
-    if (ctrl->skip) return;
+    if (ctrl->skip || !ctrl->run_sort) return;
     const SortPlan p = ctrl->plan;
     if (p.n_passes == 0) return;
     for (int i = threadIdx.x; i < kMaxPasses * kRadix; i += kHistThreads) sh[i] = 0u;
@@ -203,7 +214,7 @@ k_sort_pass(int pass, uint64_t n, BatchCtrl *ctrl, DevState *state, const uint32
     __shared__ uint32_t s_delta[kRadix];
     __shared__ uint32_t s_warp_tot[kRadix / 32], s_hist_tot[kRadix / 32];
     __shared__ uint32_t s_tile;
-    if (ctrl->skip) return;
+    if (ctrl->skip || !ctrl->run_sort) return;
     const SortPlan &pl = ctrl->plan;
     if (pass >= (int)pl.n_passes) return;
     const uint32_t lo_bits = pl.lo_bits, hi_bits = pl.hi_bits, shift = pl.shift[pass];
@@ -347,7 +358,7 @@ k_scan(const hbf_access_t *__restrict__ acc, uint64_t n, const RangeSnap *__rest
     __shared__ uint32_t s_tile;
     __shared__ long long s_die_acc[6];
     __shared__ long long s_res[3];
-    if (ctrl->skip) return;
+    if (ctrl->skip || !ctrl->run_sort) return;
     const uint64_t m = ctrl->n_ready;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) s_tile = atomicAdd(&ctrl->tile_counter[kMaxPasses], 1u);
@@ -365,6 +376,7 @@ k_scan(const hbf_access_t *__restrict__ acc, uint64_t n, const RangeSnap *__rest
     const uint64_t *keys = (np & 1u) ? keys1 : keys0;
     const uint32_t *idxs = np == 0u ? nullptr : ((np & 1u) ? idx1 : idx0);
     const int64_t q_ppm = ctrl->q_ppm;
+    const Div64 div_q = ctrl->div_q;
     const int cnt = (int)min((uint64_t)kScanTile, m - base);
 
     // this thread's consecutive items
@@ -426,7 +438,7 @@ k_scan(const hbf_access_t *__restrict__ acc, uint64_t n, const RangeSnap *__rest
             classify(rs, r_addr[j], issue[j], bytes, op, &g);
             const uint64_t off = rs.media_offset[g] + (r_addr[j] - rs.base[g]);
             const Decoded d = decode(mp, off, bytes);
-            const Terms t = service_terms(mp, bytes, d.npages, op, q_ppm);
+            const Terms t = service_terms(mp, bytes, d.npages, op, q_ppm, div_q);
             s[j] = t.s;
             if (op) { a[j] = issue[j] + t.xfer; post[j] = 0u; } else { a[j] = issue[j]; post[j] = (uint32_t)t.xfer; }
             if (d.die != run_die) { if (run_die != 0xffffffffu) flush_run(run_die); run_die = d.die; }
@@ -580,18 +592,23 @@ k_scan(const hbf_access_t *__restrict__ acc, uint64_t n, const RangeSnap *__rest
 __global__ void k_finish(uint64_t n, BatchCtrl *ctrl, DevState *state, int64_t *busy, const int64_t *busy_stage,
                          int64_t *pending, const hbf_die_stats_t *stats_stage, hbf_die_stats_t *die_stats,
                          int64_t *completion, int64_t *stall, hbf_batch_result_t *result,
-                         uint32_t n_queues, uint32_t n_dies) {
+                         const ModelParams *__restrict__ mp, uint32_t n_queues, uint32_t n_dies) {
     const int code = ctrl->code;
     const uint64_t gtid = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const uint64_t gsz = (uint64_t)gridDim.x * blockDim.x;
-    if (code == HBF_E_ACCESS_FAULT || code == HBF_E_TIMEOUT) {
+    if (code == HBF_E_ACCESS_FAULT || code == HBF_E_TIMEOUT || code == HBF_E_INVAL) {
         for (uint64_t i = gtid; i < n; i += gsz) { completion[i] = 0; stall[i] = 0; }
         if (die_stats) for (uint64_t i = gtid; i < (uint64_t)n_dies * 6u; i += gsz) reinterpret_cast<int64_t *>(die_stats)[i] = 0;
     } else if (code == HBF_OK) {
+        const bool inorder = ctrl->inorder_used != 0u;
         for (uint64_t r = gtid; r < n_queues; r += gsz) busy[r] = busy_stage[r];
         for (uint64_t d = gtid; d < n_dies; d += gsz) {
-            pending[d] += stats_stage[d].energy_pj;
-            if (die_stats) die_stats[d] = stats_stage[d];
+            hbf_die_stats_t ds = stats_stage[d];
+            // the in-order path keeps byte and access counts only: the energy is linear in them
+            if (inorder) ds.energy_pj = mp->e_cmd_read_pj * ds.n_read + mp->e_byte_read_pj * ds.bytes_read +
+                                        mp->e_cmd_prog_pj * ds.n_prog + mp->e_byte_prog_pj * ds.bytes_prog;
+            pending[d] += ds.energy_pj;
+            if (die_stats) die_stats[d] = ds;
         }
     }
     if (gtid == 0) {
@@ -622,7 +639,6 @@ __global__ void k_queue_order(const BatchCtrl *ctrl, const uint32_t *idx0, const
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 size_t workspace_layout(uint64_t n, uint32_t n_queues, Workspace *ws, void *base_ptr) {
-    (void)n_queues;
     const uint64_t nn = n ? n : 1;
     const uint64_t sort_tiles = (nn + kSortTile - 1) / kSortTile, scan_tiles = (nn + kScanTile - 1) / kScanTile;
     size_t off = 0;
@@ -632,59 +648,89 @@ size_t workspace_layout(uint64_t n, uint32_t n_queues, Workspace *ws, void *base
     void *h = take((size_t)kMaxPasses * kRadix * 4);
     void *d0 = take(sort_tiles * kRadix * 4), *d1 = take(sort_tiles * kRadix * 4);
     void *sd = take(scan_tiles * sizeof(ScanDesc));
+    const uint64_t in_tiles = std::min<uint64_t>(kInMaxTiles, (nn + 2047) / 2048);
+    const bool inorder = n_queues <= kInMaxQueues;
+    void *ia = take(inorder ? in_tiles * n_queues * 16 : 0), *ib = take(inorder ? in_tiles * n_queues * 8 : 0);
     if (ws) {
         ws->keys[0] = (uint64_t *)k0; ws->keys[1] = (uint64_t *)k1; ws->idx[0] = (uint32_t *)i0; ws->idx[1] = (uint32_t *)i1;
         ws->hist = (uint32_t *)h; ws->sort_desc[0] = (uint32_t *)d0; ws->sort_desc[1] = (uint32_t *)d1;
-        ws->scan_desc = sd; ws->inorder_desc = nullptr; ws->bytes = off;
+        ws->scan_desc = sd; ws->in_agg = (int64_t *)ia; ws->in_bin = (int64_t *)ib; ws->bytes = off;
     }
     return off;
 }
 
 unsigned long long g_kernel_launches = 0;
 
+static cudaError_t launch_sort_path(const SubmitArgs &a, cudaStream_t st) {
+    const uint64_t n = a.n;
+    auto mark = [&](int k) { if (a.ev) cudaEventRecord(a.ev[k], st); };
+    const uint64_t sort_tiles = (n + kSortTile - 1) / kSortTile, scan_tiles = (n + kScanTile - 1) / kScanTile;
+    cudaError_t e = cudaMemsetAsync(a.ws.sort_desc[0], 0, sort_tiles * kRadix * 4, st);
+    if (e != cudaSuccess) return e;
+    e = cudaMemsetAsync(a.ws.scan_desc, 0, scan_tiles * sizeof(ScanDesc), st);
+    if (e != cudaSuccess) return e;
+    mark(1);
+    const uint64_t cls_tiles = (n + kClsTile - 1) / kClsTile;
+    const unsigned cls_grid = (unsigned)std::min<uint64_t>(cls_tiles, (uint64_t)a.sm_count * 8);
+    k_classify<<<cls_grid, kClsThreads, 0, st>>>(a.acc, n, a.ranges, a.mp_dev, a.ctrl, a.ws.keys[0], a.status,
+                                                 a.completion, a.stall);
+    mark(2);
+    k_plan<<<1, 32, 0, st>>>(a.ctrl, a.path == HBF_PATH_SORT_FULL ? 1 : 0);
+    const unsigned hist_grid = (unsigned)std::min<uint64_t>((n + kHistThreads * 8 - 1) / (kHistThreads * 8), (uint64_t)a.sm_count * 4);
+    k_hist<<<hist_grid, kHistThreads, 0, st>>>(a.ws.keys[0], n, a.ctrl, a.ws.hist);
+    mark(3);
+    static bool attr_set = false;
+    if (!attr_set) {
+        e = cudaFuncSetAttribute(k_sort_pass, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSortSmem);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    for (int p = 0; p < kMaxPasses; ++p)
+        k_sort_pass<<<(unsigned)sort_tiles, kSortThreads, kSortSmem, st>>>(p, n, a.ctrl, a.state, a.ws.hist, a.ws.keys[0], a.ws.keys[1],
+                                                                           a.ws.idx[0], a.ws.idx[1], a.ws.sort_desc[0], a.ws.sort_desc[1]);
+    mark(4);
+    k_scan<<<(unsigned)scan_tiles, kScanThreads, 0, st>>>(a.acc, n, a.ranges, a.mp_dev, a.ctrl, a.state, a.ws.keys[0], a.ws.keys[1],
+                                                         a.ws.idx[0], a.ws.idx[1], (ScanDesc *)a.ws.scan_desc, a.busy,
+                                                         a.busy_stage, a.stats_stage, a.completion, a.stall);
+    g_kernel_launches += 4 + kMaxPasses;
+    return cudaSuccess;
+}
+
+// Kernel order of one batch.  AUTO: begin, the in-order kernels (they serve the batch when its records
+// arrive in non-decreasing issue order), a second begin and the sort kernels (they do nothing unless the
+// in-order attempt handed the batch over), finish.  SORT / SORT_FULL: begin, sort kernels, finish.
 cudaError_t launch_submit(const SubmitArgs &a, cudaStream_t st) {
     const uint64_t n = a.n;
     auto mark = [&](int k) { if (a.ev) cudaEventRecord(a.ev[k], st); };
+    const bool try_inorder = a.inorder_ok && (a.path == HBF_PATH_AUTO || a.path == HBF_PATH_INORDER);
+    const bool sort_kernels = a.path != HBF_PATH_INORDER || !a.inorder_ok;
     mark(0);
-    k_begin<<<1, 256, 0, st>>>(a.ctrl, a.state, a.busy, a.busy_stage, a.stats_stage, a.ws.hist, a.mp.n_queues, a.mp.n_dies);
+    k_begin<<<1, 256, 0, st>>>(a.ctrl, a.state, a.busy, a.busy_stage, a.stats_stage, a.ws.hist, a.mp.n_queues, a.mp.n_dies,
+                               0, try_inorder ? 0 : 1);
     g_kernel_launches += 1;
     if (n > 0) {
-        const uint64_t sort_tiles = (n + kSortTile - 1) / kSortTile, scan_tiles = (n + kScanTile - 1) / kScanTile;
-        cudaError_t e = cudaMemsetAsync(a.ws.sort_desc[0], 0, sort_tiles * kRadix * 4, st);
-        if (e != cudaSuccess) return e;
-        e = cudaMemsetAsync(a.ws.scan_desc, 0, scan_tiles * sizeof(ScanDesc), st);
-        if (e != cudaSuccess) return e;
-        mark(1);
-        const uint64_t cls_tiles = (n + kClsTile - 1) / kClsTile;
-        const unsigned cls_grid = (unsigned)std::min<uint64_t>(cls_tiles, (uint64_t)a.sm_count * 8);
-        k_classify<<<cls_grid, kClsThreads, 0, st>>>(a.acc, n, a.ranges, a.mp_dev, a.ctrl, a.ws.keys[0], a.status,
-                                                     a.completion, a.stall);
-        mark(2);
-        k_plan<<<1, 32, 0, st>>>(a.ctrl, a.path == HBF_PATH_SORT_FULL ? 1 : 0);
-        const unsigned hist_grid = (unsigned)std::min<uint64_t>((n + kHistThreads * 8 - 1) / (kHistThreads * 8), (uint64_t)a.sm_count * 4);
-        k_hist<<<hist_grid, kHistThreads, 0, st>>>(a.ws.keys[0], n, a.ctrl, a.ws.hist);
-        mark(3);
-        static bool attr_set = false;
-        if (!attr_set) {
-            e = cudaFuncSetAttribute(k_sort_pass, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSortSmem);
+        if (try_inorder) {
+            mark(7);
+            cudaError_t e = launch_inorder(a, st);
             if (e != cudaSuccess) return e;
-            attr_set = true;
+            mark(8);
+            if (sort_kernels) {
+                k_begin<<<1, 256, 0, st>>>(a.ctrl, a.state, a.busy, a.busy_stage, a.stats_stage, a.ws.hist, a.mp.n_queues,
+                                           a.mp.n_dies, 1, 1);
+                g_kernel_launches += 1;
+            }
         }
-        for (int p = 0; p < kMaxPasses; ++p)
-            k_sort_pass<<<(unsigned)sort_tiles, kSortThreads, kSortSmem, st>>>(p, n, a.ctrl, a.state, a.ws.hist, a.ws.keys[0], a.ws.keys[1],
-                                                                               a.ws.idx[0], a.ws.idx[1], a.ws.sort_desc[0], a.ws.sort_desc[1]);
-        mark(4);
-        k_scan<<<(unsigned)scan_tiles, kScanThreads, 0, st>>>(a.acc, n, a.ranges, a.mp_dev, a.ctrl, a.state, a.ws.keys[0], a.ws.keys[1],
-                                                             a.ws.idx[0], a.ws.idx[1], (ScanDesc *)a.ws.scan_desc, a.busy,
-                                                             a.busy_stage, a.stats_stage, a.completion, a.stall);
-        g_kernel_launches += 4 + kMaxPasses;
+        if (sort_kernels) {
+            cudaError_t e = launch_sort_path(a, st);
+            if (e != cudaSuccess) return e;
+        } else { mark(1); mark(2); mark(3); mark(4); }
     } else {
         mark(1); mark(2); mark(3); mark(4);
     }
     mark(5);
     const unsigned fin_grid = (unsigned)std::max<uint64_t>(1, std::min<uint64_t>((n + 1023) / 1024, (uint64_t)a.sm_count * 4));
     k_finish<<<fin_grid, 256, 0, st>>>(n, a.ctrl, a.state, a.busy, a.busy_stage, a.pending, a.stats_stage, a.die_stats,
-                                       a.completion, a.stall, a.result, a.mp.n_queues, a.mp.n_dies);
+                                       a.completion, a.stall, a.result, a.mp_dev, a.mp.n_queues, a.mp.n_dies);
     g_kernel_launches += 1;
     mark(6);
     return cudaGetLastError();

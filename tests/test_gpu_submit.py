@@ -203,3 +203,73 @@ def test_state_blob_round_trip(hbf):
     compare_batch(g2, o, w.acc[4000:])
     with pytest.raises(hbf.HbfError):
         g2.set_state(blob[:-8])
+
+
+# ---- the in-order path (batches whose records arrive in non-decreasing issue order) ---------------------
+
+def issue_sorted(acc):
+    return np.sort(acc, order="issue_ns", kind="stable")
+
+
+@pytest.mark.parametrize("n", [1, 2, 2047, 2048, 2049, 4096, 10_000, 100_003])
+def test_inorder_path_mixed_status(hbf, n):
+    w = wl.mixed_status(n, seed=n + 1)
+    acc = issue_sorted(w.acc)
+    for path in (hbf.PATH_INORDER, hbf.PATH_AUTO, hbf.PATH_SORT):
+        g, o = contexts(hbf, w.profile, w.ranges, path)
+        cut = n // 2
+        compare_batch(g, o, acc[:cut])
+        compare_batch(g, o, acc[cut:])
+
+
+def test_inorder_path_is_the_one_auto_takes(hbf):
+    w = wl.tiny_uniform(30_000)
+    g, o = contexts(hbf, w.profile, w.ranges, hbf.PATH_AUTO)
+    compare_batch(g, o, w.acc)
+    with pytest.raises(hbf.HbfError):                       # no sorted index array exists after an in-order batch
+        g.queue_order(w.n)
+    shuffled = w.acc[np.random.default_rng(0).permutation(w.n)]
+    compare_batch(g, o, shuffled, check_order=True)         # falls back to the sort path
+
+
+def test_forced_inorder_refuses_unsorted_batches(hbf):
+    w = wl.mixed_status(5000, seed=3)
+    g, o = contexts(hbf, w.profile, w.ranges, hbf.PATH_INORDER)
+    rc, comp, stall, _, ds = g.submit_host(w.acc, check=False)
+    assert rc == hbf.E_INVAL and not comp.any() and not stall.any() and not ds["busy_ns"].any()
+    assert not g.get_busy_until().any()
+    compare_batch(g, o, issue_sorted(w.acc))
+
+
+def test_inorder_path_faults_and_throttle(hbf):
+    wf = wl.mixed_status(9000, seed=6, faults=True)
+    w = wl.mixed_status(9000, seed=6)
+    g, o = contexts(hbf, w.profile, w.ranges, hbf.PATH_AUTO)
+    assert compare_batch(g, o, issue_sorted(wf.acc)) == hbfo.E_ACCESS_FAULT
+    g.force_mode(hbf.MODE_LIGHT, 700_001); o.force_mode(hbfo.MODE_LIGHT, 700_001)
+    compare_batch(g, o, issue_sorted(w.acc))
+
+
+def test_inorder_hot_queue_and_equal_issue(hbf):
+    rng = np.random.default_rng(8)
+    n = 60_000
+    acc = np.zeros(n, hbfo.ACCESS_DTYPE)
+    acc["addr"] = wl.RANGE_BASE + rng.integers(0, 3, n).astype(np.uint64) * np.uint64(16384) + rng.integers(0, 4, n).astype(np.uint64) * np.uint64(4096)
+    acc["issue_ns"] = np.sort(rng.integers(0, 2000, n))
+    acc["bytes"] = rng.choice([64, 4096, 16384, 40000], n)
+    acc["flags"] = rng.random(n) < 0.3
+    prof = wl.load_profile("nominal", **wl.GEOMETRY["tiny"])
+    g, o = contexts(hbf, prof, [(wl.RANGE_BASE, wl.GIB, 3, 0, 0, 0)], hbf.PATH_INORDER)
+    compare_batch(g, o, acc)
+    compare_batch(g, o, acc)
+
+
+@pytest.mark.parametrize("geo", [dict(channels=3, dies=5, planes=2, page_bytes=4096, stripe_bytes=16384),
+                                 dict(channels=8, dies=4, planes=2, page_bytes=16384, stripe_bytes=16384, queue_level=1),
+                                 dict(channels=32, dies=8, planes=8, page_bytes=16384, stripe_bytes=16384),
+                                 dict(channels=1, dies=1, planes=1, page_bytes=16384, stripe_bytes=16384)])
+def test_inorder_other_geometries(hbf, geo):
+    w = wl.mixed_status(40_000, seed=5)
+    prof = dict(w.profile); prof.update(geo)
+    g, o = contexts(hbf, prof, w.ranges, hbf.PATH_INORDER)
+    compare_batch(g, o, issue_sorted(w.acc))
