@@ -177,6 +177,34 @@ HBF_API int hbf_get_profile(hbf_ctx *ctx, float *ms_out, uint32_t cap);
 /* Number of kernels this library has launched in the calling process so far. */
 HBF_API uint64_t hbf_kernel_launches(void);
 
+/* Explicit-Euler substeps of the package RC network without any allocation.  (The paper has no
+ * counterpart: this entry point exists for callers that are not allowed to allocate device memory,
+ * for example a serving loop that cannot afford the device-wide synchronisation cudaMalloc may cause,
+ * or a plug-in that must work inside the buffers its host application hands it.)
+ *
+ * It needs no context.  The caller passes every input and output as device pointers:
+ * d_cell_C, d_cell_Gx, d_cell_Gy, d_cell_Gsink, d_cell_power_w [grid_h*grid_w] are read only (same
+ * meaning and layout as in hbf_config_t; power in watts per cell); d_theta [grid_h*grid_w] is the
+ * field as rise above ambient, advanced in place by n_sub substeps of dt_sub_s seconds (same
+ * arithmetic as hbf_thermal_step); d_comp [grid_h*grid_w] is the per-cell compensation term that
+ * belongs to d_theta (zero for a fresh field, carried from call to call).  Work is enqueued on
+ * cuda_stream (a cudaStream_t, NULL = default stream); the call does not wait for it.
+ *
+ * The second field buffer the update needs lives in an array built into the library: 256 KiB of
+ * device memory on every GPU that loads the library, held until the process exits.  Grids of more
+ * than HBF_STATIC_MAX_CELLS cells are refused with HBF_E_WORKSPACE.  No cudaMalloc, cudaFree or
+ * allocating library routine is called.  The first call on each device looks the array's device
+ * address up (with that device current); make that first call before any stream capture begins.
+ * All calls on one GPU share the array, which keeps whatever the last call left in it; nothing in
+ * it has to be cleared, because every cell is written before it is read.  Two calls whose kernels
+ * overlap on the GPU (different streams) race on it: order them.  The stability limit of the
+ * explicit step is not checked here; hbf_euler_limit_ns gives it for a context's floorplan. */
+#define HBF_STATIC_MAX_CELLS 65536
+HBF_API int hbf_euler_substeps_static(const float *d_cell_C, const float *d_cell_Gx, const float *d_cell_Gy,
+                                      const float *d_cell_Gsink, const float *d_cell_power_w, float *d_theta,
+                                      float *d_comp, uint32_t grid_h, uint32_t grid_w, uint32_t n_sub,
+                                      float dt_sub_s, void *cuda_stream);
+
 HBF_API const char *hbf_strerror(int code);
 
 #ifdef __cplusplus

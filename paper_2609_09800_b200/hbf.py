@@ -28,7 +28,8 @@ EXPORTS = ("hbf_create", "hbf_destroy", "hbf_register_range", "hbf_clear_ranges"
            "hbf_submit_batch", "hbf_last_result", "hbf_thermal_step", "hbf_force_mode", "hbf_get_mode",
            "hbf_reset", "hbf_set_path", "hbf_get_state", "hbf_set_state", "hbf_get_busy_until",
            "hbf_get_pending_energy", "hbf_get_temps", "hbf_euler_limit_ns", "hbf_queue_order", "hbf_strerror",
-           "hbf_set_profiling", "hbf_get_profile", "hbf_kernel_launches")
+           "hbf_set_profiling", "hbf_get_profile", "hbf_kernel_launches", "hbf_euler_substeps_static")
+STATIC_MAX_CELLS = 65536
 PROF_STAGES = ("begin", "classify", "plan_hist", "sort", "scan", "finish", "inorder", "thermal")
 
 
@@ -101,6 +102,7 @@ def lib():
         L.hbf_get_profile.argtypes = [vp, vp, u32]
         L.hbf_kernel_launches.argtypes = []
         L.hbf_kernel_launches.restype = u64
+        L.hbf_euler_substeps_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, u32, u32, u32, C.c_float, vp]
         L.hbf_strerror.argtypes = [C.c_int]
         L.hbf_strerror.restype = C.c_char_p
         _lib = L
@@ -109,6 +111,17 @@ def lib():
 
 def kernel_launches() -> int:
     return lib().hbf_kernel_launches()
+
+
+def euler_substeps_static(d_cell_C, d_cell_Gx, d_cell_Gy, d_cell_Gsink, d_cell_power_w, d_theta, d_comp,
+                          grid_h, grid_w, n_sub, dt_sub_s, stream=None) -> int:
+    """``hbf_euler_substeps_static``: advances ``d_theta`` (torch CUDA float32 tensors throughout) in place
+    using the scratch array built into the library; allocates nothing.  Returns the C return code."""
+    import torch
+    st = stream if stream is not None else torch.cuda.current_stream()
+    return lib().hbf_euler_substeps_static(_ptr(d_cell_C), _ptr(d_cell_Gx), _ptr(d_cell_Gy), _ptr(d_cell_Gsink),
+                                           _ptr(d_cell_power_w), _ptr(d_theta), _ptr(d_comp), grid_h, grid_w, n_sub,
+                                           dt_sub_s, C.c_void_p(st.cuda_stream))
 
 
 class HbfError(RuntimeError):
