@@ -72,9 +72,14 @@ __device__ __forceinline__ unsigned long long warp_and(unsigned long long v) {
 __device__ __forceinline__ int classify(const RangeSnap &rs, uint64_t addr, int64_t issue, uint32_t bytes,
                                         uint32_t flags, int *g) {
     if (bytes == 0u || (flags & ~1u) != 0u || issue < 0 || issue >= HBF_ISSUE_LIMIT) return HBF_ST_UNSUPPORTED;
-    int lo = 0, hi = (int)rs.count;              // last range with base <= addr
-    while (lo < hi) { int mid = (lo + hi) >> 1; if (rs.base[mid] <= addr) lo = mid + 1; else hi = mid; }
-    int k = lo - 1;
+    int k;
+    if (rs.count == 1u) {                        // the common registration: one range
+        k = addr >= rs.base[0] ? 0 : -1;
+    } else {
+        int lo = 0, hi = (int)rs.count;          // last range with base <= addr
+        while (lo < hi) { int mid = (lo + hi) >> 1; if (rs.base[mid] <= addr) lo = mid + 1; else hi = mid; }
+        k = lo - 1;
+    }
     if (k < 0) return HBF_ST_NATIVE;
     uint64_t rel = addr - rs.base[k];
     if (rel >= rs.length[k]) return HBF_ST_NATIVE;

@@ -70,17 +70,17 @@ k_inorder(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_record
     unsigned char *fixed = in_smem + kInWorkBytes;
     int64_t *aggS = reinterpret_cast<int64_t *>(fixed);                            // reduce: [R] ; apply: busy-until [R]
     int64_t *aggM = aggS + R;                                                      // reduce only
-    unsigned long long *st_br = reinterpret_cast<unsigned long long *>(aggM + R);  // reduce only, per die
-    unsigned long long *st_bp = st_br + n_dies;
-    uint32_t *st_nr = reinterpret_cast<uint32_t *>(st_bp + n_dies);
-    uint32_t *st_np = st_nr + n_dies;
+    // reduce only, per die: charged bytes as low/high 32-bit halves (native 32-bit shared atomics), access counts
+    uint32_t *st_br_lo = reinterpret_cast<uint32_t *>(aggM + R), *st_br_hi = st_br_lo + n_dies;
+    uint32_t *st_bp_lo = st_br_hi + n_dies, *st_bp_hi = st_bp_lo + n_dies;
+    uint32_t *st_nr = st_bp_hi + n_dies, *st_np = st_nr + n_dies;
 
     const uint32_t tile = blockIdx.x;
     const uint64_t tile_begin = (uint64_t)tile * tile_records;
     const uint64_t tile_end = min(n, tile_begin + tile_records);
     if (MODE == 0) {
         for (uint32_t r = tid; r < R; r += kInThreads) { aggS[r] = 0; aggM[r] = kNegInf; }
-        for (uint32_t d = tid; d < n_dies; d += kInThreads) { st_br[d] = 0; st_bp[d] = 0; st_nr[d] = 0; st_np[d] = 0; }
+        for (uint32_t d = tid; d < n_dies * 6u; d += kInThreads) st_br_lo[d] = 0u;
     } else {
         for (uint32_t r = tid; r < R; r += kInThreads) aggS[r] = in_bin[(uint64_t)tile * R + r];
     }
@@ -142,8 +142,13 @@ k_inorder(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_record
                     xo[j] = (uint32_t)t.xfer | (op << 31);
                     if (MODE == 0) {
                         ++c_ready;
-                        if (op) { atomicAdd(&st_np[d.die], 1u); atomicAdd(&st_bp[d.die], (unsigned long long)t.cb); }
-                        else    { atomicAdd(&st_nr[d.die], 1u); atomicAdd(&st_br[d.die], (unsigned long long)t.cb); }
+                        // charged bytes < 2^33: add the low word, carry into the high word when it wraps
+                        const uint32_t lo = (uint32_t)t.cb, hi = (uint32_t)((uint64_t)t.cb >> 32);
+                        uint32_t *plo = op ? st_bp_lo : st_br_lo, *phi = op ? st_bp_hi : st_br_hi;
+                        atomicAdd(op ? &st_np[d.die] : &st_nr[d.die], 1u);
+                        const uint32_t old = atomicAdd(&plo[d.die], lo);
+                        const uint32_t carry = hi + ((old + lo) < old ? 1u : 0u);
+                        if (carry) atomicAdd(&phi[d.die], carry);
                     }
                 } else if (st == HBF_ST_NATIVE) {
                     S[j] = issue;                            // apply: completion = issue, stall = 0
@@ -282,8 +287,10 @@ k_inorder(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_record
         for (uint32_t r = tid; r < R; r += kInThreads) out[r] = make_longlong2(aggS[r], aggM[r]);
         for (uint32_t d = tid; d < n_dies; d += kInThreads) {
             unsigned long long *g = reinterpret_cast<unsigned long long *>(stats_stage + d);
-            if (st_br[d]) atomicAdd(&g[1], st_br[d]);
-            if (st_bp[d]) atomicAdd(&g[2], st_bp[d]);
+            const unsigned long long br = ((unsigned long long)st_br_hi[d] << 32) | st_br_lo[d];
+            const unsigned long long bp = ((unsigned long long)st_bp_hi[d] << 32) | st_bp_lo[d];
+            if (br) atomicAdd(&g[1], br);
+            if (bp) atomicAdd(&g[2], bp);
             if (st_nr[d]) atomicAdd(&g[4], (unsigned long long)st_nr[d]);
             if (st_np[d]) atomicAdd(&g[5], (unsigned long long)st_np[d]);
         }
@@ -309,7 +316,8 @@ k_inorder(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_record
 }
 
 // scan over tiles, one thread per queue; also decides what happens to the batch
-constexpr int kInScanThreads = 128;
+constexpr int kInScanThreads = 32;
+constexpr int kInScanDepth = 16;
 
 __global__ void __launch_bounds__(kInScanThreads)
 k_inorder_scan(BatchCtrl *ctrl, const ModelParams *__restrict__ mp, uint32_t n_tiles, const int64_t *__restrict__ in_agg,
@@ -334,12 +342,12 @@ k_inorder_scan(BatchCtrl *ctrl, const ModelParams *__restrict__ mp, uint32_t n_t
         int64_t B = busy[r];
         const longlong2 *a = reinterpret_cast<const longlong2 *>(in_agg) + r;
         uint32_t t = 0;
-        for (; t + 8 <= n_tiles; t += 8) {
-            longlong2 v[8];
+        for (; t + kInScanDepth <= n_tiles; t += kInScanDepth) {
+            longlong2 v[kInScanDepth];
 #pragma unroll
-            for (int k = 0; k < 8; ++k) v[k] = a[(uint64_t)(t + k) * R];
+            for (int k = 0; k < kInScanDepth; ++k) v[k] = a[(uint64_t)(t + k) * R];
 #pragma unroll
-            for (int k = 0; k < 8; ++k) { in_bin[(uint64_t)(t + k) * R + r] = B; B = max((int64_t)(B + v[k].x), (int64_t)v[k].y); tot += v[k].x; }
+            for (int k = 0; k < kInScanDepth; ++k) { in_bin[(uint64_t)(t + k) * R + r] = B; B = max((int64_t)(B + v[k].x), (int64_t)v[k].y); tot += v[k].x; }
         }
         for (; t < n_tiles; ++t) {
             const longlong2 v = a[(uint64_t)t * R];

@@ -227,10 +227,14 @@ k_sort_pass(int pass, uint64_t n, BatchCtrl *ctrl, DevState *state, const uint32
     uint32_t *desc_next = (pass & 1) ? desc0 : desc1;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
+    const uint32_t n_tiles = (uint32_t)((n + kSortTile - 1) / kSortTile);
+  for (;;) {                                  // persistent: tiles are taken in order from a counter
+    __syncthreads();                          // shared memory of the previous tile is no longer read
     if (tid == 0) s_tile = atomicAdd(&ctrl->tile_counter[pass], 1u);
     for (int i = tid; i < kSortWarps * kRadix; i += kSortThreads) s_cnt[i] = 0u;
     __syncthreads();
     const uint32_t tile = s_tile;
+    if (tile >= n_tiles) break;
     const uint64_t base = (uint64_t)tile * kSortTile;
     if (tid < kRadix) desc_next[(uint64_t)tile * kRadix + tid] = 0u;     // ready for the pass after this one
 
@@ -319,6 +323,7 @@ k_sort_pass(int pass, uint64_t n, BatchCtrl *ctrl, DevState *state, const uint32
         const uint32_t g = (uint32_t)i + s_delta[d];
         kout[g] = k; iout[g] = s_idx[i];
     }
+  }
 }
 
 // =====================================================================================================
@@ -361,17 +366,19 @@ k_scan(const hbf_access_t *__restrict__ acc, uint64_t n, const RangeSnap *__rest
     if (ctrl->skip || !ctrl->run_sort) return;
     const uint64_t m = ctrl->n_ready;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    if (tid == 0) s_tile = atomicAdd(&ctrl->tile_counter[kMaxPasses], 1u);
     for (int i = tid; i < (int)(sizeof(RangeSnap) / 4); i += kScanThreads)
         reinterpret_cast<uint32_t *>(&rs)[i] = reinterpret_cast<const uint32_t *>(ranges_g)[i];
     for (int i = tid; i < (int)(sizeof(ModelParams) / 4); i += kScanThreads)
         reinterpret_cast<uint32_t *>(&mp)[i] = reinterpret_cast<const uint32_t *>(mp_g)[i];
+  for (;;) {                                  // persistent: tiles are taken in order from a counter
+    __syncthreads();
+    if (tid == 0) s_tile = atomicAdd(&ctrl->tile_counter[kMaxPasses], 1u);
     if (tid < 6) s_die_acc[tid] = 0;
     if (tid < 3) s_res[tid] = tid == 2 ? INT64_MIN : 0;
     __syncthreads();
     const uint32_t tile = s_tile;
     const uint64_t base = (uint64_t)tile * kScanTile;
-    if (base >= m) return;
+    if (base >= m) break;
     const uint32_t np = ctrl->plan.n_passes;
     const uint64_t *keys = (np & 1u) ? keys1 : keys0;
     const uint32_t *idxs = np == 0u ? nullptr : ((np & 1u) ? idx1 : idx0);
@@ -584,6 +591,7 @@ k_scan(const hbf_access_t *__restrict__ acc, uint64_t n, const RangeSnap *__rest
             atomicMax(&ctrl->max_completion_ns, s_res[2]);
         }
     }
+  }
 }
 
 // =====================================================================================================
@@ -685,11 +693,12 @@ static cudaError_t launch_sort_path(const SubmitArgs &a, cudaStream_t st) {
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
+    const unsigned sort_grid = (unsigned)std::min<uint64_t>(sort_tiles, (uint64_t)a.sm_count * 3);
     for (int p = 0; p < kMaxPasses; ++p)
-        k_sort_pass<<<(unsigned)sort_tiles, kSortThreads, kSortSmem, st>>>(p, n, a.ctrl, a.state, a.ws.hist, a.ws.keys[0], a.ws.keys[1],
+        k_sort_pass<<<sort_grid, kSortThreads, kSortSmem, st>>>(p, n, a.ctrl, a.state, a.ws.hist, a.ws.keys[0], a.ws.keys[1],
                                                                            a.ws.idx[0], a.ws.idx[1], a.ws.sort_desc[0], a.ws.sort_desc[1]);
     mark(4);
-    k_scan<<<(unsigned)scan_tiles, kScanThreads, 0, st>>>(a.acc, n, a.ranges, a.mp_dev, a.ctrl, a.state, a.ws.keys[0], a.ws.keys[1],
+    k_scan<<<(unsigned)std::min<uint64_t>(scan_tiles, (uint64_t)a.sm_count * 8), kScanThreads, 0, st>>>(a.acc, n, a.ranges, a.mp_dev, a.ctrl, a.state, a.ws.keys[0], a.ws.keys[1],
                                                          a.ws.idx[0], a.ws.idx[1], (ScanDesc *)a.ws.scan_desc, a.busy,
                                                          a.busy_stage, a.stats_stage, a.completion, a.stall);
     g_kernel_launches += 4 + kMaxPasses;
