@@ -8,8 +8,12 @@
 //   apply   every tile re-reads its records and, starting from its entering busy-until vector, serves them
 //           chunk by chunk; completions and stalls leave through shared memory in batch order.
 // Every global access is coalesced (records in, results out); nothing waits on another thread block.
-// Inside a chunk the per-queue order is recovered with a stable shared-memory radix sort of
-// (queue, position) words and a segmented max-plus scan.
+//
+// Inside a 2,048-record chunk the records are bucketed by queue in shared memory (one atomic per
+// record for its slot, an exclusive scan of the per-queue counts for the bucket starts) and thread t
+// serves queues t, t+256, ... one access after the other, keeping those queues' state in registers.
+// A bucket is put in index order by a selection pass when it is short (the common case: a chunk holds
+// about one access per queue); a chunk with a long bucket is bucketed by a stable radix sort instead.
 #include <algorithm>
 
 #include "device_utils.cuh"
@@ -20,25 +24,21 @@ constexpr int kInThreads = 256;
 constexpr int kInItems = 8;
 constexpr int kInChunk = kInThreads * kInItems;          // 2048 records
 constexpr int kInWarps = kInThreads / 32;
-constexpr int kInPosBits = 11;                           // position inside the chunk
+constexpr int kInQPT = kInMaxQueues / kInThreads;        // queues owned by one thread (8)
 constexpr int kInDigitBits = 6;
 constexpr int kInBins = 1 << kInDigitBits;
-constexpr int kInWorkBytes = kInChunk * 28;              // S 8 + M 8 + xfer/op 4 + two key buffers 2*4
-static_assert(kInWorkBytes >= kInChunk * 24, "the raw records are staged in the work region");
-
-struct InMap { int64_t S, M; int f; };
-__device__ __forceinline__ InMap in_compose(const InMap &x, const InMap &y) {     // x earlier, y later
-    if (y.f) return y;
-    InMap r; r.f = x.f; r.S = x.S + y.S; r.M = max(x.M + y.S, y.M); return r;
-}
-__device__ __forceinline__ InMap in_shfl_up(const InMap &m, int o) {
-    InMap r; r.S = __shfl_up_sync(0xffffffffu, m.S, o); r.M = __shfl_up_sync(0xffffffffu, m.M, o);
-    r.f = __shfl_up_sync(0xffffffffu, m.f, o); return r;
-}
+constexpr int kInMaxBucket = 16;                         // longer buckets take the radix route
+constexpr uint32_t kInNoQueue = 0xffffu;                 // record is not modeled (native or refused)
+// dynamic shared memory: the 24-byte record slots (reused in place), the per-queue counts / bucket
+// starts, two position buffers, and (reduce only) the per-die byte and access counters
+constexpr int kInSlotBytes = kInChunk * 24;
+constexpr int kInCntBytes = (kInMaxQueues + 64) * 4;
+constexpr int kInPosBytes = kInChunk * 2;
+constexpr int kInWorkBytes = kInSlotBytes + kInCntBytes + 2 * kInPosBytes;
 
 // MODE 0 = reduce, MODE 1 = apply
 template <int MODE>
-__global__ void __launch_bounds__(kInThreads, 2)
+__global__ void __launch_bounds__(kInThreads, MODE == 1 ? 3 : 2)
 k_inorder(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_records, const RangeSnap *__restrict__ ranges_g,
           const ModelParams *__restrict__ mp_g, BatchCtrl *ctrl, uint8_t *__restrict__ status, int64_t *__restrict__ in_agg,
           const int64_t *__restrict__ in_bin, hbf_die_stats_t *stats_stage, int64_t *__restrict__ completion,
@@ -46,10 +46,10 @@ k_inorder(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_record
     extern __shared__ __align__(16) unsigned char in_smem[];
     __shared__ RangeSnap rs;
     __shared__ ModelParams mp;
-    __shared__ uint32_t s_cnt[kInWarps * kInBins];
+    __shared__ uint32_t s_cnt[kInWarps * kInBins];        // radix route only
     __shared__ uint32_t s_bin_start[kInBins];
     __shared__ uint32_t s_bin_warp[2];
-    __shared__ InMap s_warp_map[kInWarps];
+    __shared__ uint32_t s_warp_tot[kInWarps];
     __shared__ long long s_red[2];
 
     if (ctrl->skip) return;
@@ -61,34 +61,34 @@ k_inorder(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_record
         reinterpret_cast<uint32_t *>(&mp)[i] = reinterpret_cast<const uint32_t *>(mp_g)[i];
     const uint32_t R = mp_g->n_queues, n_dies = mp_g->n_dies;
 
-    // shared-memory carve-up
-    uint64_t *raw = reinterpret_cast<uint64_t *>(in_smem);                        // [chunk*3], dead after the terms are in registers
-    int64_t *sS = reinterpret_cast<int64_t *>(in_smem);                           // [chunk]  service; later the completion
-    int64_t *sM = sS + kInChunk;                                                   // [chunk]  arrival + service; later the stall
-    uint32_t *sX = reinterpret_cast<uint32_t *>(sM + kInChunk);                    // [chunk]  transfer ns | op << 31
-    uint32_t *keyA = sX + kInChunk, *keyB = keyA + kInChunk;                       // [chunk] each
-    unsigned char *fixed = in_smem + kInWorkBytes;
-    int64_t *aggS = reinterpret_cast<int64_t *>(fixed);                            // reduce: [R] ; apply: busy-until [R]
-    int64_t *aggM = aggS + R;                                                      // reduce only
-    // reduce only, per die: charged bytes as low/high 32-bit halves (native 32-bit shared atomics), access counts
-    uint32_t *st_br_lo = reinterpret_cast<uint32_t *>(aggM + R), *st_br_hi = st_br_lo + n_dies;
+    // slot e holds record e on arrival; then word0 = service (later: completion), word1 = arrival + service
+    // (later: stall), word2 = transfer ns | op << 31 | queue << 32 | slot-in-bucket << 48
+    uint64_t *slot = reinterpret_cast<uint64_t *>(in_smem);
+    uint32_t *qcnt = reinterpret_cast<uint32_t *>(in_smem + kInSlotBytes);             // [R + 1] counts, then starts
+    uint16_t *posA = reinterpret_cast<uint16_t *>(in_smem + kInSlotBytes + kInCntBytes);
+    uint16_t *posB = posA + kInChunk;
+    uint32_t *st_br_lo = reinterpret_cast<uint32_t *>(in_smem + kInWorkBytes), *st_br_hi = st_br_lo + n_dies;   // reduce only
     uint32_t *st_bp_lo = st_br_hi + n_dies, *st_bp_hi = st_bp_lo + n_dies;
     uint32_t *st_nr = st_bp_hi + n_dies, *st_np = st_nr + n_dies;
 
     const uint32_t tile = blockIdx.x;
     const uint64_t tile_begin = (uint64_t)tile * tile_records;
     const uint64_t tile_end = min(n, tile_begin + tile_records);
-    if (MODE == 0) {
-        for (uint32_t r = tid; r < R; r += kInThreads) { aggS[r] = 0; aggM[r] = kNegInf; }
-        for (uint32_t d = tid; d < n_dies * 6u; d += kInThreads) st_br_lo[d] = 0u;
-    } else {
-        for (uint32_t r = tid; r < R; r += kInThreads) aggS[r] = in_bin[(uint64_t)tile * R + r];
+
+    // state of the queues this thread owns (t, t+256, ...): reduce: aggregate (S, M); apply: busy-until in qM
+    int64_t qS[kInQPT], qM[kInQPT];
+#pragma unroll
+    for (int b = 0; b < kInQPT; ++b) {
+        const uint32_t q = (uint32_t)b * kInThreads + tid;
+        qS[b] = 0; qM[b] = kNegInf;
+        if (MODE == 1 && q < R) qM[b] = in_bin[(uint64_t)tile * R + q];
     }
+    if (MODE == 0) for (uint32_t d = tid; d < n_dies * 6u; d += kInThreads) st_br_lo[d] = 0u;
     if (tid < 2) s_red[tid] = tid == 1 ? INT64_MIN : 0;
 
-    // radix plan of the chunk sort: queue ids 0..R (R marks records that are not modeled)
     const uint32_t qbits = 32u - (uint32_t)__clz((int)R);
     const uint32_t n_pass = (qbits + kInDigitBits - 1) / kInDigitBits;
+    const uint32_t bins_per_thread = (R + kInThreads - 1) / kInThreads;
     const int64_t q_ppm = ctrl->q_ppm;
     const Div64 div_q = ctrl->div_q;
     const bool aligned16 = (reinterpret_cast<uintptr_t>(acc) & 15u) == 0;
@@ -99,47 +99,53 @@ k_inorder(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_record
 
     for (uint64_t cbase = tile_begin; cbase < tile_end; cbase += kInChunk) {
         const int cnt = (int)min((uint64_t)kInChunk, tile_end - cbase);
-        __syncthreads();                                   // the work region is free again
-        // ---- load: 16-byte coalesced loads of the 24-byte records ---------------------------------
+        __syncthreads();                                   // the previous chunk has left shared memory
+        // ---- load: 16-byte coalesced loads of the 24-byte records; clear the per-queue counts ----------
         const uint64_t *src = reinterpret_cast<const uint64_t *>(acc + cbase);
         if (cnt == kInChunk && aligned16) {
             const uint4 *s4 = reinterpret_cast<const uint4 *>(src);
-            uint4 *d4 = reinterpret_cast<uint4 *>(raw);
+            uint4 *d4 = reinterpret_cast<uint4 *>(slot);
 #pragma unroll
             for (int k = 0; k < kInChunk * 24 / 16 / kInThreads; ++k) d4[tid + k * kInThreads] = __ldg(s4 + tid + k * kInThreads);
         } else {
-            for (int i = tid; i < cnt * 3; i += kInThreads) raw[i] = __ldg(src + i);
+            for (int i = tid; i < cnt * 3; i += kInThreads) slot[i] = __ldg(src + i);
         }
+        for (uint32_t q = tid; q <= R; q += kInThreads) qcnt[q] = 0u;
         __syncthreads();
-        // ---- terms: classify, decode, service; warp-striped so that memory order = (item, lane) order ----
-        uint32_t key[kInItems], xo[kInItems];
-        int64_t S[kInItems], M[kInItems];
+        if (MODE == 0) {                                   // issue order, checked before the slots are reused
+#pragma unroll
+            for (int j = 0; j < kInItems; ++j) {
+                const int e = j * kInThreads + tid;
+                if (e < cnt) {
+                    const int64_t issue = (int64_t)slot[e * 3 + 1];
+                    const int64_t prev = e > 0 ? (int64_t)slot[e * 3 - 2] : (cbase > 0 ? acc[cbase - 1].issue_ns : INT64_MIN);
+                    c_unsorted |= issue < prev ? 1u : 0u;
+                }
+            }
+            __syncthreads();
+        }
+        // ---- terms, in place: classify, decode, service; take a slot in the queue's bucket ----------------
 #pragma unroll
         for (int j = 0; j < kInItems; ++j) {
-            const int e = warp * (32 * kInItems) + j * 32 + lane;
-            key[j] = (R << kInPosBits) | (uint32_t)e; xo[j] = 0u; S[j] = 0; M[j] = 0;
+            const int e = j * kInThreads + tid;
             if (e < cnt) {
-                const uint64_t addr = raw[e * 3];
-                const int64_t issue = (int64_t)raw[e * 3 + 1];
-                const uint64_t bf = raw[e * 3 + 2];
+                const uint64_t addr = slot[e * 3];
+                const int64_t issue = (int64_t)slot[e * 3 + 1];
+                const uint64_t bf = slot[e * 3 + 2];
                 const uint32_t bytes = (uint32_t)bf, flags = (uint32_t)(bf >> 32);
                 int g = 0;
                 const int st = classify(rs, addr, issue, bytes, flags, &g);
-                if (MODE == 0) {
-                    int64_t prev;
-                    if (e > 0) prev = (int64_t)raw[e * 3 - 2];
-                    else prev = cbase > 0 ? acc[cbase - 1].issue_ns : INT64_MIN;
-                    c_unsorted |= issue < prev ? 1u : 0u;
-                    if (status) status[cbase + e] = (uint8_t)st;
-                }
+                if (MODE == 0 && status) status[cbase + e] = (uint8_t)st;
+                uint64_t w0 = 0, w1 = 0, w2 = (uint64_t)kInNoQueue << 32;
                 if (st == HBF_ST_READY) {
                     const uint64_t off = rs.media_offset[g] + (addr - rs.base[g]);
                     const Decoded d = decode(mp, off, bytes);
                     const uint32_t op = flags & 1u;
                     const Terms t = service_terms(mp, bytes, d.npages, op, q_ppm, div_q);
-                    key[j] = (d.queue << kInPosBits) | (uint32_t)e;
-                    S[j] = t.s; M[j] = issue + (op ? t.xfer : 0) + t.s;
-                    xo[j] = (uint32_t)t.xfer | (op << 31);
+                    const uint32_t o = atomicAdd(&qcnt[d.queue], 1u);
+                    w0 = (uint64_t)t.s;
+                    w1 = (uint64_t)(issue + (op ? t.xfer : 0) + t.s);
+                    w2 = (uint64_t)((uint32_t)t.xfer | (op << 31)) | ((uint64_t)d.queue << 32) | ((uint64_t)o << 48);
                     if (MODE == 0) {
                         ++c_ready;
                         // charged bytes < 2^33: add the low word, carry into the high word when it wraps
@@ -151,140 +157,165 @@ k_inorder(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_record
                         if (carry) atomicAdd(&phi[d.die], carry);
                     }
                 } else if (st == HBF_ST_NATIVE) {
-                    S[j] = issue;                            // apply: completion = issue, stall = 0
+                    w0 = (uint64_t)issue;                    // apply: completion = issue, stall = 0
                     if (MODE == 0) ++c_native;
                 } else if (MODE == 0) {
                     ++c_fault;
                 }
+                slot[e * 3] = w0; slot[e * 3 + 1] = w1; slot[e * 3 + 2] = w2;
             }
         }
-        __syncthreads();                                   // every raw record has been read
-#pragma unroll
-        for (int j = 0; j < kInItems; ++j) {
-            const int e = warp * (32 * kInItems) + j * 32 + lane;
-            sS[e] = S[j]; sM[e] = M[j]; sX[e] = xo[j];
-        }
-        // ---- stable radix sort of (queue, position) words by queue -----------------------------------
-        uint32_t shift = kInPosBits;
-        for (uint32_t p = 0; p < n_pass; ++p) {
-            const uint32_t width = qbits / n_pass + (p < qbits % n_pass ? 1u : 0u);
-            const uint32_t dmask = (1u << width) - 1u;
-            uint32_t *dst = (p & 1u) ? keyB : keyA;
-            const uint32_t *srcb = (p & 1u) ? keyA : keyB;
-            for (int i = tid; i < kInWarps * kInBins; i += kInThreads) s_cnt[i] = 0u;
-            if (p > 0) {
-#pragma unroll
-                for (int j = 0; j < kInItems; ++j) key[j] = srcb[warp * (32 * kInItems) + j * 32 + lane];
-            }
-            __syncthreads();
-            uint32_t rank[kInItems];
-            uint32_t *wcnt = s_cnt + warp * kInBins;
-#pragma unroll
-            for (int j = 0; j < kInItems; ++j) {
-                const uint32_t d = (key[j] >> shift) & dmask;
-                const unsigned peers = __match_any_sync(0xffffffffu, d);
-                const uint32_t before = wcnt[d];
-                rank[j] = before + (uint32_t)__popc(peers & lanemask_lt());
-                __syncwarp();
-                if ((peers >> lane) <= 1u) wcnt[d] = before + (uint32_t)__popc(peers);
-                __syncwarp();
-            }
-            __syncthreads();
-            if (tid < kInBins) {                            // per bin: exclusive over warps, then exclusive over bins
-                uint32_t run = 0;
-#pragma unroll
-                for (int w = 0; w < kInWarps; ++w) { const uint32_t c = s_cnt[w * kInBins + tid]; s_cnt[w * kInBins + tid] = run; run += c; }
-                uint32_t incl = run;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += t; }
-                if (lane == 31) s_bin_warp[warp] = incl;
-                s_bin_start[tid] = incl - run;
-            }
-            __syncthreads();
-#pragma unroll
-            for (int j = 0; j < kInItems; ++j) {
-                const uint32_t d = (key[j] >> shift) & dmask;
-                const uint32_t pos = s_bin_start[d] + (d >= 32u ? s_bin_warp[0] : 0u) + wcnt[d] + rank[j];
-                dst[pos] = key[j];
-            }
-            shift += width;
-            __syncthreads();
-        }
-        const uint32_t *sorted = (n_pass & 1u) ? keyA : keyB;
-        // ---- segmented max-plus scan over the sorted order (blocked: 8 consecutive positions per thread) ----
-        uint32_t sk[kInItems];
-        {
-            const uint4 *k4 = reinterpret_cast<const uint4 *>(sorted + tid * kInItems);
-            const uint4 a = k4[0], b = k4[1];
-            sk[0] = a.x; sk[1] = a.y; sk[2] = a.z; sk[3] = a.w; sk[4] = b.x; sk[5] = b.y; sk[6] = b.z; sk[7] = b.w;
-        }
-        const uint32_t prev_q = tid > 0 ? (sorted[tid * kInItems - 1] >> kInPosBits) : 0xffffffffu;
-        const uint32_t next_q = tid < kInThreads - 1 ? (sorted[(tid + 1) * kInItems] >> kInPosBits) : 0xffffffffu;
-        InMap tm; tm.f = 0; tm.S = 0; tm.M = kNegInf;
-        {
-            uint32_t pq = prev_q;
-#pragma unroll
-            for (int j = 0; j < kInItems; ++j) {
-                const uint32_t q = sk[j] >> kInPosBits, e = sk[j] & (kInChunk - 1);
-                S[j] = 0; M[j] = kNegInf;
-                if (q < R) {
-                    S[j] = sS[e]; M[j] = sM[e];
-                    InMap el; el.S = S[j]; el.f = q != pq;
-                    if (MODE == 1 && el.f) M[j] = max(aggS[q] + S[j], M[j]);      // head: enter with the queue's busy-until
-                    el.M = M[j];
-                    tm = in_compose(tm, el);
-                }
-                pq = q;
-            }
-        }
-        InMap incl = tm;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) { const InMap up = in_shfl_up(incl, o); if (lane >= o) incl = in_compose(up, incl); }
-        if (lane == 31) s_warp_map[warp] = incl;
         __syncthreads();
-        InMap cur; cur.f = 0; cur.S = 0; cur.M = kNegInf;
-        for (int w = 0; w < warp; ++w) cur = in_compose(cur, s_warp_map[w]);
+        // ---- bucket starts: exclusive scan of the counts in queue order; qcnt[R] = modeled records ---------
+        uint32_t longest = 0;
         {
-            InMap ex = in_shfl_up(incl, 1);
-            if (lane == 0) { ex.f = 0; ex.S = 0; ex.M = kNegInf; }
-            cur = in_compose(cur, ex);
+            const uint32_t q0 = (uint32_t)tid * bins_per_thread;
+            uint32_t c[kInQPT], tot = 0;
+            if (bins_per_thread == (uint32_t)kInQPT) {     // full width: two 16-byte loads, free of bank conflicts
+                const uint4 lo = *reinterpret_cast<const uint4 *>(qcnt + q0), hi = *reinterpret_cast<const uint4 *>(qcnt + q0 + 4);
+                c[0] = lo.x; c[1] = lo.y; c[2] = lo.z; c[3] = lo.w; c[4] = hi.x; c[5] = hi.y; c[6] = hi.z; c[7] = hi.w;
+            } else {
+#pragma unroll
+                for (int b = 0; b < kInQPT; ++b) c[b] = ((uint32_t)b < bins_per_thread && q0 + b < R) ? qcnt[q0 + b] : 0u;
+            }
+#pragma unroll
+            for (int b = 0; b < kInQPT; ++b) {
+                longest = max(longest, c[b]);
+                const uint32_t t = c[b]; c[b] = tot; tot += t;
+            }
+            uint32_t incl = tot;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += t; }
+            if (lane == 31) s_warp_tot[warp] = incl;
+            const int use_radix = __syncthreads_or(longest > (uint32_t)kInMaxBucket);
+            uint32_t woff = 0;
+            for (int w = 0; w < warp; ++w) woff += s_warp_tot[w];
+            const uint32_t base = woff + incl - tot;
+            if (bins_per_thread == (uint32_t)kInQPT) {
+                *reinterpret_cast<uint4 *>(qcnt + q0) = make_uint4(base + c[0], base + c[1], base + c[2], base + c[3]);
+                *reinterpret_cast<uint4 *>(qcnt + q0 + 4) = make_uint4(base + c[4], base + c[5], base + c[6], base + c[7]);
+            } else {
+#pragma unroll
+                for (int b = 0; b < kInQPT; ++b)
+                    if ((uint32_t)b < bins_per_thread && q0 + b < R) qcnt[q0 + b] = base + c[b];
+            }
+            if (tid == kInThreads - 1) qcnt[R] = base + tot;
+            longest = (uint32_t)use_radix;
         }
-        {
-            uint32_t pq = prev_q;
+        const uint16_t *pos;
+        if (!longest) {
+            // ---- short buckets: every record goes to the slot it took; order inside a bucket is fixed later ----
+            __syncthreads();
 #pragma unroll
             for (int j = 0; j < kInItems; ++j) {
-                const uint32_t q = sk[j] >> kInPosBits, e = sk[j] & (kInChunk - 1);
-                if (q < R) {
-                    InMap el; el.S = S[j]; el.M = M[j]; el.f = q != pq;
-                    cur = in_compose(cur, el);
-                    const uint32_t nq = j + 1 < kInItems ? (sk[j + 1] >> kInPosBits) : next_q;
-                    if (MODE == 1) {
-                        const uint32_t x = sX[e];
+                const int e = j * kInThreads + tid;
+                if (e < cnt) {
+                    const uint64_t w2 = slot[e * 3 + 2];
+                    const uint32_t q = (uint32_t)(w2 >> 32) & 0xffffu;
+                    if (q != kInNoQueue) posA[qcnt[q] + (uint32_t)(w2 >> 48)] = (uint16_t)e;
+                }
+            }
+            pos = posA;
+        } else {
+            // ---- a long bucket: stable radix sort of the positions by queue (6-bit digits, warp ranking) ----
+            uint32_t shift = 0;
+            for (uint32_t p = 0; p < n_pass; ++p) {
+                const uint32_t width = qbits / n_pass + (p < qbits % n_pass ? 1u : 0u);
+                const uint32_t dmask = (1u << width) - 1u;
+                uint16_t *dst = (p & 1u) ? posB : posA;
+                const uint16_t *srcp = (p & 1u) ? posA : posB;
+                for (int i = tid; i < kInWarps * kInBins; i += kInThreads) s_cnt[i] = 0u;
+                uint32_t e_[kInItems], dig[kInItems], rank[kInItems];
+                __syncthreads();
+#pragma unroll
+                for (int j = 0; j < kInItems; ++j) {
+                    const int i = warp * (32 * kInItems) + j * 32 + lane;       // memory order = (item, lane) order
+                    e_[j] = p == 0 ? (uint32_t)i : (uint32_t)srcp[i];
+                    uint32_t q = R;                                                // not modeled: behind every queue
+                    if ((int)e_[j] < cnt) { const uint32_t qq = (uint32_t)(slot[e_[j] * 3 + 2] >> 32) & 0xffffu; if (qq != kInNoQueue) q = qq; }
+                    dig[j] = (q >> shift) & dmask;
+                }
+                uint32_t *wcnt = s_cnt + warp * kInBins;
+#pragma unroll
+                for (int j = 0; j < kInItems; ++j) {
+                    const unsigned peers = __match_any_sync(0xffffffffu, dig[j]);
+                    const uint32_t before = wcnt[dig[j]];
+                    rank[j] = before + (uint32_t)__popc(peers & lanemask_lt());
+                    __syncwarp();
+                    if ((peers >> lane) <= 1u) wcnt[dig[j]] = before + (uint32_t)__popc(peers);
+                    __syncwarp();
+                }
+                __syncthreads();
+                if (tid < kInBins) {
+                    uint32_t run = 0;
+#pragma unroll
+                    for (int w = 0; w < kInWarps; ++w) { const uint32_t c = s_cnt[w * kInBins + tid]; s_cnt[w * kInBins + tid] = run; run += c; }
+                    uint32_t incl = run;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += t; }
+                    if (lane == 31) s_bin_warp[warp] = incl;
+                    s_bin_start[tid] = incl - run;
+                }
+                __syncthreads();
+#pragma unroll
+                for (int j = 0; j < kInItems; ++j) {
+                    const uint32_t d = dig[j];
+                    dst[s_bin_start[d] + (d >= 32u ? s_bin_warp[0] : 0u) + wcnt[d] + rank[j]] = (uint16_t)e_[j];
+                }
+                shift += width;
+                __syncthreads();                           // the warp counters are cleared again by the next pass
+            }
+            pos = (n_pass & 1u) ? posA : posB;
+        }
+        __syncthreads();
+        // ---- serve: thread t walks the buckets of queues t, t+256, ... in index order -------------------------
+#pragma unroll
+        for (int b = 0; b < kInQPT; ++b) {
+            const uint32_t q = (uint32_t)b * kInThreads + tid;
+            if (q < R) {
+                const uint32_t st0 = qcnt[q], c = qcnt[q + 1] - st0;
+                int last = -1;
+                for (uint32_t k = 0; k < c; ++k) {
+                    int e;
+                    if (longest) {
+                        e = pos[st0 + k];                   // already in index order
+                    } else {                                // next position above the last one served
+                        e = 0x7fffffff;
+                        for (uint32_t i = 0; i < c; ++i) { const int p = pos[st0 + i]; if (p > last && p < e) e = p; }
+                        last = e;
+                    }
+                    const int64_t s = (int64_t)slot[e * 3], m = (int64_t)slot[e * 3 + 1];
+                    if (MODE == 0) {
+                        qM[b] = max(qM[b] + s, m); qS[b] += s;               // aggregate o access
+                    } else {
+                        const uint32_t x = (uint32_t)slot[e * 3 + 2];
                         const int64_t xfer = (int64_t)(x & 0x7fffffffu);
                         const bool op = (x >> 31) != 0u;
-                        const int64_t c = cur.M + (op ? 0 : xfer);
-                        const int64_t issue = sM[e] - S[j] - (op ? xfer : 0);
-                        sS[e] = c; sM[e] = c - issue;
-                        sum_stall += c - issue; max_c = max(max_c, (long long)c);
-                        if (nq != q) aggS[q] = cur.M;                               // last access of the queue in this chunk
-                    } else if (nq != q) {
-                        aggM[q] = max(aggM[q] + cur.S, cur.M); aggS[q] += cur.S;    // queue aggregate o chunk segment
+                        const int64_t B = max(qM[b] + s, m);                 // busy-until after this access
+                        qM[b] = B;
+                        const int64_t done = B + (op ? 0 : xfer);
+                        const int64_t wait = done - (m - s - (op ? xfer : 0));
+                        slot[e * 3] = (uint64_t)done; slot[e * 3 + 1] = (uint64_t)wait;
+                        sum_stall += wait; max_c = max(max_c, (long long)done);
                     }
                 }
-                pq = q;
             }
         }
         // ---- results leave in batch order ---------------------------------------------------------------
         if (MODE == 1) {
             __syncthreads();
-            for (int e = tid; e < cnt; e += kInThreads) { completion[cbase + e] = sS[e]; stall[cbase + e] = sM[e]; }
+            for (int e = tid; e < cnt; e += kInThreads) { completion[cbase + e] = (int64_t)slot[e * 3]; stall[cbase + e] = (int64_t)slot[e * 3 + 1]; }
         }
     }
 
-    __syncthreads();
     if (MODE == 0) {
         longlong2 *out = reinterpret_cast<longlong2 *>(in_agg) + (uint64_t)tile * R;
-        for (uint32_t r = tid; r < R; r += kInThreads) out[r] = make_longlong2(aggS[r], aggM[r]);
+#pragma unroll
+        for (int b = 0; b < kInQPT; ++b) {
+            const uint32_t q = (uint32_t)b * kInThreads + tid;
+            if (q < R) out[q] = make_longlong2(qS[b], qM[b]);
+        }
+        __syncthreads();
         for (uint32_t d = tid; d < n_dies; d += kInThreads) {
             unsigned long long *g = reinterpret_cast<unsigned long long *>(stats_stage + d);
             const unsigned long long br = ((unsigned long long)st_br_hi[d] << 32) | st_br_lo[d];
@@ -323,7 +354,6 @@ __global__ void __launch_bounds__(kInScanThreads)
 k_inorder_scan(BatchCtrl *ctrl, const ModelParams *__restrict__ mp, uint32_t n_tiles, const int64_t *__restrict__ in_agg,
                int64_t *__restrict__ in_bin, const int64_t *__restrict__ busy, int64_t *busy_stage,
                hbf_die_stats_t *stats_stage, int forced) {
-    __shared__ long long s_tot;
     if (ctrl->skip) return;
     const bool fault = ctrl->n_fault != 0, unsorted = ctrl->unsorted != 0u;
     if (blockIdx.x == 0 && threadIdx.x == 0) {
@@ -333,8 +363,6 @@ k_inorder_scan(BatchCtrl *ctrl, const ModelParams *__restrict__ mp, uint32_t n_t
         else ctrl->inorder_used = 1u;
     }
     if (fault || unsorted) return;
-    if (threadIdx.x == 0) s_tot = 0;
-    __syncthreads();
     const uint32_t R = mp->n_queues;
     const uint32_t r = blockIdx.x * kInScanThreads + threadIdx.x;
     long long tot = 0;
@@ -347,7 +375,9 @@ k_inorder_scan(BatchCtrl *ctrl, const ModelParams *__restrict__ mp, uint32_t n_t
 #pragma unroll
             for (int k = 0; k < kInScanDepth; ++k) v[k] = a[(uint64_t)(t + k) * R];
 #pragma unroll
-            for (int k = 0; k < kInScanDepth; ++k) { in_bin[(uint64_t)(t + k) * R + r] = B; B = max((int64_t)(B + v[k].x), (int64_t)v[k].y); tot += v[k].x; }
+            for (int k = 0; k < kInScanDepth; ++k) {
+                in_bin[(uint64_t)(t + k) * R + r] = B; B = max((int64_t)(B + v[k].x), (int64_t)v[k].y); tot += v[k].x;
+            }
         }
         for (; t < n_tiles; ++t) {
             const longlong2 v = a[(uint64_t)t * R];
@@ -358,9 +388,7 @@ k_inorder_scan(BatchCtrl *ctrl, const ModelParams *__restrict__ mp, uint32_t n_t
         if (tot) atomicAdd(reinterpret_cast<unsigned long long *>(&stats_stage[die].busy_ns), (unsigned long long)tot);
     }
     tot = warp_sum(tot);
-    if ((threadIdx.x & 31) == 0 && tot) atomicAdd((unsigned long long *)&s_tot, (unsigned long long)tot);
-    __syncthreads();
-    if (threadIdx.x == 0 && s_tot) atomicAdd((unsigned long long *)&ctrl->service_ns, (unsigned long long)s_tot);
+    if (threadIdx.x == 0 && tot) atomicAdd((unsigned long long *)&ctrl->service_ns, (unsigned long long)tot);
 }
 
 uint64_t inorder_tile_records(uint64_t n, int sm_count) {
@@ -375,8 +403,8 @@ cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st) {
     const uint64_t tile_records = inorder_tile_records(n, a.sm_count);
     const unsigned n_tiles = (unsigned)((n + tile_records - 1) / tile_records);
     const uint32_t R = a.mp.n_queues, nd = a.mp.n_dies;
-    const size_t smem_reduce = (size_t)kInWorkBytes + (size_t)R * 16 + (size_t)nd * 24;
-    const size_t smem_apply = (size_t)kInWorkBytes + (size_t)R * 8;
+    const size_t smem_reduce = (size_t)kInWorkBytes + (size_t)nd * 24;
+    const size_t smem_apply = (size_t)kInWorkBytes;
     static size_t set_reduce = 0, set_apply = 0;
     if (smem_reduce > set_reduce) {
         cudaError_t e = cudaFuncSetAttribute(k_inorder<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_reduce);
