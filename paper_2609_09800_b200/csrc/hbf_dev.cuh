@@ -84,6 +84,8 @@ struct Workspace {
     void *scan_desc;                     // [scan tiles] ScanDesc
     int64_t *in_agg;                     // [tiles][queues][2]: per-tile, per-queue max-plus aggregate (S, M)
     int64_t *in_bin;                     // [tiles][queues]: busy-until entering each tile
+    uint64_t *in_img;                    // [n][3]: served image of every record (in-order path)
+    uint16_t *in_start;                  // per 2,048-record chunk: first queue-major position of each thread's queues
     size_t bytes;
 };
 
@@ -104,6 +106,7 @@ constexpr uint32_t kInMaxTiles = 1024;
 size_t workspace_layout(uint64_t n, uint32_t n_queues, Workspace *ws, void *base);
 // tile size (records) of the in-order path for a batch of n on a device with sm_count SMs
 uint64_t inorder_tile_records(uint64_t n, int sm_count);
+size_t inorder_start_bytes(uint64_t n);
 cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st);
 cudaError_t launch_submit(const SubmitArgs &a, cudaStream_t st);
 cudaError_t launch_queue_order(const BatchCtrl *ctrl, const Workspace &ws, uint32_t *out, uint64_t n, cudaStream_t st);
