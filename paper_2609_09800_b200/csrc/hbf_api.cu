@@ -156,7 +156,7 @@ int hbf_create(const hbf_config_t *cfg, void *cuda_stream, hbf_ctx **out) {
     {   // the in-order path packs the transfer time of an access into 31 bits and keeps per-queue state in shared memory
         const unsigned __int128 worst = ((unsigned __int128)0xffffffffull + std::max(cfg->read_granule, cfg->prog_granule)) * 1000u;
         c->inorder_ok = nq <= kInMaxQueues && worst / cfg->chan_bytes_per_us < ((unsigned __int128)1 << 31) &&
-                        66u * 1024u + nd * 24u <= 200u * 1024u;
+                        100u * 1024u + nd * 24u <= 220u * 1024u;
     }
     DevState st0; st0.mode = HBF_MODE_NORMAL; st0.poisoned = 0; st0.q_ppm = 1000000;
     if ((rc = dev_copy(c, &c->d_ranges, nullptr, 1))) return fail(rc);

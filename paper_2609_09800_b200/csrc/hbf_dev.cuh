@@ -84,8 +84,12 @@ struct Workspace {
     void *scan_desc;                     // [scan tiles] ScanDesc
     int64_t *in_agg;                     // [tiles][queues][2]: per-tile, per-queue max-plus aggregate (S, M)
     int64_t *in_bin;                     // [tiles][queues]: busy-until entering each tile
-    uint64_t *in_img;                    // [n][3]: served image of every record (in-order path)
-    uint16_t *in_start;                  // per 2,048-record chunk: first queue-major position of each thread's queues
+    uint16_t *in_pos;                    // [n]: per 2,048-record chunk, the positions of its modeled records in queue-major order
+    uint16_t *in_start;                  // per chunk: [queues + 1] first queue-major position of every queue
+    void *in_tile;                       // [tiles] stall bookkeeping of the in-order path
+    void *in_head;                       // [tiles][queues][8]: the first accesses of every (tile, queue), for the fix-up
+    uint8_t *in_headcnt;                 // [tiles][queues]: how many of them exist
+    uint32_t *in_list;                   // [1 + tiles*queues]: count, then the (tile, queue) pairs the long fix-up handles
     size_t bytes;
 };
 
@@ -102,11 +106,12 @@ constexpr int kProfEvents = 10;
 extern unsigned long long g_kernel_launches;
 
 constexpr uint32_t kInMaxQueues = 2048;  // the in-order path keeps per-queue state in shared memory
-constexpr uint32_t kInMaxTiles = 1024;
+constexpr uint32_t kInMaxTiles = 512;
 size_t workspace_layout(uint64_t n, uint32_t n_queues, Workspace *ws, void *base);
 // tile size (records) of the in-order path for a batch of n on a device with sm_count SMs
 uint64_t inorder_tile_records(uint64_t n, int sm_count);
-size_t inorder_start_bytes(uint64_t n);
+size_t inorder_start_bytes(uint64_t n, uint32_t n_queues);
+size_t inorder_head_bytes(uint64_t tiles, uint32_t n_queues);
 cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st);
 cudaError_t launch_submit(const SubmitArgs &a, cudaStream_t st);
 cudaError_t launch_queue_order(const BatchCtrl *ctrl, const Workspace &ws, uint32_t *out, uint64_t n, cudaStream_t st);

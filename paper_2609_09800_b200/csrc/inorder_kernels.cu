@@ -1,16 +1,20 @@
 // In-order path of hbf_submit_batch: serves a batch whose records arrive in non-decreasing issue order
 // without a global sort.  In such a batch the (issue, index) order of every queue is plain index order,
-// so the batch can be cut into a few hundred contiguous tiles and handled as reduce - scan - apply over
-// vectors of per-queue max-plus maps:
-//   reduce  every tile classifies and decodes its records, writes status[], counts, sums per-die bytes,
-//           and composes, per queue, the maps B -> max(B + s, a + s) of its accesses in index order into
-//           one aggregate (S, M).  It also leaves a 24-byte "served image" of every record in the
-//           workspace: service, arrival + service, transfer time, queue and the record's place in its
-//           chunk's queue-major order, so that the apply pass repeats none of this work;
-//   scan    one thread per queue walks the tiles in order: busy-until entering each tile, final busy-until;
-//   apply   every tile reads its images and, starting from its entering busy-until vector, serves them
-//           chunk by chunk; completions and stalls leave through shared memory in batch order.
-// Every global access is coalesced; nothing waits on another thread block.
+// so the batch is cut into a few hundred contiguous tiles that are served independently, in one pass:
+//   serve   every tile classifies and decodes its records, writes status[], counts, sums per-die bytes, and
+//           serves its accesses AS IF every queue were idle when the tile begins; completions and stalls
+//           leave through shared memory in batch order.  Per queue it also keeps the composition (S, M) of
+//           the maps B -> max(B + s, a + s) of its accesses (M is exactly the busy-until of the as-if run),
+//           and per 2,048-record chunk it leaves the queue-major order of the chunk in the workspace;
+//   scan    one thread per queue walks the tiles' aggregates in order: the true busy-until entering each
+//           tile, and the final busy-until;
+//   fix-up  one thread per (tile, queue) starts from the true entering busy-until and re-serves that queue's
+//           accesses of the tile in order, until it meets an access that arrives when the queue is idle:
+//           from there on the as-if run and the true run coincide (busy-until is monotone in its start
+//           value, so the as-if run was idle there too).  At moderate load this touches a few accesses
+//           per (tile, queue); under overload it degrades to re-serving everything, still exactly.
+// The serve pass is the only one that streams the batch: 24 B read and 16 B + 1 B written per access, plus
+// 4 B of order information.  Every global access of it is coalesced; nothing waits on another thread block.
 //
 // Inside a 2,048-record chunk the records are bucketed by queue in shared memory: one atomic per record
 // takes a slot in its queue's bucket, an exclusive scan of the per-queue counts gives the bucket starts,
@@ -29,29 +33,59 @@ constexpr int kInChunk = kInThreads * kInItems;          // 2048 records
 constexpr int kInWarps = kInThreads / 32;
 constexpr int kInDigitBits = 6;
 constexpr int kInBins = 1 << kInDigitBits;
+constexpr int kInGroup = 4;                              // accesses a thread loads at once while serving
 constexpr int kInMaxBucket = 16;                         // longer buckets take the radix route
 constexpr uint32_t kInNoQueue = 0xffffu;                 // record is not modeled (native or refused)
 constexpr int kInSlotBytes = kInChunk * 24;
 constexpr int kInCntBytes = (kInMaxQueues + 64) * 4;
 constexpr int kInPosBytes = kInChunk * 2;
-constexpr int kInStartRow = kInThreads + 8;              // u16 per chunk: first sorted position of each thread's queues, + end
+constexpr int kInStartRow = kInThreads + 8;              // shared: first queue-major position of each thread's queues, + end
 
-// word 2 of a served image: transfer ns (31 bits) | op << 31 | queue << 32 | place in the chunk's queue-major order << 48
+// word 2 of a slot: transfer ns (31 bits) | op << 31 | queue << 32 | slot taken in the queue's bucket << 48
 __device__ __forceinline__ uint32_t img_queue(uint64_t w2) { return (uint32_t)(w2 >> 32) & 0xffffu; }
 __device__ __forceinline__ uint32_t img_place(uint64_t w2) { return (uint32_t)(w2 >> 48); }
+
+// One access, from its record: status, and for a modeled access its queue, die and service terms.
+struct Served { int st; uint32_t queue, die, op; int64_t s, xfer, cb; };
+__device__ __forceinline__ Served serve_terms(const RangeSnap &rs, const ModelParams &mp, uint64_t addr, int64_t issue,
+                                              uint64_t bf, int64_t q_ppm, const Div64 &div_q) {
+    Served r; r.queue = 0; r.die = 0; r.op = 0; r.s = 0; r.xfer = 0; r.cb = 0;
+    const uint32_t bytes = (uint32_t)bf, flags = (uint32_t)(bf >> 32);
+    int g = 0;
+    r.st = classify(rs, addr, issue, bytes, flags, &g);
+    if (r.st == HBF_ST_READY) {
+        const uint64_t off = rs.media_offset[g] + (addr - rs.base[g]);
+        const Decoded d = decode(mp, off, bytes);
+        r.op = flags & 1u;
+        const Terms t = service_terms(mp, bytes, d.npages, r.op, q_ppm, div_q);
+        r.queue = d.queue; r.die = d.die; r.s = t.s; r.xfer = t.xfer; r.cb = t.cb;
+    }
+    return r;
+}
 
 // state arrays are laid out so that thread t's queues sit in different banks than thread t+1's
 __device__ __forceinline__ uint32_t state_index(uint32_t q, uint32_t qpt_shift) {
     return ((q & ((1u << qpt_shift) - 1u)) << 8) | (q >> qpt_shift);
 }
 
+// per-tile bookkeeping of the stall total: as-if-idle sum, fix-up corrections, and the exact sum of a re-served tile
+struct InTile { long long spec_sum, fix_delta, true_sum; uint32_t reserve; uint32_t stragglers; };
+// The first kInHead accesses of every (tile, queue), as the serve pass saw them: all the fix-up needs in the common case.
+constexpr int kInHead = 8;
+struct InHead { int64_t m, s; uint32_t xo, idx; };       // arrival + service, service, transfer | op << 31, batch index
+
 // ======================================================================================================
-// reduce
+// serve.  RESERVE = false: the streaming pass over every tile, every queue taken as idle at the tile's start.
+// RESERVE = true: only for tiles the fix-up flagged (a queue stayed backlogged far into the tile): the same
+// pass from the true entering busy-until, writing the exact results and nothing else.
 // ======================================================================================================
+template <bool RESERVE>
 __global__ void __launch_bounds__(kInThreads, 2)
-k_inorder_reduce(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_records, const RangeSnap *__restrict__ ranges_g,
-                 const ModelParams *__restrict__ mp_g, BatchCtrl *ctrl, uint8_t *__restrict__ status, int64_t *__restrict__ in_agg,
-                 uint64_t *__restrict__ in_img, uint16_t *__restrict__ in_start, hbf_die_stats_t *stats_stage) {
+k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_records, const RangeSnap *__restrict__ ranges_g,
+                const ModelParams *__restrict__ mp_g, BatchCtrl *ctrl, uint8_t *__restrict__ status, int64_t *__restrict__ in_agg,
+                uint16_t *__restrict__ in_pos, uint16_t *__restrict__ in_start, uint32_t row_stride,
+                hbf_die_stats_t *stats_stage, int64_t *__restrict__ completion, int64_t *__restrict__ stall,
+                const int64_t *__restrict__ in_bin, InTile *in_tile, InHead *__restrict__ in_head, uint8_t *__restrict__ in_headcnt) {
     extern __shared__ __align__(16) unsigned char in_smem[];
     __shared__ ModelParams mp;
     __shared__ uint32_t s_cnt[kInWarps * kInBins];        // radix route only
@@ -59,8 +93,10 @@ k_inorder_reduce(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile
     __shared__ uint32_t s_bin_warp[2];
     __shared__ uint32_t s_warp_tot[kInWarps];
     __shared__ uint16_t s_tstart[kInStartRow];
+    __shared__ long long s_red[2];
 
     if (ctrl->skip) return;
+    if (RESERVE && (ctrl->run_sort || !ctrl->inorder_used || !in_tile[blockIdx.x].reserve)) return;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const RangeSnap &rs = *ranges_g;                      // read through the cache: shared memory is needed elsewhere
     for (int i = tid; i < (int)(sizeof(ModelParams) / 4); i += kInThreads)
@@ -77,6 +113,8 @@ k_inorder_reduce(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile
     uint32_t *st_br_lo = reinterpret_cast<uint32_t *>(aggM + kInMaxQueues), *st_br_hi = st_br_lo + n_dies;   // per die
     uint32_t *st_bp_lo = st_br_hi + n_dies, *st_bp_hi = st_bp_lo + n_dies;
     uint32_t *st_nr = st_bp_hi + n_dies, *st_np = st_nr + n_dies;
+    // head-table fill count per queue, one nibble each; the two nibbles of a byte belong to the same thread
+    uint8_t *hfill = reinterpret_cast<uint8_t *>(st_np + n_dies);
 
     const uint32_t tile = blockIdx.x;
     const uint64_t tile_begin = (uint64_t)tile * tile_records;
@@ -88,7 +126,13 @@ k_inorder_reduce(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile
     const uint32_t qpt = 1u << qpt_shift;
 
     for (uint32_t i = tid; i < kInMaxQueues; i += kInThreads) { aggS[i] = 0; aggM[i] = kNegInf; }
-    for (uint32_t d = tid; d < n_dies * 6u; d += kInThreads) st_br_lo[d] = 0u;
+    if (RESERVE) {
+        __syncthreads();
+        for (uint32_t q = tid; q < R; q += kInThreads) aggM[state_index(q, qpt_shift)] = in_bin[(uint64_t)blockIdx.x * R + q];
+    } else {
+        for (uint32_t d = tid; d < n_dies * 6u; d += kInThreads) st_br_lo[d] = 0u;
+        for (uint32_t i = tid; i < kInMaxQueues / 2; i += kInThreads) hfill[i] = 0;
+    }
 
     const uint32_t qbits = 32u - (uint32_t)__clz((int)R);
     const uint32_t n_pass = (qbits + kInDigitBits - 1) / kInDigitBits;
@@ -98,6 +142,11 @@ k_inorder_reduce(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile
 
     unsigned long long c_native = 0, c_ready = 0, c_fault = 0;
     unsigned c_unsorted = 0;
+    long long sum_stall = 0, max_c = INT64_MIN;
+    bool heads_open = !RESERVE;                           // this thread still fills head entries of its queues
+    uint32_t heads_full = 0;
+    const uint32_t owned_queues = min(qpt, R > (uint32_t)tid * qpt ? R - (uint32_t)tid * qpt : 0u);
+    if (tid < 2) s_red[tid] = tid == 1 ? INT64_MIN : 0;
 
     for (uint64_t cbase = tile_begin; cbase < tile_end; cbase += kInChunk) {
         const int cnt = (int)min((uint64_t)kInChunk, tile_end - cbase);
@@ -121,7 +170,7 @@ k_inorder_reduce(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile
             if (e < cnt) {
                 const int64_t issue = (int64_t)slot[e * 3 + 1];
                 const int64_t prev = e > 0 ? (int64_t)slot[e * 3 - 2] : (cbase > 0 ? acc[cbase - 1].issue_ns : INT64_MIN);
-                c_unsorted |= issue < prev ? 1u : 0u;
+                if (!RESERVE) c_unsorted |= issue < prev ? 1u : 0u;
             }
         }
         __syncthreads();
@@ -132,31 +181,26 @@ k_inorder_reduce(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile
             if (e < cnt) {
                 const uint64_t addr = slot[e * 3];
                 const int64_t issue = (int64_t)slot[e * 3 + 1];
-                const uint64_t bf = slot[e * 3 + 2];
-                const uint32_t bytes = (uint32_t)bf, flags = (uint32_t)(bf >> 32);
-                int g = 0;
-                const int st = classify(rs, addr, issue, bytes, flags, &g);
-                if (status) status[cbase + e] = (uint8_t)st;
+                const Served v = serve_terms(rs, mp, addr, issue, slot[e * 3 + 2], q_ppm, div_q);
+                if (!RESERVE && status) status[cbase + e] = (uint8_t)v.st;
                 uint64_t w0 = 0, w1 = 0, w2 = (uint64_t)kInNoQueue << 32;
-                if (st == HBF_ST_READY) {
-                    const uint64_t off = rs.media_offset[g] + (addr - rs.base[g]);
-                    const Decoded d = decode(mp, off, bytes);
-                    const uint32_t op = flags & 1u;
-                    const Terms t = service_terms(mp, bytes, d.npages, op, q_ppm, div_q);
-                    const uint32_t o = atomicAdd(&qcnt[d.queue], 1u);
-                    w0 = (uint64_t)t.s;
-                    w1 = (uint64_t)(issue + (op ? t.xfer : 0) + t.s);
-                    w2 = (uint64_t)((uint32_t)t.xfer | (op << 31)) | ((uint64_t)d.queue << 32) | ((uint64_t)o << 48);
-                    ++c_ready;
-                    // charged bytes < 2^33: add the low word, carry into the high word when it wraps
-                    const uint32_t lo = (uint32_t)t.cb, hi = (uint32_t)((uint64_t)t.cb >> 32);
-                    uint32_t *plo = op ? st_bp_lo : st_br_lo, *phi = op ? st_bp_hi : st_br_hi;
-                    atomicAdd(op ? &st_np[d.die] : &st_nr[d.die], 1u);
-                    const uint32_t old = atomicAdd(&plo[d.die], lo);
-                    const uint32_t carry = hi + ((old + lo) < old ? 1u : 0u);
-                    if (carry) atomicAdd(&phi[d.die], carry);
-                } else if (st == HBF_ST_NATIVE) {
-                    w0 = (uint64_t)issue;                    // apply: completion = issue, stall = 0
+                if (v.st == HBF_ST_READY) {
+                    const uint32_t o = atomicAdd(&qcnt[v.queue], 1u);
+                    w0 = (uint64_t)v.s;
+                    w1 = (uint64_t)(issue + (v.op ? v.xfer : 0) + v.s);
+                    w2 = (uint64_t)((uint32_t)v.xfer | (v.op << 31)) | ((uint64_t)v.queue << 32) | ((uint64_t)o << 48);
+                    if (!RESERVE) {
+                        ++c_ready;
+                        // charged bytes < 2^33: add the low word, carry into the high word when it wraps
+                        const uint32_t lo = (uint32_t)v.cb, hi = (uint32_t)((uint64_t)v.cb >> 32);
+                        uint32_t *plo = v.op ? st_bp_lo : st_br_lo, *phi = v.op ? st_bp_hi : st_br_hi;
+                        atomicAdd(v.op ? &st_np[v.die] : &st_nr[v.die], 1u);
+                        const uint32_t old = atomicAdd(&plo[v.die], lo);
+                        const uint32_t carry = hi + ((old + lo) < old ? 1u : 0u);
+                        if (carry) atomicAdd(&phi[v.die], carry);
+                    }
+                } else if (v.st == HBF_ST_NATIVE) {
+                    w0 = (uint64_t)issue;                    // native: completion = issue, stall = 0
                     ++c_native;
                 } else {
                     ++c_fault;
@@ -224,10 +268,9 @@ k_inorder_reduce(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile
                     if (q != kInNoQueue) {
                         const uint32_t st0 = qcnt[q], c = qcnt[q + 1] - st0;
                         uint32_t rank = 0;
-                        for (uint32_t i = 0; i < c; ++i) rank += (uint32_t)posA[st0 + i] < (uint32_t)e ? 1u : 0u;
-                        const uint32_t p = st0 + rank;
-                        posB[p] = (uint16_t)e;
-                        slot[e * 3 + 2] = (w2 & 0x0000ffffffffffffull) | ((uint64_t)p << 48);
+                        if (c > 1u)
+                            for (uint32_t i = 0; i < c; ++i) rank += (uint32_t)posA[st0 + i] < (uint32_t)e ? 1u : 0u;
+                        posB[st0 + rank] = (uint16_t)e;
                     }
                 }
             }
@@ -281,51 +324,89 @@ k_inorder_reduce(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile
                 shift += width;
                 __syncthreads();                           // the warp counters are cleared again by the next pass
             }
-            const uint32_t modeled = qcnt[R];
-            for (uint32_t k = tid; k < modeled; k += kInThreads) {
-                const uint32_t e = posB[k];
-                slot[e * 3 + 2] = (slot[e * 3 + 2] & 0x0000ffffffffffffull) | ((uint64_t)k << 48);
-            }
         }
         __syncthreads();
-        // ---- aggregate: thread t walks its queues' accesses, which are consecutive in queue-major order --------
+        // ---- serve: thread t walks its queues' accesses, which are consecutive in queue-major order --------
+        // (four at a time: the loads of a group are independent, only the max-plus chain is serial).
+        // M is the aggregate's constant term and, at the same time, the busy-until of the as-if-idle run.
         {
             const uint32_t k0 = s_tstart[tid], k1 = s_tstart[tid + 1];
-            uint32_t cur = kInNoQueue, ci = 0;
+            uint32_t cur = kInNoQueue, ci = 0, hf = 0;
             int64_t S = 0, M = kNegInf;
-            for (uint32_t k = k0; k < k1; ++k) {
-                const uint32_t e = posB[k];
-                const int64_t s = (int64_t)slot[e * 3], m = (int64_t)slot[e * 3 + 1];
-                const uint32_t q = img_queue(slot[e * 3 + 2]);
-                if (q != cur) {
-                    if (cur != kInNoQueue) { aggS[ci] = S; aggM[ci] = M; }
-                    cur = q; ci = state_index(q, qpt_shift); S = aggS[ci]; M = aggM[ci];
+            auto close_queue = [&]() {
+                aggS[ci] = S; aggM[ci] = M;
+                if (!RESERVE && heads_open) {
+                    uint8_t *hb = hfill + (((ci >> 9) << 8) | (ci & 255u));
+                    const uint32_t old = ((ci >> 8) & 1u) ? (uint32_t)(*hb >> 4) : (uint32_t)(*hb & 0x0fu);
+                    *hb = ((ci >> 8) & 1u) ? (uint8_t)((*hb & 0x0fu) | (hf << 4)) : (uint8_t)((*hb & 0xf0u) | hf);
+                    if (old < (uint32_t)kInHead && hf == (uint32_t)kInHead) ++heads_full;
                 }
-                M = max(M + s, m); S += s;                  // aggregate o access
+            };
+            for (uint32_t k = k0; k < k1; k += kInGroup) {
+                uint32_t e[kInGroup], qi[kInGroup];
+                int64_t s_[kInGroup], m_[kInGroup], aS[kInGroup], aM[kInGroup];
+                uint64_t w2[kInGroup];
+#pragma unroll
+                for (int j = 0; j < kInGroup; ++j) e[j] = k + j < k1 ? (uint32_t)posB[k + j] : 0u;
+#pragma unroll
+                for (int j = 0; j < kInGroup; ++j) {
+                    s_[j] = (int64_t)slot[e[j] * 3]; m_[j] = (int64_t)slot[e[j] * 3 + 1]; w2[j] = slot[e[j] * 3 + 2];
+                }
+#pragma unroll
+                for (int j = 0; j < kInGroup; ++j) {
+                    qi[j] = state_index(img_queue(w2[j]) & (kInMaxQueues - 1), qpt_shift);
+                    aS[j] = aggS[qi[j]]; aM[j] = aggM[qi[j]];       // used only if this access opens its queue here
+                }
+#pragma unroll
+                for (int j = 0; j < kInGroup; ++j) {
+                    if (k + j < k1) {
+                        const uint32_t q = img_queue(w2[j]);
+                        if (q != cur) {
+                            if (cur != kInNoQueue) close_queue();
+                            cur = q; ci = qi[j]; S = aS[j]; M = aM[j];
+                            if (!RESERVE && heads_open) {
+                                const uint8_t hb = hfill[((ci >> 9) << 8) | (ci & 255u)];
+                                hf = ((ci >> 8) & 1u) ? (uint32_t)(hb >> 4) : (uint32_t)(hb & 0x0fu);
+                            }
+                        }
+                        if (!RESERVE && heads_open && hf < (uint32_t)kInHead) {    // among the first accesses of this queue in the tile
+                            InHead h; h.m = m_[j]; h.s = s_[j]; h.xo = (uint32_t)w2[j]; h.idx = (uint32_t)(cbase + e[j]);
+                            in_head[((uint64_t)tile * kInHead + hf) * R + q] = h;
+                            ++hf;
+                        }
+                        M = max(M + s_[j], m_[j]); S += s_[j];      // aggregate o access; M = busy-until after it
+                        const int64_t xfer = (int64_t)((uint32_t)w2[j] & 0x7fffffffu);
+                        const bool op = (((uint32_t)w2[j]) >> 31) != 0u;
+                        const int64_t done = M + (op ? 0 : xfer);
+                        const int64_t wait = done - (m_[j] - s_[j] - (op ? xfer : 0));
+                        slot[e[j] * 3] = (uint64_t)done; slot[e[j] * 3 + 1] = (uint64_t)wait;
+                        sum_stall += wait; max_c = max(max_c, (long long)done);
+                    }
+                }
             }
-            if (cur != kInNoQueue) { aggS[ci] = S; aggM[ci] = M; }
+            if (cur != kInNoQueue) close_queue();
+            if (heads_full >= owned_queues) heads_open = false;          // every queue of this thread has its head entries
         }
         __syncthreads();
-        // ---- the served images and the threads' starts leave for the apply pass ----------------------------
-        {
-            uint64_t *dst = in_img + cbase * 3;
-            if (cnt == kInChunk) {
-                const uint4 *s4 = reinterpret_cast<const uint4 *>(slot);
-                uint4 *d4 = reinterpret_cast<uint4 *>(dst);
-#pragma unroll
-                for (int k = 0; k < kInChunk * 24 / 16 / kInThreads; ++k) d4[tid + k * kInThreads] = s4[tid + k * kInThreads];
-            } else {
-                for (int i = tid; i < cnt * 3; i += kInThreads) dst[i] = slot[i];
-            }
-            uint16_t *row = in_start + (cbase / kInChunk) * kInStartRow;
-            for (int i = tid; i <= kInThreads; i += kInThreads) row[i] = s_tstart[i];
+        // ---- results leave in batch order; the chunk's queue-major order stays behind for the fix-up ----------
+        for (int e = tid; e < cnt; e += kInThreads) { completion[cbase + e] = (int64_t)slot[e * 3]; stall[cbase + e] = (int64_t)slot[e * 3 + 1]; }
+        if (!RESERVE) {
+            const uint32_t modeled = qcnt[R];
+            for (uint32_t k = tid; k < modeled; k += kInThreads) in_pos[cbase + k] = posB[k];
+            uint16_t *row = in_start + (cbase / kInChunk) * row_stride;
+            for (uint32_t q = tid; q <= R; q += kInThreads) row[q] = (uint16_t)qcnt[q];
         }
     }
 
     __syncthreads();
-    {
+    if (!RESERVE) {
         longlong2 *out = reinterpret_cast<longlong2 *>(in_agg) + (uint64_t)tile * R;
-        for (uint32_t q = tid; q < R; q += kInThreads) { const uint32_t i = state_index(q, qpt_shift); out[q] = make_longlong2(aggS[i], aggM[i]); }
+        for (uint32_t q = tid; q < R; q += kInThreads) {
+            const uint32_t i = state_index(q, qpt_shift);
+            out[q] = make_longlong2(aggS[i], aggM[i]);
+            const uint8_t hb = hfill[((i >> 9) << 8) | (i & 255u)];
+            in_headcnt[(uint64_t)tile * R + q] = ((i >> 8) & 1u) ? (uint8_t)(hb >> 4) : (uint8_t)(hb & 0x0fu);
+        }
         for (uint32_t d = tid; d < n_dies; d += kInThreads) {
             unsigned long long *g = reinterpret_cast<unsigned long long *>(stats_stage + d);
             const unsigned long long br = ((unsigned long long)st_br_hi[d] << 32) | st_br_lo[d];
@@ -345,6 +426,14 @@ k_inorder_reduce(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile
             if (c_fault) atomicAdd(&ctrl->n_fault, c_fault);
             if (c_unsorted) atomicOr(&ctrl->unsorted, 1u);
         }
+    }
+    sum_stall = warp_sum(sum_stall); max_c = warp_max(max_c);
+    if (lane == 0) { atomicAdd((unsigned long long *)&s_red[0], (unsigned long long)sum_stall); atomicMax(&s_red[1], max_c); }
+    __syncthreads();
+    if (tid == 0) {
+        if (RESERVE) in_tile[tile].true_sum = s_red[0];
+        else { InTile t; t.spec_sum = s_red[0]; t.fix_delta = 0; t.true_sum = 0; t.reserve = 0u; t.stragglers = 0u; in_tile[tile] = t; }
+        atomicMax(&ctrl->max_completion_ns, s_red[1]);
     }
 }
 
@@ -396,125 +485,194 @@ k_inorder_scan(BatchCtrl *ctrl, const ModelParams *__restrict__ mp, uint32_t n_t
 }
 
 // ======================================================================================================
-// apply
+// fix-up: the true run differs from the as-if-idle run only at the head of each (tile, queue)
 // ======================================================================================================
-__global__ void __launch_bounds__(kInThreads, 3)
-k_inorder_apply(uint64_t n, uint64_t tile_records, uint32_t R, BatchCtrl *ctrl, const uint64_t *__restrict__ in_img,
-                const uint16_t *__restrict__ in_start, const int64_t *__restrict__ in_bin, int64_t *__restrict__ completion,
-                int64_t *__restrict__ stall) {
-    extern __shared__ __align__(16) unsigned char in_smem[];
-    __shared__ uint16_t s_tstart[kInStartRow];
-    __shared__ long long s_red[2];
+constexpr int kInFixThreads = 128;
+
+// Phase 1, one thread per (tile, queue): walk the head table.  A queue that is still backlogged after
+// kInHead accesses is a straggler: it goes on a list for phase 2, or, when a tile has many of them (the
+// batch arrived on queues that were far behind), the whole tile is flagged to be served again.
+__global__ void __launch_bounds__(kInFixThreads)
+k_inorder_fixup(uint32_t R, uint32_t n_tiles, BatchCtrl *ctrl, const int64_t *__restrict__ in_bin,
+                const InHead *__restrict__ in_head, const uint8_t *__restrict__ in_headcnt, int64_t *completion, int64_t *stall,
+                InTile *in_tile, uint32_t *in_list) {
     if (ctrl->skip || ctrl->run_sort || !ctrl->inorder_used) return;
-    const int tid = threadIdx.x, lane = tid & 31;
-    uint64_t *slot = reinterpret_cast<uint64_t *>(in_smem);
-    uint16_t *pos = reinterpret_cast<uint16_t *>(in_smem + kInSlotBytes);
-    int64_t *busy = reinterpret_cast<int64_t *>(in_smem + kInSlotBytes + kInPosBytes);        // [2048], state_index order
-
-    const uint32_t tile = blockIdx.x;
-    const uint64_t tile_begin = (uint64_t)tile * tile_records;
-    const uint64_t tile_end = min(n, tile_begin + tile_records);
-    uint32_t qpt_shift = 0;
-    while (((uint32_t)kInThreads << qpt_shift) < R) ++qpt_shift;
-    for (uint32_t q = tid; q < R; q += kInThreads) busy[state_index(q, qpt_shift)] = in_bin[(uint64_t)tile * R + q];
-    if (tid < 2) s_red[tid] = tid == 1 ? INT64_MIN : 0;
-    long long sum_stall = 0, max_c = INT64_MIN;
-
-    for (uint64_t cbase = tile_begin; cbase < tile_end; cbase += kInChunk) {
-        const int cnt = (int)min((uint64_t)kInChunk, tile_end - cbase);
-        __syncthreads();
-        const uint64_t *src = in_img + cbase * 3;
-        if (cnt == kInChunk) {
-            const uint4 *s4 = reinterpret_cast<const uint4 *>(src);
-            uint4 *d4 = reinterpret_cast<uint4 *>(slot);
-#pragma unroll
-            for (int k = 0; k < kInChunk * 24 / 16 / kInThreads; ++k) d4[tid + k * kInThreads] = __ldg(s4 + tid + k * kInThreads);
-        } else {
-            for (int i = tid; i < cnt * 3; i += kInThreads) slot[i] = __ldg(src + i);
+    const uint64_t idx = (uint64_t)blockIdx.x * kInFixThreads + threadIdx.x;          // tile * R + queue
+    long long max_c = INT64_MIN;
+    if (idx < (uint64_t)n_tiles * R) {
+        const uint32_t tile = (uint32_t)(idx / R);
+        const uint32_t q = (uint32_t)(idx % R);
+        const uint32_t c = in_headcnt[idx];
+        int64_t B = in_bin[idx];                             // true busy-until of the queue entering the tile
+        int64_t Bs = kNegInf;                                // busy-until of the as-if-idle run, to know what it wrote
+        long long dstall = 0;
+        bool settled = false;
+        for (uint32_t k = 0; k < c; ++k) {
+            const InHead h = in_head[((uint64_t)tile * kInHead + k) * R + q];
+            if (B <= h.m - h.s) { settled = true; break; }   // idle on arrival: from here on the as-if run was right
+            B += h.s;                                          // it waited for the queue: starts at B
+            Bs = max(Bs + h.s, h.m);
+            const bool op = (h.xo >> 31) != 0u;
+            const int64_t xfer = (int64_t)(h.xo & 0x7fffffffu);
+            const int64_t done = B + (op ? 0 : xfer);
+            dstall += B - Bs;                                  // completion moved from Bs + post to B + post
+            completion[h.idx] = done; stall[h.idx] = done - (h.m - h.s - (op ? xfer : 0));
+            max_c = max(max_c, (long long)done);
         }
-        const uint16_t *row = in_start + (cbase / kInChunk) * kInStartRow;
-        for (int i = tid; i <= kInThreads; i += kInThreads) s_tstart[i] = row[i];
-        __syncthreads();
-        // positions in queue-major order
-#pragma unroll
-        for (int j = 0; j < kInItems; ++j) {
-            const int e = j * kInThreads + tid;
-            if (e < cnt) {
-                const uint64_t w2 = slot[e * 3 + 2];
-                if (img_queue(w2) != kInNoQueue) pos[img_place(w2)] = (uint16_t)e;
-            }
+        if (dstall) atomicAdd((unsigned long long *)&in_tile[tile].fix_delta, (unsigned long long)dstall);
+        if (!settled && c == (uint32_t)kInHead) {
+            const uint32_t rank = atomicAdd(&in_tile[tile].stragglers, 1u);
+            if (rank >= max(8u, R / 16u)) in_tile[tile].reserve = 1u;
+            else in_list[1 + atomicAdd(&in_list[0], 1u)] = (uint32_t)idx;
         }
-        __syncthreads();
-        // serve: thread t walks the accesses of its queues one after the other
-        {
-            const uint32_t k0 = s_tstart[tid], k1 = s_tstart[tid + 1];
-            uint32_t cur = kInNoQueue, ci = 0;
-            int64_t B = 0;
-            for (uint32_t k = k0; k < k1; ++k) {
-                const uint32_t e = pos[k];
-                const int64_t s = (int64_t)slot[e * 3], m = (int64_t)slot[e * 3 + 1];
-                const uint64_t w2 = slot[e * 3 + 2];
-                const uint32_t q = img_queue(w2);
-                if (q != cur) {
-                    if (cur != kInNoQueue) busy[ci] = B;
-                    cur = q; ci = state_index(q, qpt_shift); B = busy[ci];
-                }
-                const int64_t xfer = (int64_t)((uint32_t)w2 & 0x7fffffffu);
-                const bool op = (((uint32_t)w2) >> 31) != 0u;
-                B = max(B + s, m);                          // busy-until after this access
-                const int64_t done = B + (op ? 0 : xfer);
-                const int64_t wait = done - (m - s - (op ? xfer : 0));
-                slot[e * 3] = (uint64_t)done; slot[e * 3 + 1] = (uint64_t)wait;
-                sum_stall += wait; max_c = max(max_c, (long long)done);
-            }
-            if (cur != kInNoQueue) busy[ci] = B;
-        }
-        __syncthreads();
-        for (int e = tid; e < cnt; e += kInThreads) { completion[cbase + e] = (int64_t)slot[e * 3]; stall[cbase + e] = (int64_t)slot[e * 3 + 1]; }
     }
-    sum_stall = warp_sum(sum_stall); max_c = warp_max(max_c);
-    if (lane == 0) { atomicAdd((unsigned long long *)&s_red[0], (unsigned long long)sum_stall); atomicMax(&s_red[1], max_c); }
+    max_c = warp_max(max_c);
+    if ((threadIdx.x & 31) == 0 && max_c != INT64_MIN) atomicMax(&ctrl->max_completion_ns, max_c);
+}
+
+// Phase 2, one warp per straggler: re-serve the queue's accesses of the tile from the records until an
+// access arrives on an idle queue.  The lanes take 32 consecutive chunks at a time: each composes the
+// maps of the queue's accesses in its chunk, a warp scan over the lanes gives the true busy-until
+// entering every chunk, and each lane then re-serves its chunk.  Past the point where the queue falls
+// idle the re-served values equal what is already there, so lanes need not agree on where to stop.
+constexpr uint32_t kInLongBudget = 4096;                  // accesses re-served for one (tile, queue) before the tile is re-served whole
+
+__global__ void __launch_bounds__(kInFixThreads)
+k_inorder_fixup_long(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_records,
+                     const RangeSnap *__restrict__ ranges_g, const ModelParams *__restrict__ mp_g, BatchCtrl *ctrl,
+                     const int64_t *__restrict__ in_bin, const uint16_t *__restrict__ in_pos, const uint16_t *__restrict__ in_start,
+                     uint32_t row_stride, int64_t *completion, int64_t *stall, InTile *in_tile, const uint32_t *__restrict__ in_list) {
+    __shared__ ModelParams mp;
+    if (ctrl->skip || ctrl->run_sort || !ctrl->inorder_used) return;
+    const RangeSnap &rs = *ranges_g;
+    for (int i = threadIdx.x; i < (int)(sizeof(ModelParams) / 4); i += kInFixThreads)
+        reinterpret_cast<uint32_t *>(&mp)[i] = reinterpret_cast<const uint32_t *>(mp_g)[i];
     __syncthreads();
-    if (tid == 0) {
-        atomicAdd((unsigned long long *)&ctrl->modeled_ns, (unsigned long long)s_red[0]);
-        atomicMax(&ctrl->max_completion_ns, s_red[1]);
+    const uint32_t R = mp.n_queues, count = in_list[0];
+    const int64_t q_ppm = ctrl->q_ppm;
+    const Div64 div_q = ctrl->div_q;
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint32_t warp_global = (blockIdx.x * kInFixThreads + threadIdx.x) >> 5, n_warps = (gridDim.x * kInFixThreads) >> 5;
+    long long max_c = INT64_MIN;
+    for (uint32_t w = warp_global; w < count; w += n_warps) {
+        const uint32_t idx = in_list[1 + w];
+        const uint32_t tile = idx / R, q = idx % R;
+        if (in_tile[tile].reserve) continue;
+        int64_t B = in_bin[idx];                             // true busy-until entering the next group of chunks
+        long long dstall = 0;
+        const uint64_t tile_begin = (uint64_t)tile * tile_records, tile_end = min(n, tile_begin + tile_records);
+        uint32_t served = 0;
+        for (uint64_t gbase = tile_begin; gbase < tile_end; gbase += 32ull * kInChunk) {
+            const uint64_t cbase = gbase + (uint64_t)lane * kInChunk;
+            uint32_t k0 = 0, k1 = 0;
+            if (cbase < tile_end) {
+                const uint16_t *row = in_start + (cbase / kInChunk) * row_stride;
+                k0 = row[q]; k1 = row[q + 1];
+            }
+            // this lane's chunk as one map B -> max(B + S, M)
+            int64_t S = 0, M = kNegInf;
+            for (uint32_t k = k0; k < k1; ++k) {
+                const uint64_t *rec = reinterpret_cast<const uint64_t *>(acc + cbase + in_pos[cbase + k]);
+                const int64_t issue = (int64_t)rec[1];
+                const Served v = serve_terms(rs, mp, rec[0], issue, rec[2], q_ppm, div_q);
+                M = max(M + v.s, issue + (v.op ? v.xfer : 0) + v.s); S += v.s;
+            }
+            // exclusive scan of the maps over the lanes, applied to B
+            int64_t iS = S, iM = M;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int64_t uS = __shfl_up_sync(0xffffffffu, iS, o), uM = __shfl_up_sync(0xffffffffu, iM, o);
+                if ((int)lane >= o) { iM = max(uM + iS, iM); iS += uS; }
+            }
+            int64_t eS = __shfl_up_sync(0xffffffffu, iS, 1), eM = __shfl_up_sync(0xffffffffu, iM, 1);
+            if (lane == 0) { eS = 0; eM = kNegInf; }
+            int64_t Bl = max(B + eS, eM);                    // true busy-until entering this lane's chunk
+            // re-serve the chunk
+            bool idle_seen = false;
+            for (uint32_t k = k0; k < k1; ++k) {
+                const uint64_t i = cbase + in_pos[cbase + k];
+                const uint64_t *rec = reinterpret_cast<const uint64_t *>(acc + i);
+                const int64_t issue = (int64_t)rec[1];
+                const Served v = serve_terms(rs, mp, rec[0], issue, rec[2], q_ppm, div_q);
+                const int64_t a = issue + (v.op ? v.xfer : 0);
+                if (Bl <= a) idle_seen = true;
+                Bl = max(a, Bl) + v.s;
+                const int64_t done = Bl + (v.op ? 0 : v.xfer);
+                const int64_t old = completion[i];
+                if (done != old) { dstall += done - old; completion[i] = done; stall[i] = done - issue; max_c = max(max_c, (long long)done); }
+            }
+            served += __reduce_add_sync(0xffffffffu, k1 - k0);
+            B = max(B + __shfl_sync(0xffffffffu, iS, 31), __shfl_sync(0xffffffffu, iM, 31));
+            if (__any_sync(0xffffffffu, idle_seen)) break;   // the queue fell idle: the rest of the tile was served right
+            if (served > kInLongBudget) { if (lane == 0) in_tile[tile].reserve = 1u; break; }
+        }
+        dstall = warp_sum(dstall);
+        if (lane == 0 && dstall) atomicAdd((unsigned long long *)&in_tile[tile].fix_delta, (unsigned long long)dstall);
     }
+    max_c = warp_max(max_c);
+    if (lane == 0 && max_c != INT64_MIN) atomicMax(&ctrl->max_completion_ns, max_c);
+}
+
+// stall total of the batch: per tile the exact sum if it was re-served, else the as-if sum plus its corrections
+__global__ void k_inorder_total(BatchCtrl *ctrl, const InTile *__restrict__ in_tile, uint32_t n_tiles) {
+    if (ctrl->skip || ctrl->run_sort || !ctrl->inorder_used) return;
+    long long tot = 0;
+    for (uint32_t t = threadIdx.x; t < n_tiles; t += blockDim.x) {
+        const InTile v = in_tile[t];
+        tot += v.reserve ? v.true_sum : v.spec_sum + v.fix_delta;
+    }
+    tot = warp_sum(tot);
+    if ((threadIdx.x & 31) == 0 && tot) atomicAdd((unsigned long long *)&ctrl->modeled_ns, (unsigned long long)tot);
 }
 
 uint64_t inorder_tile_records(uint64_t n, int sm_count) {
-    const uint64_t want_tiles = std::min<uint64_t>(kInMaxTiles, (uint64_t)std::max(1, sm_count) * 4);
+    const uint64_t want_tiles = std::min<uint64_t>(kInMaxTiles, (uint64_t)std::max(1, sm_count) * 2);   // two thread blocks per SM: one wave
     uint64_t t = (n + want_tiles - 1) / want_tiles;
     t = (t + kInChunk - 1) / kInChunk * kInChunk;
     return std::max<uint64_t>(t, kInChunk);
 }
 
-size_t inorder_start_bytes(uint64_t n) { return ((n + kInChunk - 1) / kInChunk + 1) * kInStartRow * sizeof(uint16_t); }
+static uint32_t inorder_row_stride(uint32_t n_queues) { return (n_queues + 1u + 7u) / 8u * 8u; }
+size_t inorder_head_bytes(uint64_t tiles, uint32_t n_queues) { return tiles * n_queues * (size_t)kInHead * sizeof(InHead); }
+size_t inorder_start_bytes(uint64_t n, uint32_t n_queues) {
+    return ((n + kInChunk - 1) / kInChunk + 1) * (size_t)inorder_row_stride(n_queues) * sizeof(uint16_t);
+}
 
 cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st) {
     const uint64_t n = a.n;
     const uint64_t tile_records = inorder_tile_records(n, a.sm_count);
     const unsigned n_tiles = (unsigned)((n + tile_records - 1) / tile_records);
-    const uint32_t R = a.mp.n_queues, nd = a.mp.n_dies;
-    const size_t smem_reduce = (size_t)kInSlotBytes + kInCntBytes + 2 * kInPosBytes + (size_t)kInMaxQueues * 16 + (size_t)nd * 24;
-    const size_t smem_apply = (size_t)kInSlotBytes + kInPosBytes + (size_t)kInMaxQueues * 8;
-    static size_t set_reduce = 0, set_apply = 0;
-    if (smem_reduce > set_reduce) {
-        cudaError_t e = cudaFuncSetAttribute(k_inorder_reduce, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_reduce);
+    const uint32_t R = a.mp.n_queues, nd = a.mp.n_dies, row_stride = inorder_row_stride(R);
+    const size_t smem_serve = (size_t)kInSlotBytes + kInCntBytes + 2 * kInPosBytes + (size_t)kInMaxQueues * 16 + (size_t)nd * 24 +
+                              kInMaxQueues / 2;
+    static size_t set_serve = 0;
+    if (smem_serve > set_serve) {
+        cudaError_t e = cudaFuncSetAttribute(k_inorder_serve<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_serve);
         if (e != cudaSuccess) return e;
-        set_reduce = smem_reduce;
-    }
-    if (smem_apply > set_apply) {
-        cudaError_t e = cudaFuncSetAttribute(k_inorder_apply, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_apply);
+        e = cudaFuncSetAttribute(k_inorder_serve<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_serve);
         if (e != cudaSuccess) return e;
-        set_apply = smem_apply;
+        set_serve = smem_serve;
     }
-    k_inorder_reduce<<<n_tiles, kInThreads, smem_reduce, st>>>(a.acc, n, tile_records, a.ranges, a.mp_dev, a.ctrl, a.status, a.ws.in_agg,
-                                                               a.ws.in_img, a.ws.in_start, a.stats_stage);
+    InTile *tiles = reinterpret_cast<InTile *>(a.ws.in_tile);
+    InHead *heads = reinterpret_cast<InHead *>(a.ws.in_head);
+    cudaError_t em = cudaMemsetAsync(a.ws.in_list, 0, sizeof(uint32_t), st);
+    if (em != cudaSuccess) return em;
+    k_inorder_serve<false><<<n_tiles, kInThreads, smem_serve, st>>>(a.acc, n, tile_records, a.ranges, a.mp_dev, a.ctrl, a.status,
+                                                                    a.ws.in_agg, a.ws.in_pos, a.ws.in_start, row_stride, a.stats_stage,
+                                                                    a.completion, a.stall, a.ws.in_bin, tiles, heads, a.ws.in_headcnt);
     k_inorder_scan<<<(R + kInScanThreads - 1) / kInScanThreads, kInScanThreads, 0, st>>>(
         a.ctrl, a.mp_dev, n_tiles, a.ws.in_agg, a.ws.in_bin, a.busy, a.busy_stage, a.stats_stage, a.path == HBF_PATH_INORDER ? 1 : 0);
-    k_inorder_apply<<<n_tiles, kInThreads, smem_apply, st>>>(n, tile_records, R, a.ctrl, a.ws.in_img, a.ws.in_start, a.ws.in_bin,
-                                                             a.completion, a.stall);
-    g_kernel_launches += 3;
+    const uint64_t fix_threads = (uint64_t)n_tiles * R;
+    k_inorder_fixup<<<(unsigned)((fix_threads + kInFixThreads - 1) / kInFixThreads), kInFixThreads, 0, st>>>(
+        R, n_tiles, a.ctrl, a.ws.in_bin, heads, a.ws.in_headcnt, a.completion, a.stall, tiles, a.ws.in_list);
+    k_inorder_fixup_long<<<(unsigned)std::max(1, a.sm_count * 4), kInFixThreads, 0, st>>>(
+        a.acc, n, tile_records, a.ranges, a.mp_dev, a.ctrl, a.ws.in_bin, a.ws.in_pos, a.ws.in_start, row_stride, a.completion, a.stall,
+        tiles, a.ws.in_list);
+    k_inorder_serve<true><<<n_tiles, kInThreads, smem_serve, st>>>(a.acc, n, tile_records, a.ranges, a.mp_dev, a.ctrl, a.status,
+                                                                   a.ws.in_agg, a.ws.in_pos, a.ws.in_start, row_stride, a.stats_stage,
+                                                                   a.completion, a.stall, a.ws.in_bin, tiles, heads, a.ws.in_headcnt);
+    k_inorder_total<<<1, 256, 0, st>>>(a.ctrl, tiles, n_tiles);
+    g_kernel_launches += 6;
     return cudaGetLastError();
 }
 

@@ -72,10 +72,11 @@ def lib():
     """The loaded CUDA library.  Raises if it has not been built (python -m paper_2609_09800_b200.build)."""
     global _lib
     if _lib is None:
-        if not os.path.exists(_SO):
+        path = os.environ.get("HBF_LIBRARY", _SO)          # an explicitly chosen build of the same library
+        if not os.path.exists(path):
             raise RuntimeError("libhbf.so is missing: build it with `python -m paper_2609_09800_b200.build` "
                                "(nvcc, sm_100a); there is no CPU fallback")
-        L = C.CDLL(_SO)
+        L = C.CDLL(path)
         vp, u64, u32, i64, i32 = C.c_void_p, C.c_uint64, C.c_uint32, C.c_int64, C.c_int32
         L.hbf_create.argtypes = [C.POINTER(hbf_config_t), vp, C.POINTER(vp)]
         L.hbf_destroy.argtypes = [vp]
