@@ -31,7 +31,10 @@ METRIC = "simulated HBF accesses/s"
 UNIT = "accesses/s"
 ALGO_BYTES_PER_ACCESS = 41            # 24 B record in, 8 B completion + 8 B stall + 1 B status out
 # algorithmic bytes per access of each kernel group (what the kernel itself must move)
-STAGE_BYTES = {"classify": 24 + 8 + 1, "plan_hist": 8, "scan": 8 + 4 + 24 + 16, "inorder": 24 + 16 + 1}
+STAGE_BYTES = {"classify": 24 + 8 + 1, "plan_hist": 8, "scan": 8 + 4 + 24 + 16, "inorder": 24 + 16 + 1 + 4}
+# DRAM bytes per access of the in-order serve kernel from one ncu capture (dram__bytes_read + write over a
+# 20 M-access launch, profiles/inorder_path_capacity_20M.md); traffic grows in proportion to the batch
+NCU_TRAFFIC_BYTES_PER_ACCESS = {"inorder": 60.7}
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -62,7 +65,7 @@ def measured_peak():
 
 
 class ClockSampler:
-    """nvidia-smi clocks and throttle reasons, sampled every 200 ms while the timed region runs."""
+    """nvidia-smi clocks and throttle reasons, sampled every 20 ms from the warm-up to the end of the timed region."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -72,7 +75,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.Q,
-                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except Exception:
             self.proc = None
@@ -288,9 +291,10 @@ def main():
         else:
             dom_bytes = STAGE_BYTES[dom]; per_launch_ms = med[dom]
         achieved = dom_bytes * n / (per_launch_ms * 1e-3) / 1e9 if per_launch_ms > 0 else 0.0
+        traffic = NCU_TRAFFIC_BYTES_PER_ACCESS.get(dom)
         roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
-                    "frac": achieved / peak, "traffic": None, "algorithmic_bytes_per_access": dom_bytes,
-                    "ms_per_launch": per_launch_ms}
+                    "frac": achieved / peak, "traffic": traffic * n if traffic else None,
+                    "algorithmic_bytes_per_access": dom_bytes, "ms_per_launch": per_launch_ms}
         path_gbs = ALGO_BYTES_PER_ACCESS * value / world / 1e9
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
                 "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,

@@ -163,31 +163,24 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
         }
         for (uint32_t q = tid; q <= R; q += kInThreads) qcnt[q] = 0u;
         __syncthreads();
-        // ---- issue order, checked before the slots are reused ------------------------------------------
-#pragma unroll
-        for (int j = 0; j < kInItems; ++j) {
-            const int e = j * kInThreads + tid;
-            if (e < cnt) {
-                const int64_t issue = (int64_t)slot[e * 3 + 1];
-                const int64_t prev = e > 0 ? (int64_t)slot[e * 3 - 2] : (cbase > 0 ? acc[cbase - 1].issue_ns : INT64_MIN);
-                if (!RESERVE) c_unsorted |= issue < prev ? 1u : 0u;
-            }
-        }
-        __syncthreads();
-        // ---- terms, in place: classify, decode, service; take a slot in the queue's bucket ----------------
+        // ---- terms, in place: classify, decode, service; take a slot in the queue's bucket.  Word 1 (the issue
+        // time) stays as it is until the queues are served, so the issue-order check can read the neighbour's.
 #pragma unroll
         for (int j = 0; j < kInItems; ++j) {
             const int e = j * kInThreads + tid;
             if (e < cnt) {
                 const uint64_t addr = slot[e * 3];
                 const int64_t issue = (int64_t)slot[e * 3 + 1];
+                if (!RESERVE) {
+                    const int64_t prev = e > 0 ? (int64_t)slot[e * 3 - 2] : (cbase > 0 ? acc[cbase - 1].issue_ns : INT64_MIN);
+                    c_unsorted |= issue < prev ? 1u : 0u;
+                }
                 const Served v = serve_terms(rs, mp, addr, issue, slot[e * 3 + 2], q_ppm, div_q);
                 if (!RESERVE && status) status[cbase + e] = (uint8_t)v.st;
-                uint64_t w0 = 0, w1 = 0, w2 = (uint64_t)kInNoQueue << 32;
+                uint64_t w0 = 0, w2 = (uint64_t)kInNoQueue << 32;
                 if (v.st == HBF_ST_READY) {
                     const uint32_t o = atomicAdd(&qcnt[v.queue], 1u);
                     w0 = (uint64_t)v.s;
-                    w1 = (uint64_t)(issue + (v.op ? v.xfer : 0) + v.s);
                     w2 = (uint64_t)((uint32_t)v.xfer | (v.op << 31)) | ((uint64_t)v.queue << 32) | ((uint64_t)o << 48);
                     if (!RESERVE) {
                         ++c_ready;
@@ -205,7 +198,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
                 } else {
                     ++c_fault;
                 }
-                slot[e * 3] = w0; slot[e * 3 + 1] = w1; slot[e * 3 + 2] = w2;
+                slot[e * 3] = w0; slot[e * 3 + 2] = w2;
             }
         }
         __syncthreads();
@@ -256,6 +249,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
                     const uint64_t w2 = slot[e * 3 + 2];
                     const uint32_t q = img_queue(w2);
                     if (q != kInNoQueue) posA[qcnt[q] + img_place(w2)] = (uint16_t)e;
+                    else slot[e * 3 + 1] = 0;              // native or refused: no stall
                 }
             }
             __syncthreads();
@@ -291,7 +285,10 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
                     const int i = warp * (32 * kInItems) + j * 32 + lane;       // memory order = (item, lane) order
                     e_[j] = p == 0 ? (uint32_t)i : (uint32_t)srcp[i];
                     uint32_t q = R;                                                // not modeled: behind every queue
-                    if ((int)e_[j] < cnt) { const uint32_t qq = img_queue(slot[e_[j] * 3 + 2]); if (qq != kInNoQueue) q = qq; }
+                    if ((int)e_[j] < cnt) {
+                        const uint32_t qq = img_queue(slot[e_[j] * 3 + 2]);
+                        if (qq != kInNoQueue) q = qq; else if (p == 0) slot[e_[j] * 3 + 1] = 0;     // native or refused: no stall
+                    }
                     dig[j] = (q >> shift) & dmask;
                 }
                 uint32_t *wcnt = s_cnt + warp * kInBins;
@@ -351,6 +348,8 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
 #pragma unroll
                 for (int j = 0; j < kInGroup; ++j) {
                     s_[j] = (int64_t)slot[e[j] * 3]; m_[j] = (int64_t)slot[e[j] * 3 + 1]; w2[j] = slot[e[j] * 3 + 2];
+                    // word 1 is the issue time: arrival + service = issue (+ transfer, for a program) + service
+                    m_[j] += s_[j] + ((((uint32_t)w2[j]) >> 31) ? (int64_t)((uint32_t)w2[j] & 0x7fffffffu) : 0);
                 }
 #pragma unroll
                 for (int j = 0; j < kInGroup; ++j) {
