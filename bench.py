@@ -50,6 +50,9 @@ def parse_args():
     ap.add_argument("--cpu-sample", type=int, default=20_000_000)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--workload", default="capacity_mode", choices=["capacity_mode", "coupled_thermal"],
+                    help="coupled_thermal: the prefix-KV stream in 1 ms batches, each followed by a thermal step (not the headline)")
+    ap.add_argument("--horizon-ms", type=int, default=1000, help="simulated time of the coupled_thermal run")
     return ap.parse_args()
 
 
@@ -163,6 +166,55 @@ def run_reference(args, rank: int):
     print(json.dumps(line), flush=True)
 
 
+def run_coupled(args):
+    """Long-run coupled mode on one GPU: 1 ms batches of the prefix-KV stream, a thermal step after each."""
+    import torch
+    from paper_2609_09800_b200 import build as hbf_build, hbf
+    hbf_build.build()
+    t0 = time.time()
+    w = wl.prefix_kv()
+    fp = wl.package_floorplan()
+    batches = [b for _, b in wl.timed_batches(w, args.horizon_ms * 1_000_000)]
+    sizes = [b.shape[0] for b in batches]
+    allrec = np.concatenate(batches)
+    gen_s = time.time() - t0
+    ctx = hbf.Context(w.profile, fp)
+    for r in w.ranges:
+        ctx.register_range(*r)
+    d_all = torch.from_numpy(allrec.view(np.int64).reshape(-1, 3)).cuda()
+    nmax = max(sizes)
+    d_comp = torch.empty(nmax, dtype=torch.int64, device="cuda"); d_stall = torch.empty_like(d_comp)
+    d_stats = torch.empty(ctx.n_dies * 6, dtype=torch.int64, device="cuda")
+    ws = ctx.workspace(nmax)
+    offs = np.concatenate([[0], np.cumsum(sizes)])
+    ext = fp["ext_power_w"]
+
+    def run():
+        for k, nk in enumerate(sizes):
+            rc = ctx.submit_batch(d_all[offs[k]:offs[k + 1]], nk, d_comp, d_stall, None, d_stats, ws)
+            assert rc == 0, rc
+            ctx.thermal_step(1_000_000, ext, None, want_hot=False)
+    ctx.reset(); run(); torch.cuda.synchronize()               # warm-up pass over the same horizon
+    ctx.reset()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    l0 = hbf.kernel_launches()
+    t_host = time.perf_counter()
+    e0.record(); run(); e1.record(); torch.cuda.synchronize()
+    wall = time.perf_counter() - t_host
+    ms = e0.elapsed_time(e1)
+    hot = ctx.thermal_step(1_000_000, ext)
+    mode, q = ctx.get_mode()
+    n_acc = int(offs[-1])
+    line = {"metric": METRIC, "value": n_acc / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": len(sizes), "warmup": len(sizes),
+            "ms_per_step": ms / len(sizes), "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64",
+            "data": "synthetic",
+            "config": {"workload": "coupled_thermal", "accesses": n_acc, "mean_accesses_per_step": n_acc / len(sizes),
+                       "simulated_ms": args.horizon_ms, "geometry": "32x8x4", "thermal_grid": "128x128", "gen_seconds": round(gen_s, 1)},
+            "gpu_launches": int(hbf.kernel_launches() - l0), "host_wall_s": round(wall, 3),
+            "final": {"hot_c": [round(float(x), 3) for x in hot], "mode": mode, "q_ppm": q}}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     args = parse_args()
     rank = int(os.environ.get("RANK", "0"))
@@ -171,10 +223,14 @@ def main():
     if args.impl == "reference":
         run_reference(args, rank)
         return
+    if args.workload == "coupled_thermal":
+        if rank == 0:
+            run_coupled(args)
+        return
 
     import torch
     import torch.distributed as dist
-    from paper_2609_09800_b200 import build as hbf_build, hbf
+    from paper_2609_09800_b200 import build as hbf_build, hbf, replicas
 
     assert torch.cuda.is_available(), "bench.py needs a CUDA device (no CPU fallback)"
     torch.cuda.set_device(local_rank)
@@ -186,7 +242,7 @@ def main():
         dist.barrier()
 
     n = args.n
-    w, gen_s = make_stream(n, seed=rank)               # every rank: an independent replica on its own stream
+    w, gen_s = make_stream(n, seed=replicas.rank_seed(0, rank))   # every rank: an independent replica on its own stream
     fp = wl.package_floorplan(channels=w.profile["channels"], dies=w.profile["dies"])
     ctx = hbf.Context(w.profile, fp)
     for r in w.ranges:
@@ -250,11 +306,8 @@ def main():
     # the same batch replayed on the queues it has just filled: every queue is backlogged from its first access on
     e0.record(stream); step(); e1.record(stream); e1.synchronize()
     replay_ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
-    value = world * n * args.steps / (total_ms * 1e-3)
+    units, total_ms = replicas.combine(n * args.steps, total_ms, device="cuda")     # sum of units, max of device times
+    value = units / (total_ms * 1e-3)
 
     # end to end through the C ABI with host buffers: H2D of the records, submit + thermal step, D2H of results
     e2e = None
@@ -272,11 +325,8 @@ def main():
         ctx.reset(); e2e_step(); sync_all()
         ms = timed(args.e2e_steps, e2e_step)
         sync_all()
-        if world > 1:
-            t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        e2e = {"value": world * n * args.e2e_steps / (ms * 1e-3), "unit": UNIT, "steps": args.e2e_steps,
+        e2e_units, ms = replicas.combine(n * args.e2e_steps, ms, device="cuda")
+        e2e = {"value": e2e_units / (ms * 1e-3), "unit": UNIT, "steps": args.e2e_steps,
                "h2d_bytes_per_step": n * 24, "d2h_bytes_per_step": n * 16 + ctx.n_dies * 48}
 
     if rank == 0:

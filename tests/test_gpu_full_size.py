@@ -1,0 +1,83 @@
+"""Parity at the benchmark's full size: the 200 M-access capacity-mode batch, device-resident, in the launch
+configuration bench.py times.  The oracle cannot serve 200 M accesses in seconds, but queues are independent:
+the sub-stream of one queue, served alone by the oracle, must give exactly the completions the library gave
+those accesses.  A handful of sampled queues are checked that way, element by element, on a fresh batch and
+on a replay (every queue backlogged); totals are checked against closed forms over the whole batch."""
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+from oracle import hbfo
+from paper_2609_09800_b200 import workloads as wl
+
+N_FULL = 200_000_000
+
+
+@pytest.fixture(scope="module")
+def full():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    if torch.cuda.get_device_properties(0).total_memory < 60 * (1 << 30):
+        pytest.skip("needs a large-memory GPU")
+    from paper_2609_09800_b200 import build, hbf
+    build.build()
+    w = wl.capacity_mode(n=N_FULL)
+    u = ((w.acc["addr"] - np.uint64(wl.RANGE_BASE)) >> np.uint64(16)).astype(np.int64)   # 64 KiB stripe units
+    queue = ((u % 64) * 8 + (u // 64) % 8) * 4 + (u // 512) % 4
+    return hbf, w, queue.astype(np.int32)
+
+
+def run_gpu(hbf, ctx, w):
+    import torch
+    n = w.n
+    d_acc = torch.from_numpy(w.acc.view(np.int64).reshape(-1)).cuda()
+    d_comp = torch.empty(n, dtype=torch.int64, device="cuda")
+    d_stall = torch.empty(n, dtype=torch.int64, device="cuda")
+    d_status = torch.empty(n, dtype=torch.uint8, device="cuda")
+    d_ds = torch.empty(ctx.n_dies * 6, dtype=torch.int64, device="cuda")
+    ws = ctx.workspace(n)
+    out = []
+    for _ in range(2):                                     # fresh batch, then the same batch on backlogged queues
+        assert ctx.submit_batch(d_acc, n, d_comp, d_stall, d_status, d_ds, ws) == 0
+        res = ctx.last_result()
+        assert res["code"] == 0
+        out.append((d_comp.cpu().numpy(), d_stall.cpu().numpy(), d_ds.cpu().numpy().view(hbf.DIE_STATS_DTYPE).copy(),
+                    ctx.get_busy_until(), res))
+        assert bool((d_status == 1).all())
+    del d_acc, d_comp, d_stall, d_status, d_ds
+    return out
+
+
+@pytest.mark.parametrize("path", ["auto", "sort"])
+def test_full_size_batch_against_per_queue_oracle(full, path):
+    hbf, w, queue = full
+    ctx = hbf.Context(w.profile)
+    for r in w.ranges:
+        ctx.register_range(*r)
+    ctx.set_path(hbf.PATH_AUTO if path == "auto" else hbf.PATH_SORT)
+    runs = run_gpu(hbf, ctx, w)
+    issue = w.acc["issue_ns"]
+    sample = [0, 1, 777, 1500, 2047]
+    oracles = {}
+    for q in sample:
+        o = hbfo.Oracle(w.profile)
+        for r in w.ranges:
+            o.register_range(*r)
+        oracles[q] = o
+    npages = np.maximum(1, w.acc["bytes"].astype(np.int64) >> 14)            # size-aligned reads: 1, 2 or 4 pages
+    for step, (comp, stall, ds, busy, res) in enumerate(runs):
+        assert np.array_equal(stall, comp - issue)
+        assert res["n_modeled"] == N_FULL and res["n_native"] == 0
+        assert res["service_ns"] == int(npages.sum()) * 20000 == int(ds["busy_ns"].sum())
+        assert int(ds["n_read"].sum()) == N_FULL and int(ds["bytes_read"].sum()) == int(np.maximum(w.acc["bytes"], 64).astype(np.int64).sum())
+        assert res["modeled_ns"] == int(stall.sum()) and res["max_completion_ns"] == int(comp.max())
+        assert (stall >= npages * 20000).all()
+        for q in sample:
+            idx = np.flatnonzero(queue == q)
+            _, c_o, s_o, _, _ = oracles[q].submit(w.acc[idx])
+            bad = np.flatnonzero(comp[idx] != c_o)
+            assert bad.size == 0, (path, step, q, int(idx[bad[0]]), int(comp[idx][bad[0]]), int(c_o[bad[0]]))
+            assert int(busy[q]) == int(oracles[q].busy_until()[q])
+    ctx.destroy()
