@@ -150,6 +150,10 @@ HBF_API int hbf_reset(hbf_ctx *ctx);                                            
  * HBF_PATH_SORT always sorts (a batch already in issue order is sorted on its queue bits only, which a
  * stable sort allows); HBF_PATH_SORT_FULL sorts on every key bit regardless.  All give identical results. */
 HBF_API int hbf_set_path(hbf_ctx *ctx, int32_t path);
+/* Thermal step implementation: 0 (default) runs the whole step in one launch of a thread-block cluster when
+ * the grid fits its shared memory (up to 32,768 cells), else one launch per substep; 1 always uses the latter.
+ * Both perform the same arithmetic in the same order (Eq. 1). */
+HBF_API int hbf_set_thermal_path(hbf_ctx *ctx, int32_t generic_only);
 
 /* State snapshot (host blob): header, busy_until[queues], pending energy[dies], thermal field and
  * its compensation term.  Call with host_buf NULL to get the size. */

@@ -42,7 +42,7 @@ struct hbf_ctx {
     bool profiling = false; cudaEvent_t ev[kProfEvents] = {}; cudaEvent_t ev_th[2] = {}; bool ev_made = false;
     bool prof_submit = false, prof_thermal = false, prof_inorder = false, inorder_ok = false;
     // thermal
-    bool thermal = false; ThermalDev td{}; int cur = 0; double euler_limit_s = 0.0;
+    bool thermal = false; ThermalDev td{}; int cur = 0; double euler_limit_s = 0.0; bool thermal_generic = false;
     std::vector<void *> owned;
 };
 
@@ -267,6 +267,12 @@ size_t hbf_workspace_bytes(const hbf_ctx *c, uint64_t n) {
     return workspace_layout(n, c->mp.n_queues, nullptr, nullptr);
 }
 
+int hbf_set_thermal_path(hbf_ctx *c, int32_t generic_only) {
+    if (!c) return HBF_E_INVAL;
+    c->thermal_generic = generic_only != 0;
+    return HBF_OK;
+}
+
 int hbf_set_path(hbf_ctx *c, int32_t path) {
     if (!c || path < 0 || path > 3) return HBF_E_INVAL;
     c->path = path;
@@ -328,7 +334,7 @@ int hbf_thermal_step(hbf_ctx *c, int64_t dt_ns, const float *ext_power_w, uint32
     if (n_ext)      // pageable source: the runtime stages the bytes before returning, so the caller's array is free at once
         CK(cudaMemcpyAsync(c->td.ext_power, ext_power_w, n_ext * sizeof(float), cudaMemcpyHostToDevice, c->stream));
     if (c->profiling) CK(cudaEventRecord(c->ev_th[0], c->stream));
-    CK(launch_thermal_step(c->td, c->d_state, c->d_pending, dt_ns, n_ext != 0, d_temps_out, &c->cur, c->stream));
+    CK(launch_thermal_step(c->td, c->d_state, c->d_pending, dt_ns, n_ext != 0, d_temps_out, &c->cur, c->thermal_generic ? 1 : 0, c->stream));
     if (c->profiling) { CK(cudaEventRecord(c->ev_th[1], c->stream)); c->prof_thermal = true; }
     if (hot_c_out) {
         CK(cudaMemcpyAsync(c->h_hot, c->td.hot, 3 * sizeof(float), cudaMemcpyDeviceToHost, c->stream));

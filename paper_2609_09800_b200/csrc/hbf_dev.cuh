@@ -129,6 +129,6 @@ struct ThermalDev {
     float *hot;                          // [3] device
 };
 cudaError_t launch_thermal_step(const ThermalDev &t, DevState *state, int64_t *pending, int64_t dt_ns,
-                                int has_ext, float *d_temps_out, int *cur, cudaStream_t st);
+                                int has_ext, float *d_temps_out, int *cur, int generic_only, cudaStream_t st);
 
 }  // namespace hbf

@@ -6,7 +6,11 @@
 // 10^4..10^5 substeps and stalls once an increment drops under half an ulp of the state.
 #include <algorithm>
 
+#include <cooperative_groups.h>
+
 #include "device_utils.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace hbf {
 
@@ -100,8 +104,8 @@ k_controller(ThermalDev t, const float *__restrict__ th, DevState *state, float 
     }
 }
 
-cudaError_t launch_thermal_step(const ThermalDev &t, DevState *state, int64_t *pending, int64_t dt_ns, int has_ext,
-                                float *d_temps_out, int *cur, cudaStream_t st) {
+static cudaError_t launch_thermal_generic(const ThermalDev &t, DevState *state, int64_t *pending, int64_t dt_ns, int has_ext,
+                                          float *d_temps_out, int *cur, cudaStream_t st) {
     k_power_map<<<1, 1024, 0, st>>>(t, pending, dt_ns, has_ext);
     const float dt_sub = (float)((double)dt_ns * 1e-9 / (double)t.n_sub);
     dim3 grid((t.W + 31) / 32, (t.H + 7) / 8);
@@ -114,6 +118,186 @@ cudaError_t launch_thermal_step(const ThermalDev &t, DevState *state, int64_t *p
     g_kernel_launches += 2ull + t.n_sub;
     k_controller<<<1, 1024, 0, st>>>(t, t.theta[c], state, d_temps_out);
     return cudaGetLastError();
+}
+
+
+// ======================================================================================================
+// The whole step in one launch, for grids that fit the shared memory of one thread-block cluster: eight
+// blocks each keep a band of rows of the field (both Jacobi buffers, with one halo row above and below) in
+// shared memory and every cell's constants, power and compensation term in registers.  After each substep
+// a block writes its first and last row into its neighbours' halo rows through distributed shared memory
+// and the cluster barrier separates the substeps.  The arithmetic of a cell is the same, in the same
+// order, as in k_euler_substep; the power map is formed by every block for its own cells and the
+// hotspots are reduced through block 0.
+// ======================================================================================================
+constexpr int kThClusterBlocks = 8;
+constexpr int kThThreads = 512;
+constexpr int kThCellsPerThread = 8;
+constexpr int kThMaxRegions = 1024;
+
+__global__ void __cluster_dims__(kThClusterBlocks, 1, 1) __launch_bounds__(kThThreads)
+k_thermal_cluster(ThermalDev t, float *theta, DevState *state, int64_t *pending, int64_t dt_ns, int has_ext, float dt_sub,
+                  float *temps_out) {
+    extern __shared__ __align__(16) unsigned char th_smem[];
+    __shared__ double s_region_power[kThMaxRegions];
+    __shared__ float s_hot[kThClusterBlocks][3];
+    __shared__ float s_part[3][kThThreads / 32];
+    cg::cluster_group cluster = cg::this_cluster();
+    const uint32_t rank = cluster.block_rank();
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t H = t.H, W = t.W;
+    const uint32_t rows = (H + kThClusterBlocks - 1) / kThClusterBlocks;
+    const uint32_t y0 = min(H, rank * rows), y1 = min(H, y0 + rows);
+    const uint32_t band_cells = (y1 - y0) * W;
+    const uint32_t pitch = (rows + 2) * W;                    // one buffer: halo row, band, halo row
+    float *buf0 = reinterpret_cast<float *>(th_smem), *buf1 = buf0 + pitch;
+
+    // power of every region over the window (every block forms the same values), then of this block's cells
+    for (uint32_t g = tid; g < t.n_regions; g += kThThreads) {
+        double p = 0.0;
+        for (int32_t k = t.region_die_ptr[g]; k < t.region_die_ptr[g + 1]; ++k)
+            p += ((double)pending[t.region_die_list[k]] * 1e-12) / ((double)dt_ns * 1e-9);
+        p += (double)t.region_idle_w[g];
+        if (has_ext) p += (double)t.ext_power[g];
+        s_region_power[g] = p;
+    }
+    // field: own rows and the neighbours' boundary rows, from global memory
+    for (uint32_t i = tid; i < (y1 - y0 + 2) * W && y1 > y0; i += kThThreads) {
+        const uint32_t r = i / W, x = i - r * W;
+        const int64_t y = (int64_t)y0 + r - 1;
+        buf0[r * W + x] = (y >= 0 && y < (int64_t)H) ? theta[(uint64_t)y * W + x] : 0.0f;
+    }
+    __syncthreads();
+    // this thread's cells: constants, power and compensation in registers
+    float kC[kThCellsPerThread], gE[kThCellsPerThread], gW_[kThCellsPerThread], gS[kThCellsPerThread], gN[kThCellsPerThread],
+          gs[kThCellsPerThread], P[kThCellsPerThread], cmp[kThCellsPerThread];
+    uint32_t off[kThCellsPerThread];
+    uint32_t flags[kThCellsPerThread];
+#pragma unroll
+    for (int c = 0; c < kThCellsPerThread; ++c) {
+        const uint32_t li = (uint32_t)c * kThThreads + tid;   // cell of the band, row-major
+        flags[c] = 0; off[c] = 0; kC[c] = gE[c] = gW_[c] = gS[c] = gN[c] = gs[c] = P[c] = cmp[c] = 0.0f;
+        if (li < band_cells) {
+            const uint32_t r = li / W, x = li - r * W, y = y0 + r;
+            const uint64_t i = (uint64_t)y * W + x;
+            off[c] = (r + 1) * W + x;
+            flags[c] = 1u | (x + 1 < W ? 2u : 0u) | (x > 0 ? 4u : 0u) | (y + 1 < H ? 8u : 0u) | (y > 0 ? 16u : 0u);
+            kC[c] = dt_sub / t.C[i];
+            gE[c] = t.Gx[i]; gW_[c] = x > 0 ? t.Gx[i - 1] : 0.0f; gS[c] = t.Gy[i]; gN[c] = y > 0 ? t.Gy[i - W] : 0.0f;
+            gs[c] = t.Gs[i]; cmp[c] = t.comp[i];
+            const int32_t g = t.cell_region[i];
+            P[c] = g >= 0 ? (float)(s_region_power[g] * (double)t.region_inv_cells[g]) : 0.0f;
+        }
+    }
+    float *upper_halo0 = nullptr, *upper_halo1 = nullptr, *lower_halo0 = nullptr, *lower_halo1 = nullptr;
+    if (rank > 0 && y1 > y0) {                                   // the block above: its lower halo row sits after its band
+        const uint32_t rows_above = min(H, rank * rows) - min(H, (rank - 1) * rows);
+        upper_halo0 = cluster.map_shared_rank(buf0, rank - 1) + (rows_above + 1) * W;
+        upper_halo1 = cluster.map_shared_rank(buf1, rank - 1) + (rows_above + 1) * W;
+    }
+    if (rank + 1 < (uint32_t)kThClusterBlocks && y1 < H) {      // the block below: its upper halo row is row 0
+        lower_halo0 = cluster.map_shared_rank(buf0, rank + 1);
+        lower_halo1 = cluster.map_shared_rank(buf1, rank + 1);
+    }
+    cluster.sync();
+    if (rank == 0) for (uint32_t d = tid; d < t.n_dies; d += kThThreads) pending[d] = 0;   // every block has read it
+
+    float *in = buf0, *out = buf1;
+    for (uint32_t k = 0; k < t.n_sub; ++k) {
+        float *up = (out == buf0) ? upper_halo0 : upper_halo1, *down = (out == buf0) ? lower_halo0 : lower_halo1;
+#pragma unroll
+        for (int c = 0; c < kThCellsPerThread; ++c) {
+            if (flags[c] & 1u) {
+                const uint32_t o = off[c];
+                const float Ti = in[o];
+                float flow = 0.0f;
+                if (flags[c] & 2u)  flow += gE[c] * (Ti - in[o + 1]);
+                if (flags[c] & 4u)  flow += gW_[c] * (Ti - in[o - 1]);
+                if (flags[c] & 8u)  flow += gS[c] * (Ti - in[o + W]);
+                if (flags[c] & 16u) flow += gN[c] * (Ti - in[o - W]);
+                const float inc = kC[c] * (P[c] - flow - gs[c] * Ti);
+                const float yv = inc - cmp[c];
+                const float tn = Ti + yv;
+                cmp[c] = (tn - Ti) - yv;
+                out[o] = tn;
+                const uint32_t r = o / W;                        // first / last row of the band: also the neighbours' halo
+                if (r == 1 && up) up[o - W] = tn;
+                if (r == y1 - y0 && down) down[o - (y1 - y0) * W] = tn;
+            }
+        }
+        cluster.sync();
+        float *tmp = in; in = out; out = tmp;
+    }
+    // results: field and compensation back to global memory, hotspots to block 0
+    float hot[3] = {-INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+    for (int c = 0; c < kThCellsPerThread; ++c) {
+        if (flags[c] & 1u) {
+            const uint32_t li = (uint32_t)c * kThThreads + tid;
+            const uint64_t i = (uint64_t)y0 * W + li;
+            const float th = in[off[c]];
+            theta[i] = th; t.comp[i] = cmp[c];
+            const float T = t.ambient_c + th;
+            if (temps_out) temps_out[i] = T;
+            const int32_t g = t.cell_region[i];
+            if (g >= 0) {
+                const int32_t kind = t.region_kind[g];
+                if (kind == HBF_KIND_HBF) hot[0] = fmaxf(hot[0], T); else if (kind == HBF_KIND_HBM) hot[1] = fmaxf(hot[1], T);
+                else if (kind == HBF_KIND_GPU) hot[2] = fmaxf(hot[2], T);
+            }
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < 3; ++k) {
+        for (int o = 16; o > 0; o >>= 1) hot[k] = fmaxf(hot[k], __shfl_xor_sync(0xffffffffu, hot[k], o));
+        if (lane == 0) s_part[k][warp] = hot[k];
+    }
+    __syncthreads();
+    if (tid < 3) {
+        float v = -INFINITY;
+        for (int w = 0; w < kThThreads / 32; ++w) v = fmaxf(v, s_part[tid][w]);
+        float *dst = cluster.map_shared_rank(&s_hot[0][0], 0);
+        dst[rank * 3 + tid] = v;
+    }
+    cluster.sync();
+    if (rank == 0 && tid == 0) {
+        float h[3];
+        for (int k = 0; k < 3; ++k) {
+            float v = -INFINITY;
+            for (int b = 0; b < kThClusterBlocks; ++b) v = fmaxf(v, s_hot[b][k]);
+            h[k] = v == -INFINITY ? t.ambient_c : v;
+            t.hot[k] = h[k];
+        }
+        const int mode = next_mode(t, state->mode, quantise_mk(h[0]));
+        state->mode = mode;
+        if (mode == HBF_MODE_NORMAL) state->q_ppm = 1000000;
+        else if (mode == HBF_MODE_LIGHT) state->q_ppm = t.q_light_ppm;
+    }
+}
+
+static bool thermal_cluster_fits(const ThermalDev &t, size_t *smem_bytes) {
+    const uint32_t rows = (t.H + kThClusterBlocks - 1) / kThClusterBlocks;
+    const size_t smem = (size_t)2 * (rows + 2) * t.W * sizeof(float);
+    *smem_bytes = smem;
+    return (size_t)rows * t.W <= (size_t)kThThreads * kThCellsPerThread && smem <= 200u * 1024u && t.n_regions <= (uint32_t)kThMaxRegions;
+}
+
+cudaError_t launch_thermal_step(const ThermalDev &t, DevState *state, int64_t *pending, int64_t dt_ns, int has_ext,
+                                float *d_temps_out, int *cur, int generic_only, cudaStream_t st) {
+    const float dt_sub_f = (float)((double)dt_ns * 1e-9 / (double)t.n_sub);
+    size_t smem = 0;
+    if (!generic_only && thermal_cluster_fits(t, &smem)) {
+        static size_t set_smem = 0;
+        if (smem > set_smem) {
+            cudaError_t e = cudaFuncSetAttribute(k_thermal_cluster, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+            set_smem = smem;
+        }
+        k_thermal_cluster<<<kThClusterBlocks, kThThreads, smem, st>>>(t, t.theta[*cur], state, pending, dt_ns, has_ext, dt_sub_f, d_temps_out);
+        g_kernel_launches += 1;
+        return cudaGetLastError();
+    }
+    return launch_thermal_generic(t, state, pending, dt_ns, has_ext, d_temps_out, cur, st);
 }
 
 }  // namespace hbf

@@ -28,7 +28,7 @@ EXPORTS = ("hbf_create", "hbf_destroy", "hbf_register_range", "hbf_clear_ranges"
            "hbf_submit_batch", "hbf_last_result", "hbf_thermal_step", "hbf_force_mode", "hbf_get_mode",
            "hbf_reset", "hbf_set_path", "hbf_get_state", "hbf_set_state", "hbf_get_busy_until",
            "hbf_get_pending_energy", "hbf_get_temps", "hbf_euler_limit_ns", "hbf_queue_order", "hbf_strerror",
-           "hbf_set_profiling", "hbf_get_profile", "hbf_kernel_launches", "hbf_euler_substeps_static")
+           "hbf_set_profiling", "hbf_get_profile", "hbf_kernel_launches", "hbf_euler_substeps_static", "hbf_set_thermal_path")
 STATIC_MAX_CELLS = 65536
 PROF_STAGES = ("begin", "classify", "plan_hist", "sort", "scan", "finish", "inorder", "thermal")
 
@@ -91,6 +91,7 @@ def lib():
         L.hbf_get_mode.argtypes = [vp, C.POINTER(i32), C.POINTER(i64)]
         L.hbf_reset.argtypes = [vp]
         L.hbf_set_path.argtypes = [vp, i32]
+        L.hbf_set_thermal_path.argtypes = [vp, i32]
         L.hbf_get_state.argtypes = [vp, vp, C.POINTER(C.c_size_t)]
         L.hbf_set_state.argtypes = [vp, vp, C.c_size_t]
         L.hbf_get_busy_until.argtypes = [vp, vp, u64]
@@ -244,6 +245,11 @@ class Context:
             raise HbfError(rc, "hbf_set_path")
 
     # ---- thermal ------------------------------------------------------------------------------
+    def set_thermal_path(self, generic_only: bool):
+        rc = lib().hbf_set_thermal_path(self._h, 1 if generic_only else 0)
+        if rc != 0:
+            raise HbfError(rc, "hbf_set_thermal_path")
+
     def thermal_step(self, dt_ns, ext_power_w=None, d_temps_out=None, want_hot=True):
         hot = np.empty(3, np.float32) if want_hot else None
         if ext_power_w is None:

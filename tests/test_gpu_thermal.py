@@ -148,3 +148,24 @@ def test_reset_and_state_round_trip(hbf):
     assert np.array_equal(g.get_temps(), T)
     for _ in range(25):
         step_both(hbf, g, o, prof, dt, fp["ext_power_w"])
+
+
+@pytest.mark.parametrize("shape", [(128, 128), (17, 45), (3, 40), (130, 131), (64, 64)])
+def test_cluster_step_equals_per_substep_launches(hbf, shape):
+    """The one-launch cluster kernel and the launch-per-substep kernels perform the same arithmetic."""
+    import torch
+    h, w_ = shape
+    fp = wl.package_floorplan() if shape == (128, 128) else wl.toy_floorplan(h, w_, 8, 4, seed=h + w_)
+    geo = wl.GEOMETRY["serving"] if shape == (128, 128) else wl.GEOMETRY["tiny"]
+    prof = wl.load_profile("nominal", **geo, n_sub=9)
+    a, b = hbf.Context(prof, fp), hbf.Context(prof, fp)
+    b.set_thermal_path(True)
+    dt = int(0.8 * a.euler_limit_ns() * 9)
+    Ta = torch.empty(a.n_cells, dtype=torch.float32, device="cuda"); Tb = torch.empty_like(Ta)
+    for k in range(30):
+        ext = fp["ext_power_w"] * np.float32(1 + k % 4)
+        hot_a = a.thermal_step(dt, ext, Ta)
+        hot_b = b.thermal_step(dt, ext, Tb)
+        assert torch.equal(Ta, Tb), k
+        assert np.array_equal(hot_a, hot_b) and a.get_mode() == b.get_mode()
+    assert np.array_equal(a.get_temps(), b.get_temps())
