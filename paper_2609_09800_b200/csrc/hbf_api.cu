@@ -158,6 +158,22 @@ int hbf_create(const hbf_config_t *cfg, void *cuda_stream, hbf_ctx **out) {
         c->inorder_ok = nq <= kInMaxQueues && worst / cfg->chan_bytes_per_us < ((unsigned __int128)1 << 31) &&
                         100u * 1024u + nd * 24u <= 220u * 1024u;
     }
+    {   // transfer times of the small charged sizes, looked up instead of divided (every charged size is a multiple of its granule)
+        const uint32_t g = std::min(mp.read_gran_shift, mp.prog_gran_shift);
+        std::vector<uint32_t> tab(1025);
+        bool fits = true;
+        for (uint32_t k = 0; k <= 1024; ++k) {
+            const unsigned __int128 x = (((unsigned __int128)k << g) * 1000u + cfg->chan_bytes_per_us - 1) / cfg->chan_bytes_per_us;
+            if (x >> 31) fits = false;
+            tab[k] = (uint32_t)x;
+        }
+        mp.xfer_tab = nullptr; mp.xfer_tab_shift = g; mp.xfer_tab_max_cb = 0;
+        if (fits && g < 21) {
+            uint32_t *d = nullptr;
+            if ((rc = dev_copy(c, &d, tab.data(), tab.size()))) return fail(rc);
+            mp.xfer_tab = d; mp.xfer_tab_max_cb = 1024u << g;
+        }
+    }
     DevState st0; st0.mode = HBF_MODE_NORMAL; st0.poisoned = 0; st0.q_ppm = 1000000;
     if ((rc = dev_copy(c, &c->d_ranges, nullptr, 1))) return fail(rc);
     if ((rc = dev_copy(c, &c->d_mp, &mp, 1))) return fail(rc);

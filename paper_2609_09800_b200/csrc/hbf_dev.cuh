@@ -40,6 +40,8 @@ struct ModelParams {
     int64_t t_read_ns, t_prog_ns;
     uint64_t chan_bytes_per_us;
     Div64 div_chan;                      // division by chan_bytes_per_us
+    const uint32_t *xfer_tab;            // device: transfer ns of charged bytes k << xfer_tab_shift, k = 0..1024
+    uint32_t xfer_tab_shift, xfer_tab_max_cb;
     int64_t e_cmd_read_pj, e_byte_read_pj, e_cmd_prog_pj, e_byte_prog_pj;
 };
 

@@ -39,7 +39,6 @@ constexpr uint32_t kInNoQueue = 0xffffu;                 // record is not modele
 constexpr int kInSlotBytes = kInChunk * 24;
 constexpr int kInCntBytes = (kInMaxQueues + 64) * 4;
 constexpr int kInPosBytes = kInChunk * 2;
-constexpr int kInStartRow = kInThreads + 8;              // shared: first queue-major position of each thread's queues, + end
 
 // word 2 of a slot: transfer ns (31 bits) | op << 31 | queue << 32 | slot taken in the queue's bucket << 48
 __device__ __forceinline__ uint32_t img_queue(uint64_t w2) { return (uint32_t)(w2 >> 32) & 0xffffu; }
@@ -63,9 +62,40 @@ __device__ __forceinline__ Served serve_terms(const RangeSnap &rs, const ModelPa
     return r;
 }
 
-// state arrays are laid out so that thread t's queues sit in different banks than thread t+1's
+// The same terms for the common configuration (one registered range, power-of-two geometry, no thermal
+// scaling in force, transfer table present): 32-bit arithmetic wherever the values allow it.
+struct FastRange { uint64_t base, length, media_offset; uint32_t perms, on; };
+__device__ __forceinline__ Served serve_terms_fast(const FastRange &f, const ModelParams &mp, uint64_t addr, int64_t issue, uint64_t bf) {
+    Served r; r.queue = 0; r.die = 0; r.op = 0; r.s = 0; r.xfer = 0; r.cb = 0;
+    const uint32_t bytes = (uint32_t)bf, flags = (uint32_t)(bf >> 32);
+    const uint64_t rel = addr - f.base;                       // wraps to a huge value below the base
+    if (bytes == 0u || (flags & ~1u) != 0u || (uint32_t)((uint64_t)issue >> 32) >= (1u << (kIssueBits - 32))) { r.st = HBF_ST_UNSUPPORTED; return r; }
+    if (rel >= f.length) { r.st = HBF_ST_NATIVE; return r; }
+    if ((uint64_t)bytes > f.length - rel) { r.st = HBF_ST_FAULT_PARTIAL; return r; }
+    r.op = flags & 1u;
+    if (!(f.perms & (1u << r.op))) { r.st = HBF_ST_FAULT_PERM; return r; }
+    r.st = HBF_ST_READY;
+    const uint64_t off = f.media_offset + rel;
+    const uint32_t u = (uint32_t)(off >> mp.stripe_shift);    // only the low interleave bits are used
+    const uint32_t ch = u & (mp.channels - 1u), di = (u >> mp.ch_shift) & (mp.dies - 1u);
+    const uint32_t pl = (u >> (mp.ch_shift + mp.die_shift)) & (mp.planes - 1u);
+    r.die = ch * mp.dies + di;
+    r.queue = mp.queue_level == 0u ? r.die * mp.planes + pl : r.die;
+    const uint32_t page_mask = (1u << mp.page_shift) - 1u;
+    const uint32_t npages = (uint32_t)(((uint64_t)((uint32_t)off & page_mask) + bytes + page_mask) >> mp.page_shift);
+    const uint32_t gs = r.op ? mp.prog_gran_shift : mp.read_gran_shift;
+    const uint64_t cb = (((uint64_t)bytes + ((1ull << gs) - 1ull)) >> gs) << gs;
+    r.cb = (int64_t)cb;
+    r.xfer = cb <= (uint64_t)mp.xfer_tab_max_cb ? (int64_t)__ldg(mp.xfer_tab + (uint32_t)(cb >> mp.xfer_tab_shift))
+                                                 : (int64_t)div64(cb * 1000ull + mp.chan_bytes_per_us - 1ull, mp.div_chan);
+    r.s = (int64_t)npages * (r.op ? mp.t_prog_ns : mp.t_read_ns);
+    return r;
+}
+
+// index of a queue's state in the shared-memory arrays
 __device__ __forceinline__ uint32_t state_index(uint32_t q, uint32_t qpt_shift) {
-    return ((q & ((1u << qpt_shift) - 1u)) << 8) | (q >> qpt_shift);
+    (void)qpt_shift;
+    return q;
 }
 
 // per-tile bookkeeping of the stall total: as-if-idle sum, fix-up corrections, and the exact sum of a re-served tile
@@ -92,8 +122,9 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
     __shared__ uint32_t s_bin_start[kInBins];
     __shared__ uint32_t s_bin_warp[2];
     __shared__ uint32_t s_warp_tot[kInWarps];
-    __shared__ uint16_t s_tstart[kInStartRow];
     __shared__ long long s_red[2];
+    __shared__ FastRange s_fast;
+    __shared__ uint32_t s_heads_full;                     // queues whose head entries are complete
 
     if (ctrl->skip) return;
     if (RESERVE && (ctrl->run_sort || !ctrl->inorder_used || !in_tile[blockIdx.x].reserve)) return;
@@ -102,6 +133,11 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
     for (int i = tid; i < (int)(sizeof(ModelParams) / 4); i += kInThreads)
         reinterpret_cast<uint32_t *>(&mp)[i] = reinterpret_cast<const uint32_t *>(mp_g)[i];
     const uint32_t R = mp_g->n_queues, n_dies = mp_g->n_dies;
+    if (tid == 0) {
+        FastRange f; f.base = rs.base[0]; f.length = rs.length[0]; f.media_offset = rs.media_offset[0]; f.perms = rs.perms[0];
+        f.on = (rs.count == 1u && mp_g->pow2_geom && mp_g->xfer_tab_max_cb != 0u && ctrl->q_ppm == 1000000) ? 1u : 0u;
+        s_fast = f;
+    }
 
     // slot e holds record e on arrival, then its served image (in place)
     uint64_t *slot = reinterpret_cast<uint64_t *>(in_smem);
@@ -113,8 +149,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
     uint32_t *st_br_lo = reinterpret_cast<uint32_t *>(aggM + kInMaxQueues), *st_br_hi = st_br_lo + n_dies;   // per die
     uint32_t *st_bp_lo = st_br_hi + n_dies, *st_bp_hi = st_bp_lo + n_dies;
     uint32_t *st_nr = st_bp_hi + n_dies, *st_np = st_nr + n_dies;
-    // head-table fill count per queue, one nibble each; the two nibbles of a byte belong to the same thread
-    uint8_t *hfill = reinterpret_cast<uint8_t *>(st_np + n_dies);
+    uint8_t *hfill = reinterpret_cast<uint8_t *>(st_np + n_dies);                  // head-table entries written per queue
 
     const uint32_t tile = blockIdx.x;
     const uint64_t tile_begin = (uint64_t)tile * tile_records;
@@ -131,7 +166,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
         for (uint32_t q = tid; q < R; q += kInThreads) aggM[state_index(q, qpt_shift)] = in_bin[(uint64_t)blockIdx.x * R + q];
     } else {
         for (uint32_t d = tid; d < n_dies * 6u; d += kInThreads) st_br_lo[d] = 0u;
-        for (uint32_t i = tid; i < kInMaxQueues / 2; i += kInThreads) hfill[i] = 0;
+        for (uint32_t i = tid; i < kInMaxQueues; i += kInThreads) hfill[i] = 0;
     }
 
     const uint32_t qbits = 32u - (uint32_t)__clz((int)R);
@@ -143,10 +178,9 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
     unsigned long long c_native = 0, c_ready = 0, c_fault = 0;
     unsigned c_unsorted = 0;
     long long sum_stall = 0, max_c = INT64_MIN;
-    bool heads_open = !RESERVE;                           // this thread still fills head entries of its queues
-    uint32_t heads_full = 0;
-    const uint32_t owned_queues = min(qpt, R > (uint32_t)tid * qpt ? R - (uint32_t)tid * qpt : 0u);
+
     if (tid < 2) s_red[tid] = tid == 1 ? INT64_MIN : 0;
+    if (tid == 0) s_heads_full = 0u;
 
     for (uint64_t cbase = tile_begin; cbase < tile_end; cbase += kInChunk) {
         const int cnt = (int)min((uint64_t)kInChunk, tile_end - cbase);
@@ -175,7 +209,8 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
                     const int64_t prev = e > 0 ? (int64_t)slot[e * 3 - 2] : (cbase > 0 ? acc[cbase - 1].issue_ns : INT64_MIN);
                     c_unsorted |= issue < prev ? 1u : 0u;
                 }
-                const Served v = serve_terms(rs, mp, addr, issue, slot[e * 3 + 2], q_ppm, div_q);
+                const Served v = s_fast.on ? serve_terms_fast(s_fast, mp, addr, issue, slot[e * 3 + 2])
+                                           : serve_terms(rs, mp, addr, issue, slot[e * 3 + 2], q_ppm, div_q);
                 if (!RESERVE && status) status[cbase + e] = (uint8_t)v.st;
                 uint64_t w0 = 0, w2 = (uint64_t)kInNoQueue << 32;
                 if (v.st == HBF_ST_READY) {
@@ -236,8 +271,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
                 for (int b = 0; b < 8; ++b)
                     if ((uint32_t)b < qpt && q0 + b < R) qcnt[q0 + b] = base + c[b];
             }
-            s_tstart[tid] = (uint16_t)base;
-            if (tid == kInThreads - 1) { qcnt[R] = base + tot; s_tstart[kInThreads] = (uint16_t)(base + tot); }
+            if (tid == kInThreads - 1) qcnt[R] = base + tot;
         }
         __syncthreads();
         if (!use_radix) {
@@ -323,68 +357,77 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
             }
         }
         __syncthreads();
-        // ---- serve: thread t walks its queues' accesses, which are consecutive in queue-major order --------
-        // (four at a time: the loads of a group are independent, only the max-plus chain is serial).
-        // M is the aggregate's constant term and, at the same time, the busy-until of the as-if-idle run.
+        // ---- serve.  In queue-major order a queue's accesses are consecutive.  Thread t takes positions
+        // [8t, 8t+8) and serves every queue whose first access of the chunk lies there, to that queue's last
+        // access (which may lie past 8t+8; the thread owning those positions skips them).  Every thread thus
+        // does about eight accesses, and a queue is touched by one thread only.  Loads go four at a time: they
+        // are independent, only the max-plus chain is serial.  M is the aggregate's constant term and, at the
+        // same time, the busy-until of the as-if-idle run.
         {
-            const uint32_t k0 = s_tstart[tid], k1 = s_tstart[tid + 1];
-            uint32_t cur = kInNoQueue, ci = 0, hf = 0;
-            int64_t S = 0, M = kNegInf;
-            auto close_queue = [&]() {
-                aggS[ci] = S; aggM[ci] = M;
-                if (!RESERVE && heads_open) {
-                    uint8_t *hb = hfill + (((ci >> 9) << 8) | (ci & 255u));
-                    const uint32_t old = ((ci >> 8) & 1u) ? (uint32_t)(*hb >> 4) : (uint32_t)(*hb & 0x0fu);
-                    *hb = ((ci >> 8) & 1u) ? (uint8_t)((*hb & 0x0fu) | (hf << 4)) : (uint8_t)((*hb & 0xf0u) | hf);
-                    if (old < (uint32_t)kInHead && hf == (uint32_t)kInHead) ++heads_full;
-                }
-            };
-            for (uint32_t k = k0; k < k1; k += kInGroup) {
-                uint32_t e[kInGroup], qi[kInGroup];
-                int64_t s_[kInGroup], m_[kInGroup], aS[kInGroup], aM[kInGroup];
-                uint64_t w2[kInGroup];
+            const uint32_t modeled = qcnt[R];
+            const uint32_t p0 = (uint32_t)tid * kInItems;
+            const bool heads_on = !RESERVE && s_heads_full < R;
+            if (p0 < modeled) {
+                uint32_t cur = kInNoQueue, hf = 0;
+                bool mine = false;                            // the queue being served was opened by this thread
+                int64_t S = 0, M = kNegInf;
+                uint32_t prev_q = p0 > 0 ? img_queue(slot[(uint32_t)posB[p0 - 1] * 3 + 2]) : kInNoQueue;
+                auto close_queue = [&]() {
+                    aggS[cur] = S; aggM[cur] = M;
+                    if (heads_on) {
+                        if (hfill[cur] < (uint8_t)kInHead && hf == (uint32_t)kInHead) atomicAdd(&s_heads_full, 1u);
+                        hfill[cur] = (uint8_t)hf;
+                    }
+                };
+                auto serve_one = [&](uint32_t e, int64_t sv, int64_t issue, uint64_t w2) {
+                    const uint32_t x = (uint32_t)w2;
+                    const int64_t xfer = (int64_t)(x & 0x7fffffffu);
+                    const bool op = (x >> 31) != 0u;
+                    const int64_t m = issue + (op ? xfer : 0) + sv;          // arrival + service
+                    if (heads_on && hf < (uint32_t)kInHead) {                 // among the first accesses of this queue in the tile
+                        InHead h; h.m = m; h.s = sv; h.xo = x; h.idx = (uint32_t)(cbase + e);
+                        in_head[((uint64_t)tile * kInHead + hf) * R + cur] = h;
+                        ++hf;
+                    }
+                    M = max(M + sv, m); S += sv;                              // aggregate o access; M = busy-until after it
+                    const int64_t done = M + (op ? 0 : xfer);
+                    slot[e * 3] = (uint64_t)done; slot[e * 3 + 1] = (uint64_t)(done - issue);
+                    sum_stall += done - issue; max_c = max(max_c, (long long)done);
+                };
 #pragma unroll
-                for (int j = 0; j < kInGroup; ++j) e[j] = k + j < k1 ? (uint32_t)posB[k + j] : 0u;
+                for (int g = 0; g < kInItems / kInGroup; ++g) {
+                    const uint32_t pg = p0 + g * kInGroup;
+                    uint32_t e[kInGroup];
+                    int64_t s_[kInGroup], i_[kInGroup];
+                    uint64_t w2[kInGroup];
 #pragma unroll
-                for (int j = 0; j < kInGroup; ++j) {
-                    s_[j] = (int64_t)slot[e[j] * 3]; m_[j] = (int64_t)slot[e[j] * 3 + 1]; w2[j] = slot[e[j] * 3 + 2];
-                    // word 1 is the issue time: arrival + service = issue (+ transfer, for a program) + service
-                    m_[j] += s_[j] + ((((uint32_t)w2[j]) >> 31) ? (int64_t)((uint32_t)w2[j] & 0x7fffffffu) : 0);
-                }
+                    for (int j = 0; j < kInGroup; ++j) e[j] = pg + j < modeled ? (uint32_t)posB[pg + j] : 0u;
 #pragma unroll
-                for (int j = 0; j < kInGroup; ++j) {
-                    qi[j] = state_index(img_queue(w2[j]) & (kInMaxQueues - 1), qpt_shift);
-                    aS[j] = aggS[qi[j]]; aM[j] = aggM[qi[j]];       // used only if this access opens its queue here
-                }
+                    for (int j = 0; j < kInGroup; ++j) { s_[j] = (int64_t)slot[e[j] * 3]; i_[j] = (int64_t)slot[e[j] * 3 + 1]; w2[j] = slot[e[j] * 3 + 2]; }
 #pragma unroll
-                for (int j = 0; j < kInGroup; ++j) {
-                    if (k + j < k1) {
-                        const uint32_t q = img_queue(w2[j]);
-                        if (q != cur) {
-                            if (cur != kInNoQueue) close_queue();
-                            cur = q; ci = qi[j]; S = aS[j]; M = aM[j];
-                            if (!RESERVE && heads_open) {
-                                const uint8_t hb = hfill[((ci >> 9) << 8) | (ci & 255u)];
-                                hf = ((ci >> 8) & 1u) ? (uint32_t)(hb >> 4) : (uint32_t)(hb & 0x0fu);
+                    for (int j = 0; j < kInGroup; ++j) {
+                        if (pg + j < modeled) {
+                            const uint32_t q = img_queue(w2[j]);
+                            if (q != prev_q) {                                // first access of queue q in this chunk
+                                if (mine) close_queue();
+                                cur = q; mine = true; S = aggS[q]; M = aggM[q];
+                                if (heads_on) hf = hfill[q];
                             }
+                            if (mine) serve_one(e[j], s_[j], i_[j], w2[j]);
+                            prev_q = q;
                         }
-                        if (!RESERVE && heads_open && hf < (uint32_t)kInHead) {    // among the first accesses of this queue in the tile
-                            InHead h; h.m = m_[j]; h.s = s_[j]; h.xo = (uint32_t)w2[j]; h.idx = (uint32_t)(cbase + e[j]);
-                            in_head[((uint64_t)tile * kInHead + hf) * R + q] = h;
-                            ++hf;
-                        }
-                        M = max(M + s_[j], m_[j]); S += s_[j];      // aggregate o access; M = busy-until after it
-                        const int64_t xfer = (int64_t)((uint32_t)w2[j] & 0x7fffffffu);
-                        const bool op = (((uint32_t)w2[j]) >> 31) != 0u;
-                        const int64_t done = M + (op ? 0 : xfer);
-                        const int64_t wait = done - (m_[j] - s_[j] - (op ? xfer : 0));
-                        slot[e[j] * 3] = (uint64_t)done; slot[e[j] * 3 + 1] = (uint64_t)wait;
-                        sum_stall += wait; max_c = max(max_c, (long long)done);
                     }
                 }
+                if (mine) {                                    // the last queue opened here may go on past this thread's positions
+                    for (uint32_t p = p0 + kInItems; p < modeled; ++p) {
+                        const uint32_t e = posB[p];
+                        const uint64_t w2 = slot[e * 3 + 2];
+                        if (img_queue(w2) != cur) break;
+                        serve_one(e, (int64_t)slot[e * 3], (int64_t)slot[e * 3 + 1], w2);
+                    }
+                    close_queue();
+                }
             }
-            if (cur != kInNoQueue) close_queue();
-            if (heads_full >= owned_queues) heads_open = false;          // every queue of this thread has its head entries
         }
         __syncthreads();
         // ---- results leave in batch order; the chunk's queue-major order stays behind for the fix-up ----------
@@ -403,8 +446,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
         for (uint32_t q = tid; q < R; q += kInThreads) {
             const uint32_t i = state_index(q, qpt_shift);
             out[q] = make_longlong2(aggS[i], aggM[i]);
-            const uint8_t hb = hfill[((i >> 9) << 8) | (i & 255u)];
-            in_headcnt[(uint64_t)tile * R + q] = ((i >> 8) & 1u) ? (uint8_t)(hb >> 4) : (uint8_t)(hb & 0x0fu);
+            in_headcnt[(uint64_t)tile * R + q] = hfill[q];
         }
         for (uint32_t d = tid; d < n_dies; d += kInThreads) {
             unsigned long long *g = reinterpret_cast<unsigned long long *>(stats_stage + d);
@@ -643,7 +685,7 @@ cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st) {
     const unsigned n_tiles = (unsigned)((n + tile_records - 1) / tile_records);
     const uint32_t R = a.mp.n_queues, nd = a.mp.n_dies, row_stride = inorder_row_stride(R);
     const size_t smem_serve = (size_t)kInSlotBytes + kInCntBytes + 2 * kInPosBytes + (size_t)kInMaxQueues * 16 + (size_t)nd * 24 +
-                              kInMaxQueues / 2;
+                              kInMaxQueues;
     static size_t set_serve = 0;
     if (smem_serve > set_serve) {
         cudaError_t e = cudaFuncSetAttribute(k_inorder_serve<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_serve);
