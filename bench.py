@@ -12,6 +12,7 @@ Prints ONE JSON line.  ``--impl reference`` times the CPU oracle instead (rank 0
 from __future__ import annotations
 
 import argparse
+import datetime
 import json
 import os
 import statistics
@@ -34,7 +35,7 @@ ALGO_BYTES_PER_ACCESS = 41            # 24 B record in, 8 B completion + 8 B sta
 STAGE_BYTES = {"classify": 24 + 8 + 1, "plan_hist": 8, "scan": 8 + 4 + 24 + 16, "inorder": 24 + 16 + 1 + 4}
 # DRAM bytes per access of the in-order serve kernel from one ncu capture (dram__bytes_read + write over a
 # 20 M-access launch, profiles/inorder_path_capacity_20M.md); traffic grows in proportion to the batch
-NCU_TRAFFIC_BYTES_PER_ACCESS = {"inorder": 60.7}
+NCU_TRAFFIC_BYTES_PER_ACCESS = {"inorder": 60.9}
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -68,12 +69,13 @@ def measured_peak():
 
 
 class ClockSampler:
-    """nvidia-smi clocks and throttle reasons, sampled every 20 ms from the warm-up to the end of the timed region."""
-    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+    """nvidia-smi clocks and throttle reasons, sampled every 20 ms.  The sampler is started early (it needs a few
+    hundred ms to come up); only samples taken between mark_start() and mark_end() are reported."""
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
     def __init__(self, gpu_index: int):
-        self.gpu, self.proc = gpu_index, None
+        self.gpu, self.proc, self.t0, self.t1 = gpu_index, None, None, None
 
     def start(self):
         try:
@@ -83,6 +85,12 @@ class ClockSampler:
         except Exception:
             self.proc = None
 
+    def mark_start(self):
+        self.t0 = datetime.datetime.now()
+
+    def mark_end(self):
+        self.t1 = datetime.datetime.now()
+
     def stop(self) -> dict:
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
@@ -91,21 +99,26 @@ class ClockSampler:
             out, _ = self.proc.communicate(timeout=5)
         except Exception:
             self.proc.kill(); out = ""
-        sm, smax, reasons = [], [], set()
+        sm, smax, reasons, all_sm = [], [], set(), []
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in out.strip().splitlines():
             f = [x.strip() for x in line.split(",")]
             if len(f) < 9:
                 continue
             try:
-                sm.append(float(f[1])); smax.append(float(f[2]))
+                ts = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f")
+                mhz, mx = float(f[1]), float(f[2])
             except ValueError:
                 continue
+            all_sm.append(mhz)
+            if self.t0 is not None and self.t1 is not None and not (self.t0 <= ts <= self.t1):
+                continue
+            sm.append(mhz); smax.append(mx)
             for name, v in zip(names, f[5:9]):
                 if v.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "samples_whole_run": len(all_sm), "reasons": sorted(reasons)}
 
 
 # The batch spans seconds of simulated time while the thermal window that follows it is 1 ms, so the
@@ -241,6 +254,8 @@ def main():
     if world > 1:
         dist.barrier()
 
+    sampler = ClockSampler(local_rank)         # started now: it takes a few hundred ms before the first sample
+    sampler.start()
     n = args.n
     w, gen_s = make_stream(n, seed=replicas.rank_seed(0, rank))   # every rank: an independent replica on its own stream
     fp = wl.package_floorplan(channels=w.profile["channels"], dies=w.profile["dies"])
@@ -282,9 +297,8 @@ def main():
         return total
 
     ctx.set_profiling(True)
-    sampler = ClockSampler(local_rank)         # started before the warm-up (same load) so that short runs get samples
-    sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.mark_start()                       # the warm-up runs the same load as the timed steps
     timed(args.warmup, step)
     sync_all()
     res = ctx.last_result()
@@ -294,6 +308,7 @@ def main():
     sync_all()
     total_ms = timed(args.steps, step)
     sync_all()
+    sampler.mark_end()
     clocks = sampler.stop()
     launches = hbf.kernel_launches() - launches0
     # per-stage device times of a few more steps (events recorded between kernel groups on the same stream)
