@@ -86,7 +86,7 @@ struct Workspace {
     void *scan_desc;                     // [scan tiles] ScanDesc
     int64_t *in_agg;                     // [tiles][queues][2]: per-tile, per-queue max-plus aggregate (S, M)
     int64_t *in_bin;                     // [tiles][queues]: busy-until entering each tile
-    uint16_t *in_pos;                    // [n]: per 2,048-record chunk, the positions of its modeled records in queue-major order
+    uint16_t *in_pos;                    // [n]: per chunk, the positions of its modeled records in queue-major order
     uint16_t *in_start;                  // per chunk: [queues + 1] first queue-major position of every queue
     void *in_tile;                       // [tiles] stall bookkeeping of the in-order path
     void *in_head;                       // [tiles][queues][8]: the first accesses of every (tile, queue), for the fix-up

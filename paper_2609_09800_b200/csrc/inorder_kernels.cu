@@ -5,7 +5,7 @@
 //           serves its accesses AS IF every queue were idle when the tile begins; completions and stalls
 //           leave through shared memory in batch order.  Per queue it also keeps the composition (S, M) of
 //           the maps B -> max(B + s, a + s) of its accesses (M is exactly the busy-until of the as-if run),
-//           and per 2,048-record chunk it leaves the queue-major order of the chunk in the workspace;
+//           and per chunk it leaves the queue-major order of the chunk in the workspace;
 //   scan    one thread per queue walks the tiles' aggregates in order: the true busy-until entering each
 //           tile, and the final busy-until;
 //   fix-up  one thread per (tile, queue) starts from the true entering busy-until and re-serves that queue's
@@ -16,20 +16,29 @@
 // The serve pass is the only one that streams the batch: 24 B read and 16 B + 1 B written per access, plus
 // 4 B of order information.  Every global access of it is coalesced; nothing waits on another thread block.
 //
-// Inside a 2,048-record chunk the records are bucketed by queue in shared memory: one atomic per record
+// Inside a chunk (4,096 records) the records are bucketed by queue in shared memory: one atomic per record
 // takes a slot in its queue's bucket, an exclusive scan of the per-queue counts gives the bucket starts,
 // and each record then finds its index-order rank inside its (short) bucket by counting the smaller
 // positions.  A chunk with a long bucket is bucketed by a stable radix sort instead.  Thread t serves
-// the consecutive queues [t*qpt, (t+1)*qpt) one access after the other.
+// the queues whose first access of the chunk falls into its own positions of that order.
 #include <algorithm>
 
 #include "device_utils.cuh"
 
 namespace hbf {
 
-constexpr int kInThreads = 256;
-constexpr int kInItems = 8;
-constexpr int kInChunk = kInThreads * kInItems;          // 2048 records
+// Block shape of the serve kernel.  Measured on the 20 M capacity-mode batch (ms for the in-order group):
+// 256 x 8 records, 2 blocks/SM: 0.88; 512 x 4, 2 blocks/SM: 0.92; 512 x 8, 1 block/SM: 0.77; 1024 x 4, 1 block/SM: 0.72.
+// Larger chunks amortise the per-chunk work over the 2,048 queue bins; more warps hide shared-memory latency.
+#ifndef HBF_IN_THREADS
+#define HBF_IN_THREADS 1024
+#define HBF_IN_ITEMS 4
+#define HBF_IN_BLOCKS 1
+#endif
+constexpr int kInThreads = HBF_IN_THREADS;               // threads of a serve block
+constexpr int kInItems = HBF_IN_ITEMS;                   // records per thread and chunk
+constexpr int kInBlocksPerSM = HBF_IN_BLOCKS;            // resident serve blocks per SM (shared memory decides)
+constexpr int kInChunk = kInThreads * kInItems;          // 4096 records
 constexpr int kInWarps = kInThreads / 32;
 constexpr int kInDigitBits = 6;
 constexpr int kInBins = 1 << kInDigitBits;
@@ -110,7 +119,7 @@ struct InHead { int64_t m, s; uint32_t xo, idx; };       // arrival + service, s
 // pass from the true entering busy-until, writing the exact results and nothing else.
 // ======================================================================================================
 template <bool RESERVE>
-__global__ void __launch_bounds__(kInThreads, 2)
+__global__ void __launch_bounds__(kInThreads, kInBlocksPerSM)
 k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_records, const RangeSnap *__restrict__ ranges_g,
                 const ModelParams *__restrict__ mp_g, BatchCtrl *ctrl, uint8_t *__restrict__ status, int64_t *__restrict__ in_agg,
                 uint16_t *__restrict__ in_pos, uint16_t *__restrict__ in_start, uint32_t row_stride,
@@ -144,7 +153,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
     uint32_t *qcnt = reinterpret_cast<uint32_t *>(in_smem + kInSlotBytes);             // [R + 1] counts, then bucket starts
     uint16_t *posA = reinterpret_cast<uint16_t *>(in_smem + kInSlotBytes + kInCntBytes);
     uint16_t *posB = posA + kInChunk;                                                  // positions in queue-major order
-    int64_t *aggS = reinterpret_cast<int64_t *>(posB + kInChunk);                      // [2048] per-queue aggregate of the tile
+    int64_t *aggS = reinterpret_cast<int64_t *>(posB + kInChunk);                      // [queues] per-queue aggregate of the tile
     int64_t *aggM = aggS + kInMaxQueues;
     uint32_t *st_br_lo = reinterpret_cast<uint32_t *>(aggM + kInMaxQueues), *st_br_hi = st_br_lo + n_dies;   // per die
     uint32_t *st_bp_lo = st_br_hi + n_dies, *st_bp_hi = st_bp_lo + n_dies;
@@ -667,7 +676,7 @@ __global__ void k_inorder_total(BatchCtrl *ctrl, const InTile *__restrict__ in_t
 }
 
 uint64_t inorder_tile_records(uint64_t n, int sm_count) {
-    const uint64_t want_tiles = std::min<uint64_t>(kInMaxTiles, (uint64_t)std::max(1, sm_count) * 2);   // two thread blocks per SM: one wave
+    const uint64_t want_tiles = std::min<uint64_t>(kInMaxTiles, (uint64_t)std::max(1, sm_count) * kInBlocksPerSM);   // one wave of resident blocks
     uint64_t t = (n + want_tiles - 1) / want_tiles;
     t = (t + kInChunk - 1) / kInChunk * kInChunk;
     return std::max<uint64_t>(t, kInChunk);

@@ -659,7 +659,7 @@ size_t workspace_layout(uint64_t n, uint32_t n_queues, Workspace *ws, void *base
     const uint64_t in_tiles = std::min<uint64_t>(kInMaxTiles, (nn + 2047) / 2048);
     const bool inorder = n_queues <= kInMaxQueues;
     void *ia = take(inorder ? in_tiles * n_queues * 16 : 0), *ib = take(inorder ? in_tiles * n_queues * 8 : 0);
-    void *ii = take(inorder ? (nn + 2048) * 2 : 0), *is = take(inorder ? inorder_start_bytes(nn, n_queues) : 0);
+    void *ii = take(inorder ? (nn + 8192) * 2 : 0), *is = take(inorder ? inorder_start_bytes(nn, n_queues) : 0);
     void *it = take(inorder ? in_tiles * 32 : 0), *ih = take(inorder ? inorder_head_bytes(in_tiles, n_queues) : 0);
     void *ic = take(inorder ? in_tiles * n_queues : 0), *il = take(inorder ? (1 + in_tiles * n_queues) * 4 : 0);
     if (ws) {
