@@ -34,7 +34,7 @@ ALGO_BYTES_PER_ACCESS = 41            # 24 B record in, 8 B completion + 8 B sta
 # algorithmic bytes per access of each kernel group (what the kernel itself must move)
 STAGE_BYTES = {"classify": 24 + 8 + 1, "plan_hist": 8, "scan": 8 + 4 + 24 + 16, "inorder": 24 + 16 + 1 + 4}
 # DRAM bytes per access of the in-order serve kernel from one ncu capture (dram__bytes_read + write over a
-# 20 M-access launch, profiles/inorder_path_capacity_20M.md); traffic grows in proportion to the batch
+# 20 M-access launch, see the summary under profiles/); traffic grows in proportion to the batch
 NCU_TRAFFIC_BYTES_PER_ACCESS = {"inorder": 49.3}
 FALLBACK_HBM_GBS = 6650.0
 
