@@ -156,7 +156,7 @@ int hbf_create(const hbf_config_t *cfg, void *cuda_stream, hbf_ctx **out) {
     {   // the in-order path packs the transfer time of an access into 31 bits and keeps per-queue state in shared memory
         const unsigned __int128 worst = ((unsigned __int128)0xffffffffull + std::max(cfg->read_granule, cfg->prog_granule)) * 1000u;
         c->inorder_ok = nq <= kInMaxQueues && worst / cfg->chan_bytes_per_us < ((unsigned __int128)1 << 31) &&
-                        172u * 1024u + nd * 24u <= 224u * 1024u;
+                        inorder_serve_smem((uint32_t)nd) + 8u * 1024u <= 227u * 1024u;
     }
     {   // transfer times of the small charged sizes, looked up instead of divided (every charged size is a multiple of its granule)
         const uint32_t g = std::min(mp.read_gran_shift, mp.prog_gran_shift);

@@ -114,6 +114,7 @@ size_t workspace_layout(uint64_t n, uint32_t n_queues, Workspace *ws, void *base
 uint64_t inorder_tile_records(uint64_t n, int sm_count);
 size_t inorder_start_bytes(uint64_t n, uint32_t n_queues);
 size_t inorder_head_bytes(uint64_t tiles, uint32_t n_queues);
+size_t inorder_serve_smem(uint32_t n_dies);
 cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st);
 cudaError_t launch_submit(const SubmitArgs &a, cudaStream_t st);
 cudaError_t launch_queue_order(const BatchCtrl *ctrl, const Workspace &ws, uint32_t *out, uint64_t n, cudaStream_t st);

@@ -30,8 +30,10 @@ namespace hbf {
 // Block shape of the serve kernel.  Measured on the 20 M capacity-mode batch (ms for the in-order group):
 // 256 x 8 records, 2 blocks/SM: 0.88; 512 x 4, 2 blocks/SM: 0.92; 512 x 8, 1 block/SM: 0.77; 1024 x 4, 1 block/SM: 0.72.
 // Larger chunks amortise the per-chunk work over the 2,048 queue bins; more warps hide shared-memory latency.
+// With one block per SM nothing hides the chunk's load, so the records arrive by bulk asynchronous copy (TMA)
+// into one of two buffers while the previous chunk is being served; two 3,072-record buffers fit, two 4,096 do not.
 #ifndef HBF_IN_THREADS
-#define HBF_IN_THREADS 1024
+#define HBF_IN_THREADS 768
 #define HBF_IN_ITEMS 4
 #define HBF_IN_BLOCKS 1
 #endif
@@ -134,6 +136,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
     __shared__ long long s_red[2];
     __shared__ FastRange s_fast;
     __shared__ uint32_t s_heads_full;                     // queues whose head entries are complete
+    __shared__ __align__(8) uint64_t s_mbar[2];           // one per record buffer: completion of its bulk load
 
     if (ctrl->skip) return;
     if (RESERVE && (ctrl->run_sort || !ctrl->inorder_used || !in_tile[blockIdx.x].reserve)) return;
@@ -149,9 +152,9 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
     }
 
     // slot e holds record e on arrival, then its served image (in place)
-    uint64_t *slot = reinterpret_cast<uint64_t *>(in_smem);
-    uint32_t *qcnt = reinterpret_cast<uint32_t *>(in_smem + kInSlotBytes);             // [R + 1] counts, then bucket starts
-    uint16_t *posA = reinterpret_cast<uint16_t *>(in_smem + kInSlotBytes + kInCntBytes);
+    uint64_t *slot_buf[2] = {reinterpret_cast<uint64_t *>(in_smem), reinterpret_cast<uint64_t *>(in_smem + kInSlotBytes)};
+    uint32_t *qcnt = reinterpret_cast<uint32_t *>(in_smem + 2 * kInSlotBytes);         // [R + 1] counts, then bucket starts
+    uint16_t *posA = reinterpret_cast<uint16_t *>(in_smem + 2 * kInSlotBytes + kInCntBytes);
     uint16_t *posB = posA + kInChunk;                                                  // positions in queue-major order
     int64_t *aggS = reinterpret_cast<int64_t *>(posB + kInChunk);                      // [queues] per-queue aggregate of the tile
     int64_t *aggM = aggS + kInMaxQueues;
@@ -191,16 +194,37 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
     if (tid < 2) s_red[tid] = tid == 1 ? INT64_MIN : 0;
     if (tid == 0) s_heads_full = 0u;
 
-    for (uint64_t cbase = tile_begin; cbase < tile_end; cbase += kInChunk) {
+    // Full chunks of a 16-byte aligned batch arrive by bulk asynchronous copy; the last, partial chunk of a tile
+    // and unaligned batches are loaded by the threads.
+    constexpr uint32_t kChunkBytes = (uint32_t)kInChunk * 24u;
+    auto prefetch = [&](uint64_t cb, uint32_t buf) {       // thread 0, after a block barrier that retired the buffer's last use
+        if (aligned16 && cb < tile_end && tile_end - cb >= (uint64_t)kInChunk) {
+            mbar_expect_tx(&s_mbar[buf], kChunkBytes);
+            bulk_load(slot_buf[buf], acc + cb, kChunkBytes, &s_mbar[buf]);
+        }
+    };
+    if (tid == 0) { mbar_init(&s_mbar[0], 1u); mbar_init(&s_mbar[1], 1u); }
+    __syncthreads();
+    if (tid == 0) prefetch(tile_begin, 0u);
+    uint32_t parity_bits = 0u;                              // bit b: parity of buffer b's next completed phase
+    uint32_t chunk_no = 0u;
+
+    for (uint64_t cbase = tile_begin; cbase < tile_end; cbase += kInChunk, ++chunk_no) {
         const int cnt = (int)min((uint64_t)kInChunk, tile_end - cbase);
+        const uint32_t buf = chunk_no & 1u;
+        uint64_t *slot = slot_buf[buf];
         __syncthreads();                                   // the previous chunk has left shared memory
-        // ---- load: 16-byte coalesced loads of the 24-byte records; clear the per-queue counts ----------
+        if (tid == 0) prefetch(cbase + kInChunk, buf ^ 1u);   // the next chunk lands while this one is served
+        // ---- load: bulk copy issued one chunk ahead, or 16-byte coalesced loads; clear the per-queue counts ----------
         const uint64_t *src = reinterpret_cast<const uint64_t *>(acc + cbase);
         if (cnt == kInChunk && aligned16) {
-            const uint4 *s4 = reinterpret_cast<const uint4 *>(src);
-            uint4 *d4 = reinterpret_cast<uint4 *>(slot);
-#pragma unroll
-            for (int k = 0; k < kInChunk * 24 / 16 / kInThreads; ++k) d4[tid + k * kInThreads] = __ldg(s4 + tid + k * kInThreads);
+            const bool arrived = mbar_wait_bounded(&s_mbar[buf], (parity_bits >> buf) & 1u);
+            parity_bits ^= 1u << buf;
+            if (__syncthreads_or(arrived ? 0 : 1)) {       // the copy did not complete in time: give the batch up
+                if (tid == 0) atomicExch(&ctrl->code, (int)HBF_E_TIMEOUT);
+                mbar_wait_bounded(&s_mbar[buf ^ 1u], (parity_bits >> (buf ^ 1u)) & 1u);   // let the copy in flight land, within the same limit
+                return;
+            }
         } else {
             for (int i = tid; i < cnt * 3; i += kInThreads) slot[i] = __ldg(src + i);
         }
@@ -682,6 +706,11 @@ uint64_t inorder_tile_records(uint64_t n, int sm_count) {
     return std::max<uint64_t>(t, kInChunk);
 }
 
+// dynamic shared memory of the serve kernel: two record buffers, counts, two position buffers, aggregates, per-die counters, head fill
+size_t inorder_serve_smem(uint32_t n_dies) {
+    return (size_t)2 * kInSlotBytes + kInCntBytes + 2 * kInPosBytes + (size_t)kInMaxQueues * 16 + (size_t)n_dies * 24 + kInMaxQueues;
+}
+
 static uint32_t inorder_row_stride(uint32_t n_queues) { return (n_queues + 1u + 7u) / 8u * 8u; }
 size_t inorder_head_bytes(uint64_t tiles, uint32_t n_queues) { return tiles * n_queues * (size_t)kInHead * sizeof(InHead); }
 size_t inorder_start_bytes(uint64_t n, uint32_t n_queues) {
@@ -693,8 +722,7 @@ cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st) {
     const uint64_t tile_records = inorder_tile_records(n, a.sm_count);
     const unsigned n_tiles = (unsigned)((n + tile_records - 1) / tile_records);
     const uint32_t R = a.mp.n_queues, nd = a.mp.n_dies, row_stride = inorder_row_stride(R);
-    const size_t smem_serve = (size_t)kInSlotBytes + kInCntBytes + 2 * kInPosBytes + (size_t)kInMaxQueues * 16 + (size_t)nd * 24 +
-                              kInMaxQueues;
+    const size_t smem_serve = inorder_serve_smem(nd);
     static size_t set_serve = 0;
     if (smem_serve > set_serve) {
         cudaError_t e = cudaFuncSetAttribute(k_inorder_serve<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_serve);

@@ -603,6 +603,7 @@ __global__ void k_finish(uint64_t n, BatchCtrl *ctrl, DevState *state, int64_t *
                          const ModelParams *__restrict__ mp, uint32_t n_queues, uint32_t n_dies) {
     const int code = ctrl->code;
     const uint64_t gtid = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (code == HBF_E_TIMEOUT && gtid == 0) state->poisoned = 1;         // a bounded device-side wait expired
     const uint64_t gsz = (uint64_t)gridDim.x * blockDim.x;
     if (code == HBF_E_ACCESS_FAULT || code == HBF_E_TIMEOUT || code == HBF_E_INVAL) {
         for (uint64_t i = gtid; i < n; i += gsz) { completion[i] = 0; stall[i] = 0; }
