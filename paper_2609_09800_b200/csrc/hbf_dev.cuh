@@ -86,12 +86,9 @@ struct Workspace {
     void *scan_desc;                     // [scan tiles] ScanDesc
     int64_t *in_agg;                     // [tiles][queues][2]: per-tile, per-queue max-plus aggregate (S, M)
     int64_t *in_bin;                     // [tiles][queues]: busy-until entering each tile
-    uint16_t *in_pos;                    // [n]: per chunk, the positions of its modeled records in queue-major order
-    uint16_t *in_start;                  // per chunk: [queues + 1] first queue-major position of every queue
     void *in_tile;                       // [tiles] stall bookkeeping of the in-order path
     void *in_head;                       // [tiles][queues][8]: the first accesses of every (tile, queue), for the fix-up
-    uint8_t *in_headcnt;                 // [tiles][queues]: how many of them exist
-    uint32_t *in_list;                   // [1 + tiles*queues]: count, then the (tile, queue) pairs the long fix-up handles
+    uint8_t *in_headcnt;                 // [tiles][queues]: how many of them exist; 0xff marks a queue for the straggle pass
     size_t bytes;
 };
 
@@ -112,7 +109,6 @@ constexpr uint32_t kInMaxTiles = 512;
 size_t workspace_layout(uint64_t n, uint32_t n_queues, Workspace *ws, void *base);
 // tile size (records) of the in-order path for a batch of n on a device with sm_count SMs
 uint64_t inorder_tile_records(uint64_t n, int sm_count);
-size_t inorder_start_bytes(uint64_t n, uint32_t n_queues);
 size_t inorder_head_bytes(uint64_t tiles, uint32_t n_queues);
 size_t inorder_serve_smem(uint32_t n_dies);
 cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st);

@@ -1,59 +1,74 @@
 // In-order path of hbf_submit_batch: serves a batch whose records arrive in non-decreasing issue order
 // without a global sort.  In such a batch the (issue, index) order of every queue is plain index order,
-// so the batch is cut into a few hundred contiguous tiles that are served independently, in one pass:
-//   serve   every tile classifies and decodes its records, writes status[], counts, sums per-die bytes, and
-//           serves its accesses AS IF every queue were idle when the tile begins; completions and stalls
-//           leave through shared memory in batch order.  Per queue it also keeps the composition (S, M) of
-//           the maps B -> max(B + s, a + s) of its accesses (M is exactly the busy-until of the as-if run),
-//           and per chunk it leaves the queue-major order of the chunk in the workspace;
-//   scan    one thread per queue walks the tiles' aggregates in order: the true busy-until entering each
-//           tile, and the final busy-until;
-//   fix-up  one thread per (tile, queue) starts from the true entering busy-until and re-serves that queue's
-//           accesses of the tile in order, until it meets an access that arrives when the queue is idle:
-//           from there on the as-if run and the true run coincide (busy-until is monotone in its start
-//           value, so the as-if run was idle there too).  At moderate load this touches a few accesses
-//           per (tile, queue); under overload it degrades to re-serving everything, still exactly.
-// The serve pass is the only one that streams the batch: 24 B read and 16 B + 1 B written per access, plus
-// 4 B of order information.  Every global access of it is coalesced; nothing waits on another thread block.
+// so the batch is cut into contiguous tiles, one per SM, that are served independently, in one pass:
+//   serve     every tile classifies and decodes its records, writes status[], counts, sums per-die bytes, and
+//             serves its accesses AS IF every queue were idle when the tile begins; completions and stalls
+//             leave through shared memory in batch order.  Per queue it also keeps the composition (S, M) of
+//             the maps B -> max(B + s, a + s) of its accesses (M is exactly the busy-until of the as-if run)
+//             and the first few accesses of the queue in the tile (the head table);
+//   scan      one thread per queue walks the tiles' aggregates in order: the true busy-until entering each
+//             tile, and the final busy-until;
+//   fix-up    one thread per (tile, queue) starts from the true entering busy-until and re-serves the head
+//             table's accesses in order, until it meets an access that arrives when the queue is idle: from
+//             there on the as-if run and the true run coincide (busy-until is monotone in its start value, so
+//             the as-if run was idle there too);
+//   straggle  a queue still backlogged past its head entries is re-served from the records: the tile's
+//             block streams the tile again, keeps only that tile's straggling queues, and stops as soon as
+//             each of them has fallen idle;
+//   re-serve  a tile with many stragglers (the batch arrived on queues that were far behind) is served
+//             again from the true entering busy-until, exactly.
+// The serve pass is the only one that streams the whole batch: 24 B read and 16 B + 1 B written per access.
+// Every global access of it is coalesced; nothing waits on another thread block.
 //
-// Inside a chunk (4,096 records) the records are bucketed by queue in shared memory: one atomic per record
-// takes a slot in its queue's bucket, an exclusive scan of the per-queue counts gives the bucket starts,
-// and each record then finds its index-order rank inside its (short) bucket by counting the smaller
-// positions.  A chunk with a long bucket is bucketed by a stable radix sort instead.  Thread t serves
-// the queues whose first access of the chunk falls into its own positions of that order.
+// Inside a chunk (3,072 records) the queue dependency is resolved by the warps acting as servers: queues are
+// hashed onto the block's warps, every record is appended, in batch order, to the list of its queue's warp
+// (ranking by warp match, offsets by a small scan), and each warp then walks its list 32 records at a time.
+// The busy-until of every queue lives in shared memory; records of one queue that fall into the same group
+// of 32 are chained in registers with shuffles.  Different warps never touch the same queue.
 #include <algorithm>
 
 #include "device_utils.cuh"
 
 namespace hbf {
 
-// Block shape of the serve kernel.  Measured on the 20 M capacity-mode batch (ms for the in-order group):
-// 256 x 8 records, 2 blocks/SM: 0.88; 512 x 4, 2 blocks/SM: 0.92; 512 x 8, 1 block/SM: 0.77; 1024 x 4, 1 block/SM: 0.72.
-// Larger chunks amortise the per-chunk work over the 2,048 queue bins; more warps hide shared-memory latency.
-// With one block per SM nothing hides the chunk's load, so the records arrive by bulk asynchronous copy (TMA)
-// into one of two buffers while the previous chunk is being served; two 3,072-record buffers fit, two 4,096 do not.
+// Block shape of the serve kernel: one block per SM; the records arrive by bulk asynchronous copy (TMA)
+// into one of two buffers while the previous chunk is being served.
 #ifndef HBF_IN_THREADS
-#define HBF_IN_THREADS 768
-#define HBF_IN_ITEMS 4
-#define HBF_IN_BLOCKS 1
+#define HBF_IN_THREADS 640
+#define HBF_IN_ITEMS 5
 #endif
 constexpr int kInThreads = HBF_IN_THREADS;               // threads of a serve block
 constexpr int kInItems = HBF_IN_ITEMS;                   // records per thread and chunk
-constexpr int kInBlocksPerSM = HBF_IN_BLOCKS;            // resident serve blocks per SM (shared memory decides)
-constexpr int kInChunk = kInThreads * kInItems;          // 4096 records
+constexpr int kInBlocksPerSM = 1;
+constexpr int kInChunk = kInThreads * kInItems;          // records per chunk
 constexpr int kInWarps = kInThreads / 32;
-constexpr int kInDigitBits = 6;
-constexpr int kInBins = 1 << kInDigitBits;
-constexpr int kInGroup = 4;                              // accesses a thread loads at once while serving
-constexpr int kInMaxBucket = 16;                         // longer buckets take the radix route
-constexpr uint32_t kInNoQueue = 0xffffu;                 // record is not modeled (native or refused)
+constexpr int kInServers = kInWarps;                     // every warp serves the queues hashed onto it
+constexpr int kInCells = kInItems * kInWarps;            // (row, warp) cells of one server's line of the count matrix
+constexpr int kInCellsPerLane = (kInCells + 31) / 32;
 constexpr int kInSlotBytes = kInChunk * 24;
-constexpr int kInCntBytes = (kInMaxQueues + 64) * 4;
-constexpr int kInPosBytes = kInChunk * 2;
+constexpr int kInServerBits = kInServers < 16 ? 4 : (kInServers < 32 ? 5 : 6);   // bits of a server number, "none" included
+static_assert(kInServers <= 32, "one lane per server in the offset scan");
+static_assert(kInChunk <= 65536, "positions inside a chunk are 16-bit");
+static_assert((kInServers * kInCells) % 2 == 0, "count matrix is cleared by 32-bit words");
 
-// word 2 of a slot: transfer ns (31 bits) | op << 31 | queue << 32 | slot taken in the queue's bucket << 48
-__device__ __forceinline__ uint32_t img_queue(uint64_t w2) { return (uint32_t)(w2 >> 32) & 0xffffu; }
-__device__ __forceinline__ uint32_t img_place(uint64_t w2) { return (uint32_t)(w2 >> 48); }
+// Lanes of the warp whose low BITS bits of v equal this lane's: one ballot per bit.
+template <int BITS>
+__device__ __forceinline__ unsigned match_bits(uint32_t v) {
+    unsigned m = 0xffffffffu;
+#pragma unroll
+    for (int b = 0; b < BITS; ++b) {
+        const bool one = ((v >> b) & 1u) != 0u;
+        const unsigned bal = __ballot_sync(0xffffffffu, one);
+        m &= one ? bal : ~bal;
+    }
+    return m;
+}
+
+// Which warp serves queue q.  A multiplicative hash, so that streams that step through channels, dies or
+// planes at a fixed stride still spread over all warps.
+__device__ __forceinline__ uint32_t server_of(uint32_t q) {
+    return ((((q + 1u) * 0x9E3779B1u) >> 16) * (uint32_t)kInServers) >> 16;
+}
 
 // One access, from its record: status, and for a modeled access its queue, die and service terms.
 struct Served { int st; uint32_t queue, die, op; int64_t s, xfer, cb; };
@@ -102,37 +117,37 @@ __device__ __forceinline__ Served serve_terms_fast(const FastRange &f, const Mod
     r.s = (int64_t)npages * (r.op ? mp.t_prog_ns : mp.t_read_ns);
     return r;
 }
-
-// index of a queue's state in the shared-memory arrays
-__device__ __forceinline__ uint32_t state_index(uint32_t q, uint32_t qpt_shift) {
-    (void)qpt_shift;
-    return q;
-}
-
 // per-tile bookkeeping of the stall total: as-if-idle sum, fix-up corrections, and the exact sum of a re-served tile
 struct InTile { long long spec_sum, fix_delta, true_sum; uint32_t reserve; uint32_t stragglers; };
 // The first kInHead accesses of every (tile, queue), as the serve pass saw them: all the fix-up needs in the common case.
 constexpr int kInHead = 8;
+constexpr uint8_t kInStraggler = 0xffu;                   // head count of a (tile, queue) the fix-up hands to the straggle pass
 struct InHead { int64_t m, s; uint32_t xo, idx; };       // arrival + service, service, transfer | op << 31, batch index
+
+// A served record in shared memory (three 64-bit words, in place of the record it came from):
+//   word 0  service ns (32 bits) | transfer ns (20 bits) << 32 | op << 52 | queue << 53
+//   word 1  issue time, as it arrived
+//   word 2  arrival at the queue (issue, plus the transfer for a program) until the record has been served,
+//           its completion time afterwards
+// (for a record that is not modeled word 2 holds the issue time from the start: completion = issue, no stall).
+// A batch with a service time of 2^32 ns or a transfer of 2^20 ns or more in one access goes to the sort path.
+constexpr uint32_t kInXferBits = 20;
+static_assert(kInMaxQueues <= (1u << (64 - 53)), "queue field of a served record");
 
 // ======================================================================================================
 // serve.  RESERVE = false: the streaming pass over every tile, every queue taken as idle at the tile's start.
-// RESERVE = true: only for tiles the fix-up flagged (a queue stayed backlogged far into the tile): the same
-// pass from the true entering busy-until, writing the exact results and nothing else.
+// RESERVE = true: only for tiles the fix-up flagged (many queues stayed backlogged far into the tile): the
+// same pass from the true entering busy-until, writing the exact results and nothing else.
 // ======================================================================================================
 template <bool RESERVE>
 __global__ void __launch_bounds__(kInThreads, kInBlocksPerSM)
 k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_records, const RangeSnap *__restrict__ ranges_g,
                 const ModelParams *__restrict__ mp_g, BatchCtrl *ctrl, uint8_t *__restrict__ status, int64_t *__restrict__ in_agg,
-                uint16_t *__restrict__ in_pos, uint16_t *__restrict__ in_start, uint32_t row_stride,
                 hbf_die_stats_t *stats_stage, int64_t *__restrict__ completion, int64_t *__restrict__ stall,
                 const int64_t *__restrict__ in_bin, InTile *in_tile, InHead *__restrict__ in_head, uint8_t *__restrict__ in_headcnt) {
     extern __shared__ __align__(16) unsigned char in_smem[];
     __shared__ ModelParams mp;
-    __shared__ uint32_t s_cnt[kInWarps * kInBins];        // radix route only
-    __shared__ uint32_t s_bin_start[kInBins];
-    __shared__ uint32_t s_bin_warp[2];
-    __shared__ uint32_t s_warp_tot[kInWarps];
+    __shared__ uint32_t s_stot[32];                       // records of the chunk per server
     __shared__ long long s_red[2];
     __shared__ FastRange s_fast;
     __shared__ uint32_t s_heads_full;                     // queues whose head entries are complete
@@ -151,38 +166,28 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
         s_fast = f;
     }
 
-    // slot e holds record e on arrival, then its served image (in place)
     uint64_t *slot_buf[2] = {reinterpret_cast<uint64_t *>(in_smem), reinterpret_cast<uint64_t *>(in_smem + kInSlotBytes)};
-    uint32_t *qcnt = reinterpret_cast<uint32_t *>(in_smem + 2 * kInSlotBytes);         // [R + 1] counts, then bucket starts
-    uint16_t *posA = reinterpret_cast<uint16_t *>(in_smem + 2 * kInSlotBytes + kInCntBytes);
-    uint16_t *posB = posA + kInChunk;                                                  // positions in queue-major order
-    int64_t *aggS = reinterpret_cast<int64_t *>(posB + kInChunk);                      // [queues] per-queue aggregate of the tile
-    int64_t *aggM = aggS + kInMaxQueues;
-    uint32_t *st_br_lo = reinterpret_cast<uint32_t *>(aggM + kInMaxQueues), *st_br_hi = st_br_lo + n_dies;   // per die
+    // [queues] x: busy-until of the run in progress; y: service time served in this tile << 8 | head-table entries written
+    longlong2 *qst = reinterpret_cast<longlong2 *>(in_smem + 2 * kInSlotBytes);
+    uint16_t *list = reinterpret_cast<uint16_t *>(qst + kInMaxQueues);                 // [chunk] positions, server-major, batch order inside
+    uint16_t *cntm = list + kInChunk;                                                  // [server][row][warp] counts, then offsets
+    uint32_t *st_br_lo = reinterpret_cast<uint32_t *>(cntm + kInServers * kInCells), *st_br_hi = st_br_lo + n_dies;   // per die
     uint32_t *st_bp_lo = st_br_hi + n_dies, *st_bp_hi = st_bp_lo + n_dies;
     uint32_t *st_nr = st_bp_hi + n_dies, *st_np = st_nr + n_dies;
-    uint8_t *hfill = reinterpret_cast<uint8_t *>(st_np + n_dies);                  // head-table entries written per queue
 
     const uint32_t tile = blockIdx.x;
     const uint64_t tile_begin = (uint64_t)tile * tile_records;
     const uint64_t tile_end = min(n, tile_begin + tile_records);
 
-    // queues per thread, rounded up to a power of two
-    uint32_t qpt_shift = 0;
-    while (((uint32_t)kInThreads << qpt_shift) < R) ++qpt_shift;
-    const uint32_t qpt = 1u << qpt_shift;
-
-    for (uint32_t i = tid; i < kInMaxQueues; i += kInThreads) { aggS[i] = 0; aggM[i] = kNegInf; }
+    for (uint32_t i = tid; i < kInMaxQueues; i += kInThreads) qst[i] = make_longlong2(kNegInf, 0);
+    for (uint32_t i = tid; i < (uint32_t)(kInServers * kInCells / 2); i += kInThreads) reinterpret_cast<uint32_t *>(cntm)[i] = 0u;
     if (RESERVE) {
         __syncthreads();
-        for (uint32_t q = tid; q < R; q += kInThreads) aggM[state_index(q, qpt_shift)] = in_bin[(uint64_t)blockIdx.x * R + q];
+        for (uint32_t q = tid; q < R; q += kInThreads) qst[q].x = in_bin[(uint64_t)blockIdx.x * R + q];
     } else {
         for (uint32_t d = tid; d < n_dies * 6u; d += kInThreads) st_br_lo[d] = 0u;
-        for (uint32_t i = tid; i < kInMaxQueues; i += kInThreads) hfill[i] = 0;
     }
 
-    const uint32_t qbits = 32u - (uint32_t)__clz((int)R);
-    const uint32_t n_pass = (qbits + kInDigitBits - 1) / kInDigitBits;
     const int64_t q_ppm = ctrl->q_ppm;
     const Div64 div_q = ctrl->div_q;
     const bool aligned16 = (reinterpret_cast<uintptr_t>(acc) & 15u) == 0;
@@ -213,28 +218,26 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
         const int cnt = (int)min((uint64_t)kInChunk, tile_end - cbase);
         const uint32_t buf = chunk_no & 1u;
         uint64_t *slot = slot_buf[buf];
-        __syncthreads();                                   // the previous chunk has left shared memory
-        if (tid == 0) prefetch(cbase + kInChunk, buf ^ 1u);   // the next chunk lands while this one is served
-        // ---- load: bulk copy issued one chunk ahead, or 16-byte coalesced loads; clear the per-queue counts ----------
-        const uint64_t *src = reinterpret_cast<const uint64_t *>(acc + cbase);
-        if (cnt == kInChunk && aligned16) {
-            const bool arrived = mbar_wait_bounded(&s_mbar[buf], (parity_bits >> buf) & 1u);
-            parity_bits ^= 1u << buf;
-            if (__syncthreads_or(arrived ? 0 : 1)) {       // the copy did not complete in time: give the batch up
-                if (tid == 0) atomicExch(&ctrl->code, (int)HBF_E_TIMEOUT);
-                mbar_wait_bounded(&s_mbar[buf ^ 1u], (parity_bits >> (buf ^ 1u)) & 1u);   // let the copy in flight land, within the same limit
-                return;
-            }
+                // ---- load: bulk copy issued one chunk ahead, or 16-byte coalesced loads.  The buffer's last readers (the
+        // write-out of two chunks ago) finished before the previous chunk's first barrier.
+        const bool bulk = cnt == kInChunk && aligned16;
+        const uint32_t par = (parity_bits >> buf) & 1u;
+        int timed_out = 0;
+        if (bulk) {
+            timed_out = mbar_wait_bounded(&s_mbar[buf], par) ? 0 : 1;   // on expiry the buffer's content is arbitrary but every
+            parity_bits ^= 1u << buf;                                    // index derived from it stays in range; the barrier below ends the batch
         } else {
+            const uint64_t *src = reinterpret_cast<const uint64_t *>(acc + cbase);
             for (int i = tid; i < cnt * 3; i += kInThreads) slot[i] = __ldg(src + i);
+            __syncthreads();
         }
-        for (uint32_t q = tid; q <= R; q += kInThreads) qcnt[q] = 0u;
-        __syncthreads();
-        // ---- terms, in place: classify, decode, service; take a slot in the queue's bucket.  Word 1 (the issue
-        // time) stays as it is until the queues are served, so the issue-order check can read the neighbour's.
+        // ---- terms, in place: classify, decode, service; rank the record among its warp's records for the same
+        // server.  Word 1 (the issue time) stays as it is, so the issue-order check can read the neighbour's.
+        uint32_t pk[kInItems];                               // rank among the warp's records of this row for the same server | server << 5
 #pragma unroll
         for (int j = 0; j < kInItems; ++j) {
             const int e = j * kInThreads + tid;
+            uint32_t srv = (uint32_t)kInServers;             // not modeled
             if (e < cnt) {
                 const uint64_t addr = slot[e * 3];
                 const int64_t issue = (int64_t)slot[e * 3 + 1];
@@ -245,12 +248,15 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
                 const Served v = s_fast.on ? serve_terms_fast(s_fast, mp, addr, issue, slot[e * 3 + 2])
                                            : serve_terms(rs, mp, addr, issue, slot[e * 3 + 2], q_ppm, div_q);
                 if (!RESERVE && status) status[cbase + e] = (uint8_t)v.st;
-                uint64_t w0 = 0, w2 = (uint64_t)kInNoQueue << 32;
+                uint64_t w2 = (uint64_t)issue;               // not modeled: completion = issue (a refused batch is cleared at the end)
                 if (v.st == HBF_ST_READY) {
-                    const uint32_t o = atomicAdd(&qcnt[v.queue], 1u);
-                    w0 = (uint64_t)v.s;
-                    w2 = (uint64_t)((uint32_t)v.xfer | (v.op << 31)) | ((uint64_t)v.queue << 32) | ((uint64_t)o << 48);
+                    srv = server_of(v.queue);
+                    const uint32_t xq = ((uint32_t)v.xfer & ((1u << kInXferBits) - 1u)) | (v.op << kInXferBits) | (v.queue << (kInXferBits + 1));
+                    slot[e * 3] = (uint64_t)(uint32_t)v.s | ((uint64_t)xq << 32);
+                    w2 = (uint64_t)(issue + (v.op ? v.xfer : 0));
                     if (!RESERVE) {
+                        // a service time beyond 32 bits or a transfer beyond 20 bits goes to the sort path
+                        c_unsorted |= (((uint64_t)v.s >> 32) | ((uint64_t)v.xfer >> kInXferBits)) != 0ull ? 1u : 0u;
                         ++c_ready;
                         // charged bytes < 2^33: add the low word, carry into the high word when it wraps
                         const uint32_t lo = (uint32_t)v.cb, hi = (uint32_t)((uint64_t)v.cb >> 32);
@@ -261,215 +267,129 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
                         if (carry) atomicAdd(&phi[v.die], carry);
                     }
                 } else if (v.st == HBF_ST_NATIVE) {
-                    w0 = (uint64_t)issue;                    // native: completion = issue, stall = 0
                     ++c_native;
                 } else {
                     ++c_fault;
                 }
-                slot[e * 3] = w0; slot[e * 3 + 2] = w2;
+                slot[e * 3 + 2] = w2;
             }
+            const unsigned peers = match_bits<kInServerBits>(srv);     // five ballots: measured faster here than match.any
+            const uint32_t rk = (uint32_t)__popc(peers & lanemask_lt());
+            if (rk == 0u && srv < (uint32_t)kInServers) cntm[(srv * kInItems + j) * kInWarps + warp] = (uint16_t)__popc(peers);
+            pk[j] = rk | (srv << 5);
         }
-        __syncthreads();
-        // ---- bucket starts: exclusive scan of the counts in queue order; qcnt[R] = modeled records ---------
-        int use_radix;
+        if (__syncthreads_or(timed_out)) {                 // a bulk copy did not complete in time: give the batch up
+            if (tid == 0) atomicExch(&ctrl->code, (int)HBF_E_TIMEOUT);
+            if (bulk) mbar_wait_bounded(&s_mbar[buf], par);  // let the copy in flight land, within the same limit
+            return;
+        }
+        if (tid == 0) prefetch(cbase + kInChunk, buf ^ 1u);   // the next chunk lands while this one is served
+        // ---- offsets: warp w turns the counts of server w, in (row, warp) order, into offsets inside its list --------
         {
-            const uint32_t q0 = (uint32_t)tid * qpt;
-            uint32_t c[8], tot = 0, longest = 0;
-            if (qpt == 8u) {                               // full width: two 16-byte loads, free of bank conflicts
-                const uint4 lo = *reinterpret_cast<const uint4 *>(qcnt + q0), hi = *reinterpret_cast<const uint4 *>(qcnt + q0 + 4);
-                c[0] = lo.x; c[1] = lo.y; c[2] = lo.z; c[3] = lo.w; c[4] = hi.x; c[5] = hi.y; c[6] = hi.z; c[7] = hi.w;
-            } else {
+            uint16_t *m = cntm + warp * kInCells;
+            uint32_t c[kInCellsPerLane], tot = 0;
 #pragma unroll
-                for (int b = 0; b < 8; ++b) c[b] = ((uint32_t)b < qpt && q0 + b < R) ? qcnt[q0 + b] : 0u;
-            }
-#pragma unroll
-            for (int b = 0; b < 8; ++b) {
-                if (q0 + b >= R) c[b] = 0u;
-                longest = max(longest, c[b]);
-                const uint32_t t = c[b]; c[b] = tot; tot += t;
+            for (int b = 0; b < kInCellsPerLane; ++b) {
+                const int i = lane * kInCellsPerLane + b;
+                c[b] = i < kInCells ? (uint32_t)m[i] : 0u;
+                tot += c[b];
             }
             uint32_t incl = tot;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += t; }
-            if (lane == 31) s_warp_tot[warp] = incl;
-            use_radix = __syncthreads_or(longest > (uint32_t)kInMaxBucket);
-            uint32_t woff = 0;
-            for (int w = 0; w < warp; ++w) woff += s_warp_tot[w];
-            const uint32_t base = woff + incl - tot;
-            if (qpt == 8u) {
-                *reinterpret_cast<uint4 *>(qcnt + q0) = make_uint4(base + c[0], base + c[1], base + c[2], base + c[3]);
-                *reinterpret_cast<uint4 *>(qcnt + q0 + 4) = make_uint4(base + c[4], base + c[5], base + c[6], base + c[7]);
-            } else {
+            uint32_t run = incl - tot;
 #pragma unroll
-                for (int b = 0; b < 8; ++b)
-                    if ((uint32_t)b < qpt && q0 + b < R) qcnt[q0 + b] = base + c[b];
+            for (int b = 0; b < kInCellsPerLane; ++b) {
+                const int i = lane * kInCellsPerLane + b;
+                if (i < kInCells) { m[i] = (uint16_t)run; run += c[b]; }
             }
-            if (tid == kInThreads - 1) qcnt[R] = base + tot;
+            if (lane == 31) s_stot[warp] = incl;
         }
         __syncthreads();
-        if (!use_radix) {
-            // ---- short buckets: records go to the slot they took, then find their index-order rank ------------
-#pragma unroll
-            for (int j = 0; j < kInItems; ++j) {
-                const int e = j * kInThreads + tid;
-                if (e < cnt) {
-                    const uint64_t w2 = slot[e * 3 + 2];
-                    const uint32_t q = img_queue(w2);
-                    if (q != kInNoQueue) posA[qcnt[q] + img_place(w2)] = (uint16_t)e;
-                    else slot[e * 3 + 1] = 0;              // native or refused: no stall
-                }
-            }
-            __syncthreads();
-#pragma unroll
-            for (int j = 0; j < kInItems; ++j) {
-                const int e = j * kInThreads + tid;
-                if (e < cnt) {
-                    const uint64_t w2 = slot[e * 3 + 2];
-                    const uint32_t q = img_queue(w2);
-                    if (q != kInNoQueue) {
-                        const uint32_t st0 = qcnt[q], c = qcnt[q + 1] - st0;
-                        uint32_t rank = 0;
-                        if (c > 1u)
-                            for (uint32_t i = 0; i < c; ++i) rank += (uint32_t)posA[st0 + i] < (uint32_t)e ? 1u : 0u;
-                        posB[st0 + rank] = (uint16_t)e;
-                    }
-                }
-            }
-        } else {
-            // ---- a long bucket: stable radix sort of the positions by queue (6-bit digits, warp ranking) ----
-            uint32_t shift = 0;
-            for (uint32_t p = 0; p < n_pass; ++p) {
-                const uint32_t width = qbits / n_pass + (p < qbits % n_pass ? 1u : 0u);
-                const uint32_t dmask = (1u << width) - 1u;
-                const bool to_b = ((n_pass - 1u - p) & 1u) == 0u;            // the last pass lands in posB
-                uint16_t *dst = to_b ? posB : posA;
-                const uint16_t *srcp = to_b ? posA : posB;
-                for (int i = tid; i < kInWarps * kInBins; i += kInThreads) s_cnt[i] = 0u;
-                uint32_t e_[kInItems], dig[kInItems], rank[kInItems];
-                __syncthreads();
-#pragma unroll
-                for (int j = 0; j < kInItems; ++j) {
-                    const int i = warp * (32 * kInItems) + j * 32 + lane;       // memory order = (item, lane) order
-                    e_[j] = p == 0 ? (uint32_t)i : (uint32_t)srcp[i];
-                    uint32_t q = R;                                                // not modeled: behind every queue
-                    if ((int)e_[j] < cnt) {
-                        const uint32_t qq = img_queue(slot[e_[j] * 3 + 2]);
-                        if (qq != kInNoQueue) q = qq; else if (p == 0) slot[e_[j] * 3 + 1] = 0;     // native or refused: no stall
-                    }
-                    dig[j] = (q >> shift) & dmask;
-                }
-                uint32_t *wcnt = s_cnt + warp * kInBins;
-#pragma unroll
-                for (int j = 0; j < kInItems; ++j) {
-                    const unsigned peers = __match_any_sync(0xffffffffu, dig[j]);
-                    const uint32_t before = wcnt[dig[j]];
-                    rank[j] = before + (uint32_t)__popc(peers & lanemask_lt());
-                    __syncwarp();
-                    if ((peers >> lane) <= 1u) wcnt[dig[j]] = before + (uint32_t)__popc(peers);
-                    __syncwarp();
-                }
-                __syncthreads();
-                if (tid < kInBins) {
-                    uint32_t run = 0;
-#pragma unroll
-                    for (int w = 0; w < kInWarps; ++w) { const uint32_t c = s_cnt[w * kInBins + tid]; s_cnt[w * kInBins + tid] = run; run += c; }
-                    uint32_t incl = run;
-#pragma unroll
-                    for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += t; }
-                    if (lane == 31) s_bin_warp[warp] = incl;
-                    s_bin_start[tid] = incl - run;
-                }
-                __syncthreads();
-#pragma unroll
-                for (int j = 0; j < kInItems; ++j) {
-                    const uint32_t d = dig[j];
-                    dst[s_bin_start[d] + (d >= 32u ? s_bin_warp[0] : 0u) + wcnt[d] + rank[j]] = (uint16_t)e_[j];
-                }
-                shift += width;
-                __syncthreads();                           // the warp counters are cleared again by the next pass
-            }
-        }
-        __syncthreads();
-        // ---- serve.  In queue-major order a queue's accesses are consecutive.  Thread t takes positions
-        // [8t, 8t+8) and serves every queue whose first access of the chunk lies there, to that queue's last
-        // access (which may lie past 8t+8; the thread owning those positions skips them).  Every thread thus
-        // does about eight accesses, and a queue is touched by one thread only.  Loads go four at a time: they
-        // are independent, only the max-plus chain is serial.  M is the aggregate's constant term and, at the
-        // same time, the busy-until of the as-if-idle run.
+        uint32_t lo, hi;                                     // this warp's list
         {
-            const uint32_t modeled = qcnt[R];
-            const uint32_t p0 = (uint32_t)tid * kInItems;
-            const bool heads_on = !RESERVE && s_heads_full < R;
-            if (p0 < modeled) {
-                uint32_t cur = kInNoQueue, hf = 0;
-                bool mine = false;                            // the queue being served was opened by this thread
-                int64_t S = 0, M = kNegInf;
-                uint32_t prev_q = p0 > 0 ? img_queue(slot[(uint32_t)posB[p0 - 1] * 3 + 2]) : kInNoQueue;
-                auto close_queue = [&]() {
-                    aggS[cur] = S; aggM[cur] = M;
-                    if (heads_on) {
-                        if (hfill[cur] < (uint8_t)kInHead && hf == (uint32_t)kInHead) atomicAdd(&s_heads_full, 1u);
-                        hfill[cur] = (uint8_t)hf;
-                    }
-                };
-                auto serve_one = [&](uint32_t e, int64_t sv, int64_t issue, uint64_t w2) {
-                    const uint32_t x = (uint32_t)w2;
-                    const int64_t xfer = (int64_t)(x & 0x7fffffffu);
-                    const bool op = (x >> 31) != 0u;
-                    const int64_t m = issue + (op ? xfer : 0) + sv;          // arrival + service
-                    if (heads_on && hf < (uint32_t)kInHead) {                 // among the first accesses of this queue in the tile
-                        InHead h; h.m = m; h.s = sv; h.xo = x; h.idx = (uint32_t)(cbase + e);
-                        in_head[((uint64_t)tile * kInHead + hf) * R + cur] = h;
-                        ++hf;
-                    }
-                    M = max(M + sv, m); S += sv;                              // aggregate o access; M = busy-until after it
-                    const int64_t done = M + (op ? 0 : xfer);
-                    slot[e * 3] = (uint64_t)done; slot[e * 3 + 1] = (uint64_t)(done - issue);
-                    sum_stall += done - issue; max_c = max(max_c, (long long)done);
-                };
+            const uint32_t mine = lane < kInServers ? s_stot[lane] : 0u;
+            uint32_t incl = mine;
 #pragma unroll
-                for (int g = 0; g < kInItems / kInGroup; ++g) {
-                    const uint32_t pg = p0 + g * kInGroup;
-                    uint32_t e[kInGroup];
-                    int64_t s_[kInGroup], i_[kInGroup];
-                    uint64_t w2[kInGroup];
+            for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += t; }
+            const uint32_t sbase = incl - mine;
 #pragma unroll
-                    for (int j = 0; j < kInGroup; ++j) e[j] = pg + j < modeled ? (uint32_t)posB[pg + j] : 0u;
-#pragma unroll
-                    for (int j = 0; j < kInGroup; ++j) { s_[j] = (int64_t)slot[e[j] * 3]; i_[j] = (int64_t)slot[e[j] * 3 + 1]; w2[j] = slot[e[j] * 3 + 2]; }
-#pragma unroll
-                    for (int j = 0; j < kInGroup; ++j) {
-                        if (pg + j < modeled) {
-                            const uint32_t q = img_queue(w2[j]);
-                            if (q != prev_q) {                                // first access of queue q in this chunk
-                                if (mine) close_queue();
-                                cur = q; mine = true; S = aggS[q]; M = aggM[q];
-                                if (heads_on) hf = hfill[q];
-                            }
-                            if (mine) serve_one(e[j], s_[j], i_[j], w2[j]);
-                            prev_q = q;
-                        }
+            for (int j = 0; j < kInItems; ++j) {
+                const uint32_t srv = pk[j] >> 5;
+                const uint32_t base = __shfl_sync(0xffffffffu, sbase, (int)srv);
+                if (srv < (uint32_t)kInServers)
+                    list[base + cntm[(srv * kInItems + j) * kInWarps + warp] + (pk[j] & 31u)] = (uint16_t)(j * kInThreads + tid);
+            }
+            lo = __shfl_sync(0xffffffffu, sbase, warp);
+            hi = lo + __shfl_sync(0xffffffffu, mine, warp);
+        }
+        __syncthreads();
+        for (uint32_t i = tid; i < (uint32_t)(kInServers * kInCells / 2); i += kInThreads) reinterpret_cast<uint32_t *>(cntm)[i] = 0u;
+        // ---- serve: each warp walks its list, 32 records at a time.  Lanes holding records of the same queue
+        // chain them in lane (= batch) order: every lane composes the accesses of its queue up to its own.
+        {
+            const bool heads_on = !RESERVE && *reinterpret_cast<volatile uint32_t *>(&s_heads_full) < R;
+            const unsigned le_mask = lanemask_lt() | (1u << lane);
+            for (uint32_t t = lo; t < hi; t += 32u) {
+                const uint32_t k = t + (uint32_t)lane;
+                const bool act = k < hi;
+                const uint32_t e = act ? min((uint32_t)list[k], (uint32_t)(kInChunk - 1)) : 0u;
+                const uint64_t sx = slot[e * 3];
+                const int64_t a = (int64_t)slot[e * 3 + 2];
+                const uint32_t sv = (uint32_t)sx, xq = (uint32_t)(sx >> 32);
+                const uint32_t q = act ? min(xq >> (kInXferBits + 1), R - 1u) : (0x10000u | (uint32_t)lane);
+                const int64_t post = (xq >> kInXferBits) & 1u ? 0 : (int64_t)(xq & ((1u << kInXferBits) - 1u));   // a read's transfer follows its service
+                const unsigned peers = __match_any_sync(0xffffffffu, q);
+                const unsigned le = peers & le_mask;
+                const uint32_t rank1 = (uint32_t)__popc(le);                  // this access is the rank1-th of its queue in the group
+                const uint32_t n_it = __reduce_max_sync(0xffffffffu, rank1);
+                const uint32_t qi = act ? q : 0u;
+                const longlong2 state = qst[qi];
+                int64_t B = state.x;
+                const uint32_t c0 = heads_on ? (uint32_t)state.y & 0xffu : (uint32_t)kInHead;
+                int64_t sumS = (int64_t)sv;
+                if (n_it == 1u) {
+                    B = max(a, B) + (int64_t)sv;
+                } else {
+                    unsigned rem = le;
+                    sumS = 0;
+                    for (uint32_t it = 0; it < n_it; ++it) {
+                        const int src = rem ? __ffs((int)rem) - 1 : lane;
+                        const int64_t ab = __shfl_sync(0xffffffffu, a, src);
+                        const uint32_t sb = __shfl_sync(0xffffffffu, sv, src);
+                        if (rem) { B = max(ab, B) + (int64_t)sb; sumS += (int64_t)sb; }
+                        rem &= rem - 1u;
                     }
                 }
-                if (mine) {                                    // the last queue opened here may go on past this thread's positions
-                    for (uint32_t p = p0 + kInItems; p < modeled; ++p) {
-                        const uint32_t e = posB[p];
-                        const uint64_t w2 = slot[e * 3 + 2];
-                        if (img_queue(w2) != cur) break;
-                        serve_one(e, (int64_t)slot[e * 3], (int64_t)slot[e * 3 + 1], w2);
+                if (act) {
+                    slot[e * 3 + 2] = (uint64_t)(B + post);
+                    const uint32_t ci = c0 + rank1 - 1u;
+                    if (ci < (uint32_t)kInHead) {
+                        const uint32_t xfer = xq & ((1u << kInXferBits) - 1u), op = (xq >> kInXferBits) & 1u;
+                        InHead h; h.m = a + (int64_t)sv; h.s = (int64_t)sv; h.xo = xfer | (op << 31); h.idx = (uint32_t)(cbase + e);
+                        in_head[((uint64_t)tile * kInHead + ci) * R + q] = h;
                     }
-                    close_queue();
+                    if ((peers >> lane) == 1u) {                                // no later access of this queue in the group
+                        const uint32_t c1 = min(c0 + (uint32_t)__popc(peers), (uint32_t)kInHead);
+                        qst[q] = make_longlong2(B, state.y + (sumS << 8) + (long long)(c1 - c0));
+                        if (c1 != c0 && c1 == (uint32_t)kInHead) atomicAdd(&s_heads_full, 1u);
+                    }
                 }
+                __syncwarp();                                // the next group may meet the same queues
             }
         }
         __syncthreads();
-        // ---- results leave in batch order; the chunk's queue-major order stays behind for the fix-up ----------
-        for (int e = tid; e < cnt; e += kInThreads) { completion[cbase + e] = (int64_t)slot[e * 3]; stall[cbase + e] = (int64_t)slot[e * 3 + 1]; }
-        if (!RESERVE) {
-            const uint32_t modeled = qcnt[R];
-            for (uint32_t k = tid; k < modeled; k += kInThreads) in_pos[cbase + k] = posB[k];
-            uint16_t *row = in_start + (cbase / kInChunk) * row_stride;
-            for (uint32_t q = tid; q <= R; q += kInThreads) row[q] = (uint16_t)qcnt[q];
+        // ---- results leave in batch order ----------------------------------------------------------------------
+#pragma unroll
+        for (int j = 0; j < kInItems; ++j) {
+            const int e = j * kInThreads + tid;
+            if (e < cnt) {
+                const int64_t issue = (int64_t)slot[e * 3 + 1], done = (int64_t)slot[e * 3 + 2];
+                const int64_t st = done - issue;             // a modeled access always waits for its service: st > 0
+                completion[cbase + e] = done; stall[cbase + e] = st;
+                sum_stall += st;
+                if (st != 0) max_c = max(max_c, (long long)done);
+            }
         }
     }
 
@@ -477,9 +397,9 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
     if (!RESERVE) {
         longlong2 *out = reinterpret_cast<longlong2 *>(in_agg) + (uint64_t)tile * R;
         for (uint32_t q = tid; q < R; q += kInThreads) {
-            const uint32_t i = state_index(q, qpt_shift);
-            out[q] = make_longlong2(aggS[i], aggM[i]);
-            in_headcnt[(uint64_t)tile * R + q] = hfill[q];
+            const longlong2 v = qst[q];
+            out[q] = make_longlong2(v.y >> 8, v.x);
+            in_headcnt[(uint64_t)tile * R + q] = (uint8_t)(v.y & 0xff);
         }
         for (uint32_t d = tid; d < n_dies; d += kInThreads) {
             unsigned long long *g = reinterpret_cast<unsigned long long *>(stats_stage + d);
@@ -507,7 +427,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
     if (tid == 0) {
         if (RESERVE) in_tile[tile].true_sum = s_red[0];
         else { InTile t; t.spec_sum = s_red[0]; t.fix_delta = 0; t.true_sum = 0; t.reserve = 0u; t.stragglers = 0u; in_tile[tile] = t; }
-        atomicMax(&ctrl->max_completion_ns, s_red[1]);
+        if (s_red[1] != INT64_MIN) atomicMax(&ctrl->max_completion_ns, s_red[1]);
     }
 }
 
@@ -563,13 +483,13 @@ k_inorder_scan(BatchCtrl *ctrl, const ModelParams *__restrict__ mp, uint32_t n_t
 // ======================================================================================================
 constexpr int kInFixThreads = 128;
 
-// Phase 1, one thread per (tile, queue): walk the head table.  A queue that is still backlogged after
-// kInHead accesses is a straggler: it goes on a list for phase 2, or, when a tile has many of them (the
-// batch arrived on queues that were far behind), the whole tile is flagged to be served again.
+// One thread per (tile, queue): walk the head table.  A queue that is still backlogged after kInHead
+// accesses is a straggler: its head count is replaced by a mark for the straggle pass, or, when a tile has
+// many of them (the batch arrived on queues that were far behind), the whole tile is flagged to be served again.
 __global__ void __launch_bounds__(kInFixThreads)
 k_inorder_fixup(uint32_t R, uint32_t n_tiles, BatchCtrl *ctrl, const int64_t *__restrict__ in_bin,
-                const InHead *__restrict__ in_head, const uint8_t *__restrict__ in_headcnt, int64_t *completion, int64_t *stall,
-                InTile *in_tile, uint32_t *in_list) {
+                const InHead *__restrict__ in_head, uint8_t *__restrict__ in_headcnt, int64_t *completion, int64_t *stall,
+                InTile *in_tile) {
     if (ctrl->skip || ctrl->run_sort || !ctrl->inorder_used) return;
     const uint64_t idx = (uint64_t)blockIdx.x * kInFixThreads + threadIdx.x;          // tile * R + queue
     long long max_c = INT64_MIN;
@@ -593,98 +513,187 @@ k_inorder_fixup(uint32_t R, uint32_t n_tiles, BatchCtrl *ctrl, const int64_t *__
             completion[h.idx] = done; stall[h.idx] = done - (h.m - h.s - (op ? xfer : 0));
             max_c = max(max_c, (long long)done);
         }
-        if (dstall) atomicAdd((unsigned long long *)&in_tile[tile].fix_delta, (unsigned long long)dstall);
         if (!settled && c == (uint32_t)kInHead) {
+            // the straggle pass serves this queue again from the tile's start and accounts for all of its corrections
+            in_headcnt[idx] = kInStraggler;
             const uint32_t rank = atomicAdd(&in_tile[tile].stragglers, 1u);
             if (rank >= max(8u, R / 16u)) in_tile[tile].reserve = 1u;
-            else in_list[1 + atomicAdd(&in_list[0], 1u)] = (uint32_t)idx;
+        } else if (dstall) {
+            atomicAdd((unsigned long long *)&in_tile[tile].fix_delta, (unsigned long long)dstall);
         }
     }
     max_c = warp_max(max_c);
     if ((threadIdx.x & 31) == 0 && max_c != INT64_MIN) atomicMax(&ctrl->max_completion_ns, max_c);
 }
 
-// Phase 2, one warp per straggler: re-serve the queue's accesses of the tile from the records until an
-// access arrives on an idle queue.  The lanes take 32 consecutive chunks at a time: each composes the
-// maps of the queue's accesses in its chunk, a warp scan over the lanes gives the true busy-until
-// entering every chunk, and each lane then re-serves its chunk.  Past the point where the queue falls
-// idle the re-served values equal what is already there, so lanes need not agree on where to stop.
-constexpr uint32_t kInLongBudget = 4096;                  // accesses re-served for one (tile, queue) before the tile is re-served whole
+// ======================================================================================================
+// straggle: one block per tile that has stragglers (and is not re-served whole).  The block streams the
+// tile's records again, keeps the modeled records of the straggling queues in batch order, and its first
+// warp re-serves them 32 at a time, carrying both the true run (from the true entering busy-until) and the
+// as-if-idle run (to know what the serve pass wrote).  A queue is done when the two runs meet: from there
+// on the serve pass was right.  The block stops at the chunk in which its last queue is done.
+// ======================================================================================================
+constexpr int kInStrThreads = 512;
+constexpr int kInStrItems = 8;
+constexpr int kInStrChunk = kInStrThreads * kInStrItems;
+constexpr int kInStrWarps = kInStrThreads / 32;
+constexpr int kInStrCells = kInStrItems * kInStrWarps;    // (row, warp) cells of the kept-record counts
+constexpr int kInStrCellsPerLane = kInStrCells / 32;
+static_assert(kInStrCells % 32 == 0, "the offset scan gives every lane the same number of cells");
 
-__global__ void __launch_bounds__(kInFixThreads)
-k_inorder_fixup_long(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_records,
-                     const RangeSnap *__restrict__ ranges_g, const ModelParams *__restrict__ mp_g, BatchCtrl *ctrl,
-                     const int64_t *__restrict__ in_bin, const uint16_t *__restrict__ in_pos, const uint16_t *__restrict__ in_start,
-                     uint32_t row_stride, int64_t *completion, int64_t *stall, InTile *in_tile, const uint32_t *__restrict__ in_list) {
+// Queue of an access of the common configuration (one range, power-of-two geometry), or ~0 when the address
+// lies outside the range.  In a batch that was not refused every access inside the range is modeled.
+__device__ __forceinline__ uint32_t fast_queue(const FastRange &f, const ModelParams &mp, uint64_t addr) {
+    const uint64_t rel = addr - f.base;
+    if (rel >= f.length) return 0xffffffffu;
+    const uint32_t u = (uint32_t)((f.media_offset + rel) >> mp.stripe_shift);
+    const uint32_t ch = u & (mp.channels - 1u), di = (u >> mp.ch_shift) & (mp.dies - 1u);
+    const uint32_t pl = (u >> (mp.ch_shift + mp.die_shift)) & (mp.planes - 1u);
+    const uint32_t die = ch * mp.dies + di;
+    return mp.queue_level == 0u ? die * mp.planes + pl : die;
+}
+
+__global__ void __launch_bounds__(kInStrThreads)
+k_inorder_straggle(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_records,
+                   const RangeSnap *__restrict__ ranges_g, const ModelParams *__restrict__ mp_g, BatchCtrl *ctrl,
+                   const int64_t *__restrict__ in_bin, const uint8_t *__restrict__ in_headcnt, int64_t *completion,
+                   int64_t *stall, InTile *in_tile) {
+    extern __shared__ __align__(16) unsigned char str_smem[];
     __shared__ ModelParams mp;
+    __shared__ uint32_t s_cells[kInStrCells];
+    __shared__ uint32_t s_total;
+    __shared__ int s_open;                                   // straggling queues whose two runs have not met yet
+    __shared__ FastRange s_fast;
+
     if (ctrl->skip || ctrl->run_sort || !ctrl->inorder_used) return;
+    const uint32_t tile = blockIdx.x;
+    if (in_tile[tile].stragglers == 0u || in_tile[tile].reserve) return;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const RangeSnap &rs = *ranges_g;
-    for (int i = threadIdx.x; i < (int)(sizeof(ModelParams) / 4); i += kInFixThreads)
+    for (int i = tid; i < (int)(sizeof(ModelParams) / 4); i += kInStrThreads)
         reinterpret_cast<uint32_t *>(&mp)[i] = reinterpret_cast<const uint32_t *>(mp_g)[i];
+    const uint32_t R = mp_g->n_queues;
+    int64_t *Bt = reinterpret_cast<int64_t *>(str_smem);                       // [queues] true run
+    int64_t *Ba = Bt + kInMaxQueues;                                           // [queues] as-if-idle run
+    uint16_t *list = reinterpret_cast<uint16_t *>(Ba + kInMaxQueues);          // [chunk] positions of the kept records, batch order
+    uint8_t *open = reinterpret_cast<uint8_t *>(list + kInStrChunk);           // [queues] 1: straggler, runs have not met
+    if (tid == 0) {
+        s_open = 0;
+        FastRange f; f.base = rs.base[0]; f.length = rs.length[0]; f.media_offset = rs.media_offset[0]; f.perms = rs.perms[0];
+        f.on = (rs.count == 1u && mp_g->pow2_geom) ? 1u : 0u;
+        s_fast = f;
+    }
     __syncthreads();
-    const uint32_t R = mp.n_queues, count = in_list[0];
+    {
+        int mine = 0;
+        for (uint32_t q = tid; q < kInMaxQueues; q += kInStrThreads) {
+            const bool s = q < R && in_headcnt[(uint64_t)tile * R + q] == kInStraggler;
+            open[q] = s ? 1 : 0;
+            Ba[q] = kNegInf;
+            Bt[q] = s ? in_bin[(uint64_t)tile * R + q] : kNegInf;
+            mine += s ? 1 : 0;
+        }
+        if (mine) atomicAdd(&s_open, mine);
+    }
     const int64_t q_ppm = ctrl->q_ppm;
     const Div64 div_q = ctrl->div_q;
-    const uint32_t lane = threadIdx.x & 31u;
-    const uint32_t warp_global = (blockIdx.x * kInFixThreads + threadIdx.x) >> 5, n_warps = (gridDim.x * kInFixThreads) >> 5;
-    long long max_c = INT64_MIN;
-    for (uint32_t w = warp_global; w < count; w += n_warps) {
-        const uint32_t idx = in_list[1 + w];
-        const uint32_t tile = idx / R, q = idx % R;
-        if (in_tile[tile].reserve) continue;
-        int64_t B = in_bin[idx];                             // true busy-until entering the next group of chunks
-        long long dstall = 0;
-        const uint64_t tile_begin = (uint64_t)tile * tile_records, tile_end = min(n, tile_begin + tile_records);
-        uint32_t served = 0;
-        for (uint64_t gbase = tile_begin; gbase < tile_end; gbase += 32ull * kInChunk) {
-            const uint64_t cbase = gbase + (uint64_t)lane * kInChunk;
-            uint32_t k0 = 0, k1 = 0;
-            if (cbase < tile_end) {
-                const uint16_t *row = in_start + (cbase / kInChunk) * row_stride;
-                k0 = row[q]; k1 = row[q + 1];
-            }
-            // this lane's chunk as one map B -> max(B + S, M)
-            int64_t S = 0, M = kNegInf;
-            for (uint32_t k = k0; k < k1; ++k) {
-                const uint64_t *rec = reinterpret_cast<const uint64_t *>(acc + cbase + in_pos[cbase + k]);
-                const int64_t issue = (int64_t)rec[1];
-                const Served v = serve_terms(rs, mp, rec[0], issue, rec[2], q_ppm, div_q);
-                M = max(M + v.s, issue + (v.op ? v.xfer : 0) + v.s); S += v.s;
-            }
-            // exclusive scan of the maps over the lanes, applied to B
-            int64_t iS = S, iM = M;
+    const uint64_t tile_begin = (uint64_t)tile * tile_records, tile_end = min(n, tile_begin + tile_records);
+    long long dstall = 0, max_c = INT64_MIN;
+    __syncthreads();
+
+    for (uint64_t cbase = tile_begin; cbase < tile_end; cbase += kInStrChunk) {
+        // ---- keep the modeled records of the open queues, in batch order -----------------------------------
+        uint32_t keep = 0, rk[kInStrItems];
 #pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int64_t uS = __shfl_up_sync(0xffffffffu, iS, o), uM = __shfl_up_sync(0xffffffffu, iM, o);
-                if ((int)lane >= o) { iM = max(uM + iS, iM); iS += uS; }
-            }
-            int64_t eS = __shfl_up_sync(0xffffffffu, iS, 1), eM = __shfl_up_sync(0xffffffffu, iM, 1);
-            if (lane == 0) { eS = 0; eM = kNegInf; }
-            int64_t Bl = max(B + eS, eM);                    // true busy-until entering this lane's chunk
-            // re-serve the chunk
-            bool idle_seen = false;
-            for (uint32_t k = k0; k < k1; ++k) {
-                const uint64_t i = cbase + in_pos[cbase + k];
+        for (int j = 0; j < kInStrItems; ++j) {
+            const uint64_t i = cbase + (uint64_t)(j * kInStrThreads + tid);
+            bool k = false;
+            if (i < tile_end) {
                 const uint64_t *rec = reinterpret_cast<const uint64_t *>(acc + i);
-                const int64_t issue = (int64_t)rec[1];
-                const Served v = serve_terms(rs, mp, rec[0], issue, rec[2], q_ppm, div_q);
-                const int64_t a = issue + (v.op ? v.xfer : 0);
-                if (Bl <= a) idle_seen = true;
-                Bl = max(a, Bl) + v.s;
-                const int64_t done = Bl + (v.op ? 0 : v.xfer);
-                const int64_t old = completion[i];
-                if (done != old) { dstall += done - old; completion[i] = done; stall[i] = done - issue; max_c = max(max_c, (long long)done); }
+                if (s_fast.on) {
+                    const uint32_t q = fast_queue(s_fast, mp, __ldg(rec));
+                    k = q != 0xffffffffu && open[q] != 0;
+                } else {
+                    const Served v = serve_terms(rs, mp, __ldg(rec), (int64_t)__ldg(rec + 1), __ldg(rec + 2), q_ppm, div_q);
+                    k = v.st == HBF_ST_READY && open[v.queue] != 0;
+                }
             }
-            served += __reduce_add_sync(0xffffffffu, k1 - k0);
-            B = max(B + __shfl_sync(0xffffffffu, iS, 31), __shfl_sync(0xffffffffu, iM, 31));
-            if (__any_sync(0xffffffffu, idle_seen)) break;   // the queue fell idle: the rest of the tile was served right
-            if (served > kInLongBudget) { if (lane == 0) in_tile[tile].reserve = 1u; break; }
+            const unsigned bal = __ballot_sync(0xffffffffu, k);
+            rk[j] = (uint32_t)__popc(bal & lanemask_lt());
+            if (lane == 0) s_cells[j * kInStrWarps + warp] = (uint32_t)__popc(bal);
+            keep |= k ? 1u << j : 0u;
         }
-        dstall = warp_sum(dstall);
-        if (lane == 0 && dstall) atomicAdd((unsigned long long *)&in_tile[tile].fix_delta, (unsigned long long)dstall);
+        __syncthreads();
+        if (warp == 0) {
+            uint32_t c[kInStrCellsPerLane], tot = 0;
+#pragma unroll
+            for (int b = 0; b < kInStrCellsPerLane; ++b) { c[b] = s_cells[lane * kInStrCellsPerLane + b]; tot += c[b]; }
+            uint32_t incl = tot;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += t; }
+            uint32_t run = incl - tot;
+#pragma unroll
+            for (int b = 0; b < kInStrCellsPerLane; ++b) { s_cells[lane * kInStrCellsPerLane + b] = run; run += c[b]; }
+            if (lane == 31) s_total = incl;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int j = 0; j < kInStrItems; ++j)
+            if (keep & (1u << j)) list[s_cells[j * kInStrWarps + warp] + rk[j]] = (uint16_t)(j * kInStrThreads + tid);
+        __syncthreads();
+        // ---- the first warp re-serves them ---------------------------------------------------------------
+        if (warp == 0) {
+            const uint32_t total = s_total;
+            const unsigned le_mask = lanemask_lt() | (1u << lane);
+            for (uint32_t t = 0; t < total; t += 32u) {
+                const uint32_t k = t + (uint32_t)lane;
+                const bool act = k < total;
+                uint64_t i = cbase;
+                uint32_t q = 0x10000u | (uint32_t)lane;
+                int64_t issue = 0, a = 0, sv = 0, post = 0;
+                if (act) {
+                    i = min(cbase + list[k], tile_end - 1);
+                    const uint64_t *rec = reinterpret_cast<const uint64_t *>(acc + i);
+                    issue = (int64_t)__ldg(rec + 1);
+                    const Served v = serve_terms(rs, mp, __ldg(rec), issue, __ldg(rec + 2), q_ppm, div_q);
+                    q = v.queue; sv = v.s; a = issue + (v.op ? v.xfer : 0); post = v.op ? 0 : v.xfer;
+                }
+                const unsigned peers = __match_any_sync(0xffffffffu, q);
+                const unsigned le = peers & le_mask;
+                const uint32_t n_it = __reduce_max_sync(0xffffffffu, (uint32_t)__popc(le));
+                const uint32_t qi = act ? q : 0u;
+                int64_t BT = Bt[qi], BA = Ba[qi];
+                unsigned rem = le;
+                for (uint32_t it = 0; it < n_it; ++it) {
+                    const int src = rem ? __ffs((int)rem) - 1 : lane;
+                    const int64_t ab = __shfl_sync(0xffffffffu, a, src), sb = __shfl_sync(0xffffffffu, sv, src);
+                    if (rem) { BT = max(ab, BT) + sb; BA = max(ab, BA) + sb; }
+                    rem &= rem - 1u;
+                }
+                if (act) {
+                    if ((peers >> lane) == 1u) {               // last access of this queue in the group
+                        Bt[q] = BT; Ba[q] = BA;
+                        if (BT == BA && open[q]) { open[q] = 0; atomicSub(&s_open, 1); }
+                    }
+                    if (BT != BA) {                             // the serve pass wrote BA + post
+                        const int64_t done = BT + post;
+                        completion[i] = done; stall[i] = done - issue;
+                        dstall += BT - BA; max_c = max(max_c, (long long)done);
+                    }
+                }
+                __syncwarp();
+            }
+        }
+        __syncthreads();
+        if (*reinterpret_cast<volatile int *>(&s_open) <= 0) break;
     }
-    max_c = warp_max(max_c);
-    if (lane == 0 && max_c != INT64_MIN) atomicMax(&ctrl->max_completion_ns, max_c);
+    if (warp == 0) {
+        dstall = warp_sum(dstall); max_c = warp_max(max_c);
+        if (lane == 0) {
+            if (dstall) atomicAdd((unsigned long long *)&in_tile[tile].fix_delta, (unsigned long long)dstall);
+            if (max_c != INT64_MIN) atomicMax(&ctrl->max_completion_ns, max_c);
+        }
+    }
 }
 
 // stall total of the batch: per tile the exact sum if it was re-served, else the as-if sum plus its corrections
@@ -706,49 +715,47 @@ uint64_t inorder_tile_records(uint64_t n, int sm_count) {
     return std::max<uint64_t>(t, kInChunk);
 }
 
-// dynamic shared memory of the serve kernel: two record buffers, counts, two position buffers, aggregates, per-die counters, head fill
+// dynamic shared memory of the serve kernel: two record buffers, the per-queue state, the servers' lists, the
+// count matrix, per-die counters
 size_t inorder_serve_smem(uint32_t n_dies) {
-    return (size_t)2 * kInSlotBytes + kInCntBytes + 2 * kInPosBytes + (size_t)kInMaxQueues * 16 + (size_t)n_dies * 24 + kInMaxQueues;
+    return (size_t)2 * kInSlotBytes + (size_t)kInMaxQueues * 16 + (size_t)kInChunk * 2 + (size_t)kInServers * kInCells * 2 +
+           (size_t)n_dies * 24;
 }
+static size_t inorder_straggle_smem() { return (size_t)kInMaxQueues * 16 + (size_t)kInStrChunk * 2 + kInMaxQueues; }
 
-static uint32_t inorder_row_stride(uint32_t n_queues) { return (n_queues + 1u + 7u) / 8u * 8u; }
 size_t inorder_head_bytes(uint64_t tiles, uint32_t n_queues) { return tiles * n_queues * (size_t)kInHead * sizeof(InHead); }
-size_t inorder_start_bytes(uint64_t n, uint32_t n_queues) {
-    return ((n + kInChunk - 1) / kInChunk + 1) * (size_t)inorder_row_stride(n_queues) * sizeof(uint16_t);
-}
 
 cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st) {
     const uint64_t n = a.n;
     const uint64_t tile_records = inorder_tile_records(n, a.sm_count);
     const unsigned n_tiles = (unsigned)((n + tile_records - 1) / tile_records);
-    const uint32_t R = a.mp.n_queues, nd = a.mp.n_dies, row_stride = inorder_row_stride(R);
-    const size_t smem_serve = inorder_serve_smem(nd);
+    const uint32_t R = a.mp.n_queues, nd = a.mp.n_dies;
+    const size_t smem_serve = inorder_serve_smem(nd), smem_str = inorder_straggle_smem();
     static size_t set_serve = 0;
     if (smem_serve > set_serve) {
         cudaError_t e = cudaFuncSetAttribute(k_inorder_serve<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_serve);
         if (e != cudaSuccess) return e;
         e = cudaFuncSetAttribute(k_inorder_serve<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_serve);
         if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(k_inorder_straggle, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_str);
+        if (e != cudaSuccess) return e;
         set_serve = smem_serve;
     }
     InTile *tiles = reinterpret_cast<InTile *>(a.ws.in_tile);
     InHead *heads = reinterpret_cast<InHead *>(a.ws.in_head);
-    cudaError_t em = cudaMemsetAsync(a.ws.in_list, 0, sizeof(uint32_t), st);
-    if (em != cudaSuccess) return em;
     k_inorder_serve<false><<<n_tiles, kInThreads, smem_serve, st>>>(a.acc, n, tile_records, a.ranges, a.mp_dev, a.ctrl, a.status,
-                                                                    a.ws.in_agg, a.ws.in_pos, a.ws.in_start, row_stride, a.stats_stage,
-                                                                    a.completion, a.stall, a.ws.in_bin, tiles, heads, a.ws.in_headcnt);
+                                                                    a.ws.in_agg, a.stats_stage, a.completion, a.stall, a.ws.in_bin,
+                                                                    tiles, heads, a.ws.in_headcnt);
     k_inorder_scan<<<(R + kInScanThreads - 1) / kInScanThreads, kInScanThreads, 0, st>>>(
         a.ctrl, a.mp_dev, n_tiles, a.ws.in_agg, a.ws.in_bin, a.busy, a.busy_stage, a.stats_stage, a.path == HBF_PATH_INORDER ? 1 : 0);
     const uint64_t fix_threads = (uint64_t)n_tiles * R;
     k_inorder_fixup<<<(unsigned)((fix_threads + kInFixThreads - 1) / kInFixThreads), kInFixThreads, 0, st>>>(
-        R, n_tiles, a.ctrl, a.ws.in_bin, heads, a.ws.in_headcnt, a.completion, a.stall, tiles, a.ws.in_list);
-    k_inorder_fixup_long<<<(unsigned)std::max(1, a.sm_count * 4), kInFixThreads, 0, st>>>(
-        a.acc, n, tile_records, a.ranges, a.mp_dev, a.ctrl, a.ws.in_bin, a.ws.in_pos, a.ws.in_start, row_stride, a.completion, a.stall,
-        tiles, a.ws.in_list);
+        R, n_tiles, a.ctrl, a.ws.in_bin, heads, a.ws.in_headcnt, a.completion, a.stall, tiles);
+    k_inorder_straggle<<<n_tiles, kInStrThreads, smem_str, st>>>(a.acc, n, tile_records, a.ranges, a.mp_dev, a.ctrl, a.ws.in_bin,
+                                                                a.ws.in_headcnt, a.completion, a.stall, tiles);
     k_inorder_serve<true><<<n_tiles, kInThreads, smem_serve, st>>>(a.acc, n, tile_records, a.ranges, a.mp_dev, a.ctrl, a.status,
-                                                                   a.ws.in_agg, a.ws.in_pos, a.ws.in_start, row_stride, a.stats_stage,
-                                                                   a.completion, a.stall, a.ws.in_bin, tiles, heads, a.ws.in_headcnt);
+                                                                   a.ws.in_agg, a.stats_stage, a.completion, a.stall, a.ws.in_bin,
+                                                                   tiles, heads, a.ws.in_headcnt);
     k_inorder_total<<<1, 256, 0, st>>>(a.ctrl, tiles, n_tiles);
     g_kernel_launches += 6;
     return cudaGetLastError();

@@ -660,14 +660,13 @@ size_t workspace_layout(uint64_t n, uint32_t n_queues, Workspace *ws, void *base
     const uint64_t in_tiles = std::min<uint64_t>(kInMaxTiles, (nn + 2047) / 2048);
     const bool inorder = n_queues <= kInMaxQueues;
     void *ia = take(inorder ? in_tiles * n_queues * 16 : 0), *ib = take(inorder ? in_tiles * n_queues * 8 : 0);
-    void *ii = take(inorder ? (nn + 8192) * 2 : 0), *is = take(inorder ? inorder_start_bytes(nn, n_queues) : 0);
     void *it = take(inorder ? in_tiles * 32 : 0), *ih = take(inorder ? inorder_head_bytes(in_tiles, n_queues) : 0);
-    void *ic = take(inorder ? in_tiles * n_queues : 0), *il = take(inorder ? (1 + in_tiles * n_queues) * 4 : 0);
+    void *ic = take(inorder ? in_tiles * n_queues : 0);
     if (ws) {
         ws->keys[0] = (uint64_t *)k0; ws->keys[1] = (uint64_t *)k1; ws->idx[0] = (uint32_t *)i0; ws->idx[1] = (uint32_t *)i1;
         ws->hist = (uint32_t *)h; ws->sort_desc[0] = (uint32_t *)d0; ws->sort_desc[1] = (uint32_t *)d1;
         ws->scan_desc = sd; ws->in_agg = (int64_t *)ia; ws->in_bin = (int64_t *)ib;
-        ws->in_pos = (uint16_t *)ii; ws->in_tile = it; ws->in_head = ih; ws->in_headcnt = (uint8_t *)ic; ws->in_list = (uint32_t *)il; ws->in_start = (uint16_t *)is; ws->bytes = off;
+        ws->in_tile = it; ws->in_head = ih; ws->in_headcnt = (uint8_t *)ic; ws->bytes = off;
     }
     return off;
 }
