@@ -106,6 +106,12 @@ extern unsigned long long g_kernel_launches;
 
 constexpr uint32_t kInMaxQueues = 2048;  // the in-order path keeps per-queue state in shared memory
 constexpr uint32_t kInMaxTiles = 512;
+constexpr uint32_t kInTileQuantum = 1024; // tiles of the in-order path are a multiple of this many records
+// upper bound of the number of tiles of a batch of n records, on any device: what the workspace is carved for
+inline uint64_t inorder_tiles_bound(uint64_t n) {
+    const uint64_t t = (n + kInTileQuantum - 1) / kInTileQuantum;
+    return t < 1 ? 1 : (t < kInMaxTiles ? t : kInMaxTiles);
+}
 size_t workspace_layout(uint64_t n, uint32_t n_queues, Workspace *ws, void *base);
 // tile size (records) of the in-order path for a batch of n on a device with sm_count SMs
 uint64_t inorder_tile_records(uint64_t n, int sm_count);

@@ -1,11 +1,11 @@
 // In-order path of hbf_submit_batch: serves a batch whose records arrive in non-decreasing issue order
 // without a global sort.  In such a batch the (issue, index) order of every queue is plain index order,
-// so the batch is cut into contiguous tiles, one per SM, that are served independently, in one pass:
+// so the batch is cut into contiguous tiles, one per resident thread block, that are served independently:
 //   serve     every tile classifies and decodes its records, writes status[], counts, sums per-die bytes, and
 //             serves its accesses AS IF every queue were idle when the tile begins; completions and stalls
-//             leave through shared memory in batch order.  Per queue it also keeps the composition (S, M) of
-//             the maps B -> max(B + s, a + s) of its accesses (M is exactly the busy-until of the as-if run)
-//             and the first few accesses of the queue in the tile (the head table);
+//             are written as they are computed, in batch order.  Per queue it also keeps the composition
+//             (S, M) of the maps B -> max(B + s, a + s) of its accesses (M is exactly the busy-until of the
+//             as-if run) and the first few accesses of the queue in the tile (the head table);
 //   scan      one thread per queue walks the tiles' aggregates in order: the true busy-until entering each
 //             tile, and the final busy-until;
 //   fix-up    one thread per (tile, queue) starts from the true entering busy-until and re-serves the head
@@ -18,57 +18,31 @@
 //   re-serve  a tile with many stragglers (the batch arrived on queues that were far behind) is served
 //             again from the true entering busy-until, exactly.
 // The serve pass is the only one that streams the whole batch: 24 B read and 16 B + 1 B written per access.
-// Every global access of it is coalesced; nothing waits on another thread block.
+// Every global access of it is coalesced; nothing waits on another thread block, and no thread spins.
 //
-// Inside a chunk (3,072 records) the queue dependency is resolved by the warps acting as servers: queues are
-// hashed onto the block's warps, every record is appended, in batch order, to the list of its queue's warp
-// (ranking by warp match, offsets by a small scan), and each warp then walks its list 32 records at a time.
-// The busy-until of every queue lives in shared memory; records of one queue that fall into the same group
-// of 32 are chained in registers with shuffles.  Different warps never touch the same queue.
+// Inside a tile the busy-until of every queue lives in shared memory.  The records are taken 32 at a time
+// (a row per warp, rows dealt round-robin to the block's warps); all the per-record arithmetic runs in
+// parallel, and only the read-serve-write of the queue state is done row after row, handed from warp to
+// warp through the hardware's named barriers.  Records of one queue that fall into the same row are chained
+// in registers with shuffles.
 #include <algorithm>
 
 #include "device_utils.cuh"
 
 namespace hbf {
 
-// Block shape of the serve kernel: one block per SM; the records arrive by bulk asynchronous copy (TMA)
-// into one of two buffers while the previous chunk is being served.
+// Block shape of the serve kernel.  The per-queue state (32 KB) is all the shared memory a block needs, so
+// several blocks share an SM, each with its own tile and its own row-after-row chain of queue updates.
 #ifndef HBF_IN_THREADS
-#define HBF_IN_THREADS 640
-#define HBF_IN_ITEMS 5
+#define HBF_IN_THREADS 384
+#endif
+#ifndef HBF_IN_BLOCKS
+#define HBF_IN_BLOCKS 2
 #endif
 constexpr int kInThreads = HBF_IN_THREADS;               // threads of a serve block
-constexpr int kInItems = HBF_IN_ITEMS;                   // records per thread and chunk
-constexpr int kInBlocksPerSM = 1;
-constexpr int kInChunk = kInThreads * kInItems;          // records per chunk
+constexpr int kInBlocksPerSM = HBF_IN_BLOCKS;            // resident serve blocks per SM
 constexpr int kInWarps = kInThreads / 32;
-constexpr int kInServers = kInWarps;                     // every warp serves the queues hashed onto it
-constexpr int kInCells = kInItems * kInWarps;            // (row, warp) cells of one server's line of the count matrix
-constexpr int kInCellsPerLane = (kInCells + 31) / 32;
-constexpr int kInSlotBytes = kInChunk * 24;
-constexpr int kInServerBits = kInServers < 16 ? 4 : (kInServers < 32 ? 5 : 6);   // bits of a server number, "none" included
-static_assert(kInServers <= 32, "one lane per server in the offset scan");
-static_assert(kInChunk <= 65536, "positions inside a chunk are 16-bit");
-static_assert((kInServers * kInCells) % 2 == 0, "count matrix is cleared by 32-bit words");
-
-// Lanes of the warp whose low BITS bits of v equal this lane's: one ballot per bit.
-template <int BITS>
-__device__ __forceinline__ unsigned match_bits(uint32_t v) {
-    unsigned m = 0xffffffffu;
-#pragma unroll
-    for (int b = 0; b < BITS; ++b) {
-        const bool one = ((v >> b) & 1u) != 0u;
-        const unsigned bal = __ballot_sync(0xffffffffu, one);
-        m &= one ? bal : ~bal;
-    }
-    return m;
-}
-
-// Which warp serves queue q.  A multiplicative hash, so that streams that step through channels, dies or
-// planes at a fixed stride still spread over all warps.
-__device__ __forceinline__ uint32_t server_of(uint32_t q) {
-    return ((((q + 1u) * 0x9E3779B1u) >> 16) * (uint32_t)kInServers) >> 16;
-}
+static_assert(kInWarps >= 2 && kInWarps <= 15, "every warp owns one of the hardware barriers 1..15");
 
 // One access, from its record: status, and for a modeled access its queue, die and service terms.
 struct Served { int st; uint32_t queue, die, op; int64_t s, xfer, cb; };
@@ -124,21 +98,21 @@ constexpr int kInHead = 8;
 constexpr uint8_t kInStraggler = 0xffu;                   // head count of a (tile, queue) the fix-up hands to the straggle pass
 struct InHead { int64_t m, s; uint32_t xo, idx; };       // arrival + service, service, transfer | op << 31, batch index
 
-// A served record in shared memory (three 64-bit words, in place of the record it came from):
-//   word 0  service ns (32 bits) | transfer ns (20 bits) << 32 | op << 52 | queue << 53
-//   word 1  issue time, as it arrived
-//   word 2  arrival at the queue (issue, plus the transfer for a program) until the record has been served,
-//           its completion time afterwards
-// (for a record that is not modeled word 2 holds the issue time from the start: completion = issue, no stall).
-// A batch with a service time of 2^32 ns or a transfer of 2^20 ns or more in one access goes to the sort path.
-constexpr uint32_t kInXferBits = 20;
-static_assert(kInMaxQueues <= (1u << (64 - 53)), "queue field of a served record");
-
 // ======================================================================================================
 // serve.  RESERVE = false: the streaming pass over every tile, every queue taken as idle at the tile's start.
 // RESERVE = true: only for tiles the fix-up flagged (many queues stayed backlogged far into the tile): the
 // same pass from the true entering busy-until, writing the exact results and nothing else.
+//
+// A tile is cut into rows of 32 consecutive records; warp w takes rows w, w + W, w + 2W, ...  Everything that
+// does not depend on the queues' state (load, classification, decode, service terms, the ranking of lanes that
+// hold the same queue) happens in parallel.  The queue update itself (read the busy-until, serve, write it
+// back: a handful of instructions) is done row after row: the warp of row r waits on a hardware barrier that
+// the warp of row r - 1 arrives at when its update is in shared memory.  Warp w owns barrier 1 + w: it is the
+// only one that waits on it, and warp w - 1 the only one that arrives, so uses of a barrier cannot overlap.
 // ======================================================================================================
+__device__ __forceinline__ void row_wait(int id) { asm volatile("barrier.cta.sync %0, 64;" ::"r"(id) : "memory"); }
+__device__ __forceinline__ void row_pass(int id) { asm volatile("barrier.cta.arrive %0, 64;" ::"r"(id) : "memory"); }
+
 template <bool RESERVE>
 __global__ void __launch_bounds__(kInThreads, kInBlocksPerSM)
 k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_records, const RangeSnap *__restrict__ ranges_g,
@@ -147,16 +121,14 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
                 const int64_t *__restrict__ in_bin, InTile *in_tile, InHead *__restrict__ in_head, uint8_t *__restrict__ in_headcnt) {
     extern __shared__ __align__(16) unsigned char in_smem[];
     __shared__ ModelParams mp;
-    __shared__ uint32_t s_stot[32];                       // records of the chunk per server
     __shared__ long long s_red[2];
     __shared__ FastRange s_fast;
     __shared__ uint32_t s_heads_full;                     // queues whose head entries are complete
-    __shared__ __align__(8) uint64_t s_mbar[2];           // one per record buffer: completion of its bulk load
 
     if (ctrl->skip) return;
     if (RESERVE && (ctrl->run_sort || !ctrl->inorder_used || !in_tile[blockIdx.x].reserve)) return;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const RangeSnap &rs = *ranges_g;                      // read through the cache: shared memory is needed elsewhere
+    const RangeSnap &rs = *ranges_g;                      // read through the cache
     for (int i = tid; i < (int)(sizeof(ModelParams) / 4); i += kInThreads)
         reinterpret_cast<uint32_t *>(&mp)[i] = reinterpret_cast<const uint32_t *>(mp_g)[i];
     const uint32_t R = mp_g->n_queues, n_dies = mp_g->n_dies;
@@ -166,12 +138,9 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
         s_fast = f;
     }
 
-    uint64_t *slot_buf[2] = {reinterpret_cast<uint64_t *>(in_smem), reinterpret_cast<uint64_t *>(in_smem + kInSlotBytes)};
     // [queues] x: busy-until of the run in progress; y: service time served in this tile << 8 | head-table entries written
-    longlong2 *qst = reinterpret_cast<longlong2 *>(in_smem + 2 * kInSlotBytes);
-    uint16_t *list = reinterpret_cast<uint16_t *>(qst + kInMaxQueues);                 // [chunk] positions, server-major, batch order inside
-    uint16_t *cntm = list + kInChunk;                                                  // [server][row][warp] counts, then offsets
-    uint32_t *st_br_lo = reinterpret_cast<uint32_t *>(cntm + kInServers * kInCells), *st_br_hi = st_br_lo + n_dies;   // per die
+    longlong2 *qst = reinterpret_cast<longlong2 *>(in_smem);
+    uint32_t *st_br_lo = reinterpret_cast<uint32_t *>(qst + kInMaxQueues), *st_br_hi = st_br_lo + n_dies;   // per die
     uint32_t *st_bp_lo = st_br_hi + n_dies, *st_bp_hi = st_bp_lo + n_dies;
     uint32_t *st_nr = st_bp_hi + n_dies, *st_np = st_nr + n_dies;
 
@@ -180,17 +149,14 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
     const uint64_t tile_end = min(n, tile_begin + tile_records);
 
     for (uint32_t i = tid; i < kInMaxQueues; i += kInThreads) qst[i] = make_longlong2(kNegInf, 0);
-    for (uint32_t i = tid; i < (uint32_t)(kInServers * kInCells / 2); i += kInThreads) reinterpret_cast<uint32_t *>(cntm)[i] = 0u;
     if (RESERVE) {
         __syncthreads();
         for (uint32_t q = tid; q < R; q += kInThreads) qst[q].x = in_bin[(uint64_t)blockIdx.x * R + q];
     } else {
         for (uint32_t d = tid; d < n_dies * 6u; d += kInThreads) st_br_lo[d] = 0u;
     }
-
     const int64_t q_ppm = ctrl->q_ppm;
     const Div64 div_q = ctrl->div_q;
-    const bool aligned16 = (reinterpret_cast<uintptr_t>(acc) & 15u) == 0;
 
     unsigned long long c_native = 0, c_ready = 0, c_fault = 0;
     unsigned c_unsorted = 0;
@@ -198,198 +164,104 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
 
     if (tid < 2) s_red[tid] = tid == 1 ? INT64_MIN : 0;
     if (tid == 0) s_heads_full = 0u;
+    __syncthreads();
 
-    // Full chunks of a 16-byte aligned batch arrive by bulk asynchronous copy; the last, partial chunk of a tile
-    // and unaligned batches are loaded by the threads.
-    constexpr uint32_t kChunkBytes = (uint32_t)kInChunk * 24u;
-    auto prefetch = [&](uint64_t cb, uint32_t buf) {       // thread 0, after a block barrier that retired the buffer's last use
-        if (aligned16 && cb < tile_end && tile_end - cb >= (uint64_t)kInChunk) {
-            mbar_expect_tx(&s_mbar[buf], kChunkBytes);
-            bulk_load(slot_buf[buf], acc + cb, kChunkBytes, &s_mbar[buf]);
+    const uint64_t rows = tile_end > tile_begin ? (tile_end - tile_begin + 31) / 32 : 0;
+    const unsigned le_mask = lanemask_lt() | (1u << lane);
+    const int my_bar = 1 + warp, next_bar = 1 + (warp + 1 == kInWarps ? 0 : warp + 1);
+
+    // the row after this one is already on its way while this one is served
+    uint64_t nx_addr = 0, nx_issue = 0, nx_bf = 0;
+    auto fetch = [&](uint64_t row) {
+        const uint64_t i = tile_begin + row * 32 + (uint64_t)lane;
+        if (row < rows && i < tile_end) {
+            const uint64_t *rec = reinterpret_cast<const uint64_t *>(acc + i);
+            nx_addr = __ldg(rec); nx_issue = __ldg(rec + 1); nx_bf = __ldg(rec + 2);
         }
     };
-    if (tid == 0) { mbar_init(&s_mbar[0], 1u); mbar_init(&s_mbar[1], 1u); }
-    __syncthreads();
-    if (tid == 0) prefetch(tile_begin, 0u);
-    uint32_t parity_bits = 0u;                              // bit b: parity of buffer b's next completed phase
-    uint32_t chunk_no = 0u;
+    fetch((uint64_t)warp);
 
-    for (uint64_t cbase = tile_begin; cbase < tile_end; cbase += kInChunk, ++chunk_no) {
-        const int cnt = (int)min((uint64_t)kInChunk, tile_end - cbase);
-        const uint32_t buf = chunk_no & 1u;
-        uint64_t *slot = slot_buf[buf];
-                // ---- load: bulk copy issued one chunk ahead, or 16-byte coalesced loads.  The buffer's last readers (the
-        // write-out of two chunks ago) finished before the previous chunk's first barrier.
-        const bool bulk = cnt == kInChunk && aligned16;
-        const uint32_t par = (parity_bits >> buf) & 1u;
-        int timed_out = 0;
-        if (bulk) {
-            timed_out = mbar_wait_bounded(&s_mbar[buf], par) ? 0 : 1;   // on expiry the buffer's content is arbitrary but every
-            parity_bits ^= 1u << buf;                                    // index derived from it stays in range; the barrier below ends the batch
-        } else {
-            const uint64_t *src = reinterpret_cast<const uint64_t *>(acc + cbase);
-            for (int i = tid; i < cnt * 3; i += kInThreads) slot[i] = __ldg(src + i);
-            __syncthreads();
+    for (uint64_t row = (uint64_t)warp; row < rows; row += kInWarps) {
+        const uint64_t i = tile_begin + row * 32 + (uint64_t)lane;
+        const bool valid = i < tile_end;
+        const uint64_t addr = nx_addr, bf = nx_bf;
+        const int64_t issue = (int64_t)nx_issue;
+        fetch(row + kInWarps);
+        if (tile_begin + (row + 2 * kInWarps + 1) * 32 <= tile_end) {   // and the (full) row after that is called into the L2
+            const char *p = reinterpret_cast<const char *>(acc + tile_begin + (row + 2 * kInWarps) * 32) + lane * 32;
+            if (lane < 24) asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
         }
-        // ---- terms, in place: classify, decode, service; rank the record among its warp's records for the same
-        // server.  Word 1 (the issue time) stays as it is, so the issue-order check can read the neighbour's.
-        uint32_t pk[kInItems];                               // rank among the warp's records of this row for the same server | server << 5
-#pragma unroll
-        for (int j = 0; j < kInItems; ++j) {
-            const int e = j * kInThreads + tid;
-            uint32_t srv = (uint32_t)kInServers;             // not modeled
-            if (e < cnt) {
-                const uint64_t addr = slot[e * 3];
-                const int64_t issue = (int64_t)slot[e * 3 + 1];
-                if (!RESERVE) {
-                    const int64_t prev = e > 0 ? (int64_t)slot[e * 3 - 2] : (cbase > 0 ? acc[cbase - 1].issue_ns : INT64_MIN);
-                    c_unsorted |= issue < prev ? 1u : 0u;
-                }
-                const Served v = s_fast.on ? serve_terms_fast(s_fast, mp, addr, issue, slot[e * 3 + 2])
-                                           : serve_terms(rs, mp, addr, issue, slot[e * 3 + 2], q_ppm, div_q);
-                if (!RESERVE && status) status[cbase + e] = (uint8_t)v.st;
-                uint64_t w2 = (uint64_t)issue;               // not modeled: completion = issue (a refused batch is cleared at the end)
-                if (v.st == HBF_ST_READY) {
-                    srv = server_of(v.queue);
-                    const uint32_t xq = ((uint32_t)v.xfer & ((1u << kInXferBits) - 1u)) | (v.op << kInXferBits) | (v.queue << (kInXferBits + 1));
-                    slot[e * 3] = (uint64_t)(uint32_t)v.s | ((uint64_t)xq << 32);
-                    w2 = (uint64_t)(issue + (v.op ? v.xfer : 0));
-                    if (!RESERVE) {
-                        // a service time beyond 32 bits or a transfer beyond 20 bits goes to the sort path
-                        c_unsorted |= (((uint64_t)v.s >> 32) | ((uint64_t)v.xfer >> kInXferBits)) != 0ull ? 1u : 0u;
-                        ++c_ready;
-                        // charged bytes < 2^33: add the low word, carry into the high word when it wraps
-                        const uint32_t lo = (uint32_t)v.cb, hi = (uint32_t)((uint64_t)v.cb >> 32);
-                        uint32_t *plo = v.op ? st_bp_lo : st_br_lo, *phi = v.op ? st_bp_hi : st_br_hi;
-                        atomicAdd(v.op ? &st_np[v.die] : &st_nr[v.die], 1u);
-                        const uint32_t old = atomicAdd(&plo[v.die], lo);
-                        const uint32_t carry = hi + ((old + lo) < old ? 1u : 0u);
-                        if (carry) atomicAdd(&phi[v.die], carry);
-                    }
+        // ---- terms ---------------------------------------------------------------------------------------
+        Served v; v.st = HBF_ST_NATIVE; v.queue = 0; v.die = 0; v.op = 0; v.s = 0; v.xfer = 0; v.cb = 0;
+        if (valid)
+            v = s_fast.on ? serve_terms_fast(s_fast, mp, addr, issue, bf) : serve_terms(rs, mp, addr, issue, bf, q_ppm, div_q);
+        const bool ready = valid && v.st == HBF_ST_READY;
+        if (!RESERVE) {
+            int64_t prev = __shfl_up_sync(0xffffffffu, issue, 1);
+            if (lane == 0) prev = i > 0 ? acc[i - 1].issue_ns : INT64_MIN;
+            if (valid) {
+                c_unsorted |= issue < prev ? 1u : 0u;
+                if (status) status[i] = (uint8_t)v.st;
+                if (ready) {
+                    ++c_ready;
+                    // charged bytes < 2^33: add the low word, carry into the high word when it wraps
+                    const uint32_t lo = (uint32_t)v.cb, hi = (uint32_t)((uint64_t)v.cb >> 32);
+                    uint32_t *plo = v.op ? st_bp_lo : st_br_lo, *phi = v.op ? st_bp_hi : st_br_hi;
+                    atomicAdd(v.op ? &st_np[v.die] : &st_nr[v.die], 1u);
+                    const uint32_t old = atomicAdd(&plo[v.die], lo);
+                    const uint32_t carry = hi + ((old + lo) < old ? 1u : 0u);
+                    if (carry) atomicAdd(&phi[v.die], carry);
                 } else if (v.st == HBF_ST_NATIVE) {
                     ++c_native;
                 } else {
                     ++c_fault;
                 }
-                slot[e * 3 + 2] = w2;
             }
-            const unsigned peers = match_bits<kInServerBits>(srv);     // five ballots: measured faster here than match.any
-            const uint32_t rk = (uint32_t)__popc(peers & lanemask_lt());
-            if (rk == 0u && srv < (uint32_t)kInServers) cntm[(srv * kInItems + j) * kInWarps + warp] = (uint16_t)__popc(peers);
-            pk[j] = rk | (srv << 5);
         }
-        if (__syncthreads_or(timed_out)) {                 // a bulk copy did not complete in time: give the batch up
-            if (tid == 0) atomicExch(&ctrl->code, (int)HBF_E_TIMEOUT);
-            if (bulk) mbar_wait_bounded(&s_mbar[buf], par);  // let the copy in flight land, within the same limit
-            return;
-        }
-        if (tid == 0) prefetch(cbase + kInChunk, buf ^ 1u);   // the next chunk lands while this one is served
-        // ---- offsets: warp w turns the counts of server w, in (row, warp) order, into offsets inside its list --------
-        {
-            uint16_t *m = cntm + warp * kInCells;
-            uint32_t c[kInCellsPerLane], tot = 0;
-#pragma unroll
-            for (int b = 0; b < kInCellsPerLane; ++b) {
-                const int i = lane * kInCellsPerLane + b;
-                c[b] = i < kInCells ? (uint32_t)m[i] : 0u;
-                tot += c[b];
+        const int64_t a = issue + (v.op ? v.xfer : 0);      // arrival at the queue: a program's data is transferred first
+        const uint32_t q = ready ? v.queue : (0x10000u | (uint32_t)lane);
+        const unsigned peers = __match_any_sync(0xffffffffu, q);
+        const unsigned le = peers & le_mask;
+        const uint32_t rank1 = (uint32_t)__popc(le);        // this access is the rank1-th of its queue in the row
+        const uint32_t n_it = __reduce_max_sync(0xffffffffu, rank1);
+        const bool last = ready && (peers >> lane) == 1u;    // no later access of this queue in the row
+        const uint32_t qi = ready ? v.queue : 0u;
+        const bool heads_on = !RESERVE && *reinterpret_cast<volatile uint32_t *>(&s_heads_full) < R;
+        // ---- the queue update, in row order -----------------------------------------------------------------
+        if (row > 0) row_wait(my_bar);
+        const longlong2 state = qst[qi];
+        int64_t B = state.x, sumS = v.s;
+        if (n_it == 1u) {
+            B = max(a, B) + v.s;
+        } else {                                             // lanes holding the same queue chain their accesses in lane order
+            unsigned rem = le;
+            sumS = 0;
+            for (uint32_t it = 0; it < n_it; ++it) {
+                const int src = rem ? __ffs((int)rem) - 1 : lane;
+                const int64_t ab = __shfl_sync(0xffffffffu, a, src), sb = __shfl_sync(0xffffffffu, (int64_t)v.s, src);
+                if (rem) { B = max(ab, B) + sb; sumS += sb; }
+                rem &= rem - 1u;
             }
-            uint32_t incl = tot;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += t; }
-            uint32_t run = incl - tot;
-#pragma unroll
-            for (int b = 0; b < kInCellsPerLane; ++b) {
-                const int i = lane * kInCellsPerLane + b;
-                if (i < kInCells) { m[i] = (uint16_t)run; run += c[b]; }
-            }
-            if (lane == 31) s_stot[warp] = incl;
         }
-        __syncthreads();
-        uint32_t lo, hi;                                     // this warp's list
-        {
-            const uint32_t mine = lane < kInServers ? s_stot[lane] : 0u;
-            uint32_t incl = mine;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += t; }
-            const uint32_t sbase = incl - mine;
-#pragma unroll
-            for (int j = 0; j < kInItems; ++j) {
-                const uint32_t srv = pk[j] >> 5;
-                const uint32_t base = __shfl_sync(0xffffffffu, sbase, (int)srv);
-                if (srv < (uint32_t)kInServers)
-                    list[base + cntm[(srv * kInItems + j) * kInWarps + warp] + (pk[j] & 31u)] = (uint16_t)(j * kInThreads + tid);
-            }
-            lo = __shfl_sync(0xffffffffu, sbase, warp);
-            hi = lo + __shfl_sync(0xffffffffu, mine, warp);
-        }
-        __syncthreads();
-        for (uint32_t i = tid; i < (uint32_t)(kInServers * kInCells / 2); i += kInThreads) reinterpret_cast<uint32_t *>(cntm)[i] = 0u;
-        // ---- serve: each warp walks its list, 32 records at a time.  Lanes holding records of the same queue
-        // chain them in lane (= batch) order: every lane composes the accesses of its queue up to its own.
-        {
-            const bool heads_on = !RESERVE && *reinterpret_cast<volatile uint32_t *>(&s_heads_full) < R;
-            const unsigned le_mask = lanemask_lt() | (1u << lane);
-            for (uint32_t t = lo; t < hi; t += 32u) {
-                const uint32_t k = t + (uint32_t)lane;
-                const bool act = k < hi;
-                const uint32_t e = act ? min((uint32_t)list[k], (uint32_t)(kInChunk - 1)) : 0u;
-                const uint64_t sx = slot[e * 3];
-                const int64_t a = (int64_t)slot[e * 3 + 2];
-                const uint32_t sv = (uint32_t)sx, xq = (uint32_t)(sx >> 32);
-                const uint32_t q = act ? min(xq >> (kInXferBits + 1), R - 1u) : (0x10000u | (uint32_t)lane);
-                const int64_t post = (xq >> kInXferBits) & 1u ? 0 : (int64_t)(xq & ((1u << kInXferBits) - 1u));   // a read's transfer follows its service
-                const unsigned peers = __match_any_sync(0xffffffffu, q);
-                const unsigned le = peers & le_mask;
-                const uint32_t rank1 = (uint32_t)__popc(le);                  // this access is the rank1-th of its queue in the group
-                const uint32_t n_it = __reduce_max_sync(0xffffffffu, rank1);
-                const uint32_t qi = act ? q : 0u;
-                const longlong2 state = qst[qi];
-                int64_t B = state.x;
-                const uint32_t c0 = heads_on ? (uint32_t)state.y & 0xffu : (uint32_t)kInHead;
-                int64_t sumS = (int64_t)sv;
-                if (n_it == 1u) {
-                    B = max(a, B) + (int64_t)sv;
-                } else {
-                    unsigned rem = le;
-                    sumS = 0;
-                    for (uint32_t it = 0; it < n_it; ++it) {
-                        const int src = rem ? __ffs((int)rem) - 1 : lane;
-                        const int64_t ab = __shfl_sync(0xffffffffu, a, src);
-                        const uint32_t sb = __shfl_sync(0xffffffffu, sv, src);
-                        if (rem) { B = max(ab, B) + (int64_t)sb; sumS += (int64_t)sb; }
-                        rem &= rem - 1u;
-                    }
+        const uint32_t c0 = heads_on ? (uint32_t)state.y & 0xffu : (uint32_t)kInHead;
+        const uint32_t c1 = min(c0 + (uint32_t)__popc(peers), (uint32_t)kInHead);
+        if (last) qst[qi] = make_longlong2(B, state.y + (sumS << 8) + (long long)(c1 - c0));
+        if (row + 1 < rows) row_pass(next_bar);
+        // ---- results ---------------------------------------------------------------------------------------
+        if (valid) {
+            int64_t done = issue, st = 0;                    // not modeled: completion = issue, no stall (a refused batch is cleared at the end)
+            if (ready) {
+                done = B + (v.op ? 0 : v.xfer);              // a read's data is transferred after its service
+                st = done - issue;
+                sum_stall += st; max_c = max(max_c, (long long)done);
+                const uint32_t ci = c0 + rank1 - 1u;
+                if (ci < (uint32_t)kInHead) {
+                    InHead h; h.m = a + v.s; h.s = v.s; h.xo = (uint32_t)v.xfer | (v.op << 31); h.idx = (uint32_t)i;
+                    in_head[((uint64_t)tile * kInHead + ci) * R + qi] = h;
                 }
-                if (act) {
-                    slot[e * 3 + 2] = (uint64_t)(B + post);
-                    const uint32_t ci = c0 + rank1 - 1u;
-                    if (ci < (uint32_t)kInHead) {
-                        const uint32_t xfer = xq & ((1u << kInXferBits) - 1u), op = (xq >> kInXferBits) & 1u;
-                        InHead h; h.m = a + (int64_t)sv; h.s = (int64_t)sv; h.xo = xfer | (op << 31); h.idx = (uint32_t)(cbase + e);
-                        in_head[((uint64_t)tile * kInHead + ci) * R + q] = h;
-                    }
-                    if ((peers >> lane) == 1u) {                                // no later access of this queue in the group
-                        const uint32_t c1 = min(c0 + (uint32_t)__popc(peers), (uint32_t)kInHead);
-                        qst[q] = make_longlong2(B, state.y + (sumS << 8) + (long long)(c1 - c0));
-                        if (c1 != c0 && c1 == (uint32_t)kInHead) atomicAdd(&s_heads_full, 1u);
-                    }
-                }
-                __syncwarp();                                // the next group may meet the same queues
+                if (last && c1 != c0 && c1 == (uint32_t)kInHead) atomicAdd(&s_heads_full, 1u);
             }
-        }
-        __syncthreads();
-        // ---- results leave in batch order ----------------------------------------------------------------------
-#pragma unroll
-        for (int j = 0; j < kInItems; ++j) {
-            const int e = j * kInThreads + tid;
-            if (e < cnt) {
-                const int64_t issue = (int64_t)slot[e * 3 + 1], done = (int64_t)slot[e * 3 + 2];
-                const int64_t st = done - issue;             // a modeled access always waits for its service: st > 0
-                completion[cbase + e] = done; stall[cbase + e] = st;
-                sum_stall += st;
-                if (st != 0) max_c = max(max_c, (long long)done);
-            }
+            completion[i] = done; stall[i] = st;
         }
     }
 
@@ -711,16 +583,12 @@ __global__ void k_inorder_total(BatchCtrl *ctrl, const InTile *__restrict__ in_t
 uint64_t inorder_tile_records(uint64_t n, int sm_count) {
     const uint64_t want_tiles = std::min<uint64_t>(kInMaxTiles, (uint64_t)std::max(1, sm_count) * kInBlocksPerSM);   // one wave of resident blocks
     uint64_t t = (n + want_tiles - 1) / want_tiles;
-    t = (t + kInChunk - 1) / kInChunk * kInChunk;
-    return std::max<uint64_t>(t, kInChunk);
+    t = (t + kInTileQuantum - 1) / kInTileQuantum * kInTileQuantum;
+    return std::max<uint64_t>(t, kInTileQuantum);
 }
 
-// dynamic shared memory of the serve kernel: two record buffers, the per-queue state, the servers' lists, the
-// count matrix, per-die counters
-size_t inorder_serve_smem(uint32_t n_dies) {
-    return (size_t)2 * kInSlotBytes + (size_t)kInMaxQueues * 16 + (size_t)kInChunk * 2 + (size_t)kInServers * kInCells * 2 +
-           (size_t)n_dies * 24;
-}
+// dynamic shared memory of the serve kernel: the per-queue state and the per-die counters
+size_t inorder_serve_smem(uint32_t n_dies) { return (size_t)kInMaxQueues * 16 + (size_t)n_dies * 24; }
 static size_t inorder_straggle_smem() { return (size_t)kInMaxQueues * 16 + (size_t)kInStrChunk * 2 + kInMaxQueues; }
 
 size_t inorder_head_bytes(uint64_t tiles, uint32_t n_queues) { return tiles * n_queues * (size_t)kInHead * sizeof(InHead); }
@@ -729,6 +597,7 @@ cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st) {
     const uint64_t n = a.n;
     const uint64_t tile_records = inorder_tile_records(n, a.sm_count);
     const unsigned n_tiles = (unsigned)((n + tile_records - 1) / tile_records);
+    if (n_tiles > inorder_tiles_bound(n)) return cudaErrorInvalidValue;       // the workspace is carved for that many
     const uint32_t R = a.mp.n_queues, nd = a.mp.n_dies;
     const size_t smem_serve = inorder_serve_smem(nd), smem_str = inorder_straggle_smem();
     static size_t set_serve = 0;

@@ -657,7 +657,7 @@ size_t workspace_layout(uint64_t n, uint32_t n_queues, Workspace *ws, void *base
     void *h = take((size_t)kMaxPasses * kRadix * 4);
     void *d0 = take(sort_tiles * kRadix * 4), *d1 = take(sort_tiles * kRadix * 4);
     void *sd = take(scan_tiles * sizeof(ScanDesc));
-    const uint64_t in_tiles = std::min<uint64_t>(kInMaxTiles, (nn + 2047) / 2048);
+    const uint64_t in_tiles = inorder_tiles_bound(nn);
     const bool inorder = n_queues <= kInMaxQueues;
     void *ia = take(inorder ? in_tiles * n_queues * 16 : 0), *ib = take(inorder ? in_tiles * n_queues * 8 : 0);
     void *it = take(inorder ? in_tiles * 32 : 0), *ih = take(inorder ? inorder_head_bytes(in_tiles, n_queues) : 0);

@@ -275,20 +275,17 @@ def test_inorder_other_geometries(hbf, geo):
     compare_batch(g, o, issue_sorted(w.acc))
 
 
-def test_inorder_long_accesses_take_the_sort_path(hbf):
-    """The in-order kernels pack an access's service time into 32 bits of ns and its transfer into 20; a batch
-    with a longer one is served by the sort path (which also leaves the served order behind)."""
+def test_inorder_long_accesses(hbf):
+    """Accesses with a service time beyond 32 bits of ns and a transfer of milliseconds, among ordinary ones."""
     w = wl.tiny_uniform(20_000, seed=4)
     for nbytes, flags in ((32 << 20, 0), (256 << 20, 1)):
         acc = w.acc.copy()
         acc["bytes"][7777] = nbytes
         acc["flags"][7777] = flags
         acc["addr"][7777] = wl.RANGE_BASE                   # the whole span stays inside the 1 GiB range
-        g, o = contexts(hbf, w.profile, w.ranges, hbf.PATH_AUTO)
-        compare_batch(g, o, acc, check_order=True)
-        g, o = contexts(hbf, w.profile, w.ranges, hbf.PATH_INORDER)
-        rc, comp, stall, _, _ = g.submit_host(acc, check=False)
-        assert rc == hbf.E_INVAL and not comp.any() and not stall.any()
+        for path in (hbf.PATH_AUTO, hbf.PATH_INORDER, hbf.PATH_SORT):
+            g, o = contexts(hbf, w.profile, w.ranges, path)
+            compare_batch(g, o, acc)
 
 
 @pytest.mark.parametrize("rho", [0.8, 0.95, 1.2])
