@@ -105,7 +105,7 @@ constexpr int kProfEvents = 10;
 extern unsigned long long g_kernel_launches;
 
 constexpr uint32_t kInMaxQueues = 2048;  // the in-order path keeps per-queue state in shared memory
-constexpr uint32_t kInMaxTiles = 512;
+constexpr uint32_t kInMaxTiles = 1024;
 constexpr uint32_t kInTileQuantum = 1024; // tiles of the in-order path are a multiple of this many records
 // upper bound of the number of tiles of a batch of n records, on any device: what the workspace is carved for
 inline uint64_t inorder_tiles_bound(uint64_t n) {

@@ -110,7 +110,11 @@ struct InHead { int64_t m, s; uint32_t xo, idx; };       // arrival + service, s
 // the warp of row r - 1 arrives at when its update is in shared memory.  Warp w owns barrier 1 + w: it is the
 // only one that waits on it, and warp w - 1 the only one that arrives, so uses of a barrier cannot overlap.
 // ======================================================================================================
-__device__ __forceinline__ void row_wait(int id) { asm volatile("barrier.cta.sync %0, 64;" ::"r"(id) : "memory"); }
+// The extra operands are not used by the instruction: naming them makes the compiler finish computing them
+// before the wait instead of after it.
+__device__ __forceinline__ void row_wait(int id, int64_t m, long long s8, const void *pq, uint32_t pc, bool last) {
+    asm volatile("barrier.cta.sync %0, 64;" ::"r"(id), "l"(m), "l"(s8), "l"(pq), "r"(pc), "r"((int)last) : "memory");
+}
 __device__ __forceinline__ void row_pass(int id) { asm volatile("barrier.cta.arrive %0, 64;" ::"r"(id) : "memory"); }
 
 template <bool RESERVE>
@@ -225,28 +229,33 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
         const uint32_t rank1 = (uint32_t)__popc(le);        // this access is the rank1-th of its queue in the row
         const uint32_t n_it = __reduce_max_sync(0xffffffffu, rank1);
         const bool last = ready && (peers >> lane) == 1u;    // no later access of this queue in the row
-        const uint32_t qi = ready ? v.queue : 0u;
-        const bool heads_on = !RESERVE && *reinterpret_cast<volatile uint32_t *>(&s_heads_full) < R;
-        // ---- the queue update, in row order -----------------------------------------------------------------
-        if (row > 0) row_wait(my_bar);
-        const longlong2 state = qst[qi];
-        int64_t B = state.x, sumS = v.s;
-        if (n_it == 1u) {
-            B = max(a, B) + v.s;
-        } else {                                             // lanes holding the same queue chain their accesses in lane order
-            unsigned rem = le;
-            sumS = 0;
+        // The accesses of this lane's queue in the row, up to this lane's, as one map B -> max(B + S, M): composed
+        // here, in lane order, so that the ordered part below is one application of it whatever the row holds.
+        int64_t S = v.s, M = a + v.s;
+        if (n_it > 1u) {
+            unsigned rem = le & ~(1u << lane);               // earlier lanes of the same queue, lowest first
+            S = 0; M = kNegInf;
             for (uint32_t it = 0; it < n_it; ++it) {
                 const int src = rem ? __ffs((int)rem) - 1 : lane;
                 const int64_t ab = __shfl_sync(0xffffffffu, a, src), sb = __shfl_sync(0xffffffffu, (int64_t)v.s, src);
-                if (rem) { B = max(ab, B) + sb; sumS += sb; }
+                if (rem || it + 1u == rank1) { M = max(M, ab) + sb; S += sb; }     // its peers first, then the lane's own access
                 rem &= rem - 1u;
             }
         }
-        const uint32_t c0 = heads_on ? (uint32_t)state.y & 0xffu : (uint32_t)kInHead;
-        const uint32_t c1 = min(c0 + (uint32_t)__popc(peers), (uint32_t)kInHead);
-        if (last) qst[qi] = make_longlong2(B, state.y + (sumS << 8) + (long long)(c1 - c0));
+        const uint32_t qi = ready ? v.queue : 0u;
+        longlong2 *const pq = qst + qi;
+        const bool heads_on = !RESERVE && *reinterpret_cast<volatile uint32_t *>(&s_heads_full) < R;
+        const long long S8 = S << 8;
+        const uint32_t pc = heads_on ? (uint32_t)__popc(peers) : 0u;
+        // ---- the queue update, in row order: everything it needs is in registers before the wait ------------------
+        if (row > 0) row_wait(my_bar, M, S8, pq, pc, last);
+        const longlong2 state = *pq;
+        const int64_t B = max((int64_t)(state.x + S), M);
+        const uint32_t c0 = min((uint32_t)state.y & 0xffu, (uint32_t)kInHead);
+        const uint32_t inc = min(pc, (uint32_t)kInHead - c0);
+        if (last) *pq = make_longlong2(B, state.y + S8 + (long long)inc);
         if (row + 1 < rows) row_pass(next_bar);
+        const uint32_t c1 = c0 + inc;
         // ---- results ---------------------------------------------------------------------------------------
         if (valid) {
             int64_t done = issue, st = 0;                    // not modeled: completion = issue, no stall (a refused batch is cleared at the end)
@@ -255,7 +264,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
                 st = done - issue;
                 sum_stall += st; max_c = max(max_c, (long long)done);
                 const uint32_t ci = c0 + rank1 - 1u;
-                if (ci < (uint32_t)kInHead) {
+                if (heads_on && ci < (uint32_t)kInHead) {
                     InHead h; h.m = a + v.s; h.s = v.s; h.xo = (uint32_t)v.xfer | (v.op << 31); h.idx = (uint32_t)i;
                     in_head[((uint64_t)tile * kInHead + ci) * R + qi] = h;
                 }
