@@ -311,6 +311,10 @@ int hbf_submit_batch(hbf_ctx *c, const hbf_access_t *d_acc, uint64_t n, int64_t 
     a.ranges = c->d_ranges; a.mp_dev = c->d_mp; a.mp = c->mp; a.state = c->d_state; a.ctrl = c->d_ctrl; a.result = c->d_result;
     a.busy = c->d_busy; a.busy_stage = c->d_busy_stage; a.pending = c->d_pending; a.stats_stage = c->d_stats_stage;
     a.path = c->path; a.sm_count = c->sm_count; a.inorder_ok = c->inorder_ok ? 1 : 0;
+    if (c->ranges.size() == 1) {
+        const HostRange &r = c->ranges[0];
+        a.fast.base = r.base; a.fast.length = r.length; a.fast.media_offset = r.media_offset; a.fast.perms = r.perms; a.fast.on = 1u;
+    }
     c->prof_inorder = c->profiling && n > 0 && c->inorder_ok && (c->path == HBF_PATH_AUTO || c->path == HBF_PATH_INORDER);
     a.ev = c->profiling ? c->ev : nullptr;
     c->prof_submit = c->profiling;

@@ -92,6 +92,10 @@ struct Workspace {
     size_t bytes;
 };
 
+// The registered ranges when there is exactly one of them (on == 0 otherwise): what the in-order kernels take as
+// a kernel argument, so that the common configuration reads nothing from memory to classify an access.
+struct FastRange { uint64_t base, length, media_offset; uint32_t perms, on; };
+
 struct SubmitArgs {
     const hbf_access_t *acc; uint64_t n;
     int64_t *completion, *stall; uint8_t *status; hbf_die_stats_t *die_stats;
@@ -99,6 +103,7 @@ struct SubmitArgs {
     DevState *state; BatchCtrl *ctrl; hbf_batch_result_t *result;
     int64_t *busy, *busy_stage, *pending; hbf_die_stats_t *stats_stage;
     Workspace ws; int32_t path; int sm_count; int inorder_ok;
+    FastRange fast;
     cudaEvent_t *ev;                     // [kProfEvents] or null: recorded between kernel groups
 };
 constexpr int kProfEvents = 10;

@@ -42,6 +42,10 @@ namespace hbf {
 constexpr int kInThreads = HBF_IN_THREADS;               // threads of a serve block
 constexpr int kInBlocksPerSM = HBF_IN_BLOCKS;            // resident serve blocks per SM
 constexpr int kInWarps = kInThreads / 32;
+#ifndef HBF_IN_ROWS
+#define HBF_IN_ROWS 1
+#endif
+constexpr int kInRows = HBF_IN_ROWS;                     // rows of 32 records a warp serves per turn
 static_assert(kInWarps >= 2 && kInWarps <= 15, "every warp owns one of the hardware barriers 1..15");
 
 // One access, from its record: status, and for a modeled access its queue, die and service terms.
@@ -64,7 +68,6 @@ __device__ __forceinline__ Served serve_terms(const RangeSnap &rs, const ModelPa
 
 // The same terms for the common configuration (one registered range, power-of-two geometry, no thermal
 // scaling in force, transfer table present): 32-bit arithmetic wherever the values allow it.
-struct FastRange { uint64_t base, length, media_offset; uint32_t perms, on; };
 __device__ __forceinline__ Served serve_terms_fast(const FastRange &f, const ModelParams &mp, uint64_t addr, int64_t issue, uint64_t bf) {
     Served r; r.queue = 0; r.die = 0; r.op = 0; r.s = 0; r.xfer = 0; r.cb = 0;
     const uint32_t bytes = (uint32_t)bf, flags = (uint32_t)(bf >> 32);
@@ -117,30 +120,34 @@ __device__ __forceinline__ void row_wait(int id, int64_t m, long long s8, const 
 }
 __device__ __forceinline__ void row_pass(int id) { asm volatile("barrier.cta.arrive %0, 64;" ::"r"(id) : "memory"); }
 
+__device__ __forceinline__ void row_wait2(int id, int64_t m, long long s8, const void *pq, uint32_t pc, bool last,
+                                          int64_t m2, long long s82, const void *pq2, uint32_t pc2, bool last2) {
+    asm volatile("barrier.cta.sync %0, 64;" ::"r"(id), "l"(m), "l"(s8), "l"(pq), "r"(pc), "r"((int)last),
+                 "l"(m2), "l"(s82), "l"(pq2), "r"(pc2), "r"((int)last2) : "memory");
+}
+
 template <bool RESERVE>
 __global__ void __launch_bounds__(kInThreads, kInBlocksPerSM)
 k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_records, const RangeSnap *__restrict__ ranges_g,
-                const ModelParams *__restrict__ mp_g, BatchCtrl *ctrl, uint8_t *__restrict__ status, int64_t *__restrict__ in_agg,
+                const __grid_constant__ ModelParams mp_arg, const __grid_constant__ FastRange fast_arg, BatchCtrl *ctrl, uint8_t *__restrict__ status, int64_t *__restrict__ in_agg,
                 hbf_die_stats_t *stats_stage, int64_t *__restrict__ completion, int64_t *__restrict__ stall,
                 const int64_t *__restrict__ in_bin, InTile *in_tile, InHead *__restrict__ in_head, uint8_t *__restrict__ in_headcnt) {
     extern __shared__ __align__(16) unsigned char in_smem[];
-    __shared__ ModelParams mp;
     __shared__ long long s_red[2];
-    __shared__ FastRange s_fast;
     __shared__ uint32_t s_heads_full;                     // queues whose head entries are complete
+    __shared__ ModelParams mp;                            // measured: reads from shared memory beat reads of the argument
+    __shared__ FastRange fast_range;
 
     if (ctrl->skip) return;
     if (RESERVE && (ctrl->run_sort || !ctrl->inorder_used || !in_tile[blockIdx.x].reserve)) return;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const RangeSnap &rs = *ranges_g;                      // read through the cache
-    for (int i = tid; i < (int)(sizeof(ModelParams) / 4); i += kInThreads)
-        reinterpret_cast<uint32_t *>(&mp)[i] = reinterpret_cast<const uint32_t *>(mp_g)[i];
-    const uint32_t R = mp_g->n_queues, n_dies = mp_g->n_dies;
-    if (tid == 0) {
-        FastRange f; f.base = rs.base[0]; f.length = rs.length[0]; f.media_offset = rs.media_offset[0]; f.perms = rs.perms[0];
-        f.on = (rs.count == 1u && mp_g->pow2_geom && mp_g->xfer_tab_max_cb != 0u && ctrl->q_ppm == 1000000) ? 1u : 0u;
-        s_fast = f;
-    }
+    const RangeSnap &rs = *ranges_g;                      // read through the cache; the common configuration does not touch it
+    if (tid == 0) { mp = mp_arg; fast_range = fast_arg; }
+    const uint32_t R = mp_arg.n_queues, n_dies = mp_arg.n_dies;
+    const int64_t q_ppm = ctrl->q_ppm;
+    const Div64 div_q = ctrl->div_q;
+    // one range, power-of-two geometry, transfer table, no thermal scaling in force: the short form of the terms
+    const bool fast_on = fast_arg.on != 0u && mp_arg.pow2_geom != 0u && mp_arg.xfer_tab_max_cb != 0u && q_ppm == 1000000;
 
     // [queues] x: busy-until of the run in progress; y: service time served in this tile << 8 | head-table entries written
     longlong2 *qst = reinterpret_cast<longlong2 *>(in_smem);
@@ -159,9 +166,6 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
     } else {
         for (uint32_t d = tid; d < n_dies * 6u; d += kInThreads) st_br_lo[d] = 0u;
     }
-    const int64_t q_ppm = ctrl->q_ppm;
-    const Div64 div_q = ctrl->div_q;
-
     unsigned long long c_native = 0, c_ready = 0, c_fault = 0;
     unsigned c_unsorted = 0;
     long long sum_stall = 0, max_c = INT64_MIN;
@@ -170,107 +174,153 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
     if (tid == 0) s_heads_full = 0u;
     __syncthreads();
 
+    // A warp's turn covers kInRows consecutive rows: their arithmetic interleaves, and their queue updates
+    // follow one another inside one wait/pass pair.
+    constexpr int K = kInRows;
     const uint64_t rows = tile_end > tile_begin ? (tile_end - tile_begin + 31) / 32 : 0;
+    const uint64_t turns = (rows + K - 1) / K;
     const unsigned le_mask = lanemask_lt() | (1u << lane);
     const int my_bar = 1 + warp, next_bar = 1 + (warp + 1 == kInWarps ? 0 : warp + 1);
 
-    // the row after this one is already on its way while this one is served
-    uint64_t nx_addr = 0, nx_issue = 0, nx_bf = 0;
-    auto fetch = [&](uint64_t row) {
-        const uint64_t i = tile_begin + row * 32 + (uint64_t)lane;
-        if (row < rows && i < tile_end) {
-            const uint64_t *rec = reinterpret_cast<const uint64_t *>(acc + i);
-            nx_addr = __ldg(rec); nx_issue = __ldg(rec + 1); nx_bf = __ldg(rec + 2);
+    // the records of the warp's next turn are already on their way while this one is served
+    uint64_t nx_addr[K], nx_issue[K], nx_bf[K];
+    int64_t nx_prev = INT64_MIN;                             // lane 0: issue time of the record before the turn's first
+#pragma unroll
+    for (int u = 0; u < K; ++u) { nx_addr[u] = 0; nx_issue[u] = 0; nx_bf[u] = 0; }
+    auto fetch = [&](uint64_t turn) {
+#pragma unroll
+        for (int u = 0; u < K; ++u) {
+            const uint64_t i = tile_begin + (turn * K + u) * 32 + (uint64_t)lane;
+            if (i < tile_end) {
+                const uint64_t *rec = reinterpret_cast<const uint64_t *>(acc + i);
+                nx_addr[u] = __ldg(rec); nx_issue[u] = __ldg(rec + 1); nx_bf[u] = __ldg(rec + 2);
+                if (!RESERVE && u == 0 && lane == 0 && i > 0) nx_prev = (int64_t)__ldg(rec - 2);
+            }
         }
     };
     fetch((uint64_t)warp);
 
-    for (uint64_t row = (uint64_t)warp; row < rows; row += kInWarps) {
-        const uint64_t i = tile_begin + row * 32 + (uint64_t)lane;
-        const bool valid = i < tile_end;
-        const uint64_t addr = nx_addr, bf = nx_bf;
-        const int64_t issue = (int64_t)nx_issue;
-        fetch(row + kInWarps);
-        if (tile_begin + (row + 2 * kInWarps + 1) * 32 <= tile_end) {   // and the (full) row after that is called into the L2
-            const char *p = reinterpret_cast<const char *>(acc + tile_begin + (row + 2 * kInWarps) * 32) + lane * 32;
-            if (lane < 24) asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+    for (uint64_t turn = (uint64_t)warp; turn < turns; turn += kInWarps) {
+        uint64_t i[K];
+        bool valid[K], ready[K], last[K];
+        int64_t issue[K], a[K], S[K], M[K], B[K];
+        Served v[K];
+        uint32_t rank1[K], pc[K], c0[K], c1[K], qi[K];
+        longlong2 *pq[K];
+        const int64_t turn_prev = nx_prev;
+        uint64_t addr[K], bf[K];
+#pragma unroll
+        for (int u = 0; u < K; ++u) {
+            i[u] = tile_begin + (turn * K + u) * 32 + (uint64_t)lane;
+            valid[u] = i[u] < tile_end;
+            addr[u] = nx_addr[u]; bf[u] = nx_bf[u]; issue[u] = (int64_t)nx_issue[u];
+        }
+        fetch(turn + kInWarps);
+        {                                                    // and the turn after that is called into the L2
+            const uint64_t first = tile_begin + (turn + 2 * kInWarps) * (uint64_t)(K * 32);
+            if (first + K * 32 <= tile_end) {
+                const char *p = reinterpret_cast<const char *>(acc + first) + lane * 32;
+#pragma unroll
+                for (int u = 0; u < K; ++u)
+                    if (lane < 24) asm volatile("prefetch.global.L2 [%0];" ::"l"(p + u * 768));
+            }
         }
         // ---- terms ---------------------------------------------------------------------------------------
-        Served v; v.st = HBF_ST_NATIVE; v.queue = 0; v.die = 0; v.op = 0; v.s = 0; v.xfer = 0; v.cb = 0;
-        if (valid)
-            v = s_fast.on ? serve_terms_fast(s_fast, mp, addr, issue, bf) : serve_terms(rs, mp, addr, issue, bf, q_ppm, div_q);
-        const bool ready = valid && v.st == HBF_ST_READY;
+#pragma unroll
+        for (int u = 0; u < K; ++u) {
+            v[u].st = HBF_ST_NATIVE; v[u].queue = 0; v[u].die = 0; v[u].op = 0; v[u].s = 0; v[u].xfer = 0; v[u].cb = 0;
+            if (valid[u])
+                v[u] = fast_on ? serve_terms_fast(fast_range, mp, addr[u], issue[u], bf[u])
+                                 : serve_terms(rs, mp, addr[u], issue[u], bf[u], q_ppm, div_q);
+            ready[u] = valid[u] && v[u].st == HBF_ST_READY;
+        }
         if (!RESERVE) {
-            int64_t prev = __shfl_up_sync(0xffffffffu, issue, 1);
-            if (lane == 0) prev = i > 0 ? acc[i - 1].issue_ns : INT64_MIN;
-            if (valid) {
-                c_unsorted |= issue < prev ? 1u : 0u;
-                if (status) status[i] = (uint8_t)v.st;
-                if (ready) {
-                    ++c_ready;
-                    // charged bytes < 2^33: add the low word, carry into the high word when it wraps
-                    const uint32_t lo = (uint32_t)v.cb, hi = (uint32_t)((uint64_t)v.cb >> 32);
-                    uint32_t *plo = v.op ? st_bp_lo : st_br_lo, *phi = v.op ? st_bp_hi : st_br_hi;
-                    atomicAdd(v.op ? &st_np[v.die] : &st_nr[v.die], 1u);
-                    const uint32_t old = atomicAdd(&plo[v.die], lo);
-                    const uint32_t carry = hi + ((old + lo) < old ? 1u : 0u);
-                    if (carry) atomicAdd(&phi[v.die], carry);
-                } else if (v.st == HBF_ST_NATIVE) {
-                    ++c_native;
-                } else {
-                    ++c_fault;
+#pragma unroll
+            for (int u = 0; u < K; ++u) {
+                int64_t prev = __shfl_up_sync(0xffffffffu, issue[u], 1);
+                const int64_t before = u == 0 ? turn_prev : __shfl_sync(0xffffffffu, issue[u == 0 ? 0 : u - 1], 31);
+                if (lane == 0) prev = before;
+                if (valid[u]) {
+                    c_unsorted |= issue[u] < prev ? 1u : 0u;
+                    if (status) status[i[u]] = (uint8_t)v[u].st;
+                    if (ready[u]) {
+                        ++c_ready;
+                        // charged bytes < 2^33: add the low word, carry into the high word when it wraps
+                        const uint32_t lo = (uint32_t)v[u].cb, hi = (uint32_t)((uint64_t)v[u].cb >> 32);
+                        uint32_t *plo = v[u].op ? st_bp_lo : st_br_lo, *phi = v[u].op ? st_bp_hi : st_br_hi;
+                        atomicAdd(v[u].op ? &st_np[v[u].die] : &st_nr[v[u].die], 1u);
+                        const uint32_t old = atomicAdd(&plo[v[u].die], lo);
+                        const uint32_t carry = hi + ((old + lo) < old ? 1u : 0u);
+                        if (carry) atomicAdd(&phi[v[u].die], carry);
+                    } else if (v[u].st == HBF_ST_NATIVE) {
+                        ++c_native;
+                    } else {
+                        ++c_fault;
+                    }
                 }
             }
         }
-        const int64_t a = issue + (v.op ? v.xfer : 0);      // arrival at the queue: a program's data is transferred first
-        const uint32_t q = ready ? v.queue : (0x10000u | (uint32_t)lane);
-        const unsigned peers = __match_any_sync(0xffffffffu, q);
-        const unsigned le = peers & le_mask;
-        const uint32_t rank1 = (uint32_t)__popc(le);        // this access is the rank1-th of its queue in the row
-        const uint32_t n_it = __reduce_max_sync(0xffffffffu, rank1);
-        const bool last = ready && (peers >> lane) == 1u;    // no later access of this queue in the row
-        // The accesses of this lane's queue in the row, up to this lane's, as one map B -> max(B + S, M): composed
-        // here, in lane order, so that the ordered part below is one application of it whatever the row holds.
-        int64_t S = v.s, M = a + v.s;
-        if (n_it > 1u) {
-            unsigned rem = le & ~(1u << lane);               // earlier lanes of the same queue, lowest first
-            S = 0; M = kNegInf;
-            for (uint32_t it = 0; it < n_it; ++it) {
-                const int src = rem ? __ffs((int)rem) - 1 : lane;
-                const int64_t ab = __shfl_sync(0xffffffffu, a, src), sb = __shfl_sync(0xffffffffu, (int64_t)v.s, src);
-                if (rem || it + 1u == rank1) { M = max(M, ab) + sb; S += sb; }     // its peers first, then the lane's own access
-                rem &= rem - 1u;
-            }
-        }
-        const uint32_t qi = ready ? v.queue : 0u;
-        longlong2 *const pq = qst + qi;
         const bool heads_on = !RESERVE && *reinterpret_cast<volatile uint32_t *>(&s_heads_full) < R;
-        const long long S8 = S << 8;
-        const uint32_t pc = heads_on ? (uint32_t)__popc(peers) : 0u;
-        // ---- the queue update, in row order: everything it needs is in registers before the wait ------------------
-        if (row > 0) row_wait(my_bar, M, S8, pq, pc, last);
-        const longlong2 state = *pq;
-        const int64_t B = max((int64_t)(state.x + S), M);
-        const uint32_t c0 = min((uint32_t)state.y & 0xffu, (uint32_t)kInHead);
-        const uint32_t inc = min(pc, (uint32_t)kInHead - c0);
-        if (last) *pq = make_longlong2(B, state.y + S8 + (long long)inc);
-        if (row + 1 < rows) row_pass(next_bar);
-        const uint32_t c1 = c0 + inc;
-        // ---- results ---------------------------------------------------------------------------------------
-        if (valid) {
-            int64_t done = issue, st = 0;                    // not modeled: completion = issue, no stall (a refused batch is cleared at the end)
-            if (ready) {
-                done = B + (v.op ? 0 : v.xfer);              // a read's data is transferred after its service
-                st = done - issue;
-                sum_stall += st; max_c = max(max_c, (long long)done);
-                const uint32_t ci = c0 + rank1 - 1u;
-                if (heads_on && ci < (uint32_t)kInHead) {
-                    InHead h; h.m = a + v.s; h.s = v.s; h.xo = (uint32_t)v.xfer | (v.op << 31); h.idx = (uint32_t)i;
-                    in_head[((uint64_t)tile * kInHead + ci) * R + qi] = h;
+        // ---- per row: the accesses of a lane's queue, up to the lane's own, as one map B -> max(B + S, M), composed
+        // in lane order, so that the ordered part below is one application of it whatever the row holds
+#pragma unroll
+        for (int u = 0; u < K; ++u) {
+            a[u] = issue[u] + (v[u].op ? v[u].xfer : 0);   // arrival at the queue: a program's data is transferred first
+            const uint32_t q = ready[u] ? v[u].queue : (0x10000u | (uint32_t)lane);
+            const unsigned peers = __match_any_sync(0xffffffffu, q);
+            const unsigned le = peers & le_mask;
+            rank1[u] = (uint32_t)__popc(le);               // this access is the rank1-th of its queue in the row
+            const uint32_t n_it = __reduce_max_sync(0xffffffffu, rank1[u]);
+            last[u] = ready[u] && (peers >> lane) == 1u;    // no later access of this queue in the row
+            S[u] = v[u].s; M[u] = a[u] + v[u].s;
+            if (n_it > 1u) {
+                unsigned rem = le & ~(1u << lane);           // earlier lanes of the same queue, lowest first
+                S[u] = 0; M[u] = kNegInf;
+                for (uint32_t it = 0; it < n_it; ++it) {
+                    const int src = rem ? __ffs((int)rem) - 1 : lane;
+                    const int64_t ab = __shfl_sync(0xffffffffu, a[u], src), sb = __shfl_sync(0xffffffffu, (int64_t)v[u].s, src);
+                    if (rem || it + 1u == rank1[u]) { M[u] = max(M[u], ab) + sb; S[u] += sb; }   // its peers first, then the lane's own
+                    rem &= rem - 1u;
                 }
-                if (last && c1 != c0 && c1 == (uint32_t)kInHead) atomicAdd(&s_heads_full, 1u);
             }
-            completion[i] = done; stall[i] = st;
+            qi[u] = ready[u] ? v[u].queue : 0u;
+            pq[u] = qst + qi[u];
+            pc[u] = heads_on ? (uint32_t)__popc(peers) : 0u;
+        }
+        // ---- the queue updates, in row order: everything they need is in registers before the wait ---------------
+        if (turn > 0) {
+            if (K == 1) row_wait(my_bar, M[0], S[0], pq[0], pc[0], last[0]);
+            else row_wait2(my_bar, M[0], S[0], pq[0], pc[0], last[0], M[K - 1], S[K - 1], pq[K - 1], pc[K - 1], last[K - 1]);
+        }
+#pragma unroll
+        for (int u = 0; u < K; ++u) {
+            const longlong2 state = *pq[u];
+            B[u] = max((int64_t)(state.x + S[u]), M[u]);
+            c0[u] = min((uint32_t)state.y & 0xffu, (uint32_t)kInHead);
+            const uint32_t inc = min(pc[u], (uint32_t)kInHead - c0[u]);
+            c1[u] = c0[u] + inc;
+            if (last[u]) *pq[u] = make_longlong2(B[u], state.y + (S[u] << 8) + (long long)inc);
+            if (u + 1 < K) __syncwarp();                     // the next row may hold the same queues
+        }
+        if (turn + 1 < turns) row_pass(next_bar);
+        // ---- results ---------------------------------------------------------------------------------------
+#pragma unroll
+        for (int u = 0; u < K; ++u) {
+            if (valid[u]) {
+                int64_t done = issue[u], st = 0;             // not modeled: completion = issue, no stall (a refused batch is cleared at the end)
+                if (ready[u]) {
+                    done = B[u] + (v[u].op ? 0 : v[u].xfer); // a read's data is transferred after its service
+                    st = done - issue[u];
+                    sum_stall += st; max_c = max(max_c, (long long)done);
+                    const uint32_t ci = c0[u] + rank1[u] - 1u;
+                    if (heads_on && ci < (uint32_t)kInHead) {
+                        InHead h; h.m = a[u] + v[u].s; h.s = v[u].s; h.xo = (uint32_t)v[u].xfer | (v[u].op << 31); h.idx = (uint32_t)i[u];
+                        in_head[((uint64_t)tile * kInHead + ci) * R + qi[u]] = h;
+                    }
+                    if (last[u] && c1[u] != c0[u] && c1[u] == (uint32_t)kInHead) atomicAdd(&s_heads_full, 1u);
+                }
+                completion[i[u]] = done; stall[i[u]] = st;
+            }
         }
     }
 
@@ -621,7 +671,7 @@ cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st) {
     }
     InTile *tiles = reinterpret_cast<InTile *>(a.ws.in_tile);
     InHead *heads = reinterpret_cast<InHead *>(a.ws.in_head);
-    k_inorder_serve<false><<<n_tiles, kInThreads, smem_serve, st>>>(a.acc, n, tile_records, a.ranges, a.mp_dev, a.ctrl, a.status,
+    k_inorder_serve<false><<<n_tiles, kInThreads, smem_serve, st>>>(a.acc, n, tile_records, a.ranges, a.mp, a.fast, a.ctrl, a.status,
                                                                     a.ws.in_agg, a.stats_stage, a.completion, a.stall, a.ws.in_bin,
                                                                     tiles, heads, a.ws.in_headcnt);
     k_inorder_scan<<<(R + kInScanThreads - 1) / kInScanThreads, kInScanThreads, 0, st>>>(
@@ -631,7 +681,7 @@ cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st) {
         R, n_tiles, a.ctrl, a.ws.in_bin, heads, a.ws.in_headcnt, a.completion, a.stall, tiles);
     k_inorder_straggle<<<n_tiles, kInStrThreads, smem_str, st>>>(a.acc, n, tile_records, a.ranges, a.mp_dev, a.ctrl, a.ws.in_bin,
                                                                 a.ws.in_headcnt, a.completion, a.stall, tiles);
-    k_inorder_serve<true><<<n_tiles, kInThreads, smem_serve, st>>>(a.acc, n, tile_records, a.ranges, a.mp_dev, a.ctrl, a.status,
+    k_inorder_serve<true><<<n_tiles, kInThreads, smem_serve, st>>>(a.acc, n, tile_records, a.ranges, a.mp, a.fast, a.ctrl, a.status,
                                                                    a.ws.in_agg, a.stats_stage, a.completion, a.stall, a.ws.in_bin,
                                                                    tiles, heads, a.ws.in_headcnt);
     k_inorder_total<<<1, 256, 0, st>>>(a.ctrl, tiles, n_tiles);
