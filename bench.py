@@ -32,10 +32,10 @@ METRIC = "simulated HBF accesses/s"
 UNIT = "accesses/s"
 ALGO_BYTES_PER_ACCESS = 41            # 24 B record in, 8 B completion + 8 B stall + 1 B status out
 # algorithmic bytes per access of each kernel group (what the kernel itself must move)
-STAGE_BYTES = {"classify": 24 + 8 + 1, "plan_hist": 8, "scan": 8 + 4 + 24 + 16, "inorder": 24 + 16 + 1 + 4}
-# DRAM bytes per access of the in-order serve kernel from one ncu capture (dram__bytes_read + write over a
-# 20 M-access launch, see the summary under profiles/); traffic grows in proportion to the batch
-NCU_TRAFFIC_BYTES_PER_ACCESS = {"inorder": 49.3}
+STAGE_BYTES = {"classify": 24 + 8 + 1, "plan_hist": 8, "scan": 8 + 4 + 24 + 16, "inorder": 24 + 16 + 1}
+# DRAM bytes per access of the in-order serve kernel from one one-pass ncu capture at the full 200 M size
+# (dram__bytes_read + write of one launch, see the summary under profiles/); scaled to the batch in use
+NCU_TRAFFIC_BYTES_PER_ACCESS = {"inorder": 42.6}
 FALLBACK_HBM_GBS = 6650.0
 
 
