@@ -465,7 +465,7 @@ k_inorder_fixup(uint32_t R, uint32_t n_tiles, BatchCtrl *ctrl, const int64_t *__
 // on the serve pass was right.  The block stops at the chunk in which its last queue is done.
 // ======================================================================================================
 constexpr int kInStrThreads = 512;
-constexpr int kInStrItems = 8;
+constexpr int kInStrItems = 4;
 constexpr int kInStrChunk = kInStrThreads * kInStrItems;
 constexpr int kInStrWarps = kInStrThreads / 32;
 constexpr int kInStrCells = kInStrItems * kInStrWarps;    // (row, warp) cells of the kept-record counts
@@ -486,66 +486,79 @@ __device__ __forceinline__ uint32_t fast_queue(const FastRange &f, const ModelPa
 
 __global__ void __launch_bounds__(kInStrThreads)
 k_inorder_straggle(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_records,
-                   const RangeSnap *__restrict__ ranges_g, const ModelParams *__restrict__ mp_g, BatchCtrl *ctrl,
+                   const RangeSnap *__restrict__ ranges_g, const __grid_constant__ ModelParams mp_arg,
+                   const __grid_constant__ FastRange fast_arg, BatchCtrl *ctrl,
                    const int64_t *__restrict__ in_bin, const uint8_t *__restrict__ in_headcnt, int64_t *completion,
                    int64_t *stall, InTile *in_tile) {
     extern __shared__ __align__(16) unsigned char str_smem[];
     __shared__ ModelParams mp;
+    __shared__ FastRange fast_range;
     __shared__ uint32_t s_cells[kInStrCells];
     __shared__ uint32_t s_total;
-    __shared__ int s_open;                                   // straggling queues whose two runs have not met yet
-    __shared__ FastRange s_fast;
+    __shared__ uint32_t s_stragglers;                        // straggling queues of the tile
+    __shared__ int s_open;                                   // those whose two runs have not met yet
+    __shared__ long long s_red[2];
 
     if (ctrl->skip || ctrl->run_sort || !ctrl->inorder_used) return;
     const uint32_t tile = blockIdx.x;
     if (in_tile[tile].stragglers == 0u || in_tile[tile].reserve) return;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const RangeSnap &rs = *ranges_g;
-    for (int i = tid; i < (int)(sizeof(ModelParams) / 4); i += kInStrThreads)
-        reinterpret_cast<uint32_t *>(&mp)[i] = reinterpret_cast<const uint32_t *>(mp_g)[i];
-    const uint32_t R = mp_g->n_queues;
+    const uint32_t R = mp_arg.n_queues;
     int64_t *Bt = reinterpret_cast<int64_t *>(str_smem);                       // [queues] true run
     int64_t *Ba = Bt + kInMaxQueues;                                           // [queues] as-if-idle run
-    uint16_t *list = reinterpret_cast<uint16_t *>(Ba + kInMaxQueues);          // [chunk] positions of the kept records, batch order
-    uint8_t *open = reinterpret_cast<uint8_t *>(list + kInStrChunk);           // [queues] 1: straggler, runs have not met
-    if (tid == 0) {
-        s_open = 0;
-        FastRange f; f.base = rs.base[0]; f.length = rs.length[0]; f.media_offset = rs.media_offset[0]; f.perms = rs.perms[0];
-        f.on = (rs.count == 1u && mp_g->pow2_geom) ? 1u : 0u;
-        s_fast = f;
-    }
+    longlong2 *ent_as = reinterpret_cast<longlong2 *>(Ba + kInMaxQueues);      // [chunk] kept records, batch order: issue time, service time
+    uint2 *ent_pq = reinterpret_cast<uint2 *>(ent_as + kInStrChunk);           //         transfer | op << 31, queue | position << 16
+    uint16_t *oq = reinterpret_cast<uint16_t *>(ent_pq + kInStrChunk);         // [stragglers] their queues
+    uint8_t *open = reinterpret_cast<uint8_t *>(oq + kInMaxQueues);            // [queues] 1: straggler, runs have not met
+    if (tid == 0) { mp = mp_arg; fast_range = fast_arg; s_stragglers = 0u; s_red[0] = 0; s_red[1] = INT64_MIN; }
     __syncthreads();
-    {
-        int mine = 0;
-        for (uint32_t q = tid; q < kInMaxQueues; q += kInStrThreads) {
-            const bool s = q < R && in_headcnt[(uint64_t)tile * R + q] == kInStraggler;
-            open[q] = s ? 1 : 0;
-            Ba[q] = kNegInf;
-            Bt[q] = s ? in_bin[(uint64_t)tile * R + q] : kNegInf;
-            mine += s ? 1 : 0;
-        }
-        if (mine) atomicAdd(&s_open, mine);
+    for (uint32_t q = tid; q < kInMaxQueues; q += kInStrThreads) {
+        const bool s = q < R && in_headcnt[(uint64_t)tile * R + q] == kInStraggler;
+        open[q] = s ? 1 : 0;
+        Ba[q] = kNegInf;
+        Bt[q] = s ? in_bin[(uint64_t)tile * R + q] : kNegInf;
+        if (s) oq[atomicAdd(&s_stragglers, 1u)] = (uint16_t)q;
     }
     const int64_t q_ppm = ctrl->q_ppm;
     const Div64 div_q = ctrl->div_q;
+    const bool one_range = fast_arg.on != 0u && mp_arg.pow2_geom != 0u;
+    const bool fast_terms = one_range && mp_arg.xfer_tab_max_cb != 0u && q_ppm == 1000000;
     const uint64_t tile_begin = (uint64_t)tile * tile_records, tile_end = min(n, tile_begin + tile_records);
     long long dstall = 0, max_c = INT64_MIN;
     __syncthreads();
+    const uint32_t stragglers = s_stragglers;
+    if (tid == 0) s_open = (int)stragglers;
+
+    // the addresses of the next chunk are on their way while this one is filtered
+    uint64_t nx_addr[kInStrItems];
+    auto fetch = [&](uint64_t cb) {
+#pragma unroll
+        for (int j = 0; j < kInStrItems; ++j) {
+            const uint64_t i = cb + (uint64_t)(j * kInStrThreads + tid);
+            nx_addr[j] = i < tile_end ? __ldg(reinterpret_cast<const uint64_t *>(acc + i)) : 0ull;
+        }
+    };
+    fetch(tile_begin);
 
     for (uint64_t cbase = tile_begin; cbase < tile_end; cbase += kInStrChunk) {
         // ---- keep the modeled records of the open queues, in batch order -----------------------------------
+        uint64_t addr[kInStrItems];
+#pragma unroll
+        for (int j = 0; j < kInStrItems; ++j) addr[j] = nx_addr[j];
+        fetch(cbase + kInStrChunk);
         uint32_t keep = 0, rk[kInStrItems];
 #pragma unroll
         for (int j = 0; j < kInStrItems; ++j) {
             const uint64_t i = cbase + (uint64_t)(j * kInStrThreads + tid);
             bool k = false;
             if (i < tile_end) {
-                const uint64_t *rec = reinterpret_cast<const uint64_t *>(acc + i);
-                if (s_fast.on) {
-                    const uint32_t q = fast_queue(s_fast, mp, __ldg(rec));
+                if (one_range) {
+                    const uint32_t q = fast_queue(fast_range, mp, addr[j]);
                     k = q != 0xffffffffu && open[q] != 0;
                 } else {
-                    const Served v = serve_terms(rs, mp, __ldg(rec), (int64_t)__ldg(rec + 1), __ldg(rec + 2), q_ppm, div_q);
+                    const uint64_t *rec = reinterpret_cast<const uint64_t *>(acc + i);
+                    const Served v = serve_terms(rs, mp, addr[j], (int64_t)__ldg(rec + 1), __ldg(rec + 2), q_ppm, div_q);
                     k = v.st == HBF_ST_READY && open[v.queue] != 0;
                 }
             }
@@ -570,60 +583,55 @@ k_inorder_straggle(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t ti
         __syncthreads();
 #pragma unroll
         for (int j = 0; j < kInStrItems; ++j)
-            if (keep & (1u << j)) list[s_cells[j * kInStrWarps + warp] + rk[j]] = (uint16_t)(j * kInStrThreads + tid);
-        __syncthreads();
-        // ---- the first warp re-serves them ---------------------------------------------------------------
-        if (warp == 0) {
-            const uint32_t total = s_total;
-            const unsigned le_mask = lanemask_lt() | (1u << lane);
-            for (uint32_t t = 0; t < total; t += 32u) {
-                const uint32_t k = t + (uint32_t)lane;
-                const bool act = k < total;
-                uint64_t i = cbase;
-                uint32_t q = 0x10000u | (uint32_t)lane;
-                int64_t issue = 0, a = 0, sv = 0, post = 0;
-                if (act) {
-                    i = min(cbase + list[k], tile_end - 1);
-                    const uint64_t *rec = reinterpret_cast<const uint64_t *>(acc + i);
-                    issue = (int64_t)__ldg(rec + 1);
-                    const Served v = serve_terms(rs, mp, __ldg(rec), issue, __ldg(rec + 2), q_ppm, div_q);
-                    q = v.queue; sv = v.s; a = issue + (v.op ? v.xfer : 0); post = v.op ? 0 : v.xfer;
-                }
-                const unsigned peers = __match_any_sync(0xffffffffu, q);
-                const unsigned le = peers & le_mask;
-                const uint32_t n_it = __reduce_max_sync(0xffffffffu, (uint32_t)__popc(le));
-                const uint32_t qi = act ? q : 0u;
-                int64_t BT = Bt[qi], BA = Ba[qi];
-                unsigned rem = le;
-                for (uint32_t it = 0; it < n_it; ++it) {
-                    const int src = rem ? __ffs((int)rem) - 1 : lane;
-                    const int64_t ab = __shfl_sync(0xffffffffu, a, src), sb = __shfl_sync(0xffffffffu, sv, src);
-                    if (rem) { BT = max(ab, BT) + sb; BA = max(ab, BA) + sb; }
-                    rem &= rem - 1u;
-                }
-                if (act) {
-                    if ((peers >> lane) == 1u) {               // last access of this queue in the group
-                        Bt[q] = BT; Ba[q] = BA;
-                        if (BT == BA && open[q]) { open[q] = 0; atomicSub(&s_open, 1); }
-                    }
-                    if (BT != BA) {                             // the serve pass wrote BA + post
-                        const int64_t done = BT + post;
-                        completion[i] = done; stall[i] = done - issue;
-                        dstall += BT - BA; max_c = max(max_c, (long long)done);
-                    }
-                }
-                __syncwarp();
+            if (keep & (1u << j)) {                          // few records are kept: their terms are computed here, once
+                const uint32_t e = (uint32_t)(j * kInStrThreads + tid);
+                const uint64_t *rec = reinterpret_cast<const uint64_t *>(acc + cbase + e);
+                const int64_t issue = (int64_t)__ldg(rec + 1);
+                const uint64_t bf = __ldg(rec + 2);
+                const Served v = fast_terms ? serve_terms_fast(fast_range, mp, addr[j], issue, bf)
+                                            : serve_terms(rs, mp, addr[j], issue, bf, q_ppm, div_q);
+                const uint32_t pos = s_cells[j * kInStrWarps + warp] + rk[j];
+                ent_as[pos] = make_longlong2(issue, v.s);
+                ent_pq[pos] = make_uint2((uint32_t)v.xfer | (v.op << 31), v.queue | (e << 16));
             }
+        __syncthreads();
+        // ---- one thread per straggling queue walks the kept records (they are in batch order) and re-serves its own
+        // (spread over the warps first, then over their lanes: lanes of a warp that find their records diverge)
+        for (uint32_t t = (uint32_t)(lane * kInStrWarps + warp); t < stragglers; t += kInStrThreads) {
+            const uint32_t q = oq[t];
+            if (!open[q]) continue;
+            const uint32_t total = min(s_total, (uint32_t)kInStrChunk);
+            int64_t BT = Bt[q], BA = Ba[q];
+            for (uint32_t k = 0; k < total; ++k) {
+                const uint2 pq = ent_pq[k];
+                if ((pq.y & 0xffffu) != q) continue;
+                const longlong2 as = ent_as[k];
+                const int64_t xfer = (int64_t)(pq.x & 0x7fffffffu);
+                const bool op = (pq.x >> 31) != 0u;
+                const int64_t a = as.x + (op ? xfer : 0);
+                BT = max(a, BT) + as.y; BA = max(a, BA) + as.y;
+                if (BT != BA) {                               // the serve pass wrote BA + post
+                    const uint64_t i = min(cbase + (pq.y >> 16), tile_end - 1);
+                    const int64_t done = BT + (op ? 0 : xfer);
+                    completion[i] = done; stall[i] = done - as.x;
+                    dstall += BT - BA; max_c = max(max_c, (long long)done);
+                }
+            }
+            Bt[q] = BT; Ba[q] = BA;
+            if (BT == BA) { open[q] = 0; atomicSub(&s_open, 1); }   // the runs have met: the rest of the tile was served right
         }
         __syncthreads();
         if (*reinterpret_cast<volatile int *>(&s_open) <= 0) break;
     }
-    if (warp == 0) {
-        dstall = warp_sum(dstall); max_c = warp_max(max_c);
-        if (lane == 0) {
-            if (dstall) atomicAdd((unsigned long long *)&in_tile[tile].fix_delta, (unsigned long long)dstall);
-            if (max_c != INT64_MIN) atomicMax(&ctrl->max_completion_ns, max_c);
-        }
+    dstall = warp_sum(dstall); max_c = warp_max(max_c);
+    if (lane == 0) {
+        if (dstall) atomicAdd((unsigned long long *)&s_red[0], (unsigned long long)dstall);
+        if (max_c != INT64_MIN) atomicMax(&s_red[1], max_c);
+    }
+    __syncthreads();
+    if (tid == 0) {
+        if (s_red[0]) atomicAdd((unsigned long long *)&in_tile[tile].fix_delta, (unsigned long long)s_red[0]);
+        if (s_red[1] != INT64_MIN) atomicMax(&ctrl->max_completion_ns, s_red[1]);
     }
 }
 
@@ -648,7 +656,7 @@ uint64_t inorder_tile_records(uint64_t n, int sm_count) {
 
 // dynamic shared memory of the serve kernel: the per-queue state and the per-die counters
 size_t inorder_serve_smem(uint32_t n_dies) { return (size_t)kInMaxQueues * 16 + (size_t)n_dies * 24; }
-static size_t inorder_straggle_smem() { return (size_t)kInMaxQueues * 16 + (size_t)kInStrChunk * 2 + kInMaxQueues; }
+static size_t inorder_straggle_smem() { return (size_t)kInMaxQueues * 16 + (size_t)kInStrChunk * 24 + (size_t)kInMaxQueues * 3; }
 
 size_t inorder_head_bytes(uint64_t tiles, uint32_t n_queues) { return tiles * n_queues * (size_t)kInHead * sizeof(InHead); }
 
@@ -679,7 +687,7 @@ cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st) {
     const uint64_t fix_threads = (uint64_t)n_tiles * R;
     k_inorder_fixup<<<(unsigned)((fix_threads + kInFixThreads - 1) / kInFixThreads), kInFixThreads, 0, st>>>(
         R, n_tiles, a.ctrl, a.ws.in_bin, heads, a.ws.in_headcnt, a.completion, a.stall, tiles);
-    k_inorder_straggle<<<n_tiles, kInStrThreads, smem_str, st>>>(a.acc, n, tile_records, a.ranges, a.mp_dev, a.ctrl, a.ws.in_bin,
+    k_inorder_straggle<<<n_tiles, kInStrThreads, smem_str, st>>>(a.acc, n, tile_records, a.ranges, a.mp, a.fast, a.ctrl, a.ws.in_bin,
                                                                 a.ws.in_headcnt, a.completion, a.stall, tiles);
     k_inorder_serve<true><<<n_tiles, kInThreads, smem_serve, st>>>(a.acc, n, tile_records, a.ranges, a.mp, a.fast, a.ctrl, a.status,
                                                                    a.ws.in_agg, a.stats_stage, a.completion, a.stall, a.ws.in_bin,
