@@ -77,6 +77,11 @@ int  hbfo_register_range(hbfo_ctx *ctx, uint64_t base, uint64_t length, uint32_t
 int  hbfo_clear_ranges(hbfo_ctx *ctx);
 int  hbfo_submit_batch(hbfo_ctx *ctx, const hbfo_access_t *acc, uint64_t n, int64_t *completion_ns,
                        int64_t *stall_ns, uint8_t *status, hbfo_die_stats_t *die_stats);
+/* Page-granular variant (this build's extension; the paper's back end is a page-based flash simulator but the
+ * text does not spell the splitting out): every page of a modeled access is a request of its own, queued by
+ * its own decode; the access completes with its last part.  Same arguments as hbfo_submit_batch. */
+int  hbfo_submit_batch_paged(hbfo_ctx *ctx, const hbfo_access_t *acc, uint64_t n, int64_t *completion_ns,
+                             int64_t *stall_ns, uint8_t *status, hbfo_die_stats_t *die_stats);
 int  hbfo_last_result(hbfo_ctx *ctx, hbfo_batch_result_t *out);
 /* The order in which the last accepted batch was served: indices, queue-major. */
 int  hbfo_last_order(hbfo_ctx *ctx, uint32_t *order, uint64_t cap, uint64_t *count);

@@ -87,6 +87,8 @@ def lib():
         L.hbfo_clear_ranges.argtypes = [C.c_void_p]
         L.hbfo_submit_batch.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p, C.c_void_p,
                                         C.c_void_p, C.c_void_p]
+        L.hbfo_submit_batch_paged.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p, C.c_void_p,
+                                        C.c_void_p, C.c_void_p]
         L.hbfo_last_result.argtypes = [C.c_void_p, C.POINTER(BatchResult)]
         L.hbfo_last_order.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.POINTER(C.c_uint64)]
         L.hbfo_thermal_step.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p]
@@ -170,16 +172,16 @@ class Oracle:
     def clear_ranges(self):
         lib().hbfo_clear_ranges(self._h)
 
-    def submit(self, acc: np.ndarray, check=True):
-        """Returns (code, completion, stall, status, die_stats)."""
+    def submit(self, acc: np.ndarray, check=True, paged=False):
+        """Returns (code, completion, stall, status, die_stats).  paged: every page of an access is a request of its own."""
         acc = np.ascontiguousarray(acc, dtype=ACCESS_DTYPE)
         n = acc.shape[0]
         comp = np.empty(n, np.int64)
         stall = np.empty(n, np.int64)
         status = np.empty(n, np.uint8)
         ds = np.zeros(self.n_dies, DIE_STATS_DTYPE)
-        rc = lib().hbfo_submit_batch(self._h, acc.ctypes.data, n, comp.ctypes.data, stall.ctypes.data,
-                                     status.ctypes.data, ds.ctypes.data)
+        fn = lib().hbfo_submit_batch_paged if paged else lib().hbfo_submit_batch
+        rc = fn(self._h, acc.ctypes.data, n, comp.ctypes.data, stall.ctypes.data, status.ctypes.data, ds.ctypes.data)
         if check and rc != 0:
             raise OracleError(rc)
         return rc, comp, stall, status, ds
