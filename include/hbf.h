@@ -126,6 +126,25 @@ HBF_API int hbf_submit_batch(hbf_ctx *ctx, const hbf_access_t *d_acc, uint64_t n
                      int64_t *d_stall_ns, uint8_t *d_status, hbf_die_stats_t *d_die_stats,
                      void *d_workspace, size_t workspace_bytes);
 
+/* Page-granular variant of hbf_submit_batch (an extension: the paper's back end is a page-based flash simulator,
+ * Section "Design", but the text does not define the splitting; this is the library's definition).  A modeled
+ * access is cut at the page boundaries of the media; every part is a request of its own: decoded by its own
+ * first byte (so consecutive pages follow the stripe interleave), charged one page of array time (Eq. 3) and
+ * the transfer of its own bytes in whole granules, queued in (issue_ns, access index, part index) order.  The
+ * access completes when its last part does; d_stall_ns[i] = completion - issue.  d_die_stats counts parts
+ * (page operations); the batch summary read with hbf_last_result counts accesses.  An access that is not
+ * modeled (native, or failing) is one part.
+ * parts_capacity: upper bound, chosen by the caller, of the number of parts of the batch (at least n; e.g.
+ * n * (largest access / page_bytes + 2)); it sizes the workspace, hbf_workspace_bytes_paged(ctx, n, capacity).
+ * The call counts the parts on the device and waits for that count (one stream synchronisation) before it
+ * launches the rest; with more parts than parts_capacity it returns HBF_E_WORKSPACE and nothing has changed.
+ * Other arguments, ownership and error behaviour as for hbf_submit_batch.  hbf_queue_order afterwards refers
+ * to parts, not accesses. */
+HBF_API size_t hbf_workspace_bytes_paged(const hbf_ctx *ctx, uint64_t n, uint64_t parts_capacity);
+HBF_API int hbf_submit_batch_paged(hbf_ctx *ctx, const hbf_access_t *d_acc, uint64_t n, uint64_t parts_capacity,
+                           int64_t *d_completion_ns, int64_t *d_stall_ns, uint8_t *d_status,
+                           hbf_die_stats_t *d_die_stats, void *d_workspace, size_t workspace_bytes);
+
 /* Waits for the last submitted batch and copies its summary to host_out; returns its code. */
 HBF_API int hbf_last_result(hbf_ctx *ctx, hbf_batch_result_t *host_out);
 

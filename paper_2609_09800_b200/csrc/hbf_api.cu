@@ -323,6 +323,53 @@ int hbf_submit_batch(hbf_ctx *c, const hbf_access_t *d_acc, uint64_t n, int64_t 
     return HBF_OK;
 }
 
+size_t hbf_workspace_bytes_paged(const hbf_ctx *c, uint64_t n, uint64_t parts_capacity) {
+    if (!c) return 0;
+    return paged_layout(n, std::max<uint64_t>(parts_capacity, n), c->mp.n_queues, nullptr, nullptr);
+}
+
+int hbf_submit_batch_paged(hbf_ctx *c, const hbf_access_t *d_acc, uint64_t n, uint64_t parts_capacity,
+                           int64_t *d_completion_ns, int64_t *d_stall_ns, uint8_t *d_status, hbf_die_stats_t *d_die_stats,
+                           void *d_workspace, size_t workspace_bytes) {
+    if (!c) return HBF_E_INVAL;
+    if (n == 0)                                             // nothing to split: the ordinary path reports the empty batch
+        return hbf_submit_batch(c, d_acc, 0, d_completion_ns, d_stall_ns, d_status, d_die_stats, d_workspace, workspace_bytes);
+    if (c->terminal) return HBF_E_LINK_SHUTDOWN;
+    if (n > HBF_MAX_BATCH) return HBF_E_INVAL;
+    if (!d_acc || !d_completion_ns || !d_stall_ns) return HBF_E_INVAL;
+    if ((reinterpret_cast<uintptr_t>(d_acc) & 7u) || (reinterpret_cast<uintptr_t>(d_completion_ns) & 7u) ||
+        (reinterpret_cast<uintptr_t>(d_stall_ns) & 7u) || (reinterpret_cast<uintptr_t>(d_die_stats) & 7u)) return HBF_E_INVAL;
+    const uint64_t capacity = std::min<uint64_t>(std::max<uint64_t>(parts_capacity, n), HBF_MAX_BATCH);
+    PagedWorkspace pw{};
+    const size_t need = paged_layout(n, capacity, c->mp.n_queues, &pw, d_workspace);
+    if (!d_workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(d_workspace) & 255u)) return HBF_E_WORKSPACE;
+    // how many parts: the one point where the host waits for the device inside a submit
+    CK(launch_paged_count(d_acc, n, c->d_ranges, c->d_mp, pw, c->stream));
+    unsigned long long *h_total = reinterpret_cast<unsigned long long *>(c->h_result);     // pinned, free between calls
+    CK(cudaMemcpyAsync(h_total, pw.total, sizeof(unsigned long long), cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    const uint64_t total = *h_total;
+    if (total > capacity) return HBF_E_WORKSPACE;            // nothing has changed: the caller may come back with more room
+    CK(launch_paged_expand(d_acc, n, c->d_ranges, c->d_mp, capacity, pw, c->stream));
+    SubmitArgs a{};
+    workspace_layout(total, c->mp.n_queues, &a.ws, pw.inner);
+    a.acc = pw.parts; a.n = total; a.completion = pw.part_completion; a.stall = pw.part_stall; a.status = pw.part_status;
+    a.die_stats = d_die_stats;
+    a.ranges = c->d_ranges; a.mp_dev = c->d_mp; a.mp = c->mp; a.state = c->d_state; a.ctrl = c->d_ctrl; a.result = c->d_result;
+    a.busy = c->d_busy; a.busy_stage = c->d_busy_stage; a.pending = c->d_pending; a.stats_stage = c->d_stats_stage;
+    a.path = c->path; a.sm_count = c->sm_count; a.inorder_ok = c->inorder_ok ? 1 : 0;
+    if (c->ranges.size() == 1) {
+        const HostRange &r = c->ranges[0];
+        a.fast.base = r.base; a.fast.length = r.length; a.fast.media_offset = r.media_offset; a.fast.perms = r.perms; a.fast.on = 1u;
+    }
+    c->prof_inorder = false; c->prof_submit = false;
+    a.ev = nullptr;
+    CK(launch_submit(a, c->stream));
+    CK(launch_paged_join(d_acc, n, pw, c->d_result, d_completion_ns, d_stall_ns, d_status, c->sm_count, c->stream));
+    c->submitted = true;
+    return HBF_OK;
+}
+
 int hbf_last_result(hbf_ctx *c, hbf_batch_result_t *host_out) {
     if (!c || !host_out) return HBF_E_INVAL;
     if (!c->submitted) { memset(host_out, 0, sizeof(*host_out)); return HBF_OK; }

@@ -126,6 +126,25 @@ cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st);
 cudaError_t launch_submit(const SubmitArgs &a, cudaStream_t st);
 cudaError_t launch_queue_order(const BatchCtrl *ctrl, const Workspace &ws, uint32_t *out, uint64_t n, cudaStream_t st);
 
+// ---- page-granular submit ---------------------------------------------------------------------------
+struct PagedWorkspace {
+    unsigned long long *tile_sum;        // [tiles of 2,048 accesses] parts per tile, then exclusive offsets
+    unsigned long long *total;           // parts of the batch
+    void *sums;                          // accesses served and their stall total
+    uint32_t *part_first;                // [n + 1] first part of every access
+    hbf_access_t *parts;                 // [capacity] the parts as access records
+    int64_t *part_completion, *part_stall; uint8_t *part_status;
+    void *inner; size_t inner_bytes;     // workspace of the ordinary path for `capacity` records
+    size_t bytes;
+};
+size_t paged_layout(uint64_t n, uint64_t capacity, uint32_t n_queues, PagedWorkspace *pw, void *base);
+cudaError_t launch_paged_count(const hbf_access_t *acc, uint64_t n, const RangeSnap *ranges, const ModelParams *mp_dev,
+                               const PagedWorkspace &pw, cudaStream_t st);
+cudaError_t launch_paged_expand(const hbf_access_t *acc, uint64_t n, const RangeSnap *ranges, const ModelParams *mp_dev,
+                                uint64_t capacity, const PagedWorkspace &pw, cudaStream_t st);
+cudaError_t launch_paged_join(const hbf_access_t *acc, uint64_t n, const PagedWorkspace &pw, hbf_batch_result_t *result,
+                              int64_t *completion, int64_t *stall, uint8_t *status, int sm_count, cudaStream_t st);
+
 // ---- thermal -------------------------------------------------------------------------------------
 struct ThermalDev {
     uint32_t H, W, n_regions, n_dies, n_sub;

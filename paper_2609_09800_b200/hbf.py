@@ -28,7 +28,8 @@ EXPORTS = ("hbf_create", "hbf_destroy", "hbf_register_range", "hbf_clear_ranges"
            "hbf_submit_batch", "hbf_last_result", "hbf_thermal_step", "hbf_force_mode", "hbf_get_mode",
            "hbf_reset", "hbf_set_path", "hbf_get_state", "hbf_set_state", "hbf_get_busy_until",
            "hbf_get_pending_energy", "hbf_get_temps", "hbf_euler_limit_ns", "hbf_queue_order", "hbf_strerror",
-           "hbf_set_profiling", "hbf_get_profile", "hbf_kernel_launches", "hbf_euler_substeps_static", "hbf_set_thermal_path")
+           "hbf_set_profiling", "hbf_get_profile", "hbf_kernel_launches", "hbf_euler_substeps_static", "hbf_set_thermal_path",
+           "hbf_workspace_bytes_paged", "hbf_submit_batch_paged")
 STATIC_MAX_CELLS = 65536
 PROF_STAGES = ("begin", "classify", "plan_hist", "sort", "scan", "finish", "inorder", "thermal")
 
@@ -85,6 +86,9 @@ def lib():
         L.hbf_workspace_bytes.argtypes = [vp, u64]
         L.hbf_workspace_bytes.restype = C.c_size_t
         L.hbf_submit_batch.argtypes = [vp, vp, u64, vp, vp, vp, vp, vp, C.c_size_t]
+        L.hbf_workspace_bytes_paged.argtypes = [vp, u64, u64]
+        L.hbf_workspace_bytes_paged.restype = C.c_size_t
+        L.hbf_submit_batch_paged.argtypes = [vp, vp, u64, u64, vp, vp, vp, vp, vp, C.c_size_t]
         L.hbf_last_result.argtypes = [vp, C.POINTER(hbf_batch_result_t)]
         L.hbf_thermal_step.argtypes = [vp, i64, vp, u32, vp, vp]
         L.hbf_force_mode.argtypes = [vp, i32, i64]
@@ -225,6 +229,21 @@ class Context:
         return lib().hbf_submit_batch(self._h, _ptr(d_acc), n, _ptr(d_completion), _ptr(d_stall), _ptr(d_status),
                                       _ptr(d_die_stats), _ptr(ws), ws.numel() * ws.element_size())
 
+    def workspace_bytes_paged(self, n: int, parts_capacity: int) -> int:
+        return lib().hbf_workspace_bytes_paged(self._h, n, parts_capacity)
+
+    def submit_batch_paged(self, d_acc, n, parts_capacity, d_completion, d_stall, d_status=None, d_die_stats=None,
+                           d_workspace=None):
+        """Page-granular submit: every page of an access is queued on its own (see hbf_submit_batch_paged)."""
+        if d_workspace is None:
+            need = self.workspace_bytes_paged(n, parts_capacity)
+            if self._ws is None or self._ws.numel() < need:
+                self._ws = self._torch.empty(need, dtype=self._torch.uint8, device="cuda")
+            d_workspace = self._ws
+        return lib().hbf_submit_batch_paged(self._h, _ptr(d_acc), n, parts_capacity, _ptr(d_completion), _ptr(d_stall),
+                                            _ptr(d_status), _ptr(d_die_stats), _ptr(d_workspace),
+                                            d_workspace.numel() * d_workspace.element_size())
+
     def last_result(self) -> dict:
         r = hbf_batch_result_t()
         lib().hbf_last_result(self._h, C.byref(r))
@@ -329,9 +348,10 @@ class Context:
             raise HbfError(rc, "hbf_set_state")
 
     # ---- host-buffer convenience: copies in, one submit, copies out ---------------------------------
-    def submit_host(self, acc: np.ndarray, want_status=True, check=True):
-        """Marshals a host batch through the device: H2D of the records, ``hbf_submit_batch``, D2H of
-        completions, stalls, status and per-die stats.  Returns (code, completion, stall, status, die_stats)."""
+    def submit_host(self, acc: np.ndarray, want_status=True, check=True, parts_capacity=None):
+        """Marshals a host batch through the device: H2D of the records, ``hbf_submit_batch`` (or, with
+        parts_capacity given, ``hbf_submit_batch_paged``), D2H of completions, stalls, status and per-die stats.
+        Returns (code, completion, stall, status, die_stats)."""
         torch = self._torch
         acc = np.ascontiguousarray(acc, dtype=ACCESS_DTYPE)
         n = acc.shape[0]
@@ -341,7 +361,10 @@ class Context:
             d_stall = torch.empty(n, dtype=torch.int64, device="cuda")
             d_status = torch.empty(n, dtype=torch.uint8, device="cuda") if want_status else None
             d_ds = torch.empty(self.n_dies * 6, dtype=torch.int64, device="cuda")
-            rc = self.submit_batch(d_acc, n, d_comp, d_stall, d_status, d_ds)
+            if parts_capacity is None:
+                rc = self.submit_batch(d_acc, n, d_comp, d_stall, d_status, d_ds)
+            else:
+                rc = self.submit_batch_paged(d_acc, n, parts_capacity, d_comp, d_stall, d_status, d_ds)
             if rc != 0:
                 if check:
                     raise HbfError(rc, "hbf_submit_batch")
