@@ -51,8 +51,9 @@ def parse_args():
     ap.add_argument("--cpu-sample", type=int, default=20_000_000)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--workload", default="capacity_mode", choices=["capacity_mode", "coupled_thermal"],
-                    help="coupled_thermal: the prefix-KV stream in 1 ms batches, each followed by a thermal step (not the headline)")
+    ap.add_argument("--workload", default="capacity_mode", choices=["capacity_mode", "coupled_thermal", "capacity_paged"],
+                    help="coupled_thermal: the prefix-KV stream in 1 ms batches, each followed by a thermal step; "
+                         "capacity_paged: the capacity-mode batch through the page-granular submit (neither is the headline)")
     ap.add_argument("--horizon-ms", type=int, default=1000, help="simulated time of the coupled_thermal run")
     return ap.parse_args()
 
@@ -228,6 +229,67 @@ def run_coupled(args):
     print(json.dumps(line), flush=True)
 
 
+def run_paged(args):
+    """The capacity-mode batch through hbf_submit_batch_paged on one GPU: every page of a read queued on its own."""
+    import torch
+    from paper_2609_09800_b200 import build as hbf_build, hbf
+    hbf_build.build()
+    n = args.n
+    w, gen_s = make_stream(n, seed=0)
+    fp = wl.package_floorplan(channels=w.profile["channels"], dies=w.profile["dies"])
+    ctx = hbf.Context(w.profile, fp)
+    for r in w.ranges:
+        ctx.register_range(*r)
+    page = w.profile["page_bytes"]
+    off = w.acc["addr"] - np.uint64(w.ranges[0][0])
+    parts = int(((off % np.uint64(page) + w.acc["bytes"] + np.uint64(page - 1)) // np.uint64(page)).sum())
+    d_acc = torch.from_numpy(w.acc.view(np.int64).reshape(-1)).cuda()
+    d_comp = torch.empty(n, dtype=torch.int64, device="cuda"); d_stall = torch.empty_like(d_comp)
+    d_status = torch.empty(n, dtype=torch.uint8, device="cuda")
+    d_stats = torch.empty(ctx.n_dies * 6, dtype=torch.int64, device="cuda")
+    ws = torch.empty(ctx.workspace_bytes_paged(n, parts), dtype=torch.uint8, device="cuda")
+    ext = fp["ext_power_w"]
+    stream = torch.cuda.current_stream()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def step():
+        rc = ctx.submit_batch_paged(d_acc, n, parts, d_comp, d_stall, d_status, d_stats, ws)
+        assert rc == 0, rc
+        ctx.thermal_step(1_000_000, ext, None, want_hot=False)
+
+    def timed(k):
+        total = 0.0
+        for _ in range(k):
+            ctx.reset()
+            e0.record(stream); step(); e1.record(stream)
+            e1.synchronize()
+            total += e0.elapsed_time(e1)
+        return total
+    timed(args.warmup)
+    res = ctx.last_result()
+    assert res["code"] == 0, res
+    l0 = hbf.kernel_launches()
+    ms = timed(args.steps)
+    launches = hbf.kernel_launches() - l0
+    peak, kind = measured_peak()
+    rate = n * args.steps / (ms * 1e-3)
+    # what the split path must move: the records in, the part records out and in again, their results out and in, the results out
+    moved = 24 * n + 2 * 24 * parts + 2 * 17 * parts + 17 * n
+    line = {"metric": METRIC, "value": rate, "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64",
+            "data": "synthetic",
+            "config": {"workload": "capacity_mode_paged", "accesses_per_step": n, "parts_per_step": parts, "geometry": "64x8x4",
+                       "queues": 2048, "thermal_grid": "128x128",
+                       "gen_seconds": round(gen_s, 1), "state": "queues idle at the start of every step"},
+            "gpu_launches": int(launches),
+            "roofline": {"bound": "hbm", "kernel": "paged submit, all kernels", "achieved": moved * args.steps / (ms * 1e-3) / 1e9,
+                         "peak": peak, "peak_kind": kind, "unit": "GB/s",
+                         "frac": moved * args.steps / (ms * 1e-3) / 1e9 / peak, "traffic": None,
+                         "algorithmic_bytes_per_access": moved / n},
+            "batch_result": {k: res[k] for k in ("n_modeled", "n_native", "max_completion_ns")}}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     args = parse_args()
     rank = int(os.environ.get("RANK", "0"))
@@ -235,6 +297,10 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     if args.impl == "reference":
         run_reference(args, rank)
+        return
+    if args.workload == "capacity_paged":
+        if rank == 0:
+            run_paged(args)
         return
     if args.workload == "coupled_thermal":
         if rank == 0:

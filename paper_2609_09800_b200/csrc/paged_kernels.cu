@@ -78,21 +78,25 @@ k_paged_tile_scan(unsigned long long *tile_sum, uint64_t n_tiles, unsigned long 
     if (tid == 0) *total = s_carry;
 }
 
-// Thread t of a tile takes kPgItems consecutive accesses, so that the parts leave in (access, part) order.
+// A tile first lays out where the parts of each of its accesses go (thread t takes kPgItems consecutive accesses,
+// block scan of the counts); then the threads walk the tile's OUTPUT slots, consecutive threads writing
+// consecutive part records: each finds its access by binary search in the tile's offsets and cuts its part out.
 __global__ void __launch_bounds__(kPgThreads)
 k_paged_expand(const hbf_access_t *__restrict__ acc, uint64_t n, const RangeSnap *__restrict__ ranges, const ModelParams *__restrict__ mp,
                const unsigned long long *__restrict__ tile_off, uint64_t capacity, hbf_access_t *__restrict__ parts,
                uint32_t *__restrict__ part_first) {
     __shared__ unsigned long long s_warp[kPgThreads / 32];
+    __shared__ uint32_t s_first[kPgTile + 1];               // first part of every access of the tile, relative to the tile's first
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint64_t first = (uint64_t)blockIdx.x * kPgTile + (uint64_t)tid * kPgItems;
+    const uint64_t tile_base = (uint64_t)blockIdx.x * kPgTile;
+    const uint32_t in_tile = (uint32_t)min((uint64_t)kPgTile, n - tile_base);
+    const uint64_t first = tile_base + (uint64_t)tid * kPgItems;
     uint32_t cnt[kPgItems];
-    uint64_t fb[kPgItems];
     unsigned long long mine = 0;
 #pragma unroll
     for (int j = 0; j < kPgItems; ++j) {
-        cnt[j] = 0; fb[j] = 0;
-        if (first + j < n) cnt[j] = parts_of(*ranges, *mp, reinterpret_cast<const uint64_t *>(acc + first + j), &fb[j]);
+        uint64_t fb;
+        cnt[j] = first + j < n ? parts_of(*ranges, *mp, reinterpret_cast<const uint64_t *>(acc + first + j), &fb) : 0u;
         mine += cnt[j];
     }
     unsigned long long incl = mine;
@@ -100,26 +104,41 @@ k_paged_expand(const hbf_access_t *__restrict__ acc, uint64_t n, const RangeSnap
     for (int o = 1; o < 32; o <<= 1) { const unsigned long long t = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += t; }
     if (lane == 31) s_warp[warp] = incl;
     __syncthreads();
-    unsigned long long at = tile_off[blockIdx.x] + incl - mine;
-    for (int w = 0; w < warp; ++w) at += s_warp[w];
-    const uint64_t page = 1ull << mp->page_shift;
+    unsigned long long local = incl - mine;
+    for (int w = 0; w < warp; ++w) local += s_warp[w];
+    const unsigned long long off0 = tile_off[blockIdx.x];
 #pragma unroll
     for (int j = 0; j < kPgItems; ++j) {
-        if (first + j >= n) break;
-        part_first[first + j] = (uint32_t)at;
-        hbf_access_t r = acc[first + j];
-        uint64_t left = r.bytes, take = fb[j];
-        for (uint32_t k = 0; k < cnt[j]; ++k) {
-            if (at < capacity) {                             // the host checked the total against the capacity before this launch
-                hbf_access_t p; p.addr = r.addr; p.issue_ns = r.issue_ns; p.bytes = (uint32_t)take; p.flags = r.flags;
-                parts[at] = p;
-            }
-            ++at;
-            r.addr += take; left -= take;
-            take = min(left, page);
+        if (first + j < n) {
+            s_first[tid * kPgItems + j] = (uint32_t)local;
+            part_first[first + j] = (uint32_t)(off0 + local);
+            local += cnt[j];
         }
     }
-    if (first <= n - 1 && n - 1 < first + kPgItems) part_first[n] = (uint32_t)at;   // the thread that holds the last access
+    unsigned long long tile_total = 0;
+    for (int w = 0; w < kPgThreads / 32; ++w) tile_total += s_warp[w];
+    if (tid == 0) {
+        s_first[in_tile] = (uint32_t)tile_total;
+        if (tile_base + in_tile == n) part_first[n] = (uint32_t)(off0 + tile_total);     // the tile that holds the last access
+    }
+    __syncthreads();
+    const uint64_t page = 1ull << mp->page_shift;
+    for (unsigned long long k = (unsigned long long)tid; k < tile_total; k += kPgThreads) {
+        uint32_t lo = 0, hi = in_tile;                       // last access e with s_first[e] <= k
+        while (hi - lo > 1u) { const uint32_t mid = (lo + hi) >> 1; if ((unsigned long long)s_first[mid] <= k) lo = mid; else hi = mid; }
+        const uint32_t e = lo, part = (uint32_t)(k - s_first[e]), of = s_first[e + 1] - s_first[e];
+        hbf_access_t r = acc[tile_base + e];
+        if (of > 1u) {                                       // a modeled access of several pages
+            int g = 0;
+            classify(*ranges, r.addr, r.issue_ns, r.bytes, r.flags, &g);
+            const uint64_t off = ranges->media_offset[g] + (r.addr - ranges->base[g]);
+            const uint64_t head = page - (off & (page - 1ull));          // bytes in its first page
+            const uint64_t skip = part == 0u ? 0ull : head + (uint64_t)(part - 1u) * page;
+            const uint64_t len = part == 0u ? head : min((uint64_t)r.bytes - skip, page);
+            r.addr += skip; r.bytes = (uint32_t)len;
+        }
+        if (off0 + k < capacity) parts[off0 + k] = r;       // the host checked the total against the capacity before this launch
+    }
 }
 
 struct PagedSums { unsigned long long n_ready, stall_sum; };
