@@ -24,6 +24,9 @@ struct hbfo_ctx {
     int32_t mode; int64_t q_ppm;
     hbfo_batch_result_t last;
     uint32_t *order; uint64_t order_count, order_cap;
+    /* time-bin energy ledger (off while bin_ns == 0) */
+    int64_t bin_ns; uint32_t n_bins; int64_t cur_bin;
+    int64_t *ledger;           /* [n_bins][n_dies], row = bin index modulo n_bins */
     /* thermal */
     int thermal;
     double *C, *Gx, *Gy, *Gs, *T, *Tn, *P;
@@ -71,7 +74,7 @@ const char *hbfo_strerror(int code) {
 
 static void free_ctx(hbfo_ctx *c) {
     if (!c) return;
-    free(c->busy_until); free(c->pending_pj); free(c->order);
+    free(c->busy_until); free(c->pending_pj); free(c->order); free(c->ledger);
     free(c->C); free(c->Gx); free(c->Gy); free(c->Gs); free(c->T); free(c->Tn); free(c->P);
     free(c->cell_region); free(c->die_region); free(c->region_kind);
     free(c->region_idle_w); free(c->region_cells);
@@ -165,6 +168,8 @@ int hbfo_reset(hbfo_ctx *c) {
     c->mode = HBFO_MODE_NORMAL; c->q_ppm = 1000000;
     memset(&c->last, 0, sizeof(c->last));
     c->order_count = 0;
+    c->cur_bin = 0;
+    if (c->ledger) memset(c->ledger, 0, (size_t)c->n_bins * c->n_dies * sizeof(int64_t));
     if (c->thermal) for (size_t i = 0; i < c->n_cells; ++i) c->T[i] = (double)c->cfg.ambient_c;
     return HBFO_OK;
 }
@@ -264,6 +269,52 @@ int hbfo_service_terms(hbfo_ctx *c, uint32_t bytes, uint64_t npages, uint32_t op
     if (s_ns) *s_ns = s;
     if (energy_pj) *energy_pj = e;
     return HBFO_OK;
+}
+
+/* ---- time-bin power integration (Section "Design", the paragraph on the event-based energy model) -------
+ * Event energies accumulate in bins of bin_ns; an event that spans more than one bin has its energy split
+ * across the bins in proportion to the time overlap.  The event of an access is its array service interval
+ * [start, start + s) on its die.  Shares are whole pJ: floor(E * overlap / s) for every bin but the event's
+ * last, which takes what is left, so a die's bins always add up to its events' energy.  The ledger is a ring
+ * of n_bins bins starting at the bin the thermal clock stands in: time before it counts into that bin, time
+ * past the ring's end into the ring's last bin. */
+int hbfo_enable_energy_bins(hbfo_ctx *c, int64_t bin_ns, uint32_t n_bins) {
+    if (!c || bin_ns <= 0 || n_bins == 0) return HBFO_E_INVAL;
+    int64_t *l = (int64_t *)calloc((size_t)n_bins * c->n_dies, sizeof(int64_t));
+    if (!l) return HBFO_E_NOMEM;
+    free(c->ledger);
+    c->ledger = l; c->bin_ns = bin_ns; c->n_bins = n_bins; c->cur_bin = 0;
+    memset(c->pending_pj, 0, c->n_dies * sizeof(int64_t));
+    return HBFO_OK;
+}
+
+int hbfo_get_energy_bins(hbfo_ctx *c, int64_t *out, uint64_t cap, int64_t *first_bin) {
+    if (!c || !c->ledger || !out || cap < (uint64_t)c->n_bins * c->n_dies) return HBFO_E_INVAL;
+    for (uint32_t k = 0; k < c->n_bins; ++k) {              /* row k of the output is bin cur_bin + k */
+        int64_t b = c->cur_bin + k;
+        memcpy(out + (size_t)k * c->n_dies, c->ledger + (size_t)(b % c->n_bins) * c->n_dies, c->n_dies * sizeof(int64_t));
+    }
+    if (first_bin) *first_bin = c->cur_bin;
+    return HBFO_OK;
+}
+
+static void ledger_add(hbfo_ctx *c, uint32_t die, int64_t bin, int64_t pj) {
+    if (bin < c->cur_bin) bin = c->cur_bin;
+    if (bin > c->cur_bin + (int64_t)c->n_bins - 1) bin = c->cur_bin + (int64_t)c->n_bins - 1;
+    c->ledger[(size_t)(bin % c->n_bins) * c->n_dies + die] += pj;
+}
+
+static void ledger_event(hbfo_ctx *c, uint32_t die, int64_t start, int64_t s, int64_t energy_pj) {
+    const int64_t end = start + s, w = c->bin_ns;             /* s >= 1 */
+    const int64_t b0 = start / w, b1 = (end - 1) / w;
+    int64_t given = 0;
+    for (int64_t b = b0; b < b1; ++b) {
+        int64_t lo = b * w > start ? b * w : start, hi = (b + 1) * w;
+        int64_t share = (int64_t)(((__int128)energy_pj * (hi - lo)) / s);
+        ledger_add(c, die, b, share);
+        given += share;
+    }
+    ledger_add(c, die, b1, energy_pj - given);
 }
 
 /* ---- submit --------------------------------------------------------------------------------- */
@@ -371,6 +422,7 @@ int hbfo_submit_batch(hbfo_ctx *c, const hbfo_access_t *acc, uint64_t n, int64_t
             stall_ns[i] = done_ns - acc[i].issue_ns;
             hbfo_die_stats_t *d = &ds[die[i]];
             d->busy_ns += s_ns[i]; d->energy_pj += eng[i];
+            if (c->bin_ns) ledger_event(c, die[i], start, s_ns[i], eng[i]);
             if (acc[i].flags & 1u) { d->bytes_prog += cbs[i]; d->n_prog += 1; }
             else                   { d->bytes_read += cbs[i]; d->n_read += 1; }
             res.modeled_ns += stall_ns[i]; res.service_ns += s_ns[i];
@@ -380,7 +432,7 @@ int hbfo_submit_batch(hbfo_ctx *c, const hbfo_access_t *acc, uint64_t n, int64_t
         c->busy_until[r] = B;
     }
     c->order_count = n_ready;
-    for (uint32_t d = 0; d < c->n_dies; ++d) c->pending_pj[d] += ds[d].energy_pj;
+    if (!c->bin_ns) for (uint32_t d = 0; d < c->n_dies; ++d) c->pending_pj[d] += ds[d].energy_pj;
     if (die_stats) memcpy(die_stats, ds, c->n_dies * sizeof(hbfo_die_stats_t));
     free(ds);
     res.code = HBFO_OK; res.n_native = n_native; res.n_modeled = n_ready;
@@ -607,6 +659,12 @@ int hbfo_thermal_step(hbfo_ctx *c, int64_t dt_ns, const float *ext_power_w, uint
     if (dt_sub > c->euler_limit_s) return HBFO_E_INVAL;                    /* explicit step would be unstable */
     const double amb = (double)c->cfg.ambient_c;
 
+    if (c->bin_ns) {                                          /* the step is the bin the thermal clock stands in */
+        if (dt_ns != c->bin_ns) return HBFO_E_INVAL;
+        int64_t *row = c->ledger + (size_t)(c->cur_bin % c->n_bins) * c->n_dies;
+        for (uint32_t d = 0; d < c->n_dies; ++d) { c->pending_pj[d] += row[d]; row[d] = 0; }
+        c->cur_bin += 1;
+    }
     /* power map: energy of the window / window length + idle + external, spread over the region */
     double *Pr = (double *)calloc(NR, sizeof(double));
     if (!Pr) return HBFO_E_NOMEM;

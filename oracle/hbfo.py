@@ -89,6 +89,8 @@ def lib():
                                         C.c_void_p, C.c_void_p]
         L.hbfo_submit_batch_paged.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p, C.c_void_p,
                                         C.c_void_p, C.c_void_p]
+        L.hbfo_enable_energy_bins.argtypes = [C.c_void_p, C.c_int64, C.c_uint32]
+        L.hbfo_get_energy_bins.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.POINTER(C.c_int64)]
         L.hbfo_last_result.argtypes = [C.c_void_p, C.POINTER(BatchResult)]
         L.hbfo_last_order.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.POINTER(C.c_uint64)]
         L.hbfo_thermal_step.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p]
@@ -185,6 +187,21 @@ class Oracle:
         if check and rc != 0:
             raise OracleError(rc)
         return rc, comp, stall, status, ds
+
+    def enable_energy_bins(self, bin_ns: int, n_bins: int):
+        rc = lib().hbfo_enable_energy_bins(self._h, bin_ns, n_bins)
+        if rc != 0:
+            raise OracleError(rc)
+        self._n_bins = n_bins
+
+    def energy_bins(self):
+        """(first_bin, array [n_bins][n_dies] of pJ): row k is bin first_bin + k."""
+        out = np.zeros((self._n_bins, self.n_dies), np.int64)
+        first = C.c_int64()
+        rc = lib().hbfo_get_energy_bins(self._h, out.ctypes.data, out.size, C.byref(first))
+        if rc != 0:
+            raise OracleError(rc)
+        return first.value, out
 
     def last_result(self) -> dict:
         r = BatchResult()
