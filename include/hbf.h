@@ -145,6 +145,21 @@ HBF_API int hbf_submit_batch_paged(hbf_ctx *ctx, const hbf_access_t *d_acc, uint
                            int64_t *d_completion_ns, int64_t *d_stall_ns, uint8_t *d_status,
                            hbf_die_stats_t *d_die_stats, void *d_workspace, size_t workspace_bytes);
 
+/* Time-bin power integration (Section "Design", the event-based energy model: event energies accumulate in
+ * bins; an event that spans more than one bin has its energy split across the bins in proportion to the time
+ * overlap; P = E / dt + P_idle).  After hbf_enable_energy_bins, hbf_submit_batch books the energy of every
+ * modeled access into the bins its array service interval [start, start + s) overlaps, instead of adding the
+ * batch's energy to the pending totals: whole pJ, floor(E * overlap / s) per bin, the event's last bin takes
+ * what is left.  The ledger is a ring of n_bins bins of bin_ns each, starting at the bin the thermal clock
+ * stands in (bin 0 after enable or hbf_reset); time before that bin is booked into it, time past the ring's
+ * end into its last bin.  hbf_thermal_step must then be called with dt_ns == bin_ns (HBF_E_INVAL otherwise):
+ * it consumes the clock's bin and advances the clock by one.  hbf_get_energy_bins synchronises and copies the
+ * ring to host_out [n_bins][channels*dies] (row k = bin *first_bin + k).  The ledger is library-owned device
+ * memory allocated by hbf_enable_energy_bins; it is not part of the hbf_get_state blob.
+ * hbf_submit_batch_paged is refused (HBF_E_INVAL) while the ledger is on. */
+HBF_API int hbf_enable_energy_bins(hbf_ctx *ctx, int64_t bin_ns, uint32_t n_bins);
+HBF_API int hbf_get_energy_bins(hbf_ctx *ctx, int64_t *host_out, uint64_t cap, int64_t *first_bin);
+
 /* Waits for the last submitted batch and copies its summary to host_out; returns its code. */
 HBF_API int hbf_last_result(hbf_ctx *ctx, hbf_batch_result_t *host_out);
 

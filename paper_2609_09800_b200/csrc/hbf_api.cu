@@ -36,6 +36,8 @@ struct hbf_ctx {
     BatchCtrl *d_ctrl = nullptr; hbf_batch_result_t *d_result = nullptr;
     int64_t *d_busy = nullptr, *d_busy_stage = nullptr, *d_pending = nullptr; hbf_die_stats_t *d_stats_stage = nullptr;
     hbf_batch_result_t *h_result = nullptr;      // pinned
+    // time-bin energy ledger (off while bin_ns == 0)
+    int64_t bin_ns = 0, cur_bin = 0; uint32_t n_bins = 0; unsigned long long *d_ledger = nullptr;
     float *h_hot = nullptr;                      // pinned [3]
     float *h_ext = nullptr;                      // pinned [n_regions]
     bool submitted = false;
@@ -111,6 +113,7 @@ int hbf_destroy(hbf_ctx *c) {
     for (void *p : c->owned) cudaFree(p);
     if (c->ev_made) { for (auto &e : c->ev) cudaEventDestroy(e); for (auto &e : c->ev_th) cudaEventDestroy(e); }
     if (c->h_result) cudaFreeHost(c->h_result);
+    if (c->d_ledger) cudaFree(c->d_ledger);
     if (c->h_hot) cudaFreeHost(c->h_hot);
     if (c->h_ext) cudaFreeHost(c->h_ext);
     delete c;
@@ -318,7 +321,11 @@ int hbf_submit_batch(hbf_ctx *c, const hbf_access_t *d_acc, uint64_t n, int64_t 
     c->prof_inorder = c->profiling && n > 0 && c->inorder_ok && (c->path == HBF_PATH_AUTO || c->path == HBF_PATH_INORDER);
     a.ev = c->profiling ? c->ev : nullptr;
     c->prof_submit = c->profiling;
+    a.binned = c->bin_ns != 0;
     CK(launch_submit(a, c->stream));
+    if (a.binned)
+        CK(launch_energy_bins(d_acc, n, d_completion_ns, c->d_ranges, c->d_mp, c->d_ctrl, c->d_result, c->d_ledger, c->bin_ns,
+                              c->n_bins, c->cur_bin, c->sm_count, c->stream));
     c->submitted = true;
     return HBF_OK;
 }
@@ -335,7 +342,7 @@ int hbf_submit_batch_paged(hbf_ctx *c, const hbf_access_t *d_acc, uint64_t n, ui
     if (n == 0)                                             // nothing to split: the ordinary path reports the empty batch
         return hbf_submit_batch(c, d_acc, 0, d_completion_ns, d_stall_ns, d_status, d_die_stats, d_workspace, workspace_bytes);
     if (c->terminal) return HBF_E_LINK_SHUTDOWN;
-    if (n > HBF_MAX_BATCH) return HBF_E_INVAL;
+    if (n > HBF_MAX_BATCH || c->bin_ns != 0) return HBF_E_INVAL;          // the time-bin ledger books whole accesses only
     if (!d_acc || !d_completion_ns || !d_stall_ns) return HBF_E_INVAL;
     if ((reinterpret_cast<uintptr_t>(d_acc) & 7u) || (reinterpret_cast<uintptr_t>(d_completion_ns) & 7u) ||
         (reinterpret_cast<uintptr_t>(d_stall_ns) & 7u) || (reinterpret_cast<uintptr_t>(d_die_stats) & 7u)) return HBF_E_INVAL;
@@ -370,6 +377,30 @@ int hbf_submit_batch_paged(hbf_ctx *c, const hbf_access_t *d_acc, uint64_t n, ui
     return HBF_OK;
 }
 
+int hbf_enable_energy_bins(hbf_ctx *c, int64_t bin_ns, uint32_t n_bins) {
+    if (!c || bin_ns <= 0 || n_bins == 0) return HBF_E_INVAL;
+    CK(cudaStreamSynchronize(c->stream));
+    unsigned long long *l = nullptr;
+    if (cudaMalloc(&l, (size_t)n_bins * c->mp.n_dies * 8) != cudaSuccess) return HBF_E_NOMEM;
+    if (c->d_ledger) cudaFree(c->d_ledger);
+    c->d_ledger = l; c->bin_ns = bin_ns; c->n_bins = n_bins; c->cur_bin = 0;
+    CK(cudaMemsetAsync(c->d_ledger, 0, (size_t)n_bins * c->mp.n_dies * 8, c->stream));
+    CK(cudaMemsetAsync(c->d_pending, 0, c->mp.n_dies * sizeof(int64_t), c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    return HBF_OK;
+}
+
+int hbf_get_energy_bins(hbf_ctx *c, int64_t *host_out, uint64_t cap, int64_t *first_bin) {
+    if (!c || !c->d_ledger || !host_out || cap < (uint64_t)c->n_bins * c->mp.n_dies) return HBF_E_INVAL;
+    const size_t row = (size_t)c->mp.n_dies * 8;
+    for (uint32_t k = 0; k < c->n_bins; ++k)                // row k of the output is bin cur_bin + k
+        CK(cudaMemcpyAsync(host_out + (size_t)k * c->mp.n_dies, c->d_ledger + (size_t)((c->cur_bin + k) % c->n_bins) * c->mp.n_dies,
+                           row, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    if (first_bin) *first_bin = c->cur_bin;
+    return HBF_OK;
+}
+
 int hbf_last_result(hbf_ctx *c, hbf_batch_result_t *host_out) {
     if (!c || !host_out) return HBF_E_INVAL;
     if (!c->submitted) { memset(host_out, 0, sizeof(*host_out)); return HBF_OK; }
@@ -400,6 +431,11 @@ int hbf_thermal_step(hbf_ctx *c, int64_t dt_ns, const float *ext_power_w, uint32
     if (dt_sub > c->euler_limit_s) return HBF_E_INVAL;
     if (n_ext)      // pageable source: the runtime stages the bytes before returning, so the caller's array is free at once
         CK(cudaMemcpyAsync(c->td.ext_power, ext_power_w, n_ext * sizeof(float), cudaMemcpyHostToDevice, c->stream));
+    if (c->bin_ns) {                                         // the step is the bin the thermal clock stands in
+        if (dt_ns != c->bin_ns) return HBF_E_INVAL;
+        CK(launch_take_bin(c->d_ledger + (size_t)(c->cur_bin % c->n_bins) * c->mp.n_dies, c->d_pending, c->mp.n_dies, c->stream));
+        c->cur_bin += 1;
+    }
     if (c->profiling) CK(cudaEventRecord(c->ev_th[0], c->stream));
     CK(launch_thermal_step(c->td, c->d_state, c->d_pending, dt_ns, n_ext != 0, d_temps_out, &c->cur, c->thermal_generic ? 1 : 0, c->stream));
     if (c->profiling) { CK(cudaEventRecord(c->ev_th[1], c->stream)); c->prof_thermal = true; }
@@ -441,6 +477,7 @@ int hbf_reset(hbf_ctx *c) {
     CK(cudaMemsetAsync(c->d_busy, 0, c->mp.n_queues * sizeof(int64_t), c->stream));
     CK(cudaMemsetAsync(c->d_pending, 0, c->mp.n_dies * sizeof(int64_t), c->stream));
     CK(cudaMemsetAsync(c->d_result, 0, sizeof(hbf_batch_result_t), c->stream));
+    if (c->bin_ns) { CK(cudaMemsetAsync(c->d_ledger, 0, (size_t)c->n_bins * c->mp.n_dies * 8, c->stream)); c->cur_bin = 0; }
     if (c->thermal) {
         const size_t nc = (size_t)c->td.H * c->td.W;
         CK(cudaMemsetAsync(c->td.theta[0], 0, nc * sizeof(float), c->stream));

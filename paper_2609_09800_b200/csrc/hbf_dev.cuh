@@ -104,6 +104,7 @@ struct SubmitArgs {
     int64_t *busy, *busy_stage, *pending; hbf_die_stats_t *stats_stage;
     Workspace ws; int32_t path; int sm_count; int inorder_ok;
     FastRange fast;
+    int binned;                          // the batch's energy goes to the time-bin ledger, not to the pending totals
     cudaEvent_t *ev;                     // [kProfEvents] or null: recorded between kernel groups
 };
 constexpr int kProfEvents = 10;
@@ -144,6 +145,13 @@ cudaError_t launch_paged_expand(const hbf_access_t *acc, uint64_t n, const Range
                                 uint64_t capacity, const PagedWorkspace &pw, cudaStream_t st);
 cudaError_t launch_paged_join(const hbf_access_t *acc, uint64_t n, const PagedWorkspace &pw, hbf_batch_result_t *result,
                               int64_t *completion, int64_t *stall, uint8_t *status, int sm_count, cudaStream_t st);
+
+// ---- time-bin energy ledger ----------------------------------------------------------------------------
+cudaError_t launch_energy_bins(const hbf_access_t *acc, uint64_t n, const int64_t *completion, const RangeSnap *ranges,
+                               const ModelParams *mp_dev, const BatchCtrl *ctrl, const hbf_batch_result_t *result,
+                               unsigned long long *ledger, int64_t bin_ns, uint32_t n_bins, int64_t cur_bin, int sm_count,
+                               cudaStream_t st);
+cudaError_t launch_take_bin(unsigned long long *row, int64_t *pending, uint32_t n_dies, cudaStream_t st);
 
 // ---- thermal -------------------------------------------------------------------------------------
 struct ThermalDev {

@@ -600,7 +600,7 @@ k_scan(const hbf_access_t *__restrict__ acc, uint64_t n, const RangeSnap *__rest
 __global__ void k_finish(uint64_t n, BatchCtrl *ctrl, DevState *state, int64_t *busy, const int64_t *busy_stage,
                          int64_t *pending, const hbf_die_stats_t *stats_stage, hbf_die_stats_t *die_stats,
                          int64_t *completion, int64_t *stall, hbf_batch_result_t *result,
-                         const ModelParams *__restrict__ mp, uint32_t n_queues, uint32_t n_dies) {
+                         const ModelParams *__restrict__ mp, uint32_t n_queues, uint32_t n_dies, int binned) {
     const int code = ctrl->code;
     const uint64_t gtid = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (code == HBF_E_TIMEOUT && gtid == 0) state->poisoned = 1;         // a bounded device-side wait expired
@@ -616,7 +616,7 @@ __global__ void k_finish(uint64_t n, BatchCtrl *ctrl, DevState *state, int64_t *
             // the in-order path keeps byte and access counts only: the energy is linear in them
             if (inorder) ds.energy_pj = mp->e_cmd_read_pj * ds.n_read + mp->e_byte_read_pj * ds.bytes_read +
                                         mp->e_cmd_prog_pj * ds.n_prog + mp->e_byte_prog_pj * ds.bytes_prog;
-            pending[d] += ds.energy_pj;
+            if (!binned) pending[d] += ds.energy_pj;          // with the time-bin ledger on, the energy is booked per event
             if (die_stats) die_stats[d] = ds;
         }
     }
@@ -743,7 +743,7 @@ cudaError_t launch_submit(const SubmitArgs &a, cudaStream_t st) {
     mark(5);
     const unsigned fin_grid = (unsigned)std::max<uint64_t>(1, std::min<uint64_t>((n + 1023) / 1024, (uint64_t)a.sm_count * 4));
     k_finish<<<fin_grid, 256, 0, st>>>(n, a.ctrl, a.state, a.busy, a.busy_stage, a.pending, a.stats_stage, a.die_stats,
-                                       a.completion, a.stall, a.result, a.mp_dev, a.mp.n_queues, a.mp.n_dies);
+                                       a.completion, a.stall, a.result, a.mp_dev, a.mp.n_queues, a.mp.n_dies, a.binned);
     g_kernel_launches += 1;
     mark(6);
     return cudaGetLastError();

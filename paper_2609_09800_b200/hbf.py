@@ -29,7 +29,8 @@ EXPORTS = ("hbf_create", "hbf_destroy", "hbf_register_range", "hbf_clear_ranges"
            "hbf_reset", "hbf_set_path", "hbf_get_state", "hbf_set_state", "hbf_get_busy_until",
            "hbf_get_pending_energy", "hbf_get_temps", "hbf_euler_limit_ns", "hbf_queue_order", "hbf_strerror",
            "hbf_set_profiling", "hbf_get_profile", "hbf_kernel_launches", "hbf_euler_substeps_static", "hbf_set_thermal_path",
-           "hbf_workspace_bytes_paged", "hbf_submit_batch_paged")
+           "hbf_workspace_bytes_paged", "hbf_submit_batch_paged",
+           "hbf_enable_energy_bins", "hbf_get_energy_bins")
 STATIC_MAX_CELLS = 65536
 PROF_STAGES = ("begin", "classify", "plan_hist", "sort", "scan", "finish", "inorder", "thermal")
 
@@ -89,6 +90,8 @@ def lib():
         L.hbf_workspace_bytes_paged.argtypes = [vp, u64, u64]
         L.hbf_workspace_bytes_paged.restype = C.c_size_t
         L.hbf_submit_batch_paged.argtypes = [vp, vp, u64, u64, vp, vp, vp, vp, vp, C.c_size_t]
+        L.hbf_enable_energy_bins.argtypes = [vp, i64, u32]
+        L.hbf_get_energy_bins.argtypes = [vp, vp, u64, C.POINTER(i64)]
         L.hbf_last_result.argtypes = [vp, C.POINTER(hbf_batch_result_t)]
         L.hbf_thermal_step.argtypes = [vp, i64, vp, u32, vp, vp]
         L.hbf_force_mode.argtypes = [vp, i32, i64]
@@ -243,6 +246,21 @@ class Context:
         return lib().hbf_submit_batch_paged(self._h, _ptr(d_acc), n, parts_capacity, _ptr(d_completion), _ptr(d_stall),
                                             _ptr(d_status), _ptr(d_die_stats), _ptr(d_workspace),
                                             d_workspace.numel() * d_workspace.element_size())
+
+    def enable_energy_bins(self, bin_ns: int, n_bins: int):
+        rc = lib().hbf_enable_energy_bins(self._h, bin_ns, n_bins)
+        if rc != 0:
+            raise HbfError(rc, "hbf_enable_energy_bins")
+        self._n_bins = n_bins
+
+    def energy_bins(self):
+        """(first_bin, array [n_bins][n_dies] of pJ): row k is bin first_bin + k."""
+        out = np.zeros((self._n_bins, self.n_dies), np.int64)
+        first = C.c_int64()
+        rc = lib().hbf_get_energy_bins(self._h, out.ctypes.data, out.size, C.byref(first))
+        if rc != 0:
+            raise HbfError(rc, "hbf_get_energy_bins")
+        return first.value, out
 
     def last_result(self) -> dict:
         r = hbf_batch_result_t()

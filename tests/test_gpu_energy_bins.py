@@ -1,0 +1,113 @@
+"""Parity of the time-bin energy ledger (hbf_enable_energy_bins) with the oracle's: bins bit for bit, temperatures
+within 1e-3 K when the thermal steps consume them."""
+import json
+import os
+
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+from oracle import hbfo
+from paper_2609_09800_b200 import workloads as wl
+
+
+@pytest.fixture(scope="module")
+def hbf():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2609_09800_b200 import build, hbf as mod
+    build.build()
+    return mod
+
+
+def contexts(hbf, profile, ranges, fp=None, path=None):
+    g, o = hbf.Context(profile, fp), hbfo.Oracle(profile, fp)
+    for r in ranges:
+        g.register_range(*r)
+        o.register_range(*r)
+    if path is not None:
+        g.set_path(path)
+    return g, o
+
+
+def same_bins(g, o):
+    fg, bg = g.energy_bins()
+    fo, bo = o.energy_bins()
+    assert fg == fo
+    bad = np.argwhere(bg != bo)
+    assert bad.size == 0, "first difference at bin %d die %d: gpu %d oracle %d" % (bad[0][0], bad[0][1], bg[tuple(bad[0])], bo[tuple(bad[0])])
+
+
+def test_hand_examples(hbf, golden_dir):
+    with open(os.path.join(golden_dir, "energy_bin_examples.json")) as f:
+        examples = json.load(f)["examples"]
+    prof = wl.load_profile("nominal", **wl.GEOMETRY["tiny"])
+    for ex in examples:
+        g = hbf.Context(prof)
+        g.register_range(wl.RANGE_BASE, wl.GIB)
+        g.enable_energy_bins(ex["bin_ns"], len(ex["bins"]))
+        acc = np.zeros(len(ex["acc"]), hbfo.ACCESS_DTYPE)
+        for i, (off, issue, nbytes, op) in enumerate(ex["acc"]):
+            acc[i] = (wl.RANGE_BASE + off, issue, nbytes, op)
+        g.submit_host(acc)
+        first, bins = g.energy_bins()
+        assert first == 0 and bins[:, 0].tolist() == ex["bins"], ex["name"]
+        assert not bins[:, 1:].any() and not g.get_pending_energy().any()
+
+
+@pytest.mark.parametrize("path", ["auto", "sort"])
+@pytest.mark.parametrize("bin_ns", [7_000, 1_000_000])
+def test_mixed_stream_in_two_batches(hbf, bin_ns, path):
+    rng = np.random.default_rng(bin_ns)
+    n = 60_000
+    acc = np.zeros(n, hbfo.ACCESS_DTYPE)
+    acc["addr"] = wl.RANGE_BASE + rng.integers(0, 1 << 26, n).astype(np.uint64)
+    acc["issue_ns"] = np.sort(rng.integers(0, 40_000_000, n))
+    acc["bytes"] = rng.choice([1, 64, 4096, 16384, 65536, 300_000], n)
+    acc["flags"] = rng.random(n) < 0.05
+    prof = wl.load_profile("nominal", **wl.GEOMETRY["tiny"])
+    g, o = contexts(hbf, prof, [(wl.RANGE_BASE, wl.GIB, 3, 0, 0, 0)], path=hbf.PATH_AUTO if path == "auto" else hbf.PATH_SORT)
+    n_bins = 500                                              # the stream runs past the ring: its end collects the rest
+    g.enable_energy_bins(bin_ns, n_bins); o.enable_energy_bins(bin_ns, n_bins)
+    for part in (acc[:35_000], acc[35_000:]):
+        rc_o, c_o, s_o, _, ds_o = o.submit(part)
+        rc_g, c_g, s_g, _, ds_g = g.submit_host(part)
+        assert np.array_equal(c_g, c_o) and np.array_equal(ds_g["energy_pj"], ds_o["energy_pj"])
+        same_bins(g, o)
+    _, bins = g.energy_bins()
+    assert bins.sum() > 0 and not g.get_pending_energy().any()
+
+
+def test_refused_batches_book_nothing_and_paged_is_refused(hbf):
+    wf = wl.mixed_status(5000, seed=2, faults=True)
+    g, o = contexts(hbf, wf.profile, wf.ranges)
+    g.enable_energy_bins(100_000, 64); o.enable_energy_bins(100_000, 64)
+    rc, *_ = g.submit_host(wf.acc, check=False)
+    assert rc == hbf.E_ACCESS_FAULT and not g.energy_bins()[1].any()
+    rc, *_ = g.submit_host(wf.acc, check=False, parts_capacity=100_000)
+    assert rc == hbf.E_INVAL
+
+
+def test_thermal_steps_consume_the_bins(hbf):
+    w = wl.prefix_kv(epochs=1, steps=1, batch=4, kv_tokens=256, layers=2)
+    fp = wl.package_floorplan()
+    g, o = contexts(hbf, w.profile, w.ranges, fp)
+    g.enable_energy_bins(1_000_000, 16); o.enable_energy_bins(1_000_000, 16)
+    ext = fp["ext_power_w"]
+    k = 0
+    for _, batch in wl.timed_batches(w, 12_000_000):
+        g.submit_host(batch); o.submit(batch)
+        same_bins(g, o)
+        hot_g = g.thermal_step(1_000_000, ext)
+        hot_o, _ = o.thermal_step(1_000_000, ext)
+        assert np.abs(np.asarray(hot_g, np.float64) - hot_o).max() < 1e-3
+        k += 1
+    assert k >= 10
+    same_bins(g, o)
+    assert np.abs(g.get_temps().astype(np.float64) - o.temps()).max() < 1e-3
+    with pytest.raises(hbf.HbfError):
+        g.thermal_step(2_000_000, ext)                        # in binned mode a step is one bin long
+    g.reset(); o.reset()
+    same_bins(g, o)
