@@ -712,3 +712,69 @@ int hbfo_thermal_step(hbfo_ctx *c, int64_t dt_ns, const float *ext_power_w, uint
     if (hot_c_out) { hot_c_out[0] = hot[0]; hot_c_out[1] = hot[1]; hot_c_out[2] = hot[2]; }
     return HBFO_OK;
 }
+
+/* ---- reduced-order thermal model (Eq. 2): x' = A x + B p + b,  T = C x + D p + d, with x the state BEFORE
+ * the update.  Plain loops in double; matrices row-major. */
+struct hbfo_rom {
+    uint32_t n, m, o;
+    double *A, *B, *b, *C, *D, *d, *x, *xn;
+};
+
+static double *dup_f64(const double *src, size_t n) {
+    double *p = (double *)malloc((n ? n : 1) * sizeof(double));
+    if (p && src) memcpy(p, src, n * sizeof(double));
+    else if (p) memset(p, 0, (n ? n : 1) * sizeof(double));
+    return p;
+}
+
+int hbfo_rom_destroy(hbfo_rom *r) {
+    if (!r) return HBFO_E_INVAL;
+    free(r->A); free(r->B); free(r->b); free(r->C); free(r->D); free(r->d); free(r->x); free(r->xn); free(r);
+    return HBFO_OK;
+}
+
+int hbfo_rom_create(uint32_t n_states, uint32_t n_inputs, uint32_t n_outputs, const double *A, const double *B,
+                    const double *b, const double *C, const double *D, const double *d, hbfo_rom **out) {
+    if (!out || !n_states || !n_inputs || !n_outputs || !A || !B || !C) return HBFO_E_INVAL;
+    hbfo_rom *r = (hbfo_rom *)calloc(1, sizeof(hbfo_rom));
+    if (!r) return HBFO_E_NOMEM;
+    r->n = n_states; r->m = n_inputs; r->o = n_outputs;
+    r->A = dup_f64(A, (size_t)n_states * n_states); r->B = dup_f64(B, (size_t)n_states * n_inputs);
+    r->b = dup_f64(b, n_states); r->C = dup_f64(C, (size_t)n_outputs * n_states);
+    r->D = dup_f64(D, (size_t)n_outputs * n_inputs); r->d = dup_f64(d, n_outputs);
+    r->x = dup_f64(NULL, n_states); r->xn = dup_f64(NULL, n_states);
+    if (!r->A || !r->B || !r->b || !r->C || !r->D || !r->d || !r->x || !r->xn) { hbfo_rom_destroy(r); return HBFO_E_NOMEM; }
+    *out = r;
+    return HBFO_OK;
+}
+
+int hbfo_rom_reset(hbfo_rom *r) { if (!r) return HBFO_E_INVAL; memset(r->x, 0, r->n * sizeof(double)); return HBFO_OK; }
+
+/* n_steps steps: power [n_steps][n_inputs] in, temps_out [n_steps][n_outputs] out */
+int hbfo_rom_step(hbfo_rom *r, const double *power, uint32_t n_steps, double *temps_out) {
+    if (!r || !power || !temps_out) return HBFO_E_INVAL;
+    for (uint32_t k = 0; k < n_steps; ++k) {
+        const double *p = power + (size_t)k * r->m;
+        double *T = temps_out + (size_t)k * r->o;
+        for (uint32_t i = 0; i < r->o; ++i) {
+            double acc = r->d[i];
+            for (uint32_t j = 0; j < r->n; ++j) acc += r->C[(size_t)i * r->n + j] * r->x[j];
+            for (uint32_t j = 0; j < r->m; ++j) acc += r->D[(size_t)i * r->m + j] * p[j];
+            T[i] = acc;
+        }
+        for (uint32_t i = 0; i < r->n; ++i) {
+            double acc = r->b[i];
+            for (uint32_t j = 0; j < r->n; ++j) acc += r->A[(size_t)i * r->n + j] * r->x[j];
+            for (uint32_t j = 0; j < r->m; ++j) acc += r->B[(size_t)i * r->m + j] * p[j];
+            r->xn[i] = acc;
+        }
+        double *t = r->x; r->x = r->xn; r->xn = t;
+    }
+    return HBFO_OK;
+}
+
+int hbfo_rom_get_state(hbfo_rom *r, double *out, uint64_t cap) {
+    if (!r || !out || cap < r->n) return HBFO_E_INVAL;
+    memcpy(out, r->x, r->n * sizeof(double));
+    return HBFO_OK;
+}

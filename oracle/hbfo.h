@@ -113,6 +113,16 @@ int32_t hbfo_next_mode(hbfo_ctx *ctx, int32_t mode, int64_t t_hot_mk);
 int64_t hbfo_quantise_mk(double t_c);
 const char *hbfo_strerror(int code);
 
+/* Reduced-order thermal model (Eq. 2): x' = A x + B p + b, T = C x + D p + d (x before the update).  Matrices
+ * row-major, double, copied at create; b, D, d may be NULL (zero).  The state starts at zero. */
+typedef struct hbfo_rom hbfo_rom;
+int  hbfo_rom_create(uint32_t n_states, uint32_t n_inputs, uint32_t n_outputs, const double *A, const double *B,
+                     const double *b, const double *C, const double *D, const double *d, hbfo_rom **out);
+int  hbfo_rom_destroy(hbfo_rom *rom);
+int  hbfo_rom_reset(hbfo_rom *rom);
+int  hbfo_rom_step(hbfo_rom *rom, const double *power, uint32_t n_steps, double *temps_out);
+int  hbfo_rom_get_state(hbfo_rom *rom, double *out, uint64_t cap);
+
 #ifdef __cplusplus
 }
 #endif

@@ -91,6 +91,11 @@ def lib():
                                         C.c_void_p, C.c_void_p]
         L.hbfo_enable_energy_bins.argtypes = [C.c_void_p, C.c_int64, C.c_uint32]
         L.hbfo_get_energy_bins.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.POINTER(C.c_int64)]
+        L.hbfo_rom_create.argtypes = [C.c_uint32, C.c_uint32, C.c_uint32] + [C.c_void_p] * 6 + [C.POINTER(C.c_void_p)]
+        L.hbfo_rom_destroy.argtypes = [C.c_void_p]
+        L.hbfo_rom_reset.argtypes = [C.c_void_p]
+        L.hbfo_rom_step.argtypes = [C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p]
+        L.hbfo_rom_get_state.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64]
         L.hbfo_last_result.argtypes = [C.c_void_p, C.POINTER(BatchResult)]
         L.hbfo_last_order.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.POINTER(C.c_uint64)]
         L.hbfo_thermal_step.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p]
@@ -298,3 +303,43 @@ class Oracle:
 
 def quantise_mk(t_c: float) -> int:
     return lib().hbfo_quantise_mk(t_c)
+
+
+class Rom:
+    """Reduced-order thermal model (Eq. 2) stepped in double by plain loops."""
+
+    def __init__(self, A, B, C_, D=None, b=None, d=None):
+        A = np.ascontiguousarray(A, np.float64); B = np.ascontiguousarray(B, np.float64); C_ = np.ascontiguousarray(C_, np.float64)
+        self.n, self.m, self.o = A.shape[0], B.shape[1], C_.shape[0]
+        opt = lambda v, shape: None if v is None else np.ascontiguousarray(np.broadcast_to(np.asarray(v, np.float64), shape))
+        D, b, d = opt(D, (self.o, self.m)), opt(b, (self.n,)), opt(d, (self.o,))
+        ptr = lambda v: None if v is None else v.ctypes.data
+        h = C.c_void_p()
+        rc = lib().hbfo_rom_create(self.n, self.m, self.o, ptr(A), ptr(B), ptr(b), ptr(C_), ptr(D), ptr(d), C.byref(h))
+        if rc != 0:
+            raise OracleError(rc)
+        self._h = h
+
+    def __del__(self):
+        try:
+            if getattr(self, "_h", None):
+                lib().hbfo_rom_destroy(self._h); self._h = None
+        except Exception:
+            pass
+
+    def reset(self):
+        lib().hbfo_rom_reset(self._h)
+
+    def step(self, power):
+        """power [n_steps][n_inputs] -> temperatures [n_steps][n_outputs]"""
+        p = np.ascontiguousarray(np.atleast_2d(power), np.float64)
+        out = np.empty((p.shape[0], self.o), np.float64)
+        rc = lib().hbfo_rom_step(self._h, p.ctypes.data, p.shape[0], out.ctypes.data)
+        if rc != 0:
+            raise OracleError(rc)
+        return out
+
+    def state(self):
+        x = np.empty(self.n, np.float64)
+        lib().hbfo_rom_get_state(self._h, x.ctypes.data, self.n)
+        return x
