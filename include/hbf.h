@@ -243,6 +243,22 @@ HBF_API int hbf_euler_substeps_static(const float *d_cell_C, const float *d_cell
                                       float *d_comp, uint32_t grid_h, uint32_t grid_w, uint32_t n_sub,
                                       float dt_sub_s, void *cuda_stream);
 
+/* Reduced-order thermal model at run time (Eq. 2): x[k+1] = A x[k] + B p[k] + b, T[k] = C x[k] + D p[k] + d.
+ * The paper fits such a model offline (ERA on unit-step responses of the package operator) and steps it instead
+ * of the full grid; the fit is not part of this library (the Python package carries one, era.py), the step is.
+ * hbf_rom_create copies the matrices (host, row-major, double; b, D, d may be NULL = zero) to the current device;
+ * the state starts at zero.  2 * n_states + n_inputs doubles must fit in 40 KiB (HBF_E_INVAL otherwise).
+ * hbf_rom_step runs n_steps steps asynchronously on the stream given at create: d_power [n_steps][n_inputs] and
+ * d_temps_out [n_steps][n_outputs] are device arrays of doubles owned by the caller.  The state carries over
+ * between calls; hbf_rom_reset zeroes it; hbf_rom_get_state synchronises and copies it to host_out [n_states]. */
+typedef struct hbf_rom hbf_rom;
+HBF_API int hbf_rom_create(uint32_t n_states, uint32_t n_inputs, uint32_t n_outputs, const double *A, const double *B,
+                   const double *b, const double *C, const double *D, const double *d, void *cuda_stream, hbf_rom **out);
+HBF_API int hbf_rom_destroy(hbf_rom *rom);
+HBF_API int hbf_rom_reset(hbf_rom *rom);
+HBF_API int hbf_rom_step(hbf_rom *rom, const double *d_power, uint32_t n_steps, double *d_temps_out);
+HBF_API int hbf_rom_get_state(hbf_rom *rom, double *host_out, uint64_t cap);
+
 HBF_API const char *hbf_strerror(int code);
 
 #ifdef __cplusplus

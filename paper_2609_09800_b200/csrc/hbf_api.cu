@@ -89,6 +89,64 @@ static int publish_ranges(hbf_ctx *c) {
 
 extern "C" {
 
+// ---- reduced-order thermal model (Eq. 2) ----------------------------------------------------------------------
+struct hbf_rom {
+    uint32_t n = 0, m = 0, o = 0;
+    cudaStream_t stream = nullptr;
+    double *d_all = nullptr;             // A, B, b, C, D, d, x in one allocation
+    double *A = nullptr, *B = nullptr, *b = nullptr, *C = nullptr, *D = nullptr, *d = nullptr, *x = nullptr;
+};
+
+int hbf_rom_create(uint32_t n_states, uint32_t n_inputs, uint32_t n_outputs, const double *A, const double *B, const double *b,
+                   const double *C, const double *D, const double *d, void *cuda_stream, hbf_rom **out) {
+    if (!out || !n_states || !n_inputs || !n_outputs || !A || !B || !C) return HBF_E_INVAL;
+    if ((size_t)(2 * n_states + n_inputs) * sizeof(double) > 40u * 1024u) return HBF_E_INVAL;   // the step keeps x, x' and p in shared memory
+    const size_t n = n_states, m = n_inputs, o = n_outputs;
+    const size_t total = n * n + n * m + n + o * n + o * m + o + n;
+    std::vector<double> h(total, 0.0);
+    double *p = h.data();
+    auto put = [&](const double *src, size_t cnt) { if (src) memcpy(p, src, cnt * sizeof(double)); double *at = p; p += cnt; return at - h.data(); };
+    const size_t oA = put(A, n * n), oB = put(B, n * m), ob = put(b, n), oC = put(C, o * n), oD = put(D, o * m), od = put(d, o), ox = put(nullptr, n);
+    hbf_rom *r = new (std::nothrow) hbf_rom();
+    if (!r) return HBF_E_NOMEM;
+    r->n = n_states; r->m = n_inputs; r->o = n_outputs; r->stream = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMalloc(&r->d_all, total * sizeof(double)) != cudaSuccess) { delete r; return HBF_E_NOMEM; }
+    if (cudaMemcpyAsync(r->d_all, h.data(), total * sizeof(double), cudaMemcpyHostToDevice, r->stream) != cudaSuccess ||
+        cudaStreamSynchronize(r->stream) != cudaSuccess) { cudaFree(r->d_all); delete r; return HBF_E_CUDA; }
+    r->A = r->d_all + oA; r->B = r->d_all + oB; r->b = r->d_all + ob; r->C = r->d_all + oC; r->D = r->d_all + oD; r->d = r->d_all + od;
+    r->x = r->d_all + ox;
+    *out = r;
+    return HBF_OK;
+}
+
+int hbf_rom_destroy(hbf_rom *r) {
+    if (!r) return HBF_E_INVAL;
+    cudaStreamSynchronize(r->stream);
+    cudaFree(r->d_all);
+    delete r;
+    return HBF_OK;
+}
+
+int hbf_rom_reset(hbf_rom *r) {
+    if (!r) return HBF_E_INVAL;
+    CK(cudaMemsetAsync(r->x, 0, r->n * sizeof(double), r->stream));
+    return HBF_OK;
+}
+
+int hbf_rom_step(hbf_rom *r, const double *d_power, uint32_t n_steps, double *d_temps_out) {
+    if (!r || !d_power || !d_temps_out) return HBF_E_INVAL;
+    if (n_steps == 0) return HBF_OK;
+    CK(launch_rom_steps(r->n, r->m, r->o, r->A, r->B, r->b, r->C, r->D, r->d, r->x, d_power, n_steps, d_temps_out, r->stream));
+    return HBF_OK;
+}
+
+int hbf_rom_get_state(hbf_rom *r, double *host_out, uint64_t cap) {
+    if (!r || !host_out || cap < r->n) return HBF_E_INVAL;
+    CK(cudaMemcpyAsync(host_out, r->x, r->n * sizeof(double), cudaMemcpyDeviceToHost, r->stream));
+    CK(cudaStreamSynchronize(r->stream));
+    return HBF_OK;
+}
+
 const char *hbf_strerror(int code) {
     switch (code) {
     case HBF_OK: return "ok";

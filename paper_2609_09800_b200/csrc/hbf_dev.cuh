@@ -153,6 +153,11 @@ cudaError_t launch_energy_bins(const hbf_access_t *acc, uint64_t n, const int64_
                                cudaStream_t st);
 cudaError_t launch_take_bin(unsigned long long *row, int64_t *pending, uint32_t n_dies, cudaStream_t st);
 
+// ---- reduced-order thermal model -------------------------------------------------------------------------
+cudaError_t launch_rom_steps(uint32_t n, uint32_t m, uint32_t o, const double *A, const double *B, const double *b,
+                             const double *C, const double *D, const double *d, double *x, const double *power,
+                             uint32_t n_steps, double *temps_out, cudaStream_t st);
+
 // ---- thermal -------------------------------------------------------------------------------------
 struct ThermalDev {
     uint32_t H, W, n_regions, n_dies, n_sub;

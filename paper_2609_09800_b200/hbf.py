@@ -30,7 +30,8 @@ EXPORTS = ("hbf_create", "hbf_destroy", "hbf_register_range", "hbf_clear_ranges"
            "hbf_get_pending_energy", "hbf_get_temps", "hbf_euler_limit_ns", "hbf_queue_order", "hbf_strerror",
            "hbf_set_profiling", "hbf_get_profile", "hbf_kernel_launches", "hbf_euler_substeps_static", "hbf_set_thermal_path",
            "hbf_workspace_bytes_paged", "hbf_submit_batch_paged",
-           "hbf_enable_energy_bins", "hbf_get_energy_bins")
+           "hbf_enable_energy_bins", "hbf_get_energy_bins",
+           "hbf_rom_create", "hbf_rom_destroy", "hbf_rom_reset", "hbf_rom_step", "hbf_rom_get_state")
 STATIC_MAX_CELLS = 65536
 PROF_STAGES = ("begin", "classify", "plan_hist", "sort", "scan", "finish", "inorder", "thermal")
 
@@ -92,6 +93,11 @@ def lib():
         L.hbf_submit_batch_paged.argtypes = [vp, vp, u64, u64, vp, vp, vp, vp, vp, C.c_size_t]
         L.hbf_enable_energy_bins.argtypes = [vp, i64, u32]
         L.hbf_get_energy_bins.argtypes = [vp, vp, u64, C.POINTER(i64)]
+        L.hbf_rom_create.argtypes = [u32, u32, u32, vp, vp, vp, vp, vp, vp, vp, C.POINTER(vp)]
+        L.hbf_rom_destroy.argtypes = [vp]
+        L.hbf_rom_reset.argtypes = [vp]
+        L.hbf_rom_step.argtypes = [vp, vp, u32, vp]
+        L.hbf_rom_get_state.argtypes = [vp, vp, u64]
         L.hbf_last_result.argtypes = [vp, C.POINTER(hbf_batch_result_t)]
         L.hbf_thermal_step.argtypes = [vp, i64, vp, u32, vp, vp]
         L.hbf_force_mode.argtypes = [vp, i32, i64]
@@ -184,6 +190,8 @@ class Context:
         self.n_dies = cfg.channels * cfg.dies
         self.n_queues = self.n_dies * (cfg.planes if cfg.queue_level == 0 else 1)
         self.n_cells = cfg.grid_h * cfg.grid_w if floorplan is not None else 0
+        self.n_regions = cfg.n_regions if floorplan is not None else 0
+        self.ambient_c = float(cfg.ambient_c)
         self.stream = stream if stream is not None else torch.cuda.current_stream()
         h = C.c_void_p()
         rc = lib().hbf_create(C.byref(cfg), C.c_void_p(self.stream.cuda_stream), C.byref(h))
@@ -394,3 +402,53 @@ class Context:
             status = d_status.cpu().numpy() if want_status else None
             ds = d_ds.cpu().numpy().view(DIE_STATS_DTYPE)
         return res["code"], comp, stall, status, ds
+
+
+class Rom:
+    """Reduced-order thermal model (Eq. 2) on the device: ``hbf_rom_create`` / ``hbf_rom_step``."""
+
+    def __init__(self, A, B, C_, D=None, b=None, d=None, stream=None):
+        import torch
+        self._torch = torch
+        A = np.ascontiguousarray(A, np.float64); B = np.ascontiguousarray(B, np.float64); C_ = np.ascontiguousarray(C_, np.float64)
+        self.n, self.m, self.o = A.shape[0], B.shape[1], C_.shape[0]
+        opt = lambda v, shape: None if v is None else np.ascontiguousarray(np.broadcast_to(np.asarray(v, np.float64), shape))
+        D, b, d = opt(D, (self.o, self.m)), opt(b, (self.n,)), opt(d, (self.o,))
+        ptr = lambda v: None if v is None else v.ctypes.data
+        self.stream = stream if stream is not None else torch.cuda.current_stream()
+        h = C.c_void_p()
+        rc = lib().hbf_rom_create(self.n, self.m, self.o, ptr(A), ptr(B), ptr(b), ptr(C_), ptr(D), ptr(d),
+                                  self.stream.cuda_stream, C.byref(h))
+        if rc != 0:
+            raise HbfError(rc, "hbf_rom_create")
+        self._h = h
+
+    def __del__(self):
+        try:
+            if getattr(self, "_h", None):
+                lib().hbf_rom_destroy(self._h); self._h = None
+        except Exception:
+            pass
+
+    def reset(self):
+        lib().hbf_rom_reset(self._h)
+
+    def step_device(self, d_power, n_steps, d_temps_out):
+        rc = lib().hbf_rom_step(self._h, _ptr(d_power), n_steps, _ptr(d_temps_out))
+        if rc != 0:
+            raise HbfError(rc, "hbf_rom_step")
+
+    def step(self, power):
+        """Host convenience: power [n_steps][n_inputs] -> temperatures [n_steps][n_outputs] (copies in and out)."""
+        torch = self._torch
+        p = np.ascontiguousarray(np.atleast_2d(power), np.float64)
+        with torch.cuda.stream(self.stream):
+            d_p = torch.from_numpy(p).cuda()
+            d_t = torch.empty((p.shape[0], self.o), dtype=torch.float64, device="cuda")
+            self.step_device(d_p, p.shape[0], d_t)
+            return d_t.cpu().numpy()
+
+    def state(self):
+        x = np.empty(self.n, np.float64)
+        lib().hbf_rom_get_state(self._h, x.ctypes.data, self.n)
+        return x
