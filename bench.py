@@ -51,9 +51,10 @@ def parse_args():
     ap.add_argument("--cpu-sample", type=int, default=20_000_000)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--workload", default="capacity_mode", choices=["capacity_mode", "coupled_thermal", "capacity_paged"],
+    ap.add_argument("--workload", default="capacity_mode", choices=["capacity_mode", "coupled_thermal", "capacity_paged", "rom"],
                     help="coupled_thermal: the prefix-KV stream in 1 ms batches, each followed by a thermal step; "
-                         "capacity_paged: the capacity-mode batch through the page-granular submit (neither is the headline)")
+                         "capacity_paged: the capacity-mode batch through the page-granular submit; rom: fit the reduced-order "
+                         "thermal model of the package floorplan and time its step against the full grid (none is the headline)")
     ap.add_argument("--horizon-ms", type=int, default=1000, help="simulated time of the coupled_thermal run")
     ap.add_argument("--energy-bins", action="store_true",
                     help="coupled_thermal: book event energies into 1 ms bins (time-bin power integration) instead of at submit")
@@ -295,6 +296,55 @@ def run_paged(args):
     print(json.dumps(line), flush=True)
 
 
+def run_rom(args):
+    """Fits the 224-state reduced-order thermal model (Eq. 2) of the package floorplan from the CUDA grid's unit-step
+    responses (10 ms steps), compares it with the grid on three input shapes, and times both."""
+    import torch
+    from paper_2609_09800_b200 import build as hbf_build, hbf, era
+    hbf_build.build()
+    fp0 = wl.package_floorplan()
+    fp = dict(fp0); fp["region_idle_w"] = np.zeros_like(fp["region_idle_w"])
+    prof = wl.load_profile("nominal", **wl.GEOMETRY["serving"]); prof["n_sub"] = 160
+    prof.update(rtt_c=500.0, ltt_c=600.0, stt_c=700.0, shutdown_c=800.0)
+    g = hbf.Context(prof, fp)
+    dt = 10_000_000
+    region = np.asarray(fp["cell_region"]); m = len(fp["region_kind"])
+    sel = list(range(m))[::6][:11]
+    probes = [int(np.flatnonzero(region == k)[len(np.flatnonzero(region == k)) // 2]) for k in sel]
+    t0 = time.time(); steps = era.unit_step_responses(g, probes, 420, dt); resp_s = time.time() - t0
+    t0 = time.time(); fit = era.era(era.markov_from_steps(steps), n_states=224, rows=200, cols=200); fit_s = time.time() - t0
+    rom = hbf.Rom(fit["A"], fit["B"], fit["C"], D=fit["D"], d=np.full(len(probes), prof["ambient_c"]))
+    n_run = 400
+    k = np.arange(n_run)[:, None]; amp = np.asarray(fp0["ext_power_w"], np.float64)[None, :] + 0.2
+    shapes = dict(step=np.ones((n_run, 1)) * amp, ramp=(k / n_run) * amp, pulses=((k // 40) % 2) * amp)
+    d_T = torch.empty(g.n_cells, dtype=torch.float32, device="cuda"); pt = torch.as_tensor(probes, device="cuda")
+    errs = {}
+    for name, p in shapes.items():
+        g.reset(); full = np.empty((n_run, len(probes)))
+        for i in range(n_run):
+            g.thermal_step(dt, p[i].astype(np.float32), d_T, want_hot=False); full[i] = d_T[pt].cpu().numpy()
+        rom.reset(); red = rom.step(p.astype(np.float32).astype(np.float64))
+        errs[name] = {"worst_k": float(np.abs(red - full).max()), "swing_k": float(full.max() - prof["ambient_c"])}
+    d_p = torch.from_numpy(shapes["step"]).cuda(); d_o = torch.empty((n_run, len(probes)), dtype=torch.float64, device="cuda")
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    rom.step_device(d_p, n_run, d_o); torch.cuda.synchronize()
+    e0.record(); rom.step_device(d_p, n_run, d_o); e1.record(); torch.cuda.synchronize()
+    rom_us = e0.elapsed_time(e1) * 1e3 / n_run
+    ext = shapes["step"][0].astype(np.float32)
+    g.thermal_step(dt, ext, None, want_hot=False); torch.cuda.synchronize()
+    e0.record()
+    for _ in range(50):
+        g.thermal_step(dt, ext, None, want_hot=False)
+    e1.record(); torch.cuda.synchronize()
+    grid_us = e0.elapsed_time(e1) * 1e3 / 50
+    print(json.dumps({"metric": "thermal steps/s (reduced-order model, 10 ms steps)", "value": 1e6 / rom_us, "unit": "steps/s",
+                      "n_gpus": 1, "steps": n_run, "warmup": n_run, "ms_per_step": rom_us * 1e-3, "higher_is_better": True,
+                      "dtype": "f64", "data": "synthetic",
+                      "config": {"workload": "rom", "states": 224, "inputs": m, "outputs": len(probes), "grid": "128x128",
+                                 "unit_step_samples": 420, "responses_seconds": round(resp_s, 1), "fit_seconds": round(fit_s, 1)},
+                      "full_grid_us_per_step": grid_us, "rom_us_per_step": rom_us, "model_vs_grid": errs}), flush=True)
+
+
 def main():
     args = parse_args()
     rank = int(os.environ.get("RANK", "0"))
@@ -306,6 +356,10 @@ def main():
     if args.workload == "capacity_paged":
         if rank == 0:
             run_paged(args)
+        return
+    if args.workload == "rom":
+        if rank == 0:
+            run_rom(args)
         return
     if args.workload == "coupled_thermal":
         if rank == 0:
