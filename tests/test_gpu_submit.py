@@ -298,3 +298,35 @@ def test_inorder_long_busy_periods(hbf, rho):
     w = wl.capacity_mode(n=1_500_000, seed=5, rho=rho)
     g, o = contexts(hbf, w.profile, w.ranges, hbf.PATH_INORDER)
     compare_batch(g, o, w.acc)
+
+
+def test_pinned_host_pipeline_equals_one_batch(hbf):
+    """Copy-in, service and read-back of consecutive chunks on three streams: for records in issue order the
+    result is that of one batch."""
+    import torch
+    w = wl.capacity_mode(n=230_000, seed=4)
+    g, o = contexts(hbf, w.profile, w.ranges)
+    _, c_o, s_o, _, ds_o = o.submit(w.acc)
+    n = w.n
+    h_in = torch.from_numpy(w.acc.view(np.int64).reshape(-1)).pin_memory()
+    h_c, h_s = torch.empty(n, dtype=torch.int64).pin_memory(), torch.empty(n, dtype=torch.int64).pin_memory()
+    h_ds = torch.empty(g.n_dies * 6, dtype=torch.int64).pin_memory()
+    for chunk in (50_000, 230_000, 7):
+        if chunk == 7:
+            n_use = 100                                      # many tiny chunks
+        else:
+            n_use = n
+        g.reset()
+        assert g.submit_pinned(h_in, n_use, h_c, h_s, h_ds, chunk=chunk) == 0
+        torch.cuda.synchronize()
+        assert g.last_result()["code"] == 0
+        if n_use == n:
+            assert np.array_equal(h_c.numpy(), c_o) and np.array_equal(h_s.numpy(), s_o)
+            assert np.array_equal(h_ds.numpy().view(hbfo.DIE_STATS_DTYPE)["bytes_read"], ds_o["bytes_read"])
+            assert np.array_equal(g.get_busy_until(), o.busy_until())
+        else:
+            o2 = hbfo.Oracle(w.profile)
+            for r in w.ranges:
+                o2.register_range(*r)
+            _, c2, s2, _, _ = o2.submit(w.acc[:n_use])
+            assert np.array_equal(h_c.numpy()[:n_use], c2) and np.array_equal(h_s.numpy()[:n_use], s2)
