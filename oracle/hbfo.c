@@ -24,6 +24,8 @@ struct hbfo_ctx {
     int32_t mode; int64_t q_ppm;
     hbfo_batch_result_t last;
     uint32_t *order; uint64_t order_count, order_cap;
+    /* channel bus as a second queued stage (off while bus_busy == NULL) */
+    int64_t *bus_busy;         /* [channels] */
     /* time-bin energy ledger (off while bin_ns == 0) */
     int64_t bin_ns; uint32_t n_bins; int64_t cur_bin;
     int64_t *ledger;           /* [n_bins][n_dies], row = bin index modulo n_bins */
@@ -74,7 +76,7 @@ const char *hbfo_strerror(int code) {
 
 static void free_ctx(hbfo_ctx *c) {
     if (!c) return;
-    free(c->busy_until); free(c->pending_pj); free(c->order); free(c->ledger);
+    free(c->busy_until); free(c->pending_pj); free(c->order); free(c->ledger); free(c->bus_busy);
     free(c->C); free(c->Gx); free(c->Gy); free(c->Gs); free(c->T); free(c->Tn); free(c->P);
     free(c->cell_region); free(c->die_region); free(c->region_kind);
     free(c->region_idle_w); free(c->region_cells);
@@ -169,6 +171,7 @@ int hbfo_reset(hbfo_ctx *c) {
     memset(&c->last, 0, sizeof(c->last));
     c->order_count = 0;
     c->cur_bin = 0;
+    if (c->bus_busy) memset(c->bus_busy, 0, c->cfg.channels * sizeof(int64_t));
     if (c->ledger) memset(c->ledger, 0, (size_t)c->n_bins * c->n_dies * sizeof(int64_t));
     if (c->thermal) for (size_t i = 0; i < c->n_cells; ++i) c->T[i] = (double)c->cfg.ambient_c;
     return HBFO_OK;
@@ -317,6 +320,33 @@ static void ledger_event(hbfo_ctx *c, uint32_t die, int64_t start, int64_t s, in
     ledger_add(c, die, b1, energy_pj - given);
 }
 
+/* ---- channel bus as a second queued stage (this build's extension; the paper gives the package 16 host channels
+ * of 64 bits, Evaluation setup, and a flash back end, but no bus model) ---------------------------------------
+ * With the stage on, a read's data-out transfer is no longer a pure latency after its array time: when the array
+ * is done with the read (time D), the transfer queues on the bus of the read's channel, first come first served in
+ * (D, batch index) order behind whatever earlier batches left on that bus, and occupies it for the transfer time.
+ * The read completes when its transfer does.  Programs keep their transfer as a latency before the array time. */
+int hbfo_enable_channel_bus(hbfo_ctx *c) {
+    if (!c) return HBFO_E_INVAL;
+    if (!c->bus_busy) c->bus_busy = (int64_t *)calloc(c->cfg.channels, sizeof(int64_t));
+    return c->bus_busy ? HBFO_OK : HBFO_E_NOMEM;
+}
+
+int hbfo_get_bus_busy_until(hbfo_ctx *c, int64_t *out, uint64_t cap) {
+    if (!c || !c->bus_busy || !out || cap < c->cfg.channels) return HBFO_E_INVAL;
+    memcpy(out, c->bus_busy, c->cfg.channels * sizeof(int64_t));
+    return HBFO_OK;
+}
+
+typedef struct { int64_t done_ns; uint32_t idx; } bent_t;
+
+static int cmp_bent(const void *pa, const void *pb) {
+    const bent_t *a = (const bent_t *)pa, *b = (const bent_t *)pb;
+    if (a->done_ns != b->done_ns) return a->done_ns < b->done_ns ? -1 : 1;
+    if (a->idx != b->idx) return a->idx < b->idx ? -1 : 1;
+    return 0;
+}
+
 /* ---- submit --------------------------------------------------------------------------------- */
 
 typedef struct { int64_t issue_ns; uint32_t idx; } qent_t;
@@ -432,6 +462,35 @@ int hbfo_submit_batch(hbfo_ctx *c, const hbfo_access_t *acc, uint64_t n, int64_t
         c->busy_until[r] = B;
     }
     c->order_count = n_ready;
+    if (c->bus_busy) {
+        /* second stage: per channel, the reads in the order the array finished them */
+        bent_t *be = (bent_t *)malloc((n_ready ? n_ready : 1) * sizeof(bent_t));
+        if (!be) { free(ds); rc = HBFO_E_NOMEM; goto done; }
+        res.modeled_ns = 0; res.max_completion_ns = 0;
+        for (uint32_t ch = 0; ch < c->cfg.channels; ++ch) {
+            uint64_t m = 0;
+            for (uint64_t i = 0; i < n; ++i)
+                if (st[i] == HBFO_ST_READY && !(acc[i].flags & 1u) && die[i] / c->cfg.dies == ch) {
+                    be[m].done_ns = completion_ns[i] - post[i]; be[m].idx = (uint32_t)i; ++m;
+                }
+            qsort(be, (size_t)m, sizeof(bent_t), cmp_bent);
+            int64_t B = c->bus_busy[ch];
+            for (uint64_t k = 0; k < m; ++k) {
+                const uint32_t i = be[k].idx;
+                int64_t start = be[k].done_ns > B ? be[k].done_ns : B;
+                B = start + post[i];
+                completion_ns[i] = B;
+                stall_ns[i] = B - acc[i].issue_ns;
+            }
+            c->bus_busy[ch] = B;
+        }
+        free(be);
+        for (uint64_t i = 0; i < n; ++i) {
+            if (st[i] != HBFO_ST_READY) continue;
+            res.modeled_ns += stall_ns[i];
+            if (completion_ns[i] > res.max_completion_ns) res.max_completion_ns = completion_ns[i];
+        }
+    }
     if (!c->bin_ns) for (uint32_t d = 0; d < c->n_dies; ++d) c->pending_pj[d] += ds[d].energy_pj;
     if (die_stats) memcpy(die_stats, ds, c->n_dies * sizeof(hbfo_die_stats_t));
     free(ds);

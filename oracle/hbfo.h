@@ -89,6 +89,11 @@ int  hbfo_submit_batch_paged(hbfo_ctx *ctx, const hbfo_access_t *acc, uint64_t n
  * copies the ring out, row k = bin first_bin + k.  hbfo_reset clears the ring and the clock. */
 int  hbfo_enable_energy_bins(hbfo_ctx *ctx, int64_t bin_ns, uint32_t n_bins);
 int  hbfo_get_energy_bins(hbfo_ctx *ctx, int64_t *out, uint64_t cap, int64_t *first_bin);
+/* Channel bus as a second queued stage (this build's extension): after this call a read's data-out transfer
+ * queues on its channel's bus in (array-done time, batch index) order instead of being a fixed latency; programs
+ * are unchanged.  hbfo_get_bus_busy_until copies the per-channel bus state out.  hbfo_reset clears it. */
+int  hbfo_enable_channel_bus(hbfo_ctx *ctx);
+int  hbfo_get_bus_busy_until(hbfo_ctx *ctx, int64_t *out, uint64_t cap);
 int  hbfo_last_result(hbfo_ctx *ctx, hbfo_batch_result_t *out);
 /* The order in which the last accepted batch was served: indices, queue-major. */
 int  hbfo_last_order(hbfo_ctx *ctx, uint32_t *order, uint64_t cap, uint64_t *count);

@@ -89,6 +89,8 @@ def lib():
                                         C.c_void_p, C.c_void_p]
         L.hbfo_submit_batch_paged.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p, C.c_void_p,
                                         C.c_void_p, C.c_void_p]
+        L.hbfo_enable_channel_bus.argtypes = [C.c_void_p]
+        L.hbfo_get_bus_busy_until.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64]
         L.hbfo_enable_energy_bins.argtypes = [C.c_void_p, C.c_int64, C.c_uint32]
         L.hbfo_get_energy_bins.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.POINTER(C.c_int64)]
         L.hbfo_rom_create.argtypes = [C.c_uint32, C.c_uint32, C.c_uint32] + [C.c_void_p] * 6 + [C.POINTER(C.c_void_p)]
@@ -148,6 +150,7 @@ class Oracle:
             cfg.n_regions = len(floorplan["region_kind"])
         self.cfg = cfg
         self.n_dies = cfg.channels * cfg.dies
+        self.n_channels = cfg.channels
         self.n_queues = self.n_dies * (cfg.planes if cfg.queue_level == 0 else 1)
         self.n_cells = cfg.grid_h * cfg.grid_w if floorplan is not None else 0
         h = C.c_void_p()
@@ -192,6 +195,18 @@ class Oracle:
         if check and rc != 0:
             raise OracleError(rc)
         return rc, comp, stall, status, ds
+
+    def enable_channel_bus(self):
+        rc = lib().hbfo_enable_channel_bus(self._h)
+        if rc != 0:
+            raise OracleError(rc)
+
+    def bus_busy_until(self) -> np.ndarray:
+        out = np.zeros(self.n_channels, np.int64)
+        rc = lib().hbfo_get_bus_busy_until(self._h, out.ctypes.data, out.size)
+        if rc != 0:
+            raise OracleError(rc)
+        return out
 
     def enable_energy_bins(self, bin_ns: int, n_bins: int):
         rc = lib().hbfo_enable_energy_bins(self._h, bin_ns, n_bins)

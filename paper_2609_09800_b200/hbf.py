@@ -188,6 +188,7 @@ class Context:
         self._torch = torch
         cfg, keep = make_config(profile, floorplan)
         self.n_dies = cfg.channels * cfg.dies
+        self.n_channels = cfg.channels
         self.n_queues = self.n_dies * (cfg.planes if cfg.queue_level == 0 else 1)
         self.n_cells = cfg.grid_h * cfg.grid_w if floorplan is not None else 0
         self.n_regions = cfg.n_regions if floorplan is not None else 0
