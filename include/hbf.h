@@ -145,6 +145,21 @@ HBF_API int hbf_submit_batch_paged(hbf_ctx *ctx, const hbf_access_t *d_acc, uint
                            int64_t *d_completion_ns, int64_t *d_stall_ns, uint8_t *d_status,
                            hbf_die_stats_t *d_die_stats, void *d_workspace, size_t workspace_bytes);
 
+/* Channel bus as a second queued stage (an extension; the paper gives the package 16 host channels of 64 bits,
+ * Evaluation setup, but no bus model; the definition is this library's).  After hbf_enable_channel_bus, a read's
+ * data-out transfer is no longer a fixed latency after its array time: when the array is done with the read, the
+ * transfer queues on the bus of the read's channel, first come first served in (array-done time, index) order
+ * behind whatever earlier batches left there, and holds the bus for the transfer time; the read completes when its
+ * transfer does.  Programs are unchanged (their transfer stays a latency before the array time), and so are the
+ * queue state and the per-die statistics.  The stage runs inside hbf_submit_batch after the array stage (a radix
+ * sort of the reads by channel and array-done time, then a segmented max-plus scan); hbf_workspace_bytes grows by
+ * 4 bytes per access once it is on.  An array-done time of 2^47 ns or more cannot be ordered: the batch's result
+ * becomes HBF_E_INVAL after its array stage has been committed and the context is poisoned.
+ * hbf_get_bus_busy_until synchronises and copies the per-channel bus state to host_out [channels]; hbf_reset clears
+ * it.  The state blob of hbf_get_state does not carry it.  hbf_submit_batch_paged is refused while the stage is on. */
+HBF_API int hbf_enable_channel_bus(hbf_ctx *ctx);
+HBF_API int hbf_get_bus_busy_until(hbf_ctx *ctx, int64_t *host_out, uint64_t cap);
+
 /* Time-bin power integration (Section "Design", the event-based energy model: event energies accumulate in
  * bins; an event that spans more than one bin has its energy split across the bins in proportion to the time
  * overlap; P = E / dt + P_idle).  After hbf_enable_energy_bins, hbf_submit_batch books the energy of every

@@ -36,6 +36,8 @@ struct hbf_ctx {
     BatchCtrl *d_ctrl = nullptr; hbf_batch_result_t *d_result = nullptr;
     int64_t *d_busy = nullptr, *d_busy_stage = nullptr, *d_pending = nullptr; hbf_die_stats_t *d_stats_stage = nullptr;
     hbf_batch_result_t *h_result = nullptr;      // pinned
+    // channel bus as a second queued stage (off while d_bus_busy == nullptr)
+    int64_t *d_bus_busy = nullptr; BatchCtrl *d_bus_ctrl = nullptr;
     // time-bin energy ledger (off while bin_ns == 0)
     int64_t bin_ns = 0, cur_bin = 0; uint32_t n_bins = 0; unsigned long long *d_ledger = nullptr;
     float *h_hot = nullptr;                      // pinned [3]
@@ -172,6 +174,8 @@ int hbf_destroy(hbf_ctx *c) {
     if (c->ev_made) { for (auto &e : c->ev) cudaEventDestroy(e); for (auto &e : c->ev_th) cudaEventDestroy(e); }
     if (c->h_result) cudaFreeHost(c->h_result);
     if (c->d_ledger) cudaFree(c->d_ledger);
+    if (c->d_bus_busy) cudaFree(c->d_bus_busy);
+    if (c->d_bus_ctrl) cudaFree(c->d_bus_ctrl);
     if (c->h_hot) cudaFreeHost(c->h_hot);
     if (c->h_ext) cudaFreeHost(c->h_ext);
     delete c;
@@ -341,7 +345,7 @@ int hbf_clear_ranges(hbf_ctx *c) {
 
 size_t hbf_workspace_bytes(const hbf_ctx *c, uint64_t n) {
     if (!c) return 0;
-    return workspace_layout(n, c->mp.n_queues, nullptr, nullptr);
+    return workspace_layout(n, c->mp.n_queues, nullptr, nullptr, c->d_bus_busy ? 1 : 0);
 }
 
 int hbf_set_thermal_path(hbf_ctx *c, int32_t generic_only) {
@@ -366,7 +370,7 @@ int hbf_submit_batch(hbf_ctx *c, const hbf_access_t *d_acc, uint64_t n, int64_t 
     if ((reinterpret_cast<uintptr_t>(d_acc) & 7u) || (reinterpret_cast<uintptr_t>(d_completion_ns) & 7u) ||
         (reinterpret_cast<uintptr_t>(d_stall_ns) & 7u) || (reinterpret_cast<uintptr_t>(d_die_stats) & 7u)) return HBF_E_INVAL;
     SubmitArgs a{};
-    const size_t need = workspace_layout(n, c->mp.n_queues, &a.ws, d_workspace);
+    const size_t need = workspace_layout(n, c->mp.n_queues, &a.ws, d_workspace, c->d_bus_busy ? 1 : 0);
     if (!d_workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(d_workspace) & 255u)) return HBF_E_WORKSPACE;
     a.acc = d_acc; a.n = n; a.completion = d_completion_ns; a.stall = d_stall_ns; a.status = d_status; a.die_stats = d_die_stats;
     a.ranges = c->d_ranges; a.mp_dev = c->d_mp; a.mp = c->mp; a.state = c->d_state; a.ctrl = c->d_ctrl; a.result = c->d_result;
@@ -384,6 +388,8 @@ int hbf_submit_batch(hbf_ctx *c, const hbf_access_t *d_acc, uint64_t n, int64_t 
     if (a.binned)
         CK(launch_energy_bins(d_acc, n, d_completion_ns, c->d_ranges, c->d_mp, c->d_ctrl, c->d_result, c->d_ledger, c->bin_ns,
                               c->n_bins, c->cur_bin, c->sm_count, c->stream));
+    if (c->d_bus_busy)                                       // after the ledger: its events are the array intervals
+        CK(launch_bus_stage(a, c->d_bus_ctrl, c->d_bus_busy, c->stream));
     c->submitted = true;
     return HBF_OK;
 }
@@ -400,7 +406,7 @@ int hbf_submit_batch_paged(hbf_ctx *c, const hbf_access_t *d_acc, uint64_t n, ui
     if (n == 0)                                             // nothing to split: the ordinary path reports the empty batch
         return hbf_submit_batch(c, d_acc, 0, d_completion_ns, d_stall_ns, d_status, d_die_stats, d_workspace, workspace_bytes);
     if (c->terminal) return HBF_E_LINK_SHUTDOWN;
-    if (n > HBF_MAX_BATCH || c->bin_ns != 0) return HBF_E_INVAL;          // the time-bin ledger books whole accesses only
+    if (n > HBF_MAX_BATCH || c->bin_ns != 0 || c->d_bus_busy) return HBF_E_INVAL;   // ledger and bus stage take whole accesses only
     if (!d_acc || !d_completion_ns || !d_stall_ns) return HBF_E_INVAL;
     if ((reinterpret_cast<uintptr_t>(d_acc) & 7u) || (reinterpret_cast<uintptr_t>(d_completion_ns) & 7u) ||
         (reinterpret_cast<uintptr_t>(d_stall_ns) & 7u) || (reinterpret_cast<uintptr_t>(d_die_stats) & 7u)) return HBF_E_INVAL;
@@ -432,6 +438,26 @@ int hbf_submit_batch_paged(hbf_ctx *c, const hbf_access_t *d_acc, uint64_t n, ui
     CK(launch_submit(a, c->stream));
     CK(launch_paged_join(d_acc, n, pw, c->d_result, d_completion_ns, d_stall_ns, d_status, c->sm_count, c->stream));
     c->submitted = true;
+    return HBF_OK;
+}
+
+int hbf_enable_channel_bus(hbf_ctx *c) {
+    if (!c) return HBF_E_INVAL;
+    if (c->d_bus_busy) return HBF_OK;
+    CK(cudaStreamSynchronize(c->stream));
+    int64_t *b = nullptr; BatchCtrl *bc = nullptr;
+    if (cudaMalloc(&b, (size_t)c->mp.channels * 8) != cudaSuccess) return HBF_E_NOMEM;
+    if (cudaMalloc(&bc, sizeof(BatchCtrl)) != cudaSuccess) { cudaFree(b); return HBF_E_NOMEM; }
+    c->d_bus_busy = b; c->d_bus_ctrl = bc;
+    CK(cudaMemsetAsync(b, 0, (size_t)c->mp.channels * 8, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    return HBF_OK;
+}
+
+int hbf_get_bus_busy_until(hbf_ctx *c, int64_t *host_out, uint64_t cap) {
+    if (!c || !c->d_bus_busy || !host_out || cap < c->mp.channels) return HBF_E_INVAL;
+    CK(cudaMemcpyAsync(host_out, c->d_bus_busy, (size_t)c->mp.channels * 8, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
     return HBF_OK;
 }
 
@@ -536,6 +562,7 @@ int hbf_reset(hbf_ctx *c) {
     CK(cudaMemsetAsync(c->d_pending, 0, c->mp.n_dies * sizeof(int64_t), c->stream));
     CK(cudaMemsetAsync(c->d_result, 0, sizeof(hbf_batch_result_t), c->stream));
     if (c->bin_ns) { CK(cudaMemsetAsync(c->d_ledger, 0, (size_t)c->n_bins * c->mp.n_dies * 8, c->stream)); c->cur_bin = 0; }
+    if (c->d_bus_busy) CK(cudaMemsetAsync(c->d_bus_busy, 0, (size_t)c->mp.channels * 8, c->stream));
     if (c->thermal) {
         const size_t nc = (size_t)c->td.H * c->td.W;
         CK(cudaMemsetAsync(c->td.theta[0], 0, nc * sizeof(float), c->stream));

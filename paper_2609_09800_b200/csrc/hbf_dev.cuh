@@ -89,6 +89,7 @@ struct Workspace {
     void *in_tile;                       // [tiles] stall bookkeeping of the in-order path
     void *in_head;                       // [tiles][queues][8]: the first accesses of every (tile, queue), for the fix-up
     uint8_t *in_headcnt;                 // [tiles][queues]: how many of them exist; 0xff marks a queue for the straggle pass
+    uint32_t *bus_xfer;                  // [n] transfer time of every read (only with the channel-bus stage on)
     size_t bytes;
 };
 
@@ -118,7 +119,9 @@ inline uint64_t inorder_tiles_bound(uint64_t n) {
     const uint64_t t = (n + kInTileQuantum - 1) / kInTileQuantum;
     return t < 1 ? 1 : (t < kInMaxTiles ? t : kInMaxTiles);
 }
-size_t workspace_layout(uint64_t n, uint32_t n_queues, Workspace *ws, void *base);
+size_t workspace_layout(uint64_t n, uint32_t n_queues, Workspace *ws, void *base, int with_bus = 0);
+// channel bus as a second queued stage, after launch_submit on the same arguments (bc: a control block of its own)
+cudaError_t launch_bus_stage(const SubmitArgs &a, BatchCtrl *bc, int64_t *bus_busy, cudaStream_t st);
 // tile size (records) of the in-order path for a batch of n on a device with sm_count SMs
 uint64_t inorder_tile_records(uint64_t n, int sm_count);
 size_t inorder_head_bytes(uint64_t tiles, uint32_t n_queues);

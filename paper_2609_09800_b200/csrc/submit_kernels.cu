@@ -643,11 +643,277 @@ __global__ void k_queue_order(const BatchCtrl *ctrl, const uint32_t *idx0, const
 }
 
 // =====================================================================================================
+// channel bus as a second queued stage (an extension; the library's own definition).  After the array
+// stage, a read's data-out transfer queues on the bus of its channel in (array-done time, index) order and
+// holds it for the transfer time; the read completes when the transfer does.  Programs are unchanged.
+//   keys   per access: channel << 47 | array-done time (reads), a sentinel behind every channel (the rest)
+//   sort   the onesweep passes of the sort path, over the key bits that differ
+//   scan   in sorted order a read is the map B -> max(B, D) + x on its channel's bus; channels are segments
+//          whose first map starts from the bus state earlier batches left.  Three kernels, no look-back: tile
+//          aggregates, an exclusive scan of them by one block, tiles again with their carry.
+// =====================================================================================================
+struct BusMap { int64_t S, M; int f; };                    // B -> max(B + S, M); f: contains a segment head (then B does not matter)
+__device__ __forceinline__ BusMap bus_then(const BusMap &a, const BusMap &b) {       // a first, then b
+    if (b.f) return b;
+    BusMap r; r.S = a.S + b.S; r.M = max((int64_t)(a.M + b.S), b.M); r.f = a.f; return r;
+}
+__device__ __forceinline__ BusMap bus_identity() { BusMap r; r.S = 0; r.M = kNegInf; r.f = 0; return r; }
+__device__ __forceinline__ BusMap bus_shfl_up(const BusMap &v, int o) {
+    BusMap r; r.S = __shfl_up_sync(0xffffffffu, v.S, o); r.M = __shfl_up_sync(0xffffffffu, v.M, o); r.f = __shfl_up_sync(0xffffffffu, v.f, o);
+    return r;
+}
+constexpr int kBusThreads = 256;
+constexpr int kBusItems = 8;
+constexpr int kBusTile = kBusThreads * kBusItems;          // as many entries as a scan tile of the sort path: its descriptors are reused
+static_assert(kBusTile == kScanTile && sizeof(BusMap) <= sizeof(ScanDesc), "the bus stage reuses the scan descriptors");
+
+__global__ void k_bus_begin(BatchCtrl *bc, const hbf_batch_result_t *result, uint32_t *hist) {
+    uint32_t *w = reinterpret_cast<uint32_t *>(bc);
+    for (int i = threadIdx.x; i < (int)(sizeof(BatchCtrl) / 4); i += blockDim.x) w[i] = 0u;
+    for (int i = threadIdx.x; i < kMaxPasses * kRadix; i += blockDim.x) hist[i] = 0u;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        bc->key_and = ~0ull; bc->run_sort = 1u; bc->unsorted = 1u;
+        bc->max_completion_ns = INT64_MIN;
+        if (result->code != HBF_OK) bc->skip = 1;           // a refused batch has no second stage
+    }
+}
+
+__global__ void __launch_bounds__(256)
+k_bus_keys(const hbf_access_t *__restrict__ acc, uint64_t n, const int64_t *__restrict__ completion,
+           const RangeSnap *__restrict__ ranges, const ModelParams *__restrict__ mp_g, BatchCtrl *bc,
+           uint64_t *__restrict__ keys, uint32_t *__restrict__ xfer_out) {
+    __shared__ ModelParams mp;
+    if (bc->skip) return;
+    for (int i = threadIdx.x; i < (int)(sizeof(ModelParams) / 4); i += blockDim.x)
+        reinterpret_cast<uint32_t *>(&mp)[i] = reinterpret_cast<const uint32_t *>(mp_g)[i];
+    __syncthreads();
+    const RangeSnap &rs = *ranges;
+    const uint64_t sentinel = (uint64_t)mp.channels << kIssueBits;
+    const Div64 one = make_div64(1000000ull);
+    unsigned long long reads = 0, k_or = 0, k_and = ~0ull;
+    unsigned late = 0;
+    const uint64_t n_round = (n + 31ull) & ~31ull;
+    for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_round; i += (uint64_t)gridDim.x * blockDim.x) {
+        if (i >= n) continue;
+        const uint64_t *rec = reinterpret_cast<const uint64_t *>(acc + i);
+        const uint64_t addr = __ldg(rec), bf = __ldg(rec + 2);
+        const int64_t issue = (int64_t)__ldg(rec + 1);
+        const uint32_t bytes = (uint32_t)bf, flags = (uint32_t)(bf >> 32);
+        int g = 0;
+        uint64_t key = sentinel;
+        uint32_t x = 0;
+        if (classify(rs, addr, issue, bytes, flags, &g) == HBF_ST_READY && !(flags & 1u)) {
+            const Decoded d = decode(mp, rs.media_offset[g] + (addr - rs.base[g]), bytes);
+            const Terms t = service_terms(mp, bytes, d.npages, 0u, 1000000, one);      // the transfer does not depend on the throttle
+            const int64_t done = completion[i] - t.xfer;                                 // when the array is done with the read
+            x = (uint32_t)t.xfer;
+            if (done < 0 || done >= HBF_ISSUE_LIMIT) late = 1u;
+            else { key = ((uint64_t)(d.die / mp.dies) << kIssueBits) | (uint64_t)done; ++reads; }
+        }
+        keys[i] = key; xfer_out[i] = x;
+        k_or |= key; k_and &= key;
+    }
+    reads = (unsigned long long)warp_sum((long long)reads);
+    k_or = warp_or(k_or); k_and = warp_and(k_and);
+    late = __any_sync(0xffffffffu, late);
+    if (lane_id() == 0) {
+        if (reads) atomicAdd(&bc->n_ready, reads);
+        atomicOr(&bc->key_or, k_or); atomicAnd(&bc->key_and, k_and);
+        if (late) atomicExch(&bc->code, (int)HBF_E_INVAL);  // an array-done time beyond the 47-bit key field
+    }
+}
+
+__global__ void k_bus_check(BatchCtrl *bc) { if (bc->code != HBF_OK) bc->skip = 1; }
+
+// entry j of the sorted order as a map on its channel's bus
+__device__ __forceinline__ BusMap bus_entry(uint64_t j, const uint64_t *__restrict__ ks, const uint32_t *__restrict__ is, bool have_idx,
+                                            const uint32_t *__restrict__ xfer, const int64_t *__restrict__ bus_busy,
+                                            uint32_t *idx_out, uint32_t *ch_out, int64_t *plain_out) {
+    const uint64_t key = ks[j];
+    const uint32_t ch = (uint32_t)(key >> kIssueBits), idx = have_idx ? is[j] : (uint32_t)j;
+    const int64_t done = (int64_t)(key & kIssueMask), x = (int64_t)xfer[idx];
+    const bool head = j == 0 || (uint32_t)(ks[j - 1] >> kIssueBits) != ch;
+    BusMap m; m.S = x; m.M = (head ? max(bus_busy[ch], done) : done) + x; m.f = head ? 1 : 0;
+    *idx_out = idx; *ch_out = ch; *plain_out = done + x;
+    return m;
+}
+
+__global__ void __launch_bounds__(kBusThreads)
+k_bus_reduce(const BatchCtrl *bc, const uint64_t *k0, const uint64_t *k1, const uint32_t *i0, const uint32_t *i1,
+             const uint32_t *__restrict__ xfer, const int64_t *__restrict__ bus_busy, ScanDesc *agg) {
+    __shared__ BusMap s_warp[kBusThreads / 32];
+    if (bc->skip) return;
+    const uint64_t m = bc->n_ready;
+    const uint32_t np = bc->plan.n_passes;
+    const uint64_t *ks = (np & 1u) ? k1 : k0; const uint32_t *is = (np & 1u) ? i1 : i0;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    for (uint64_t tile = blockIdx.x; tile * kBusTile < m; tile += gridDim.x) {
+        BusMap mine = bus_identity();
+        const uint64_t first = tile * kBusTile + (uint64_t)tid * kBusItems;
+        for (int u = 0; u < kBusItems; ++u) {
+            const uint64_t j = first + u;
+            if (j >= m) break;
+            uint32_t idx, ch; int64_t plain;
+            mine = bus_then(mine, bus_entry(j, ks, is, np != 0u, xfer, bus_busy, &idx, &ch, &plain));
+        }
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const BusMap p = bus_shfl_up(mine, o); if (lane >= o) mine = bus_then(p, mine); }
+        __syncthreads();
+        if (lane == 31) s_warp[warp] = mine;
+        __syncthreads();
+        if (tid == 0) {
+            BusMap t = s_warp[0];
+            for (int w = 1; w < kBusThreads / 32; ++w) t = bus_then(t, s_warp[w]);
+            ScanDesc d; d.S = t.S; d.M = t.M; d.value = 0; d.status = (uint32_t)t.f; d.pad = 0;
+            agg[tile] = d;
+        }
+    }
+}
+
+// one block: exclusive scan (in tile order) of the tile aggregates, in place
+__global__ void __launch_bounds__(1024)
+k_bus_tile_scan(const BatchCtrl *bc, ScanDesc *agg) {
+    __shared__ BusMap s_warp[32];
+    if (bc->skip) return;
+    const uint64_t tiles = (bc->n_ready + kBusTile - 1) / kBusTile;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint64_t per = (tiles + 1023) / 1024, lo = (uint64_t)tid * per, hi = min(tiles, lo + per);
+    BusMap mine = bus_identity();
+    for (uint64_t t = lo; t < hi; ++t) { BusMap e; e.S = agg[t].S; e.M = agg[t].M; e.f = (int)agg[t].status; mine = bus_then(mine, e); }
+    BusMap incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const BusMap p = bus_shfl_up(incl, o); if (lane >= o) incl = bus_then(p, incl); }
+    if (lane == 31) s_warp[warp] = incl;
+    __syncthreads();
+    BusMap before = bus_identity();
+    for (int w = 0; w < warp; ++w) before = bus_then(before, s_warp[w]);
+    BusMap prev = bus_shfl_up(incl, 1);
+    if (lane == 0) prev = bus_identity();
+    BusMap run = bus_then(before, prev);                    // everything before this thread's tiles
+    for (uint64_t t = lo; t < hi; ++t) {
+        BusMap e; e.S = agg[t].S; e.M = agg[t].M; e.f = (int)agg[t].status;
+        ScanDesc d; d.S = run.S; d.M = run.M; d.value = 0; d.status = (uint32_t)run.f; d.pad = 0;
+        agg[t] = d;
+        run = bus_then(run, e);
+    }
+}
+
+__global__ void __launch_bounds__(kBusThreads)
+k_bus_apply(const hbf_access_t *__restrict__ acc, BatchCtrl *bc, const uint64_t *k0, const uint64_t *k1, const uint32_t *i0,
+            const uint32_t *i1, const uint32_t *__restrict__ xfer, int64_t *bus_busy, const ScanDesc *__restrict__ agg,
+            int64_t *__restrict__ completion, int64_t *__restrict__ stall) {
+    __shared__ BusMap s_warp[kBusThreads / 32];
+    if (bc->skip) return;
+    const uint64_t m = bc->n_ready;
+    const uint32_t np = bc->plan.n_passes;
+    const uint64_t *ks = (np & 1u) ? k1 : k0; const uint32_t *is = (np & 1u) ? i1 : i0;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    long long moved = 0, max_c = INT64_MIN;
+    for (uint64_t tile = blockIdx.x; tile * kBusTile < m; tile += gridDim.x) {
+        const uint64_t first = tile * kBusTile + (uint64_t)tid * kBusItems;
+        BusMap e[kBusItems]; uint32_t idx[kBusItems], ch[kBusItems]; int64_t plain[kBusItems];
+        BusMap mine = bus_identity();
+#pragma unroll
+        for (int u = 0; u < kBusItems; ++u) {
+            const uint64_t j = first + u;
+            if (j < m) { e[u] = bus_entry(j, ks, is, np != 0u, xfer, bus_busy, &idx[u], &ch[u], &plain[u]); mine = bus_then(mine, e[u]); }
+            else { e[u] = bus_identity(); idx[u] = 0; ch[u] = 0; plain[u] = 0; }
+        }
+        BusMap incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const BusMap p = bus_shfl_up(incl, o); if (lane >= o) incl = bus_then(p, incl); }
+        __syncthreads();
+        if (lane == 31) s_warp[warp] = incl;
+        __syncthreads();
+        BusMap run; run.S = agg[tile].S; run.M = agg[tile].M; run.f = (int)agg[tile].status;     // everything before the tile
+        for (int w = 0; w < warp; ++w) run = bus_then(run, s_warp[w]);
+        BusMap prev = bus_shfl_up(incl, 1);
+        if (lane == 0) prev = bus_identity();
+        run = bus_then(run, prev);
+        // Every prefix holds a segment head (entry 0 is one), so the composed map's constant term is the bus's
+        // busy-until after the entry: the time the read's transfer ends.
+#pragma unroll
+        for (int u = 0; u < kBusItems; ++u) {
+            const uint64_t j = first + u;
+            if (j >= m) break;
+            run = bus_then(run, e[u]);
+            const int64_t done = run.M;
+            completion[idx[u]] = done; stall[idx[u]] = done - acc[idx[u]].issue_ns;
+            moved += done - plain[u]; max_c = max(max_c, (long long)done);
+        }
+    }
+    moved = warp_sum(moved); max_c = warp_max(max_c);
+    if (lane == 0) {
+        if (moved) atomicAdd((unsigned long long *)&bc->modeled_ns, (unsigned long long)moved);
+        if (max_c != INT64_MIN) atomicMax(&bc->max_completion_ns, max_c);
+    }
+}
+
+// The bus state is written by a pass of its own, after every tile has read the old one: the last read of each
+// channel's segment holds the new busy-until in its completion.
+__global__ void __launch_bounds__(256)
+k_bus_commit(const BatchCtrl *bc, const uint64_t *k0, const uint64_t *k1, const uint32_t *i0, const uint32_t *i1,
+             const int64_t *__restrict__ completion, int64_t *bus_busy) {
+    if (bc->skip) return;
+    const uint64_t m = bc->n_ready;
+    const uint32_t np = bc->plan.n_passes;
+    const uint64_t *ks = (np & 1u) ? k1 : k0; const uint32_t *is = (np & 1u) ? i1 : i0;
+    for (uint64_t j = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; j < m; j += (uint64_t)gridDim.x * blockDim.x) {
+        const uint32_t ch = (uint32_t)(ks[j] >> kIssueBits);
+        if (j + 1 == m || (uint32_t)(ks[j + 1] >> kIssueBits) != ch) bus_busy[ch] = completion[np ? is[j] : (uint32_t)j];
+    }
+}
+
+__global__ void k_bus_finish(const BatchCtrl *bc, hbf_batch_result_t *result, DevState *state) {
+    if (bc->code != HBF_OK) { result->code = bc->code; state->poisoned = 1; return; }   // the array stage is committed: the context cannot go on
+    if (bc->skip) return;
+    result->modeled_ns += bc->modeled_ns;
+    if (bc->max_completion_ns > result->max_completion_ns) result->max_completion_ns = bc->max_completion_ns;
+}
+
+cudaError_t launch_bus_stage(const SubmitArgs &a, BatchCtrl *bc, int64_t *bus_busy, cudaStream_t st) {
+    const uint64_t n = a.n;
+    if (n == 0) return cudaSuccess;
+    const uint64_t sort_tiles = (n + kSortTile - 1) / kSortTile, bus_tiles = (n + kBusTile - 1) / kBusTile;
+    cudaError_t e = cudaMemsetAsync(a.ws.sort_desc[0], 0, sort_tiles * kRadix * 4, st);
+    if (e != cudaSuccess) return e;
+    k_bus_begin<<<1, 256, 0, st>>>(bc, a.result, a.ws.hist);
+    const unsigned wide = (unsigned)std::min<uint64_t>((n + 255) / 256, (uint64_t)a.sm_count * 8);
+    k_bus_keys<<<wide, 256, 0, st>>>(a.acc, n, a.completion, a.ranges, a.mp_dev, bc, a.ws.keys[0], a.ws.bus_xfer);
+    k_bus_check<<<1, 1, 0, st>>>(bc);
+    k_plan<<<1, 32, 0, st>>>(bc, 1);
+    const unsigned hist_grid = (unsigned)std::min<uint64_t>((n + kHistThreads * 8 - 1) / (kHistThreads * 8), (uint64_t)a.sm_count * 4);
+    k_hist<<<hist_grid, kHistThreads, 0, st>>>(a.ws.keys[0], n, bc, a.ws.hist);
+    static bool attr_set = false;
+    if (!attr_set) {
+        e = cudaFuncSetAttribute(k_sort_pass, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSortSmem);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    const unsigned sort_grid = (unsigned)std::min<uint64_t>(sort_tiles, (uint64_t)a.sm_count * 3);
+    for (int p = 0; p < kMaxPasses; ++p)
+        k_sort_pass<<<sort_grid, kSortThreads, kSortSmem, st>>>(p, n, bc, a.state, a.ws.hist, a.ws.keys[0], a.ws.keys[1],
+                                                                a.ws.idx[0], a.ws.idx[1], a.ws.sort_desc[0], a.ws.sort_desc[1]);
+    k_bus_check<<<1, 1, 0, st>>>(bc);                        // a look-back that gave up sets the code
+    const unsigned tiles_grid = (unsigned)std::min<uint64_t>(bus_tiles, (uint64_t)a.sm_count * 8);
+    ScanDesc *agg = (ScanDesc *)a.ws.scan_desc;
+    k_bus_reduce<<<tiles_grid, kBusThreads, 0, st>>>(bc, a.ws.keys[0], a.ws.keys[1], a.ws.idx[0], a.ws.idx[1], a.ws.bus_xfer, bus_busy, agg);
+    k_bus_tile_scan<<<1, 1024, 0, st>>>(bc, agg);
+    k_bus_apply<<<tiles_grid, kBusThreads, 0, st>>>(a.acc, bc, a.ws.keys[0], a.ws.keys[1], a.ws.idx[0], a.ws.idx[1], a.ws.bus_xfer, bus_busy,
+                                                    agg, a.completion, a.stall);
+    k_bus_commit<<<wide, 256, 0, st>>>(bc, a.ws.keys[0], a.ws.keys[1], a.ws.idx[0], a.ws.idx[1], a.completion, bus_busy);
+    k_bus_finish<<<1, 1, 0, st>>>(bc, a.result, a.state);
+    g_kernel_launches += 10 + kMaxPasses;
+    return cudaGetLastError();
+}
+
+// =====================================================================================================
 // host side
 // =====================================================================================================
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-size_t workspace_layout(uint64_t n, uint32_t n_queues, Workspace *ws, void *base_ptr) {
+size_t workspace_layout(uint64_t n, uint32_t n_queues, Workspace *ws, void *base_ptr, int with_bus) {
     const uint64_t nn = n ? n : 1;
     const uint64_t sort_tiles = (nn + kSortTile - 1) / kSortTile, scan_tiles = (nn + kScanTile - 1) / kScanTile;
     size_t off = 0;
@@ -662,11 +928,12 @@ size_t workspace_layout(uint64_t n, uint32_t n_queues, Workspace *ws, void *base
     void *ia = take(inorder ? in_tiles * n_queues * 16 : 0), *ib = take(inorder ? in_tiles * n_queues * 8 : 0);
     void *it = take(inorder ? in_tiles * 32 : 0), *ih = take(inorder ? inorder_head_bytes(in_tiles, n_queues) : 0);
     void *ic = take(inorder ? in_tiles * n_queues : 0);
+    void *bx = take(with_bus ? nn * 4 : 0);
     if (ws) {
         ws->keys[0] = (uint64_t *)k0; ws->keys[1] = (uint64_t *)k1; ws->idx[0] = (uint32_t *)i0; ws->idx[1] = (uint32_t *)i1;
         ws->hist = (uint32_t *)h; ws->sort_desc[0] = (uint32_t *)d0; ws->sort_desc[1] = (uint32_t *)d1;
         ws->scan_desc = sd; ws->in_agg = (int64_t *)ia; ws->in_bin = (int64_t *)ib;
-        ws->in_tile = it; ws->in_head = ih; ws->in_headcnt = (uint8_t *)ic; ws->bytes = off;
+        ws->in_tile = it; ws->in_head = ih; ws->in_headcnt = (uint8_t *)ic; ws->bus_xfer = (uint32_t *)bx; ws->bytes = off;
     }
     return off;
 }

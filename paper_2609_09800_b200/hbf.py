@@ -30,7 +30,7 @@ EXPORTS = ("hbf_create", "hbf_destroy", "hbf_register_range", "hbf_clear_ranges"
            "hbf_get_pending_energy", "hbf_get_temps", "hbf_euler_limit_ns", "hbf_queue_order", "hbf_strerror",
            "hbf_set_profiling", "hbf_get_profile", "hbf_kernel_launches", "hbf_euler_substeps_static", "hbf_set_thermal_path",
            "hbf_workspace_bytes_paged", "hbf_submit_batch_paged",
-           "hbf_enable_energy_bins", "hbf_get_energy_bins",
+           "hbf_enable_energy_bins", "hbf_get_energy_bins", "hbf_enable_channel_bus", "hbf_get_bus_busy_until",
            "hbf_rom_create", "hbf_rom_destroy", "hbf_rom_reset", "hbf_rom_step", "hbf_rom_get_state")
 STATIC_MAX_CELLS = 65536
 PROF_STAGES = ("begin", "classify", "plan_hist", "sort", "scan", "finish", "inorder", "thermal")
@@ -91,6 +91,8 @@ def lib():
         L.hbf_workspace_bytes_paged.argtypes = [vp, u64, u64]
         L.hbf_workspace_bytes_paged.restype = C.c_size_t
         L.hbf_submit_batch_paged.argtypes = [vp, vp, u64, u64, vp, vp, vp, vp, vp, C.c_size_t]
+        L.hbf_enable_channel_bus.argtypes = [vp]
+        L.hbf_get_bus_busy_until.argtypes = [vp, vp, u64]
         L.hbf_enable_energy_bins.argtypes = [vp, i64, u32]
         L.hbf_get_energy_bins.argtypes = [vp, vp, u64, C.POINTER(i64)]
         L.hbf_rom_create.argtypes = [u32, u32, u32, vp, vp, vp, vp, vp, vp, vp, C.POINTER(vp)]
@@ -255,6 +257,19 @@ class Context:
         return lib().hbf_submit_batch_paged(self._h, _ptr(d_acc), n, parts_capacity, _ptr(d_completion), _ptr(d_stall),
                                             _ptr(d_status), _ptr(d_die_stats), _ptr(d_workspace),
                                             d_workspace.numel() * d_workspace.element_size())
+
+    def enable_channel_bus(self):
+        rc = lib().hbf_enable_channel_bus(self._h)
+        if rc != 0:
+            raise HbfError(rc, "hbf_enable_channel_bus")
+        self._ws = None                                      # the workspace grows once the stage is on
+
+    def get_bus_busy_until(self):
+        out = np.zeros(self.n_channels, np.int64)
+        rc = lib().hbf_get_bus_busy_until(self._h, out.ctypes.data, out.size)
+        if rc != 0:
+            raise HbfError(rc, "hbf_get_bus_busy_until")
+        return out
 
     def enable_energy_bins(self, bin_ns: int, n_bins: int):
         rc = lib().hbf_enable_energy_bins(self._h, bin_ns, n_bins)
