@@ -57,6 +57,8 @@ def parse_args():
                          "capacity_paged: the capacity-mode batch through the page-granular submit; rom: fit the reduced-order "
                          "thermal model of the package floorplan and time its step against the full grid (none is the headline)")
     ap.add_argument("--horizon-ms", type=int, default=1000, help="simulated time of the coupled_thermal run")
+    ap.add_argument("--channel-bus", action="store_true",
+                    help="capacity_mode: also run the channel-bus stage (reads' transfers queue per channel); not the headline")
     ap.add_argument("--energy-bins", action="store_true",
                     help="coupled_thermal: book event energies into 1 ms bins (time-bin power integration) instead of at submit")
     return ap.parse_args()
@@ -389,6 +391,8 @@ def main():
     for r in w.ranges:
         ctx.register_range(*r)
     ctx.set_path({"auto": hbf.PATH_AUTO, "sort": hbf.PATH_SORT, "sort_full": hbf.PATH_SORT_FULL}[args.path])
+    if args.channel_bus:
+        ctx.enable_channel_bus()
 
     # inputs resident in HBM before the timed region
     h_acc = torch.from_numpy(w.acc.view(np.int64).reshape(-1))
@@ -495,7 +499,7 @@ def main():
                 "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": "int64", "data": "synthetic",
                 "config": {"workload": "capacity_mode", "accesses_per_step": n, "geometry": "64x8x4", "queues": 2048,
-                           "path": args.path, "thermal_grid": "128x128", "l2": "inputs (%.1f GB) larger than L2" % (n * 24 / 1e9),
+                           "path": args.path, "channel_bus_stage": bool(args.channel_bus), "thermal_grid": "128x128", "l2": "inputs (%.1f GB) larger than L2" % (n * 24 / 1e9),
                            "multi_gpu": "replicas only", "gen_seconds": round(gen_s, 1),
                            "state": "queues idle at the start of every step (reset outside the timed region)"},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
