@@ -131,7 +131,8 @@ __global__ void __launch_bounds__(kInThreads, kInBlocksPerSM)
 k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_records, const RangeSnap *__restrict__ ranges_g,
                 const __grid_constant__ ModelParams mp_arg, const __grid_constant__ FastRange fast_arg, BatchCtrl *ctrl, uint8_t *__restrict__ status, int64_t *__restrict__ in_agg,
                 hbf_die_stats_t *stats_stage, int64_t *__restrict__ completion, int64_t *__restrict__ stall,
-                const int64_t *__restrict__ in_bin, InTile *in_tile, InHead *__restrict__ in_head, uint8_t *__restrict__ in_headcnt) {
+                const int64_t *__restrict__ in_bin, InTile *in_tile, InHead *__restrict__ in_head, uint8_t *__restrict__ in_headcnt,
+                const int64_t *__restrict__ busy) {
     extern __shared__ __align__(16) unsigned char in_smem[];
     __shared__ long long s_red[2];
     __shared__ uint32_t s_heads_full;                     // queues whose head entries are complete
@@ -165,6 +166,10 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
         for (uint32_t q = tid; q < R; q += kInThreads) qst[q].x = in_bin[(uint64_t)blockIdx.x * R + q];
     } else {
         for (uint32_t d = tid; d < n_dies * 6u; d += kInThreads) st_br_lo[d] = 0u;
+        if (blockIdx.x == 0) {                               // the first tile knows its entering state: it is served exactly
+            __syncthreads();
+            for (uint32_t q = tid; q < R; q += kInThreads) qst[q].x = busy[q];
+        }
     }
     unsigned long long c_native = 0, c_ready = 0, c_fault = 0;
     unsigned c_unsorted = 0;
@@ -427,7 +432,7 @@ k_inorder_fixup(uint32_t R, uint32_t n_tiles, BatchCtrl *ctrl, const int64_t *__
     if (idx < (uint64_t)n_tiles * R) {
         const uint32_t tile = (uint32_t)(idx / R);
         const uint32_t q = (uint32_t)(idx % R);
-        const uint32_t c = in_headcnt[idx];
+        const uint32_t c = tile == 0u ? 0u : in_headcnt[idx];       // the first tile was served from its true entering state
         int64_t B = in_bin[idx];                             // true busy-until of the queue entering the tile
         int64_t Bs = kNegInf;                                // busy-until of the as-if-idle run, to know what it wrote
         long long dstall = 0;
@@ -681,7 +686,7 @@ cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st) {
     InHead *heads = reinterpret_cast<InHead *>(a.ws.in_head);
     k_inorder_serve<false><<<n_tiles, kInThreads, smem_serve, st>>>(a.acc, n, tile_records, a.ranges, a.mp, a.fast, a.ctrl, a.status,
                                                                     a.ws.in_agg, a.stats_stage, a.completion, a.stall, a.ws.in_bin,
-                                                                    tiles, heads, a.ws.in_headcnt);
+                                                                    tiles, heads, a.ws.in_headcnt, a.busy);
     k_inorder_scan<<<(R + kInScanThreads - 1) / kInScanThreads, kInScanThreads, 0, st>>>(
         a.ctrl, a.mp_dev, n_tiles, a.ws.in_agg, a.ws.in_bin, a.busy, a.busy_stage, a.stats_stage, a.path == HBF_PATH_INORDER ? 1 : 0);
     const uint64_t fix_threads = (uint64_t)n_tiles * R;
@@ -691,7 +696,7 @@ cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st) {
                                                                 a.ws.in_headcnt, a.completion, a.stall, tiles);
     k_inorder_serve<true><<<n_tiles, kInThreads, smem_serve, st>>>(a.acc, n, tile_records, a.ranges, a.mp, a.fast, a.ctrl, a.status,
                                                                    a.ws.in_agg, a.stats_stage, a.completion, a.stall, a.ws.in_bin,
-                                                                   tiles, heads, a.ws.in_headcnt);
+                                                                   tiles, heads, a.ws.in_headcnt, a.busy);
     k_inorder_total<<<1, 256, 0, st>>>(a.ctrl, tiles, n_tiles);
     g_kernel_launches += 6;
     return cudaGetLastError();
