@@ -274,6 +274,18 @@ HBF_API int hbf_rom_reset(hbf_rom *rom);
 HBF_API int hbf_rom_step(hbf_rom *rom, const double *d_power, uint32_t n_steps, double *d_temps_out);
 HBF_API int hbf_rom_get_state(hbf_rom *rom, double *host_out, uint64_t cap);
 
+/* The paper's run-time configuration: the thermal step of a context on a reduced-order model instead of the grid.
+ * After hbf_attach_rom, hbf_thermal_step(ctx, dt_ns == the dt_ns given here, ...) forms the same power vector as
+ * before (window energy / dt + idle + external, one entry per floorplan region = one model input, so the model
+ * needs n_inputs == n_regions), advances the model by one step and runs the throttle controller on the hottest
+ * output of each medium: output_kind [n_outputs] (host, copied) gives HBF_KIND_HBF / HBF_KIND_HBM / HBF_KIND_GPU
+ * per model output.  hot_c_out reports those three maxima; d_temps_out must be NULL (the grid field is not
+ * advanced, HBF_E_INVAL otherwise).  The model must have been created on the context's stream; its state is the
+ * caller's to reset (hbf_rom_reset).  hbf_attach_rom(ctx, NULL, NULL, 0) goes back to the grid.
+ * hbf_get_rom_temps synchronises and copies the last step's outputs to host_out [n_outputs]. */
+HBF_API int hbf_attach_rom(hbf_ctx *ctx, hbf_rom *rom, const int32_t *output_kind, int64_t dt_ns);
+HBF_API int hbf_get_rom_temps(hbf_ctx *ctx, double *host_out, uint64_t cap);
+
 HBF_API const char *hbf_strerror(int code);
 
 #ifdef __cplusplus

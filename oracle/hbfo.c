@@ -837,3 +837,45 @@ int hbfo_rom_get_state(hbfo_rom *r, double *out, uint64_t cap) {
     memcpy(out, r->x, r->n * sizeof(double));
     return HBFO_OK;
 }
+
+/* ---- thermal step on the reduced-order model (the paper's run-time configuration: the service simulation runs on
+ * the fitted model, Section "Evaluation", not on the full operator).  Same power vector as hbfo_thermal_step
+ * (window energy / dt + idle + external, one entry per region), one step of the model, then the controller on the
+ * hottest output of each medium (output_kind[i] = HBFO_KIND_* of output i).  The grid field is not advanced. */
+int hbfo_thermal_step_rom(hbfo_ctx *c, hbfo_rom *r, const int32_t *output_kind, int64_t dt_ns, const float *ext_power_w,
+                          uint32_t n_ext, double hot_c_out[3]) {
+    if (!c || !c->thermal || !r || !output_kind || dt_ns <= 0 || r->m != c->cfg.n_regions) return HBFO_E_INVAL;
+    if (n_ext != 0 && (n_ext != c->cfg.n_regions || !ext_power_w)) return HBFO_E_INVAL;
+    const uint32_t NR = c->cfg.n_regions;
+    const double dt_s = (double)dt_ns * 1e-9;
+    if (c->bin_ns) {
+        if (dt_ns != c->bin_ns) return HBFO_E_INVAL;
+        int64_t *row = c->ledger + (size_t)(c->cur_bin % c->n_bins) * c->n_dies;
+        for (uint32_t d = 0; d < c->n_dies; ++d) { c->pending_pj[d] += row[d]; row[d] = 0; }
+        c->cur_bin += 1;
+    }
+    double *Pr = (double *)calloc(NR, sizeof(double)), *T = (double *)calloc(r->o, sizeof(double));
+    if (!Pr || !T) { free(Pr); free(T); return HBFO_E_NOMEM; }
+    for (uint32_t d = 0; d < c->n_dies; ++d)
+        Pr[c->die_region[d]] += ((double)c->pending_pj[d] * 1e-12) / dt_s;
+    for (uint32_t g = 0; g < NR; ++g) {
+        Pr[g] += c->region_idle_w[g];
+        if (n_ext) Pr[g] += (double)ext_power_w[g];
+    }
+    memset(c->pending_pj, 0, c->n_dies * sizeof(int64_t));
+    int rc = hbfo_rom_step(r, Pr, 1, T);
+    if (rc == HBFO_OK) {
+        double hot[3] = {-1e300, -1e300, -1e300};
+        for (uint32_t i = 0; i < r->o; ++i) {
+            int slot = output_kind[i] == HBFO_KIND_HBF ? 0 : output_kind[i] == HBFO_KIND_HBM ? 1 : output_kind[i] == HBFO_KIND_GPU ? 2 : -1;
+            if (slot >= 0 && T[i] > hot[slot]) hot[slot] = T[i];
+        }
+        for (int k = 0; k < 3; ++k) if (hot[k] == -1e300) hot[k] = (double)c->cfg.ambient_c;
+        c->mode = hbfo_next_mode(c, c->mode, hbfo_quantise_mk(hot[0]));
+        if (c->mode == HBFO_MODE_NORMAL) c->q_ppm = 1000000;
+        else if (c->mode == HBFO_MODE_LIGHT) c->q_ppm = c->cfg.q_light_ppm;
+        if (hot_c_out) { hot_c_out[0] = hot[0]; hot_c_out[1] = hot[1]; hot_c_out[2] = hot[2]; }
+    }
+    free(Pr); free(T);
+    return rc;
+}

@@ -128,6 +128,11 @@ int  hbfo_rom_reset(hbfo_rom *rom);
 int  hbfo_rom_step(hbfo_rom *rom, const double *power, uint32_t n_steps, double *temps_out);
 int  hbfo_rom_get_state(hbfo_rom *rom, double *out, uint64_t cap);
 
+/* One thermal step on the reduced-order model instead of the grid: the same power vector (one entry per region),
+ * one model step, the controller on the hottest output of each medium (output_kind[i] = HBFO_KIND_* of output i). */
+int  hbfo_thermal_step_rom(hbfo_ctx *ctx, hbfo_rom *rom, const int32_t *output_kind, int64_t dt_ns,
+                           const float *ext_power_w, uint32_t n_ext, double hot_c_out[3]);
+
 #ifdef __cplusplus
 }
 #endif

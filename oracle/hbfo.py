@@ -94,6 +94,7 @@ def lib():
         L.hbfo_enable_energy_bins.argtypes = [C.c_void_p, C.c_int64, C.c_uint32]
         L.hbfo_get_energy_bins.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.POINTER(C.c_int64)]
         L.hbfo_rom_create.argtypes = [C.c_uint32, C.c_uint32, C.c_uint32] + [C.c_void_p] * 6 + [C.POINTER(C.c_void_p)]
+        L.hbfo_thermal_step_rom.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_uint32, C.c_void_p]
         L.hbfo_rom_destroy.argtypes = [C.c_void_p]
         L.hbfo_rom_reset.argtypes = [C.c_void_p]
         L.hbfo_rom_step.argtypes = [C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p]
@@ -195,6 +196,20 @@ class Oracle:
         if check and rc != 0:
             raise OracleError(rc)
         return rc, comp, stall, status, ds
+
+    def thermal_step_rom(self, rom, output_kind, dt_ns, ext_power_w=None):
+        """One thermal step on the reduced-order model ``rom`` (a ``Rom``); returns hot[3]."""
+        hot = np.empty(3, np.float64)
+        kinds = np.ascontiguousarray(output_kind, np.int32)
+        if ext_power_w is None:
+            p, n = None, 0
+        else:
+            ext = np.ascontiguousarray(ext_power_w, np.float32)
+            p, n = ext.ctypes.data, ext.shape[0]
+        rc = lib().hbfo_thermal_step_rom(self._h, rom._h, kinds.ctypes.data, dt_ns, p, n, hot.ctypes.data)
+        if rc != 0:
+            raise OracleError(rc)
+        return hot
 
     def enable_channel_bus(self):
         rc = lib().hbfo_enable_channel_bus(self._h)

@@ -22,6 +22,7 @@ constexpr uint32_t kStateMagic = 0x48424631u;   // "HBF1"
 
 }  // namespace
 
+struct hbf_rom;
 struct hbf_ctx {
     hbf_config_t cfg{};
     cudaStream_t stream = nullptr;
@@ -36,6 +37,8 @@ struct hbf_ctx {
     BatchCtrl *d_ctrl = nullptr; hbf_batch_result_t *d_result = nullptr;
     int64_t *d_busy = nullptr, *d_busy_stage = nullptr, *d_pending = nullptr; hbf_die_stats_t *d_stats_stage = nullptr;
     hbf_batch_result_t *h_result = nullptr;      // pinned
+    // thermal steps on a reduced-order model instead of the grid (off while rom == nullptr)
+    hbf_rom *rom = nullptr; int64_t rom_dt_ns = 0; int32_t *d_rom_kind = nullptr; double *d_rom_p = nullptr, *d_rom_T = nullptr;
     // channel bus as a second queued stage (off while d_bus_busy == nullptr)
     int64_t *d_bus_busy = nullptr; BatchCtrl *d_bus_ctrl = nullptr;
     // time-bin energy ledger (off while bin_ns == 0)
@@ -149,6 +152,31 @@ int hbf_rom_get_state(hbf_rom *r, double *host_out, uint64_t cap) {
     return HBF_OK;
 }
 
+uint32_t hbf_rom_outputs(const hbf_rom *r) { return r ? r->o : 0u; }
+
+int hbf_attach_rom(hbf_ctx *c, hbf_rom *r, const int32_t *output_kind, int64_t dt_ns) {
+    if (!c || !c->thermal) return HBF_E_INVAL;
+    CK(cudaStreamSynchronize(c->stream));
+    if (!r) { c->rom = nullptr; return HBF_OK; }               // back to the grid
+    if (!output_kind || dt_ns <= 0 || r->m != c->td.n_regions || r->stream != c->stream) return HBF_E_INVAL;
+    if (c->d_rom_kind) { cudaFree(c->d_rom_kind); c->d_rom_kind = nullptr; }
+    if (c->d_rom_p) { cudaFree(c->d_rom_p); c->d_rom_p = nullptr; }
+    if (cudaMalloc(&c->d_rom_kind, r->o * sizeof(int32_t)) != cudaSuccess) return HBF_E_NOMEM;
+    if (cudaMalloc(&c->d_rom_p, ((size_t)r->m + r->o) * sizeof(double)) != cudaSuccess) return HBF_E_NOMEM;
+    c->d_rom_T = c->d_rom_p + r->m;
+    CK(cudaMemcpyAsync(c->d_rom_kind, output_kind, r->o * sizeof(int32_t), cudaMemcpyHostToDevice, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    c->rom = r; c->rom_dt_ns = dt_ns;
+    return HBF_OK;
+}
+
+int hbf_get_rom_temps(hbf_ctx *c, double *host_out, uint64_t cap) {
+    if (!c || !c->rom || !host_out || cap < c->rom->o) return HBF_E_INVAL;
+    CK(cudaMemcpyAsync(host_out, c->d_rom_T, c->rom->o * sizeof(double), cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    return HBF_OK;
+}
+
 const char *hbf_strerror(int code) {
     switch (code) {
     case HBF_OK: return "ok";
@@ -176,6 +204,8 @@ int hbf_destroy(hbf_ctx *c) {
     if (c->d_ledger) cudaFree(c->d_ledger);
     if (c->d_bus_busy) cudaFree(c->d_bus_busy);
     if (c->d_bus_ctrl) cudaFree(c->d_bus_ctrl);
+    if (c->d_rom_kind) cudaFree(c->d_rom_kind);
+    if (c->d_rom_p) cudaFree(c->d_rom_p);
     if (c->h_hot) cudaFreeHost(c->h_hot);
     if (c->h_ext) cudaFreeHost(c->h_ext);
     delete c;
@@ -512,7 +542,7 @@ int hbf_thermal_step(hbf_ctx *c, int64_t dt_ns, const float *ext_power_w, uint32
     if (!c || !c->thermal || dt_ns <= 0) return HBF_E_INVAL;
     if (n_ext != 0 && (n_ext != c->td.n_regions || !ext_power_w)) return HBF_E_INVAL;
     const double dt_sub = (double)dt_ns * 1e-9 / (double)c->td.n_sub;
-    if (dt_sub > c->euler_limit_s) return HBF_E_INVAL;
+    if (!c->rom && dt_sub > c->euler_limit_s) return HBF_E_INVAL;
     if (n_ext)      // pageable source: the runtime stages the bytes before returning, so the caller's array is free at once
         CK(cudaMemcpyAsync(c->td.ext_power, ext_power_w, n_ext * sizeof(float), cudaMemcpyHostToDevice, c->stream));
     if (c->bin_ns) {                                         // the step is the bin the thermal clock stands in
@@ -521,7 +551,14 @@ int hbf_thermal_step(hbf_ctx *c, int64_t dt_ns, const float *ext_power_w, uint32
         c->cur_bin += 1;
     }
     if (c->profiling) CK(cudaEventRecord(c->ev_th[0], c->stream));
-    CK(launch_thermal_step(c->td, c->d_state, c->d_pending, dt_ns, n_ext != 0, d_temps_out, &c->cur, c->thermal_generic ? 1 : 0, c->stream));
+    if (c->rom) {                                            // the attached model stands in for the grid
+        if (dt_ns != c->rom_dt_ns || d_temps_out) return HBF_E_INVAL;
+        CK(launch_rom_power(c->td, c->d_pending, dt_ns, n_ext != 0, c->d_rom_p, c->stream));
+        { const int rc_ = hbf_rom_step(c->rom, c->d_rom_p, 1, c->d_rom_T); if (rc_ != HBF_OK) return rc_; }
+        CK(launch_rom_controller(c->td, c->d_rom_T, c->d_rom_kind, hbf_rom_outputs(c->rom), c->d_state, c->stream));
+    } else {
+        CK(launch_thermal_step(c->td, c->d_state, c->d_pending, dt_ns, n_ext != 0, d_temps_out, &c->cur, c->thermal_generic ? 1 : 0, c->stream));
+    }
     if (c->profiling) { CK(cudaEventRecord(c->ev_th[1], c->stream)); c->prof_thermal = true; }
     if (hot_c_out) {
         CK(cudaMemcpyAsync(c->h_hot, c->td.hot, 3 * sizeof(float), cudaMemcpyDeviceToHost, c->stream));

@@ -176,4 +176,8 @@ struct ThermalDev {
 cudaError_t launch_thermal_step(const ThermalDev &t, DevState *state, int64_t *pending, int64_t dt_ns,
                                 int has_ext, float *d_temps_out, int *cur, int generic_only, cudaStream_t st);
 
+cudaError_t launch_rom_power(const ThermalDev &t, int64_t *pending, int64_t dt_ns, int has_ext, double *p_out, cudaStream_t st);
+cudaError_t launch_rom_controller(const ThermalDev &t, const double *temps, const int32_t *kind, uint32_t n_out, DevState *state,
+                                  cudaStream_t st);
+
 }  // namespace hbf

@@ -101,6 +101,58 @@ k_rom_steps_cluster(uint32_t n, uint32_t m, uint32_t o, uint32_t rpc, const doub
         for (uint32_t i = tid; i < n; i += kRomClusterThreads) x[i] = cur[i];
 }
 
+// ---- the thermal step of a context on a reduced-order model: power vector, one model step, controller --------
+// Power of each region over the window, as the grid's power map computes it (one thread per region walks its dies in
+// a fixed order): the model's input vector.  The window's energy is consumed.
+__global__ void k_rom_power(ThermalDev t, int64_t *pending, int64_t dt_ns, int has_ext, double *__restrict__ p_out) {
+    for (uint32_t g = threadIdx.x; g < t.n_regions; g += blockDim.x) {
+        double p = 0.0;
+        for (int32_t k = t.region_die_ptr[g]; k < t.region_die_ptr[g + 1]; ++k)
+            p += ((double)pending[t.region_die_list[k]] * 1e-12) / ((double)dt_ns * 1e-9);
+        p += (double)t.region_idle_w[g];
+        if (has_ext) p += (double)t.ext_power[g];
+        p_out[g] = p;
+    }
+    __syncthreads();
+    for (uint32_t d = threadIdx.x; d < t.n_dies; d += blockDim.x) pending[d] = 0;
+}
+
+__device__ __forceinline__ int rom_next_mode(const ThermalDev &t, int mode, long long mk) {
+    if (mode == HBF_MODE_SHUTDOWN || mk >= t.shut_mk) return HBF_MODE_SHUTDOWN;
+    if (mode == HBF_MODE_NORMAL) return mk >= t.stt_mk ? HBF_MODE_SEVERE : mk >= t.ltt_mk ? HBF_MODE_LIGHT : HBF_MODE_NORMAL;
+    if (mode == HBF_MODE_LIGHT) return mk >= t.stt_mk ? HBF_MODE_SEVERE : mk <= t.rtt_mk ? HBF_MODE_NORMAL : HBF_MODE_LIGHT;
+    return mk <= t.rtt_mk ? HBF_MODE_NORMAL : mk <= t.ltt_mk ? HBF_MODE_LIGHT : HBF_MODE_SEVERE;
+}
+
+// hottest output of each medium, the controller's transition on the HBF one (quantised to integer mK)
+__global__ void k_rom_controller(ThermalDev t, const double *__restrict__ temps, const int32_t *__restrict__ kind, uint32_t n_out,
+                                 DevState *state) {
+    if (threadIdx.x != 0) return;
+    double hot[3] = {-1e300, -1e300, -1e300};
+    for (uint32_t i = 0; i < n_out; ++i) {
+        const int slot = kind[i] == HBF_KIND_HBF ? 0 : kind[i] == HBF_KIND_HBM ? 1 : kind[i] == HBF_KIND_GPU ? 2 : -1;
+        if (slot >= 0 && temps[i] > hot[slot]) hot[slot] = temps[i];
+    }
+    for (int k = 0; k < 3; ++k) { if (hot[k] == -1e300) hot[k] = (double)t.ambient_c; t.hot[k] = (float)hot[k]; }
+    const int mode = rom_next_mode(t, state->mode, (long long)floor(hot[0] * 1000.0 + 0.5));
+    state->mode = mode;
+    if (mode == HBF_MODE_NORMAL) state->q_ppm = 1000000;
+    else if (mode == HBF_MODE_LIGHT) state->q_ppm = t.q_light_ppm;
+}
+
+cudaError_t launch_rom_power(const ThermalDev &t, int64_t *pending, int64_t dt_ns, int has_ext, double *p_out, cudaStream_t st) {
+    k_rom_power<<<1, 256, 0, st>>>(t, pending, dt_ns, has_ext, p_out);
+    g_kernel_launches += 1;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_rom_controller(const ThermalDev &t, const double *temps, const int32_t *kind, uint32_t n_out, DevState *state,
+                                  cudaStream_t st) {
+    k_rom_controller<<<1, 32, 0, st>>>(t, temps, kind, n_out, state);
+    g_kernel_launches += 1;
+    return cudaGetLastError();
+}
+
 static size_t rom_cluster_smem(uint32_t n, uint32_t m, uint32_t o, uint32_t *rpc_out) {
     const uint32_t rpc = (n + o + kRomClusterBlocks - 1) / kRomClusterBlocks;
     *rpc_out = rpc;

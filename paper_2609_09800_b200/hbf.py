@@ -31,7 +31,8 @@ EXPORTS = ("hbf_create", "hbf_destroy", "hbf_register_range", "hbf_clear_ranges"
            "hbf_set_profiling", "hbf_get_profile", "hbf_kernel_launches", "hbf_euler_substeps_static", "hbf_set_thermal_path",
            "hbf_workspace_bytes_paged", "hbf_submit_batch_paged",
            "hbf_enable_energy_bins", "hbf_get_energy_bins", "hbf_enable_channel_bus", "hbf_get_bus_busy_until",
-           "hbf_rom_create", "hbf_rom_destroy", "hbf_rom_reset", "hbf_rom_step", "hbf_rom_get_state")
+           "hbf_rom_create", "hbf_rom_destroy", "hbf_rom_reset", "hbf_rom_step", "hbf_rom_get_state",
+           "hbf_attach_rom", "hbf_get_rom_temps")
 STATIC_MAX_CELLS = 65536
 PROF_STAGES = ("begin", "classify", "plan_hist", "sort", "scan", "finish", "inorder", "thermal")
 
@@ -96,6 +97,8 @@ def lib():
         L.hbf_enable_energy_bins.argtypes = [vp, i64, u32]
         L.hbf_get_energy_bins.argtypes = [vp, vp, u64, C.POINTER(i64)]
         L.hbf_rom_create.argtypes = [u32, u32, u32, vp, vp, vp, vp, vp, vp, vp, C.POINTER(vp)]
+        L.hbf_attach_rom.argtypes = [vp, vp, vp, i64]
+        L.hbf_get_rom_temps.argtypes = [vp, vp, u64]
         L.hbf_rom_destroy.argtypes = [vp]
         L.hbf_rom_reset.argtypes = [vp]
         L.hbf_rom_step.argtypes = [vp, vp, u32, vp]
@@ -257,6 +260,25 @@ class Context:
         return lib().hbf_submit_batch_paged(self._h, _ptr(d_acc), n, parts_capacity, _ptr(d_completion), _ptr(d_stall),
                                             _ptr(d_status), _ptr(d_die_stats), _ptr(d_workspace),
                                             d_workspace.numel() * d_workspace.element_size())
+
+    def attach_rom(self, rom, output_kind=None, dt_ns=0):
+        """Thermal steps on a reduced-order model (a ``Rom`` created on this context's stream) instead of the grid;
+        ``attach_rom(None)`` goes back to the grid."""
+        if rom is None:
+            rc = lib().hbf_attach_rom(self._h, None, None, 0)
+        else:
+            kinds = np.ascontiguousarray(output_kind, np.int32)
+            rc = lib().hbf_attach_rom(self._h, rom._h, kinds.ctypes.data, dt_ns)
+        if rc != 0:
+            raise HbfError(rc, "hbf_attach_rom")
+        self._rom = rom                                       # keeps the model alive while it is attached
+
+    def get_rom_temps(self):
+        out = np.zeros(self._rom.o, np.float64)
+        rc = lib().hbf_get_rom_temps(self._h, out.ctypes.data, out.size)
+        if rc != 0:
+            raise HbfError(rc, "hbf_get_rom_temps")
+        return out
 
     def enable_channel_bus(self):
         rc = lib().hbf_enable_channel_bus(self._h)

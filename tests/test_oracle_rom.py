@@ -1,5 +1,6 @@
 """Pins of the oracle's reduced-order thermal model step (Eq. 2): closed forms and textbook special cases."""
 import numpy as np
+import pytest
 
 from oracle import hbfo
 
@@ -46,3 +47,31 @@ def test_steady_state_is_the_dc_gain_and_steps_chain():
     assert np.array_equal(T, T2)
     rom.reset()
     assert not rom.state().any()
+
+
+def test_thermal_step_on_the_model_uses_the_same_power_vector(golden_dir):
+    """A model that is pure feedthrough, T = ambient + R p, shows the power vector itself: the paper's read power,
+    384e9 B/s x 84 pJ/B + 5 W idle = 37.256 W, and the controller acting on the resulting temperature."""
+    import json, os
+    from paper_2609_09800_b200 import workloads as wl
+    with open(os.path.join(golden_dir, "paper_values.json")) as f:
+        pv = json.load(f)["hbf_read_power"]
+    prof = wl.load_profile("nominal", channels=16, dies=8, planes=1, page_bytes=16384, stripe_bytes=65536, n_sub=1)
+    prof.update(rtt_c=60.0, ltt_c=100.0, stt_c=120.0, shutdown_c=150.0)
+    fp = dict(grid_h=1, grid_w=1, cell_C=[1000.0], cell_Gx=[0.0], cell_Gy=[0.0], cell_Gsink=[1.0], cell_region=[0],
+              die_region=[0] * 128, region_kind=[wl.KIND_HBF], region_idle_w=[pv["idle_w"]])
+    o = hbfo.Oracle(prof, fp)
+    o.register_range(wl.RANGE_BASE, 1 << 40)
+    n = int(pv["bytes_per_s"]) // 65536
+    acc = np.zeros(n, hbfo.ACCESS_DTYPE)
+    acc["addr"] = wl.RANGE_BASE + np.arange(n, dtype=np.uint64) * np.uint64(65536)
+    acc["bytes"] = 65536
+    o.submit(acc)
+    rom = hbfo.Rom(np.zeros((1, 1)), np.zeros((1, 1)), np.zeros((1, 1)), D=[[2.0]], d=[prof["ambient_c"]])   # 2 K/W
+    hot = o.thermal_step_rom(rom, [wl.KIND_HBF], 1_000_000_000)
+    assert hot[0] - prof["ambient_c"] == pytest.approx(2.0 * pv["power_w"], abs=1e-9)
+    assert not o.pending_energy().any()
+    assert o.mode()[0] == hbfo.MODE_LIGHT              # 35 + 74.5 = 109.5 C: above the light threshold, below severe
+    hot = o.thermal_step_rom(rom, [wl.KIND_HBF], 1_000_000_000)    # no traffic any more: idle power only, 35 + 10 C
+    assert hot[0] - prof["ambient_c"] == pytest.approx(2.0 * pv["idle_w"], abs=1e-12)
+    assert o.mode()[0] == hbfo.MODE_NORMAL             # back below the release threshold
