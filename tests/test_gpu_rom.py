@@ -75,3 +75,44 @@ def test_model_fitted_from_the_cuda_grid_tracks_the_oracle_grid(hbf):
     for _ in range(6000):
         hot, T = o.thermal_step(dt, p1, want_temps=True)
     assert np.abs(era.dc_gain(fit)[:, 2] - (T[probes] - prof["ambient_c"])).max() < 5e-3 * (T[probes].max() - prof["ambient_c"])
+
+
+def test_context_steps_on_an_attached_model(hbf):
+    """Coupled run with the thermal step on a reduced-order model: hot spots within 1e-9 K of the oracle's (double on
+    both sides), the mode / service-fraction trace and every completion equal."""
+    w = wl.prefix_kv(epochs=1, steps=1, batch=4, kv_tokens=256, layers=2)
+    fp = wl.package_floorplan()
+    prof = dict(w.profile); prof.update(rtt_c=36.0, ltt_c=36.6, stt_c=60.0, shutdown_c=90.0)   # thresholds the run crosses
+    g, o = hbf.Context(prof, fp), hbfo.Oracle(prof, fp)
+    for r in w.ranges:
+        g.register_range(*r); o.register_range(*r)
+    m = len(fp["region_kind"])
+    rng = np.random.default_rng(5)
+    n, no = 40, 9
+    A = np.diag(rng.uniform(0.80, 0.97, n))
+    B = rng.uniform(0.0, 0.02, size=(n, m)); C = rng.uniform(0.0, 0.05, size=(no, n)); D = rng.uniform(0.0, 0.002, size=(no, m))
+    kinds = np.array([wl.KIND_HBF, wl.KIND_HBF, wl.KIND_HBF, wl.KIND_HBM, wl.KIND_HBM, wl.KIND_GPU, wl.KIND_GPU, wl.KIND_NONE, wl.KIND_HBF], np.int32)
+    d = np.full(no, prof["ambient_c"])
+    rg, ro = hbf.Rom(A, B, C, D=D, d=d, stream=g.stream), hbfo.Rom(A, B, C, D=D, d=d)
+    dt = 1_000_000
+    g.attach_rom(rg, kinds, dt)
+    ext = fp["ext_power_w"]
+    modes = set()
+    for _, batch in wl.timed_batches(w, 14_000_000):
+        rc_g, c_g, s_g, _, _ = g.submit_host(batch, check=False)
+        rc_o, c_o, s_o, _, _ = o.submit(batch, check=False)
+        assert rc_g == rc_o
+        if rc_o == 0:
+            assert np.array_equal(c_g, c_o) and np.array_equal(s_g, s_o)
+        hot_g = g.thermal_step(dt, ext)
+        hot_o = o.thermal_step_rom(ro, kinds, dt, ext)
+        assert np.abs(hot_g.astype(np.float64) - hot_o).max() < 1e-4      # hot_c_out is float32
+        assert np.abs(g.get_rom_temps()[kinds != wl.KIND_NONE].max() - hot_o.max()) < 1e-9
+        assert g.get_mode() == o.mode()
+        modes.add(o.mode()[0])
+    assert len(modes) >= 2                                                 # the trace does leave Normal
+    assert np.abs(rg.state() - ro.state()).max() < 1e-9
+    with pytest.raises(hbf.HbfError):
+        g.thermal_step(2 * dt, ext)                                        # the model was fitted for one step length
+    g.attach_rom(None)
+    g.thermal_step(dt, ext)                                                # the grid again
