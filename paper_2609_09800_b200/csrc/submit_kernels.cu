@@ -839,8 +839,10 @@ k_bus_apply(const hbf_access_t *__restrict__ acc, BatchCtrl *bc, const uint64_t 
             if (j >= m) break;
             run = bus_then(run, e[u]);
             const int64_t done = run.M;
-            completion[idx[u]] = done; stall[idx[u]] = done - acc[idx[u]].issue_ns;
-            moved += done - plain[u]; max_c = max(max_c, (long long)done);
+            if (done != plain[u]) {                          // the transfer waited for the bus: completion and stall move by the wait
+                completion[idx[u]] = done; stall[idx[u]] += done - plain[u];
+                moved += done - plain[u]; max_c = max(max_c, (long long)done);
+            }
         }
     }
     moved = warp_sum(moved); max_c = warp_max(max_c);
