@@ -144,8 +144,8 @@ k_paged_expand(const hbf_access_t *__restrict__ acc, uint64_t n, const RangeSnap
 struct PagedSums { unsigned long long n_ready, stall_sum; };
 
 __global__ void __launch_bounds__(256)
-k_paged_join(const hbf_access_t *__restrict__ acc, uint64_t n, const uint32_t *__restrict__ part_first,
-             const int64_t *__restrict__ part_completion, const uint8_t *__restrict__ part_status,
+k_paged_join(uint64_t n, const uint32_t *__restrict__ part_first, const int64_t *__restrict__ part_completion,
+             const int64_t *__restrict__ part_stall, const uint8_t *__restrict__ part_status,
              const hbf_batch_result_t *__restrict__ result, int64_t *__restrict__ completion, int64_t *__restrict__ stall,
              uint8_t *__restrict__ status, PagedSums *sums) {
     const bool served = result->code == HBF_OK;
@@ -159,7 +159,8 @@ k_paged_join(const hbf_access_t *__restrict__ acc, uint64_t n, const uint32_t *_
         if (served) {
             done = part_completion[lo];
             for (uint32_t k = lo + 1; k < hi; ++k) done = max(done, part_completion[k]);
-            if (st == HBF_ST_READY) { waited = done - acc[i].issue_ns; ++ready; stall_sum += waited; }
+            // every part carries the access's issue time: completion - stall of the first part gives it back
+            if (st == HBF_ST_READY) { waited = done - (part_completion[lo] - part_stall[lo]); ++ready; stall_sum += waited; }
         }
         completion[i] = done; stall[i] = waited;
     }
@@ -216,7 +217,7 @@ cudaError_t launch_paged_expand(const hbf_access_t *acc, uint64_t n, const Range
 cudaError_t launch_paged_join(const hbf_access_t *acc, uint64_t n, const PagedWorkspace &pw, hbf_batch_result_t *result,
                               int64_t *completion, int64_t *stall, uint8_t *status, int sm_count, cudaStream_t st) {
     const unsigned grid = (unsigned)std::min<uint64_t>((n + 255) / 256, (uint64_t)std::max(1, sm_count) * 8);
-    k_paged_join<<<grid, 256, 0, st>>>(acc, n, pw.part_first, pw.part_completion, pw.part_status, result, completion, stall, status,
+    k_paged_join<<<grid, 256, 0, st>>>(n, pw.part_first, pw.part_completion, pw.part_stall, pw.part_status, result, completion, stall, status,
                                       reinterpret_cast<PagedSums *>(pw.sums));
     k_paged_finish<<<1, 1, 0, st>>>(result, reinterpret_cast<const PagedSums *>(pw.sums));
     g_kernel_launches += 2;
