@@ -81,3 +81,38 @@ def test_full_size_batch_against_per_queue_oracle(full, path):
             assert bad.size == 0, (path, step, q, int(idx[bad[0]]), int(comp[idx][bad[0]]), int(c_o[bad[0]]))
             assert int(busy[q]) == int(oracles[q].busy_until()[q])
     ctx.destroy()
+
+
+@pytest.mark.parametrize("which", ["decode_weights", "prefix_kv"])
+def test_serving_configurations_at_full_size_element_by_element(which):
+    """The 21 M-access decode-weight stream and the 28 M-access prefix-KV stream (the two serving configurations),
+    device-resident and in one batch each as the bench would submit them: the oracle serves them whole in a few
+    seconds, so every completion, stall, status, per-die statistic and queue state is compared; then the same batch
+    again on the queues it left backlogged."""
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2609_09800_b200 import build, hbf
+    build.build()
+    w = wl.decode_weights() if which == "decode_weights" else wl.prefix_kv()
+    g, o = hbf.Context(w.profile), hbfo.Oracle(w.profile)
+    for r in w.ranges:
+        g.register_range(*r); o.register_range(*r)
+    n = w.n
+    d_acc = torch.from_numpy(w.acc.view(np.int64).reshape(-1)).cuda()
+    d_comp = torch.empty(n, dtype=torch.int64, device="cuda"); d_stall = torch.empty_like(d_comp)
+    d_status = torch.empty(n, dtype=torch.uint8, device="cuda")
+    d_ds = torch.empty(g.n_dies * 6, dtype=torch.int64, device="cuda")
+    ws = g.workspace(n)
+    for _ in range(2):
+        assert g.submit_batch(d_acc, n, d_comp, d_stall, d_status, d_ds, ws) == 0
+        _, c_o, s_o, st_o, ds_o = o.submit(w.acc)
+        assert g.last_result() == o.last_result()
+        c_g = d_comp.cpu().numpy()
+        bad = np.flatnonzero(c_g != c_o)
+        assert bad.size == 0, "first mismatch at %d: gpu %d oracle %d (%d mismatches)" % (bad[0], c_g[bad[0]], c_o[bad[0]], bad.size)
+        assert np.array_equal(d_stall.cpu().numpy(), s_o) and np.array_equal(d_status.cpu().numpy(), st_o)
+        ds_g = d_ds.cpu().numpy().view(hbf.DIE_STATS_DTYPE)
+        for k in hbfo.DIE_STATS_DTYPE.names:
+            assert np.array_equal(ds_g[k], ds_o[k]), k
+        assert np.array_equal(g.get_busy_until(), o.busy_until())
