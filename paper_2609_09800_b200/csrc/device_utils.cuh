@@ -27,36 +27,6 @@ __device__ __forceinline__ uint64_t ld_nc_u64(const uint64_t *p) {
     uint64_t v; asm volatile("ld.global.nc.u64 %0, [%1];" : "=l"(v) : "l"(p)); return v;
 }
 
-// ---- bulk asynchronous copies (TMA, one-dimensional) and their mbarrier ------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-    return ok != 0u;
-}
-// Waits for the phase with the given parity; gives up after a bounded number of polls.
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity) {
-    for (uint32_t spins = 0; spins < (1u << 22); ++spins) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (spins > 64u) __nanosleep(64);
-    }
-    return false;
-}
-// global -> shared, bytes a multiple of 16, both addresses 16-byte aligned; completion counts on the mbarrier
-__device__ __forceinline__ void bulk_load(void *smem_dst, const void *gmem_src, uint32_t bytes, uint64_t *bar) {
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // earlier generic accesses to the buffer come first
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(smem_u32(smem_dst)), "l"(gmem_src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
-}
-
 // ---- division by a run-time constant ----------------------------------------------------------------
 // For d not a power of two, l = ceil(log2 d), magic = floor(2^(63+l) / d) + 1: floor(n / d) =
 // mulhi(n, magic) >> (l - 1) for every n < 2^63 (the error term n * (magic*d - 2^(63+l)) stays below 2^(63+l)).
