@@ -35,6 +35,7 @@ struct hbfo_ctx {
     int32_t *cell_region, *die_region, *region_kind;
     double *region_idle_w, *region_cells;
     double euler_limit_s;
+    struct hbfo_retention *ret;   /* retention, refresh and wear (off while NULL) */
 };
 
 /* ---- small helpers ---------------------------------------------------------------------- */
@@ -74,8 +75,11 @@ const char *hbfo_strerror(int code) {
 
 /* ---- create / destroy --------------------------------------------------------------------- */
 
+static void free_retention(struct hbfo_retention *r);
+
 static void free_ctx(hbfo_ctx *c) {
     if (!c) return;
+    free_retention(c->ret);
     free(c->busy_until); free(c->pending_pj); free(c->order); free(c->ledger); free(c->bus_busy);
     free(c->C); free(c->Gx); free(c->Gy); free(c->Gs); free(c->T); free(c->Tn); free(c->P);
     free(c->cell_region); free(c->die_region); free(c->region_kind);
@@ -163,6 +167,8 @@ int hbfo_destroy(hbfo_ctx *ctx) { free_ctx(ctx); return HBFO_OK; }
 
 double hbfo_euler_limit_ns(hbfo_ctx *ctx) { return ctx && ctx->thermal ? ctx->euler_limit_s * 1e9 : 0.0; }
 
+static void retention_reset(struct hbfo_retention *r);
+
 int hbfo_reset(hbfo_ctx *c) {
     if (!c) return HBFO_E_INVAL;
     memset(c->busy_until, 0, c->n_queues * sizeof(int64_t));
@@ -174,6 +180,7 @@ int hbfo_reset(hbfo_ctx *c) {
     if (c->bus_busy) memset(c->bus_busy, 0, c->cfg.channels * sizeof(int64_t));
     if (c->ledger) memset(c->ledger, 0, (size_t)c->n_bins * c->n_dies * sizeof(int64_t));
     if (c->thermal) for (size_t i = 0; i < c->n_cells; ++i) c->T[i] = (double)c->cfg.ambient_c;
+    retention_reset(c->ret);
     return HBFO_OK;
 }
 
@@ -282,7 +289,7 @@ int hbfo_service_terms(hbfo_ctx *c, uint32_t bytes, uint64_t npages, uint32_t op
  * of n_bins bins starting at the bin the thermal clock stands in: time before it counts into that bin, time
  * past the ring's end into the ring's last bin. */
 int hbfo_enable_energy_bins(hbfo_ctx *c, int64_t bin_ns, uint32_t n_bins) {
-    if (!c || bin_ns <= 0 || n_bins == 0) return HBFO_E_INVAL;
+    if (!c || bin_ns <= 0 || n_bins == 0 || c->ret) return HBFO_E_INVAL;
     int64_t *l = (int64_t *)calloc((size_t)n_bins * c->n_dies, sizeof(int64_t));
     if (!l) return HBFO_E_NOMEM;
     free(c->ledger);
@@ -327,7 +334,7 @@ static void ledger_event(hbfo_ctx *c, uint32_t die, int64_t start, int64_t s, in
  * (D, batch index) order behind whatever earlier batches left on that bus, and occupies it for the transfer time.
  * The read completes when its transfer does.  Programs keep their transfer as a latency before the array time. */
 int hbfo_enable_channel_bus(hbfo_ctx *c) {
-    if (!c) return HBFO_E_INVAL;
+    if (!c || c->ret) return HBFO_E_INVAL;
     if (!c->bus_busy) c->bus_busy = (int64_t *)calloc(c->cfg.channels, sizeof(int64_t));
     return c->bus_busy ? HBFO_OK : HBFO_E_NOMEM;
 }
@@ -345,6 +352,234 @@ static int cmp_bent(const void *pa, const void *pb) {
     if (a->done_ns != b->done_ns) return a->done_ns < b->done_ns ? -1 : 1;
     if (a->idx != b->idx) return a->idx < b->idx ? -1 : 1;
     return 0;
+}
+
+/* ---- retention, refresh and wear (Design D4) --------------------------------------------------------
+ * What the paper fixes: every registered block carries retention damage, a read-disturb count, a zone, and a
+ * current and a maximum program/erase count; the retention lifetime follows the Arrhenius equation anchored at a
+ * reference condition, L(T) = L_ref * exp[(E_a / k_B) * (1/T - 1/T_ref)] (first equation of D4, E_a = 1.04 eV in
+ * the evaluation); damage accumulates as D <- D + a_t * dt / L(T) (second equation of D4); a block becomes
+ * eligible at its lead threshold or its read-disturb limit; the scheduler emits page-aligned read-rewrite pairs in
+ * the order eligibility epoch, channel round robin, die round robin, zone, block, page; the plan is published as a
+ * debt of which every admission claims at most one quantum and reserves that quantum's thermally scaled service
+ * before its own; a block commits one program/erase cycle and clears its damage and disturb counters only after
+ * all of its quanta are done; idle time drains debt on a separate account.
+ * What is a reading (the paper gives no numbers or layouts for these): a block is pages_per_block consecutive
+ * pages of one plane, block = (page / pages_per_block) mod blocks_per_plane, zone = block / blocks_per_zone; a
+ * read adds its page count to the disturb counter of the block of its first page, programs add nothing; damage
+ * and eligibility are evaluated by hbfo_retention_advance, once per call (= one epoch), with one temperature per
+ * floorplan region (given, or the hottest cell of the region in the field); within a die, blocks are ordered by
+ * (zone, plane, block); a quantum is one page, read and rewritten: t_read + t_prog of array time, scaled like any
+ * service (Eq. 3), charged on the claiming access's own queue and die, its energy booked on that die; the modeled
+ * accesses of a batch claim in index (ticket) order; commits take effect when the batch (or the decay) that
+ * claimed a block's last quantum has completed; idle time drains one quantum per scaled quantum time. */
+#define HBFO_KB_EV 8.617333262e-5                  /* Boltzmann constant, eV/K */
+
+struct hbfo_retention {
+    hbfo_retention_config_t cfg;
+    uint64_t n_blocks;
+    double *damage; uint32_t *disturb, *pec, *epoch_of; uint8_t *worn;
+    uint64_t *last_pos;          /* plan position of the block's last quantum */
+    uint32_t *plan; uint64_t plan_len, plan_cap;
+    uint64_t claimed, decayed, commits, worn_blocks;
+    uint32_t epoch;
+};
+
+static void free_retention(struct hbfo_retention *r) {
+    if (!r) return;
+    free(r->damage); free(r->disturb); free(r->pec); free(r->epoch_of); free(r->worn); free(r->last_pos); free(r->plan);
+    free(r);
+}
+
+static void retention_reset(struct hbfo_retention *r) {
+    if (!r) return;
+    memset(r->damage, 0, r->n_blocks * sizeof(double)); memset(r->disturb, 0, r->n_blocks * 4);
+    memset(r->pec, 0, r->n_blocks * 4); memset(r->epoch_of, 0, r->n_blocks * 4); memset(r->worn, 0, r->n_blocks);
+    r->plan_len = 0; r->claimed = r->decayed = r->commits = r->worn_blocks = 0; r->epoch = 0;
+}
+
+int hbfo_enable_retention(hbfo_ctx *c, const hbfo_retention_config_t *cfg) {
+    if (!c || !cfg || c->ret || c->bin_ns || c->bus_busy) return HBFO_E_INVAL;
+    if (cfg->pages_per_block == 0 || cfg->blocks_per_plane == 0 || cfg->blocks_per_zone == 0 ||
+        cfg->blocks_per_plane % cfg->blocks_per_zone != 0 || cfg->max_pec == 0) return HBFO_E_INVAL;
+    if (!(cfg->l_ref_s > 0.0) || !(cfg->t_ref_c > -273.15) || !(cfg->ea_ev >= 0.0) || !(cfg->accel > 0.0) ||
+        !(cfg->lead_threshold > 0.0)) return HBFO_E_INVAL;
+    const uint64_t nb = (uint64_t)c->cfg.channels * c->cfg.dies * c->cfg.planes * cfg->blocks_per_plane;
+    if (nb * cfg->pages_per_block > 0xffffffffull) return HBFO_E_INVAL;
+    struct hbfo_retention *r = (struct hbfo_retention *)calloc(1, sizeof(*r));
+    if (!r) return HBFO_E_NOMEM;
+    r->cfg = *cfg; r->n_blocks = nb;
+    r->damage = (double *)calloc(nb, sizeof(double)); r->disturb = (uint32_t *)calloc(nb, 4);
+    r->pec = (uint32_t *)calloc(nb, 4); r->epoch_of = (uint32_t *)calloc(nb, 4); r->worn = (uint8_t *)calloc(nb, 1);
+    r->last_pos = (uint64_t *)calloc(nb, 8);
+    if (!r->damage || !r->disturb || !r->pec || !r->epoch_of || !r->worn || !r->last_pos) { free_retention(r); return HBFO_E_NOMEM; }
+    c->ret = r;
+    return HBFO_OK;
+}
+
+double hbfo_retention_lifetime_s(hbfo_ctx *c, double temp_c) {
+    if (!c || !c->ret) return 0.0;
+    const hbfo_retention_config_t *k = &c->ret->cfg;
+    const double T = temp_c + 273.15, Tref = k->t_ref_c + 273.15;
+    return k->l_ref_s * exp((k->ea_ev / HBFO_KB_EV) * (1.0 / T - 1.0 / Tref));
+}
+
+/* the block an access's first page lies in: ((channel, die, plane) * blocks_per_plane + block) */
+static uint64_t retention_block_of(hbfo_ctx *c, uint64_t off) {
+    uint32_t ch, di, pl; uint64_t page;
+    hbfo_decode(c, off, 1, &ch, &di, &pl, NULL, &page, NULL, NULL);
+    const struct hbfo_retention *r = c->ret;
+    const uint64_t bip = (page / r->cfg.pages_per_block) % r->cfg.blocks_per_plane;
+    return (((uint64_t)ch * c->cfg.dies + di) * c->cfg.planes + pl) * r->cfg.blocks_per_plane + bip;
+}
+
+/* blocks whose last quantum lies below the watermark commit: one cycle, counters cleared */
+static void retention_commit(struct hbfo_retention *r) {
+    const uint64_t mark = r->claimed + r->decayed;
+    for (uint64_t b = 0; b < r->n_blocks; ++b) {
+        if (r->epoch_of[b] == 0 || r->last_pos[b] >= mark) continue;
+        r->pec[b] += 1; r->damage[b] = 0.0; r->disturb[b] = 0; r->epoch_of[b] = 0; r->commits += 1;
+        if (r->pec[b] >= r->cfg.max_pec) { r->worn[b] = 1; r->worn_blocks += 1; }
+    }
+}
+
+static int retention_plan_push(struct hbfo_retention *r, uint32_t quantum) {
+    if (r->plan_len == r->plan_cap) {
+        uint64_t cap = r->plan_cap ? r->plan_cap * 2 : 1024;
+        uint32_t *p = (uint32_t *)realloc(r->plan, cap * 4);
+        if (!p) return HBFO_E_NOMEM;
+        r->plan = p; r->plan_cap = cap;
+    }
+    r->plan[r->plan_len++] = quantum;
+    return HBFO_OK;
+}
+
+int hbfo_retention_advance(hbfo_ctx *c, int64_t dt_ns, const double *region_temp_c) {
+    if (!c || !c->ret || dt_ns < 0) return HBFO_E_INVAL;
+    struct hbfo_retention *r = c->ret;
+    const uint32_t NR = c->thermal ? c->cfg.n_regions : 1;
+    if (!region_temp_c && !c->thermal) return HBFO_E_INVAL;
+    double *temp = (double *)malloc(NR * sizeof(double));
+    if (!temp) return HBFO_E_NOMEM;
+    if (region_temp_c) memcpy(temp, region_temp_c, NR * sizeof(double));
+    else {                                                     /* the hottest cell of each region */
+        for (uint32_t k = 0; k < NR; ++k) temp[k] = -INFINITY;
+        for (size_t i = 0; i < c->n_cells; ++i) {
+            int32_t g = c->cell_region[i];
+            if (g >= 0 && c->T[i] > temp[g]) temp[g] = c->T[i];
+        }
+        for (uint32_t k = 0; k < NR; ++k) if (temp[k] == -INFINITY) temp[k] = (double)c->cfg.ambient_c;
+    }
+    r->epoch += 1;
+    const uint32_t Cn = c->cfg.channels, Dn = c->cfg.dies, Pn = c->cfg.planes;
+    const uint32_t bpp = r->cfg.blocks_per_plane, bpz = r->cfg.blocks_per_zone, ppb = r->cfg.pages_per_block;
+    const double dt_s = (double)dt_ns * 1e-9;
+    /* damage, then eligibility */
+    for (uint64_t b = 0; b < r->n_blocks; ++b) {
+        if (r->worn[b]) continue;
+        const uint64_t die = b / ((uint64_t)Pn * bpp);
+        const uint32_t g = c->thermal ? (uint32_t)c->die_region[die] : 0u;
+        r->damage[b] += r->cfg.accel * dt_s / hbfo_retention_lifetime_s(c, temp[g]);
+        if (r->epoch_of[b] == 0 && (r->damage[b] >= r->cfg.lead_threshold ||
+                                    (r->cfg.disturb_limit && r->disturb[b] >= r->cfg.disturb_limit)))
+            r->epoch_of[b] = r->epoch;
+    }
+    free(temp);
+    /* this epoch's quanta: per die in (zone, plane, block, page) order ... */
+    const uint32_t n_dies = Cn * Dn;
+    uint32_t **list = (uint32_t **)calloc(n_dies, sizeof(uint32_t *));
+    uint64_t *len = (uint64_t *)calloc(n_dies, 8), *pos = (uint64_t *)calloc(n_dies, 8);
+    uint32_t *die_ptr = (uint32_t *)calloc(Cn, 4);
+    int rc = HBFO_OK;
+    uint64_t remaining = 0;
+    if (!list || !len || !pos || !die_ptr) { rc = HBFO_E_NOMEM; goto done; }
+    for (uint32_t d = 0; d < n_dies; ++d) {
+        uint64_t cnt = 0;
+        for (uint32_t pl = 0; pl < Pn; ++pl)
+            for (uint32_t k = 0; k < bpp; ++k)
+                if (r->epoch_of[((uint64_t)d * Pn + pl) * bpp + k] == r->epoch) ++cnt;
+        if (!cnt) continue;
+        list[d] = (uint32_t *)malloc(cnt * ppb * 4);
+        if (!list[d]) { rc = HBFO_E_NOMEM; goto done; }
+        for (uint32_t z = 0; z < bpp / bpz; ++z)
+            for (uint32_t pl = 0; pl < Pn; ++pl)
+                for (uint32_t k = z * bpz; k < (z + 1) * bpz; ++k) {
+                    const uint64_t b = ((uint64_t)d * Pn + pl) * bpp + k;
+                    if (r->epoch_of[b] != r->epoch) continue;
+                    for (uint32_t pg = 0; pg < ppb; ++pg) list[d][len[d]++] = (uint32_t)(b * ppb + pg);
+                }
+        remaining += len[d];
+    }
+    /* ... emitted one at a time: channels in turn, within a channel its dies in turn, skipping what is exhausted */
+    for (uint32_t ch = 0; remaining; ch = (ch + 1) % Cn) {
+        int left = 0;
+        for (uint32_t di = 0; di < Dn; ++di) if (pos[ch * Dn + di] < len[ch * Dn + di]) left = 1;
+        if (!left) continue;
+        uint32_t di = die_ptr[ch];
+        while (pos[ch * Dn + di] >= len[ch * Dn + di]) di = (di + 1) % Dn;
+        const uint32_t d = ch * Dn + di;
+        const uint32_t quantum = list[d][pos[d]++];
+        r->last_pos[quantum / ppb] = r->plan_len;            /* pages go out in order: the last one stays */
+        rc = retention_plan_push(r, quantum);
+        if (rc != HBFO_OK) goto done;
+        die_ptr[ch] = (di + 1) % Dn;
+        --remaining;
+    }
+done:
+    if (list) for (uint32_t d = 0; d < n_dies; ++d) free(list[d]);
+    free(list); free(len); free(pos); free(die_ptr);
+    return rc;
+}
+
+/* scaled array time of one quantum: a page read and a page program (Eq. 3) */
+static int64_t retention_quantum_ns(hbfo_ctx *c, int64_t q_ppm) {
+    return ceil_div_i64((c->cfg.t_read_ns + c->cfg.t_prog_ns) * 1000000, q_ppm);
+}
+static int64_t retention_quantum_pj(hbfo_ctx *c) {
+    const int64_t pg = (int64_t)c->cfg.page_bytes;
+    return c->cfg.e_cmd_read_pj + c->cfg.e_byte_read_pj * pg + c->cfg.e_cmd_prog_pj + c->cfg.e_byte_prog_pj * pg;
+}
+
+int hbfo_retention_decay(hbfo_ctx *c, int64_t idle_ns) {
+    if (!c || !c->ret || idle_ns < 0) return HBFO_E_INVAL;
+    struct hbfo_retention *r = c->ret;
+    uint64_t drained = (uint64_t)(idle_ns / retention_quantum_ns(c, c->q_ppm));
+    const uint64_t debt = r->plan_len - (r->claimed + r->decayed);
+    if (drained > debt) drained = debt;
+    r->decayed += drained;
+    retention_commit(r);
+    return HBFO_OK;
+}
+
+int hbfo_get_retention_blocks(hbfo_ctx *c, double *damage, uint32_t *disturb, uint32_t *pec, uint32_t *epoch, uint64_t cap) {
+    if (!c || !c->ret || cap < c->ret->n_blocks) return HBFO_E_INVAL;
+    const struct hbfo_retention *r = c->ret;
+    if (damage) memcpy(damage, r->damage, r->n_blocks * 8);
+    if (disturb) memcpy(disturb, r->disturb, r->n_blocks * 4);
+    if (pec) memcpy(pec, r->pec, r->n_blocks * 4);
+    if (epoch) memcpy(epoch, r->epoch_of, r->n_blocks * 4);
+    return HBFO_OK;
+}
+
+int hbfo_get_retention_plan(hbfo_ctx *c, uint32_t *quanta, uint64_t cap, uint64_t *count) {
+    if (!c || !c->ret || !count) return HBFO_E_INVAL;
+    const struct hbfo_retention *r = c->ret;
+    const uint64_t mark = r->claimed + r->decayed, m = r->plan_len - mark;
+    *count = m;
+    if (!quanta) return HBFO_OK;
+    if (cap < m) return HBFO_E_INVAL;
+    memcpy(quanta, r->plan + mark, m * 4);
+    return HBFO_OK;
+}
+
+int hbfo_get_retention_totals(hbfo_ctx *c, hbfo_retention_totals_t *out) {
+    if (!c || !c->ret || !out) return HBFO_E_INVAL;
+    const struct hbfo_retention *r = c->ret;
+    out->planned = r->plan_len; out->claimed = r->claimed; out->decayed = r->decayed; out->commits = r->commits;
+    out->worn_blocks = r->worn_blocks; out->epoch = r->epoch; out->n_blocks = r->n_blocks;
+    out->waiting_blocks = 0;
+    for (uint64_t b = 0; b < r->n_blocks; ++b) if (r->epoch_of[b]) out->waiting_blocks += 1;
+    return HBFO_OK;
 }
 
 /* ---- submit --------------------------------------------------------------------------------- */
@@ -397,6 +632,7 @@ int hbfo_submit_batch(hbfo_ctx *c, const hbfo_access_t *acc, uint64_t n, int64_t
     uint64_t *cnt = (uint64_t *)calloc((size_t)c->n_queues + 1, sizeof(uint64_t));
     qent_t *ent = (qent_t *)malloc((n_ready ? n_ready : 1) * sizeof(qent_t));
     int rc = HBFO_OK;
+    uint64_t claims = 0;                                      /* refresh quanta claimed by this batch */
     if (!queue || !die || !a_ns || !s_ns || !post || !cbs || !eng || !cnt || !ent) { rc = HBFO_E_NOMEM; goto done; }
     if (c->order_cap < n_ready) {
         free(c->order); c->order = (uint32_t *)malloc((n_ready ? n_ready : 1) * sizeof(uint32_t));
@@ -414,6 +650,13 @@ int hbfo_submit_batch(hbfo_ctx *c, const hbfo_access_t *acc, uint64_t n, int64_t
         int64_t cb, xfer, s, e;
         hbfo_service_terms(c, acc[i].bytes, np, op, q, &cb, &xfer, &s, &e);
         queue[i] = qu; die[i] = ch * c->cfg.dies + di;
+        if (c->ret && c->ret->claimed + c->ret->decayed + claims < c->ret->plan_len) {
+            /* this admission claims one refresh quantum: its scaled service is reserved before the access's own */
+            s += retention_quantum_ns(c, q);
+            c->pending_pj[die[i]] += retention_quantum_pj(c);
+            ++claims;
+        }
+        if (c->ret && !op) c->ret->disturb[retention_block_of(c, off)] += (uint32_t)np;
         s_ns[i] = s; cbs[i] = cb; eng[i] = e;
         if (op) { a_ns[i] = acc[i].issue_ns + xfer; post[i] = 0; }       /* program: data moves in first */
         else    { a_ns[i] = acc[i].issue_ns;        post[i] = xfer; }    /* read: data moves out after  */
@@ -496,6 +739,7 @@ int hbfo_submit_batch(hbfo_ctx *c, const hbfo_access_t *acc, uint64_t n, int64_t
     free(ds);
     res.code = HBFO_OK; res.n_native = n_native; res.n_modeled = n_ready;
     c->last = res;
+    if (c->ret) { c->ret->claimed += claims; retention_commit(c->ret); }
 
 done:
     free(st); free(rg); free(queue); free(die); free(a_ns); free(s_ns); free(post); free(cbs); free(eng);
@@ -523,7 +767,7 @@ static int cmp_pent(const void *pa, const void *pb) {
 
 int hbfo_submit_batch_paged(hbfo_ctx *c, const hbfo_access_t *acc, uint64_t n, int64_t *completion_ns,
                             int64_t *stall_ns, uint8_t *status, hbfo_die_stats_t *die_stats) {
-    if (!c || (n && (!acc || !completion_ns || !stall_ns)) || n > 0xffffffffull) return HBFO_E_INVAL;
+    if (!c || (n && (!acc || !completion_ns || !stall_ns)) || n > 0xffffffffull || c->ret) return HBFO_E_INVAL;
     hbfo_batch_result_t res; memset(&res, 0, sizeof(res));
     const int64_t q = c->q_ppm;
     res.mode = c->mode; res.q_ppm = q;

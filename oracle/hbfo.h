@@ -118,6 +118,37 @@ int32_t hbfo_next_mode(hbfo_ctx *ctx, int32_t mode, int64_t t_hot_mk);
 int64_t hbfo_quantise_mk(double t_c);
 const char *hbfo_strerror(int code);
 
+/* Retention, refresh and wear (Design D4; the definitions and the readings are at the head of this part of
+ * hbfo.c).  Not together with the energy bins, the channel bus or the page-granular submit.
+ *   hbfo_enable_retention     block state for channels*dies*planes*blocks_per_plane blocks, all fresh
+ *   hbfo_retention_advance    one epoch: damage += accel*dt/L(T) per block with its die's region temperature
+ *                             (region_temp_c [n_regions], or NULL = hottest cell of each region in the field),
+ *                             newly eligible blocks join the plan in the deterministic order
+ *   hbfo_submit_batch         the modeled accesses claim the outstanding quanta in index order, one each; reads
+ *                             count towards read disturb; blocks whose quanta are all claimed commit
+ *   hbfo_retention_decay      idle time drains outstanding quanta, one per scaled quantum time */
+typedef struct {
+    uint32_t pages_per_block, blocks_per_plane, blocks_per_zone;
+    uint32_t max_pec;                      /* a block that has committed this many cycles is worn out */
+    uint32_t disturb_limit;                /* page reads that make a block eligible; 0 = no limit */
+    uint32_t pad;
+    double l_ref_s, t_ref_c, ea_ev;        /* lifetime at the reference temperature; activation energy */
+    double accel;                          /* a_t, reliability-time acceleration */
+    double lead_threshold;                 /* damage at which a block becomes eligible */
+} hbfo_retention_config_t;
+typedef struct {
+    uint64_t n_blocks, planned, claimed, decayed, commits, worn_blocks, waiting_blocks;
+    uint32_t epoch, pad;
+} hbfo_retention_totals_t;
+int  hbfo_enable_retention(hbfo_ctx *ctx, const hbfo_retention_config_t *cfg);
+int  hbfo_retention_advance(hbfo_ctx *ctx, int64_t dt_ns, const double *region_temp_c);
+int  hbfo_retention_decay(hbfo_ctx *ctx, int64_t idle_ns);
+int  hbfo_get_retention_blocks(hbfo_ctx *ctx, double *damage, uint32_t *disturb, uint32_t *pec, uint32_t *epoch, uint64_t cap);
+/* the outstanding quanta in plan order (quantum = block * pages_per_block + page); quanta == NULL: count only */
+int  hbfo_get_retention_plan(hbfo_ctx *ctx, uint32_t *quanta, uint64_t cap, uint64_t *count);
+int  hbfo_get_retention_totals(hbfo_ctx *ctx, hbfo_retention_totals_t *out);
+double hbfo_retention_lifetime_s(hbfo_ctx *ctx, double temp_c);
+
 /* Reduced-order thermal model (Eq. 2): x' = A x + B p + b, T = C x + D p + d (x before the update).  Matrices
  * row-major, double, copied at create; b, D, d may be NULL (zero).  The state starts at zero. */
 typedef struct hbfo_rom hbfo_rom;

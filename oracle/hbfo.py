@@ -93,6 +93,14 @@ def lib():
         L.hbfo_get_bus_busy_until.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64]
         L.hbfo_enable_energy_bins.argtypes = [C.c_void_p, C.c_int64, C.c_uint32]
         L.hbfo_get_energy_bins.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.POINTER(C.c_int64)]
+        L.hbfo_enable_retention.argtypes = [C.c_void_p, C.POINTER(RetentionConfig)]
+        L.hbfo_retention_advance.argtypes = [C.c_void_p, C.c_int64, C.c_void_p]
+        L.hbfo_retention_decay.argtypes = [C.c_void_p, C.c_int64]
+        L.hbfo_get_retention_blocks.argtypes = [C.c_void_p] + [C.c_void_p] * 4 + [C.c_uint64]
+        L.hbfo_get_retention_plan.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.POINTER(C.c_uint64)]
+        L.hbfo_get_retention_totals.argtypes = [C.c_void_p, C.POINTER(RetentionTotals)]
+        L.hbfo_retention_lifetime_s.argtypes = [C.c_void_p, C.c_double]
+        L.hbfo_retention_lifetime_s.restype = C.c_double
         L.hbfo_rom_create.argtypes = [C.c_uint32, C.c_uint32, C.c_uint32] + [C.c_void_p] * 6 + [C.POINTER(C.c_void_p)]
         L.hbfo_thermal_step_rom.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_uint32, C.c_void_p]
         L.hbfo_rom_destroy.argtypes = [C.c_void_p]
@@ -124,6 +132,18 @@ _SCALARS = ("channels", "dies", "planes", "page_bytes", "stripe_bytes", "queue_l
 _ARRAYS = (("cell_C", np.float32), ("cell_Gx", np.float32), ("cell_Gy", np.float32), ("cell_Gsink", np.float32),
            ("cell_region", np.int32), ("die_region", np.int32), ("region_kind", np.int32),
            ("region_idle_w", np.float32))
+
+
+class RetentionConfig(C.Structure):
+    _fields_ = [("pages_per_block", C.c_uint32), ("blocks_per_plane", C.c_uint32), ("blocks_per_zone", C.c_uint32),
+                ("max_pec", C.c_uint32), ("disturb_limit", C.c_uint32), ("pad", C.c_uint32),
+                ("l_ref_s", C.c_double), ("t_ref_c", C.c_double), ("ea_ev", C.c_double),
+                ("accel", C.c_double), ("lead_threshold", C.c_double)]
+
+
+class RetentionTotals(C.Structure):
+    _fields_ = [(k, C.c_uint64) for k in ("n_blocks", "planned", "claimed", "decayed", "commits", "worn_blocks",
+                                          "waiting_blocks")] + [("epoch", C.c_uint32), ("pad", C.c_uint32)]
 
 
 class OracleError(RuntimeError):
@@ -210,6 +230,57 @@ class Oracle:
         if rc != 0:
             raise OracleError(rc)
         return hot
+
+    # ---- retention, refresh and wear (Design D4) ----
+    def enable_retention(self, **kw):
+        """Keyword arguments are the fields of ``hbfo_retention_config_t``."""
+        cfg = RetentionConfig()
+        for k, v in kw.items():
+            setattr(cfg, k, v)
+        rc = lib().hbfo_enable_retention(self._h, C.byref(cfg))
+        if rc != 0:
+            raise OracleError(rc)
+        self._ret_blocks = self.n_dies * self.cfg.planes * cfg.blocks_per_plane
+
+    def retention_advance(self, dt_ns, region_temp_c=None):
+        t = None if region_temp_c is None else np.ascontiguousarray(region_temp_c, np.float64)
+        rc = lib().hbfo_retention_advance(self._h, dt_ns, None if t is None else t.ctypes.data)
+        if rc != 0:
+            raise OracleError(rc)
+
+    def retention_decay(self, idle_ns):
+        rc = lib().hbfo_retention_decay(self._h, idle_ns)
+        if rc != 0:
+            raise OracleError(rc)
+
+    def retention_blocks(self) -> dict:
+        nb = self._ret_blocks
+        out = {"damage": np.zeros(nb, np.float64), "disturb": np.zeros(nb, np.uint32), "pec": np.zeros(nb, np.uint32),
+               "epoch": np.zeros(nb, np.uint32)}
+        rc = lib().hbfo_get_retention_blocks(self._h, out["damage"].ctypes.data, out["disturb"].ctypes.data,
+                                             out["pec"].ctypes.data, out["epoch"].ctypes.data, nb)
+        if rc != 0:
+            raise OracleError(rc)
+        return out
+
+    def retention_plan(self) -> np.ndarray:
+        cnt = C.c_uint64()
+        lib().hbfo_get_retention_plan(self._h, None, 0, C.byref(cnt))
+        out = np.zeros(cnt.value, np.uint32)
+        rc = lib().hbfo_get_retention_plan(self._h, out.ctypes.data, out.size, C.byref(cnt))
+        if rc != 0:
+            raise OracleError(rc)
+        return out
+
+    def retention_totals(self) -> dict:
+        t = RetentionTotals()
+        rc = lib().hbfo_get_retention_totals(self._h, C.byref(t))
+        if rc != 0:
+            raise OracleError(rc)
+        return {k: getattr(t, k) for k, _ in t._fields_ if k != "pad"}
+
+    def retention_lifetime_s(self, temp_c) -> float:
+        return lib().hbfo_retention_lifetime_s(self._h, float(temp_c))
 
     def enable_channel_bus(self):
         rc = lib().hbfo_enable_channel_bus(self._h)
