@@ -286,6 +286,60 @@ HBF_API int hbf_rom_get_state(hbf_rom *rom, double *host_out, uint64_t cap);
 HBF_API int hbf_attach_rom(hbf_ctx *ctx, hbf_rom *rom, const int32_t *output_kind, int64_t dt_ns);
 HBF_API int hbf_get_rom_temps(hbf_ctx *ctx, double *host_out, uint64_t cap);
 
+/* Retention, refresh and wear (Design D4: "Retention, Refresh, and Wear as Injected Latency").
+ * What the paper fixes: every registered block carries retention damage, a read-disturb count, a zone and a
+ * current and maximum program/erase count; the retention lifetime is L(T) = L_ref * exp[(E_a/k_B)(1/T - 1/T_ref)]
+ * (first equation of D4; E_a = 1.04 eV in the evaluation); damage accumulates as D <- D + a_t * dt / L(T) (second
+ * equation of D4); a block becomes eligible at its lead threshold or its read-disturb limit; refresh is emitted as
+ * page-aligned read-rewrite pairs in the order eligibility epoch, channel round robin, die round robin, zone,
+ * block, page; the plan is a debt of which every admission claims at most one quantum, reserving that quantum's
+ * thermally scaled service before its own; a block commits one program/erase cycle and clears its damage and
+ * disturb counters only when all its quanta are done; idle time drains debt on a separate account.
+ * What is this library's definition (the paper gives no layout or numbers for it): a block is pages_per_block
+ * consecutive pages of one plane, block = (page / pages_per_block) mod blocks_per_plane, id = ((channel * dies +
+ * die) * planes + plane) * blocks_per_plane + block, zone = block / blocks_per_zone; a quantum is one page (id =
+ * block id * pages_per_block + page), costing t_read + t_prog of array time scaled by Eq. 3 on the CLAIMING
+ * access's queue and die, its energy (one page read + one page program) booked on that die; within a die blocks
+ * are ordered by (zone, plane, block); a read adds its page count to the disturb counter of the block of its first
+ * page, programs add nothing; the modeled accesses of a batch claim in index (ticket) order; commits take effect
+ * when the batch, or the decay, that claimed a block's last quantum has completed.
+ *
+ * hbf_enable_retention: allocates the block state (all fresh).  Not together with the energy bins, the channel bus
+ *   or the page-granular submit (HBF_E_INVAL from whichever comes second).
+ * hbf_retention_advance: one epoch, asynchronously on the context's stream.  Every block that is not worn out gains
+ *   accel * dt / L(T) of damage, T being the temperature of its die's floorplan region: region_temp_c [n_regions]
+ *   (host, deg C, copied before the call returns; one entry when the context has no thermal configuration), or
+ *   NULL = the hottest cell of each region in the context's thermal field (HBF_E_INVAL without a field, or with a
+ *   reduced-order model attached).  Blocks that reach lead_threshold or disturb_limit become eligible in this epoch
+ *   and their pages join the end of the plan in the order above.
+ * hbf_submit_batch with retention on: the first (planned - claimed - decayed) modeled accesses of the batch, by
+ *   index, claim one quantum each; d_die_stats[].busy_ns and the summary's service_ns include the claimed time,
+ *   energy_pj does not (it goes to the pending thermal energy).  A refused batch claims nothing and disturbs
+ *   nothing.  While quanta are outstanding the batch is served by the sort path; with hbf_set_path(HBF_PATH_INORDER)
+ *   such a batch's result is HBF_E_INVAL.
+ * hbf_retention_decay: idle_ns of idle time drain floor(idle_ns / scaled quantum time) outstanding quanta.
+ * hbf_get_retention_blocks / _plan / _totals synchronise the stream and copy to host memory: per-block arrays
+ *   [n_blocks] (each nullable); the outstanding quanta in plan order (quanta == NULL: count only); the counters. */
+typedef struct {
+    uint32_t pages_per_block, blocks_per_plane, blocks_per_zone;   /* blocks_per_plane a multiple of blocks_per_zone */
+    uint32_t max_pec;                      /* a block that has committed this many cycles is worn out: no more damage, never eligible */
+    uint32_t disturb_limit;                /* page reads that make a block eligible; 0 = no limit */
+    uint32_t pad;
+    double l_ref_s, t_ref_c, ea_ev;        /* lifetime (s) at the reference temperature (deg C); activation energy (eV) */
+    double accel;                          /* a_t: reliability-time acceleration */
+    double lead_threshold;                 /* damage at which a block becomes eligible */
+} hbf_retention_config_t;
+typedef struct {
+    uint64_t n_blocks, planned, claimed, decayed, commits, worn_blocks, waiting_blocks;
+    uint32_t epoch, pad;
+} hbf_retention_totals_t;
+HBF_API int hbf_enable_retention(hbf_ctx *ctx, const hbf_retention_config_t *cfg);
+HBF_API int hbf_retention_advance(hbf_ctx *ctx, int64_t dt_ns, const double *region_temp_c);
+HBF_API int hbf_retention_decay(hbf_ctx *ctx, int64_t idle_ns);
+HBF_API int hbf_get_retention_blocks(hbf_ctx *ctx, double *damage, uint32_t *disturb, uint32_t *pec, uint32_t *epoch, uint64_t cap);
+HBF_API int hbf_get_retention_plan(hbf_ctx *ctx, uint32_t *quanta, uint64_t cap, uint64_t *count);
+HBF_API int hbf_get_retention_totals(hbf_ctx *ctx, hbf_retention_totals_t *out);
+
 HBF_API const char *hbf_strerror(int code);
 
 #ifdef __cplusplus

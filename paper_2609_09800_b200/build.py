@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 SO = os.path.join(HERE, "libhbf.so")
-SOURCES = ["hbf_api.cu", "submit_kernels.cu", "inorder_kernels.cu", "paged_kernels.cu", "energy_bins.cu", "rom_kernels.cu", "thermal_kernels.cu", "noalloc_thermal.cu"]
+SOURCES = ["hbf_api.cu", "submit_kernels.cu", "inorder_kernels.cu", "paged_kernels.cu", "energy_bins.cu", "rom_kernels.cu", "retention_kernels.cu", "thermal_kernels.cu", "noalloc_thermal.cu"]
 HEADERS = ["hbf_dev.cuh", "device_utils.cuh", os.path.join("..", "..", "include", "hbf.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--shared", "-cudart", "shared"]

@@ -43,6 +43,8 @@ struct hbf_ctx {
     int64_t *d_bus_busy = nullptr; BatchCtrl *d_bus_ctrl = nullptr;
     // time-bin energy ledger (off while bin_ns == 0)
     int64_t bin_ns = 0, cur_bin = 0; uint32_t n_bins = 0; unsigned long long *d_ledger = nullptr;
+    // retention, refresh and wear (off while ret_on == false)
+    bool ret_on = false; RetDev ret{}; hbf_retention_config_t ret_cfg{};
     float *h_hot = nullptr;                      // pinned [3]
     float *h_ext = nullptr;                      // pinned [n_regions]
     bool submitted = false;
@@ -89,6 +91,19 @@ static int publish_ranges(hbf_ctx *c) {
     // ordered after every batch already enqueued, before every later one
     CK(cudaMemcpyAsync(c->d_ranges, &snap, sizeof(snap), cudaMemcpyHostToDevice, c->stream));
     CK(cudaStreamSynchronize(c->stream));
+    return HBF_OK;
+}
+
+// ---- retention, refresh and wear (Design D4) ----------------------------------------------------------------
+static int retention_clear(hbf_ctx *c) {
+    const RetDev &r = c->ret;
+    CK(cudaMemsetAsync(r.damage, 0, r.n_blocks * 8, c->stream));
+    CK(cudaMemsetAsync(r.disturb, 0, r.n_blocks * 4, c->stream));
+    CK(cudaMemsetAsync(r.pec, 0, r.n_blocks * 4, c->stream));
+    CK(cudaMemsetAsync(r.epoch_of, 0, r.n_blocks * 4, c->stream));
+    CK(cudaMemsetAsync(r.worn, 0, r.n_blocks, c->stream));
+    CK(cudaMemsetAsync(r.die_claims, 0, (size_t)c->mp.n_dies * 4, c->stream));
+    CK(cudaMemsetAsync(r.st, 0, sizeof(RetState), c->stream));
     return HBF_OK;
 }
 
@@ -414,7 +429,13 @@ int hbf_submit_batch(hbf_ctx *c, const hbf_access_t *d_acc, uint64_t n, int64_t 
     a.ev = c->profiling ? c->ev : nullptr;
     c->prof_submit = c->profiling;
     a.binned = c->bin_ns != 0;
+    if (c->ret_on) {                                         // how far the outstanding refresh quanta reach into this batch
+        CK(launch_ret_window(d_acc, n, c->d_ranges, c->ret, c->sm_count, c->stream));
+        a.claim_limit = &c->ret.st->claim_limit; a.die_claims = c->ret.die_claims;
+    }
     CK(launch_submit(a, c->stream));
+    if (c->ret_on)                                           // read disturb, commits, the claimed energy
+        CK(launch_ret_close(d_acc, n, c->d_ranges, c->d_mp, c->mp, c->d_result, c->d_pending, c->ret, c->sm_count, c->stream));
     if (a.binned)
         CK(launch_energy_bins(d_acc, n, d_completion_ns, c->d_ranges, c->d_mp, c->d_ctrl, c->d_result, c->d_ledger, c->bin_ns,
                               c->n_bins, c->cur_bin, c->sm_count, c->stream));
@@ -436,7 +457,7 @@ int hbf_submit_batch_paged(hbf_ctx *c, const hbf_access_t *d_acc, uint64_t n, ui
     if (n == 0)                                             // nothing to split: the ordinary path reports the empty batch
         return hbf_submit_batch(c, d_acc, 0, d_completion_ns, d_stall_ns, d_status, d_die_stats, d_workspace, workspace_bytes);
     if (c->terminal) return HBF_E_LINK_SHUTDOWN;
-    if (n > HBF_MAX_BATCH || c->bin_ns != 0 || c->d_bus_busy) return HBF_E_INVAL;   // ledger and bus stage take whole accesses only
+    if (n > HBF_MAX_BATCH || c->bin_ns != 0 || c->d_bus_busy || c->ret_on) return HBF_E_INVAL;   // ledger, bus stage and retention take whole accesses only
     if (!d_acc || !d_completion_ns || !d_stall_ns) return HBF_E_INVAL;
     if ((reinterpret_cast<uintptr_t>(d_acc) & 7u) || (reinterpret_cast<uintptr_t>(d_completion_ns) & 7u) ||
         (reinterpret_cast<uintptr_t>(d_stall_ns) & 7u) || (reinterpret_cast<uintptr_t>(d_die_stats) & 7u)) return HBF_E_INVAL;
@@ -472,7 +493,7 @@ int hbf_submit_batch_paged(hbf_ctx *c, const hbf_access_t *d_acc, uint64_t n, ui
 }
 
 int hbf_enable_channel_bus(hbf_ctx *c) {
-    if (!c) return HBF_E_INVAL;
+    if (!c || c->ret_on) return HBF_E_INVAL;
     if (c->d_bus_busy) return HBF_OK;
     CK(cudaStreamSynchronize(c->stream));
     int64_t *b = nullptr; BatchCtrl *bc = nullptr;
@@ -491,8 +512,106 @@ int hbf_get_bus_busy_until(hbf_ctx *c, int64_t *host_out, uint64_t cap) {
     return HBF_OK;
 }
 
+int hbf_enable_retention(hbf_ctx *c, const hbf_retention_config_t *cfg) {
+    if (!c || !cfg || c->ret_on || c->bin_ns != 0 || c->d_bus_busy) return HBF_E_INVAL;
+    if (!cfg->pages_per_block || !cfg->blocks_per_plane || !cfg->blocks_per_zone ||
+        cfg->blocks_per_plane % cfg->blocks_per_zone != 0 || !cfg->max_pec) return HBF_E_INVAL;
+    if (!(cfg->l_ref_s > 0.0) || !(cfg->t_ref_c > -273.15) || !(cfg->ea_ev >= 0.0) || !(cfg->accel > 0.0) ||
+        !(cfg->lead_threshold > 0.0)) return HBF_E_INVAL;
+    const uint64_t nb = (uint64_t)c->mp.n_dies * c->mp.planes * cfg->blocks_per_plane;
+    if (nb * cfg->pages_per_block > 0xffffffffull) return HBF_E_INVAL;      // a quantum id is 32 bits
+    CK(cudaStreamSynchronize(c->stream));
+    RetDev r{};
+    r.ppb = cfg->pages_per_block; r.bpp = cfg->blocks_per_plane; r.bpz = cfg->blocks_per_zone; r.max_pec = cfg->max_pec;
+    r.disturb_limit = cfg->disturb_limit; r.n_regions = c->thermal ? c->td.n_regions : 1u;
+    r.accel = cfg->accel; r.lead = cfg->lead_threshold; r.l_ref_s = cfg->l_ref_s; r.t_ref_k = cfg->t_ref_c + 273.15;
+    r.ea_over_kb = cfg->ea_ev / 8.617333262e-5;                             // Boltzmann constant in eV/K
+    r.n_blocks = nb; r.plan_cap = nb * cfg->pages_per_block;
+    int rc;
+    if ((rc = dev_copy<double>(c, &r.damage, nullptr, nb)) != HBF_OK) return rc;
+    if ((rc = dev_copy<uint32_t>(c, &r.disturb, nullptr, nb)) != HBF_OK) return rc;
+    if ((rc = dev_copy<uint32_t>(c, &r.pec, nullptr, nb)) != HBF_OK) return rc;
+    if ((rc = dev_copy<uint32_t>(c, &r.epoch_of, nullptr, nb)) != HBF_OK) return rc;
+    if ((rc = dev_copy<uint8_t>(c, &r.worn, nullptr, nb)) != HBF_OK) return rc;
+    if ((rc = dev_copy<unsigned long long>(c, &r.last_pos, nullptr, nb)) != HBF_OK) return rc;
+    if ((rc = dev_copy<uint32_t>(c, &r.plan, nullptr, r.plan_cap)) != HBF_OK) return rc;
+    if ((rc = dev_copy<uint32_t>(c, &r.rank, nullptr, nb)) != HBF_OK) return rc;
+    if ((rc = dev_copy<unsigned long long>(c, &r.die_len, nullptr, c->mp.n_dies)) != HBF_OK) return rc;
+    if ((rc = dev_copy<unsigned long long>(c, &r.chan_len, nullptr, c->mp.channels)) != HBF_OK) return rc;
+    if ((rc = dev_copy<uint32_t>(c, &r.die_claims, nullptr, c->mp.n_dies)) != HBF_OK) return rc;
+    if ((rc = dev_copy<uint32_t>(c, &r.tile_count, nullptr, (HBF_MAX_BATCH + 1023) / 1024 + 1)) != HBF_OK) return rc;
+    if ((rc = dev_copy<double>(c, &r.rate, nullptr, r.n_regions)) != HBF_OK) return rc;
+    if ((rc = dev_copy<double>(c, &r.region_temp, nullptr, r.n_regions)) != HBF_OK) return rc;
+    if ((rc = dev_copy<int>(c, &r.region_max, nullptr, r.n_regions)) != HBF_OK) return rc;
+    if ((rc = dev_copy<RetState>(c, &r.st, nullptr, 1)) != HBF_OK) return rc;
+    c->ret = r; c->ret_cfg = *cfg; c->ret_on = true;
+    return HBF_OK;
+}
+
+int hbf_retention_advance(hbf_ctx *c, int64_t dt_ns, const double *region_temp_c) {
+    if (!c || !c->ret_on || dt_ns < 0) return HBF_E_INVAL;
+    if (!region_temp_c && (!c->thermal || c->rom)) return HBF_E_INVAL;      // no field to read the temperatures from
+    if (region_temp_c)                                                      // pageable source: staged before the call returns
+        CK(cudaMemcpyAsync(c->ret.region_temp, region_temp_c, c->ret.n_regions * sizeof(double), cudaMemcpyHostToDevice, c->stream));
+    CK(launch_ret_advance(c->ret, c->mp, c->thermal ? &c->td : nullptr, c->thermal ? c->td.theta[c->cur] : nullptr,
+                          c->thermal ? c->td.die_region : nullptr, region_temp_c ? 1 : 0, dt_ns, c->sm_count, c->stream));
+    return HBF_OK;
+}
+
+int hbf_retention_decay(hbf_ctx *c, int64_t idle_ns) {
+    if (!c || !c->ret_on || idle_ns < 0) return HBF_E_INVAL;
+    CK(launch_ret_decay(c->ret, c->mp, c->d_state, idle_ns, c->sm_count, c->stream));
+    return HBF_OK;
+}
+
+int hbf_get_retention_blocks(hbf_ctx *c, double *damage, uint32_t *disturb, uint32_t *pec, uint32_t *epoch, uint64_t cap) {
+    if (!c || !c->ret_on || cap < c->ret.n_blocks) return HBF_E_INVAL;
+    const RetDev &r = c->ret;
+    if (damage) CK(cudaMemcpyAsync(damage, r.damage, r.n_blocks * 8, cudaMemcpyDeviceToHost, c->stream));
+    if (disturb) CK(cudaMemcpyAsync(disturb, r.disturb, r.n_blocks * 4, cudaMemcpyDeviceToHost, c->stream));
+    if (pec) CK(cudaMemcpyAsync(pec, r.pec, r.n_blocks * 4, cudaMemcpyDeviceToHost, c->stream));
+    if (epoch) CK(cudaMemcpyAsync(epoch, r.epoch_of, r.n_blocks * 4, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    return HBF_OK;
+}
+
+static int retention_state(hbf_ctx *c, RetState *out) {
+    CK(cudaMemcpyAsync(out, c->ret.st, sizeof(RetState), cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    return HBF_OK;
+}
+
+int hbf_get_retention_plan(hbf_ctx *c, uint32_t *quanta, uint64_t cap, uint64_t *count) {
+    if (!c || !c->ret_on || !count) return HBF_E_INVAL;
+    RetState s; int rc = retention_state(c, &s);
+    if (rc != HBF_OK) return rc;
+    const uint64_t mark = s.claimed + s.decayed, m = s.planned - mark;
+    *count = m;
+    if (!quanta) return HBF_OK;
+    if (cap < m) return HBF_E_INVAL;
+    const uint64_t first = mark % c->ret.plan_cap, head = std::min<uint64_t>(m, c->ret.plan_cap - first);   // the ring may wrap once
+    if (head) CK(cudaMemcpyAsync(quanta, c->ret.plan + first, head * 4, cudaMemcpyDeviceToHost, c->stream));
+    if (m > head) CK(cudaMemcpyAsync(quanta + head, c->ret.plan, (m - head) * 4, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    return HBF_OK;
+}
+
+int hbf_get_retention_totals(hbf_ctx *c, hbf_retention_totals_t *out) {
+    if (!c || !c->ret_on || !out) return HBF_E_INVAL;
+    RetState s; int rc = retention_state(c, &s);
+    if (rc != HBF_OK) return rc;
+    std::vector<uint32_t> ep(c->ret.n_blocks);
+    CK(cudaMemcpyAsync(ep.data(), c->ret.epoch_of, c->ret.n_blocks * 4, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    out->n_blocks = c->ret.n_blocks; out->planned = s.planned; out->claimed = s.claimed; out->decayed = s.decayed;
+    out->commits = s.commits; out->worn_blocks = s.worn_blocks; out->epoch = s.epoch; out->pad = 0;
+    out->waiting_blocks = 0;
+    for (uint32_t e : ep) if (e) out->waiting_blocks += 1;
+    return HBF_OK;
+}
+
 int hbf_enable_energy_bins(hbf_ctx *c, int64_t bin_ns, uint32_t n_bins) {
-    if (!c || bin_ns <= 0 || n_bins == 0) return HBF_E_INVAL;
+    if (!c || bin_ns <= 0 || n_bins == 0 || c->ret_on) return HBF_E_INVAL;
     CK(cudaStreamSynchronize(c->stream));
     unsigned long long *l = nullptr;
     if (cudaMalloc(&l, (size_t)n_bins * c->mp.n_dies * 8) != cudaSuccess) return HBF_E_NOMEM;
@@ -600,6 +719,7 @@ int hbf_reset(hbf_ctx *c) {
     CK(cudaMemsetAsync(c->d_result, 0, sizeof(hbf_batch_result_t), c->stream));
     if (c->bin_ns) { CK(cudaMemsetAsync(c->d_ledger, 0, (size_t)c->n_bins * c->mp.n_dies * 8, c->stream)); c->cur_bin = 0; }
     if (c->d_bus_busy) CK(cudaMemsetAsync(c->d_bus_busy, 0, (size_t)c->mp.channels * 8, c->stream));
+    if (c->ret_on) { int rc = retention_clear(c); if (rc != HBF_OK) return rc; }
     if (c->thermal) {
         const size_t nc = (size_t)c->td.H * c->td.W;
         CK(cudaMemsetAsync(c->td.theta[0], 0, nc * sizeof(float), c->stream));

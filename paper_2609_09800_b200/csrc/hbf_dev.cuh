@@ -106,6 +106,8 @@ struct SubmitArgs {
     Workspace ws; int32_t path; int sm_count; int inorder_ok;
     FastRange fast;
     int binned;                          // the batch's energy goes to the time-bin ledger, not to the pending totals
+    const unsigned long long *claim_limit;  // retention on: batch index below which a modeled access claims a refresh quantum
+    uint32_t *die_claims;                   // retention on: [dies] claims of the batch
     cudaEvent_t *ev;                     // [kProfEvents] or null: recorded between kernel groups
 };
 constexpr int kProfEvents = 10;
@@ -160,6 +162,39 @@ cudaError_t launch_take_bin(unsigned long long *row, int64_t *pending, uint32_t 
 cudaError_t launch_rom_steps(uint32_t n, uint32_t m, uint32_t o, const double *A, const double *B, const double *b,
                              const double *C, const double *D, const double *d, double *x, const double *power,
                              uint32_t n_steps, double *temps_out, cudaStream_t st);
+
+// ---- retention, refresh and wear (Design D4) -------------------------------------------------------------
+// Device-resident counters of the refresh plan.  planned - claimed - decayed quanta are outstanding (the debt).
+struct RetState {
+    unsigned long long planned, claimed, decayed, commits, worn_blocks;
+    unsigned long long claim_limit;      // this batch: modeled accesses with a smaller batch index claim one quantum each
+    unsigned long long claims_now;       // quanta this batch claims if it is accepted
+    unsigned long long tickets, counted; // the claim window's tile counter and the modeled accesses counted so far
+    unsigned long long epoch_total;      // quanta the epoch in progress adds
+    uint32_t epoch, pad;
+};
+struct RetDev {
+    uint32_t ppb, bpp, bpz, max_pec, disturb_limit, n_regions;
+    double accel, lead, l_ref_s, t_ref_k, ea_over_kb;
+    uint64_t n_blocks, plan_cap;
+    double *damage; uint32_t *disturb, *pec, *epoch_of; uint8_t *worn;
+    unsigned long long *last_pos;        // [blocks] plan position of the block's last quantum
+    uint32_t *plan;                      // [plan_cap] ring of quanta (block * ppb + page), position modulo plan_cap
+    uint32_t *rank;                      // [blocks] rank of a newly eligible block in its die's (zone, plane, block) order
+    unsigned long long *die_len, *chan_len;   // quanta the epoch in progress adds per die, per channel
+    uint32_t *die_claims;                // [dies] quanta claimed on each die by the batch in progress
+    uint32_t *tile_count;                // [tiles of 1,024 records] modeled accesses, claim window
+    double *rate, *region_temp;          // [regions] damage per block of this epoch; temperatures
+    int *region_max;                     // [regions] hottest cell, as an ordered integer
+    RetState *st;
+};
+cudaError_t launch_ret_window(const hbf_access_t *acc, uint64_t n, const RangeSnap *ranges, const RetDev &r, int sm_count, cudaStream_t st);
+cudaError_t launch_ret_close(const hbf_access_t *acc, uint64_t n, const RangeSnap *ranges, const ModelParams *mp_dev, const ModelParams &mp,
+                             const hbf_batch_result_t *result, int64_t *pending, const RetDev &r, int sm_count, cudaStream_t st);
+struct ThermalDev;
+cudaError_t launch_ret_advance(const RetDev &r, const ModelParams &mp, const ThermalDev *field, const float *theta, const int32_t *die_region,
+                               int have_temps, int64_t dt_ns, int sm_count, cudaStream_t st);
+cudaError_t launch_ret_decay(const RetDev &r, const ModelParams &mp, const DevState *state, int64_t idle_ns, int sm_count, cudaStream_t st);
 
 // ---- thermal -------------------------------------------------------------------------------------
 struct ThermalDev {

@@ -140,8 +140,8 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
     __shared__ ModelParams mp;                            // measured: reads from shared memory beat reads of the argument
     __shared__ FastRange fast_range;
 
-    if (ctrl->skip) return;
-    if (RESERVE && (ctrl->run_sort || !ctrl->inorder_used || !in_tile[blockIdx.x].reserve)) return;
+    if (ctrl->skip || ctrl->run_sort) return;             // (run_sort set this early: the batch went to the sort path at its start)
+    if (RESERVE && (!ctrl->inorder_used || !in_tile[blockIdx.x].reserve)) return;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const RangeSnap &rs = *ranges_g;                      // read through the cache; the common configuration does not touch it
     if (tid == 0) { mp = mp_arg; fast_range = fast_arg; }
@@ -378,7 +378,7 @@ __global__ void __launch_bounds__(kInScanThreads)
 k_inorder_scan(BatchCtrl *ctrl, const ModelParams *__restrict__ mp, uint32_t n_tiles, const int64_t *__restrict__ in_agg,
                int64_t *__restrict__ in_bin, const int64_t *__restrict__ busy, int64_t *busy_stage,
                hbf_die_stats_t *stats_stage, int forced) {
-    if (ctrl->skip) return;
+    if (ctrl->skip || ctrl->run_sort) return;
     const bool fault = ctrl->n_fault != 0, unsorted = ctrl->unsorted != 0u;
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         if (fault) { ctrl->code = HBF_E_ACCESS_FAULT; ctrl->skip = 1; }                 // fail closed: refuse the batch

@@ -18,12 +18,15 @@ namespace hbf {
 //         sort path when the in-order attempt found the records out of issue order, else does nothing.
 __global__ void k_begin(BatchCtrl *ctrl, const DevState *state, const int64_t *busy, int64_t *busy_stage,
                         hbf_die_stats_t *stats_stage, uint32_t *hist, uint32_t n_queues, uint32_t n_dies,
-                        int role, int run_sort) {
+                        int role, int run_sort, const unsigned long long *claim_limit, int sort_available) {
     const int tid = threadIdx.x;
     if (role == 1) {
         if (ctrl->skip || !ctrl->run_sort) return;
         run_sort = 1;
     }
+    // refresh quanta to be claimed (retention on): the claims are applied by the sort path
+    const bool claims = claim_limit != nullptr && *claim_limit != 0ull;
+    if (claims) run_sort = 1;
     __syncthreads();
     uint32_t *w = reinterpret_cast<uint32_t *>(ctrl);
     for (int i = tid; i < (int)(sizeof(BatchCtrl) / 4); i += blockDim.x) w[i] = 0u;
@@ -37,6 +40,7 @@ __global__ void k_begin(BatchCtrl *ctrl, const DevState *state, const int64_t *b
         if (state->poisoned) { ctrl->code = HBF_E_TIMEOUT; ctrl->skip = 1; }
         else if (mode == HBF_MODE_SHUTDOWN) { ctrl->code = HBF_E_LINK_SHUTDOWN; ctrl->skip = 1; }
         else if (mode == HBF_MODE_SEVERE) { ctrl->code = HBF_E_THROTTLED; ctrl->skip = 1; }
+        else if (claims && !sort_available) { ctrl->code = HBF_E_INVAL; ctrl->skip = 1; }
     }
     for (uint32_t r = tid; r < n_queues; r += blockDim.x) busy_stage[r] = busy[r];
     int64_t *s = reinterpret_cast<int64_t *>(stats_stage);
@@ -354,7 +358,8 @@ k_scan(const hbf_access_t *__restrict__ acc, uint64_t n, const RangeSnap *__rest
        const ModelParams *__restrict__ mp_g, BatchCtrl *ctrl, DevState *state,
        const uint64_t *keys0, const uint64_t *keys1, const uint32_t *idx0, const uint32_t *idx1,
        ScanDesc *desc, const int64_t *__restrict__ busy, int64_t *busy_stage, hbf_die_stats_t *stats_stage,
-       int64_t *__restrict__ completion, int64_t *__restrict__ stall) {
+       int64_t *__restrict__ completion, int64_t *__restrict__ stall,
+       const unsigned long long *claim_limit_p, uint32_t *die_claims) {
     __shared__ RangeSnap rs;
     __shared__ ModelParams mp;
     __shared__ uint32_t s_first_q[kScanThreads], s_last_q[kScanThreads];
@@ -385,6 +390,11 @@ k_scan(const hbf_access_t *__restrict__ acc, uint64_t n, const RangeSnap *__rest
     const int64_t q_ppm = ctrl->q_ppm;
     const Div64 div_q = ctrl->div_q;
     const int cnt = (int)min((uint64_t)kScanTile, m - base);
+    // retention on: a modeled access with a batch index below the claim limit pays one refresh quantum (a page read
+    // and a page program, scaled like any service, Eq. 3) before its own service
+    const uint64_t claim_limit = claim_limit_p ? *claim_limit_p : 0ull;
+    const int64_t quantum_ns = q_ppm == 1000000 ? mp.t_read_ns + mp.t_prog_ns
+        : (int64_t)div64((uint64_t)(mp.t_read_ns + mp.t_prog_ns) * 1000000ull + (uint64_t)q_ppm - 1ull, div_q);
 
     // this thread's consecutive items
     uint32_t queue[kScanItems], idx[kScanItems], post[kScanItems];
@@ -447,9 +457,10 @@ k_scan(const hbf_access_t *__restrict__ acc, uint64_t n, const RangeSnap *__rest
             const Decoded d = decode(mp, off, bytes);
             const Terms t = service_terms(mp, bytes, d.npages, op, q_ppm, div_q);
             s[j] = t.s;
+            if ((uint64_t)idx[j] < claim_limit) { s[j] += quantum_ns; atomicAdd(&die_claims[d.die], 1u); }
             if (op) { a[j] = issue[j] + t.xfer; post[j] = 0u; } else { a[j] = issue[j]; post[j] = (uint32_t)t.xfer; }
             if (d.die != run_die) { if (run_die != 0xffffffffu) flush_run(run_die); run_die = d.die; }
-            acc_busy += t.s; acc_e += t.energy; sum_s += t.s;
+            acc_busy += s[j]; acc_e += t.energy; sum_s += s[j];
             if (op) { acc_bp += t.cb; acc_np += 1; } else { acc_br += t.cb; acc_nr += 1; }
         }
     }
@@ -973,7 +984,8 @@ static cudaError_t launch_sort_path(const SubmitArgs &a, cudaStream_t st) {
     mark(4);
     k_scan<<<(unsigned)std::min<uint64_t>(scan_tiles, (uint64_t)a.sm_count * 8), kScanThreads, 0, st>>>(a.acc, n, a.ranges, a.mp_dev, a.ctrl, a.state, a.ws.keys[0], a.ws.keys[1],
                                                          a.ws.idx[0], a.ws.idx[1], (ScanDesc *)a.ws.scan_desc, a.busy,
-                                                         a.busy_stage, a.stats_stage, a.completion, a.stall);
+                                                         a.busy_stage, a.stats_stage, a.completion, a.stall,
+                                                         a.claim_limit, a.die_claims);
     g_kernel_launches += 4 + kMaxPasses;
     return cudaSuccess;
 }
@@ -988,7 +1000,7 @@ cudaError_t launch_submit(const SubmitArgs &a, cudaStream_t st) {
     const bool sort_kernels = a.path != HBF_PATH_INORDER || !a.inorder_ok;
     mark(0);
     k_begin<<<1, 256, 0, st>>>(a.ctrl, a.state, a.busy, a.busy_stage, a.stats_stage, a.ws.hist, a.mp.n_queues, a.mp.n_dies,
-                               0, try_inorder ? 0 : 1);
+                               0, try_inorder ? 0 : 1, a.claim_limit, sort_kernels ? 1 : 0);
     g_kernel_launches += 1;
     if (n > 0) {
         if (try_inorder) {
@@ -998,7 +1010,7 @@ cudaError_t launch_submit(const SubmitArgs &a, cudaStream_t st) {
             mark(8);
             if (sort_kernels) {
                 k_begin<<<1, 256, 0, st>>>(a.ctrl, a.state, a.busy, a.busy_stage, a.stats_stage, a.ws.hist, a.mp.n_queues,
-                                           a.mp.n_dies, 1, 1);
+                                           a.mp.n_dies, 1, 1, a.claim_limit, 1);
                 g_kernel_launches += 1;
             }
         }

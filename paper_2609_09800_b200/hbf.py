@@ -32,9 +32,23 @@ EXPORTS = ("hbf_create", "hbf_destroy", "hbf_register_range", "hbf_clear_ranges"
            "hbf_workspace_bytes_paged", "hbf_submit_batch_paged",
            "hbf_enable_energy_bins", "hbf_get_energy_bins", "hbf_enable_channel_bus", "hbf_get_bus_busy_until",
            "hbf_rom_create", "hbf_rom_destroy", "hbf_rom_reset", "hbf_rom_step", "hbf_rom_get_state",
-           "hbf_attach_rom", "hbf_get_rom_temps")
+           "hbf_attach_rom", "hbf_get_rom_temps",
+           "hbf_enable_retention", "hbf_retention_advance", "hbf_retention_decay", "hbf_get_retention_blocks",
+           "hbf_get_retention_plan", "hbf_get_retention_totals")
 STATIC_MAX_CELLS = 65536
 PROF_STAGES = ("begin", "classify", "plan_hist", "sort", "scan", "finish", "inorder", "thermal")
+
+
+class hbf_retention_config_t(C.Structure):
+    _fields_ = [("pages_per_block", C.c_uint32), ("blocks_per_plane", C.c_uint32), ("blocks_per_zone", C.c_uint32),
+                ("max_pec", C.c_uint32), ("disturb_limit", C.c_uint32), ("pad", C.c_uint32),
+                ("l_ref_s", C.c_double), ("t_ref_c", C.c_double), ("ea_ev", C.c_double),
+                ("accel", C.c_double), ("lead_threshold", C.c_double)]
+
+
+class hbf_retention_totals_t(C.Structure):
+    _fields_ = [(k, C.c_uint64) for k in ("n_blocks", "planned", "claimed", "decayed", "commits", "worn_blocks",
+                                          "waiting_blocks")] + [("epoch", C.c_uint32), ("pad", C.c_uint32)]
 
 
 class hbf_config_t(C.Structure):
@@ -95,6 +109,12 @@ def lib():
         L.hbf_enable_channel_bus.argtypes = [vp]
         L.hbf_get_bus_busy_until.argtypes = [vp, vp, u64]
         L.hbf_enable_energy_bins.argtypes = [vp, i64, u32]
+        L.hbf_enable_retention.argtypes = [vp, C.POINTER(hbf_retention_config_t)]
+        L.hbf_retention_advance.argtypes = [vp, i64, vp]
+        L.hbf_retention_decay.argtypes = [vp, i64]
+        L.hbf_get_retention_blocks.argtypes = [vp, vp, vp, vp, vp, u64]
+        L.hbf_get_retention_plan.argtypes = [vp, vp, u64, C.POINTER(u64)]
+        L.hbf_get_retention_totals.argtypes = [vp, C.POINTER(hbf_retention_totals_t)]
         L.hbf_get_energy_bins.argtypes = [vp, vp, u64, C.POINTER(i64)]
         L.hbf_rom_create.argtypes = [u32, u32, u32, vp, vp, vp, vp, vp, vp, vp, C.POINTER(vp)]
         L.hbf_attach_rom.argtypes = [vp, vp, vp, i64]
@@ -194,6 +214,7 @@ class Context:
         cfg, keep = make_config(profile, floorplan)
         self.n_dies = cfg.channels * cfg.dies
         self.n_channels = cfg.channels
+        self.n_planes = cfg.planes
         self.n_queues = self.n_dies * (cfg.planes if cfg.queue_level == 0 else 1)
         self.n_cells = cfg.grid_h * cfg.grid_w if floorplan is not None else 0
         self.n_regions = cfg.n_regions if floorplan is not None else 0
@@ -279,6 +300,56 @@ class Context:
         if rc != 0:
             raise HbfError(rc, "hbf_get_rom_temps")
         return out
+
+    # ---- retention, refresh and wear (Design D4) ----
+    def enable_retention(self, **kw):
+        """Keyword arguments are the fields of ``hbf_retention_config_t``."""
+        cfg = hbf_retention_config_t()
+        for k, v in kw.items():
+            setattr(cfg, k, v)
+        rc = lib().hbf_enable_retention(self._h, C.byref(cfg))
+        if rc != 0:
+            raise HbfError(rc, "hbf_enable_retention")
+        self._ret_blocks = self.n_dies * self.n_planes * cfg.blocks_per_plane
+
+    def retention_advance(self, dt_ns, region_temp_c=None):
+        t = None if region_temp_c is None else np.ascontiguousarray(region_temp_c, np.float64)
+        rc = lib().hbf_retention_advance(self._h, dt_ns, None if t is None else t.ctypes.data)
+        if rc != 0:
+            raise HbfError(rc, "hbf_retention_advance")
+
+    def retention_decay(self, idle_ns):
+        rc = lib().hbf_retention_decay(self._h, idle_ns)
+        if rc != 0:
+            raise HbfError(rc, "hbf_retention_decay")
+
+    def retention_blocks(self) -> dict:
+        nb = self._ret_blocks
+        out = {"damage": np.zeros(nb, np.float64), "disturb": np.zeros(nb, np.uint32), "pec": np.zeros(nb, np.uint32),
+               "epoch": np.zeros(nb, np.uint32)}
+        rc = lib().hbf_get_retention_blocks(self._h, out["damage"].ctypes.data, out["disturb"].ctypes.data,
+                                            out["pec"].ctypes.data, out["epoch"].ctypes.data, nb)
+        if rc != 0:
+            raise HbfError(rc, "hbf_get_retention_blocks")
+        return out
+
+    def retention_plan(self) -> np.ndarray:
+        cnt = C.c_uint64()
+        rc = lib().hbf_get_retention_plan(self._h, None, 0, C.byref(cnt))
+        if rc != 0:
+            raise HbfError(rc, "hbf_get_retention_plan")
+        out = np.zeros(cnt.value, np.uint32)
+        rc = lib().hbf_get_retention_plan(self._h, out.ctypes.data, out.size, C.byref(cnt))
+        if rc != 0:
+            raise HbfError(rc, "hbf_get_retention_plan")
+        return out
+
+    def retention_totals(self) -> dict:
+        t = hbf_retention_totals_t()
+        rc = lib().hbf_get_retention_totals(self._h, C.byref(t))
+        if rc != 0:
+            raise HbfError(rc, "hbf_get_retention_totals")
+        return {k: getattr(t, k) for k, _ in t._fields_ if k != "pad"}
 
     def enable_channel_bus(self):
         rc = lib().hbf_enable_channel_bus(self._h)

@@ -1,0 +1,265 @@
+"""Parity of the retention / refresh / wear part (hbf_enable_retention and friends) with the oracle's, through the C
+ABI: integers bit for bit (plan order, claims, completions, counters), damage within 1e-12 relative (the two sides
+call different exp() implementations)."""
+import json
+import os
+
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+from oracle import hbfo
+from paper_2609_09800_b200 import workloads as wl
+
+BASE = wl.RANGE_BASE
+PAGE = 16 * wl.KIB
+RET = dict(pages_per_block=4, blocks_per_plane=8, blocks_per_zone=2, max_pec=3, disturb_limit=0,
+           l_ref_s=1000.0, t_ref_c=40.0, ea_ev=1.04, accel=1.0, lead_threshold=0.5)
+
+
+@pytest.fixture(scope="module")
+def hbf():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2609_09800_b200 import build, hbf as mod
+    build.build()
+    return mod
+
+
+def contexts(hbf, ret, geometry="tiny", floorplan=None, path=None, **over):
+    prof = wl.load_profile("nominal", **wl.GEOMETRY[geometry])
+    prof.update(over)
+    g, o = hbf.Context(prof, floorplan), hbfo.Oracle(prof, floorplan)
+    g.register_range(BASE, 64 * wl.GIB); o.register_range(BASE, 64 * wl.GIB)
+    if path is not None:
+        g.set_path(path)
+    g.enable_retention(**ret); o.enable_retention(**ret)
+    return g, o, prof
+
+
+def compare_state(g, o, rtol=1e-12):
+    bg, bo = g.retention_blocks(), o.retention_blocks()
+    for k in ("disturb", "pec", "epoch"):
+        bad = np.flatnonzero(bg[k] != bo[k])
+        assert bad.size == 0, "%s: first mismatch at block %d: gpu %d oracle %d" % (k, bad[0], bg[k][bad[0]], bo[k][bad[0]])
+    assert np.allclose(bg["damage"], bo["damage"], rtol=rtol, atol=0.0)
+    assert g.retention_totals() == o.retention_totals()
+    pg, po = g.retention_plan(), o.retention_plan()
+    assert pg.shape == po.shape
+    bad = np.flatnonzero(pg != po)
+    assert bad.size == 0, "plan: first mismatch at %d: gpu %d oracle %d (%d of %d)" % (bad[0], pg[bad[0]], po[bad[0]], bad.size, pg.size)
+
+
+def compare_batch(g, o, acc, rtol=1e-12):
+    rc_o, c_o, s_o, st_o, ds_o = o.submit(acc, check=False)
+    rc_g, c_g, s_g, st_g, ds_g = g.submit_host(acc, check=False)
+    assert rc_g == rc_o
+    if rc_o == 0:
+        assert np.array_equal(st_g, st_o)
+        bad = np.flatnonzero(c_g != c_o)
+        assert bad.size == 0, "first mismatch at %d: gpu %d oracle %d (%d mismatches)" % (bad[0], c_g[bad[0]], c_o[bad[0]], bad.size)
+        assert np.array_equal(s_g, s_o)
+        for k in hbfo.DIE_STATS_DTYPE.names:
+            assert np.array_equal(ds_g[k], ds_o[k]), k
+        assert g.last_result() == o.last_result()
+    assert np.array_equal(g.get_busy_until(), o.busy_until())
+    assert np.array_equal(g.get_pending_energy(), o.pending_energy())
+    compare_state(g, o, rtol)
+    return rc_g
+
+
+def recs(rows):
+    a = np.zeros(len(rows), hbfo.ACCESS_DTYPE)
+    for i, (off, issue, nbytes, op) in enumerate(rows):
+        a[i] = (BASE + off, issue, nbytes, op)
+    return a
+
+
+def offset_of(prof, ret, ch, di, pl, block, page=0):
+    C, D, P = prof["channels"], prof["dies"], prof["planes"]
+    return (((((block * ret["pages_per_block"] + page) * P + pl) * D + di) * C + ch)) * PAGE
+
+
+def test_hand_example(hbf, golden_dir):
+    with open(os.path.join(golden_dir, "retention_examples.json")) as f:
+        ex = json.load(f)
+    ret = dict(RET, **ex["retention"])
+    prof = wl.load_profile("nominal", **wl.GEOMETRY["tiny"]); prof.update(ex["geometry"])
+    g = hbf.Context(prof)
+    g.register_range(BASE, wl.GIB)
+    g.enable_retention(**ret)
+    g.submit_host(recs([(offset_of(prof, ret, b["channel"], b["die"], b["plane"], b["block"]), 0, 64, 0) for b in ex["eligible_blocks"]]))
+    g.retention_advance(0, np.array([40.0]))
+    assert g.retention_plan().tolist() == ex["plan"]
+    rows = [(offset_of(prof, ret, 1, 1, pl, 0), 0, PAGE, 0) for pl in (0, 1)] + [(offset_of(prof, ret, 1, 0, 1, 0), 0, PAGE, 0)]
+    _, comp, _, _, _ = g.submit_host(recs(rows))
+    assert comp.tolist() == ex["claims"]["completion_first"]
+    _, comp, _, _, _ = g.submit_host(recs([(offset_of(prof, ret, 1, 1, pl, 0), 1_000_000, PAGE, 0) for pl in (0, 1)]))
+    assert comp.tolist() == ex["claims"]["completion_second"]
+    pec = g.retention_blocks()["pec"]
+    assert {str(i): int(v) for i, v in enumerate(pec) if v} == ex["claims"]["pec_after_second"]
+    assert g.retention_plan().tolist() == ex["claims"]["plan_after_second"]
+    g.retention_decay(ex["decay"]["idle_ns"])
+    pec = g.retention_blocks()["pec"]
+    assert {str(i): int(v) for i, v in enumerate(pec) if v} == ex["decay"]["pec_after"]
+    assert g.retention_plan().tolist() == ex["decay"]["plan_after"]
+    t = g.retention_totals()
+    assert (t["planned"], t["claimed"], t["decayed"], t["commits"]) == (10, 5, 2, 3)
+
+
+def mixed_batch(rng, n, t0, span_pages, natives=0.1, progs=0.1, gap=400):
+    acc = np.zeros(n, hbfo.ACCESS_DTYPE)
+    acc["addr"] = BASE + rng.integers(0, span_pages, n).astype(np.uint64) * np.uint64(PAGE) + rng.integers(0, 4, n).astype(np.uint64) * np.uint64(4096)
+    acc["issue_ns"] = t0 + np.sort(rng.integers(0, gap * n + 1, n))
+    acc["bytes"] = rng.choice([64, 4096, 16000, 40000], n)
+    acc["flags"] = rng.random(n) < progs
+    nat = rng.random(n) < natives
+    acc["addr"][nat] = 0x2000 + 64 * np.arange(int(nat.sum()), dtype=np.uint64)
+    return acc
+
+
+@pytest.mark.parametrize("path", ["auto", "sort"])
+@pytest.mark.parametrize("n", [1, 33, 2049, 70_000])
+def test_rounds_of_batches_epochs_and_decay(hbf, n, path):
+    """Blocks become eligible by read disturb and by damage, batches claim what they can, blocks commit and wear out."""
+    ret = dict(RET, disturb_limit=max(2, n // 300), lead_threshold=0.02, max_pec=2, pages_per_block=4)
+    g, o, prof = contexts(hbf, ret, path=hbf.PATH_AUTO if path == "auto" else hbf.PATH_SORT)
+    rng = np.random.default_rng(n + (7 if path == "sort" else 0))
+    span_pages = 8 * 4 * 2 * 8 * 4 * 2                                   # twice the tracked blocks: the block index wraps
+    t0 = 0
+    for round_ in range(6):
+        acc = mixed_batch(rng, n, t0, span_pages)
+        assert compare_batch(g, o, acc) == 0
+        t0 = int(acc["issue_ns"][-1]) + 50_000_000
+        temps = np.array([rng.uniform(35.0, 95.0)])
+        dt = int(rng.integers(1, 40)) * 10**9
+        g.retention_advance(dt, temps); o.retention_advance(dt, temps)
+        compare_state(g, o)
+        if round_ % 2 == 1:
+            idle = int(rng.integers(0, 30)) * 395_000 + int(rng.integers(0, 395_000))
+            g.retention_decay(idle); o.retention_decay(idle)
+            compare_state(g, o)
+    t = o.retention_totals()
+    if n >= 2049:                                                        # the scenario does exercise every stage
+        assert t["claimed"] > 0 and t["commits"] > 0 and t["worn_blocks"] > 0
+
+
+def test_whole_batch_claims_and_debt_remains(hbf):
+    ret = dict(RET, disturb_limit=1, lead_threshold=1e9, pages_per_block=64, blocks_per_plane=64, blocks_per_zone=8)
+    g, o, prof = contexts(hbf, ret)
+    rows = [(offset_of(prof, ret, c, d, 0, 0), 0, 64, 0) for c in range(8) for d in range(4)]
+    compare_batch(g, o, recs(rows))
+    g.retention_advance(0, np.array([40.0])); o.retention_advance(0, np.array([40.0]))
+    compare_state(g, o)
+    assert o.retention_totals()["planned"] == 32 * 64
+    w = wl.tiny_uniform(n=1500, seed=4, rho=0.9)
+    acc = w.acc.copy(); acc["issue_ns"] += 10**8
+    assert compare_batch(g, o, acc) == 0
+    assert o.retention_totals()["claimed"] == 1500
+    acc["issue_ns"] += 10**9
+    assert compare_batch(g, o, acc) == 0                                  # the debt ends inside this one
+    assert o.retention_totals()["claimed"] == 2048
+
+
+def test_thermally_scaled_claims(hbf):
+    ret = dict(RET, disturb_limit=1, lead_threshold=1e9)
+    g, o, prof = contexts(hbf, ret)
+    rng = np.random.default_rng(5)
+    compare_batch(g, o, mixed_batch(rng, 500, 0, 4096, natives=0.0, progs=0.0))
+    g.retention_advance(0, np.array([40.0])); o.retention_advance(0, np.array([40.0]))
+    g.force_mode(1, 612_345); hbfo.lib().hbfo_force_mode(o._h, 1, 612_345)
+    assert compare_batch(g, o, mixed_batch(rng, 3000, 10**9, 4096)) == 0
+    idle = 10 * 395_000
+    g.retention_decay(idle); o.retention_decay(idle)                      # the drain rate is scaled too
+    compare_state(g, o)
+
+
+def test_capacity_geometry_two_million_accesses(hbf):
+    """2,048 queues, a batch of many tiles, the claim limit deep inside it, natives mixed in."""
+    ret = dict(RET, pages_per_block=8, blocks_per_plane=16, blocks_per_zone=4, disturb_limit=3, lead_threshold=1e9, max_pec=100)
+    g, o, prof = contexts(hbf, ret, geometry="capacity")
+    rng = np.random.default_rng(9)
+    n = 2_000_000
+    span_pages = 64 * 8 * 4 * 16 * 8
+    acc = mixed_batch(rng, n, 0, span_pages, gap=12)
+    assert compare_batch(g, o, acc) == 0
+    g.retention_advance(10**9, np.full(1, 50.0)); o.retention_advance(10**9, np.full(1, 50.0))
+    compare_state(g, o)
+    debt = o.retention_totals()["planned"]
+    assert 50_000 < debt < n
+    acc["issue_ns"] += 10**9
+    assert compare_batch(g, o, acc) == 0
+    assert o.retention_totals()["claimed"] == debt
+    acc["issue_ns"] += 10**9
+    assert compare_batch(g, o, acc) == 0                                  # no debt: the in-order path serves it
+
+
+def test_region_temperatures_from_the_thermal_field(hbf):
+    fp = wl.toy_floorplan(16, 48, 8, 4)
+    ret = dict(RET, lead_threshold=1e9)
+    g, o, prof = contexts(hbf, ret, floorplan=fp)
+    rng = np.random.default_rng(2)
+    ext = np.asarray(fp["ext_power_w"], np.float32) if "ext_power_w" in fp else None
+    t0 = 0
+    for _ in range(5):
+        acc = mixed_batch(rng, 20_000, t0, 4096, gap=100)
+        compare_batch(g, o, acc, rtol=2e-4)                              # 1e-3 K of field tolerance is 1.3e-4 of lifetime
+        t0 = int(acc["issue_ns"][-1]) + 1
+        g.thermal_step(1_000_000, ext); o.thermal_step(1_000_000, ext)
+        g.retention_advance(10**9); o.retention_advance(10**9)
+    bg, bo = g.retention_blocks(), o.retention_blocks()
+    assert bo["damage"].max() > bo["damage"].min() > 0                    # regions differ in temperature
+    assert np.allclose(bg["damage"], bo["damage"], rtol=2e-4)
+    assert g.retention_totals() == o.retention_totals()
+
+
+def test_forced_inorder_with_debt_is_refused_and_without_it_served(hbf):
+    ret = dict(RET, disturb_limit=1, lead_threshold=1e9)
+    g, o, prof = contexts(hbf, ret, path=hbf.PATH_INORDER)
+    rng = np.random.default_rng(3)
+    acc = mixed_batch(rng, 5000, 0, 4096, natives=0.0)
+    assert compare_batch(g, o, acc) == 0                                  # no debt yet
+    g.retention_advance(0, np.array([40.0]))
+    before = g.retention_totals()
+    acc["issue_ns"] += 10**9
+    rc, *_ = g.submit_host(acc, check=False)
+    assert rc == hbf.E_INVAL
+    assert g.retention_totals() == before
+
+
+def test_refused_batch_changes_nothing(hbf):
+    ret = dict(RET, disturb_limit=1, lead_threshold=1e9)
+    g, o, prof = contexts(hbf, ret)
+    compare_batch(g, o, recs([(0, 0, 64, 0), (PAGE * 9, 5, 64, 0)]))
+    g.retention_advance(0, np.array([40.0])); o.retention_advance(0, np.array([40.0]))
+    bad = recs([(PAGE, 10**7, 64, 0), (64 * wl.GIB - 32, 10**7, 64, 0), (2 * PAGE, 10**7, 64, 0)])
+    assert compare_batch(g, o, bad) == hbfo.E_ACCESS_FAULT
+    assert compare_batch(g, o, recs([(PAGE, 2 * 10**7, 64, 0)])) == 0
+
+
+def test_not_with_the_other_extensions(hbf):
+    g, o, prof = contexts(hbf, RET)
+    with pytest.raises(hbf.HbfError):
+        g.enable_channel_bus()
+    with pytest.raises(hbf.HbfError):
+        g.enable_energy_bins(1000, 4)
+    acc = recs([(0, 0, 64, 0)])
+    rc, *_ = g.submit_host(acc, check=False, parts_capacity=4)
+    assert rc == hbf.E_INVAL
+    g2 = hbf.Context(prof); g2.enable_channel_bus()
+    with pytest.raises(hbf.HbfError):
+        g2.enable_retention(**RET)
+
+
+def test_reset_clears_the_block_state(hbf):
+    ret = dict(RET, disturb_limit=1, lead_threshold=1e9)
+    g, o, prof = contexts(hbf, ret)
+    rng = np.random.default_rng(8)
+    compare_batch(g, o, mixed_batch(rng, 3000, 0, 4096))
+    g.retention_advance(10**9, np.array([60.0])); o.retention_advance(10**9, np.array([60.0]))
+    g.reset(); hbfo.lib().hbfo_reset(o._h)
+    compare_state(g, o)
+    assert g.retention_totals()["planned"] == 0
+    assert compare_batch(g, o, mixed_batch(rng, 3000, 0, 4096)) == 0
