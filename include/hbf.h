@@ -315,8 +315,7 @@ HBF_API int hbf_get_rom_temps(hbf_ctx *ctx, double *host_out, uint64_t cap);
  * hbf_submit_batch with retention on: the first (planned - claimed - decayed) modeled accesses of the batch, by
  *   index, claim one quantum each; d_die_stats[].busy_ns and the summary's service_ns include the claimed time,
  *   energy_pj does not (it goes to the pending thermal energy).  A refused batch claims nothing and disturbs
- *   nothing.  While quanta are outstanding the batch is served by the sort path; with hbf_set_path(HBF_PATH_INORDER)
- *   such a batch's result is HBF_E_INVAL.
+ *   nothing.  Every path applies the claims.
  * hbf_retention_decay: idle_ns of idle time drain floor(idle_ns / scaled quantum time) outstanding quanta.
  * hbf_get_retention_blocks / _plan / _totals synchronise the stream and copy to host memory: per-block arrays
  *   [n_blocks] (each nullable); the outstanding quanta in plan order (quanta == NULL: count only); the counters. */

@@ -127,13 +127,16 @@ __device__ __forceinline__ void row_wait2(int id, int64_t m, long long s8, const
                  "l"(m2), "l"(s82), "l"(pq2), "r"(pc2), "r"((int)last2) : "memory");
 }
 
-template <bool RESERVE>
+// DEBT = true (retention on): a modeled access with a batch index below the claim limit pays one refresh quantum (a page
+// read and a page program, scaled like any service, Eq. 3) before its own service; the streaming pass counts the
+// claims per die.
+template <bool RESERVE, bool DEBT>
 __global__ void __launch_bounds__(kInThreads, kInBlocksPerSM)
 k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_records, const RangeSnap *__restrict__ ranges_g,
                 const __grid_constant__ ModelParams mp_arg, const __grid_constant__ FastRange fast_arg, BatchCtrl *ctrl, uint8_t *__restrict__ status, int64_t *__restrict__ in_agg,
                 hbf_die_stats_t *stats_stage, int64_t *__restrict__ completion, int64_t *__restrict__ stall,
                 const int64_t *__restrict__ in_bin, InTile *in_tile, InHead *__restrict__ in_head, uint8_t *__restrict__ in_headcnt,
-                const int64_t *__restrict__ busy) {
+                const int64_t *__restrict__ busy, const unsigned long long *claim_limit_p, uint32_t *die_claims) {
     extern __shared__ __align__(16) unsigned char in_smem[];
     __shared__ long long s_red[2];
     __shared__ uint32_t s_heads_full;                     // queues whose head entries are complete
@@ -150,6 +153,9 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
     const Div64 div_q = ctrl->div_q;
     // one range, power-of-two geometry, transfer table, no thermal scaling in force: the short form of the terms
     const bool fast_on = fast_arg.on != 0u && mp_arg.pow2_geom != 0u && mp_arg.xfer_tab_max_cb != 0u && q_ppm == 1000000;
+    const uint64_t claim_limit = DEBT ? *claim_limit_p : 0ull;
+    const int64_t quantum_ns = !DEBT ? 0 : q_ppm == 1000000 ? mp_arg.t_read_ns + mp_arg.t_prog_ns
+        : (int64_t)div64((uint64_t)(mp_arg.t_read_ns + mp_arg.t_prog_ns) * 1000000ull + (uint64_t)q_ppm - 1ull, div_q);
 
     // [queues] x: busy-until of the run in progress; y: service time served in this tile << 8 | head-table entries written
     longlong2 *qst = reinterpret_cast<longlong2 *>(in_smem);
@@ -239,6 +245,10 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
                 v[u] = fast_on ? serve_terms_fast(fast_range, mp, addr[u], issue[u], bf[u])
                                  : serve_terms(rs, mp, addr[u], issue[u], bf[u], q_ppm, div_q);
             ready[u] = valid[u] && v[u].st == HBF_ST_READY;
+            if (DEBT && ready[u] && i[u] < claim_limit) {
+                v[u].s += quantum_ns;
+                if (!RESERVE) atomicAdd(&die_claims[v[u].die], 1u);
+            }
         }
         if (!RESERVE) {
 #pragma unroll
@@ -490,12 +500,13 @@ __device__ __forceinline__ uint32_t fast_queue(const FastRange &f, const ModelPa
     return mp.queue_level == 0u ? die * mp.planes + pl : die;
 }
 
+template <bool DEBT>
 __global__ void __launch_bounds__(kInStrThreads)
 k_inorder_straggle(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_records,
                    const RangeSnap *__restrict__ ranges_g, const __grid_constant__ ModelParams mp_arg,
                    const __grid_constant__ FastRange fast_arg, BatchCtrl *ctrl,
                    const int64_t *__restrict__ in_bin, const uint8_t *__restrict__ in_headcnt, int64_t *completion,
-                   int64_t *stall, InTile *in_tile) {
+                   int64_t *stall, InTile *in_tile, const unsigned long long *claim_limit_p) {
     extern __shared__ __align__(16) unsigned char str_smem[];
     __shared__ ModelParams mp;
     __shared__ FastRange fast_range;
@@ -530,6 +541,9 @@ k_inorder_straggle(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t ti
     const Div64 div_q = ctrl->div_q;
     const bool one_range = fast_arg.on != 0u && mp_arg.pow2_geom != 0u;
     const bool fast_terms = one_range && mp_arg.xfer_tab_max_cb != 0u && q_ppm == 1000000;
+    const uint64_t claim_limit = DEBT ? *claim_limit_p : 0ull;     // as in the serve pass
+    const int64_t quantum_ns = !DEBT ? 0 : q_ppm == 1000000 ? mp_arg.t_read_ns + mp_arg.t_prog_ns
+        : (int64_t)div64((uint64_t)(mp_arg.t_read_ns + mp_arg.t_prog_ns) * 1000000ull + (uint64_t)q_ppm - 1ull, div_q);
     const uint64_t tile_begin = (uint64_t)tile * tile_records, tile_end = min(n, tile_begin + tile_records);
     long long dstall = 0, max_c = INT64_MIN;
     __syncthreads();
@@ -594,8 +608,9 @@ k_inorder_straggle(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t ti
                 const uint64_t *rec = reinterpret_cast<const uint64_t *>(acc + cbase + e);
                 const int64_t issue = (int64_t)__ldg(rec + 1);
                 const uint64_t bf = __ldg(rec + 2);
-                const Served v = fast_terms ? serve_terms_fast(fast_range, mp, addr[j], issue, bf)
-                                            : serve_terms(rs, mp, addr[j], issue, bf, q_ppm, div_q);
+                Served v = fast_terms ? serve_terms_fast(fast_range, mp, addr[j], issue, bf)
+                                      : serve_terms(rs, mp, addr[j], issue, bf, q_ppm, div_q);
+                if (DEBT && cbase + e < claim_limit) v.s += quantum_ns;
                 const uint32_t pos = s_cells[j * kInStrWarps + warp] + rk[j];
                 ent_as[pos] = make_longlong2(issue, v.s);
                 ent_pq[pos] = make_uint2((uint32_t)v.xfer | (v.op << 31), v.queue | (e << 16));
@@ -675,29 +690,37 @@ cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st) {
     const size_t smem_serve = inorder_serve_smem(nd), smem_str = inorder_straggle_smem();
     static size_t set_serve = 0;
     if (smem_serve > set_serve) {
-        cudaError_t e = cudaFuncSetAttribute(k_inorder_serve<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_serve);
+        const void *serve_fns[4] = {(const void *)k_inorder_serve<false, false>, (const void *)k_inorder_serve<true, false>,
+                                    (const void *)k_inorder_serve<false, true>, (const void *)k_inorder_serve<true, true>};
+        for (const void *f : serve_fns) {
+            cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_serve);
+            if (e != cudaSuccess) return e;
+        }
+        cudaError_t e = cudaFuncSetAttribute(k_inorder_straggle<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_str);
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(k_inorder_serve<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_serve);
-        if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(k_inorder_straggle, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_str);
+        e = cudaFuncSetAttribute(k_inorder_straggle<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_str);
         if (e != cudaSuccess) return e;
         set_serve = smem_serve;
     }
     InTile *tiles = reinterpret_cast<InTile *>(a.ws.in_tile);
     InHead *heads = reinterpret_cast<InHead *>(a.ws.in_head);
-    k_inorder_serve<false><<<n_tiles, kInThreads, smem_serve, st>>>(a.acc, n, tile_records, a.ranges, a.mp, a.fast, a.ctrl, a.status,
-                                                                    a.ws.in_agg, a.stats_stage, a.completion, a.stall, a.ws.in_bin,
-                                                                    tiles, heads, a.ws.in_headcnt, a.busy);
+    const bool debt = a.claim_limit != nullptr;              // retention on: the kernels that apply the claims
+    auto serve = [&](bool reserve) {
+        auto k = reserve ? (debt ? k_inorder_serve<true, true> : k_inorder_serve<true, false>)
+                         : (debt ? k_inorder_serve<false, true> : k_inorder_serve<false, false>);
+        k<<<n_tiles, kInThreads, smem_serve, st>>>(a.acc, n, tile_records, a.ranges, a.mp, a.fast, a.ctrl, a.status, a.ws.in_agg,
+                                                   a.stats_stage, a.completion, a.stall, a.ws.in_bin, tiles, heads, a.ws.in_headcnt,
+                                                   a.busy, a.claim_limit, a.die_claims);
+    };
+    serve(false);
     k_inorder_scan<<<(R + kInScanThreads - 1) / kInScanThreads, kInScanThreads, 0, st>>>(
         a.ctrl, a.mp_dev, n_tiles, a.ws.in_agg, a.ws.in_bin, a.busy, a.busy_stage, a.stats_stage, a.path == HBF_PATH_INORDER ? 1 : 0);
     const uint64_t fix_threads = (uint64_t)n_tiles * R;
     k_inorder_fixup<<<(unsigned)((fix_threads + kInFixThreads - 1) / kInFixThreads), kInFixThreads, 0, st>>>(
         R, n_tiles, a.ctrl, a.ws.in_bin, heads, a.ws.in_headcnt, a.completion, a.stall, tiles);
-    k_inorder_straggle<<<n_tiles, kInStrThreads, smem_str, st>>>(a.acc, n, tile_records, a.ranges, a.mp, a.fast, a.ctrl, a.ws.in_bin,
-                                                                a.ws.in_headcnt, a.completion, a.stall, tiles);
-    k_inorder_serve<true><<<n_tiles, kInThreads, smem_serve, st>>>(a.acc, n, tile_records, a.ranges, a.mp, a.fast, a.ctrl, a.status,
-                                                                   a.ws.in_agg, a.stats_stage, a.completion, a.stall, a.ws.in_bin,
-                                                                   tiles, heads, a.ws.in_headcnt, a.busy);
+    (debt ? k_inorder_straggle<true> : k_inorder_straggle<false>)<<<n_tiles, kInStrThreads, smem_str, st>>>(
+        a.acc, n, tile_records, a.ranges, a.mp, a.fast, a.ctrl, a.ws.in_bin, a.ws.in_headcnt, a.completion, a.stall, tiles, a.claim_limit);
+    serve(true);
     k_inorder_total<<<1, 256, 0, st>>>(a.ctrl, tiles, n_tiles);
     g_kernel_launches += 6;
     return cudaGetLastError();

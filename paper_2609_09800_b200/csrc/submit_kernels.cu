@@ -18,15 +18,12 @@ namespace hbf {
 //         sort path when the in-order attempt found the records out of issue order, else does nothing.
 __global__ void k_begin(BatchCtrl *ctrl, const DevState *state, const int64_t *busy, int64_t *busy_stage,
                         hbf_die_stats_t *stats_stage, uint32_t *hist, uint32_t n_queues, uint32_t n_dies,
-                        int role, int run_sort, const unsigned long long *claim_limit, int sort_available) {
+                        int role, int run_sort, uint32_t *die_claims) {
     const int tid = threadIdx.x;
     if (role == 1) {
         if (ctrl->skip || !ctrl->run_sort) return;
         run_sort = 1;
     }
-    // refresh quanta to be claimed (retention on): the claims are applied by the sort path
-    const bool claims = claim_limit != nullptr && *claim_limit != 0ull;
-    if (claims) run_sort = 1;
     __syncthreads();
     uint32_t *w = reinterpret_cast<uint32_t *>(ctrl);
     for (int i = tid; i < (int)(sizeof(BatchCtrl) / 4); i += blockDim.x) w[i] = 0u;
@@ -40,12 +37,13 @@ __global__ void k_begin(BatchCtrl *ctrl, const DevState *state, const int64_t *b
         if (state->poisoned) { ctrl->code = HBF_E_TIMEOUT; ctrl->skip = 1; }
         else if (mode == HBF_MODE_SHUTDOWN) { ctrl->code = HBF_E_LINK_SHUTDOWN; ctrl->skip = 1; }
         else if (mode == HBF_MODE_SEVERE) { ctrl->code = HBF_E_THROTTLED; ctrl->skip = 1; }
-        else if (claims && !sort_available) { ctrl->code = HBF_E_INVAL; ctrl->skip = 1; }
     }
     for (uint32_t r = tid; r < n_queues; r += blockDim.x) busy_stage[r] = busy[r];
     int64_t *s = reinterpret_cast<int64_t *>(stats_stage);
     for (uint32_t i = tid; i < n_dies * 6u; i += blockDim.x) s[i] = 0;
     for (int i = tid; i < kMaxPasses * kRadix; i += blockDim.x) hist[i] = 0u;
+    if (die_claims)                                          // retention on: an in-order attempt that was handed over counted some
+        for (uint32_t d = tid; d < n_dies; d += blockDim.x) die_claims[d] = 0u;
 }
 
 // =====================================================================================================
@@ -1000,7 +998,7 @@ cudaError_t launch_submit(const SubmitArgs &a, cudaStream_t st) {
     const bool sort_kernels = a.path != HBF_PATH_INORDER || !a.inorder_ok;
     mark(0);
     k_begin<<<1, 256, 0, st>>>(a.ctrl, a.state, a.busy, a.busy_stage, a.stats_stage, a.ws.hist, a.mp.n_queues, a.mp.n_dies,
-                               0, try_inorder ? 0 : 1, a.claim_limit, sort_kernels ? 1 : 0);
+                               0, try_inorder ? 0 : 1, a.die_claims);
     g_kernel_launches += 1;
     if (n > 0) {
         if (try_inorder) {
@@ -1010,7 +1008,7 @@ cudaError_t launch_submit(const SubmitArgs &a, cudaStream_t st) {
             mark(8);
             if (sort_kernels) {
                 k_begin<<<1, 256, 0, st>>>(a.ctrl, a.state, a.busy, a.busy_stage, a.stats_stage, a.ws.hist, a.mp.n_queues,
-                                           a.mp.n_dies, 1, 1, a.claim_limit, 1);
+                                           a.mp.n_dies, 1, 1, a.die_claims);
                 g_kernel_launches += 1;
             }
         }

@@ -215,18 +215,30 @@ def test_region_temperatures_from_the_thermal_field(hbf):
     assert g.retention_totals() == o.retention_totals()
 
 
-def test_forced_inorder_with_debt_is_refused_and_without_it_served(hbf):
-    ret = dict(RET, disturb_limit=1, lead_threshold=1e9)
+@pytest.mark.parametrize("rho_gap", [400, 40])
+def test_forced_inorder_path_applies_the_claims(hbf, rho_gap):
+    """The in-order kernels (serve, fix-up, straggle, re-serve) with claims; the dense case backlogs every queue."""
+    ret = dict(RET, disturb_limit=1, lead_threshold=1e9, pages_per_block=128)
     g, o, prof = contexts(hbf, ret, path=hbf.PATH_INORDER)
     rng = np.random.default_rng(3)
-    acc = mixed_batch(rng, 5000, 0, 4096, natives=0.0)
+    acc = mixed_batch(rng, 50_000, 0, 65536, gap=rho_gap)               # touches every tracked block
     assert compare_batch(g, o, acc) == 0                                  # no debt yet
-    g.retention_advance(0, np.array([40.0]))
-    before = g.retention_totals()
-    acc["issue_ns"] += 10**9
-    rc, *_ = g.submit_host(acc, check=False)
-    assert rc == hbf.E_INVAL
-    assert g.retention_totals() == before
+    g.retention_advance(0, np.array([40.0])); o.retention_advance(0, np.array([40.0]))
+    for k in range(3):                                                    # the debt ends inside the third batch
+        acc = mixed_batch(rng, 30_000, 10**9 * (k + 1) if rho_gap == 400 else int(acc["issue_ns"][-1]) + 1, 4096, gap=rho_gap)
+        assert compare_batch(g, o, acc) == 0
+    assert o.retention_totals()["claimed"] == o.retention_totals()["planned"] > 30_000
+
+
+def test_unsorted_batch_with_debt_goes_to_the_sort_path_and_counts_claims_once(hbf):
+    ret = dict(RET, disturb_limit=1, lead_threshold=1e9)
+    g, o, prof = contexts(hbf, ret)
+    rng = np.random.default_rng(13)
+    compare_batch(g, o, mixed_batch(rng, 20_000, 0, 4096))
+    g.retention_advance(0, np.array([40.0])); o.retention_advance(0, np.array([40.0]))
+    acc = mixed_batch(rng, 20_000, 10**9, 4096)
+    acc = acc[rng.permutation(acc.shape[0])]                              # out of issue order: the in-order attempt is abandoned
+    assert compare_batch(g, o, acc) == 0
 
 
 def test_refused_batch_changes_nothing(hbf):
