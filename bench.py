@@ -52,10 +52,12 @@ def parse_args():
     ap.add_argument("--cpu-sample", type=int, default=20_000_000)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--workload", default="capacity_mode", choices=["capacity_mode", "coupled_thermal", "capacity_paged", "rom"],
+    ap.add_argument("--workload", default="capacity_mode", choices=["capacity_mode", "coupled_thermal", "capacity_paged", "rom", "capacity_retention"],
                     help="coupled_thermal: the prefix-KV stream in 1 ms batches, each followed by a thermal step; "
                          "capacity_paged: the capacity-mode batch through the page-granular submit; rom: fit the reduced-order "
-                         "thermal model of the package floorplan and time its step against the full grid (none is the headline)")
+                         "thermal model of the package floorplan and time its step against the full grid; capacity_retention: the "
+                         "capacity-mode batch with retention on: a batch without debt, an epoch (damage, eligibility, plan), the "
+                         "same batch paying refresh claims (none is the headline)")
     ap.add_argument("--horizon-ms", type=int, default=1000, help="simulated time of the coupled_thermal run")
     ap.add_argument("--channel-bus", action="store_true",
                     help="capacity_mode: also run the channel-bus stage (reads' transfers queue per channel); not the headline")
@@ -301,6 +303,76 @@ def run_paged(args):
     print(json.dumps(line), flush=True)
 
 
+def run_retention(args):
+    """The capacity-mode batch with retention, refresh and wear on (one GPU).  A step: reset; the batch on a device without
+    refresh debt (claim window, service, read disturb, commit scan); one epoch at 60 C with a read-disturb limit of one
+    page read, so that every block the batch touched becomes eligible and its pages join the plan; the same batch again,
+    its first accesses now claiming one refresh quantum each."""
+    import torch
+    from paper_2609_09800_b200 import build as hbf_build, hbf
+    hbf_build.build()
+    n = args.n
+    w, gen_s = make_stream(n, seed=0)
+    fp = wl.package_floorplan(channels=w.profile["channels"], dies=w.profile["dies"])
+    ctx = hbf.Context(w.profile, fp)
+    for r in w.ranges:
+        ctx.register_range(*r)
+    ret = dict(pages_per_block=256, blocks_per_plane=64, blocks_per_zone=8, max_pec=3000, disturb_limit=1,
+               l_ref_s=3.15e7, t_ref_c=40.0, ea_ev=1.04, accel=1.0, lead_threshold=0.8)
+    ctx.enable_retention(**ret)
+    temps = np.full(len(fp["region_kind"]), 60.0)
+    d_acc = torch.from_numpy(w.acc.view(np.int64).reshape(-1)).cuda()
+    d_comp = torch.empty(n, dtype=torch.int64, device="cuda"); d_stall = torch.empty_like(d_comp)
+    d_status = torch.empty(n, dtype=torch.uint8, device="cuda")
+    d_stats = torch.empty(ctx.n_dies * 6, dtype=torch.int64, device="cuda")
+    ws = torch.empty(ctx.workspace_bytes(n), dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+
+    def submit():
+        rc = ctx.submit_batch(d_acc, n, d_comp, d_stall, d_status, d_stats, ws)
+        assert rc == 0, rc
+
+    def timed(k):
+        t = np.zeros(3)
+        for _ in range(k):
+            ctx.reset()
+            ev[0].record(stream); submit()
+            ev[1].record(stream); ctx.retention_advance(1_000_000_000, temps)
+            ev[2].record(stream); submit()
+            ev[3].record(stream); ev[3].synchronize()
+            t += [ev[i].elapsed_time(ev[i + 1]) for i in range(3)]
+        return t
+    timed(args.warmup)
+    res = ctx.last_result()
+    assert res["code"] == 0, res
+    tot = ctx.retention_totals()
+    l0 = hbf.kernel_launches()
+    t = timed(args.steps)
+    launches = hbf.kernel_launches() - l0
+    ms = float(t.sum())
+    peak, kind = measured_peak()
+    rate = 2 * n * args.steps / (ms * 1e-3)
+    # per batch: the records in, completion + stall + status out (41 B), the records in again for the read-disturb pass (24 B)
+    moved = 2 * (41 + 24) * n
+    line = {"metric": METRIC, "value": rate, "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64",
+            "data": "synthetic",
+            "config": {"workload": "capacity_mode_retention", "accesses_per_step": 2 * n, "geometry": "64x8x4", "queues": 2048,
+                       "blocks": tot["n_blocks"], "pages_per_block": ret["pages_per_block"], "gen_seconds": round(gen_s, 1),
+                       "state": "reset at the start of every step; two batches and one epoch per step"},
+            "gpu_launches": int(launches),
+            "retention": {"batch_without_debt_ms": t[0] / args.steps, "epoch_ms": t[1] / args.steps,
+                          "batch_with_claims_ms": t[2] / args.steps, "quanta_planned_per_epoch": tot["planned"],
+                          "quanta_claimed_by_the_batch": tot["claimed"], "blocks_committed": tot["commits"]},
+            "roofline": {"bound": "hbm", "kernel": "submit with retention, all kernels", "achieved": moved * args.steps / (ms * 1e-3) / 1e9,
+                         "peak": peak, "peak_kind": kind, "unit": "GB/s",
+                         "frac": moved * args.steps / (ms * 1e-3) / 1e9 / peak, "traffic": None,
+                         "algorithmic_bytes_per_access": 65},
+            "batch_result": {k: res[k] for k in ("n_modeled", "n_native", "max_completion_ns")}}
+    print(json.dumps(line), flush=True)
+
+
 def run_rom(args):
     """Fits the 224-state reduced-order thermal model (Eq. 2) of the package floorplan from the CUDA grid's unit-step
     responses (10 ms steps), compares it with the grid on three input shapes, and times both."""
@@ -365,6 +437,10 @@ def main():
     if args.workload == "rom":
         if rank == 0:
             run_rom(args)
+        return
+    if args.workload == "capacity_retention":
+        if rank == 0:
+            run_retention(args)
         return
     if args.workload == "coupled_thermal":
         if rank == 0:

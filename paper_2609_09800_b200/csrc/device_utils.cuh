@@ -115,6 +115,28 @@ __device__ __forceinline__ Decoded decode(const ModelParams &mp, uint64_t off, u
     return d;
 }
 
+// ---- retention: block (erase unit) that holds a media offset's page: ((channel, die, plane) * blocks_per_plane + block)
+__device__ __forceinline__ uint64_t ret_block_of(const ModelParams &mp, const RetDev &r, uint64_t off) {
+    const uint64_t u = off >> mp.stripe_shift;
+    uint32_t ch, di, pl; uint64_t row;
+    if (mp.pow2_geom) {
+        ch = (uint32_t)u & (mp.channels - 1u);
+        di = (uint32_t)(u >> mp.ch_shift) & (mp.dies - 1u);
+        pl = (uint32_t)(u >> (mp.ch_shift + mp.die_shift)) & (mp.planes - 1u);
+        row = u >> (mp.ch_shift + mp.die_shift + mp.plane_shift);
+    } else {
+        ch = (uint32_t)(u % mp.channels);
+        uint64_t v = u / mp.channels;
+        di = (uint32_t)(v % mp.dies); v /= mp.dies;
+        pl = (uint32_t)(v % mp.planes); row = v / mp.planes;
+    }
+    const uint64_t in_stripe = (off & ((1ull << mp.stripe_shift) - 1ull)) >> mp.page_shift;
+    const uint64_t page = (row << mp.pages_per_stripe_shift) + in_stripe;
+    const uint64_t blk = div64(page, r.div_ppb);             // page < 2^63 always
+    const uint64_t bip = blk - div64(blk, r.div_bpp) * r.bpp;
+    return (((uint64_t)ch * mp.dies + di) * mp.planes + pl) * r.bpp + bip;
+}
+
 // ---- service terms (Eq. 3 for the array time; transfer is pure latency) ---------------------------
 
 struct Terms { int64_t s, xfer, energy, cb; };

@@ -431,7 +431,7 @@ int hbf_submit_batch(hbf_ctx *c, const hbf_access_t *d_acc, uint64_t n, int64_t 
     a.binned = c->bin_ns != 0;
     if (c->ret_on) {                                         // how far the outstanding refresh quanta reach into this batch
         CK(launch_ret_window(d_acc, n, c->d_ranges, c->ret, c->sm_count, c->stream));
-        a.claim_limit = &c->ret.st->claim_limit; a.die_claims = c->ret.die_claims;
+        a.claim_limit = &c->ret.st->claim_limit; a.die_claims = c->ret.die_claims; a.ret = &c->ret;
     }
     CK(launch_submit(a, c->stream));
     if (c->ret_on)                                           // read disturb, commits, the claimed energy
@@ -524,6 +524,7 @@ int hbf_enable_retention(hbf_ctx *c, const hbf_retention_config_t *cfg) {
     RetDev r{};
     r.ppb = cfg->pages_per_block; r.bpp = cfg->blocks_per_plane; r.bpz = cfg->blocks_per_zone; r.max_pec = cfg->max_pec;
     r.disturb_limit = cfg->disturb_limit; r.n_regions = c->thermal ? c->td.n_regions : 1u;
+    r.div_ppb = make_div64_host(cfg->pages_per_block); r.div_bpp = make_div64_host(cfg->blocks_per_plane);
     r.accel = cfg->accel; r.lead = cfg->lead_threshold; r.l_ref_s = cfg->l_ref_s; r.t_ref_k = cfg->t_ref_c + 273.15;
     r.ea_over_kb = cfg->ea_ev / 8.617333262e-5;                             // Boltzmann constant in eV/K
     r.n_blocks = nb; r.plan_cap = nb * cfg->pages_per_block;

@@ -108,6 +108,7 @@ struct SubmitArgs {
     int binned;                          // the batch's energy goes to the time-bin ledger, not to the pending totals
     const unsigned long long *claim_limit;  // retention on: batch index below which a modeled access claims a refresh quantum
     uint32_t *die_claims;                   // retention on: [dies] claims of the batch
+    const struct RetDev *ret;               // retention on: the block state (host copy of the device pointers)
     cudaEvent_t *ev;                     // [kProfEvents] or null: recorded between kernel groups
 };
 constexpr int kProfEvents = 10;
@@ -171,10 +172,12 @@ struct RetState {
     unsigned long long claims_now;       // quanta this batch claims if it is accepted
     unsigned long long tickets, counted; // the claim window's tile counter and the modeled accesses counted so far
     unsigned long long epoch_total;      // quanta the epoch in progress adds
-    uint32_t epoch, pad;
+    uint32_t epoch;
+    uint32_t observed_inline;            // the in-order serve pass has counted this batch's reads into the disturb counters
 };
 struct RetDev {
     uint32_t ppb, bpp, bpz, max_pec, disturb_limit, n_regions;
+    Div64 div_ppb, div_bpp;              // exact division by pages_per_block and by blocks_per_plane
     double accel, lead, l_ref_s, t_ref_k, ea_over_kb;
     uint64_t n_blocks, plan_cap;
     double *damage; uint32_t *disturb, *pec, *epoch_of; uint8_t *worn;

@@ -136,7 +136,8 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
                 const __grid_constant__ ModelParams mp_arg, const __grid_constant__ FastRange fast_arg, BatchCtrl *ctrl, uint8_t *__restrict__ status, int64_t *__restrict__ in_agg,
                 hbf_die_stats_t *stats_stage, int64_t *__restrict__ completion, int64_t *__restrict__ stall,
                 const int64_t *__restrict__ in_bin, InTile *in_tile, InHead *__restrict__ in_head, uint8_t *__restrict__ in_headcnt,
-                const int64_t *__restrict__ busy, const unsigned long long *claim_limit_p, uint32_t *die_claims) {
+                const int64_t *__restrict__ busy, const unsigned long long *claim_limit_p, uint32_t *die_claims,
+                const __grid_constant__ RetDev ret) {
     extern __shared__ __align__(16) unsigned char in_smem[];
     __shared__ long long s_red[2];
     __shared__ uint32_t s_heads_full;                     // queues whose head entries are complete
@@ -148,6 +149,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const RangeSnap &rs = *ranges_g;                      // read through the cache; the common configuration does not touch it
     if (tid == 0) { mp = mp_arg; fast_range = fast_arg; }
+    if (DEBT && !RESERVE && tid == 0 && blockIdx.x == 0) ret.st->observed_inline = 1u;
     const uint32_t R = mp_arg.n_queues, n_dies = mp_arg.n_dies;
     const int64_t q_ppm = ctrl->q_ppm;
     const Div64 div_q = ctrl->div_q;
@@ -248,6 +250,14 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
             if (DEBT && ready[u] && i[u] < claim_limit) {
                 v[u].s += quantum_ns;
                 if (!RESERVE) atomicAdd(&die_claims[v[u].die], 1u);
+            }
+            if (DEBT && !RESERVE && ready[u] && !v[u].op) {  // read disturb: the read's pages, on the block of its first page
+                uint64_t off;
+                if (fast_on) off = fast_range.media_offset + (addr[u] - fast_range.base);
+                else { int g = 0; classify(rs, addr[u], issue[u], (uint32_t)bf[u], (uint32_t)(bf[u] >> 32), &g); off = rs.media_offset[g] + (addr[u] - rs.base[g]); }
+                const uint32_t page_mask = (1u << mp.page_shift) - 1u;
+                const uint32_t npages = (uint32_t)(((uint64_t)((uint32_t)off & page_mask) + (uint32_t)bf[u] + page_mask) >> mp.page_shift);
+                atomicAdd(&ret.disturb[ret_block_of(mp, ret, off)], npages);
             }
         }
         if (!RESERVE) {
@@ -710,7 +720,7 @@ cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st) {
                          : (debt ? k_inorder_serve<false, true> : k_inorder_serve<false, false>);
         k<<<n_tiles, kInThreads, smem_serve, st>>>(a.acc, n, tile_records, a.ranges, a.mp, a.fast, a.ctrl, a.status, a.ws.in_agg,
                                                    a.stats_stage, a.completion, a.stall, a.ws.in_bin, tiles, heads, a.ws.in_headcnt,
-                                                   a.busy, a.claim_limit, a.die_claims);
+                                                   a.busy, a.claim_limit, a.die_claims, debt ? *a.ret : RetDev{});
     };
     serve(false);
     k_inorder_scan<<<(R + kInScanThreads - 1) / kInScanThreads, kInScanThreads, 0, st>>>(

@@ -17,27 +17,6 @@
 
 namespace hbf {
 
-// block (erase unit) that holds a media offset's page: ((channel, die, plane) * blocks_per_plane + block)
-__device__ __forceinline__ uint64_t ret_block_of(const ModelParams &mp, const RetDev &r, uint64_t off) {
-    const uint64_t u = off >> mp.stripe_shift;
-    uint32_t ch, di, pl; uint64_t row;
-    if (mp.pow2_geom) {
-        ch = (uint32_t)u & (mp.channels - 1u);
-        di = (uint32_t)(u >> mp.ch_shift) & (mp.dies - 1u);
-        pl = (uint32_t)(u >> (mp.ch_shift + mp.die_shift)) & (mp.planes - 1u);
-        row = u >> (mp.ch_shift + mp.die_shift + mp.plane_shift);
-    } else {
-        ch = (uint32_t)(u % mp.channels);
-        uint64_t v = u / mp.channels;
-        di = (uint32_t)(v % mp.dies); v /= mp.dies;
-        pl = (uint32_t)(v % mp.planes); row = v / mp.planes;
-    }
-    const uint64_t in_stripe = (off & ((1ull << mp.stripe_shift) - 1ull)) >> mp.page_shift;
-    const uint64_t page = (row << mp.pages_per_stripe_shift) + in_stripe;
-    const uint64_t bip = (page / r.ppb) % r.bpp;
-    return (((uint64_t)ch * mp.dies + di) * mp.planes + pl) * r.bpp + bip;
-}
-
 __device__ __forceinline__ bool ret_ready(const RangeSnap &rs, const hbf_access_t *acc, uint64_t i, uint64_t *off, uint32_t *bytes, uint32_t *op) {
     const uint64_t *rec = reinterpret_cast<const uint64_t *>(acc + i);
     const uint64_t addr = __ldg(rec), bf = __ldg(rec + 2);
@@ -168,12 +147,17 @@ cudaError_t launch_ret_window(const hbf_access_t *acc, uint64_t n, const RangeSn
 // =====================================================================================================
 // after the batch: read disturb, commits, bookkeeping
 // =====================================================================================================
+// The in-order serve pass counts the reads into the disturb counters as it streams the batch (observed_inline).  This
+// pass covers the other cases: the batch was served without that pass (count now), or the pass ran and the batch was
+// then refused (take the counts back: the same reads, the same amounts).
 __global__ void __launch_bounds__(256)
 k_ret_observe(const hbf_access_t *__restrict__ acc, uint64_t n, const RangeSnap *__restrict__ ranges_g,
               const ModelParams *__restrict__ mp_g, const hbf_batch_result_t *result, RetDev r) {
     __shared__ RangeSnap rs;
     __shared__ ModelParams mp;
-    if (result->code != HBF_OK) return;
+    const bool ok = result->code == HBF_OK, inline_done = r.st->observed_inline != 0u;
+    if (ok == inline_done) return;                           // counted and accepted, or neither
+    const bool undo = inline_done;
     load_ranges(&rs, ranges_g);
     for (int i = threadIdx.x; i < (int)(sizeof(ModelParams) / 4); i += blockDim.x)
         reinterpret_cast<uint32_t *>(&mp)[i] = reinterpret_cast<const uint32_t *>(mp_g)[i];
@@ -184,7 +168,7 @@ k_ret_observe(const hbf_access_t *__restrict__ acc, uint64_t n, const RangeSnap 
         if (!ret_ready(rs, acc, i, &off, &bytes, &op) || op) continue;
         const uint64_t in_page = off & ((1ull << mp.page_shift) - 1ull);
         const uint32_t npages = (uint32_t)((in_page + bytes + (1ull << mp.page_shift) - 1ull) >> mp.page_shift);
-        atomicAdd(&r.disturb[ret_block_of(mp, r, off)], npages);
+        atomicAdd(&r.disturb[ret_block_of(mp, r, off)], undo ? 0u - npages : npages);
     }
 }
 
@@ -214,7 +198,7 @@ __global__ void k_ret_close(const hbf_batch_result_t *result, int64_t *pending, 
     if (threadIdx.x == 0) {
         RetState *st = r.st;
         if (ok) st->claimed += st->claims_now;
-        st->claims_now = 0ull; st->claim_limit = 0ull;
+        st->claims_now = 0ull; st->claim_limit = 0ull; st->observed_inline = 0u;
     }
 }
 
@@ -318,32 +302,34 @@ __global__ void k_ret_chan(RetDev r, uint32_t channels, uint32_t dies) {
     if (threadIdx.x == 0) r.st->epoch_total = s_total;
 }
 
+// one warp per block, its lanes over the block's pages
 __global__ void __launch_bounds__(256)
 k_ret_emit(RetDev r, uint32_t channels, uint32_t dies, uint32_t planes) {
     const RetState *st = r.st;
     const uint32_t epoch = st->epoch;
     const unsigned long long base = st->planned;
     const uint32_t blocks_per_die = planes * r.bpp;
-    const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
-    for (uint64_t b = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; b < r.n_blocks; b += stride) {
+    const int lane = threadIdx.x & 31;
+    const uint64_t warps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+    for (uint64_t b = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; b < r.n_blocks; b += warps) {
         if (r.epoch_of[b] != epoch) continue;
         const uint32_t die = (uint32_t)(b / blocks_per_die), ch = die / dies, di = die % dies;
-        unsigned long long pos = 0;
-        for (uint32_t pg = 0; pg < r.ppb; ++pg) {
-            const unsigned long long r_die = (unsigned long long)r.rank[b] * r.ppb + pg;
+        const unsigned long long first = (unsigned long long)r.rank[b] * r.ppb;
+        for (uint32_t pg = (uint32_t)lane; pg < r.ppb; pg += 32u) {
+            const unsigned long long r_die = first + pg;
             unsigned long long r_ch = 0;
             for (uint32_t d = 0; d < dies; ++d) {
                 const unsigned long long len = r.die_len[ch * dies + d];
                 r_ch += min(len, r_die) + ((d < di && len > r_die) ? 1ull : 0ull);
             }
-            pos = 0;
+            unsigned long long pos = 0;
             for (uint32_t c = 0; c < channels; ++c) {
                 const unsigned long long len = r.chan_len[c];
                 pos += min(len, r_ch) + ((c < ch && len > r_ch) ? 1ull : 0ull);
             }
             r.plan[(base + pos) % r.plan_cap] = (uint32_t)(b * r.ppb + pg);
+            if (pg + 1u == r.ppb) r.last_pos[b] = base + pos;       // the last page's place: a block's pages go out in order
         }
-        r.last_pos[b] = base + pos;                         // the last page's place: a block's pages go out in order
     }
 }
 
@@ -364,7 +350,7 @@ cudaError_t launch_ret_advance(const RetDev &r, const ModelParams &mp, const The
     k_ret_damage<<<ret_grid(r.n_blocks, sm_count), 256, 0, st>>>(r, die_region, mp.planes * r.bpp);
     k_ret_rank<<<mp.n_dies, kRetRankThreads, 0, st>>>(r, mp.planes);
     k_ret_chan<<<1, 256, 0, st>>>(r, mp.channels, mp.dies);
-    k_ret_emit<<<ret_grid(r.n_blocks, sm_count), 256, 0, st>>>(r, mp.channels, mp.dies, mp.planes);
+    k_ret_emit<<<ret_grid(r.n_blocks * 32, sm_count), 256, 0, st>>>(r, mp.channels, mp.dies, mp.planes);
     k_ret_epoch_close<<<1, 1, 0, st>>>(r);
     g_kernel_launches += 6;
     return cudaGetLastError();
