@@ -164,6 +164,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
     uint32_t *st_br_lo = reinterpret_cast<uint32_t *>(qst + kInMaxQueues), *st_br_hi = st_br_lo + n_dies;   // per die
     uint32_t *st_bp_lo = st_br_hi + n_dies, *st_bp_hi = st_bp_lo + n_dies;
     uint32_t *st_nr = st_bp_hi + n_dies, *st_np = st_nr + n_dies;
+    uint32_t *st_claims = st_np + n_dies;                 // refresh quanta claimed on each die (claims variant)
 
     const uint32_t tile = blockIdx.x;
     const uint64_t tile_begin = (uint64_t)tile * tile_records;
@@ -174,7 +175,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
         __syncthreads();
         for (uint32_t q = tid; q < R; q += kInThreads) qst[q].x = in_bin[(uint64_t)blockIdx.x * R + q];
     } else {
-        for (uint32_t d = tid; d < n_dies * 6u; d += kInThreads) st_br_lo[d] = 0u;
+        for (uint32_t d = tid; d < n_dies * 7u; d += kInThreads) st_br_lo[d] = 0u;
         if (blockIdx.x == 0) {                               // the first tile knows its entering state: it is served exactly
             __syncthreads();
             for (uint32_t q = tid; q < R; q += kInThreads) qst[q].x = busy[q];
@@ -249,7 +250,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
             ready[u] = valid[u] && v[u].st == HBF_ST_READY;
             if (DEBT && ready[u] && i[u] < claim_limit) {
                 v[u].s += quantum_ns;
-                if (!RESERVE) atomicAdd(&die_claims[v[u].die], 1u);
+                if (!RESERVE) atomicAdd(&st_claims[v[u].die], 1u);
             }
             if (DEBT && !RESERVE && ready[u] && !v[u].op) {  // read disturb: the read's pages, on the block of its first page
                 uint64_t off;
@@ -366,6 +367,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
             if (bp) atomicAdd(&g[2], bp);
             if (st_nr[d]) atomicAdd(&g[4], (unsigned long long)st_nr[d]);
             if (st_np[d]) atomicAdd(&g[5], (unsigned long long)st_np[d]);
+            if (DEBT && st_claims[d]) atomicAdd(&die_claims[d], st_claims[d]);
         }
         c_native = (unsigned long long)warp_sum((long long)c_native);
         c_ready = (unsigned long long)warp_sum((long long)c_ready);
@@ -686,7 +688,7 @@ uint64_t inorder_tile_records(uint64_t n, int sm_count) {
 }
 
 // dynamic shared memory of the serve kernel: the per-queue state and the per-die counters
-size_t inorder_serve_smem(uint32_t n_dies) { return (size_t)kInMaxQueues * 16 + (size_t)n_dies * 24; }
+size_t inorder_serve_smem(uint32_t n_dies) { return (size_t)kInMaxQueues * 16 + (size_t)n_dies * 28; }
 static size_t inorder_straggle_smem() { return (size_t)kInMaxQueues * 16 + (size_t)kInStrChunk * 24 + (size_t)kInMaxQueues * 3; }
 
 size_t inorder_head_bytes(uint64_t tiles, uint32_t n_queues) { return tiles * n_queues * (size_t)kInHead * sizeof(InHead); }

@@ -302,32 +302,37 @@ __global__ void k_ret_chan(RetDev r, uint32_t channels, uint32_t dies) {
     if (threadIdx.x == 0) r.st->epoch_total = s_total;
 }
 
-// one warp per block, its lanes over the block's pages
+// one warp per block, its lanes over the block's pages.  Every length and rank of an epoch is below 2^32 (a quantum id
+// is 32 bits and a block is planned at most once at a time), so the arithmetic is 32-bit.
 __global__ void __launch_bounds__(256)
 k_ret_emit(RetDev r, uint32_t channels, uint32_t dies, uint32_t planes) {
     const RetState *st = r.st;
     const uint32_t epoch = st->epoch;
     const unsigned long long base = st->planned;
+    const uint64_t base_mod = base % r.plan_cap;
     const uint32_t blocks_per_die = planes * r.bpp;
     const int lane = threadIdx.x & 31;
     const uint64_t warps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
     for (uint64_t b = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; b < r.n_blocks; b += warps) {
         if (r.epoch_of[b] != epoch) continue;
         const uint32_t die = (uint32_t)(b / blocks_per_die), ch = die / dies, di = die % dies;
-        const unsigned long long first = (unsigned long long)r.rank[b] * r.ppb;
+        const uint32_t first = r.rank[b] * r.ppb;
+        const unsigned long long *dlen = r.die_len + (size_t)ch * dies;
         for (uint32_t pg = (uint32_t)lane; pg < r.ppb; pg += 32u) {
-            const unsigned long long r_die = first + pg;
-            unsigned long long r_ch = 0;
+            const uint32_t r_die = first + pg;
+            uint32_t r_ch = 0;
             for (uint32_t d = 0; d < dies; ++d) {
-                const unsigned long long len = r.die_len[ch * dies + d];
-                r_ch += min(len, r_die) + ((d < di && len > r_die) ? 1ull : 0ull);
+                const uint32_t len = (uint32_t)__ldg(dlen + d);
+                r_ch += min(len, r_die) + ((d < di && len > r_die) ? 1u : 0u);
             }
-            unsigned long long pos = 0;
+            uint32_t pos = 0;
             for (uint32_t c = 0; c < channels; ++c) {
-                const unsigned long long len = r.chan_len[c];
-                pos += min(len, r_ch) + ((c < ch && len > r_ch) ? 1ull : 0ull);
+                const uint32_t len = (uint32_t)__ldg(r.chan_len + c);
+                pos += min(len, r_ch) + ((c < ch && len > r_ch) ? 1u : 0u);
             }
-            r.plan[(base + pos) % r.plan_cap] = (uint32_t)(b * r.ppb + pg);
+            uint64_t slot = base_mod + pos;
+            if (slot >= r.plan_cap) slot -= r.plan_cap;
+            r.plan[slot] = (uint32_t)(b * r.ppb + pg);
             if (pg + 1u == r.ppb) r.last_pos[b] = base + pos;       // the last page's place: a block's pages go out in order
         }
     }

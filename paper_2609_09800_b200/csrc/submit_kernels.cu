@@ -425,6 +425,7 @@ k_scan(const hbf_access_t *__restrict__ acc, uint64_t n, const RangeSnap *__rest
     }
     // gather the records and rebuild their service terms
     long long acc_busy = 0, acc_br = 0, acc_bp = 0, acc_e = 0, acc_nr = 0, acc_np = 0;
+    uint32_t acc_claims = 0;                                 // refresh quanta claimed on the die of the run in progress
     uint32_t run_die = 0xffffffffu;
     auto flush_run = [&](uint32_t die) {
         long long *d = reinterpret_cast<long long *>(stats_stage + die);
@@ -434,7 +435,8 @@ k_scan(const hbf_access_t *__restrict__ acc, uint64_t n, const RangeSnap *__rest
         if (acc_e) atomicAdd((unsigned long long *)&d[3], (unsigned long long)acc_e);
         if (acc_nr) atomicAdd((unsigned long long *)&d[4], (unsigned long long)acc_nr);
         if (acc_np) atomicAdd((unsigned long long *)&d[5], (unsigned long long)acc_np);
-        acc_busy = acc_br = acc_bp = acc_e = acc_nr = acc_np = 0;
+        if (acc_claims) atomicAdd(&die_claims[die], acc_claims);
+        acc_busy = acc_br = acc_bp = acc_e = acc_nr = acc_np = 0; acc_claims = 0;
     };
     uint64_t r_addr[kScanItems], r_bf[kScanItems];
 #pragma unroll
@@ -455,9 +457,9 @@ k_scan(const hbf_access_t *__restrict__ acc, uint64_t n, const RangeSnap *__rest
             const Decoded d = decode(mp, off, bytes);
             const Terms t = service_terms(mp, bytes, d.npages, op, q_ppm, div_q);
             s[j] = t.s;
-            if ((uint64_t)idx[j] < claim_limit) { s[j] += quantum_ns; atomicAdd(&die_claims[d.die], 1u); }
             if (op) { a[j] = issue[j] + t.xfer; post[j] = 0u; } else { a[j] = issue[j]; post[j] = (uint32_t)t.xfer; }
             if (d.die != run_die) { if (run_die != 0xffffffffu) flush_run(run_die); run_die = d.die; }
+            if ((uint64_t)idx[j] < claim_limit) { s[j] += quantum_ns; ++acc_claims; }
             acc_busy += s[j]; acc_e += t.energy; sum_s += s[j];
             if (op) { acc_bp += t.cb; acc_np += 1; } else { acc_br += t.cb; acc_nr += 1; }
         }
@@ -574,6 +576,8 @@ k_scan(const hbf_access_t *__restrict__ acc, uint64_t n, const RangeSnap *__rest
         if (uniform && tile_die == s_tile_die) {
             acc_busy = warp_sum(acc_busy); acc_br = warp_sum(acc_br); acc_bp = warp_sum(acc_bp);
             acc_e = warp_sum(acc_e); acc_nr = warp_sum(acc_nr); acc_np = warp_sum(acc_np);
+            acc_claims = (uint32_t)warp_sum((long long)acc_claims);
+            if (lane == 0 && acc_claims) atomicAdd(&die_claims[tile_die], acc_claims);
             if (lane == 0) {
                 atomicAdd((unsigned long long *)&s_die_acc[0], (unsigned long long)acc_busy);
                 atomicAdd((unsigned long long *)&s_die_acc[1], (unsigned long long)acc_br);
