@@ -83,6 +83,61 @@ def test_full_size_batch_against_per_queue_oracle(full, path):
     ctx.destroy()
 
 
+def test_full_size_batch_with_refresh_claims(full):
+    """Retention on, in the configuration `bench.py --workload capacity_retention` times: the batch, one epoch that
+    makes every block eligible, the batch again with its first 33.5 M accesses claiming one refresh quantum each.
+    Claims go to the modeled accesses in index order, so within one queue's sub-stream they go to a prefix too: the
+    oracle serves a sampled queue's sub-stream alone with exactly that many quanta of debt (made by an epoch of its
+    own and trimmed by idle-time decay) and must give the same completions."""
+    import torch
+    hbf, w, queue = full
+    ret = dict(pages_per_block=256, blocks_per_plane=64, blocks_per_zone=8, max_pec=3000, disturb_limit=1,
+               l_ref_s=3.15e7, t_ref_c=40.0, ea_ev=1.04, accel=1.0, lead_threshold=0.8)
+    ctx = hbf.Context(w.profile)
+    for r in w.ranges:
+        ctx.register_range(*r)
+    ctx.enable_retention(**ret)
+    n = w.n
+    d_acc = torch.from_numpy(w.acc.view(np.int64).reshape(-1)).cuda()
+    d_comp = torch.empty(n, dtype=torch.int64, device="cuda"); d_stall = torch.empty_like(d_comp)
+    d_ds = torch.empty(ctx.n_dies * 6, dtype=torch.int64, device="cuda")
+    ws = ctx.workspace(n)
+    assert ctx.submit_batch(d_acc, n, d_comp, d_stall, None, d_ds, ws) == 0
+    assert ctx.last_result()["code"] == 0 and ctx.retention_totals()["claimed"] == 0
+    ctx.retention_advance(10**9, np.array([60.0]))
+    debt = ctx.retention_totals()["planned"]
+    assert debt == 131072 * 256                               # every block was read at least once
+    assert ctx.submit_batch(d_acc, n, d_comp, d_stall, None, d_ds, ws) == 0
+    res = ctx.last_result()
+    comp = d_comp.cpu().numpy(); ds = d_ds.cpu().numpy().view(hbf.DIE_STATS_DTYPE).copy(); busy = ctx.get_busy_until()
+    tot = ctx.retention_totals()
+    assert res["code"] == 0 and tot["claimed"] == debt and tot["commits"] == 131072 and tot["waiting_blocks"] == 0
+    npages = np.maximum(1, w.acc["bytes"].astype(np.int64) >> 14)
+    assert res["service_ns"] == int(npages.sum()) * 20000 + debt * 395000 == int(ds["busy_ns"].sum())
+    assert int(ctx.retention_blocks()["pec"].sum()) == 131072
+    quantum_pj = (84 + 840) * 16384
+    read_pj = 2 * 84 * int(np.maximum(w.acc["bytes"], 64).astype(np.int64).sum())          # two batches of reads
+    assert int(ctx.get_pending_energy().sum()) == read_pj + debt * quantum_pj
+    del d_acc, d_comp, d_stall, d_ds
+    for q in [0, 1, 777, 2047]:
+        idx = np.flatnonzero(queue == q)
+        k = int(np.count_nonzero(idx < debt))                 # every access is modeled: the claim limit is the debt itself
+        o = hbfo.Oracle(w.profile)
+        for r in w.ranges:
+            o.register_range(*r)
+        o.enable_retention(**dict(ret, pages_per_block=1, blocks_per_plane=16, blocks_per_zone=8, disturb_limit=0, lead_threshold=1e-9))
+        o.submit(w.acc[idx])
+        o.retention_advance(10**9, np.array([60.0]))
+        assert o.retention_totals()["planned"] == 2048 * 16 >= k
+        o.retention_decay((2048 * 16 - k) * 395000)
+        assert o.retention_totals()["planned"] - o.retention_totals()["decayed"] == k
+        _, c_o, _, _, _ = o.submit(w.acc[idx])
+        bad = np.flatnonzero(comp[idx] != c_o)
+        assert bad.size == 0, (q, int(idx[bad[0]]), int(comp[idx][bad[0]]), int(c_o[bad[0]]))
+        assert int(busy[q]) == int(o.busy_until()[q])
+    ctx.destroy()
+
+
 @pytest.mark.parametrize("which", ["decode_weights", "prefix_kv"])
 def test_serving_configurations_at_full_size_element_by_element(which):
     """The 21 M-access decode-weight stream and the 28 M-access prefix-KV stream (the two serving configurations),
