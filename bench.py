@@ -61,6 +61,9 @@ def parse_args():
     ap.add_argument("--horizon-ms", type=int, default=1000, help="simulated time of the coupled_thermal run")
     ap.add_argument("--channel-bus", action="store_true",
                     help="capacity_mode: also run the channel-bus stage (reads' transfers queue per channel); not the headline")
+    ap.add_argument("--retention", action="store_true",
+                    help="coupled_thermal: retention on, one epoch per thermal step with the temperatures of the field "
+                         "(reliability time accelerated 2e6 times so that blocks come due within the simulated second)")
     ap.add_argument("--energy-bins", action="store_true",
                     help="coupled_thermal: book event energies into 1 ms bins (time-bin power integration) instead of at submit")
     return ap.parse_args()
@@ -206,6 +209,9 @@ def run_coupled(args):
     ctx.set_path(hbf.PATH_INORDER)             # the caller knows its stream is in issue order: no sort kernels are launched
     if args.energy_bins:
         ctx.enable_energy_bins(1_000_000, 64)
+    if args.retention:
+        ctx.enable_retention(pages_per_block=64, blocks_per_plane=64, blocks_per_zone=8, max_pec=3000, disturb_limit=0,
+                             l_ref_s=3.15e7, t_ref_c=40.0, ea_ev=1.04, accel=2.0e6, lead_threshold=0.8)
     d_all = torch.from_numpy(allrec.view(np.int64).reshape(-1, 3)).cuda()
     nmax = max(sizes)
     d_comp = torch.empty(nmax, dtype=torch.int64, device="cuda"); d_stall = torch.empty_like(d_comp)
@@ -219,6 +225,8 @@ def run_coupled(args):
             rc = ctx.submit_batch(d_all[offs[k]:offs[k + 1]], nk, d_comp, d_stall, None, d_stats, ws)
             assert rc == 0, rc
             ctx.thermal_step(1_000_000, ext, None, want_hot=False)
+            if args.retention:
+                ctx.retention_advance(1_000_000)
     ctx.reset(); run(); torch.cuda.synchronize()               # warm-up pass over the same horizon
     ctx.reset()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -239,6 +247,9 @@ def run_coupled(args):
                        "energy": "1 ms bins, split by time overlap" if args.energy_bins else "charged at submit"},
             "gpu_launches": int(hbf.kernel_launches() - l0), "host_wall_s": round(wall, 3),
             "final": {"hot_c": [round(float(x), 3) for x in hot], "mode": mode, "q_ppm": q}}
+    if args.retention:
+        line["retention"] = ctx.retention_totals()
+        line["config"]["retention"] = "one epoch per thermal step, region temperatures from the field, a_t = 2e6"
     print(json.dumps(line), flush=True)
 
 
