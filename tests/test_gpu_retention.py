@@ -275,3 +275,31 @@ def test_reset_clears_the_block_state(hbf):
     compare_state(g, o)
     assert g.retention_totals()["planned"] == 0
     assert compare_batch(g, o, mixed_batch(rng, 3000, 0, 4096)) == 0
+
+
+@pytest.mark.parametrize("geom", [dict(channels=3, dies=5, planes=3), dict(channels=4, dies=2, planes=2, queue_level=1),
+                                  dict(channels=8, dies=4, planes=2, stripe_bytes=64 * wl.KIB)])
+def test_other_geometries_and_two_ranges(hbf, geom):
+    """Channel, die and plane counts that are not powers of two (division instead of masks), one queue per die, several
+    pages per stripe unit, two registered ranges with media offsets of their own."""
+    ret = dict(RET, disturb_limit=3, lead_threshold=0.05, pages_per_block=3, blocks_per_plane=12, blocks_per_zone=4)
+    prof = wl.load_profile("nominal", **wl.GEOMETRY["tiny"]); prof.update(geom)
+    g, o = hbf.Context(prof), hbfo.Oracle(prof)
+    for c in (g, o):
+        c.register_range(BASE, wl.GIB, 3, 0, 0, 5 * PAGE)
+        c.register_range(BASE + 4 * wl.GIB, wl.GIB, 1, 0, 0, 3 * wl.GIB + 7 * PAGE)
+    g.enable_retention(**ret); o.enable_retention(**ret)
+    rng = np.random.default_rng(geom["channels"])
+    t0 = 0
+    for round_ in range(5):
+        acc = mixed_batch(rng, 20_000, t0, 3000)
+        second = rng.random(acc.shape[0]) < 0.4
+        acc["addr"][second] += np.uint64(4 * wl.GIB)
+        acc["flags"][second] = 0                                          # the second range is read-only
+        assert compare_batch(g, o, acc) == 0
+        t0 = int(acc["issue_ns"][-1]) + 10**8
+        temps = np.array([rng.uniform(40.0, 90.0)])
+        g.retention_advance(10**10, temps); o.retention_advance(10**10, temps)
+        compare_state(g, o)
+    t = o.retention_totals()
+    assert t["claimed"] > 0 and t["commits"] > 0
