@@ -26,6 +26,7 @@
 // warp through the hardware's named barriers.  Records of one queue that fall into the same row are chained
 // in registers with shuffles.
 #include <algorithm>
+#include <type_traits>
 
 #include "device_utils.cuh"
 
@@ -181,7 +182,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
             for (uint32_t q = tid; q < R; q += kInThreads) qst[q].x = busy[q];
         }
     }
-    unsigned long long c_native = 0, c_ready = 0, c_fault = 0;
+    uint32_t c_native = 0, c_ready = 0, c_fault = 0;         // per thread: far below 2^32 (a batch is below 2^30 records)
     unsigned c_unsorted = 0;
     long long sum_stall = 0, max_c = INT64_MIN;
 
@@ -199,9 +200,9 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
 
     // the records of the warp's next turn are already on their way while this one is served
     uint64_t nx_addr[K], nx_issue[K], nx_bf[K];
-    int64_t nx_prev = INT64_MIN;                             // lane 0: issue time of the record before the turn's first
+    int64_t nx_prev[K];                                      // issue time of the record before the lane's own (same cache line, mostly)
 #pragma unroll
-    for (int u = 0; u < K; ++u) { nx_addr[u] = 0; nx_issue[u] = 0; nx_bf[u] = 0; }
+    for (int u = 0; u < K; ++u) { nx_addr[u] = 0; nx_issue[u] = 0; nx_bf[u] = 0; nx_prev[u] = INT64_MIN; }
     auto fetch = [&](uint64_t turn) {
 #pragma unroll
         for (int u = 0; u < K; ++u) {
@@ -209,7 +210,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
             if (i < tile_end) {
                 const uint64_t *rec = reinterpret_cast<const uint64_t *>(acc + i);
                 nx_addr[u] = __ldg(rec); nx_issue[u] = __ldg(rec + 1); nx_bf[u] = __ldg(rec + 2);
-                if (!RESERVE && u == 0 && lane == 0 && i > 0) nx_prev = (int64_t)__ldg(rec - 2);
+                if (!RESERVE) nx_prev[u] = i > 0 ? (int64_t)__ldg(rec - 2) : INT64_MIN;
             }
         }
     };
@@ -222,13 +223,13 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
         Served v[K];
         uint32_t rank1[K], pc[K], c0[K], c1[K], qi[K];
         longlong2 *pq[K];
-        const int64_t turn_prev = nx_prev;
+        int64_t prev[K];
         uint64_t addr[K], bf[K];
 #pragma unroll
         for (int u = 0; u < K; ++u) {
             i[u] = tile_begin + (turn * K + u) * 32 + (uint64_t)lane;
             valid[u] = i[u] < tile_end;
-            addr[u] = nx_addr[u]; bf[u] = nx_bf[u]; issue[u] = (int64_t)nx_issue[u];
+            addr[u] = nx_addr[u]; bf[u] = nx_bf[u]; issue[u] = (int64_t)nx_issue[u]; prev[u] = nx_prev[u];
         }
         fetch(turn + kInWarps);
         {                                                    // and the turn after that is called into the L2
@@ -264,11 +265,8 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
         if (!RESERVE) {
 #pragma unroll
             for (int u = 0; u < K; ++u) {
-                int64_t prev = __shfl_up_sync(0xffffffffu, issue[u], 1);
-                const int64_t before = u == 0 ? turn_prev : __shfl_sync(0xffffffffu, issue[u == 0 ? 0 : u - 1], 31);
-                if (lane == 0) prev = before;
                 if (valid[u]) {
-                    c_unsorted |= issue[u] < prev ? 1u : 0u;
+                    c_unsorted |= issue[u] < prev[u] ? 1u : 0u;
                     if (status) status[i[u]] = (uint8_t)v[u].st;
                     if (ready[u]) {
                         ++c_ready;
@@ -287,7 +285,11 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
                 }
             }
         }
+        // The rest of the turn exists twice: with the head-table bookkeeping, and without it once every queue of the
+        // tile has its head entries (after a few percent of a large tile).  The flag is the same for the whole warp.
         const bool heads_on = !RESERVE && *reinterpret_cast<volatile uint32_t *>(&s_heads_full) < R;
+        auto rest_of_turn = [&](auto heads_tag) {
+        constexpr bool HEADS = decltype(heads_tag)::value;
         // ---- per row: the accesses of a lane's queue, up to the lane's own, as one map B -> max(B + S, M), composed
         // in lane order, so that the ordered part below is one application of it whatever the row holds
 #pragma unroll
@@ -312,7 +314,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
             }
             qi[u] = ready[u] ? v[u].queue : 0u;
             pq[u] = qst + qi[u];
-            pc[u] = heads_on ? (uint32_t)__popc(peers) : 0u;
+            pc[u] = HEADS ? (uint32_t)__popc(peers) : 0u;
         }
         // ---- the queue updates, in row order: everything they need is in registers before the wait ---------------
         if (turn > 0) {
@@ -323,9 +325,12 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
         for (int u = 0; u < K; ++u) {
             const longlong2 state = *pq[u];
             B[u] = max((int64_t)(state.x + S[u]), M[u]);
-            c0[u] = min((uint32_t)state.y & 0xffu, (uint32_t)kInHead);
-            const uint32_t inc = min(pc[u], (uint32_t)kInHead - c0[u]);
-            c1[u] = c0[u] + inc;
+            uint32_t inc = 0u;
+            if (HEADS) {
+                c0[u] = min((uint32_t)state.y & 0xffu, (uint32_t)kInHead);
+                inc = min(pc[u], (uint32_t)kInHead - c0[u]);
+                c1[u] = c0[u] + inc;
+            }
             if (last[u]) *pq[u] = make_longlong2(B[u], state.y + (S[u] << 8) + (long long)inc);
             if (u + 1 < K) __syncwarp();                     // the next row may hold the same queues
         }
@@ -339,16 +344,20 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
                     done = B[u] + (v[u].op ? 0 : v[u].xfer); // a read's data is transferred after its service
                     st = done - issue[u];
                     sum_stall += st; max_c = max(max_c, (long long)done);
-                    const uint32_t ci = c0[u] + rank1[u] - 1u;
-                    if (heads_on && ci < (uint32_t)kInHead) {
-                        InHead h; h.m = a[u] + v[u].s; h.s = v[u].s; h.xo = (uint32_t)v[u].xfer | (v[u].op << 31); h.idx = (uint32_t)i[u];
-                        in_head[((uint64_t)tile * kInHead + ci) * R + qi[u]] = h;
+                    if (HEADS) {
+                        const uint32_t ci = c0[u] + rank1[u] - 1u;
+                        if (ci < (uint32_t)kInHead) {
+                            InHead h; h.m = a[u] + v[u].s; h.s = v[u].s; h.xo = (uint32_t)v[u].xfer | (v[u].op << 31); h.idx = (uint32_t)i[u];
+                            in_head[((uint64_t)tile * kInHead + ci) * R + qi[u]] = h;
+                        }
+                        if (last[u] && c1[u] != c0[u] && c1[u] == (uint32_t)kInHead) atomicAdd(&s_heads_full, 1u);
                     }
-                    if (last[u] && c1[u] != c0[u] && c1[u] == (uint32_t)kInHead) atomicAdd(&s_heads_full, 1u);
                 }
                 completion[i[u]] = done; stall[i[u]] = st;
             }
         }
+        };
+        if (heads_on) rest_of_turn(std::true_type{}); else rest_of_turn(std::false_type{});
     }
 
     __syncthreads();
@@ -369,14 +378,14 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
             if (st_np[d]) atomicAdd(&g[5], (unsigned long long)st_np[d]);
             if (DEBT && st_claims[d]) atomicAdd(&die_claims[d], st_claims[d]);
         }
-        c_native = (unsigned long long)warp_sum((long long)c_native);
-        c_ready = (unsigned long long)warp_sum((long long)c_ready);
-        c_fault = (unsigned long long)warp_sum((long long)c_fault);
+        const unsigned long long w_native = (unsigned long long)warp_sum((long long)c_native);
+        const unsigned long long w_ready = (unsigned long long)warp_sum((long long)c_ready);
+        const unsigned long long w_fault = (unsigned long long)warp_sum((long long)c_fault);
         c_unsorted = __any_sync(0xffffffffu, c_unsorted);
         if (lane == 0) {
-            if (c_native) atomicAdd(&ctrl->n_native, c_native);
-            if (c_ready) atomicAdd(&ctrl->n_ready, c_ready);
-            if (c_fault) atomicAdd(&ctrl->n_fault, c_fault);
+            if (w_native) atomicAdd(&ctrl->n_native, w_native);
+            if (w_ready) atomicAdd(&ctrl->n_ready, w_ready);
+            if (w_fault) atomicAdd(&ctrl->n_fault, w_fault);
             if (c_unsorted) atomicOr(&ctrl->unsorted, 1u);
         }
     }
