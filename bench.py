@@ -36,6 +36,10 @@ STAGE_BYTES = {"classify": 24 + 8 + 1, "plan_hist": 8, "scan": 8 + 4 + 24 + 16, 
 # DRAM bytes per access of the in-order serve kernel from one one-pass ncu capture at the full 200 M size
 # (dram__bytes_read + write of one launch, see the summary under profiles/); scaled to the batch in use
 NCU_TRAFFIC_BYTES_PER_ACCESS = {"inorder": 42.6}
+# warp instructions the in-order serve pass executes per access (smsp__inst_executed.sum of a one-pass ncu capture at
+# 200 M, profiles/inorder_path_capacity_20M.md) and the SM's issue rate: 148 SMs x 4 schedulers x one instruction per cycle
+NCU_WARP_INSTR_PER_ACCESS = {"inorder": 11.0}
+SM_COUNT, SCHEDULERS_PER_SM = 148, 4
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -583,6 +587,14 @@ def main():
         roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
                     "frac": achieved / peak, "traffic": traffic * n if traffic else None,
                     "algorithmic_bytes_per_access": dom_bytes, "ms_per_launch": per_launch_ms}
+        if dom in NCU_WARP_INSTR_PER_ACCESS and per_launch_ms > 0:
+            # the same kernel against the issue rate at the clock sampled during the timed region: what actually binds it
+            mhz = (clocks or {}).get("sm_mhz") or 1965.0
+            issue_peak = SM_COUNT * SCHEDULERS_PER_SM * mhz * 1e6
+            issued = NCU_WARP_INSTR_PER_ACCESS[dom] * n / (per_launch_ms * 1e-3)
+            roofline["alu"] = {"achieved": issued / 1e12, "peak": issue_peak / 1e12, "unit": "T warp instructions/s",
+                               "frac": issued / issue_peak, "warp_instructions_per_access": NCU_WARP_INSTR_PER_ACCESS[dom],
+                               "note": "instruction count from an ncu capture, time measured live"}
         path_gbs = ALGO_BYTES_PER_ACCESS * value / world / 1e9
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
                 "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
