@@ -95,6 +95,64 @@ __device__ __forceinline__ Served serve_terms_fast(const FastRange &f, const Mod
     r.s = (int64_t)npages * (r.op ? mp.t_prog_ns : mp.t_read_ns);
     return r;
 }
+// The common configuration once more, laid out for the serve pass: seven 16-byte vectors in shared memory, every field a
+// 32-bit operand where the values allow it (page times and the transfer table's reach below 2^32).
+struct __align__(16) FastGeom {
+    uint64_t base, length;                                  // the one registered range
+    uint64_t media_offset; uint32_t perms, stripe_shift;
+    uint32_t ch_mask, ch_shift, die_mask, chdie_shift;      // stripe unit -> channel, die, plane
+    uint32_t plane_mask, dies, planes_q, plane_mask_q;      // planes_q = 1, plane_mask_q = 0 with one queue per die
+    uint32_t page_mask, page_shift, gran_shift_read, gran_shift_prog;
+    uint32_t tab_shift, tab_max_cb, t_read, t_prog;
+    const uint32_t *xfer_tab; uint64_t pad;
+};
+__device__ __forceinline__ bool fast_geom_ok(const FastRange &f, const ModelParams &mp) {
+    return f.on != 0u && mp.pow2_geom != 0u && mp.xfer_tab_max_cb != 0u && mp.t_read_ns < (1ll << 32) && mp.t_prog_ns < (1ll << 32);
+}
+__device__ __forceinline__ FastGeom make_fast_geom(const FastRange &f, const ModelParams &mp) {
+    FastGeom g;
+    g.base = f.base; g.length = f.length; g.media_offset = f.media_offset; g.perms = f.perms; g.stripe_shift = mp.stripe_shift;
+    g.ch_mask = mp.channels - 1u; g.ch_shift = mp.ch_shift; g.die_mask = mp.dies - 1u; g.chdie_shift = mp.ch_shift + mp.die_shift;
+    g.plane_mask = mp.planes - 1u; g.dies = mp.dies;
+    g.planes_q = mp.queue_level == 0u ? mp.planes : 1u; g.plane_mask_q = mp.queue_level == 0u ? mp.planes - 1u : 0u;
+    g.page_mask = (1u << mp.page_shift) - 1u; g.page_shift = mp.page_shift;
+    g.gran_shift_read = mp.read_gran_shift; g.gran_shift_prog = mp.prog_gran_shift;
+    g.tab_shift = mp.xfer_tab_shift; g.tab_max_cb = mp.xfer_tab_max_cb; g.t_read = (uint32_t)mp.t_read_ns; g.t_prog = (uint32_t)mp.t_prog_ns;
+    g.xfer_tab = mp.xfer_tab; g.pad = 0;
+    return g;
+}
+// No branches: every access computes every term, and the classification (the same tests in the same order as classify())
+// only selects the status; the terms of an access that is not READY are never used.  (Early returns cost this pass
+// about 47 instructions per row of 32 accesses, measured.)
+__device__ __forceinline__ Served serve_terms_geom(const FastGeom &g, const ModelParams &mp, uint64_t addr, int64_t issue, uint64_t bf) {
+    Served r;
+    const uint32_t bytes = (uint32_t)bf, flags = (uint32_t)(bf >> 32);
+    const uint64_t rel = addr - g.base;                       // wraps to a huge value below the base
+    const uint32_t op = flags & 1u;
+    const bool unsupported = bytes == 0u || flags > 1u || (uint32_t)((uint64_t)issue >> 32) >= (1u << (kIssueBits - 32));
+    const bool outside = rel >= g.length;
+    const bool partial = (uint64_t)bytes > g.length - rel;
+    const bool denied = ((g.perms >> op) & 1u) == 0u;
+    int st = denied ? HBF_ST_FAULT_PERM : HBF_ST_READY;
+    st = partial ? HBF_ST_FAULT_PARTIAL : st;
+    st = outside ? HBF_ST_NATIVE : st;
+    r.st = unsupported ? HBF_ST_UNSUPPORTED : st;
+    r.op = op;
+    const uint64_t off = g.media_offset + rel;
+    const uint32_t u = (uint32_t)(off >> g.stripe_shift);     // only the low interleave bits are used
+    const uint32_t ch = u & g.ch_mask, di = (u >> g.ch_shift) & g.die_mask, pl = (u >> g.chdie_shift) & g.plane_mask_q;
+    r.die = ch * g.dies + di;
+    r.queue = r.die * g.planes_q + pl;
+    const uint32_t npages = (uint32_t)(((uint64_t)((uint32_t)off & g.page_mask) + bytes + g.page_mask) >> g.page_shift);
+    const uint32_t gs = op ? g.gran_shift_prog : g.gran_shift_read;
+    const uint64_t gm = (1ull << gs) - 1ull;
+    const uint64_t cb = ((uint64_t)bytes + gm) & ~gm;
+    r.cb = (int64_t)cb;
+    r.xfer = cb <= (uint64_t)g.tab_max_cb ? (int64_t)__ldg(g.xfer_tab + ((uint32_t)cb >> g.tab_shift))
+                                            : (int64_t)div64(cb * 1000ull + mp.chan_bytes_per_us - 1ull, mp.div_chan);
+    r.s = (int64_t)((uint64_t)npages * (op ? g.t_prog : g.t_read));
+    return r;
+}
 // per-tile bookkeeping of the stall total: as-if-idle sum, fix-up corrections, and the exact sum of a re-served tile
 struct InTile { long long spec_sum, fix_delta, true_sum; uint32_t reserve; uint32_t stragglers; };
 // The first kInHead accesses of every (tile, queue), as the serve pass saw them: all the fix-up needs in the common case.
@@ -144,18 +202,19 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
     __shared__ uint32_t s_heads_full;                     // queues whose head entries are complete
     __shared__ ModelParams mp;                            // measured: reads from shared memory beat reads of the argument
     __shared__ FastRange fast_range;
+    __shared__ FastGeom geom;
 
     if (ctrl->skip || ctrl->run_sort) return;             // (run_sort set this early: the batch went to the sort path at its start)
     if (RESERVE && (!ctrl->inorder_used || !in_tile[blockIdx.x].reserve)) return;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const RangeSnap &rs = *ranges_g;                      // read through the cache; the common configuration does not touch it
-    if (tid == 0) { mp = mp_arg; fast_range = fast_arg; }
+    if (tid == 0) { mp = mp_arg; fast_range = fast_arg; geom = make_fast_geom(fast_arg, mp_arg); }
     if (DEBT && !RESERVE && tid == 0 && blockIdx.x == 0) ret.st->observed_inline = 1u;
     const uint32_t R = mp_arg.n_queues, n_dies = mp_arg.n_dies;
     const int64_t q_ppm = ctrl->q_ppm;
     const Div64 div_q = ctrl->div_q;
     // one range, power-of-two geometry, transfer table, no thermal scaling in force: the short form of the terms
-    const bool fast_on = fast_arg.on != 0u && mp_arg.pow2_geom != 0u && mp_arg.xfer_tab_max_cb != 0u && q_ppm == 1000000;
+    const bool fast_on = fast_geom_ok(fast_arg, mp_arg) && q_ppm == 1000000;
     const uint64_t claim_limit = DEBT ? *claim_limit_p : 0ull;
     const int64_t quantum_ns = !DEBT ? 0 : q_ppm == 1000000 ? mp_arg.t_read_ns + mp_arg.t_prog_ns
         : (int64_t)div64((uint64_t)(mp_arg.t_read_ns + mp_arg.t_prog_ns) * 1000000ull + (uint64_t)q_ppm - 1ull, div_q);
@@ -182,7 +241,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
             for (uint32_t q = tid; q < R; q += kInThreads) qst[q].x = busy[q];
         }
     }
-    uint32_t c_native = 0, c_ready = 0, c_fault = 0;         // per thread: far below 2^32 (a batch is below 2^30 records)
+    uint32_t c_native = 0, c_ready = 0, c_valid = 0;         // per thread: far below 2^32 (a batch is below 2^30 records)
     unsigned c_unsorted = 0;
     long long sum_stall = 0, max_c = INT64_MIN;
 
@@ -193,8 +252,13 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
     // A warp's turn covers kInRows consecutive rows: their arithmetic interleaves, and their queue updates
     // follow one another inside one wait/pass pair.
     constexpr int K = kInRows;
-    const uint64_t rows = tile_end > tile_begin ? (tile_end - tile_begin + 31) / 32 : 0;
-    const uint64_t turns = (rows + K - 1) / K;
+    // inside a tile everything is indexed by 32-bit offsets from the tile's first record (a batch is below 2^30 records)
+    const uint32_t tile_len = tile_end > tile_begin ? (uint32_t)(tile_end - tile_begin) : 0u;
+    const hbf_access_t *acc_t = acc + tile_begin;
+    int64_t *completion_t = completion + tile_begin, *stall_t = stall + tile_begin;
+    uint8_t *status_t = status ? status + tile_begin : nullptr;
+    const uint32_t rows = (tile_len + 31u) / 32u;
+    const uint32_t turns = (rows + K - 1) / K;
     const unsigned le_mask = lanemask_lt() | (1u << lane);
     const int my_bar = 1 + warp, next_bar = 1 + (warp + 1 == kInWarps ? 0 : warp + 1);
 
@@ -203,21 +267,22 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
     int64_t nx_prev[K];                                      // issue time of the record before the lane's own (same cache line, mostly)
 #pragma unroll
     for (int u = 0; u < K; ++u) { nx_addr[u] = 0; nx_issue[u] = 0; nx_bf[u] = 0; nx_prev[u] = INT64_MIN; }
-    auto fetch = [&](uint64_t turn) {
+    const bool first_tile = tile_begin == 0;
+    auto fetch = [&](uint32_t turn) {
 #pragma unroll
         for (int u = 0; u < K; ++u) {
-            const uint64_t i = tile_begin + (turn * K + u) * 32 + (uint64_t)lane;
-            if (i < tile_end) {
-                const uint64_t *rec = reinterpret_cast<const uint64_t *>(acc + i);
+            const uint32_t j = (turn * K + u) * 32u + (uint32_t)lane;
+            if (j < tile_len) {
+                const uint64_t *rec = reinterpret_cast<const uint64_t *>(acc_t + j);
                 nx_addr[u] = __ldg(rec); nx_issue[u] = __ldg(rec + 1); nx_bf[u] = __ldg(rec + 2);
-                if (!RESERVE) nx_prev[u] = i > 0 ? (int64_t)__ldg(rec - 2) : INT64_MIN;
+                if (!RESERVE) nx_prev[u] = (j > 0u || !first_tile) ? (int64_t)__ldg(rec - 2) : INT64_MIN;
             }
         }
     };
-    fetch((uint64_t)warp);
+    fetch((uint32_t)warp);
 
-    for (uint64_t turn = (uint64_t)warp; turn < turns; turn += kInWarps) {
-        uint64_t i[K];
+    for (uint32_t turn = (uint32_t)warp; turn < turns; turn += kInWarps) {
+        uint32_t i[K];                                       // offsets from the tile's first record
         bool valid[K], ready[K], last[K];
         int64_t issue[K], a[K], S[K], M[K], B[K];
         Served v[K];
@@ -227,15 +292,15 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
         uint64_t addr[K], bf[K];
 #pragma unroll
         for (int u = 0; u < K; ++u) {
-            i[u] = tile_begin + (turn * K + u) * 32 + (uint64_t)lane;
-            valid[u] = i[u] < tile_end;
+            i[u] = (turn * K + u) * 32u + (uint32_t)lane;
+            valid[u] = i[u] < tile_len;
             addr[u] = nx_addr[u]; bf[u] = nx_bf[u]; issue[u] = (int64_t)nx_issue[u]; prev[u] = nx_prev[u];
         }
         fetch(turn + kInWarps);
         {                                                    // and the turn after that is called into the L2
-            const uint64_t first = tile_begin + (turn + 2 * kInWarps) * (uint64_t)(K * 32);
-            if (first + K * 32 <= tile_end) {
-                const char *p = reinterpret_cast<const char *>(acc + first) + lane * 32;
+            const uint32_t first = (turn + 2 * kInWarps) * (uint32_t)(K * 32);
+            if (first + K * 32 <= tile_len) {
+                const char *p = reinterpret_cast<const char *>(acc_t + first) + lane * 32;
 #pragma unroll
                 for (int u = 0; u < K; ++u)
                     if (lane < 24) asm volatile("prefetch.global.L2 [%0];" ::"l"(p + u * 768));
@@ -246,10 +311,10 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
         for (int u = 0; u < K; ++u) {
             v[u].st = HBF_ST_NATIVE; v[u].queue = 0; v[u].die = 0; v[u].op = 0; v[u].s = 0; v[u].xfer = 0; v[u].cb = 0;
             if (valid[u])
-                v[u] = fast_on ? serve_terms_fast(fast_range, mp, addr[u], issue[u], bf[u])
+                v[u] = fast_on ? serve_terms_geom(geom, mp, addr[u], issue[u], bf[u])
                                  : serve_terms(rs, mp, addr[u], issue[u], bf[u], q_ppm, div_q);
             ready[u] = valid[u] && v[u].st == HBF_ST_READY;
-            if (DEBT && ready[u] && i[u] < claim_limit) {
+            if (DEBT && ready[u] && tile_begin + i[u] < claim_limit) {
                 v[u].s += quantum_ns;
                 if (!RESERVE) atomicAdd(&st_claims[v[u].die], 1u);
             }
@@ -267,9 +332,11 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
             for (int u = 0; u < K; ++u) {
                 if (valid[u]) {
                     c_unsorted |= issue[u] < prev[u] ? 1u : 0u;
-                    if (status) status[i[u]] = (uint8_t)v[u].st;
+                    if (status_t) status_t[i[u]] = (uint8_t)v[u].st;
+                    c_valid += 1u;
+                    c_ready += ready[u] ? 1u : 0u;
+                    c_native += v[u].st == HBF_ST_NATIVE ? 1u : 0u;
                     if (ready[u]) {
-                        ++c_ready;
                         // charged bytes < 2^33: add the low word, carry into the high word when it wraps
                         const uint32_t lo = (uint32_t)v[u].cb, hi = (uint32_t)((uint64_t)v[u].cb >> 32);
                         uint32_t *plo = v[u].op ? st_bp_lo : st_br_lo, *phi = v[u].op ? st_bp_hi : st_br_hi;
@@ -277,10 +344,6 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
                         const uint32_t old = atomicAdd(&plo[v[u].die], lo);
                         const uint32_t carry = hi + ((old + lo) < old ? 1u : 0u);
                         if (carry) atomicAdd(&phi[v[u].die], carry);
-                    } else if (v[u].st == HBF_ST_NATIVE) {
-                        ++c_native;
-                    } else {
-                        ++c_fault;
                     }
                 }
             }
@@ -347,13 +410,13 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
                     if (HEADS) {
                         const uint32_t ci = c0[u] + rank1[u] - 1u;
                         if (ci < (uint32_t)kInHead) {
-                            InHead h; h.m = a[u] + v[u].s; h.s = v[u].s; h.xo = (uint32_t)v[u].xfer | (v[u].op << 31); h.idx = (uint32_t)i[u];
+                            InHead h; h.m = a[u] + v[u].s; h.s = v[u].s; h.xo = (uint32_t)v[u].xfer | (v[u].op << 31); h.idx = (uint32_t)tile_begin + i[u];
                             in_head[((uint64_t)tile * kInHead + ci) * R + qi[u]] = h;
                         }
                         if (last[u] && c1[u] != c0[u] && c1[u] == (uint32_t)kInHead) atomicAdd(&s_heads_full, 1u);
                     }
                 }
-                completion[i[u]] = done; stall[i[u]] = st;
+                completion_t[i[u]] = done; stall_t[i[u]] = st;
             }
         }
         };
@@ -380,7 +443,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
         }
         const unsigned long long w_native = (unsigned long long)warp_sum((long long)c_native);
         const unsigned long long w_ready = (unsigned long long)warp_sum((long long)c_ready);
-        const unsigned long long w_fault = (unsigned long long)warp_sum((long long)c_fault);
+        const unsigned long long w_fault = (unsigned long long)warp_sum((long long)(c_valid - c_ready - c_native));   // every other status is a fault
         c_unsorted = __any_sync(0xffffffffu, c_unsorted);
         if (lane == 0) {
             if (w_native) atomicAdd(&ctrl->n_native, w_native);
