@@ -281,7 +281,11 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
     };
     fetch((uint32_t)warp);
 
+    // A turn whose rows are all complete (every turn but the last of a batch whose size is not a multiple of 32) runs
+    // a copy of the code that has no bounds tests.
     for (uint32_t turn = (uint32_t)warp; turn < turns; turn += kInWarps) {
+      auto whole_turn = [&](auto full_tag) {
+        constexpr bool FULL = decltype(full_tag)::value;
         uint32_t i[K];                                       // offsets from the tile's first record
         bool valid[K], ready[K], last[K];
         int64_t issue[K], a[K], S[K], M[K], B[K];
@@ -293,7 +297,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
 #pragma unroll
         for (int u = 0; u < K; ++u) {
             i[u] = (turn * K + u) * 32u + (uint32_t)lane;
-            valid[u] = i[u] < tile_len;
+            valid[u] = FULL || i[u] < tile_len;
             addr[u] = nx_addr[u]; bf[u] = nx_bf[u]; issue[u] = (int64_t)nx_issue[u]; prev[u] = nx_prev[u];
         }
         fetch(turn + kInWarps);
@@ -421,6 +425,8 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
         }
         };
         if (heads_on) rest_of_turn(std::true_type{}); else rest_of_turn(std::false_type{});
+      };
+      if ((turn * K + K) * 32u <= tile_len) whole_turn(std::true_type{}); else whole_turn(std::false_type{});
     }
 
     __syncthreads();
