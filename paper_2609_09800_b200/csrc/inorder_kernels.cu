@@ -46,6 +46,10 @@ constexpr int kInWarps = kInThreads / 32;
 #ifndef HBF_IN_ROWS
 #define HBF_IN_ROWS 1
 #endif
+#ifndef HBF_IN_PFDIST
+#define HBF_IN_PFDIST 2
+#endif
+constexpr int kInPrefetchTurns = HBF_IN_PFDIST;          // how many of the warp's turns ahead its records are called into the L2
 constexpr int kInRows = HBF_IN_ROWS;                     // rows of 32 records a warp serves per turn
 static_assert(kInWarps >= 2 && kInWarps <= 15, "every warp owns one of the hardware barriers 1..15");
 
@@ -302,7 +306,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
         }
         fetch(turn + kInWarps);
         {                                                    // and the turn after that is called into the L2
-            const uint32_t first = (turn + 2 * kInWarps) * (uint32_t)(K * 32);
+            const uint32_t first = (turn + kInPrefetchTurns * kInWarps) * (uint32_t)(K * 32);
             if (first + K * 32 <= tile_len) {
                 const char *p = reinterpret_cast<const char *>(acc_t + first) + lane * 32;
 #pragma unroll
@@ -366,17 +370,24 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
             const unsigned peers = __match_any_sync(0xffffffffu, q);
             const unsigned le = peers & le_mask;
             rank1[u] = (uint32_t)__popc(le);               // this access is the rank1-th of its queue in the row
-            const uint32_t n_it = __reduce_max_sync(0xffffffffu, rank1[u]);
             last[u] = ready[u] && (peers >> lane) == 1u;    // no later access of this queue in the row
             S[u] = v[u].s; M[u] = a[u] + v[u].s;
-            if (n_it > 1u) {
-                unsigned rem = le & ~(1u << lane);           // earlier lanes of the same queue, lowest first
-                S[u] = 0; M[u] = kNegInf;
-                for (uint32_t it = 0; it < n_it; ++it) {
-                    const int src = rem ? __ffs((int)rem) - 1 : lane;
-                    const int64_t ab = __shfl_sync(0xffffffffu, a[u], src), sb = __shfl_sync(0xffffffffu, (int64_t)v[u].s, src);
-                    if (rem || it + 1u == rank1[u]) { M[u] = max(M[u], ab) + sb; S[u] += sb; }   // its peers first, then the lane's own
-                    rem &= rem - 1u;
+            if (__any_sync(0xffffffffu, rank1[u] > 1u)) {    // one row in five: some queue occurs twice
+                if (!__any_sync(0xffffffffu, rank1[u] > 2u)) {
+                    // pairs only (nearly always): the second lane of a pair composes its peer's map with its own
+                    const int src = rank1[u] == 2u ? __ffs((int)(le & ~(1u << lane))) - 1 : lane;
+                    const int64_t mp_ = __shfl_sync(0xffffffffu, M[u], src), sp_ = __shfl_sync(0xffffffffu, (int64_t)v[u].s, src);
+                    if (rank1[u] == 2u) { M[u] = max(mp_, a[u]) + v[u].s; S[u] = sp_ + v[u].s; }
+                } else {
+                    const uint32_t n_it = __reduce_max_sync(0xffffffffu, rank1[u]);
+                    unsigned rem = le & ~(1u << lane);       // earlier lanes of the same queue, lowest first
+                    S[u] = 0; M[u] = kNegInf;
+                    for (uint32_t it = 0; it < n_it; ++it) {
+                        const int src = rem ? __ffs((int)rem) - 1 : lane;
+                        const int64_t ab = __shfl_sync(0xffffffffu, a[u], src), sb = __shfl_sync(0xffffffffu, (int64_t)v[u].s, src);
+                        if (rem || it + 1u == rank1[u]) { M[u] = max(M[u], ab) + sb; S[u] += sb; }   // its peers first, then the lane's own
+                        rem &= rem - 1u;
+                    }
                 }
             }
             qi[u] = ready[u] ? v[u].queue : 0u;
