@@ -54,7 +54,8 @@ constexpr int kInRows = HBF_IN_ROWS;                     // rows of 32 records a
 static_assert(kInWarps >= 2 && kInWarps <= 15, "every warp owns one of the hardware barriers 1..15");
 
 // One access, from its record: status, and for a modeled access its queue, die and service terms.
-struct Served { int st; uint32_t queue, die, op; int64_t s, xfer, cb; };
+// (the in-order path is only chosen when every transfer time fits 31 bits)
+struct Served { int st; uint32_t queue, die, op, xfer; int64_t s, cb; };
 __device__ __forceinline__ Served serve_terms(const RangeSnap &rs, const ModelParams &mp, uint64_t addr, int64_t issue,
                                               uint64_t bf, int64_t q_ppm, const Div64 &div_q) {
     Served r; r.queue = 0; r.die = 0; r.op = 0; r.s = 0; r.xfer = 0; r.cb = 0;
@@ -66,7 +67,7 @@ __device__ __forceinline__ Served serve_terms(const RangeSnap &rs, const ModelPa
         const Decoded d = decode(mp, off, bytes);
         r.op = flags & 1u;
         const Terms t = service_terms(mp, bytes, d.npages, r.op, q_ppm, div_q);
-        r.queue = d.queue; r.die = d.die; r.s = t.s; r.xfer = t.xfer; r.cb = t.cb;
+        r.queue = d.queue; r.die = d.die; r.s = t.s; r.xfer = (uint32_t)t.xfer; r.cb = t.cb;
     }
     return r;
 }
@@ -94,8 +95,8 @@ __device__ __forceinline__ Served serve_terms_fast(const FastRange &f, const Mod
     const uint32_t gs = r.op ? mp.prog_gran_shift : mp.read_gran_shift;
     const uint64_t cb = (((uint64_t)bytes + ((1ull << gs) - 1ull)) >> gs) << gs;
     r.cb = (int64_t)cb;
-    r.xfer = cb <= (uint64_t)mp.xfer_tab_max_cb ? (int64_t)__ldg(mp.xfer_tab + (uint32_t)(cb >> mp.xfer_tab_shift))
-                                                 : (int64_t)div64(cb * 1000ull + mp.chan_bytes_per_us - 1ull, mp.div_chan);
+    r.xfer = cb <= (uint64_t)mp.xfer_tab_max_cb ? __ldg(mp.xfer_tab + (uint32_t)(cb >> mp.xfer_tab_shift))
+                                                 : (uint32_t)div64(cb * 1000ull + mp.chan_bytes_per_us - 1ull, mp.div_chan);
     r.s = (int64_t)npages * (r.op ? mp.t_prog_ns : mp.t_read_ns);
     return r;
 }
@@ -152,8 +153,8 @@ __device__ __forceinline__ Served serve_terms_geom(const FastGeom &g, const Mode
     const uint64_t gm = (1ull << gs) - 1ull;
     const uint64_t cb = ((uint64_t)bytes + gm) & ~gm;
     r.cb = (int64_t)cb;
-    r.xfer = cb <= (uint64_t)g.tab_max_cb ? (int64_t)__ldg(g.xfer_tab + ((uint32_t)cb >> g.tab_shift))
-                                            : (int64_t)div64(cb * 1000ull + mp.chan_bytes_per_us - 1ull, mp.div_chan);
+    r.xfer = cb <= (uint64_t)g.tab_max_cb ? __ldg(g.xfer_tab + ((uint32_t)cb >> g.tab_shift))
+                                            : (uint32_t)div64(cb * 1000ull + mp.chan_bytes_per_us - 1ull, mp.div_chan);
     r.s = (int64_t)((uint64_t)npages * (op ? g.t_prog : g.t_read));
     return r;
 }
@@ -272,6 +273,8 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
 #pragma unroll
     for (int u = 0; u < K; ++u) { nx_addr[u] = 0; nx_issue[u] = 0; nx_bf[u] = 0; nx_prev[u] = INT64_MIN; }
     const bool first_tile = tile_begin == 0;
+    const bool pf_lane = lane < 24;
+    const char *pf_base = reinterpret_cast<const char *>(acc_t) + lane * 32;
     auto fetch = [&](uint32_t turn) {
 #pragma unroll
         for (int u = 0; u < K; ++u) {
@@ -307,11 +310,10 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
         fetch(turn + kInWarps);
         {                                                    // and the turn after that is called into the L2
             const uint32_t first = (turn + kInPrefetchTurns * kInWarps) * (uint32_t)(K * 32);
-            if (first + K * 32 <= tile_len) {
-                const char *p = reinterpret_cast<const char *>(acc_t + first) + lane * 32;
+            if (pf_lane && first + K * 32 <= tile_len) {     // 24 lanes cover a row's 768 bytes in 32-byte sectors
+                const char *p = pf_base + (size_t)first * sizeof(hbf_access_t);
 #pragma unroll
-                for (int u = 0; u < K; ++u)
-                    if (lane < 24) asm volatile("prefetch.global.L2 [%0];" ::"l"(p + u * 768));
+                for (int u = 0; u < K; ++u) asm volatile("prefetch.global.L2 [%0];" ::"l"(p + u * 768));
             }
         }
         // ---- terms ---------------------------------------------------------------------------------------
@@ -345,7 +347,8 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
                     c_ready += ready[u] ? 1u : 0u;
                     c_native += v[u].st == HBF_ST_NATIVE ? 1u : 0u;
                     if (ready[u]) {
-                        // charged bytes < 2^33: add the low word, carry into the high word when it wraps
+                        // charged bytes < 2^33: add the low word, carry into the high word when it wraps (a form that counts
+                        // granules in one word and sends oversized accesses to the 64-bit totals measured slower)
                         const uint32_t lo = (uint32_t)v[u].cb, hi = (uint32_t)((uint64_t)v[u].cb >> 32);
                         uint32_t *plo = v[u].op ? st_bp_lo : st_br_lo, *phi = v[u].op ? st_bp_hi : st_br_hi;
                         atomicAdd(v[u].op ? &st_np[v[u].die] : &st_nr[v[u].die], 1u);
@@ -365,7 +368,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
         // in lane order, so that the ordered part below is one application of it whatever the row holds
 #pragma unroll
         for (int u = 0; u < K; ++u) {
-            a[u] = issue[u] + (v[u].op ? v[u].xfer : 0);   // arrival at the queue: a program's data is transferred first
+            a[u] = issue[u] + (int64_t)(v[u].op ? v[u].xfer : 0u);   // arrival at the queue: a program's data is transferred first
             const uint32_t q = ready[u] ? v[u].queue : (0x10000u | (uint32_t)lane);
             const unsigned peers = __match_any_sync(0xffffffffu, q);
             const unsigned le = peers & le_mask;
@@ -419,13 +422,13 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
             if (valid[u]) {
                 int64_t done = issue[u], st = 0;             // not modeled: completion = issue, no stall (a refused batch is cleared at the end)
                 if (ready[u]) {
-                    done = B[u] + (v[u].op ? 0 : v[u].xfer); // a read's data is transferred after its service
+                    done = B[u] + (int64_t)(v[u].op ? 0u : v[u].xfer); // a read's data is transferred after its service
                     st = done - issue[u];
                     sum_stall += st; max_c = max(max_c, (long long)done);
                     if (HEADS) {
                         const uint32_t ci = c0[u] + rank1[u] - 1u;
                         if (ci < (uint32_t)kInHead) {
-                            InHead h; h.m = a[u] + v[u].s; h.s = v[u].s; h.xo = (uint32_t)v[u].xfer | (v[u].op << 31); h.idx = (uint32_t)tile_begin + i[u];
+                            InHead h; h.m = a[u] + v[u].s; h.s = v[u].s; h.xo = v[u].xfer | (v[u].op << 31); h.idx = (uint32_t)tile_begin + i[u];
                             in_head[((uint64_t)tile * kInHead + ci) * R + qi[u]] = h;
                         }
                         if (last[u] && c1[u] != c0[u] && c1[u] == (uint32_t)kInHead) atomicAdd(&s_heads_full, 1u);
@@ -714,7 +717,7 @@ k_inorder_straggle(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t ti
                 if (DEBT && cbase + e < claim_limit) v.s += quantum_ns;
                 const uint32_t pos = s_cells[j * kInStrWarps + warp] + rk[j];
                 ent_as[pos] = make_longlong2(issue, v.s);
-                ent_pq[pos] = make_uint2((uint32_t)v.xfer | (v.op << 31), v.queue | (e << 16));
+                ent_pq[pos] = make_uint2(v.xfer | (v.op << 31), v.queue | (e << 16));
             }
         __syncthreads();
         // ---- one thread per straggling queue walks the kept records (they are in batch order) and re-serves its own
