@@ -129,7 +129,8 @@ __device__ __forceinline__ FastGeom make_fast_geom(const FastRange &f, const Mod
 // No branches: every access computes every term, and the classification (the same tests in the same order as classify())
 // only selects the status; the terms of an access that is not READY are never used.  (Early returns cost this pass
 // about 47 instructions per row of 32 accesses, measured.)
-__device__ __forceinline__ Served serve_terms_geom(const FastGeom &g, const ModelParams &mp, uint64_t addr, int64_t issue, uint64_t bf) {
+__device__ __forceinline__ Served serve_terms_geom(const FastGeom &g, const ModelParams &mp, uint64_t addr, int64_t issue, uint64_t bf,
+                                                  int64_t q_ppm, const Div64 &div_q) {
     Served r;
     const uint32_t bytes = (uint32_t)bf, flags = (uint32_t)(bf >> 32);
     const uint64_t rel = addr - g.base;                       // wraps to a huge value below the base
@@ -155,7 +156,8 @@ __device__ __forceinline__ Served serve_terms_geom(const FastGeom &g, const Mode
     r.cb = (int64_t)cb;
     r.xfer = cb <= (uint64_t)g.tab_max_cb ? __ldg(g.xfer_tab + ((uint32_t)cb >> g.tab_shift))
                                             : (uint32_t)div64(cb * 1000ull + mp.chan_bytes_per_us - 1ull, mp.div_chan);
-    r.s = (int64_t)((uint64_t)npages * (op ? g.t_prog : g.t_read));
+    const uint64_t s0 = (uint64_t)npages * (op ? g.t_prog : g.t_read);
+    r.s = q_ppm == 1000000 ? (int64_t)s0 : (int64_t)div64(s0 * 1000000ull + (uint64_t)q_ppm - 1ull, div_q);   // Eq. 3 (s0 < 2^50)
     return r;
 }
 // per-tile bookkeeping of the stall total: as-if-idle sum, fix-up corrections, and the exact sum of a re-served tile
@@ -219,7 +221,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
     const int64_t q_ppm = ctrl->q_ppm;
     const Div64 div_q = ctrl->div_q;
     // one range, power-of-two geometry, transfer table, no thermal scaling in force: the short form of the terms
-    const bool fast_on = fast_geom_ok(fast_arg, mp_arg) && q_ppm == 1000000;
+    const bool fast_on = fast_geom_ok(fast_arg, mp_arg);
     const uint64_t claim_limit = DEBT ? *claim_limit_p : 0ull;
     const int64_t quantum_ns = !DEBT ? 0 : q_ppm == 1000000 ? mp_arg.t_read_ns + mp_arg.t_prog_ns
         : (int64_t)div64((uint64_t)(mp_arg.t_read_ns + mp_arg.t_prog_ns) * 1000000ull + (uint64_t)q_ppm - 1ull, div_q);
@@ -321,7 +323,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
         for (int u = 0; u < K; ++u) {
             v[u].st = HBF_ST_NATIVE; v[u].queue = 0; v[u].die = 0; v[u].op = 0; v[u].s = 0; v[u].xfer = 0; v[u].cb = 0;
             if (valid[u])
-                v[u] = fast_on ? serve_terms_geom(geom, mp, addr[u], issue[u], bf[u])
+                v[u] = fast_on ? serve_terms_geom(geom, mp, addr[u], issue[u], bf[u], q_ppm, div_q)
                                  : serve_terms(rs, mp, addr[u], issue[u], bf[u], q_ppm, div_q);
             ready[u] = valid[u] && v[u].st == HBF_ST_READY;
             if (DEBT && ready[u] && tile_begin + i[u] < claim_limit) {
