@@ -35,7 +35,7 @@ namespace hbf {
 // Block shape of the serve kernel.  The per-queue state (32 KB) is all the shared memory a block needs, so
 // several blocks share an SM, each with its own tile and its own row-after-row chain of queue updates.
 #ifndef HBF_IN_THREADS
-#define HBF_IN_THREADS 384
+#define HBF_IN_THREADS 320
 #endif
 #ifndef HBF_IN_BLOCKS
 #define HBF_IN_BLOCKS 2
@@ -44,7 +44,7 @@ constexpr int kInThreads = HBF_IN_THREADS;               // threads of a serve b
 constexpr int kInBlocksPerSM = HBF_IN_BLOCKS;            // resident serve blocks per SM
 constexpr int kInWarps = kInThreads / 32;
 #ifndef HBF_IN_ROWS
-#define HBF_IN_ROWS 1
+#define HBF_IN_ROWS 2
 #endif
 #ifndef HBF_IN_PFDIST
 #define HBF_IN_PFDIST 2
