@@ -38,7 +38,7 @@ STAGE_BYTES = {"classify": 24 + 8 + 1, "plan_hist": 8, "scan": 8 + 4 + 24 + 16, 
 NCU_TRAFFIC_BYTES_PER_ACCESS = {"inorder": 42.6}
 # warp instructions the in-order serve pass executes per access (smsp__inst_executed.sum of a one-pass ncu capture at
 # 200 M, profiles/inorder_path_capacity_20M.md) and the SM's issue rate: 148 SMs x 4 schedulers x one instruction per cycle
-NCU_WARP_INSTR_PER_ACCESS = {"inorder": 8.68}
+NCU_WARP_INSTR_PER_ACCESS = {"inorder": 7.76}
 SM_COUNT, SCHEDULERS_PER_SM = 148, 4
 FALLBACK_HBM_GBS = 6650.0
 
