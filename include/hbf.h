@@ -318,7 +318,9 @@ HBF_API int hbf_get_rom_temps(hbf_ctx *ctx, double *host_out, uint64_t cap);
  *   nothing.  Every path applies the claims.
  * hbf_retention_decay: idle_ns of idle time drain floor(idle_ns / scaled quantum time) outstanding quanta.
  * hbf_get_retention_blocks / _plan / _totals synchronise the stream and copy to host memory: per-block arrays
- *   [n_blocks] (each nullable); the outstanding quanta in plan order (quanta == NULL: count only); the counters. */
+ *   [n_blocks] (each nullable); the outstanding quanta in plan order (quanta == NULL: count only); the counters.
+ * hbf_reset returns every block to fresh and empties the plan.  The block state and the plan are library-owned
+ * device memory (33 bytes per block, 4 bytes per page of the medium); they are not part of the hbf_get_state blob. */
 typedef struct {
     uint32_t pages_per_block, blocks_per_plane, blocks_per_zone;   /* blocks_per_plane a multiple of blocks_per_zone */
     uint32_t max_pec;                      /* a block that has committed this many cycles is worn out: no more damage, never eligible */
