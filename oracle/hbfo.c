@@ -289,7 +289,7 @@ int hbfo_service_terms(hbfo_ctx *c, uint32_t bytes, uint64_t npages, uint32_t op
  * of n_bins bins starting at the bin the thermal clock stands in: time before it counts into that bin, time
  * past the ring's end into the ring's last bin. */
 int hbfo_enable_energy_bins(hbfo_ctx *c, int64_t bin_ns, uint32_t n_bins) {
-    if (!c || bin_ns <= 0 || n_bins == 0 || c->ret) return HBFO_E_INVAL;
+    if (!c || bin_ns <= 0 || n_bins == 0) return HBFO_E_INVAL;
     int64_t *l = (int64_t *)calloc((size_t)n_bins * c->n_dies, sizeof(int64_t));
     if (!l) return HBFO_E_NOMEM;
     free(c->ledger);
@@ -399,7 +399,7 @@ static void retention_reset(struct hbfo_retention *r) {
 }
 
 int hbfo_enable_retention(hbfo_ctx *c, const hbfo_retention_config_t *cfg) {
-    if (!c || !cfg || c->ret || c->bin_ns || c->bus_busy) return HBFO_E_INVAL;
+    if (!c || !cfg || c->ret || c->bus_busy) return HBFO_E_INVAL;
     if (cfg->pages_per_block == 0 || cfg->blocks_per_plane == 0 || cfg->blocks_per_zone == 0 ||
         cfg->blocks_per_plane % cfg->blocks_per_zone != 0 || cfg->max_pec == 0) return HBFO_E_INVAL;
     if (!(cfg->l_ref_s > 0.0) || !(cfg->t_ref_c > -273.15) || !(cfg->ea_ev >= 0.0) || !(cfg->accel > 0.0) ||
@@ -633,6 +633,8 @@ int hbfo_submit_batch(hbfo_ctx *c, const hbfo_access_t *acc, uint64_t n, int64_t
     qent_t *ent = (qent_t *)malloc((n_ready ? n_ready : 1) * sizeof(qent_t));
     int rc = HBFO_OK;
     uint64_t claims = 0;                                      /* refresh quanta claimed by this batch */
+    uint8_t *claimed = (uint8_t *)calloc(n ? n : 1, 1);
+    if (!claimed) { rc = HBFO_E_NOMEM; goto done; }
     if (!queue || !die || !a_ns || !s_ns || !post || !cbs || !eng || !cnt || !ent) { rc = HBFO_E_NOMEM; goto done; }
     if (c->order_cap < n_ready) {
         free(c->order); c->order = (uint32_t *)malloc((n_ready ? n_ready : 1) * sizeof(uint32_t));
@@ -653,7 +655,8 @@ int hbfo_submit_batch(hbfo_ctx *c, const hbfo_access_t *acc, uint64_t n, int64_t
         if (c->ret && c->ret->claimed + c->ret->decayed + claims < c->ret->plan_len) {
             /* this admission claims one refresh quantum: its scaled service is reserved before the access's own */
             s += retention_quantum_ns(c, q);
-            c->pending_pj[die[i]] += retention_quantum_pj(c);
+            if (!c->bin_ns) c->pending_pj[die[i]] += retention_quantum_pj(c);   /* with the bins on it is booked where it is served */
+            claimed[i] = 1;
             ++claims;
         }
         if (c->ret && !op) c->ret->disturb[retention_block_of(c, off)] += (uint32_t)np;
@@ -695,7 +698,11 @@ int hbfo_submit_batch(hbfo_ctx *c, const hbfo_access_t *acc, uint64_t n, int64_t
             stall_ns[i] = done_ns - acc[i].issue_ns;
             hbfo_die_stats_t *d = &ds[die[i]];
             d->busy_ns += s_ns[i]; d->energy_pj += eng[i];
-            if (c->bin_ns) ledger_event(c, die[i], start, s_ns[i], eng[i]);
+            if (c->bin_ns && claimed[i]) {                    /* the refresh quantum first, then the access's own service */
+                const int64_t qns = retention_quantum_ns(c, q);
+                ledger_event(c, die[i], start, qns, retention_quantum_pj(c));
+                ledger_event(c, die[i], start + qns, s_ns[i] - qns, eng[i]);
+            } else if (c->bin_ns) ledger_event(c, die[i], start, s_ns[i], eng[i]);
             if (acc[i].flags & 1u) { d->bytes_prog += cbs[i]; d->n_prog += 1; }
             else                   { d->bytes_read += cbs[i]; d->n_read += 1; }
             res.modeled_ns += stall_ns[i]; res.service_ns += s_ns[i];
@@ -743,7 +750,7 @@ int hbfo_submit_batch(hbfo_ctx *c, const hbfo_access_t *acc, uint64_t n, int64_t
 
 done:
     free(st); free(rg); free(queue); free(die); free(a_ns); free(s_ns); free(post); free(cbs); free(eng);
-    free(cnt); free(ent);
+    free(cnt); free(ent); free(claimed);
     return rc;
 }
 

@@ -17,12 +17,29 @@ __device__ __forceinline__ void ledger_add(unsigned long long *ledger, uint32_t 
     if (pj) atomicAdd(&ledger[(size_t)(bin % (int64_t)n_bins) * n_dies + die], (unsigned long long)pj);
 }
 
-// Runs after the batch's results are final: start = completion - (a read's transfer) - service.
+// one event: energy pj over [start, start + s), split over the bins it overlaps
+__device__ __forceinline__ void ledger_event(unsigned long long *ledger, uint32_t n_dies, uint32_t n_bins, int64_t cur_bin, int64_t bin_ns,
+                                             uint32_t die, int64_t start, int64_t s, int64_t pj) {
+    const int64_t end = start + s;
+    const int64_t b0 = start / bin_ns, b1 = (end - 1) / bin_ns;
+    if (b0 == b1) { ledger_add(ledger, n_dies, n_bins, cur_bin, die, b0, pj); return; }
+    int64_t given = 0;
+    for (int64_t b = b0; b < b1; ++b) {
+        const int64_t lo = max(b * bin_ns, start), hi = (b + 1) * bin_ns;
+        const int64_t share = (int64_t)(((unsigned __int128)(uint64_t)pj * (uint64_t)(hi - lo)) / (uint64_t)s);
+        ledger_add(ledger, n_dies, n_bins, cur_bin, die, b, share);
+        given += share;
+    }
+    ledger_add(ledger, n_dies, n_bins, cur_bin, die, b1, pj - given);
+}
+
+// Runs after the batch's results are final: start = completion - (a read's transfer) - service.  With retention on, an
+// access below the claim limit served a refresh quantum first: that is an event of its own, ahead of the access's.
 __global__ void __launch_bounds__(256)
 k_energy_bins(const hbf_access_t *__restrict__ acc, uint64_t n, const int64_t *__restrict__ completion,
               const RangeSnap *__restrict__ ranges, const ModelParams *__restrict__ mp_g, const BatchCtrl *__restrict__ ctrl,
               const hbf_batch_result_t *__restrict__ result, unsigned long long *ledger, int64_t bin_ns, uint32_t n_bins,
-              int64_t cur_bin) {
+              int64_t cur_bin, const unsigned long long *claim_limit_p, int64_t quantum_pj) {
     __shared__ ModelParams mp;
     if (result->code != HBF_OK) return;                      // a refused batch books nothing
     for (int i = threadIdx.x; i < (int)(sizeof(ModelParams) / 4); i += blockDim.x)
@@ -32,6 +49,9 @@ k_energy_bins(const hbf_access_t *__restrict__ acc, uint64_t n, const int64_t *_
     const int64_t q_ppm = ctrl->q_ppm;
     const Div64 div_q = ctrl->div_q;
     const uint32_t n_dies = mp.n_dies;
+    const uint64_t claim_limit = claim_limit_p ? *claim_limit_p : 0ull;
+    const int64_t quantum_ns = q_ppm == 1000000 ? mp.t_read_ns + mp.t_prog_ns
+        : (int64_t)div64((uint64_t)(mp.t_read_ns + mp.t_prog_ns) * 1000000ull + (uint64_t)q_ppm - 1ull, div_q);
     for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (uint64_t)gridDim.x * blockDim.x) {
         const uint64_t *rec = reinterpret_cast<const uint64_t *>(acc + i);
         const uint64_t addr = __ldg(rec), bf = __ldg(rec + 2);
@@ -42,17 +62,12 @@ k_energy_bins(const hbf_access_t *__restrict__ acc, uint64_t n, const int64_t *_
         const Decoded d = decode(mp, rs.media_offset[g] + (addr - rs.base[g]), bytes);
         const uint32_t op = flags & 1u;
         const Terms t = service_terms(mp, bytes, d.npages, op, q_ppm, div_q);
-        const int64_t end = completion[i] - (op ? 0 : t.xfer), start = end - t.s;
-        const int64_t b0 = start / bin_ns, b1 = (end - 1) / bin_ns;
-        if (b0 == b1) { ledger_add(ledger, n_dies, n_bins, cur_bin, d.die, b0, t.energy); continue; }
-        int64_t given = 0;
-        for (int64_t b = b0; b < b1; ++b) {
-            const int64_t lo = max(b * bin_ns, start), hi = (b + 1) * bin_ns;
-            const int64_t share = (int64_t)(((unsigned __int128)(uint64_t)t.energy * (uint64_t)(hi - lo)) / (uint64_t)t.s);
-            ledger_add(ledger, n_dies, n_bins, cur_bin, d.die, b, share);
-            given += share;
+        const int64_t end = completion[i] - (op ? 0 : t.xfer);
+        int64_t start = end - t.s;
+        if (i < claim_limit) {
+            ledger_event(ledger, n_dies, n_bins, cur_bin, bin_ns, d.die, start - quantum_ns, quantum_ns, quantum_pj);
         }
-        ledger_add(ledger, n_dies, n_bins, cur_bin, d.die, b1, t.energy - given);
+        ledger_event(ledger, n_dies, n_bins, cur_bin, bin_ns, d.die, start, t.s, t.energy);
     }
 }
 
@@ -65,10 +80,10 @@ __global__ void k_take_bin(unsigned long long *row, int64_t *pending, uint32_t n
 cudaError_t launch_energy_bins(const hbf_access_t *acc, uint64_t n, const int64_t *completion, const RangeSnap *ranges,
                                const ModelParams *mp_dev, const BatchCtrl *ctrl, const hbf_batch_result_t *result,
                                unsigned long long *ledger, int64_t bin_ns, uint32_t n_bins, int64_t cur_bin, int sm_count,
-                               cudaStream_t st) {
+                               const unsigned long long *claim_limit, int64_t quantum_pj, cudaStream_t st) {
     if (n == 0) return cudaSuccess;
     const unsigned grid = (unsigned)std::min<uint64_t>((n + 255) / 256, (uint64_t)std::max(1, sm_count) * 8);
-    k_energy_bins<<<grid, 256, 0, st>>>(acc, n, completion, ranges, mp_dev, ctrl, result, ledger, bin_ns, n_bins, cur_bin);
+    k_energy_bins<<<grid, 256, 0, st>>>(acc, n, completion, ranges, mp_dev, ctrl, result, ledger, bin_ns, n_bins, cur_bin, claim_limit, quantum_pj);
     g_kernel_launches += 1;
     return cudaGetLastError();
 }

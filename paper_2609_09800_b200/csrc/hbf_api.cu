@@ -434,11 +434,14 @@ int hbf_submit_batch(hbf_ctx *c, const hbf_access_t *d_acc, uint64_t n, int64_t 
         a.claim_limit = &c->ret.st->claim_limit; a.die_claims = c->ret.die_claims; a.ret = &c->ret;
     }
     CK(launch_submit(a, c->stream));
-    if (c->ret_on)                                           // read disturb, commits, the claimed energy
-        CK(launch_ret_close(d_acc, n, c->d_ranges, c->d_mp, c->mp, c->d_result, c->d_pending, c->ret, c->sm_count, c->stream));
-    if (a.binned)
+    if (a.binned) {
+        const int64_t page = (int64_t)1 << c->mp.page_shift;
+        const int64_t quantum_pj = c->mp.e_cmd_read_pj + c->mp.e_byte_read_pj * page + c->mp.e_cmd_prog_pj + c->mp.e_byte_prog_pj * page;
         CK(launch_energy_bins(d_acc, n, d_completion_ns, c->d_ranges, c->d_mp, c->d_ctrl, c->d_result, c->d_ledger, c->bin_ns,
-                              c->n_bins, c->cur_bin, c->sm_count, c->stream));
+                              c->n_bins, c->cur_bin, c->sm_count, a.claim_limit, quantum_pj, c->stream));
+    }
+    if (c->ret_on)                                           // read disturb, commits, the claimed energy (after the ledger: it needs the claim limit)
+        CK(launch_ret_close(d_acc, n, c->d_ranges, c->d_mp, c->mp, c->d_result, c->d_pending, a.binned, c->ret, c->sm_count, c->stream));
     if (c->d_bus_busy)                                       // after the ledger: its events are the array intervals
         CK(launch_bus_stage(a, c->d_bus_ctrl, c->d_bus_busy, c->stream));
     c->submitted = true;
@@ -513,7 +516,7 @@ int hbf_get_bus_busy_until(hbf_ctx *c, int64_t *host_out, uint64_t cap) {
 }
 
 int hbf_enable_retention(hbf_ctx *c, const hbf_retention_config_t *cfg) {
-    if (!c || !cfg || c->ret_on || c->bin_ns != 0 || c->d_bus_busy) return HBF_E_INVAL;
+    if (!c || !cfg || c->ret_on || c->d_bus_busy) return HBF_E_INVAL;
     if (!cfg->pages_per_block || !cfg->blocks_per_plane || !cfg->blocks_per_zone ||
         cfg->blocks_per_plane % cfg->blocks_per_zone != 0 || !cfg->max_pec) return HBF_E_INVAL;
     if (!(cfg->l_ref_s > 0.0) || !(cfg->t_ref_c > -273.15) || !(cfg->ea_ev >= 0.0) || !(cfg->accel > 0.0) ||
@@ -612,7 +615,7 @@ int hbf_get_retention_totals(hbf_ctx *c, hbf_retention_totals_t *out) {
 }
 
 int hbf_enable_energy_bins(hbf_ctx *c, int64_t bin_ns, uint32_t n_bins) {
-    if (!c || bin_ns <= 0 || n_bins == 0 || c->ret_on) return HBF_E_INVAL;
+    if (!c || bin_ns <= 0 || n_bins == 0) return HBF_E_INVAL;
     CK(cudaStreamSynchronize(c->stream));
     unsigned long long *l = nullptr;
     if (cudaMalloc(&l, (size_t)n_bins * c->mp.n_dies * 8) != cudaSuccess) return HBF_E_NOMEM;

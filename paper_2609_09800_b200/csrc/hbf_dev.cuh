@@ -156,7 +156,7 @@ cudaError_t launch_paged_join(const hbf_access_t *acc, uint64_t n, const PagedWo
 cudaError_t launch_energy_bins(const hbf_access_t *acc, uint64_t n, const int64_t *completion, const RangeSnap *ranges,
                                const ModelParams *mp_dev, const BatchCtrl *ctrl, const hbf_batch_result_t *result,
                                unsigned long long *ledger, int64_t bin_ns, uint32_t n_bins, int64_t cur_bin, int sm_count,
-                               cudaStream_t st);
+                               const unsigned long long *claim_limit, int64_t quantum_pj, cudaStream_t st);
 cudaError_t launch_take_bin(unsigned long long *row, int64_t *pending, uint32_t n_dies, cudaStream_t st);
 
 // ---- reduced-order thermal model -------------------------------------------------------------------------
@@ -193,7 +193,7 @@ struct RetDev {
 };
 cudaError_t launch_ret_window(const hbf_access_t *acc, uint64_t n, const RangeSnap *ranges, const RetDev &r, int sm_count, cudaStream_t st);
 cudaError_t launch_ret_close(const hbf_access_t *acc, uint64_t n, const RangeSnap *ranges, const ModelParams *mp_dev, const ModelParams &mp,
-                             const hbf_batch_result_t *result, int64_t *pending, const RetDev &r, int sm_count, cudaStream_t st);
+                             const hbf_batch_result_t *result, int64_t *pending, int binned, const RetDev &r, int sm_count, cudaStream_t st);
 struct ThermalDev;
 cudaError_t launch_ret_advance(const RetDev &r, const ModelParams &mp, const ThermalDev *field, const float *theta, const int32_t *die_region,
                                int have_temps, int64_t dt_ns, int sm_count, cudaStream_t st);

@@ -207,12 +207,12 @@ static unsigned ret_grid(uint64_t items, int sm_count) {
 }
 
 cudaError_t launch_ret_close(const hbf_access_t *acc, uint64_t n, const RangeSnap *ranges, const ModelParams *mp_dev, const ModelParams &mp,
-                             const hbf_batch_result_t *result, int64_t *pending, const RetDev &r, int sm_count, cudaStream_t st) {
+                             const hbf_batch_result_t *result, int64_t *pending, int binned, const RetDev &r, int sm_count, cudaStream_t st) {
     if (n) k_ret_observe<<<ret_grid(n, sm_count), 256, 0, st>>>(acc, n, ranges, mp_dev, result, r);
     k_ret_commit<<<ret_grid(r.n_blocks, sm_count), 256, 0, st>>>(result, r);
     const int64_t page = (int64_t)1 << mp.page_shift;
     const int64_t quantum_pj = mp.e_cmd_read_pj + mp.e_byte_read_pj * page + mp.e_cmd_prog_pj + mp.e_byte_prog_pj * page;
-    k_ret_close<<<1, 256, 0, st>>>(result, pending, quantum_pj, mp.n_dies, r);
+    k_ret_close<<<1, 256, 0, st>>>(result, pending, binned ? 0 : quantum_pj, mp.n_dies, r);   // with the time bins on, the ledger has it
     g_kernel_launches += n ? 3 : 2;
     return cudaGetLastError();
 }

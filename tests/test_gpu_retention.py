@@ -251,12 +251,34 @@ def test_refused_batch_changes_nothing(hbf):
     assert compare_batch(g, o, recs([(PAGE, 2 * 10**7, 64, 0)])) == 0
 
 
-def test_not_with_the_other_extensions(hbf):
+@pytest.mark.parametrize("path", ["auto", "sort"])
+def test_with_the_energy_bins(hbf, path):
+    """Claimed quanta are ledger events of their own; the ledger, the pending totals after thermal-clock steps and
+    everything else stay bit-exact."""
+    fp = wl.toy_floorplan(16, 48, 8, 4)
+    ret = dict(RET, disturb_limit=2, lead_threshold=1e9, pages_per_block=16)
+    g, o, prof = contexts(hbf, ret, floorplan=fp, path=hbf.PATH_AUTO if path == "auto" else hbf.PATH_SORT)
+    g.enable_energy_bins(200_000, 16); o.enable_energy_bins(200_000, 16)
+    rng = np.random.default_rng(21)
+    t0 = 0
+    for round_ in range(5):
+        acc = mixed_batch(rng, 6000, t0, 4096, gap=300)
+        assert compare_batch(g, o, acc) == 0
+        fg, bg = g.energy_bins(); fo, bo = o.energy_bins()
+        assert fg == fo and np.array_equal(bg, bo)
+        t0 = int(acc["issue_ns"][-1]) + 1
+        g.thermal_step(200_000); o.thermal_step(200_000)
+        assert np.array_equal(g.get_pending_energy(), o.pending_energy())
+        temps = np.full(len(fp["region_kind"]), 50.0)
+        g.retention_advance(10**9, temps); o.retention_advance(10**9, temps)
+        compare_state(g, o)
+    assert o.retention_totals()["claimed"] > 1000
+
+
+def test_not_with_the_bus_or_the_paged_submit(hbf):
     g, o, prof = contexts(hbf, RET)
     with pytest.raises(hbf.HbfError):
         g.enable_channel_bus()
-    with pytest.raises(hbf.HbfError):
-        g.enable_energy_bins(1000, 4)
     acc = recs([(0, 0, 64, 0)])
     rc, *_ = g.submit_host(acc, check=False, parts_capacity=4)
     assert rc == hbf.E_INVAL

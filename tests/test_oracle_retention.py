@@ -340,11 +340,37 @@ def test_refused_batch_changes_nothing():
         assert np.array_equal(before[1][k], after[1][k])
 
 
-def test_not_with_the_other_extensions():
+def test_not_with_the_bus_or_the_paged_submit():
     o, _ = make(RET)
     with pytest.raises(hbfo.OracleError):
         o.enable_channel_bus()
-    with pytest.raises(hbfo.OracleError):
-        o.enable_energy_bins(1000, 4)
     rc, *_ = o.submit(recs([(0, 0, 64, 0)]), check=False, paged=True)
     assert rc != 0
+
+
+def test_with_the_energy_bins_a_claimed_quantum_is_an_event_of_its_own():
+    """One claim on an idle queue, bins of 100 us: the quantum (395 us, 15.1 uJ) fills bins 10..13 in proportion to the
+    time it spends in each, the read's own 20 us and 344 nJ follow in bin 13/14; nothing goes to the pending totals."""
+    ret = dict(RET, disturb_limit=1, lead_threshold=1e9, pages_per_block=1)
+    o, prof = make(ret)
+    o.enable_energy_bins(100_000, 32)
+    o.submit(recs([(0, 0, 64, 0)]))
+    o.retention_advance(0, np.array([40.0]))
+    first, before = o.energy_bins()
+    off = offset_of(prof, ret, 3, 2, 1, 0)
+    _, comp, _, _, _ = o.submit(recs([(off, 1_000_000, 4096, 0)]))
+    assert comp[0] == 1_000_000 + 395_000 + 20_000 + 171
+    first, bins = o.energy_bins()
+    die = 3 * prof["dies"] + 2
+    got = (bins - before)[:, die]
+    quantum_pj, read_pj = (84 + 840) * PAGE, 84 * 4096
+    want = np.zeros(32, np.int64)
+    for k in range(10, 13):
+        want[k] = quantum_pj * 100_000 // 395_000
+    want[13] = quantum_pj - 3 * (quantum_pj * 100_000 // 395_000)        # the quantum's last bin takes what is left
+    want[13] += read_pj * 5_000 // 20_000                                 # the read's service runs from 1,395,000 to 1,415,000
+    want[14] = read_pj - read_pj * 5_000 // 20_000
+    assert got.tolist() == want.tolist()
+    assert int((bins - before).sum()) == quantum_pj + read_pj
+    pend = np.zeros(o.n_dies, np.int64); hbfo.lib().hbfo_get_pending_energy(o._h, pend.ctypes.data, pend.size)
+    assert int(pend.sum()) == 0
