@@ -304,8 +304,8 @@ HBF_API int hbf_get_rom_temps(hbf_ctx *ctx, double *host_out, uint64_t cap);
  * page, programs add nothing; the modeled accesses of a batch claim in index (ticket) order; commits take effect
  * when the batch, or the decay, that claimed a block's last quantum has completed.
  *
- * hbf_enable_retention: allocates the block state (all fresh).  Not together with the channel bus or the page-granular
- *   submit (HBF_E_INVAL from whichever comes second).  With the energy bins on, a claimed quantum is an event of its
+ * hbf_enable_retention: allocates the block state (all fresh).  hbf_submit_batch_paged is refused while it is on.  The
+ *   channel-bus stage works on top of it unchanged (claims lengthen the array stage only).  With the energy bins on, a claimed quantum is an event of its
  *   own in the ledger: its energy over the interval in which it was served, ahead of the claiming access's event.
  * hbf_retention_advance: one epoch, asynchronously on the context's stream.  Every block that is not worn out gains
  *   accel * dt / L(T) of damage, T being the temperature of its die's floorplan region: region_temp_c [n_regions]

@@ -334,7 +334,7 @@ static void ledger_event(hbfo_ctx *c, uint32_t die, int64_t start, int64_t s, in
  * (D, batch index) order behind whatever earlier batches left on that bus, and occupies it for the transfer time.
  * The read completes when its transfer does.  Programs keep their transfer as a latency before the array time. */
 int hbfo_enable_channel_bus(hbfo_ctx *c) {
-    if (!c || c->ret) return HBFO_E_INVAL;
+    if (!c) return HBFO_E_INVAL;
     if (!c->bus_busy) c->bus_busy = (int64_t *)calloc(c->cfg.channels, sizeof(int64_t));
     return c->bus_busy ? HBFO_OK : HBFO_E_NOMEM;
 }
@@ -399,7 +399,7 @@ static void retention_reset(struct hbfo_retention *r) {
 }
 
 int hbfo_enable_retention(hbfo_ctx *c, const hbfo_retention_config_t *cfg) {
-    if (!c || !cfg || c->ret || c->bus_busy) return HBFO_E_INVAL;
+    if (!c || !cfg || c->ret) return HBFO_E_INVAL;
     if (cfg->pages_per_block == 0 || cfg->blocks_per_plane == 0 || cfg->blocks_per_zone == 0 ||
         cfg->blocks_per_plane % cfg->blocks_per_zone != 0 || cfg->max_pec == 0) return HBFO_E_INVAL;
     if (!(cfg->l_ref_s > 0.0) || !(cfg->t_ref_c > -273.15) || !(cfg->ea_ev >= 0.0) || !(cfg->accel > 0.0) ||

@@ -119,7 +119,7 @@ int64_t hbfo_quantise_mk(double t_c);
 const char *hbfo_strerror(int code);
 
 /* Retention, refresh and wear (Design D4; the definitions and the readings are at the head of this part of
- * hbfo.c).  Not together with the channel bus or the page-granular submit; with the energy bins on, a claimed
+ * hbfo.c).  Not together with the page-granular submit; with the energy bins on, a claimed
  * quantum is booked as an event of its own ahead of the claiming access's.
  *   hbfo_enable_retention     block state for channels*dies*planes*blocks_per_plane blocks, all fresh
  *   hbfo_retention_advance    one epoch: damage += accel*dt/L(T) per block with its die's region temperature

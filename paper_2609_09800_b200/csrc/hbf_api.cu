@@ -496,7 +496,7 @@ int hbf_submit_batch_paged(hbf_ctx *c, const hbf_access_t *d_acc, uint64_t n, ui
 }
 
 int hbf_enable_channel_bus(hbf_ctx *c) {
-    if (!c || c->ret_on) return HBF_E_INVAL;
+    if (!c) return HBF_E_INVAL;
     if (c->d_bus_busy) return HBF_OK;
     CK(cudaStreamSynchronize(c->stream));
     int64_t *b = nullptr; BatchCtrl *bc = nullptr;
@@ -516,7 +516,7 @@ int hbf_get_bus_busy_until(hbf_ctx *c, int64_t *host_out, uint64_t cap) {
 }
 
 int hbf_enable_retention(hbf_ctx *c, const hbf_retention_config_t *cfg) {
-    if (!c || !cfg || c->ret_on || c->d_bus_busy) return HBF_E_INVAL;
+    if (!c || !cfg || c->ret_on) return HBF_E_INVAL;
     if (!cfg->pages_per_block || !cfg->blocks_per_plane || !cfg->blocks_per_zone ||
         cfg->blocks_per_plane % cfg->blocks_per_zone != 0 || !cfg->max_pec) return HBF_E_INVAL;
     if (!(cfg->l_ref_s > 0.0) || !(cfg->t_ref_c > -273.15) || !(cfg->ea_ev >= 0.0) || !(cfg->accel > 0.0) ||

@@ -275,16 +275,28 @@ def test_with_the_energy_bins(hbf, path):
     assert o.retention_totals()["claimed"] > 1000
 
 
-def test_not_with_the_bus_or_the_paged_submit(hbf):
+@pytest.mark.parametrize("path", ["auto", "sort"])
+def test_with_the_channel_bus(hbf, path):
+    ret = dict(RET, disturb_limit=2, lead_threshold=1e9, pages_per_block=16)
+    g, o, prof = contexts(hbf, ret, path=hbf.PATH_AUTO if path == "auto" else hbf.PATH_SORT)
+    g.enable_channel_bus(); o.enable_channel_bus()
+    rng = np.random.default_rng(31)
+    t0 = 0
+    for round_ in range(4):
+        acc = mixed_batch(rng, 8000, t0, 4096, gap=300)
+        assert compare_batch(g, o, acc) == 0
+        assert np.array_equal(g.get_bus_busy_until(), o.bus_busy_until())
+        t0 = int(acc["issue_ns"][-1]) + 1
+        g.retention_advance(10**9, np.array([50.0])); o.retention_advance(10**9, np.array([50.0]))
+        compare_state(g, o)
+    assert o.retention_totals()["claimed"] > 1000
+
+
+def test_not_with_the_paged_submit(hbf):
     g, o, prof = contexts(hbf, RET)
-    with pytest.raises(hbf.HbfError):
-        g.enable_channel_bus()
     acc = recs([(0, 0, 64, 0)])
     rc, *_ = g.submit_host(acc, check=False, parts_capacity=4)
     assert rc == hbf.E_INVAL
-    g2 = hbf.Context(prof); g2.enable_channel_bus()
-    with pytest.raises(hbf.HbfError):
-        g2.enable_retention(**RET)
 
 
 def test_reset_clears_the_block_state(hbf):

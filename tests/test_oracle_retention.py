@@ -340,12 +340,24 @@ def test_refused_batch_changes_nothing():
         assert np.array_equal(before[1][k], after[1][k])
 
 
-def test_not_with_the_bus_or_the_paged_submit():
+def test_not_with_the_paged_submit():
     o, _ = make(RET)
-    with pytest.raises(hbfo.OracleError):
-        o.enable_channel_bus()
     rc, *_ = o.submit(recs([(0, 0, 64, 0)]), check=False, paged=True)
     assert rc != 0
+
+
+def test_with_the_channel_bus_claims_lengthen_the_array_stage_only():
+    """Two reads on two dies of one channel, both claiming: the arrays finish at 415,000; the bus then moves the
+    first read's 16 KiB until 415,683 and the second's until 416,366."""
+    ret = dict(RET, disturb_limit=1, lead_threshold=1e9, pages_per_block=2)
+    o, prof = make(ret)
+    o.enable_channel_bus()
+    o.submit(recs([(offset_of(prof, ret, 5, 0, 0, 0), 0, 64, 0)]))
+    o.retention_advance(0, np.array([40.0]))
+    rows = [(offset_of(prof, ret, 0, 0, 0, 0), 10**6, PAGE, 0), (offset_of(prof, ret, 0, 1, 0, 0), 10**6, PAGE, 0)]
+    _, comp, _, _, _ = o.submit(recs(rows))
+    assert comp.tolist() == [10**6 + 415_683, 10**6 + 416_366]
+    assert o.retention_totals()["claimed"] == 2
 
 
 def test_with_the_energy_bins_a_claimed_quantum_is_an_event_of_its_own():
