@@ -21,7 +21,10 @@
  * an independent event-driven brute force on tiny inputs, the M/D/1 mean wait, the printed power
  * figure 37.256 W at 384 GB/s, thermal steady state against a direct linear solve and the lumped
  * closed form.  Parity unpinned (no value in the paper, fixed by the committed profile only):
- * program energy per byte, the threshold temperatures, q_light, the floorplan constants.
+ * program energy per byte, the threshold temperatures, q_light, the floorplan constants; of the retention part
+ * (Design D4) everything beyond the two equations, the eligibility rule, the emission order and the claim rule:
+ * the block layout, the cost and the booking of a quantum, the read-disturb increment, when a commit takes effect,
+ * the decay rate (pinned against hand-worked examples of this build's own definitions only).
  *
  * All times int64 ns on one shared origin; energies int64 pJ; temperatures double, deg C.
  */
