@@ -195,9 +195,13 @@ HBF_API int hbf_get_mode(hbf_ctx *ctx, int32_t *mode, int64_t *q_ppm);          
 HBF_API int hbf_reset(hbf_ctx *ctx);                                             /* queues idle, field at ambient, mode Normal */
 
 /* Chooses how batches are ordered: HBF_PATH_AUTO (default) serves a batch whose records arrive in
- * non-decreasing issue order without a global sort and falls back to the radix sort otherwise;
+ * non-decreasing issue order without a global sort and falls back to the radix sort otherwise (also for a batch in
+ * which a single access's service time reaches 2^33 ns, 2^32 ns with retention on: the in-order kernels keep
+ * per-tile sums of service times in 56 bits);
  * HBF_PATH_SORT always sorts (a batch already in issue order is sorted on its queue bits only, which a
- * stable sort allows); HBF_PATH_SORT_FULL sorts on every key bit regardless.  All give identical results. */
+ * stable sort allows); HBF_PATH_SORT_FULL sorts on every key bit regardless; HBF_PATH_INORDER is the caller's
+ * declaration that its batches are in issue order: only the in-order kernels are launched, and a batch that is not in
+ * issue order, or has such a long service time, is refused with HBF_E_INVAL.  All give identical results. */
 HBF_API int hbf_set_path(hbf_ctx *ctx, int32_t path);
 /* Thermal step implementation: 0 (default) runs the whole step in one launch of a thread-block cluster when
  * the grid fits its shared memory (up to 32,768 cells), else one launch per substep; 1 always uses the latter.

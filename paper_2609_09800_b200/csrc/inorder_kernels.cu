@@ -56,8 +56,12 @@ static_assert(kInWarps >= 2 && kInWarps <= 15, "every warp owns one of the hardw
 // One access, from its record: status, and for a modeled access its queue, die and service terms.
 // (the in-order path is only chosen when every transfer time fits 31 bits)
 struct Served { int st; uint32_t queue, die, op, xfer; int64_t s, cb; };
+// long_service (here and below): set when one access's service time reaches 2^long_bits ns.  The serve pass keeps a tile's
+// service-time sum per queue in 56 bits (55 and a sign); a tile has fewer than 2^22 records, so with every service below
+// 2^33 ns (8.6 s) the sum cannot overflow; with retention on a claimed refresh quantum is added to a service, and both
+// stay below 2^32.  A batch with a longer service is handed to the sort path like an unsorted one.
 __device__ __forceinline__ Served serve_terms(const RangeSnap &rs, const ModelParams &mp, uint64_t addr, int64_t issue,
-                                              uint64_t bf, int64_t q_ppm, const Div64 &div_q) {
+                                              uint64_t bf, int64_t q_ppm, const Div64 &div_q, unsigned &long_service, int long_bits) {
     Served r; r.queue = 0; r.die = 0; r.op = 0; r.s = 0; r.xfer = 0; r.cb = 0;
     const uint32_t bytes = (uint32_t)bf, flags = (uint32_t)(bf >> 32);
     int g = 0;
@@ -68,6 +72,7 @@ __device__ __forceinline__ Served serve_terms(const RangeSnap &rs, const ModelPa
         r.op = flags & 1u;
         const Terms t = service_terms(mp, bytes, d.npages, r.op, q_ppm, div_q);
         r.queue = d.queue; r.die = d.die; r.s = t.s; r.xfer = (uint32_t)t.xfer; r.cb = t.cb;
+        if ((uint64_t)t.s >> long_bits) long_service = 1u;
     }
     return r;
 }
@@ -111,8 +116,12 @@ struct __align__(16) FastGeom {
     uint32_t tab_shift, tab_max_cb, t_read, t_prog;
     const uint32_t *xfer_tab; uint64_t pad;
 };
+// (the last condition: an access within the transfer table's reach spans few pages, and their unscaled service stays
+// below 2^32 ns, so the common path needs no test of its own)
 __device__ __forceinline__ bool fast_geom_ok(const FastRange &f, const ModelParams &mp) {
-    return f.on != 0u && mp.pow2_geom != 0u && mp.xfer_tab_max_cb != 0u && mp.t_read_ns < (1ll << 32) && mp.t_prog_ns < (1ll << 32);
+    const uint64_t pages = ((uint64_t)mp.xfer_tab_max_cb >> mp.page_shift) + 2ull;
+    return f.on != 0u && mp.pow2_geom != 0u && mp.xfer_tab_max_cb != 0u && mp.t_read_ns < (1ll << 32) && mp.t_prog_ns < (1ll << 32) &&
+           pages * (uint64_t)max(mp.t_read_ns, mp.t_prog_ns) < (1ull << 32);
 }
 __device__ __forceinline__ FastGeom make_fast_geom(const FastRange &f, const ModelParams &mp) {
     FastGeom g;
@@ -130,7 +139,7 @@ __device__ __forceinline__ FastGeom make_fast_geom(const FastRange &f, const Mod
 // only selects the status; the terms of an access that is not READY are never used.  (Early returns cost this pass
 // about 47 instructions per row of 32 accesses, measured.)
 __device__ __forceinline__ Served serve_terms_geom(const FastGeom &g, const ModelParams &mp, uint64_t addr, int64_t issue, uint64_t bf,
-                                                  int64_t q_ppm, const Div64 &div_q) {
+                                                  int64_t q_ppm, const Div64 &div_q, unsigned &long_service, int long_bits) {
     Served r;
     const uint32_t bytes = (uint32_t)bf, flags = (uint32_t)(bf >> 32);
     const uint64_t rel = addr - g.base;                       // wraps to a huge value below the base
@@ -154,10 +163,19 @@ __device__ __forceinline__ Served serve_terms_geom(const FastGeom &g, const Mode
     const uint64_t gm = (1ull << gs) - 1ull;
     const uint64_t cb = ((uint64_t)bytes + gm) & ~gm;
     r.cb = (int64_t)cb;
-    r.xfer = cb <= (uint64_t)g.tab_max_cb ? __ldg(g.xfer_tab + ((uint32_t)cb >> g.tab_shift))
-                                            : (uint32_t)div64(cb * 1000ull + mp.chan_bytes_per_us - 1ull, mp.div_chan);
     const uint64_t s0 = (uint64_t)npages * (op ? g.t_prog : g.t_read);
-    r.s = q_ppm == 1000000 ? (int64_t)s0 : (int64_t)div64(s0 * 1000000ull + (uint64_t)q_ppm - 1ull, div_q);   // Eq. 3 (s0 < 2^50)
+    if (cb <= (uint64_t)g.tab_max_cb) {
+        r.xfer = __ldg(g.xfer_tab + ((uint32_t)cb >> g.tab_shift));
+    } else {                                                  // a large access: rare
+        r.xfer = (uint32_t)div64(cb * 1000ull + mp.chan_bytes_per_us - 1ull, mp.div_chan);
+        if (s0 >> long_bits) long_service = 1u;
+    }
+    if (q_ppm == 1000000) {
+        r.s = (int64_t)s0;
+    } else {                                                  // thermal scaling in force: Eq. 3 (s0 < 2^50)
+        r.s = (int64_t)div64(s0 * 1000000ull + (uint64_t)q_ppm - 1ull, div_q);
+        if ((uint64_t)r.s >> long_bits) long_service = 1u;
+    }
     return r;
 }
 // per-tile bookkeeping of the stall total: as-if-idle sum, fix-up corrections, and the exact sum of a re-served tile
@@ -249,7 +267,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
         }
     }
     uint32_t c_native = 0, c_ready = 0, c_valid = 0;         // per thread: far below 2^32 (a batch is below 2^30 records)
-    unsigned c_unsorted = 0;
+    unsigned c_unsorted = (DEBT && ((uint64_t)quantum_ns >> 32)) ? 1u : 0u;   // (or a service, or a refresh quantum, of 2^32 ns or more)
     long long sum_stall = 0, max_c = INT64_MIN;
 
     if (tid < 2) s_red[tid] = tid == 1 ? INT64_MIN : 0;
@@ -323,8 +341,8 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
         for (int u = 0; u < K; ++u) {
             v[u].st = HBF_ST_NATIVE; v[u].queue = 0; v[u].die = 0; v[u].op = 0; v[u].s = 0; v[u].xfer = 0; v[u].cb = 0;
             if (valid[u])
-                v[u] = fast_on ? serve_terms_geom(geom, mp, addr[u], issue[u], bf[u], q_ppm, div_q)
-                                 : serve_terms(rs, mp, addr[u], issue[u], bf[u], q_ppm, div_q);
+                v[u] = fast_on ? serve_terms_geom(geom, mp, addr[u], issue[u], bf[u], q_ppm, div_q, c_unsorted, DEBT ? 32 : 33)
+                                 : serve_terms(rs, mp, addr[u], issue[u], bf[u], q_ppm, div_q, c_unsorted, DEBT ? 32 : 33);
             ready[u] = valid[u] && v[u].st == HBF_ST_READY;
             if (DEBT && ready[u] && tile_begin + i[u] < claim_limit) {
                 v[u].s += quantum_ns;
@@ -652,6 +670,7 @@ k_inorder_straggle(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t ti
         : (int64_t)div64((uint64_t)(mp_arg.t_read_ns + mp_arg.t_prog_ns) * 1000000ull + (uint64_t)q_ppm - 1ull, div_q);
     const uint64_t tile_begin = (uint64_t)tile * tile_records, tile_end = min(n, tile_begin + tile_records);
     long long dstall = 0, max_c = INT64_MIN;
+    unsigned ignored = 0;                                    // (the serve pass has already vetted every service time)
     __syncthreads();
     const uint32_t stragglers = s_stragglers;
     if (tid == 0) s_open = (int)stragglers;
@@ -684,7 +703,7 @@ k_inorder_straggle(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t ti
                     k = q != 0xffffffffu && open[q] != 0;
                 } else {
                     const uint64_t *rec = reinterpret_cast<const uint64_t *>(acc + i);
-                    const Served v = serve_terms(rs, mp, addr[j], (int64_t)__ldg(rec + 1), __ldg(rec + 2), q_ppm, div_q);
+                    const Served v = serve_terms(rs, mp, addr[j], (int64_t)__ldg(rec + 1), __ldg(rec + 2), q_ppm, div_q, ignored, 33);
                     k = v.st == HBF_ST_READY && open[v.queue] != 0;
                 }
             }
@@ -715,7 +734,7 @@ k_inorder_straggle(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t ti
                 const int64_t issue = (int64_t)__ldg(rec + 1);
                 const uint64_t bf = __ldg(rec + 2);
                 Served v = fast_terms ? serve_terms_fast(fast_range, mp, addr[j], issue, bf)
-                                      : serve_terms(rs, mp, addr[j], issue, bf, q_ppm, div_q);
+                                      : serve_terms(rs, mp, addr[j], issue, bf, q_ppm, div_q, ignored, 33);
                 if (DEBT && cbase + e < claim_limit) v.s += quantum_ns;
                 const uint32_t pos = s_cells[j * kInStrWarps + warp] + rk[j];
                 ent_as[pos] = make_longlong2(issue, v.s);

@@ -276,16 +276,25 @@ def test_inorder_other_geometries(hbf, geo):
 
 
 def test_inorder_long_accesses(hbf):
-    """Accesses with a service time beyond 32 bits of ns and a transfer of milliseconds, among ordinary ones."""
+    """Accesses with a service time beyond 32 bits of ns and a transfer of milliseconds, among ordinary ones; a service
+    of 2^33 ns or more (a 512 MiB program: 12.3 s) sends the batch to the sort path, and is refused when the caller
+    has declared the in-order path."""
     w = wl.tiny_uniform(20_000, seed=4)
-    for nbytes, flags in ((32 << 20, 0), (256 << 20, 1)):
+    for nbytes, flags in ((32 << 20, 0), (256 << 20, 1), (512 << 20, 1)):
         acc = w.acc.copy()
         acc["bytes"][7777] = nbytes
         acc["flags"][7777] = flags
         acc["addr"][7777] = wl.RANGE_BASE                   # the whole span stays inside the 1 GiB range
         for path in (hbf.PATH_AUTO, hbf.PATH_INORDER, hbf.PATH_SORT):
             g, o = contexts(hbf, w.profile, w.ranges, path)
+            if path == hbf.PATH_INORDER and nbytes == 512 << 20:
+                rc, *_ = g.submit_host(acc, check=False)
+                assert rc == hbf.E_INVAL and not g.get_busy_until().any()
+                continue
             compare_batch(g, o, acc)
+    g, o = contexts(hbf, w.profile, w.ranges, hbf.PATH_AUTO)
+    g.force_mode(hbf.MODE_LIGHT, 3); o.force_mode(hbfo.MODE_LIGHT, 3)      # service scaled 333,334 times: 6.7 s per page read
+    compare_batch(g, o, w.acc[:3000])
 
 
 @pytest.mark.parametrize("rho", [0.8, 0.95, 1.2])
