@@ -1001,7 +1001,7 @@ cudaError_t launch_submit(const SubmitArgs &a, cudaStream_t st) {
     const bool try_inorder = a.inorder_ok && (a.path == HBF_PATH_AUTO || a.path == HBF_PATH_INORDER);
     const bool sort_kernels = a.path != HBF_PATH_INORDER || !a.inorder_ok;
     mark(0);
-    k_begin<<<1, 256, 0, st>>>(a.ctrl, a.state, a.busy, a.busy_stage, a.stats_stage, a.ws.hist, a.mp.n_queues, a.mp.n_dies,
+    k_begin<<<1, 1024, 0, st>>>(a.ctrl, a.state, a.busy, a.busy_stage, a.stats_stage, a.ws.hist, a.mp.n_queues, a.mp.n_dies,
                                0, try_inorder ? 0 : 1, a.die_claims);
     g_kernel_launches += 1;
     if (n > 0) {
@@ -1011,7 +1011,7 @@ cudaError_t launch_submit(const SubmitArgs &a, cudaStream_t st) {
             if (e != cudaSuccess) return e;
             mark(8);
             if (sort_kernels) {
-                k_begin<<<1, 256, 0, st>>>(a.ctrl, a.state, a.busy, a.busy_stage, a.stats_stage, a.ws.hist, a.mp.n_queues,
+                k_begin<<<1, 1024, 0, st>>>(a.ctrl, a.state, a.busy, a.busy_stage, a.stats_stage, a.ws.hist, a.mp.n_queues,
                                            a.mp.n_dies, 1, 1, a.die_claims);
                 g_kernel_launches += 1;
             }
