@@ -223,7 +223,7 @@ int hbfo_clear_ranges(hbfo_ctx *c) { if (!c) return HBFO_E_INVAL; c->n_ranges = 
  * if the whole byte span lies in that one range and the operation is permitted; otherwise it fails. */
 int hbfo_classify(hbfo_ctx *c, const hbfo_access_t *a, int32_t *range_id) {
     if (range_id) *range_id = -1;
-    if (a->bytes == 0 || (a->flags & ~1u) || a->issue_ns < 0 || a->issue_ns >= HBFO_ISSUE_LIMIT)
+    if (a->bytes == 0 || (a->flags & ~1u) || a->issue_ns < 0)              /* any issue time >= 0 is in the domain */
         return HBFO_ST_UNSUPPORTED;
     for (uint32_t g = 0; g < c->n_ranges; ++g) {                         /* linear scan, on purpose */
         const range_t *r = &c->ranges[g];

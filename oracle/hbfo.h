@@ -45,7 +45,6 @@ enum { HBFO_ST_NATIVE = 0, HBFO_ST_READY = 1, HBFO_ST_FAULT_PARTIAL = 2, HBFO_ST
 enum { HBFO_MODE_NORMAL = 0, HBFO_MODE_LIGHT = 1, HBFO_MODE_SEVERE = 2, HBFO_MODE_SHUTDOWN = 3 };
 enum { HBFO_KIND_NONE = 0, HBFO_KIND_GPU = 1, HBFO_KIND_HBM = 2, HBFO_KIND_HBF = 3 };
 #define HBFO_MAX_RANGES 64
-#define HBFO_ISSUE_LIMIT (((int64_t)1) << 47)   /* issue_ns must lie in [0, 2^47) */
 
 typedef struct { uint64_t addr; int64_t issue_ns; uint32_t bytes; uint32_t flags; } hbfo_access_t;
 typedef struct { int64_t busy_ns, bytes_read, bytes_prog, energy_pj, n_read, n_prog; } hbfo_die_stats_t;

@@ -55,6 +55,22 @@ def test_hand_examples(golden_dir):
             assert int(o.pending_energy().sum()) == ex["energy_pj"]
 
 
+def test_hand_examples_hold_at_any_time_origin(golden_dir):
+    """The model knows no clock origin: the hand-worked examples moved to start far beyond 2^47 ns (no issue time is
+    too late for the definition) give the same completions moved by the same amount, and the same stalls."""
+    for shift in (1 << 47, (1 << 60) + 12345):
+        for ex in _examples(golden_dir):
+            o = make(stripe_bytes=ex["stripe_bytes"])
+            o.force_mode(hbfo.MODE_NORMAL if ex["q_ppm"] == 1000000 else hbfo.MODE_LIGHT, ex["q_ppm"])
+            acc = recs(ex["acc"])
+            acc["issue_ns"] += shift
+            _, comp, stall, status, ds = o.submit(acc)
+            assert (status == hbfo.ST_READY).all()
+            assert comp.tolist() == [c + shift for c in ex["completion"]], ex["name"]
+            assert stall.tolist() == ex["stall"], ex["name"]
+            assert int(ds["busy_ns"].sum()) == ex["busy_ns"] and int(o.busy_until()[0]) == ex["busy_until"] + shift
+
+
 def test_thermal_service_scaling_eq3(golden_dir):
     with open(os.path.join(golden_dir, "paper_values.json")) as f:
         cases = json.load(f)["thermal_service_scaling"]["cases"]
@@ -141,8 +157,8 @@ def test_classification_truth_table():
     assert o.classify(BASE, 0)[0] == S.ST_UNSUPPORTED
     assert o.classify(BASE, 64, flags=2)[0] == S.ST_UNSUPPORTED
     assert o.classify(BASE, 64, issue_ns=-1)[0] == S.ST_UNSUPPORTED
-    assert o.classify(BASE, 64, issue_ns=(1 << 47))[0] == S.ST_UNSUPPORTED
-    assert o.classify(BASE, 64, issue_ns=(1 << 47) - 1)[0] == S.ST_READY
+    assert o.classify(BASE, 64, issue_ns=(1 << 47))[0] == S.ST_READY          # the definition has no upper bound
+    assert o.classify(BASE, 64, issue_ns=(1 << 62))[0] == S.ST_READY
     # a range that ends at the top of the address space: a span that would wrap is a partial fault
     top = (1 << 64) - L
     o2 = make(ranges=[(top - L, L, 3, 0, 0, 0)])
