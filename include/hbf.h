@@ -10,7 +10,9 @@
  * origins, Design D3); energies are int64 pJ; temperatures are float degrees C.
  *
  * Return values: 0 = HBF_OK, negative = error.  Nothing is downgraded silently (Implementation,
- * "Every failure ends the run").  Calls on one context must come from one thread at a time.
+ * "Every failure ends the run").  Calls on one context must come from one thread at a time.  A context
+ * belongs to the CUDA device that was current at hbf_create: hbf_submit_batch, hbf_submit_batch_paged and
+ * hbf_thermal_step return HBF_E_INVAL when another device is current.
  */
 #ifndef HBF_H
 #define HBF_H
@@ -47,7 +49,7 @@ enum { HBF_ST_NATIVE = 0,        /* address outside every range: native HBM path
        HBF_ST_READY = 1,         /* whole span inside one range and permitted: modeled */
        HBF_ST_FAULT_PARTIAL = 2, /* starts inside a range but leaves it (or wraps) */
        HBF_ST_FAULT_PERM = 3,    /* operation not permitted by the range */
-       HBF_ST_UNSUPPORTED = 4 }; /* bytes == 0, unknown flag bits, issue_ns outside [0, 2^47) */
+       HBF_ST_UNSUPPORTED = 4 }; /* bytes == 0, unknown flag bits, issue_ns < 0; also issue_ns >= HBF_ISSUE_LIMIT (see there) */
 
 enum { HBF_MODE_NORMAL = 0, HBF_MODE_LIGHT = 1, HBF_MODE_SEVERE = 2, HBF_MODE_SHUTDOWN = 3 };
 enum { HBF_KIND_NONE = 0, HBF_KIND_GPU = 1, HBF_KIND_HBM = 2, HBF_KIND_HBF = 3 };     /* region kinds */
@@ -57,7 +59,11 @@ enum { HBF_PATH_AUTO = 0, HBF_PATH_SORT = 1, HBF_PATH_INORDER = 2, HBF_PATH_SORT
 
 #define HBF_MAX_RANGES 64
 #define HBF_MAX_BATCH ((uint64_t)((1u << 30) - 1))      /* accesses per batch */
-#define HBF_ISSUE_LIMIT (((int64_t)1) << 47)            /* issue_ns in [0, 2^47): 39 h, above the paper's longest run (86,400 s) */
+/* A restriction of this library, not of the model: the sort path packs (queue, issue_ns) into one 64-bit key with 47 bits
+ * for the issue time, so an access with issue_ns >= 2^47 (39 h on the caller's clock; the paper's longest run is 86,400 s)
+ * is marked HBF_ST_UNSUPPORTED and its batch is refused with HBF_E_ACCESS_FAULT, nothing changed.  The model itself has
+ * no such bound; a caller with later times moves its clock origin. */
+#define HBF_ISSUE_LIMIT (((int64_t)1) << 47)
 
 /* One access record, 24 bytes.  flags bit 0: 0 = read, 1 = program; all other bits must be 0. */
 typedef struct { uint64_t addr; int64_t issue_ns; uint32_t bytes; uint32_t flags; } hbf_access_t;
@@ -153,16 +159,16 @@ HBF_API int hbf_submit_batch_paged(hbf_ctx *ctx, const hbf_access_t *d_acc, uint
  * transfer does.  Programs are unchanged (their transfer stays a latency before the array time), and so are the
  * queue state and the per-die statistics.  The stage runs inside hbf_submit_batch after the array stage (a radix
  * sort of the reads by channel and array-done time, then a segmented max-plus scan); hbf_workspace_bytes grows by
- * 4 bytes per access once it is on.  An array-done time of 2^47 ns or more cannot be ordered: the batch's result
- * becomes HBF_E_INVAL after its array stage has been committed and the context is poisoned.
+ * 4 bytes per access once it is on.  Array-done times are sort keys of 47 bits here (a restriction of this library, like
+ * HBF_ISSUE_LIMIT): a batch whose largest completion time would reach 2^47 ns is refused with HBF_E_INVAL before anything
+ * is committed (outputs zeroed, queue, bus and energy state unchanged); the context stays usable.
  * hbf_get_bus_busy_until synchronises and copies the per-channel bus state to host_out [channels]; hbf_reset clears
  * it.  The state blob of hbf_get_state does not carry it.  hbf_submit_batch_paged is refused while the stage is on. */
 HBF_API int hbf_enable_channel_bus(hbf_ctx *ctx);
 HBF_API int hbf_get_bus_busy_until(hbf_ctx *ctx, int64_t *host_out, uint64_t cap);
 
-/* Time-bin power integration (Section "Design", the event-based energy model: event energies accumulate in
- * bins; an event that spans more than one bin has its energy split across the bins in proportion to the time
- * overlap; P = E / dt + P_idle).  After hbf_enable_energy_bins, hbf_submit_batch books the energy of every
+/* Time-bin power integration (Section "Design", the event-based energy model: a ledger of energy per time bin; a
+ * long event is shared among the bins it touches by the time spent in each; P = E / dt + P_idle).  After hbf_enable_energy_bins, hbf_submit_batch books the energy of every
  * modeled access into the bins its array service interval [start, start + s) overlaps, instead of adding the
  * batch's energy to the pending totals: whole pJ, floor(E * overlap / s) per bin, the event's last bin takes
  * what is left.  The ledger is a ring of n_bins bins of bin_ns each, starting at the bin the thermal clock
@@ -291,14 +297,13 @@ HBF_API int hbf_attach_rom(hbf_ctx *ctx, hbf_rom *rom, const int32_t *output_kin
 HBF_API int hbf_get_rom_temps(hbf_ctx *ctx, double *host_out, uint64_t cap);
 
 /* Retention, refresh and wear (Design D4: "Retention, Refresh, and Wear as Injected Latency").
- * What the paper fixes: every registered block carries retention damage, a read-disturb count, a zone and a
- * current and maximum program/erase count; the retention lifetime is L(T) = L_ref * exp[(E_a/k_B)(1/T - 1/T_ref)]
- * (first equation of D4; E_a = 1.04 eV in the evaluation); damage accumulates as D <- D + a_t * dt / L(T) (second
- * equation of D4); a block becomes eligible at its lead threshold or its read-disturb limit; refresh is emitted as
- * page-aligned read-rewrite pairs in the order eligibility epoch, channel round robin, die round robin, zone,
- * block, page; the plan is a debt of which every admission claims at most one quantum, reserving that quantum's
- * thermally scaled service before its own; a block commits one program/erase cycle and clears its damage and
- * disturb counters only when all its quanta are done; idle time drains debt on a separate account.
+ * From the paper: per-block state (retention damage, read-disturb counter, zone, program/erase cycles used and
+ * allowed); lifetime L(T) = L_ref * exp[(E_a/k_B)(1/T - 1/T_ref)] (first equation of D4; E_a = 1.04 eV in the
+ * evaluation); damage update D <- D + a_t * dt / L(T) (second equation of D4); eligibility at the lead threshold or
+ * at the disturb limit; refresh work of one read + one rewrite per page, sorted by (eligibility epoch; channels in
+ * rotation; dies in rotation; zone; block; page); the work is a debt, an admitted access takes over no more than
+ * one quantum, whose Eq.-3-scaled service is reserved ahead of its own; a block's cycle count rises and its
+ * counters clear once its last quantum is served; debt drained by idle time is accounted separately.
  * What is this library's definition (the paper gives no layout or numbers for it): a block is pages_per_block
  * consecutive pages of one plane, block = (page / pages_per_block) mod blocks_per_plane, id = ((channel * dies +
  * die) * planes + plane) * blocks_per_plane + block, zone = block / blocks_per_zone; a quantum is one page (id =

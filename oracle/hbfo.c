@@ -282,8 +282,8 @@ int hbfo_service_terms(hbfo_ctx *c, uint32_t bytes, uint64_t npages, uint32_t op
 }
 
 /* ---- time-bin power integration (Section "Design", the paragraph on the event-based energy model) -------
- * Event energies accumulate in bins of bin_ns; an event that spans more than one bin has its energy split
- * across the bins in proportion to the time overlap.  The event of an access is its array service interval
+ * The ledger holds energy per (bin of bin_ns, die); an event longer than one bin gives each bin it touches the
+ * fraction of its energy that matches the time it spent there.  The event of an access is its array service interval
  * [start, start + s) on its die.  Shares are whole pJ: floor(E * overlap / s) for every bin but the event's
  * last, which takes what is left, so a die's bins always add up to its events' energy.  The ledger is a ring
  * of n_bins bins starting at the bin the thermal clock stands in: time before it counts into that bin, time
@@ -355,15 +355,15 @@ static int cmp_bent(const void *pa, const void *pb) {
 }
 
 /* ---- retention, refresh and wear (Design D4) --------------------------------------------------------
- * What the paper fixes: every registered block carries retention damage, a read-disturb count, a zone, and a
- * current and a maximum program/erase count; the retention lifetime follows the Arrhenius equation anchored at a
- * reference condition, L(T) = L_ref * exp[(E_a / k_B) * (1/T - 1/T_ref)] (first equation of D4, E_a = 1.04 eV in
- * the evaluation); damage accumulates as D <- D + a_t * dt / L(T) (second equation of D4); a block becomes
- * eligible at its lead threshold or its read-disturb limit; the scheduler emits page-aligned read-rewrite pairs in
- * the order eligibility epoch, channel round robin, die round robin, zone, block, page; the plan is published as a
- * debt of which every admission claims at most one quantum and reserves that quantum's thermally scaled service
- * before its own; a block commits one program/erase cycle and clears its damage and disturb counters only after
- * all of its quanta are done; idle time drains debt on a separate account.
+ * From the paper (Design D4): per-block state = accumulated retention damage, read-disturb counter, zone,
+ * program/erase cycles used and allowed.  Lifetime at temperature T (first equation of D4, Arrhenius form around a
+ * reference point; E_a = 1.04 eV in the evaluation): L(T) = L_ref * exp[(E_a / k_B) * (1/T - 1/T_ref)].  Damage
+ * update over dt (second equation of D4): D <- D + a_t * dt / L(T).  Eligibility: damage at the lead threshold, or
+ * disturb count at its limit.  Refresh work = one read + one rewrite per page, issued sorted by (epoch in which the
+ * block became eligible; channels in rotation; dies of a channel in rotation; zone; block; page).  That work is a
+ * debt: an admitted access takes over no more than one quantum and has the quantum's service (with Eq. 3 scaling)
+ * reserved ahead of its own.  A block's cycle count goes up, and its damage and disturb counters go back to zero,
+ * once its last quantum has been served; debt drained by idle time is accounted separately from claimed debt.
  * What is a reading (the paper gives no numbers or layouts for these): a block is pages_per_block consecutive
  * pages of one plane, block = (page / pages_per_block) mod blocks_per_plane, zone = block / blocks_per_zone; a
  * read adds its page count to the disturb counter of the block of its first page, programs add nothing; damage

@@ -84,8 +84,8 @@ int  hbfo_submit_batch(hbfo_ctx *ctx, const hbfo_access_t *acc, uint64_t n, int6
  * its own decode; the access completes with its last part.  Same arguments as hbfo_submit_batch. */
 int  hbfo_submit_batch_paged(hbfo_ctx *ctx, const hbfo_access_t *acc, uint64_t n, int64_t *completion_ns,
                              int64_t *stall_ns, uint8_t *status, hbfo_die_stats_t *die_stats);
-/* Time-bin power integration (Section "Design": event energies accumulate in bins; an event spanning several
- * bins is split in proportion to the time overlap).  After this call hbfo_submit_batch books every access's
+/* Time-bin power integration (Section "Design", event-based energy model: a ledger of energy per time bin, a long
+ * event shared among its bins by time spent in each).  After this call hbfo_submit_batch books every access's
  * energy into the bins its array service interval overlaps instead of the pending total, and
  * hbfo_thermal_step(dt_ns == bin_ns) consumes the bin the thermal clock stands in.  hbfo_get_energy_bins
  * copies the ring out, row k = bin first_bin + k.  hbfo_reset clears the ring and the clock. */

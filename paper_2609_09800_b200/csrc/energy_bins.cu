@@ -1,6 +1,6 @@
-// Time-bin power integration (Section "Design", the event-based energy model): event energies accumulate in
-// bins; an event that spans more than one bin has its energy split across the bins in proportion to the time
-// overlap.  The event of an access is its array service interval [start, start + s) on its die; shares are
+// Time-bin power integration (Section "Design", event-based energy model).  The ledger keeps energy per (bin, die);
+// an event longer than one bin contributes to each bin it touches by the fraction of its duration spent there.
+// Here the event of an access is its array service interval [start, start + s) on its die; shares are
 // whole pJ, floor(E * overlap / s), and the event's last bin takes what is left.  The ledger is a ring of bins
 // that starts at the bin the thermal clock stands in; time before it is booked into that bin, time past the
 // ring's end into the ring's last bin.  Integer adds in any order: the result does not depend on scheduling.
@@ -17,19 +17,32 @@ __device__ __forceinline__ void ledger_add(unsigned long long *ledger, uint32_t 
     if (pj) atomicAdd(&ledger[(size_t)(bin % (int64_t)n_bins) * n_dies + die], (unsigned long long)pj);
 }
 
-// one event: energy pj over [start, start + s), split over the bins it overlaps
+// one event: energy pj over [start, start + s), split over the bins it overlaps.  Every bin before the event's last one
+// gets floor(pj * overlap / s); the overlap is a whole bin for all of them but the first, so the bins that the ring clamps
+// into its first or last slot are booked in one step each and the loop only walks bins inside the ring: at most n_bins
+// turns, whatever the ratio of service time to bin width.
 __device__ __forceinline__ void ledger_event(unsigned long long *ledger, uint32_t n_dies, uint32_t n_bins, int64_t cur_bin, int64_t bin_ns,
                                              uint32_t die, int64_t start, int64_t s, int64_t pj) {
     const int64_t end = start + s;
     const int64_t b0 = start / bin_ns, b1 = (end - 1) / bin_ns;
     if (b0 == b1) { ledger_add(ledger, n_dies, n_bins, cur_bin, die, b0, pj); return; }
+    const int64_t ring_hi = cur_bin + (int64_t)n_bins - 1;
+    const int64_t first = (int64_t)(((unsigned __int128)(uint64_t)pj * (uint64_t)((b0 + 1) * bin_ns - start)) / (uint64_t)s);
+    const int64_t full = (int64_t)(((unsigned __int128)(uint64_t)pj * (uint64_t)bin_ns) / (uint64_t)s);
+    auto run = [&](int64_t from, int64_t to) {               // shares of the bins [from, to), from >= b0, to <= b1
+        return to <= from ? (int64_t)0 : (from == b0 ? first + (to - from - 1) * full : (to - from) * full);
+    };
+    const int64_t below_end = min(b1, max(b0, cur_bin));     // bins [b0, below_end) lie before the ring
+    const int64_t above_begin = min(b1, max(below_end, ring_hi));   // bins [above_begin, b1) lie at or past its last slot
     int64_t given = 0;
-    for (int64_t b = b0; b < b1; ++b) {
-        const int64_t lo = max(b * bin_ns, start), hi = (b + 1) * bin_ns;
-        const int64_t share = (int64_t)(((unsigned __int128)(uint64_t)pj * (uint64_t)(hi - lo)) / (uint64_t)s);
-        ledger_add(ledger, n_dies, n_bins, cur_bin, die, b, share);
-        given += share;
+    const int64_t below = run(b0, below_end);
+    ledger_add(ledger, n_dies, n_bins, cur_bin, die, cur_bin, below); given += below;
+    for (int64_t b = below_end; b < above_begin; ++b) {
+        const int64_t share = b == b0 ? first : full;
+        ledger_add(ledger, n_dies, n_bins, cur_bin, die, b, share); given += share;
     }
+    const int64_t above = run(above_begin, b1);
+    ledger_add(ledger, n_dies, n_bins, cur_bin, die, ring_hi, above); given += above;
     ledger_add(ledger, n_dies, n_bins, cur_bin, die, b1, pj - given);
 }
 

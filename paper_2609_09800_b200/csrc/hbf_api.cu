@@ -65,6 +65,9 @@ static Div64 make_div64_host(uint64_t d) {       // same construction as the dev
     return r;
 }
 
+// the context's device state, kernels' attributes and stream belong to the device it was created on
+static bool on_own_device(const hbf_ctx *c) { int d = -1; return cudaGetDevice(&d) == cudaSuccess && d == c->device; }
+
 static bool is_pow2(uint64_t v) { return v && !(v & (v - 1)); }
 static uint32_t log2u(uint64_t v) { uint32_t s = 0; while ((1ull << s) < v) ++s; return s; }
 
@@ -408,7 +411,7 @@ int hbf_set_path(hbf_ctx *c, int32_t path) {
 int hbf_submit_batch(hbf_ctx *c, const hbf_access_t *d_acc, uint64_t n, int64_t *d_completion_ns,
                      int64_t *d_stall_ns, uint8_t *d_status, hbf_die_stats_t *d_die_stats,
                      void *d_workspace, size_t workspace_bytes) {
-    if (!c) return HBF_E_INVAL;
+    if (!c || !on_own_device(c)) return HBF_E_INVAL;
     if (c->terminal) return HBF_E_LINK_SHUTDOWN;
     if (n > HBF_MAX_BATCH) return HBF_E_INVAL;
     if (n && (!d_acc || !d_completion_ns || !d_stall_ns)) return HBF_E_INVAL;
@@ -428,7 +431,7 @@ int hbf_submit_batch(hbf_ctx *c, const hbf_access_t *d_acc, uint64_t n, int64_t 
     c->prof_inorder = c->profiling && n > 0 && c->inorder_ok && (c->path == HBF_PATH_AUTO || c->path == HBF_PATH_INORDER);
     a.ev = c->profiling ? c->ev : nullptr;
     c->prof_submit = c->profiling;
-    a.binned = c->bin_ns != 0;
+    a.binned = c->bin_ns != 0; a.bus_on = c->d_bus_busy ? 1 : 0;
     if (c->ret_on) {                                         // how far the outstanding refresh quanta reach into this batch
         CK(launch_ret_window(d_acc, n, c->d_ranges, c->ret, c->sm_count, c->stream));
         a.claim_limit = &c->ret.st->claim_limit; a.die_claims = c->ret.die_claims; a.ret = &c->ret;
@@ -459,6 +462,7 @@ int hbf_submit_batch_paged(hbf_ctx *c, const hbf_access_t *d_acc, uint64_t n, ui
     if (!c) return HBF_E_INVAL;
     if (n == 0)                                             // nothing to split: the ordinary path reports the empty batch
         return hbf_submit_batch(c, d_acc, 0, d_completion_ns, d_stall_ns, d_status, d_die_stats, d_workspace, workspace_bytes);
+    if (!on_own_device(c)) return HBF_E_INVAL;
     if (c->terminal) return HBF_E_LINK_SHUTDOWN;
     if (n > HBF_MAX_BATCH || c->bin_ns != 0 || c->d_bus_busy || c->ret_on) return HBF_E_INVAL;   // ledger, bus stage and retention take whole accesses only
     if (!d_acc || !d_completion_ns || !d_stall_ns) return HBF_E_INVAL;
@@ -662,20 +666,21 @@ int hbf_queue_order(hbf_ctx *c, const void *d_workspace, uint64_t n, uint32_t *d
 }
 
 int hbf_thermal_step(hbf_ctx *c, int64_t dt_ns, const float *ext_power_w, uint32_t n_ext, float *d_temps_out, float *hot_c_out) {
-    if (!c || !c->thermal || dt_ns <= 0) return HBF_E_INVAL;
+    if (!c || !c->thermal || dt_ns <= 0 || !on_own_device(c)) return HBF_E_INVAL;
     if (n_ext != 0 && (n_ext != c->td.n_regions || !ext_power_w)) return HBF_E_INVAL;
     const double dt_sub = (double)dt_ns * 1e-9 / (double)c->td.n_sub;
+    // every refusal comes before the first enqueue: a refused call leaves the ledger, the clock and the stream as they were
     if (!c->rom && dt_sub > c->euler_limit_s) return HBF_E_INVAL;
+    if (c->bin_ns && dt_ns != c->bin_ns) return HBF_E_INVAL;
+    if (c->rom && (dt_ns != c->rom_dt_ns || d_temps_out)) return HBF_E_INVAL;
     if (n_ext)      // pageable source: the runtime stages the bytes before returning, so the caller's array is free at once
         CK(cudaMemcpyAsync(c->td.ext_power, ext_power_w, n_ext * sizeof(float), cudaMemcpyHostToDevice, c->stream));
     if (c->bin_ns) {                                         // the step is the bin the thermal clock stands in
-        if (dt_ns != c->bin_ns) return HBF_E_INVAL;
         CK(launch_take_bin(c->d_ledger + (size_t)(c->cur_bin % c->n_bins) * c->mp.n_dies, c->d_pending, c->mp.n_dies, c->stream));
         c->cur_bin += 1;
     }
     if (c->profiling) CK(cudaEventRecord(c->ev_th[0], c->stream));
     if (c->rom) {                                            // the attached model stands in for the grid
-        if (dt_ns != c->rom_dt_ns || d_temps_out) return HBF_E_INVAL;
         CK(launch_rom_power(c->td, c->d_pending, dt_ns, n_ext != 0, c->d_rom_p, c->stream));
         { const int rc_ = hbf_rom_step(c->rom, c->d_rom_p, 1, c->d_rom_T); if (rc_ != HBF_OK) return rc_; }
         CK(launch_rom_controller(c->td, c->d_rom_T, c->d_rom_kind, hbf_rom_outputs(c->rom), c->d_state, c->stream));
@@ -789,7 +794,7 @@ int hbf_get_profile(hbf_ctx *c, float *ms_out, uint32_t cap) {
     return HBF_OK;
 }
 
-uint64_t hbf_kernel_launches(void) { return g_kernel_launches; }
+uint64_t hbf_kernel_launches(void) { return g_kernel_launches.load(); }
 
 double hbf_euler_limit_ns(const hbf_ctx *c) { return c && c->thermal ? c->euler_limit_s * 1e9 : 0.0; }
 

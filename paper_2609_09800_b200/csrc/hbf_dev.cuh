@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "../../include/hbf.h"
 
 namespace hbf {
@@ -106,13 +108,17 @@ struct SubmitArgs {
     Workspace ws; int32_t path; int sm_count; int inorder_ok;
     FastRange fast;
     int binned;                          // the batch's energy goes to the time-bin ledger, not to the pending totals
+    int bus_on;                          // the channel-bus stage follows: array-done times must fit its 47-bit key field
     const unsigned long long *claim_limit;  // retention on: batch index below which a modeled access claims a refresh quantum
     uint32_t *die_claims;                   // retention on: [dies] claims of the batch
     const struct RetDev *ret;               // retention on: the block state (host copy of the device pointers)
     cudaEvent_t *ev;                     // [kProfEvents] or null: recorded between kernel groups
 };
 constexpr int kProfEvents = 10;
-extern unsigned long long g_kernel_launches;
+extern std::atomic<unsigned long long> g_kernel_launches;
+// The dynamic shared memory a kernel may use is an attribute of the (device, kernel) pair: raises it on the current device
+// when `bytes` exceeds what this process has set there so far.  Thread-safe.
+cudaError_t ensure_dyn_smem(const void *kernel, size_t bytes);
 
 constexpr uint32_t kInMaxQueues = 2048;  // the in-order path keeps per-queue state in shared memory
 constexpr uint32_t kInMaxTiles = 1024;

@@ -813,19 +813,14 @@ cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st) {
     if (n_tiles > inorder_tiles_bound(n)) return cudaErrorInvalidValue;       // the workspace is carved for that many
     const uint32_t R = a.mp.n_queues, nd = a.mp.n_dies;
     const size_t smem_serve = inorder_serve_smem(nd), smem_str = inorder_straggle_smem();
-    static size_t set_serve = 0;
-    if (smem_serve > set_serve) {
+    {
         const void *serve_fns[4] = {(const void *)k_inorder_serve<false, false>, (const void *)k_inorder_serve<true, false>,
                                     (const void *)k_inorder_serve<false, true>, (const void *)k_inorder_serve<true, true>};
-        for (const void *f : serve_fns) {
-            cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_serve);
-            if (e != cudaSuccess) return e;
-        }
-        cudaError_t e = cudaFuncSetAttribute(k_inorder_straggle<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_str);
+        for (const void *f : serve_fns) { cudaError_t e = ensure_dyn_smem(f, smem_serve); if (e != cudaSuccess) return e; }
+        cudaError_t e = ensure_dyn_smem((const void *)k_inorder_straggle<false>, smem_str);
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(k_inorder_straggle<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_str);
+        e = ensure_dyn_smem((const void *)k_inorder_straggle<true>, smem_str);
         if (e != cudaSuccess) return e;
-        set_serve = smem_serve;
     }
     InTile *tiles = reinterpret_cast<InTile *>(a.ws.in_tile);
     InHead *heads = reinterpret_cast<InHead *>(a.ws.in_head);

@@ -165,12 +165,7 @@ cudaError_t launch_rom_steps(uint32_t n, uint32_t m, uint32_t o, const double *A
     uint32_t rpc = 0;
     const size_t csmem = rom_cluster_smem(n, m, o, &rpc);
     if (csmem <= 200u * 1024u) {                             // the rows fit the shared memory of eight blocks
-        static size_t set_smem = 0;
-        if (csmem > set_smem) {
-            cudaError_t e = cudaFuncSetAttribute(k_rom_steps_cluster, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)csmem);
-            if (e != cudaSuccess) return e;
-            set_smem = csmem;
-        }
+        { cudaError_t e = ensure_dyn_smem((const void *)k_rom_steps_cluster, csmem); if (e != cudaSuccess) return e; }
         k_rom_steps_cluster<<<kRomClusterBlocks, kRomClusterThreads, csmem, st>>>(n, m, o, rpc, A, B, b, C, D, d, x, power, n_steps, temps_out);
         g_kernel_launches += 1;
         return cudaGetLastError();

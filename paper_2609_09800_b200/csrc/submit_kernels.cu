@@ -5,6 +5,8 @@
 // Every kernel reads the batch control block first and does nothing once the batch is refused, so the
 // whole sequence can be enqueued without a host round trip.
 #include <algorithm>
+#include <mutex>
+#include <vector>
 
 #include "device_utils.cuh"
 
@@ -613,8 +615,12 @@ k_scan(const hbf_access_t *__restrict__ acc, uint64_t n, const RangeSnap *__rest
 __global__ void k_finish(uint64_t n, BatchCtrl *ctrl, DevState *state, int64_t *busy, const int64_t *busy_stage,
                          int64_t *pending, const hbf_die_stats_t *stats_stage, hbf_die_stats_t *die_stats,
                          int64_t *completion, int64_t *stall, hbf_batch_result_t *result,
-                         const ModelParams *__restrict__ mp, uint32_t n_queues, uint32_t n_dies, int binned) {
-    const int code = ctrl->code;
+                         const ModelParams *__restrict__ mp, uint32_t n_queues, uint32_t n_dies, int binned, int bus_on) {
+    int code = ctrl->code;
+    // With the channel-bus stage on, array-done times become sort keys of 47 bits: a batch that reaches 2^47 ns is refused
+    // here, before anything is committed (every array-done time is at most the largest completion).  Every thread reads
+    // the same settled values, so every thread takes the same decision.
+    if (bus_on && code == HBF_OK && ctrl->n_ready && ctrl->max_completion_ns >= HBF_ISSUE_LIMIT) code = HBF_E_INVAL;
     const uint64_t gtid = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (code == HBF_E_TIMEOUT && gtid == 0) state->poisoned = 1;         // a bounded device-side wait expired
     const uint64_t gsz = (uint64_t)gridDim.x * blockDim.x;
@@ -900,12 +906,8 @@ cudaError_t launch_bus_stage(const SubmitArgs &a, BatchCtrl *bc, int64_t *bus_bu
     k_plan<<<1, 32, 0, st>>>(bc, 1);
     const unsigned hist_grid = (unsigned)std::min<uint64_t>((n + kHistThreads * 8 - 1) / (kHistThreads * 8), (uint64_t)a.sm_count * 4);
     k_hist<<<hist_grid, kHistThreads, 0, st>>>(a.ws.keys[0], n, bc, a.ws.hist);
-    static bool attr_set = false;
-    if (!attr_set) {
-        e = cudaFuncSetAttribute(k_sort_pass, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSortSmem);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
+    e = ensure_dyn_smem((const void *)k_sort_pass, kSortSmem);
+    if (e != cudaSuccess) return e;
     const unsigned sort_grid = (unsigned)std::min<uint64_t>(sort_tiles, (uint64_t)a.sm_count * 3);
     for (int p = 0; p < kMaxPasses; ++p)
         k_sort_pass<<<sort_grid, kSortThreads, kSortSmem, st>>>(p, n, bc, a.state, a.ws.hist, a.ws.keys[0], a.ws.keys[1],
@@ -953,7 +955,27 @@ size_t workspace_layout(uint64_t n, uint32_t n_queues, Workspace *ws, void *base
     return off;
 }
 
-unsigned long long g_kernel_launches = 0;
+std::atomic<unsigned long long> g_kernel_launches{0};
+
+cudaError_t ensure_dyn_smem(const void *kernel, size_t bytes) {
+    struct Entry { int device; const void *kernel; size_t bytes; };
+    static std::mutex mu;
+    static std::vector<Entry> set;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    std::lock_guard<std::mutex> lock(mu);
+    for (Entry &en : set)
+        if (en.device == dev && en.kernel == kernel) {
+            if (bytes <= en.bytes) return cudaSuccess;
+            e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+            if (e == cudaSuccess) en.bytes = bytes;
+            return e;
+        }
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e == cudaSuccess) set.push_back(Entry{dev, kernel, bytes});
+    return e;
+}
 
 static cudaError_t launch_sort_path(const SubmitArgs &a, cudaStream_t st) {
     const uint64_t n = a.n;
@@ -973,12 +995,8 @@ static cudaError_t launch_sort_path(const SubmitArgs &a, cudaStream_t st) {
     const unsigned hist_grid = (unsigned)std::min<uint64_t>((n + kHistThreads * 8 - 1) / (kHistThreads * 8), (uint64_t)a.sm_count * 4);
     k_hist<<<hist_grid, kHistThreads, 0, st>>>(a.ws.keys[0], n, a.ctrl, a.ws.hist);
     mark(3);
-    static bool attr_set = false;
-    if (!attr_set) {
-        e = cudaFuncSetAttribute(k_sort_pass, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSortSmem);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
+    e = ensure_dyn_smem((const void *)k_sort_pass, kSortSmem);
+    if (e != cudaSuccess) return e;
     const unsigned sort_grid = (unsigned)std::min<uint64_t>(sort_tiles, (uint64_t)a.sm_count * 3);
     for (int p = 0; p < kMaxPasses; ++p)
         k_sort_pass<<<sort_grid, kSortThreads, kSortSmem, st>>>(p, n, a.ctrl, a.state, a.ws.hist, a.ws.keys[0], a.ws.keys[1],
@@ -1026,7 +1044,7 @@ cudaError_t launch_submit(const SubmitArgs &a, cudaStream_t st) {
     mark(5);
     const unsigned fin_grid = (unsigned)std::max<uint64_t>(1, std::min<uint64_t>((n + 1023) / 1024, (uint64_t)a.sm_count * 4));
     k_finish<<<fin_grid, 256, 0, st>>>(n, a.ctrl, a.state, a.busy, a.busy_stage, a.pending, a.stats_stage, a.die_stats,
-                                       a.completion, a.stall, a.result, a.mp_dev, a.mp.n_queues, a.mp.n_dies, a.binned);
+                                       a.completion, a.stall, a.result, a.mp_dev, a.mp.n_queues, a.mp.n_dies, a.binned, a.bus_on);
     g_kernel_launches += 1;
     mark(6);
     return cudaGetLastError();

@@ -287,12 +287,7 @@ cudaError_t launch_thermal_step(const ThermalDev &t, DevState *state, int64_t *p
     const float dt_sub_f = (float)((double)dt_ns * 1e-9 / (double)t.n_sub);
     size_t smem = 0;
     if (!generic_only && thermal_cluster_fits(t, &smem)) {
-        static size_t set_smem = 0;
-        if (smem > set_smem) {
-            cudaError_t e = cudaFuncSetAttribute(k_thermal_cluster, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-            if (e != cudaSuccess) return e;
-            set_smem = smem;
-        }
+        { cudaError_t e = ensure_dyn_smem((const void *)k_thermal_cluster, smem); if (e != cudaSuccess) return e; }
         k_thermal_cluster<<<kThClusterBlocks, kThThreads, smem, st>>>(t, t.theta[*cur], state, pending, dt_ns, has_ext, dt_sub_f, d_temps_out);
         g_kernel_launches += 1;
         return cudaGetLastError();

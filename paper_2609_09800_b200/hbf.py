@@ -18,6 +18,7 @@ OK, E_INVAL, E_RANGE_OVERLAP, E_RANGE_FULL, E_CAPACITY, E_WORKSPACE, E_CUDA = 0,
 E_ACCESS_FAULT, E_THROTTLED, E_LINK_SHUTDOWN, E_TIMEOUT, E_NOMEM = -7, -8, -9, -10, -11
 ST_NATIVE, ST_READY, ST_FAULT_PARTIAL, ST_FAULT_PERM, ST_UNSUPPORTED = range(5)
 MODE_NORMAL, MODE_LIGHT, MODE_SEVERE, MODE_SHUTDOWN = range(4)
+KIND_NONE, KIND_GPU, KIND_HBM, KIND_HBF = range(4)
 PATH_AUTO, PATH_SORT, PATH_INORDER, PATH_SORT_FULL = range(4)
 
 ACCESS_DTYPE = np.dtype([("addr", "<u8"), ("issue_ns", "<i8"), ("bytes", "<u4"), ("flags", "<u4")])
@@ -404,7 +405,7 @@ class Context:
         if rc != 0:
             raise HbfError(rc, "hbf_set_thermal_path")
 
-    def thermal_step(self, dt_ns, ext_power_w=None, d_temps_out=None, want_hot=True):
+    def thermal_step(self, dt_ns, ext_power_w=None, d_temps_out=None, want_hot=True, check=True):
         hot = np.empty(3, np.float32) if want_hot else None
         if ext_power_w is None:
             p, n = None, 0
@@ -413,7 +414,9 @@ class Context:
             p, n = ext.ctypes.data, ext.shape[0]
         rc = lib().hbf_thermal_step(self._h, dt_ns, p, n, _ptr(d_temps_out), hot.ctypes.data if want_hot else None)
         if rc != 0:
-            raise HbfError(rc, "hbf_thermal_step")
+            if check:
+                raise HbfError(rc, "hbf_thermal_step")
+            return rc
         return hot
 
     def force_mode(self, mode, q_ppm):

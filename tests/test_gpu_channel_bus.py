@@ -109,3 +109,25 @@ def test_with_the_energy_ledger_on(hbf):
     compare(g, o, w.acc)
     (fg, bg), (fo, bo) = g.energy_bins(), o.energy_bins()
     assert fg == fo and np.array_equal(bg, bo)                             # the ledger's events are the array intervals, bus or not
+
+
+@pytest.mark.parametrize("path", ["auto", "sort"])
+def test_completion_past_the_key_width_is_refused_before_anything_is_committed(hbf, path):
+    """With the bus stage on, array-done times are 47-bit sort keys in this library.  A batch issued just below 2^47 ns
+    completes beyond it: the library refuses it (HBF_E_INVAL) with outputs zeroed and queue, bus and energy state
+    unchanged, and goes on serving; the oracle, which has no such bound, serves the batch."""
+    w = wl.tiny_uniform(4000, seed=11)
+    g, o = contexts(hbf, w.profile, w.ranges, hbf.PATH_AUTO if path == "auto" else hbf.PATH_SORT)
+    compare(g, o, w.acc[:2000])
+    late = w.acc[2000:].copy()
+    late["issue_ns"] += (1 << 47) - 1 - int(late["issue_ns"].max())
+    busy0, bus0, pend0 = g.get_busy_until(), g.get_bus_busy_until(), g.get_pending_energy()
+    rc_g, c_g, s_g, _, ds_g = g.submit_host(late, check=False)
+    assert rc_g == hbf.E_INVAL and not c_g.any() and not s_g.any() and not ds_g["n_read"].any()
+    assert np.array_equal(g.get_busy_until(), busy0) and np.array_equal(g.get_bus_busy_until(), bus0)
+    assert np.array_equal(g.get_pending_energy(), pend0)
+    o_late = hbfo.Oracle(w.profile); o_late.register_range(*w.ranges[0]); o_late.enable_channel_bus()
+    o_late.submit(w.acc[:2000])
+    rc_o, c_o, *_ = o_late.submit(late, check=False)
+    assert rc_o == 0 and int(c_o.max()) >= (1 << 47)
+    compare(g, o, w.acc[2000:])                              # the refusal left the context usable and its state exact

@@ -111,3 +111,54 @@ def test_thermal_steps_consume_the_bins(hbf):
         g.thermal_step(2_000_000, ext)                        # in binned mode a step is one bin long
     g.reset(); o.reset()
     same_bins(g, o)
+
+
+@pytest.mark.parametrize("path", ["auto", "sort"])
+def test_events_far_longer_than_the_ring(hbf, path):
+    """A ring of two bins and events that span about five bins each (and, after a thermal step, events that begin before
+    the ring): the bins the ring clamps into its first and last slot are booked in one step each on the device, and must
+    add up to what the oracle's bin-by-bin walk gives."""
+    prof = wl.load_profile("nominal", **wl.GEOMETRY["tiny"])
+    fp = wl.package_floorplan()
+    g, o = contexts(hbf, prof, [(wl.RANGE_BASE, wl.GIB, 3, 0, 0, 0)], fp, path=hbf.PATH_AUTO if path == "auto" else hbf.PATH_SORT)
+    bin_ns = 4_001                                            # a read of one page (20,000 ns) spans five or six bins
+    g.enable_energy_bins(bin_ns, 2); o.enable_energy_bins(bin_ns, 2)
+    rng = np.random.default_rng(5)
+    n = 3000
+    acc = np.zeros(n, hbfo.ACCESS_DTYPE)
+    acc["addr"] = wl.RANGE_BASE + rng.integers(0, 1 << 22, n).astype(np.uint64)
+    acc["issue_ns"] = np.sort(rng.integers(0, 60_000, n))
+    acc["bytes"] = rng.choice([64, 4096, 40_000], n)
+    acc["flags"] = rng.random(n) < 0.1
+    for part in (acc[:1500], acc[1500:]):
+        o.submit(part); g.submit_host(part)
+        same_bins(g, o)
+        for _ in range(3):                                    # the clock moves on: later events begin before the ring
+            g.thermal_step(bin_ns, fp["ext_power_w"]); o.thermal_step(bin_ns, fp["ext_power_w"])
+        same_bins(g, o)
+        assert np.array_equal(g.get_pending_energy(), o.pending_energy())
+
+
+def test_refused_thermal_step_changes_nothing(hbf):
+    """Bins on and a reduced-order model attached: a call the model must refuse (a field output is asked for) returns
+    HBF_E_INVAL before anything is enqueued: the ledger rows, the clock's bin and the pending energy stay as they were."""
+    w = wl.prefix_kv(epochs=1, steps=1, batch=4, kv_tokens=256, layers=2)
+    fp = wl.package_floorplan()
+    g, _ = contexts(hbf, w.profile, w.ranges, fp)
+    g.enable_energy_bins(1_000_000, 8)
+    g.submit_host(w.acc[:20_000])
+    n_regions = len(fp["region_kind"])
+    rom = hbf.Rom(np.zeros((2, 2)), np.zeros((2, n_regions)), np.zeros((3, 2)), stream=g.stream)
+    g.attach_rom(rom, [hbf.KIND_HBF, hbf.KIND_HBM, hbf.KIND_GPU], 1_000_000)
+    first0, bins0 = g.energy_bins()
+    pend0 = g.get_pending_energy()
+    assert bins0.any()
+    import torch
+    d_t = torch.zeros(fp["grid_h"] * fp["grid_w"], dtype=torch.float32, device="cuda")
+    assert g.thermal_step(1_000_000, fp["ext_power_w"], d_temps_out=d_t, check=False) == hbf.E_INVAL
+    assert g.thermal_step(2_000_000, fp["ext_power_w"], check=False) == hbf.E_INVAL
+    first1, bins1 = g.energy_bins()
+    assert first1 == first0 and np.array_equal(bins1, bins0) and np.array_equal(g.get_pending_energy(), pend0)
+    g.thermal_step(1_000_000, fp["ext_power_w"])             # an accepted step consumes the clock's bin
+    first2, bins2 = g.energy_bins()
+    assert first2 == first0 + 1 and np.array_equal(bins2[:-1], bins0[1:])

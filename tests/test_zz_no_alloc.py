@@ -4,8 +4,9 @@ Some callers of this library may not allocate device memory (a serving loop that
 device-wide stall cudaMalloc can cause; a plug-in confined to buffers its host hands it).  For them
 ``hbf_euler_substeps_static`` keeps its second field buffer in an array built into the library.  This
 test drives it twice in a row on caller-owned buffers and compares the field with what the regular,
-context-based ``hbf_thermal_step`` produces for the same floorplan and power, within the 1e-3 K
-tolerance the thermal parity tests use.  The file sorts last so that a run which stops at the first
+context-based ``hbf_thermal_step`` produces for the same floorplan and power, and with the float64 CPU
+oracle's thermal step, within the 1e-3 K tolerance the thermal parity tests use; the free device
+memory the CUDA runtime reports must not move across the call.  The file sorts last so that a run which stops at the first
 failure has already run everything else.
 """
 import numpy as np
@@ -13,6 +14,7 @@ import pytest
 
 pytestmark = pytest.mark.gpu
 
+from oracle import hbfo
 from paper_2609_09800_b200 import workloads as wl
 
 TOL_K = 1e-3
@@ -54,19 +56,28 @@ def test_static_entry_matches_thermal_step_on_two_calls_in_a_row(hbf, plan):
     theta = torch.zeros(n_cells, dtype=torch.float32, device="cuda")
     comp = torch.zeros(n_cells, dtype=torch.float32, device="cuda")
     d_T = torch.empty(n_cells, dtype=torch.float32, device="cuda")
-    allocated = torch.cuda.memory_allocated()
+    orc = hbfo.Oracle(prof, fp)                             # float64, cell by cell: the independent reference
+    # warm-up on scratch buffers of its own: module load and the look-up of the built-in array's address happen here
+    w_theta, w_comp = torch.zeros_like(theta), torch.zeros_like(comp)
+    P0 = dev(cell_power(fp, fp["ext_power_w"]))
+    assert hbf.euler_substeps_static(C_, Gx, Gy, Gs, P0, w_theta, w_comp, fp["grid_h"], fp["grid_w"], 1, float(dt_sub)) == hbf.OK
+    torch.cuda.synchronize()
     for call, scale in enumerate((1.0, 2.5)):               # two calls in a row, the second with other power
         ext = fp["ext_power_w"] * np.float32(scale)
         P = dev(cell_power(fp, ext))
-        allocated = torch.cuda.memory_allocated()
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]          # what cudaMemGetInfo reports: sees any cudaMalloc, torch's or not
         rc = hbf.euler_substeps_static(C_, Gx, Gy, Gs, P, theta, comp, fp["grid_h"], fp["grid_w"], n_sub, float(dt_sub))
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free_before
         assert rc == hbf.OK
         ctx.thermal_step(dt_ns, ext, d_T)
+        _, t_o = orc.thermal_step(dt_ns, ext, want_temps=True)
         torch.cuda.synchronize()
-        assert torch.cuda.memory_allocated() == allocated
         got = theta.cpu().numpy().astype(np.float64) + prof["ambient_c"]
         want = d_T.cpu().numpy().astype(np.float64)
         assert np.abs(got - want).max() < TOL_K, (plan, call)
+        assert np.abs(got - t_o).max() < TOL_K, (plan, call, "oracle")
         assert want.max() > prof["ambient_c"] + 1e-4        # the step did something
     # odd substep counts end in the built-in buffer and are copied back
     theta2 = torch.zeros(n_cells, dtype=torch.float32, device="cuda"); comp2 = torch.zeros_like(theta2)
