@@ -1,8 +1,12 @@
 """Parity at the benchmark's full size: the 200 M-access capacity-mode batch, device-resident, in the launch
-configuration bench.py times.  The oracle cannot serve 200 M accesses in seconds, but queues are independent:
-the sub-stream of one queue, served alone by the oracle, must give exactly the completions the library gave
-those accesses.  A handful of sampled queues are checked that way, element by element, on a fresh batch and
-on a replay (every queue backlogged); totals are checked against closed forms over the whole batch."""
+configuration bench.py times.  Queues are independent, so the oracle is run on sub-streams of whole queues: the
+2,048 queues are dealt to as many oracle instances as the host has cores, each serves its own sub-stream (plain
+sequential code, one instance per thread), and every completion, stall, per-die total, queue state and summary of the
+library is compared with them: all 200 M accesses, on a fresh batch and on a replay (every queue backlogged)."""
+import os
+import time
+from concurrent.futures import ThreadPoolExecutor
+
 import numpy as np
 import pytest
 
@@ -25,8 +29,10 @@ def full():
     build.build()
     w = wl.capacity_mode(n=N_FULL)
     u = ((w.acc["addr"] - np.uint64(wl.RANGE_BASE)) >> np.uint64(16)).astype(np.int64)   # 64 KiB stripe units
-    queue = ((u % 64) * 8 + (u // 64) % 8) * 4 + (u // 512) % 4
-    return hbf, w, queue.astype(np.int32)
+    queue = (((u % 64) * 8 + (u // 64) % 8) * 4 + (u // 512) % 4).astype(np.int32)
+    shards = shards_of(queue, host_workers())
+    assert sum(s.size for s in shards) == N_FULL
+    return hbf, w, shards, [w.acc[s] for s in shards]
 
 
 def run_gpu(hbf, ctx, w):
@@ -50,47 +56,78 @@ def run_gpu(hbf, ctx, w):
     return out
 
 
+def host_workers():
+    return max(1, min(32, len(os.sched_getaffinity(0))))
+
+
+def shards_of(queue, groups):
+    """Record indices of each group of queues (queue q belongs to group q mod groups), in batch order."""
+    grp = (queue % groups).astype(np.int8)
+    return [np.flatnonzero(grp == k) for k in range(groups)]
+
+
+def make_oracle(w, setup=None):
+    o = hbfo.Oracle(w.profile)
+    for r in w.ranges:
+        o.register_range(*r)
+    if setup:
+        setup(o)
+    return o
+
+
+def compare_shard(o, sub, idx, comp, stall):
+    """One oracle instance serves its sub-stream; returns its per-die totals, queue state and summary."""
+    _, c_o, s_o, st_o, ds_o = o.submit(sub)
+    bad = np.flatnonzero(comp[idx] != c_o)
+    assert bad.size == 0, (int(idx[bad[0]]), int(comp[idx[bad[0]]]), int(c_o[bad[0]]), int(bad.size))
+    assert np.array_equal(stall[idx], s_o) and (st_o == hbfo.ST_READY).all()
+    return ds_o, o.busy_until(), o.last_result()
+
+
+def check_against_shards(hbf, pool, oracles, subs, shards, comp, stall, ds, busy, res):
+    t0 = time.perf_counter()
+    outs = list(pool.map(lambda k: compare_shard(oracles[k], subs[k], shards[k], comp, stall), range(len(shards))))
+    dt = time.perf_counter() - t0
+    ds_sum = np.zeros_like(outs[0][0])
+    for f in hbfo.DIE_STATS_DTYPE.names:
+        ds_sum[f] = sum(o[0][f] for o in outs)
+        assert np.array_equal(ds[f], ds_sum[f]), f
+    assert np.array_equal(busy, sum(o[1] for o in outs))     # an instance leaves the queues of the others at zero
+    assert res["n_modeled"] == sum(o[2]["n_modeled"] for o in outs) and res["n_native"] == 0
+    assert res["modeled_ns"] == sum(o[2]["modeled_ns"] for o in outs)
+    assert res["service_ns"] == sum(o[2]["service_ns"] for o in outs)
+    assert res["max_completion_ns"] == max(o[2]["max_completion_ns"] for o in outs)
+    return dt
+
+
 @pytest.mark.parametrize("path", ["auto", "sort"])
-def test_full_size_batch_against_per_queue_oracle(full, path):
-    hbf, w, queue = full
+def test_full_size_batch_against_the_oracle_on_every_queue(full, path):
+    hbf, w, shards, subs = full
     ctx = hbf.Context(w.profile)
     for r in w.ranges:
         ctx.register_range(*r)
     ctx.set_path(hbf.PATH_AUTO if path == "auto" else hbf.PATH_SORT)
     runs = run_gpu(hbf, ctx, w)
     issue = w.acc["issue_ns"]
-    sample = [0, 1, 777, 1500, 2047]
-    oracles = {}
-    for q in sample:
-        o = hbfo.Oracle(w.profile)
-        for r in w.ranges:
-            o.register_range(*r)
-        oracles[q] = o
-    npages = np.maximum(1, w.acc["bytes"].astype(np.int64) >> 14)            # size-aligned reads: 1, 2 or 4 pages
-    for step, (comp, stall, ds, busy, res) in enumerate(runs):
-        assert np.array_equal(stall, comp - issue)
-        assert res["n_modeled"] == N_FULL and res["n_native"] == 0
-        assert res["service_ns"] == int(npages.sum()) * 20000 == int(ds["busy_ns"].sum())
-        assert int(ds["n_read"].sum()) == N_FULL and int(ds["bytes_read"].sum()) == int(np.maximum(w.acc["bytes"], 64).astype(np.int64).sum())
-        assert res["modeled_ns"] == int(stall.sum()) and res["max_completion_ns"] == int(comp.max())
-        assert (stall >= npages * 20000).all()
-        for q in sample:
-            idx = np.flatnonzero(queue == q)
-            _, c_o, s_o, _, _ = oracles[q].submit(w.acc[idx])
-            bad = np.flatnonzero(comp[idx] != c_o)
-            assert bad.size == 0, (path, step, q, int(idx[bad[0]]), int(comp[idx][bad[0]]), int(c_o[bad[0]]))
-            assert int(busy[q]) == int(oracles[q].busy_until()[q])
+    groups = len(shards)
+    oracles = [make_oracle(w) for _ in range(groups)]
+    with ThreadPoolExecutor(groups) as pool:
+        for step, (comp, stall, ds, busy, res) in enumerate(runs):
+            assert np.array_equal(stall, comp - issue)
+            dt = check_against_shards(hbf, pool, oracles, subs, shards, comp, stall, ds, busy, res)
+            print("\n%s path, pass %d: the oracle served and checked %d accesses on %d threads in %.1f s (%.1f M accesses/s)"
+                  % (path, step, N_FULL, groups, dt, N_FULL / dt / 1e6))
     ctx.destroy()
 
 
 def test_full_size_batch_with_refresh_claims(full):
     """Retention on, in the configuration `bench.py --workload capacity_retention` times: the batch, one epoch that
     makes every block eligible, the batch again with its first 33.5 M accesses claiming one refresh quantum each.
-    Claims go to the modeled accesses in index order, so within one queue's sub-stream they go to a prefix too: the
-    oracle serves a sampled queue's sub-stream alone with exactly that many quanta of debt (made by an epoch of its
-    own and trimmed by idle-time decay) and must give the same completions."""
+    Claims go to the modeled accesses in index order, so within a sub-stream of whole queues they go to a prefix too:
+    every oracle instance serves its sub-stream with exactly that many quanta of debt (made by an epoch of its own and
+    trimmed by idle-time decay) and must give the same completions, per-die totals and queue state: all 200 M accesses."""
     import torch
-    hbf, w, queue = full
+    hbf, w, shards, subs = full
     ret = dict(pages_per_block=256, blocks_per_plane=64, blocks_per_zone=8, max_pec=3000, disturb_limit=1,
                l_ref_s=3.15e7, t_ref_c=40.0, ea_ev=1.04, accel=1.0, lead_threshold=0.8)
     ctx = hbf.Context(w.profile)
@@ -119,22 +156,28 @@ def test_full_size_batch_with_refresh_claims(full):
     read_pj = 2 * 84 * int(np.maximum(w.acc["bytes"], 64).astype(np.int64).sum())          # two batches of reads
     assert int(ctx.get_pending_energy().sum()) == read_pj + debt * quantum_pj
     del d_acc, d_comp, d_stall, d_ds
-    for q in [0, 1, 777, 2047]:
-        idx = np.flatnonzero(queue == q)
-        k = int(np.count_nonzero(idx < debt))                 # every access is modeled: the claim limit is the debt itself
-        o = hbfo.Oracle(w.profile)
-        for r in w.ranges:
-            o.register_range(*r)
-        o.enable_retention(**dict(ret, pages_per_block=1, blocks_per_plane=16, blocks_per_zone=8, disturb_limit=0, lead_threshold=1e-9))
-        o.submit(w.acc[idx])
-        o.retention_advance(10**9, np.array([60.0]))
-        assert o.retention_totals()["planned"] == 2048 * 16 >= k
-        o.retention_decay((2048 * 16 - k) * 395000)
-        assert o.retention_totals()["planned"] - o.retention_totals()["decayed"] == k
-        _, c_o, _, _, _ = o.submit(w.acc[idx])
-        bad = np.flatnonzero(comp[idx] != c_o)
-        assert bad.size == 0, (q, int(idx[bad[0]]), int(comp[idx][bad[0]]), int(c_o[bad[0]]))
-        assert int(busy[q]) == int(o.busy_until()[q])
+    stall = comp - w.acc["issue_ns"]
+
+    def with_debt(k, sub):
+        def setup(o):                                         # every block eligible after one epoch; all but k quanta drained
+            o.enable_retention(**dict(ret, disturb_limit=0, lead_threshold=1e-9))
+            o.submit(sub)
+            o.retention_advance(10**9, np.array([60.0]))
+            assert o.retention_totals()["planned"] == debt
+            o.retention_decay((debt - k) * 395000)
+            assert o.retention_totals()["planned"] - o.retention_totals()["decayed"] == k
+        return setup
+
+    ks = [int(np.count_nonzero(idx < debt)) for idx in shards]   # every access is modeled: the claim limit is the debt itself
+    assert sum(ks) == debt
+    with ThreadPoolExecutor(len(shards)) as pool:
+        oracles = list(pool.map(lambda j: make_oracle(w, with_debt(ks[j], subs[j])), range(len(shards))))
+        outs = list(pool.map(lambda j: compare_shard(oracles[j], subs[j], shards[j], comp, stall), range(len(shards))))
+    for f in ("busy_ns", "bytes_read", "n_read", "energy_pj"):
+        assert np.array_equal(ds[f], sum(o[0][f] for o in outs)), f
+    assert np.array_equal(busy, sum(o[1] for o in outs))
+    assert res["service_ns"] == sum(o[2]["service_ns"] for o in outs)
+    assert ctx.last_result()["modeled_ns"] == sum(o[2]["modeled_ns"] for o in outs)
     ctx.destroy()
 
 
