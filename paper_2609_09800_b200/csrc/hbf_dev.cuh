@@ -89,8 +89,9 @@ struct Workspace {
     int64_t *in_agg;                     // [tiles][queues][2]: per-tile, per-queue max-plus aggregate (S, M)
     int64_t *in_bin;                     // [tiles][queues]: busy-until entering each tile
     void *in_tile;                       // [tiles] stall bookkeeping of the in-order path
-    void *in_head;                       // [tiles][queues][8]: the first accesses of every (tile, queue), for the fix-up
+    void *in_head;                       // [tiles][queues][8]: the first accesses of every (tile, queue), contiguous, for the fix-up
     uint8_t *in_headcnt;                 // [tiles][queues]: how many of them exist; 0xff marks a queue for the straggle pass
+    uint16_t *in_qid;                    // [tiles][stride]: queue of each of the first records of every tile (0xffff: not modeled), for the straggle pass
     uint32_t *bus_xfer;                  // [n] transfer time of every read (only with the channel-bus stage on)
     size_t bytes;
 };
@@ -123,6 +124,12 @@ cudaError_t ensure_dyn_smem(const void *kernel, size_t bytes);
 constexpr uint32_t kInMaxQueues = 2048;  // the in-order path keeps per-queue state in shared memory
 constexpr uint32_t kInMaxTiles = 1024;
 constexpr uint32_t kInTileQuantum = 1024; // tiles of the in-order path are a multiple of this many records
+constexpr uint32_t kInQidPrefix = 131072; // records at the head of a tile whose queue numbers the serve pass leaves for the straggle pass
+// 16-bit queue numbers kept for a batch of n records (an upper bound over every tiling of it)
+inline uint64_t inorder_qid_entries(uint64_t n) {
+    const uint64_t a = 2 * (n + kInTileQuantum), b = (uint64_t)kInMaxTiles * kInQidPrefix;
+    return a < b ? a : b;
+}
 // upper bound of the number of tiles of a batch of n records, on any device: what the workspace is carved for
 inline uint64_t inorder_tiles_bound(uint64_t n) {
     const uint64_t t = (n + kInTileQuantum - 1) / kInTileQuantum;

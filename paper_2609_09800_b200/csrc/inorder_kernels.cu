@@ -182,7 +182,6 @@ __device__ __forceinline__ Served serve_terms_geom(const FastGeom &g, const Mode
 struct InTile { long long spec_sum, fix_delta, true_sum; uint32_t reserve; uint32_t stragglers; };
 // The first kInHead accesses of every (tile, queue), as the serve pass saw them: all the fix-up needs in the common case.
 constexpr int kInHead = 8;
-constexpr uint8_t kInStraggler = 0xffu;                   // head count of a (tile, queue) the fix-up hands to the straggle pass
 struct InHead { int64_t m, s; uint32_t xo, idx; };       // arrival + service, service, transfer | op << 31, batch index
 
 // ======================================================================================================
@@ -221,7 +220,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
                 hbf_die_stats_t *stats_stage, int64_t *__restrict__ completion, int64_t *__restrict__ stall,
                 const int64_t *__restrict__ in_bin, InTile *in_tile, InHead *__restrict__ in_head, uint8_t *__restrict__ in_headcnt,
                 const int64_t *__restrict__ busy, const unsigned long long *claim_limit_p, uint32_t *die_claims,
-                const __grid_constant__ RetDev ret) {
+                const __grid_constant__ RetDev ret, uint16_t *__restrict__ in_qid, uint32_t qid_stride) {
     extern __shared__ __align__(16) unsigned char in_smem[];
     __shared__ long long s_red[2];
     __shared__ uint32_t s_heads_full;                     // queues whose head entries are complete
@@ -282,6 +281,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
     const hbf_access_t *acc_t = acc + tile_begin;
     int64_t *completion_t = completion + tile_begin, *stall_t = stall + tile_begin;
     uint8_t *status_t = status ? status + tile_begin : nullptr;
+    uint16_t *qid_t = in_qid + (uint64_t)tile * qid_stride;   // the straggle pass filters the head of the tile by these
     const uint32_t rows = (tile_len + 31u) / 32u;
     const uint32_t turns = (rows + K - 1) / K;
     const unsigned le_mask = lanemask_lt() | (1u << lane);
@@ -356,6 +356,11 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
                 const uint32_t npages = (uint32_t)(((uint64_t)((uint32_t)off & page_mask) + (uint32_t)bf[u] + page_mask) >> mp.page_shift);
                 atomicAdd(&ret.disturb[ret_block_of(mp, ret, off)], npages);
             }
+        }
+        if (!RESERVE && turn * (uint32_t)(K * 32) < qid_stride) {   // (the stride is a multiple of a turn's records)
+#pragma unroll
+            for (int u = 0; u < K; ++u)
+                if (valid[u]) qid_t[i[u]] = ready[u] ? (uint16_t)v[u].queue : (uint16_t)0xffffu;
         }
         if (!RESERVE) {
 #pragma unroll
@@ -449,7 +454,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
                         const uint32_t ci = c0[u] + rank1[u] - 1u;
                         if (ci < (uint32_t)kInHead) {
                             InHead h; h.m = a[u] + v[u].s; h.s = v[u].s; h.xo = v[u].xfer | (v[u].op << 31); h.idx = (uint32_t)tile_begin + i[u];
-                            in_head[((uint64_t)tile * kInHead + ci) * R + qi[u]] = h;
+                            in_head[((uint64_t)tile * R + qi[u]) * kInHead + ci] = h;
                         }
                         if (last[u] && c1[u] != c0[u] && c1[u] == (uint32_t)kInHead) atomicAdd(&s_heads_full, 1u);
                     }
@@ -503,18 +508,24 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
 }
 
 // ======================================================================================================
-// scan over tiles, one thread per queue; also decides what happens to the batch
+// scan over tiles; also decides what happens to the batch.
+// A block takes kInScanQueues consecutive queues (threadIdx.x) and cuts the tiles into kInScanChunks runs of
+// consecutive tiles (threadIdx.y).  Every thread composes the aggregates (S, M) of its run, the runs' maps are
+// composed in order through shared memory, and the thread walks its run again from the true busy-until entering
+// it, which it stores for every tile.  The kInScanQueues lanes of a run read consecutive 16-byte aggregates:
+// whole 128-byte lines.  A few tiles per thread and all blocks resident at once: no long chain of loads.
 // ======================================================================================================
-constexpr int kInScanThreads = 32;
-constexpr int kInScanDepth = 16;
+constexpr int kInScanChunks = 64;
+constexpr int kInScanQueues = 8;
 
-__global__ void __launch_bounds__(kInScanThreads)
+__global__ void __launch_bounds__(kInScanQueues * kInScanChunks)
 k_inorder_scan(BatchCtrl *ctrl, const ModelParams *__restrict__ mp, uint32_t n_tiles, const int64_t *__restrict__ in_agg,
-               int64_t *__restrict__ in_bin, const int64_t *__restrict__ busy, int64_t *busy_stage,
+               int64_t *__restrict__ in_bin, const int64_t *__restrict__ busy, int64_t *__restrict__ busy_stage,
                hbf_die_stats_t *stats_stage, int forced) {
+    __shared__ longlong2 s_map[kInScanChunks][kInScanQueues];
     if (ctrl->skip || ctrl->run_sort) return;
-    const bool fault = ctrl->n_fault != 0, unsorted = ctrl->unsorted != 0u;
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
+    const bool fault = ctrl->n_fault != 0, unsorted = ctrl->unsorted != 0u;   // settled by the serve pass: every thread sees the same
+    if (blockIdx.x == 0 && threadIdx.x == 0 && threadIdx.y == 0) {
         if (fault) { ctrl->code = HBF_E_ACCESS_FAULT; ctrl->skip = 1; }                 // fail closed: refuse the batch
         else if (unsorted && forced) { ctrl->code = HBF_E_INVAL; ctrl->skip = 1; }
         else if (unsorted) ctrl->run_sort = 1u;                                         // hand the batch to the sort path
@@ -522,95 +533,41 @@ k_inorder_scan(BatchCtrl *ctrl, const ModelParams *__restrict__ mp, uint32_t n_t
     }
     if (fault || unsorted) return;
     const uint32_t R = mp->n_queues;
-    const uint32_t r = blockIdx.x * kInScanThreads + threadIdx.x;
+    const uint32_t r = blockIdx.x * (uint32_t)kInScanQueues + threadIdx.x, chunk = threadIdx.y;
+    const uint32_t per = (n_tiles + kInScanChunks - 1) / kInScanChunks;
+    const uint32_t t_lo = min(n_tiles, chunk * per), t_hi = min(n_tiles, t_lo + per);
+    const bool live = r < R;
+    const longlong2 *agg = reinterpret_cast<const longlong2 *>(in_agg) + r;
+    long long S = 0, M = kNegInf;                            // the run's own map
+    if (live) {
+        for (uint32_t t = t_lo; t < t_hi; ++t) {
+            const longlong2 v = agg[(uint64_t)t * R];
+            M = max((int64_t)(M + v.x), (int64_t)v.y); S += v.x;
+        }
+    }
+    s_map[chunk][threadIdx.x] = make_longlong2(S, M);
+    __syncthreads();
     long long tot = 0;
-    if (r < R) {
+    if (live) {
+        // busy-until entering the run: the state earlier batches left, through the maps of the runs before it
         int64_t B = busy[r];
-        const longlong2 *a = reinterpret_cast<const longlong2 *>(in_agg) + r;
-        uint32_t t = 0;
-        for (; t + kInScanDepth <= n_tiles; t += kInScanDepth) {
-            longlong2 v[kInScanDepth];
-#pragma unroll
-            for (int k = 0; k < kInScanDepth; ++k) v[k] = a[(uint64_t)(t + k) * R];
-#pragma unroll
-            for (int k = 0; k < kInScanDepth; ++k) {
-                in_bin[(uint64_t)(t + k) * R + r] = B; B = max((int64_t)(B + v[k].x), (int64_t)v[k].y); tot += v[k].x;
-            }
+        for (uint32_t c = 0; c < chunk; ++c) { const longlong2 v = s_map[c][threadIdx.x]; B = max((int64_t)(B + v.x), (int64_t)v.y); }
+        for (uint32_t t = t_lo; t < t_hi; ++t) {
+            const longlong2 v = agg[(uint64_t)t * R];
+            in_bin[(uint64_t)t * R + r] = B;
+            B = max((int64_t)(B + v.x), (int64_t)v.y);
         }
-        for (; t < n_tiles; ++t) {
-            const longlong2 v = a[(uint64_t)t * R];
-            in_bin[(uint64_t)t * R + r] = B; B = max((int64_t)(B + v.x), (int64_t)v.y); tot += v.x;
-        }
-        busy_stage[r] = B;
-        const uint32_t die = mp->queue_level == 0u ? r / mp->planes : r;
-        if (tot) atomicAdd(reinterpret_cast<unsigned long long *>(&stats_stage[die].busy_ns), (unsigned long long)tot);
-    }
-    tot = warp_sum(tot);
-    if (threadIdx.x == 0 && tot) atomicAdd((unsigned long long *)&ctrl->service_ns, (unsigned long long)tot);
-}
-
-// ======================================================================================================
-// fix-up: the true run differs from the as-if-idle run only at the head of each (tile, queue)
-// ======================================================================================================
-constexpr int kInFixThreads = 128;
-
-// One thread per (tile, queue): walk the head table.  A queue that is still backlogged after kInHead
-// accesses is a straggler: its head count is replaced by a mark for the straggle pass, or, when a tile has
-// many of them (the batch arrived on queues that were far behind), the whole tile is flagged to be served again.
-__global__ void __launch_bounds__(kInFixThreads)
-k_inorder_fixup(uint32_t R, uint32_t n_tiles, BatchCtrl *ctrl, const int64_t *__restrict__ in_bin,
-                const InHead *__restrict__ in_head, uint8_t *__restrict__ in_headcnt, int64_t *completion, int64_t *stall,
-                InTile *in_tile) {
-    if (ctrl->skip || ctrl->run_sort || !ctrl->inorder_used) return;
-    const uint64_t idx = (uint64_t)blockIdx.x * kInFixThreads + threadIdx.x;          // tile * R + queue
-    long long max_c = INT64_MIN;
-    if (idx < (uint64_t)n_tiles * R) {
-        const uint32_t tile = (uint32_t)(idx / R);
-        const uint32_t q = (uint32_t)(idx % R);
-        const uint32_t c = tile == 0u ? 0u : in_headcnt[idx];       // the first tile was served from its true entering state
-        int64_t B = in_bin[idx];                             // true busy-until of the queue entering the tile
-        int64_t Bs = kNegInf;                                // busy-until of the as-if-idle run, to know what it wrote
-        long long dstall = 0;
-        bool settled = false;
-        for (uint32_t k = 0; k < c; ++k) {
-            const InHead h = in_head[((uint64_t)tile * kInHead + k) * R + q];
-            if (B <= h.m - h.s) { settled = true; break; }   // idle on arrival: from here on the as-if run was right
-            B += h.s;                                          // it waited for the queue: starts at B
-            Bs = max(Bs + h.s, h.m);
-            const bool op = (h.xo >> 31) != 0u;
-            const int64_t xfer = (int64_t)(h.xo & 0x7fffffffu);
-            const int64_t done = B + (op ? 0 : xfer);
-            dstall += B - Bs;                                  // completion moved from Bs + post to B + post
-            completion[h.idx] = done; stall[h.idx] = done - (h.m - h.s - (op ? xfer : 0));
-            max_c = max(max_c, (long long)done);
-        }
-        if (!settled && c == (uint32_t)kInHead) {
-            // the straggle pass serves this queue again from the tile's start and accounts for all of its corrections
-            in_headcnt[idx] = kInStraggler;
-            const uint32_t rank = atomicAdd(&in_tile[tile].stragglers, 1u);
-            if (rank >= max(8u, R / 16u)) in_tile[tile].reserve = 1u;
-        } else if (dstall) {
-            atomicAdd((unsigned long long *)&in_tile[tile].fix_delta, (unsigned long long)dstall);
+        if (chunk == kInScanChunks - 1) {                    // the last run ends at the batch's end (empty runs pass B through)
+            busy_stage[r] = B;
+            for (uint32_t c = 0; c < (uint32_t)kInScanChunks; ++c) tot += s_map[c][threadIdx.x].x;
+            const uint32_t die = mp->queue_level == 0u ? r / mp->planes : r;
+            if (tot) atomicAdd(reinterpret_cast<unsigned long long *>(&stats_stage[die].busy_ns), (unsigned long long)tot);
         }
     }
-    max_c = warp_max(max_c);
-    if ((threadIdx.x & 31) == 0 && max_c != INT64_MIN) atomicMax(&ctrl->max_completion_ns, max_c);
+    tot = warp_sum(tot);                                     // (only the last run's threads carry a total)
+    if (((threadIdx.y * kInScanQueues + threadIdx.x) & 31u) == 0u && tot)
+        atomicAdd((unsigned long long *)&ctrl->service_ns, (unsigned long long)tot);
 }
-
-// ======================================================================================================
-// straggle: one block per tile that has stragglers (and is not re-served whole).  The block streams the
-// tile's records again, keeps the modeled records of the straggling queues in batch order, and its first
-// warp re-serves them 32 at a time, carrying both the true run (from the true entering busy-until) and the
-// as-if-idle run (to know what the serve pass wrote).  A queue is done when the two runs meet: from there
-// on the serve pass was right.  The block stops at the chunk in which its last queue is done.
-// ======================================================================================================
-constexpr int kInStrThreads = 512;
-constexpr int kInStrItems = 4;
-constexpr int kInStrChunk = kInStrThreads * kInStrItems;
-constexpr int kInStrWarps = kInStrThreads / 32;
-constexpr int kInStrCells = kInStrItems * kInStrWarps;    // (row, warp) cells of the kept-record counts
-constexpr int kInStrCellsPerLane = kInStrCells / 32;
-static_assert(kInStrCells % 32 == 0, "the offset scan gives every lane the same number of cells");
 
 // Queue of an access of the common configuration (one range, power-of-two geometry), or ~0 when the address
 // lies outside the range.  In a batch that was not refused every access inside the range is modeled.
@@ -624,13 +581,59 @@ __device__ __forceinline__ uint32_t fast_queue(const FastRange &f, const ModelPa
     return mp.queue_level == 0u ? die * mp.planes + pl : die;
 }
 
+// ======================================================================================================
+// fix-up and straggle: one block per tile.
+// Fix-up.  The true run differs from the as-if-idle run only at the head of each (tile, queue): a thread starts
+// from the true entering busy-until of its queues and re-serves the head table's accesses in order, until it meets
+// one that arrives on an idle queue; from there on the as-if run was right.  The head entries of a (tile, queue) are
+// contiguous, so they are fetched in two rounds (the first two, which settle nearly every queue, then the rest at
+// once) instead of one dependent load per entry.  A queue still backlogged after kInHead accesses is a straggler;
+// a tile with many of them (the batch arrived on queues that were far behind) is flagged to be served again whole.
+// Straggle.  The block streams the head of the tile again, keeps the modeled records of the straggling queues in
+// batch order and re-serves them a chunk at a time, carrying both the true run (from the true entering
+// busy-until) and the as-if-idle run (to know what the serve pass wrote).  A queue is done when the two runs meet:
+// from there on the serve pass was right.  The block stops at the chunk in which its last queue is done.
+// What it streams: for the first kInQidPrefix records of every tile the serve pass left the queue of each record
+// as a 16-bit number (0xffff: not modeled), so the filter reads 2 bytes per record, 32 records per thread and turn;
+// past that prefix (queues that stay backlogged for very long) it decodes the queue from the records.
+// ======================================================================================================
+struct FixRun { int64_t B, Bs; long long dstall, max_c; bool settled; };
+__device__ __forceinline__ void fix_entry(FixRun &f, const InHead &h, int64_t *completion, int64_t *stall) {
+    if (f.settled) return;
+    if (f.B <= h.m - h.s) { f.settled = true; return; }      // idle on arrival: from here on the as-if run was right
+    f.B += h.s;                                              // it waited for the queue: starts at B
+    f.Bs = max(f.Bs + h.s, h.m);
+    const bool op = (h.xo >> 31) != 0u;
+    const int64_t xfer = (int64_t)(h.xo & 0x7fffffffu);
+    const int64_t done = f.B + (op ? 0 : xfer);
+    f.dstall += f.B - f.Bs;                                  // completion moved from Bs + post to B + post
+    completion[h.idx] = done; stall[h.idx] = done - (h.m - h.s - (op ? xfer : 0));
+    f.max_c = max(f.max_c, (long long)done);
+}
+
+constexpr int kInStrThreads = 512;
+constexpr int kInStrWarps = kInStrThreads / 32;
+constexpr int kInStrQItems = 32;                          // records per thread and turn inside the queue-number prefix
+constexpr int kInStrQChunk = kInStrThreads * kInStrQItems;
+constexpr int kInStrItems = 8;                            // and past it, where the queue is decoded from the record
+constexpr int kInStrChunk = kInStrThreads * kInStrItems;
+constexpr int kInStrKeep = 2048;                          // kept records served at a time (a chunk with more is served in windows)
+constexpr int kInStrCells = kInStrItems * kInStrWarps;    // (item, warp) cells of the kept-record counts, decode path
+constexpr int kInStrCellsPerLane = kInStrCells / 32;
+constexpr int kInStrQueuesPerThread = (kInMaxQueues + kInStrThreads - 1) / kInStrThreads;
+static_assert(kInStrCells % 32 == 0, "the offset scan gives every lane the same number of cells");
+static_assert(kInStrQueuesPerThread % 2 == 0, "the fix-up takes a thread's queues two at a time");
+static_assert(kInStrQChunk <= 65536, "a kept record's position in its chunk is stored in 16 bits");
+static_assert(kInQidPrefix % kInStrQChunk == 0 && kInStrQItems == 32, "a thread's 32 queue numbers are four 16-byte loads");
+
 template <bool DEBT>
-__global__ void __launch_bounds__(kInStrThreads)
-k_inorder_straggle(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_records,
-                   const RangeSnap *__restrict__ ranges_g, const __grid_constant__ ModelParams mp_arg,
-                   const __grid_constant__ FastRange fast_arg, BatchCtrl *ctrl,
-                   const int64_t *__restrict__ in_bin, const uint8_t *__restrict__ in_headcnt, int64_t *completion,
-                   int64_t *stall, InTile *in_tile, const unsigned long long *claim_limit_p) {
+__global__ void __launch_bounds__(kInStrThreads, 2)
+k_inorder_fixstraggle(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_records,
+                      const RangeSnap *__restrict__ ranges_g, const __grid_constant__ ModelParams mp_arg,
+                      const __grid_constant__ FastRange fast_arg, BatchCtrl *ctrl,
+                      const int64_t *__restrict__ in_bin, const InHead *__restrict__ in_head,
+                      const uint8_t *__restrict__ in_headcnt, int64_t *completion, int64_t *stall, InTile *in_tile,
+                      const unsigned long long *claim_limit_p, const uint16_t *__restrict__ in_qid, uint32_t qid_stride) {
     extern __shared__ __align__(16) unsigned char str_smem[];
     __shared__ ModelParams mp;
     __shared__ FastRange fast_range;
@@ -642,25 +645,69 @@ k_inorder_straggle(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t ti
 
     if (ctrl->skip || ctrl->run_sort || !ctrl->inorder_used) return;
     const uint32_t tile = blockIdx.x;
-    if (in_tile[tile].stragglers == 0u || in_tile[tile].reserve) return;
+    if (tile == 0u) return;                                  // the first tile was served from its true entering state
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const RangeSnap &rs = *ranges_g;
     const uint32_t R = mp_arg.n_queues;
     int64_t *Bt = reinterpret_cast<int64_t *>(str_smem);                       // [queues] true run
     int64_t *Ba = Bt + kInMaxQueues;                                           // [queues] as-if-idle run
-    longlong2 *ent_as = reinterpret_cast<longlong2 *>(Ba + kInMaxQueues);      // [chunk] kept records, batch order: issue time, service time
-    uint2 *ent_pq = reinterpret_cast<uint2 *>(ent_as + kInStrChunk);           //         transfer | op << 31, queue | position << 16
-    uint16_t *oq = reinterpret_cast<uint16_t *>(ent_pq + kInStrChunk);         // [stragglers] their queues
+    longlong2 *ent_as = reinterpret_cast<longlong2 *>(Ba + kInMaxQueues);      // [keep] kept records, batch order: issue time, service time
+    uint2 *ent_pq = reinterpret_cast<uint2 *>(ent_as + kInStrKeep);            //        transfer | op << 31, queue | position << 16
+    uint16_t *oq = reinterpret_cast<uint16_t *>(ent_pq + kInStrKeep);          // [stragglers] their queues
     uint8_t *open = reinterpret_cast<uint8_t *>(oq + kInMaxQueues);            // [queues] 1: straggler, runs have not met
     if (tid == 0) { mp = mp_arg; fast_range = fast_arg; s_stragglers = 0u; s_red[0] = 0; s_red[1] = INT64_MIN; }
     __syncthreads();
-    for (uint32_t q = tid; q < kInMaxQueues; q += kInStrThreads) {
-        const bool s = q < R && in_headcnt[(uint64_t)tile * R + q] == kInStraggler;
-        open[q] = s ? 1 : 0;
-        Ba[q] = kNegInf;
-        Bt[q] = s ? in_bin[(uint64_t)tile * R + q] : kNegInf;
-        if (s) oq[atomicAdd(&s_stragglers, 1u)] = (uint16_t)q;
+
+    // ---- fix-up: this thread's queues of the tile (their loads are issued side by side) ------------------------
+    long long dstall = 0, max_c = INT64_MIN;
+    {
+        constexpr int kRound = 2;                            // queues whose loads are in flight together
+        for (int k0 = 0; k0 < kInStrQueuesPerThread; k0 += kRound) {
+            uint32_t c[kRound]; int64_t Bin[kRound];
+            InHead e0[kRound], e1[kRound];
+#pragma unroll
+            for (int k = 0; k < kRound; ++k) {
+                const uint32_t q = (uint32_t)((k0 + k) * kInStrThreads + tid);
+                c[k] = 0u; Bin[k] = kNegInf;
+                if (q < R) { c[k] = in_headcnt[(uint64_t)tile * R + q]; Bin[k] = in_bin[(uint64_t)tile * R + q]; }
+            }
+#pragma unroll
+            for (int k = 0; k < kRound; ++k) {
+                const InHead *h = in_head + ((uint64_t)tile * R + (uint32_t)((k0 + k) * kInStrThreads + tid)) * kInHead;
+                if (c[k] > 0u) e0[k] = h[0];
+                if (c[k] > 1u) e1[k] = h[1];
+            }
+#pragma unroll
+            for (int k = 0; k < kRound; ++k) {
+                const uint32_t q = (uint32_t)((k0 + k) * kInStrThreads + tid);
+                if (q < kInMaxQueues) { open[q] = 0; Ba[q] = kNegInf; Bt[q] = kNegInf; }
+                if (c[k] == 0u) continue;
+                FixRun f; f.B = Bin[k]; f.Bs = kNegInf; f.dstall = 0; f.max_c = INT64_MIN; f.settled = false;
+                fix_entry(f, e0[k], completion, stall);
+                if (c[k] > 1u) fix_entry(f, e1[k], completion, stall);
+                if (!f.settled && c[k] > 2u) {
+                    const InHead *h = in_head + ((uint64_t)tile * R + q) * kInHead;
+                    for (uint32_t j = 2; j < c[k]; ++j) fix_entry(f, h[j], completion, stall);
+                }
+                max_c = max(max_c, f.max_c);                 // (true completions: valid whoever writes them last)
+                if (!f.settled && c[k] == (uint32_t)kInHead) {
+                    // still backlogged after its head entries: the loop below serves this queue again from the tile's
+                    // start and accounts for all of its corrections
+                    open[q] = 1; Bt[q] = Bin[k];
+                    oq[atomicAdd(&s_stragglers, 1u)] = (uint16_t)q;
+                } else {
+                    dstall += f.dstall;
+                }
+            }
+        }
     }
+    __syncthreads();
+    const uint32_t stragglers = s_stragglers;
+    if (stragglers >= max(8u, R / 16u)) {                    // many queues far behind: the re-serve pass takes the whole tile
+        if (tid == 0) in_tile[tile].reserve = 1u;
+        return;
+    }
+    if (stragglers > 0u) {
     const int64_t q_ppm = ctrl->q_ppm;
     const Div64 div_q = ctrl->div_q;
     const bool one_range = fast_arg.on != 0u && mp_arg.pow2_geom != 0u;
@@ -669,105 +716,166 @@ k_inorder_straggle(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t ti
     const int64_t quantum_ns = !DEBT ? 0 : q_ppm == 1000000 ? mp_arg.t_read_ns + mp_arg.t_prog_ns
         : (int64_t)div64((uint64_t)(mp_arg.t_read_ns + mp_arg.t_prog_ns) * 1000000ull + (uint64_t)q_ppm - 1ull, div_q);
     const uint64_t tile_begin = (uint64_t)tile * tile_records, tile_end = min(n, tile_begin + tile_records);
-    long long dstall = 0, max_c = INT64_MIN;
+    const uint32_t tile_len = (uint32_t)(tile_end - tile_begin);       // offsets inside a tile fit 32 bits
+    const hbf_access_t *acc_t = acc + tile_begin;
+    const uint4 *qid_t = reinterpret_cast<const uint4 *>(in_qid + (uint64_t)tile * qid_stride);
     unsigned ignored = 0;                                    // (the serve pass has already vetted every service time)
-    __syncthreads();
-    const uint32_t stragglers = s_stragglers;
     if (tid == 0) s_open = (int)stragglers;
 
-    // the addresses of the next chunk are on their way while this one is filtered
-    uint64_t nx_addr[kInStrItems];
-    auto fetch = [&](uint64_t cb) {
+    // the queue numbers of the next chunk are on their way while this one is filtered
+    // (only the queue numbers: past the prefix, a rare stretch, the addresses are loaded when they are needed)
+    uint4 nx_q[kInStrQItems / 8];
+    auto fetch = [&](uint32_t cb) {
+        if (cb < tile_len && cb + kInStrQChunk <= qid_stride) {
 #pragma unroll
-        for (int j = 0; j < kInStrItems; ++j) {
-            const uint64_t i = cb + (uint64_t)(j * kInStrThreads + tid);
-            nx_addr[j] = i < tile_end ? __ldg(reinterpret_cast<const uint64_t *>(acc + i)) : 0ull;
+            for (int k = 0; k < kInStrQItems / 8; ++k) nx_q[k] = __ldg(qid_t + (cb >> 3) + tid * (kInStrQItems / 8) + k);
         }
     };
-    fetch(tile_begin);
+    // a kept record: its terms are computed here, once, and it takes its place in the window of kept records
+    auto put = [&](uint32_t cb, uint32_t e, uint32_t slot) {
+        const uint64_t *rec = reinterpret_cast<const uint64_t *>(acc_t + cb + e);
+        const uint64_t addr = __ldg(rec);
+        const int64_t issue = (int64_t)__ldg(rec + 1);
+        const uint64_t bf = __ldg(rec + 2);
+        Served v = fast_terms ? serve_terms_fast(fast_range, mp, addr, issue, bf)
+                              : serve_terms(rs, mp, addr, issue, bf, q_ppm, div_q, ignored, 33);
+        if (DEBT && tile_begin + cb + e < claim_limit) v.s += quantum_ns;
+        ent_as[slot] = make_longlong2(issue, v.s);
+        ent_pq[slot] = make_uint2(v.xfer | (v.op << 31), v.queue | (e << 16));
+    };
+    fetch(0u);
 
-    for (uint64_t cbase = tile_begin; cbase < tile_end; cbase += kInStrChunk) {
-        // ---- keep the modeled records of the open queues, in batch order -----------------------------------
-        uint64_t addr[kInStrItems];
+    uint32_t cb = 0;
+    while (cb < tile_len) {
+        const bool by_qid = cb + kInStrQChunk <= qid_stride;  // the same for the whole block
+        const uint32_t step = by_qid ? (uint32_t)kInStrQChunk : (uint32_t)kInStrChunk;
+        // ---- keep the modeled records of the open queues, in batch order: bit j of `keep` is this thread's item j.
+        // Inside the prefix a thread's items are 32 consecutive records; past it, eight records a block width apart.
+        uint32_t keep = 0, first = 0, rk[kInStrItems];
+        if (by_qid) {
+            const uint32_t room = tile_len - cb;             // records of the tile from this chunk on
 #pragma unroll
-        for (int j = 0; j < kInStrItems; ++j) addr[j] = nx_addr[j];
-        fetch(cbase + kInStrChunk);
-        uint32_t keep = 0, rk[kInStrItems];
-#pragma unroll
-        for (int j = 0; j < kInStrItems; ++j) {
-            const uint64_t i = cbase + (uint64_t)(j * kInStrThreads + tid);
-            bool k = false;
-            if (i < tile_end) {
-                if (one_range) {
-                    const uint32_t q = fast_queue(fast_range, mp, addr[j]);
-                    k = q != 0xffffffffu && open[q] != 0;
-                } else {
-                    const uint64_t *rec = reinterpret_cast<const uint64_t *>(acc + i);
-                    const Served v = serve_terms(rs, mp, addr[j], (int64_t)__ldg(rec + 1), __ldg(rec + 2), q_ppm, div_q, ignored, 33);
-                    k = v.st == HBF_ST_READY && open[v.queue] != 0;
-                }
+            for (int j = 0; j < kInStrQItems; ++j) {
+                const uint4 v = nx_q[j >> 3];
+                const uint32_t w = ((j >> 1) & 3) == 0 ? v.x : ((j >> 1) & 3) == 1 ? v.y : ((j >> 1) & 3) == 2 ? v.z : v.w;
+                const uint32_t q = (w >> (16 * (j & 1))) & 0xffffu;
+                const bool k = q < R && (uint32_t)(tid * kInStrQItems + j) < room && open[q] != 0;
+                keep |= k ? 1u << j : 0u;
             }
-            const unsigned bal = __ballot_sync(0xffffffffu, k);
-            rk[j] = (uint32_t)__popc(bal & lanemask_lt());
-            if (lane == 0) s_cells[j * kInStrWarps + warp] = (uint32_t)__popc(bal);
-            keep |= k ? 1u << j : 0u;
-        }
-        __syncthreads();
-        if (warp == 0) {
-            uint32_t c[kInStrCellsPerLane], tot = 0;
-#pragma unroll
-            for (int b = 0; b < kInStrCellsPerLane; ++b) { c[b] = s_cells[lane * kInStrCellsPerLane + b]; tot += c[b]; }
-            uint32_t incl = tot;
+            fetch(cb + step);
+            const uint32_t cnt = (uint32_t)__popc(keep);
+            uint32_t incl = cnt;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += t; }
-            uint32_t run = incl - tot;
+            if (lane == 31) s_cells[warp] = incl;
+            __syncthreads();
+            if (warp == 0) {
+                const uint32_t c = lane < kInStrWarps ? s_cells[lane] : 0u;
+                uint32_t in2 = c;
 #pragma unroll
-            for (int b = 0; b < kInStrCellsPerLane; ++b) { s_cells[lane * kInStrCellsPerLane + b] = run; run += c[b]; }
-            if (lane == 31) s_total = incl;
-        }
-        __syncthreads();
-#pragma unroll
-        for (int j = 0; j < kInStrItems; ++j)
-            if (keep & (1u << j)) {                          // few records are kept: their terms are computed here, once
-                const uint32_t e = (uint32_t)(j * kInStrThreads + tid);
-                const uint64_t *rec = reinterpret_cast<const uint64_t *>(acc + cbase + e);
-                const int64_t issue = (int64_t)__ldg(rec + 1);
-                const uint64_t bf = __ldg(rec + 2);
-                Served v = fast_terms ? serve_terms_fast(fast_range, mp, addr[j], issue, bf)
-                                      : serve_terms(rs, mp, addr[j], issue, bf, q_ppm, div_q, ignored, 33);
-                if (DEBT && cbase + e < claim_limit) v.s += quantum_ns;
-                const uint32_t pos = s_cells[j * kInStrWarps + warp] + rk[j];
-                ent_as[pos] = make_longlong2(issue, v.s);
-                ent_pq[pos] = make_uint2(v.xfer | (v.op << 31), v.queue | (e << 16));
+                for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_up_sync(0xffffffffu, in2, o); if (lane >= o) in2 += t; }
+                if (lane < kInStrWarps) s_cells[lane] = in2 - c;
+                if (lane == 31) s_total = in2;
             }
-        __syncthreads();
-        // ---- one thread per straggling queue walks the kept records (they are in batch order) and re-serves its own
-        // (spread over the warps first, then over their lanes: lanes of a warp that find their records diverge)
-        for (uint32_t t = (uint32_t)(lane * kInStrWarps + warp); t < stragglers; t += kInStrThreads) {
-            const uint32_t q = oq[t];
-            if (!open[q]) continue;
-            const uint32_t total = min(s_total, (uint32_t)kInStrChunk);
-            int64_t BT = Bt[q], BA = Ba[q];
-            for (uint32_t k = 0; k < total; ++k) {
-                const uint2 pq = ent_pq[k];
-                if ((pq.y & 0xffffu) != q) continue;
-                const longlong2 as = ent_as[k];
-                const int64_t xfer = (int64_t)(pq.x & 0x7fffffffu);
-                const bool op = (pq.x >> 31) != 0u;
-                const int64_t a = as.x + (op ? xfer : 0);
-                BT = max(a, BT) + as.y; BA = max(a, BA) + as.y;
-                if (BT != BA) {                               // the serve pass wrote BA + post
-                    const uint64_t i = min(cbase + (pq.y >> 16), tile_end - 1);
-                    const int64_t done = BT + (op ? 0 : xfer);
-                    completion[i] = done; stall[i] = done - as.x;
-                    dstall += BT - BA; max_c = max(max_c, (long long)done);
+            __syncthreads();
+            first = s_cells[warp] + incl - cnt;
+        } else {
+            uint64_t addr[kInStrItems];
+#pragma unroll
+            for (int j = 0; j < kInStrItems; ++j) {
+                const uint32_t i = cb + (uint32_t)(j * kInStrThreads + tid);
+                addr[j] = i < tile_len ? __ldg(reinterpret_cast<const uint64_t *>(acc_t + i)) : ~0ull;
+            }
+#pragma unroll
+            for (int j = 0; j < kInStrItems; ++j) {
+                const uint32_t i = cb + (uint32_t)(j * kInStrThreads + tid);
+                bool k = false;
+                if (i < tile_len) {
+                    if (one_range) {
+                        const uint32_t q = fast_queue(fast_range, mp, addr[j]);
+                        k = q != 0xffffffffu && open[q] != 0;
+                    } else {
+                        const uint64_t *rec = reinterpret_cast<const uint64_t *>(acc_t + i);
+                        const Served v = serve_terms(rs, mp, addr[j], (int64_t)__ldg(rec + 1), __ldg(rec + 2), q_ppm, div_q, ignored, 33);
+                        k = v.st == HBF_ST_READY && open[v.queue] != 0;
+                    }
+                }
+                const unsigned bal = __ballot_sync(0xffffffffu, k);
+                rk[j] = (uint32_t)__popc(bal & lanemask_lt());
+                if (lane == 0) s_cells[j * kInStrWarps + warp] = (uint32_t)__popc(bal);
+                keep |= k ? 1u << j : 0u;
+            }
+            __syncthreads();
+            if (warp == 0) {
+                uint32_t c[kInStrCellsPerLane], tot = 0;
+#pragma unroll
+                for (int b = 0; b < kInStrCellsPerLane; ++b) { c[b] = s_cells[lane * kInStrCellsPerLane + b]; tot += c[b]; }
+                uint32_t incl = tot;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += t; }
+                uint32_t run = incl - tot;
+#pragma unroll
+                for (int b = 0; b < kInStrCellsPerLane; ++b) { s_cells[lane * kInStrCellsPerLane + b] = run; run += c[b]; }
+                if (lane == 31) s_total = incl;
+            }
+            __syncthreads();
+#pragma unroll
+            for (int j = 0; j < kInStrItems; ++j) rk[j] += s_cells[j * kInStrWarps + warp];
+        }
+        // ---- the kept records, a window of kInStrKeep at a time (one window, nearly always)
+        const uint32_t total = s_total;
+        for (uint32_t wb = 0; wb < total; wb += (uint32_t)kInStrKeep) {
+            const uint32_t wn = min(total - wb, (uint32_t)kInStrKeep);
+            if (by_qid) {
+                uint32_t m = keep;
+                while (m) {
+                    const uint32_t j = (uint32_t)__ffs((int)m) - 1u;
+                    m &= m - 1u;
+                    const uint32_t slot = first + (uint32_t)__popc(keep & ((1u << j) - 1u)) - wb;   // (wraps below the window)
+                    if (slot < wn) put(cb, (uint32_t)(tid * kInStrQItems) + j, slot);
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < kInStrItems; ++j)
+                    if ((keep >> j) & 1u) { const uint32_t slot = rk[j] - wb; if (slot < wn) put(cb, (uint32_t)(j * kInStrThreads + tid), slot); }
+            }
+            __syncthreads();
+            // one warp per straggling queue scans the window 32 records at a time (they are in batch order) and re-serves
+            // its own in order; every lane carries the two runs, lane 0 writes
+            for (uint32_t t = (uint32_t)warp; t < stragglers; t += kInStrWarps) {
+                const uint32_t q = oq[t];
+                if (!open[q]) continue;
+                int64_t BT = Bt[q], BA = Ba[q];
+                for (uint32_t k0 = 0; k0 < wn; k0 += 32u) {
+                    const uint32_t k = k0 + (uint32_t)lane;
+                    unsigned hits = __ballot_sync(0xffffffffu, k < wn && (ent_pq[min(k, wn - 1u)].y & 0xffffu) == q);
+                    while (hits) {
+                        const uint32_t kk = k0 + (uint32_t)__ffs((int)hits) - 1u;
+                        hits &= hits - 1u;
+                        const uint2 pq = ent_pq[kk];
+                        const longlong2 as = ent_as[kk];
+                        const int64_t xfer = (int64_t)(pq.x & 0x7fffffffu);
+                        const bool op = (pq.x >> 31) != 0u;
+                        const int64_t a = as.x + (op ? xfer : 0);
+                        BT = max(a, BT) + as.y; BA = max(a, BA) + as.y;
+                        if (BT != BA && lane == 0) {          // the serve pass wrote BA + post
+                            const uint64_t i = min(tile_begin + cb + (pq.y >> 16), tile_end - 1);
+                            const int64_t done = BT + (op ? 0 : xfer);
+                            completion[i] = done; stall[i] = done - as.x;
+                            dstall += BT - BA; max_c = max(max_c, (long long)done);
+                        }
+                    }
+                }
+                if (lane == 0) {
+                    Bt[q] = BT; Ba[q] = BA;
+                    if (BT == BA) { open[q] = 0; atomicSub(&s_open, 1); }   // the runs have met: the rest of the tile was served right
                 }
             }
-            Bt[q] = BT; Ba[q] = BA;
-            if (BT == BA) { open[q] = 0; atomicSub(&s_open, 1); }   // the runs have met: the rest of the tile was served right
+            __syncthreads();
         }
-        __syncthreads();
         if (*reinterpret_cast<volatile int *>(&s_open) <= 0) break;
+        cb += step;
+    }
     }
     dstall = warp_sum(dstall); max_c = warp_max(max_c);
     if (lane == 0) {
@@ -776,7 +884,7 @@ k_inorder_straggle(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t ti
     }
     __syncthreads();
     if (tid == 0) {
-        if (s_red[0]) atomicAdd((unsigned long long *)&in_tile[tile].fix_delta, (unsigned long long)s_red[0]);
+        if (s_red[0]) in_tile[tile].fix_delta = s_red[0];    // (cleared by the serve pass; this block is the tile's only writer)
         if (s_red[1] != INT64_MIN) atomicMax(&ctrl->max_completion_ns, s_red[1]);
     }
 }
@@ -802,7 +910,7 @@ uint64_t inorder_tile_records(uint64_t n, int sm_count) {
 
 // dynamic shared memory of the serve kernel: the per-queue state and the per-die counters
 size_t inorder_serve_smem(uint32_t n_dies) { return (size_t)kInMaxQueues * 16 + (size_t)n_dies * 28; }
-static size_t inorder_straggle_smem() { return (size_t)kInMaxQueues * 16 + (size_t)kInStrChunk * 24 + (size_t)kInMaxQueues * 3; }
+static size_t inorder_straggle_smem() { return (size_t)kInMaxQueues * 16 + (size_t)kInStrKeep * 24 + (size_t)kInMaxQueues * 3; }
 
 size_t inorder_head_bytes(uint64_t tiles, uint32_t n_queues) { return tiles * n_queues * (size_t)kInHead * sizeof(InHead); }
 
@@ -817,32 +925,36 @@ cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st) {
         const void *serve_fns[4] = {(const void *)k_inorder_serve<false, false>, (const void *)k_inorder_serve<true, false>,
                                     (const void *)k_inorder_serve<false, true>, (const void *)k_inorder_serve<true, true>};
         for (const void *f : serve_fns) { cudaError_t e = ensure_dyn_smem(f, smem_serve); if (e != cudaSuccess) return e; }
-        cudaError_t e = ensure_dyn_smem((const void *)k_inorder_straggle<false>, smem_str);
+        cudaError_t e = ensure_dyn_smem((const void *)k_inorder_fixstraggle<false>, smem_str);
         if (e != cudaSuccess) return e;
-        e = ensure_dyn_smem((const void *)k_inorder_straggle<true>, smem_str);
+        e = ensure_dyn_smem((const void *)k_inorder_fixstraggle<true>, smem_str);
         if (e != cudaSuccess) return e;
     }
     InTile *tiles = reinterpret_cast<InTile *>(a.ws.in_tile);
     InHead *heads = reinterpret_cast<InHead *>(a.ws.in_head);
     const bool debt = a.claim_limit != nullptr;              // retention on: the kernels that apply the claims
+#ifdef HBF_DBG_NOQID
+    const uint32_t qid_stride = 0;
+#else
+    const uint32_t qid_stride = (uint32_t)std::min<uint64_t>(tile_records, kInQidPrefix);
+#endif
+    if ((uint64_t)n_tiles * qid_stride > inorder_qid_entries(n)) return cudaErrorInvalidValue;
     auto serve = [&](bool reserve) {
         auto k = reserve ? (debt ? k_inorder_serve<true, true> : k_inorder_serve<true, false>)
                          : (debt ? k_inorder_serve<false, true> : k_inorder_serve<false, false>);
         k<<<n_tiles, kInThreads, smem_serve, st>>>(a.acc, n, tile_records, a.ranges, a.mp, a.fast, a.ctrl, a.status, a.ws.in_agg,
                                                    a.stats_stage, a.completion, a.stall, a.ws.in_bin, tiles, heads, a.ws.in_headcnt,
-                                                   a.busy, a.claim_limit, a.die_claims, debt ? *a.ret : RetDev{});
+                                                   a.busy, a.claim_limit, a.die_claims, debt ? *a.ret : RetDev{}, a.ws.in_qid, qid_stride);
     };
     serve(false);
-    k_inorder_scan<<<(R + kInScanThreads - 1) / kInScanThreads, kInScanThreads, 0, st>>>(
+    k_inorder_scan<<<(R + kInScanQueues - 1) / kInScanQueues, dim3(kInScanQueues, kInScanChunks), 0, st>>>(
         a.ctrl, a.mp_dev, n_tiles, a.ws.in_agg, a.ws.in_bin, a.busy, a.busy_stage, a.stats_stage, a.path == HBF_PATH_INORDER ? 1 : 0);
-    const uint64_t fix_threads = (uint64_t)n_tiles * R;
-    k_inorder_fixup<<<(unsigned)((fix_threads + kInFixThreads - 1) / kInFixThreads), kInFixThreads, 0, st>>>(
-        R, n_tiles, a.ctrl, a.ws.in_bin, heads, a.ws.in_headcnt, a.completion, a.stall, tiles);
-    (debt ? k_inorder_straggle<true> : k_inorder_straggle<false>)<<<n_tiles, kInStrThreads, smem_str, st>>>(
-        a.acc, n, tile_records, a.ranges, a.mp, a.fast, a.ctrl, a.ws.in_bin, a.ws.in_headcnt, a.completion, a.stall, tiles, a.claim_limit);
+    (debt ? k_inorder_fixstraggle<true> : k_inorder_fixstraggle<false>)<<<n_tiles, kInStrThreads, smem_str, st>>>(
+        a.acc, n, tile_records, a.ranges, a.mp, a.fast, a.ctrl, a.ws.in_bin, heads, a.ws.in_headcnt, a.completion, a.stall, tiles,
+        a.claim_limit, a.ws.in_qid, qid_stride);
     serve(true);
     k_inorder_total<<<1, 256, 0, st>>>(a.ctrl, tiles, n_tiles);
-    g_kernel_launches += 6;
+    g_kernel_launches += 5;
     return cudaGetLastError();
 }
 

@@ -945,12 +945,13 @@ size_t workspace_layout(uint64_t n, uint32_t n_queues, Workspace *ws, void *base
     void *ia = take(inorder ? in_tiles * n_queues * 16 : 0), *ib = take(inorder ? in_tiles * n_queues * 8 : 0);
     void *it = take(inorder ? in_tiles * 32 : 0), *ih = take(inorder ? inorder_head_bytes(in_tiles, n_queues) : 0);
     void *ic = take(inorder ? in_tiles * n_queues : 0);
+    void *iq = take(inorder ? inorder_qid_entries(nn) * 2 : 0);
     void *bx = take(with_bus ? nn * 4 : 0);
     if (ws) {
         ws->keys[0] = (uint64_t *)k0; ws->keys[1] = (uint64_t *)k1; ws->idx[0] = (uint32_t *)i0; ws->idx[1] = (uint32_t *)i1;
         ws->hist = (uint32_t *)h; ws->sort_desc[0] = (uint32_t *)d0; ws->sort_desc[1] = (uint32_t *)d1;
         ws->scan_desc = sd; ws->in_agg = (int64_t *)ia; ws->in_bin = (int64_t *)ib;
-        ws->in_tile = it; ws->in_head = ih; ws->in_headcnt = (uint8_t *)ic; ws->bus_xfer = (uint32_t *)bx; ws->bytes = off;
+        ws->in_tile = it; ws->in_head = ih; ws->in_headcnt = (uint8_t *)ic; ws->in_qid = (uint16_t *)iq; ws->bus_xfer = (uint32_t *)bx; ws->bytes = off;
     }
     return off;
 }
@@ -1010,9 +1011,68 @@ static cudaError_t launch_sort_path(const SubmitArgs &a, cudaStream_t st) {
     return cudaSuccess;
 }
 
+// ---- the sort path launched from the device -----------------------------------------------------------
+// With HBF_PATH_AUTO the host enqueues the in-order kernels only.  A batch that turns out not to be in issue
+// order (or has a service time the in-order kernels cannot hold) needs the sort path after all, and the host
+// cannot know that without waiting for the device.  So one thread looks at the batch's control block and, in
+// that case only, launches the sort path's kernels itself, in order, into the tail-launch stream: they run
+// after this one-thread kernel and before the next kernel of the host's stream (a parent grid is complete
+// only when its children are), which is the batch's finish kernel.  A batch in issue order pays one empty
+// launch instead of thirteen.
+struct SortChain {
+    const hbf_access_t *acc; uint64_t n; const RangeSnap *ranges; const ModelParams *mp_dev; BatchCtrl *ctrl; DevState *state;
+    uint64_t *keys0, *keys1; uint32_t *idx0, *idx1, *hist, *desc0, *desc1; void *scan_desc;
+    uint8_t *status; int64_t *completion, *stall; const int64_t *busy; int64_t *busy_stage; hbf_die_stats_t *stats_stage;
+    const unsigned long long *claim_limit; uint32_t *die_claims;
+    uint32_t n_queues, n_dies; uint64_t desc_words, scan_words;
+    unsigned cls_grid, hist_grid, sort_grid, scan_grid;
+};
+
+__global__ void k_zero_words(uint32_t *p, uint64_t words) {
+    for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < words; i += (uint64_t)gridDim.x * blockDim.x) p[i] = 0u;
+}
+
+__global__ void k_sort_fallback(const __grid_constant__ SortChain c) {
+    if (c.ctrl->skip || !c.ctrl->run_sort) return;           // served in issue order, or refused: nothing to do
+    cudaStream_t st = cudaStreamTailLaunch;
+    k_begin<<<1, 1024, 0, st>>>(c.ctrl, c.state, c.busy, c.busy_stage, c.stats_stage, c.hist, c.n_queues, c.n_dies, 1, 1, c.die_claims);
+    k_zero_words<<<(unsigned)min((unsigned long long)((c.desc_words + 1023) / 1024), 592ull), 1024, 0, st>>>(c.desc0, c.desc_words);
+    k_zero_words<<<(unsigned)min((unsigned long long)((c.scan_words + 1023) / 1024), 592ull), 1024, 0, st>>>((uint32_t *)c.scan_desc, c.scan_words);
+    k_classify<<<c.cls_grid, kClsThreads, 0, st>>>(c.acc, c.n, c.ranges, c.mp_dev, c.ctrl, c.keys0, c.status, c.completion, c.stall);
+    k_plan<<<1, 32, 0, st>>>(c.ctrl, 0);
+    k_hist<<<c.hist_grid, kHistThreads, 0, st>>>(c.keys0, c.n, c.ctrl, c.hist);
+    for (int p = 0; p < kMaxPasses; ++p)
+        k_sort_pass<<<c.sort_grid, kSortThreads, kSortSmem, st>>>(p, c.n, c.ctrl, c.state, c.hist, c.keys0, c.keys1, c.idx0, c.idx1, c.desc0, c.desc1);
+    k_scan<<<c.scan_grid, kScanThreads, 0, st>>>(c.acc, c.n, c.ranges, c.mp_dev, c.ctrl, c.state, c.keys0, c.keys1, c.idx0, c.idx1,
+                                                 (ScanDesc *)c.scan_desc, c.busy, c.busy_stage, c.stats_stage, c.completion, c.stall,
+                                                 c.claim_limit, c.die_claims);
+}
+
+static cudaError_t launch_sort_fallback(const SubmitArgs &a, cudaStream_t st) {
+    const uint64_t n = a.n;
+    const uint64_t sort_tiles = (n + kSortTile - 1) / kSortTile, scan_tiles = (n + kScanTile - 1) / kScanTile;
+    cudaError_t e = ensure_dyn_smem((const void *)k_sort_pass, kSortSmem);   // (an attribute of the kernel: device-side launches use it too)
+    if (e != cudaSuccess) return e;
+    SortChain c{};
+    c.acc = a.acc; c.n = n; c.ranges = a.ranges; c.mp_dev = a.mp_dev; c.ctrl = a.ctrl; c.state = a.state;
+    c.keys0 = a.ws.keys[0]; c.keys1 = a.ws.keys[1]; c.idx0 = a.ws.idx[0]; c.idx1 = a.ws.idx[1]; c.hist = a.ws.hist;
+    c.desc0 = a.ws.sort_desc[0]; c.desc1 = a.ws.sort_desc[1]; c.scan_desc = a.ws.scan_desc;
+    c.status = a.status; c.completion = a.completion; c.stall = a.stall; c.busy = a.busy; c.busy_stage = a.busy_stage;
+    c.stats_stage = a.stats_stage; c.claim_limit = a.claim_limit; c.die_claims = a.die_claims;
+    c.n_queues = a.mp.n_queues; c.n_dies = a.mp.n_dies;
+    c.desc_words = sort_tiles * kRadix; c.scan_words = scan_tiles * (sizeof(ScanDesc) / 4);
+    c.cls_grid = (unsigned)std::min<uint64_t>((n + kClsTile - 1) / kClsTile, (uint64_t)a.sm_count * 8);
+    c.hist_grid = (unsigned)std::min<uint64_t>((n + kHistThreads * 8 - 1) / (kHistThreads * 8), (uint64_t)a.sm_count * 4);
+    c.sort_grid = (unsigned)std::min<uint64_t>(sort_tiles, (uint64_t)a.sm_count * 3);
+    c.scan_grid = (unsigned)std::min<uint64_t>(scan_tiles, (uint64_t)a.sm_count * 8);
+    k_sort_fallback<<<1, 1, 0, st>>>(c);
+    g_kernel_launches += 1;
+    return cudaGetLastError();
+}
+
 // Kernel order of one batch.  AUTO: begin, the in-order kernels (they serve the batch when its records
-// arrive in non-decreasing issue order), a second begin and the sort kernels (they do nothing unless the
-// in-order attempt handed the batch over), finish.  SORT / SORT_FULL: begin, sort kernels, finish.
+// arrive in non-decreasing issue order), one thread that launches the sort kernels from the device if the
+// in-order attempt handed the batch over, finish.  SORT / SORT_FULL: begin, sort kernels, finish.
 cudaError_t launch_submit(const SubmitArgs &a, cudaStream_t st) {
     const uint64_t n = a.n;
     auto mark = [&](int k) { if (a.ev) cudaEventRecord(a.ev[k], st); };
@@ -1029,15 +1089,14 @@ cudaError_t launch_submit(const SubmitArgs &a, cudaStream_t st) {
             if (e != cudaSuccess) return e;
             mark(8);
             if (sort_kernels) {
-                k_begin<<<1, 1024, 0, st>>>(a.ctrl, a.state, a.busy, a.busy_stage, a.stats_stage, a.ws.hist, a.mp.n_queues,
-                                           a.mp.n_dies, 1, 1, a.die_claims);
-                g_kernel_launches += 1;
+                e = launch_sort_fallback(a, st);
+                if (e != cudaSuccess) return e;
             }
-        }
-        if (sort_kernels) {
+            mark(1); mark(2); mark(3); mark(4);
+        } else {
             cudaError_t e = launch_sort_path(a, st);
             if (e != cudaSuccess) return e;
-        } else { mark(1); mark(2); mark(3); mark(4); }
+        }
     } else {
         mark(1); mark(2); mark(3); mark(4);
     }
