@@ -68,6 +68,7 @@ struct BatchCtrl {
     uint32_t inorder_used;               // the in-order path served this batch
     uint32_t run_sort;                   // the sort path has to serve this batch
     uint32_t pad1;
+    uint32_t role_count[2];              // in-order serve pass: tiles handed out so far, per size class
     uint32_t tile_counter[kMaxPasses + 2];
     long long modeled_ns, service_ns, max_completion_ns;
     SortPlan plan;
@@ -138,8 +139,17 @@ inline uint64_t inorder_tiles_bound(uint64_t n) {
 size_t workspace_layout(uint64_t n, uint32_t n_queues, Workspace *ws, void *base, int with_bus = 0);
 // channel bus as a second queued stage, after launch_submit on the same arguments (bc: a control block of its own)
 cudaError_t launch_bus_stage(const SubmitArgs &a, BatchCtrl *bc, int64_t *bus_busy, cudaStream_t st);
-// tile size (records) of the in-order path for a batch of n on a device with sm_count SMs
-uint64_t inorder_tile_records(uint64_t n, int sm_count);
+// How the in-order path cuts a batch of n records into contiguous tiles: n_big tiles of `big` records, then tiles of
+// `small` records (the last one ragged).  All sizes are multiples of kInTileQuantum.  n_big == 0: one size only.
+struct InTileMap { uint64_t n; uint32_t n_tiles, n_big; uint32_t big, small; };
+__host__ __device__ inline uint64_t tile_first(const InTileMap &m, uint32_t t) {
+    return t < m.n_big ? (uint64_t)t * m.big : (uint64_t)m.n_big * m.big + (uint64_t)(t - m.n_big) * m.small;
+}
+__host__ __device__ inline uint64_t tile_last(const InTileMap &m, uint32_t t) {      // one past the tile's last record
+    const uint64_t e = tile_first(m, t) + (t < m.n_big ? m.big : m.small);
+    return e < m.n ? e : m.n;
+}
+InTileMap inorder_tile_map(uint64_t n, int sm_count);
 size_t inorder_head_bytes(uint64_t tiles, uint32_t n_queues);
 size_t inorder_serve_smem(uint32_t n_dies);
 cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st);

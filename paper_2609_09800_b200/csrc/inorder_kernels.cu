@@ -215,7 +215,7 @@ __device__ __forceinline__ void row_wait2(int id, int64_t m, long long s8, const
 // claims per die.
 template <bool RESERVE, bool DEBT>
 __global__ void __launch_bounds__(kInThreads, kInBlocksPerSM)
-k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_records, const RangeSnap *__restrict__ ranges_g,
+k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, const __grid_constant__ InTileMap tmap, const RangeSnap *__restrict__ ranges_g,
                 const __grid_constant__ ModelParams mp_arg, const __grid_constant__ FastRange fast_arg, BatchCtrl *ctrl, uint8_t *__restrict__ status, int64_t *__restrict__ in_agg,
                 hbf_die_stats_t *stats_stage, int64_t *__restrict__ completion, int64_t *__restrict__ stall,
                 const int64_t *__restrict__ in_bin, InTile *in_tile, InHead *__restrict__ in_head, uint8_t *__restrict__ in_headcnt,
@@ -250,9 +250,30 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
     uint32_t *st_nr = st_bp_hi + n_dies, *st_np = st_nr + n_dies;
     uint32_t *st_claims = st_np + n_dies;                 // refresh quanta claimed on each die (claims variant)
 
-    const uint32_t tile = blockIdx.x;
-    const uint64_t tile_begin = (uint64_t)tile * tile_records;
-    const uint64_t tile_end = min(n, tile_begin + tile_records);
+    // Which tile this block serves.  Two blocks share an SM, and the hardware favours the one in the lower warp slots: with
+    // equal tiles it finishes about 12 % earlier (measured) and the pass lasts as long as the other one.  So the tiles come in
+    // two sizes; a block reads off its warp slot which kind of block it is and takes the next tile of the matching size (or,
+    // should one size run out, of the other: every tile is handed out exactly once whatever the slots say).
+    __shared__ uint32_t s_tile_id;
+    if (!RESERVE) {
+        if (tid == 0) {
+            uint32_t t = blockIdx.x;
+            if (tmap.n_big != 0u) {
+                unsigned slot;
+                asm volatile("mov.u32 %0, %%warpid;" : "=r"(slot));
+                const uint32_t late = slot >= 4u ? 1u : 0u;   // warp 0 of the block that came second sits past the first four slots
+                const uint32_t have[2] = {tmap.n_big, tmap.n_tiles - tmap.n_big};
+                uint32_t k = atomicAdd(&ctrl->role_count[late], 1u);
+                if (k < have[late]) t = late ? tmap.n_big + k : k;
+                else { k = atomicAdd(&ctrl->role_count[1u - late], 1u); t = late ? k : tmap.n_big + k; }
+            }
+            s_tile_id = t;
+        }
+        __syncthreads();
+    }
+    const uint32_t tile = RESERVE ? blockIdx.x : s_tile_id;
+    const uint64_t tile_begin = tile_first(tmap, tile);
+    const uint64_t tile_end = tile_last(tmap, tile);
 
     for (uint32_t i = tid; i < kInMaxQueues; i += kInThreads) qst[i] = make_longlong2(kNegInf, 0);
     if (RESERVE) {
@@ -260,7 +281,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
         for (uint32_t q = tid; q < R; q += kInThreads) qst[q].x = in_bin[(uint64_t)blockIdx.x * R + q];
     } else {
         for (uint32_t d = tid; d < n_dies * 7u; d += kInThreads) st_br_lo[d] = 0u;
-        if (blockIdx.x == 0) {                               // the first tile knows its entering state: it is served exactly
+        if (tile == 0u) {                                    // the first tile knows its entering state: it is served exactly
             __syncthreads();
             for (uint32_t q = tid; q < R; q += kInThreads) qst[q].x = busy[q];
         }
@@ -301,7 +322,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
             const uint32_t j = (turn * K + u) * 32u + (uint32_t)lane;
             if (j < tile_len) {
                 const uint64_t *rec = reinterpret_cast<const uint64_t *>(acc_t + j);
-                nx_addr[u] = __ldg(rec); nx_issue[u] = __ldg(rec + 1); nx_bf[u] = __ldg(rec + 2);
+                nx_addr[u] = __ldcs(rec); nx_issue[u] = __ldcs(rec + 1); nx_bf[u] = __ldcs(rec + 2);   // read once: streaming loads
                 if (!RESERVE) nx_prev[u] = (j > 0u || !first_tile) ? (int64_t)__ldg(rec - 2) : INT64_MIN;
             }
         }
@@ -459,7 +480,9 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_
                         if (last[u] && c1[u] != c0[u] && c1[u] == (uint32_t)kInHead) atomicAdd(&s_heads_full, 1u);
                     }
                 }
-                completion_t[i[u]] = done; stall_t[i[u]] = st;
+                // results are written once and not read again by this pass: streaming stores
+                __stcs(reinterpret_cast<long long *>(completion_t + i[u]), (long long)done);
+                __stcs(reinterpret_cast<long long *>(stall_t + i[u]), (long long)st);
             }
         }
         };
@@ -628,7 +651,7 @@ static_assert(kInQidPrefix % kInStrQChunk == 0 && kInStrQItems == 32, "a thread'
 
 template <bool DEBT>
 __global__ void __launch_bounds__(kInStrThreads, 2)
-k_inorder_fixstraggle(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t tile_records,
+k_inorder_fixstraggle(const hbf_access_t *__restrict__ acc, uint64_t n, const __grid_constant__ InTileMap tmap,
                       const RangeSnap *__restrict__ ranges_g, const __grid_constant__ ModelParams mp_arg,
                       const __grid_constant__ FastRange fast_arg, BatchCtrl *ctrl,
                       const int64_t *__restrict__ in_bin, const InHead *__restrict__ in_head,
@@ -715,7 +738,7 @@ k_inorder_fixstraggle(const hbf_access_t *__restrict__ acc, uint64_t n, uint64_t
     const uint64_t claim_limit = DEBT ? *claim_limit_p : 0ull;     // as in the serve pass
     const int64_t quantum_ns = !DEBT ? 0 : q_ppm == 1000000 ? mp_arg.t_read_ns + mp_arg.t_prog_ns
         : (int64_t)div64((uint64_t)(mp_arg.t_read_ns + mp_arg.t_prog_ns) * 1000000ull + (uint64_t)q_ppm - 1ull, div_q);
-    const uint64_t tile_begin = (uint64_t)tile * tile_records, tile_end = min(n, tile_begin + tile_records);
+    const uint64_t tile_begin = tile_first(tmap, tile), tile_end = tile_last(tmap, tile);
     const uint32_t tile_len = (uint32_t)(tile_end - tile_begin);       // offsets inside a tile fit 32 bits
     const hbf_access_t *acc_t = acc + tile_begin;
     const uint4 *qid_t = reinterpret_cast<const uint4 *>(in_qid + (uint64_t)tile * qid_stride);
@@ -901,11 +924,32 @@ __global__ void k_inorder_total(BatchCtrl *ctrl, const InTile *__restrict__ in_t
     if ((threadIdx.x & 31) == 0 && tot) atomicAdd((unsigned long long *)&ctrl->modeled_ns, (unsigned long long)tot);
 }
 
-uint64_t inorder_tile_records(uint64_t n, int sm_count) {
-    const uint64_t want_tiles = std::min<uint64_t>(kInMaxTiles, (uint64_t)std::max(1, sm_count) * kInBlocksPerSM);   // one wave of resident blocks
-    uint64_t t = (n + want_tiles - 1) / want_tiles;
-    t = (t + kInTileQuantum - 1) / kInTileQuantum * kInTileQuantum;
-    return std::max<uint64_t>(t, kInTileQuantum);
+#ifndef HBF_IN_SKEW_PERMILLE
+#define HBF_IN_SKEW_PERMILLE 60
+#endif
+// One wave of resident blocks: as many tiles as the device holds serve blocks.  When the batch is large enough to fill
+// that wave, the tiles of the blocks that the hardware favours (one per SM) are larger by the skew, the others smaller,
+// so that both blocks of an SM finish together.
+InTileMap inorder_tile_map(uint64_t n, int sm_count) {
+    InTileMap m{};
+    m.n = n;
+    const uint64_t sms = (uint64_t)std::max(1, sm_count);
+    const uint64_t want_tiles = std::min<uint64_t>(kInMaxTiles, sms * kInBlocksPerSM);
+    auto round_up = [](uint64_t v) { return std::max<uint64_t>((v + kInTileQuantum - 1) / kInTileQuantum * kInTileQuantum, kInTileQuantum); };
+    const uint64_t even = round_up((n + want_tiles - 1) / want_tiles);
+    if (kInBlocksPerSM == 2 && want_tiles == 2 * sms && even >= 64 * kInTileQuantum && HBF_IN_SKEW_PERMILLE > 0) {
+        const uint64_t big = round_up(even * (1000 + HBF_IN_SKEW_PERMILLE) / 1000);
+        if (big * sms < n) {
+            const uint64_t rest = n - big * sms;
+            const uint64_t small = round_up((rest + sms - 1) / sms);
+            m.n_big = (uint32_t)sms; m.big = (uint32_t)big; m.small = (uint32_t)small;
+            m.n_tiles = (uint32_t)(sms + (rest + small - 1) / small);
+            return m;
+        }
+    }
+    m.n_big = 0; m.big = m.small = (uint32_t)even;
+    m.n_tiles = (uint32_t)((n + even - 1) / even);
+    return m;
 }
 
 // dynamic shared memory of the serve kernel: the per-queue state and the per-die counters
@@ -916,8 +960,9 @@ size_t inorder_head_bytes(uint64_t tiles, uint32_t n_queues) { return tiles * n_
 
 cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st) {
     const uint64_t n = a.n;
-    const uint64_t tile_records = inorder_tile_records(n, a.sm_count);
-    const unsigned n_tiles = (unsigned)((n + tile_records - 1) / tile_records);
+    const InTileMap tmap = inorder_tile_map(n, a.sm_count);
+    const unsigned n_tiles = tmap.n_tiles;
+    const uint64_t tile_records = std::max(tmap.big, tmap.small);
     if (n_tiles > inorder_tiles_bound(n)) return cudaErrorInvalidValue;       // the workspace is carved for that many
     const uint32_t R = a.mp.n_queues, nd = a.mp.n_dies;
     const size_t smem_serve = inorder_serve_smem(nd), smem_str = inorder_straggle_smem();
@@ -933,16 +978,12 @@ cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st) {
     InTile *tiles = reinterpret_cast<InTile *>(a.ws.in_tile);
     InHead *heads = reinterpret_cast<InHead *>(a.ws.in_head);
     const bool debt = a.claim_limit != nullptr;              // retention on: the kernels that apply the claims
-#ifdef HBF_DBG_NOQID
-    const uint32_t qid_stride = 0;
-#else
     const uint32_t qid_stride = (uint32_t)std::min<uint64_t>(tile_records, kInQidPrefix);
-#endif
     if ((uint64_t)n_tiles * qid_stride > inorder_qid_entries(n)) return cudaErrorInvalidValue;
     auto serve = [&](bool reserve) {
         auto k = reserve ? (debt ? k_inorder_serve<true, true> : k_inorder_serve<true, false>)
                          : (debt ? k_inorder_serve<false, true> : k_inorder_serve<false, false>);
-        k<<<n_tiles, kInThreads, smem_serve, st>>>(a.acc, n, tile_records, a.ranges, a.mp, a.fast, a.ctrl, a.status, a.ws.in_agg,
+        k<<<n_tiles, kInThreads, smem_serve, st>>>(a.acc, n, tmap, a.ranges, a.mp, a.fast, a.ctrl, a.status, a.ws.in_agg,
                                                    a.stats_stage, a.completion, a.stall, a.ws.in_bin, tiles, heads, a.ws.in_headcnt,
                                                    a.busy, a.claim_limit, a.die_claims, debt ? *a.ret : RetDev{}, a.ws.in_qid, qid_stride);
     };
@@ -950,7 +991,7 @@ cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st) {
     k_inorder_scan<<<(R + kInScanQueues - 1) / kInScanQueues, dim3(kInScanQueues, kInScanChunks), 0, st>>>(
         a.ctrl, a.mp_dev, n_tiles, a.ws.in_agg, a.ws.in_bin, a.busy, a.busy_stage, a.stats_stage, a.path == HBF_PATH_INORDER ? 1 : 0);
     (debt ? k_inorder_fixstraggle<true> : k_inorder_fixstraggle<false>)<<<n_tiles, kInStrThreads, smem_str, st>>>(
-        a.acc, n, tile_records, a.ranges, a.mp, a.fast, a.ctrl, a.ws.in_bin, heads, a.ws.in_headcnt, a.completion, a.stall, tiles,
+        a.acc, n, tmap, a.ranges, a.mp, a.fast, a.ctrl, a.ws.in_bin, heads, a.ws.in_headcnt, a.completion, a.stall, tiles,
         a.claim_limit, a.ws.in_qid, qid_stride);
     serve(true);
     k_inorder_total<<<1, 256, 0, st>>>(a.ctrl, tiles, n_tiles);
