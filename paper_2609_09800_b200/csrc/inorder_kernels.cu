@@ -640,12 +640,13 @@ constexpr int kInStrQItems = 32;                          // records per thread 
 constexpr int kInStrQChunk = kInStrThreads * kInStrQItems;
 constexpr int kInStrItems = 8;                            // and past it, where the queue is decoded from the record
 constexpr int kInStrChunk = kInStrThreads * kInStrItems;
-constexpr int kInStrKeep = 2048;                          // kept records served at a time (a chunk with more is served in windows)
+constexpr int kInStrKeep = 1024;                          // kept records served at a time (a chunk with more is served in windows)
+constexpr int kInStrMaxStragglers = 128;                   // a tile with as many is served again whole instead
+constexpr int kInStrList = 32;                            // records of one queue in a window that its list holds (more: the window is scanned)
 constexpr int kInStrCells = kInStrItems * kInStrWarps;    // (item, warp) cells of the kept-record counts, decode path
 constexpr int kInStrCellsPerLane = kInStrCells / 32;
 constexpr int kInStrQueuesPerThread = (kInMaxQueues + kInStrThreads - 1) / kInStrThreads;
 static_assert(kInStrCells % 32 == 0, "the offset scan gives every lane the same number of cells");
-static_assert(kInStrQueuesPerThread % 2 == 0, "the fix-up takes a thread's queues two at a time");
 static_assert(kInStrQChunk <= 65536, "a kept record's position in its chunk is stored in 16 bits");
 static_assert(kInQidPrefix % kInStrQChunk == 0 && kInStrQItems == 32, "a thread's 32 queue numbers are four 16-byte loads");
 
@@ -677,60 +678,84 @@ k_inorder_fixstraggle(const hbf_access_t *__restrict__ acc, uint64_t n, const __
     longlong2 *ent_as = reinterpret_cast<longlong2 *>(Ba + kInMaxQueues);      // [keep] kept records, batch order: issue time, service time
     uint2 *ent_pq = reinterpret_cast<uint2 *>(ent_as + kInStrKeep);            //        transfer | op << 31, queue | position << 16
     uint16_t *oq = reinterpret_cast<uint16_t *>(ent_pq + kInStrKeep);          // [stragglers] their queues
-    uint8_t *open = reinterpret_cast<uint8_t *>(oq + kInMaxQueues);            // [queues] 1: straggler, runs have not met
-    if (tid == 0) { mp = mp_arg; fast_range = fast_arg; s_stragglers = 0u; s_red[0] = 0; s_red[1] = INT64_MIN; }
+    uint8_t *open = reinterpret_cast<uint8_t *>(oq + kInMaxQueues);            // [queues] 0, or 1 + the queue's place in oq while its runs have not met
+    uint16_t *lst = reinterpret_cast<uint16_t *>(open + kInMaxQueues);         // [stragglers][kInStrList] the window's records of each queue
+    uint32_t *lcount = reinterpret_cast<uint32_t *>(lst + kInStrMaxStragglers * kInStrList);   // [stragglers] how many
+    __shared__ uint32_t s_overflow;
+    if (tid < kInStrMaxStragglers) lcount[tid] = 0u;
+    if (tid == 0) { mp = mp_arg; fast_range = fast_arg; s_stragglers = 0u; s_total = 0u; s_overflow = 0u; s_red[0] = 0; s_red[1] = INT64_MIN; }
     __syncthreads();
 
-    // ---- fix-up: this thread's queues of the tile (their loads are issued side by side) ------------------------
+    // ---- fix-up, first entry: this thread's queues of the tile, their loads issued side by side.  Four queues in five
+    // are idle when their first access of the tile arrives: they are done here.  The others go on a list.
     long long dstall = 0, max_c = INT64_MIN;
+    uint16_t *deep = reinterpret_cast<uint16_t *>(ent_pq);   // [queues] the list (the record windows are not in use yet)
     {
-        constexpr int kRound = 2;                            // queues whose loads are in flight together
-        for (int k0 = 0; k0 < kInStrQueuesPerThread; k0 += kRound) {
-            uint32_t c[kRound]; int64_t Bin[kRound];
-            InHead e0[kRound], e1[kRound];
+        uint32_t c[kInStrQueuesPerThread]; int64_t Bin[kInStrQueuesPerThread];
+        InHead e0[kInStrQueuesPerThread];
 #pragma unroll
-            for (int k = 0; k < kRound; ++k) {
-                const uint32_t q = (uint32_t)((k0 + k) * kInStrThreads + tid);
-                c[k] = 0u; Bin[k] = kNegInf;
-                if (q < R) { c[k] = in_headcnt[(uint64_t)tile * R + q]; Bin[k] = in_bin[(uint64_t)tile * R + q]; }
+        for (int k = 0; k < kInStrQueuesPerThread; ++k) {
+            const uint32_t q = (uint32_t)(k * kInStrThreads + tid);
+            c[k] = 0u; Bin[k] = kNegInf;
+            if (q < R) { c[k] = in_headcnt[(uint64_t)tile * R + q]; Bin[k] = in_bin[(uint64_t)tile * R + q]; }
+        }
+#pragma unroll
+        for (int k = 0; k < kInStrQueuesPerThread; ++k)
+            if (c[k] > 0u) e0[k] = in_head[((uint64_t)tile * R + (uint32_t)(k * kInStrThreads + tid)) * kInHead];
+#pragma unroll
+        for (int k = 0; k < kInStrQueuesPerThread; ++k) {
+            const uint32_t q = (uint32_t)(k * kInStrThreads + tid);
+            if (q < kInMaxQueues) { open[q] = 0; Ba[q] = kNegInf; Bt[q] = Bin[k]; }
+            if (c[k] == 0u) continue;
+            if (Bin[k] <= e0[k].m - e0[k].s) continue;       // idle on arrival: the as-if run was right from the start
+            deep[atomicAdd(&s_total, 1u)] = (uint16_t)q;
+        }
+    }
+    __syncthreads();
+    // ---- fix-up, the rest: one thread per listed queue walks its head entries (fetched in two rounds) from the true
+    // entering busy-until until an access arrives on an idle queue
+    {
+        const uint32_t n_deep = s_total;
+        for (uint32_t d = (uint32_t)tid; d < n_deep; d += kInStrThreads) {
+            const uint32_t q = deep[d];
+            const uint64_t idx = (uint64_t)tile * R + q;
+            const uint32_t c = in_headcnt[idx];
+            const InHead *h = in_head + idx * kInHead;
+            FixRun f; f.B = Bt[q]; f.Bs = kNegInf; f.dstall = 0; f.max_c = INT64_MIN; f.settled = false;
+            InHead g[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) if ((uint32_t)j < c) g[j] = h[j];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) if ((uint32_t)j < c) fix_entry(f, g[j], completion, stall);
+            if (!f.settled && c > 4u) {
+#pragma unroll
+                for (int j = 4; j < kInHead; ++j) if ((uint32_t)j < c) g[j - 4] = h[j];
+#pragma unroll
+                for (int j = 4; j < kInHead; ++j) if ((uint32_t)j < c) fix_entry(f, g[j - 4], completion, stall);
             }
-#pragma unroll
-            for (int k = 0; k < kRound; ++k) {
-                const InHead *h = in_head + ((uint64_t)tile * R + (uint32_t)((k0 + k) * kInStrThreads + tid)) * kInHead;
-                if (c[k] > 0u) e0[k] = h[0];
-                if (c[k] > 1u) e1[k] = h[1];
-            }
-#pragma unroll
-            for (int k = 0; k < kRound; ++k) {
-                const uint32_t q = (uint32_t)((k0 + k) * kInStrThreads + tid);
-                if (q < kInMaxQueues) { open[q] = 0; Ba[q] = kNegInf; Bt[q] = kNegInf; }
-                if (c[k] == 0u) continue;
-                FixRun f; f.B = Bin[k]; f.Bs = kNegInf; f.dstall = 0; f.max_c = INT64_MIN; f.settled = false;
-                fix_entry(f, e0[k], completion, stall);
-                if (c[k] > 1u) fix_entry(f, e1[k], completion, stall);
-                if (!f.settled && c[k] > 2u) {
-                    const InHead *h = in_head + ((uint64_t)tile * R + q) * kInHead;
-                    for (uint32_t j = 2; j < c[k]; ++j) fix_entry(f, h[j], completion, stall);
-                }
-                max_c = max(max_c, f.max_c);                 // (true completions: valid whoever writes them last)
-                if (!f.settled && c[k] == (uint32_t)kInHead) {
-                    // still backlogged after its head entries: the loop below serves this queue again from the tile's
-                    // start and accounts for all of its corrections
-                    open[q] = 1; Bt[q] = Bin[k];
-                    oq[atomicAdd(&s_stragglers, 1u)] = (uint16_t)q;
-                } else {
-                    dstall += f.dstall;
-                }
+            max_c = max(max_c, f.max_c);                     // (true completions: valid whoever writes them last)
+            if (!f.settled && c == (uint32_t)kInHead) {
+                // still backlogged after its head entries: the loop below serves this queue again from the tile's
+                // start (Bt[q] still holds the entering value) and accounts for all of its corrections
+                const uint32_t place = atomicAdd(&s_stragglers, 1u);
+                oq[place] = (uint16_t)q;
+                open[q] = (uint8_t)min(place + 1u, 255u);   // (a tile with more than kInStrMaxStragglers - 1 of them leaves below)
+            } else {
+                dstall += f.dstall;
             }
         }
     }
     __syncthreads();
     const uint32_t stragglers = s_stragglers;
-    if (stragglers >= max(8u, R / 16u)) {                    // many queues far behind: the re-serve pass takes the whole tile
+    if (stragglers >= min(max(8u, R / 16u), (uint32_t)kInStrMaxStragglers)) {   // many queues far behind: the re-serve pass takes the whole tile
         if (tid == 0) in_tile[tile].reserve = 1u;
         return;
     }
+#ifdef HBF_DBG_FIXONLY
+    if (false) {
+#else
     if (stragglers > 0u) {
+#endif
     const int64_t q_ppm = ctrl->q_ppm;
     const Div64 div_q = ctrl->div_q;
     const bool one_range = fast_arg.on != 0u && mp_arg.pow2_geom != 0u;
@@ -754,17 +779,36 @@ k_inorder_fixstraggle(const hbf_access_t *__restrict__ acc, uint64_t n, const __
             for (int k = 0; k < kInStrQItems / 8; ++k) nx_q[k] = __ldg(qid_t + (cb >> 3) + tid * (kInStrQItems / 8) + k);
         }
     };
-    // a kept record: its terms are computed here, once, and it takes its place in the window of kept records
-    auto put = [&](uint32_t cb, uint32_t e, uint32_t slot) {
-        const uint64_t *rec = reinterpret_cast<const uint64_t *>(acc_t + cb + e);
-        const uint64_t addr = __ldg(rec);
-        const int64_t issue = (int64_t)__ldg(rec + 1);
-        const uint64_t bf = __ldg(rec + 2);
-        Served v = fast_terms ? serve_terms_fast(fast_range, mp, addr, issue, bf)
-                              : serve_terms(rs, mp, addr, issue, bf, q_ppm, div_q, ignored, 33);
-        if (DEBT && tile_begin + cb + e < claim_limit) v.s += quantum_ns;
-        ent_as[slot] = make_longlong2(issue, v.s);
-        ent_pq[slot] = make_uint2(v.xfer | (v.op << 31), v.queue | (e << 16));
+    // the kept records of a window, one per thread (their positions in the chunk are in the window already): the records are
+    // fetched side by side, their terms computed once, and they take their places in the window
+    constexpr int kPerThread = kInStrKeep / kInStrThreads;
+    auto fill_window = [&](uint32_t cb, uint32_t wn) {
+        uint64_t r_addr[kPerThread], r_bf[kPerThread]; int64_t r_issue[kPerThread]; uint32_t r_e[kPerThread];
+#pragma unroll
+        for (int k = 0; k < kPerThread; ++k) {
+            const uint32_t slot = (uint32_t)(k * kInStrThreads + tid);
+            if (slot < wn) {
+                r_e[k] = ent_pq[slot].y;
+                const uint64_t *rec = reinterpret_cast<const uint64_t *>(acc_t + cb + r_e[k]);
+                r_addr[k] = __ldg(rec); r_issue[k] = (int64_t)__ldg(rec + 1); r_bf[k] = __ldg(rec + 2);
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < kPerThread; ++k) {
+            const uint32_t slot = (uint32_t)(k * kInStrThreads + tid);
+            if (slot < wn) {
+                Served v = fast_terms ? serve_terms_fast(fast_range, mp, r_addr[k], r_issue[k], r_bf[k])
+                                      : serve_terms(rs, mp, r_addr[k], r_issue[k], r_bf[k], q_ppm, div_q, ignored, 33);
+                if (DEBT && tile_begin + cb + r_e[k] < claim_limit) v.s += quantum_ns;
+                ent_as[slot] = make_longlong2(r_issue[k], v.s);
+                ent_pq[slot] = make_uint2(v.xfer | (v.op << 31), v.queue | (r_e[k] << 16));
+                const uint32_t place = open[v.queue];         // (0: the queue's runs met in an earlier window of this chunk)
+                if (place) {
+                    const uint32_t at = atomicAdd(&lcount[place - 1u], 1u);
+                    if (at < (uint32_t)kInStrList) lst[(place - 1u) * kInStrList + at] = (uint16_t)slot; else s_overflow = 1u;
+                }
+            }
+        }
     };
     fetch(0u);
 
@@ -855,47 +899,81 @@ k_inorder_fixstraggle(const hbf_access_t *__restrict__ acc, uint64_t n, const __
                     const uint32_t j = (uint32_t)__ffs((int)m) - 1u;
                     m &= m - 1u;
                     const uint32_t slot = first + (uint32_t)__popc(keep & ((1u << j) - 1u)) - wb;   // (wraps below the window)
-                    if (slot < wn) put(cb, (uint32_t)(tid * kInStrQItems) + j, slot);
+                    if (slot < wn) ent_pq[slot].y = (uint32_t)(tid * kInStrQItems) + j;
                 }
             } else {
 #pragma unroll
                 for (int j = 0; j < kInStrItems; ++j)
-                    if ((keep >> j) & 1u) { const uint32_t slot = rk[j] - wb; if (slot < wn) put(cb, (uint32_t)(j * kInStrThreads + tid), slot); }
+                    if ((keep >> j) & 1u) { const uint32_t slot = rk[j] - wb; if (slot < wn) ent_pq[slot].y = (uint32_t)(j * kInStrThreads + tid); }
             }
             __syncthreads();
-            // one warp per straggling queue scans the window 32 records at a time (they are in batch order) and re-serves
-            // its own in order; every lane carries the two runs, lane 0 writes
-            for (uint32_t t = (uint32_t)warp; t < stragglers; t += kInStrWarps) {
-                const uint32_t q = oq[t];
-                if (!open[q]) continue;
-                int64_t BT = Bt[q], BA = Ba[q];
-                for (uint32_t k0 = 0; k0 < wn; k0 += 32u) {
-                    const uint32_t k = k0 + (uint32_t)lane;
-                    unsigned hits = __ballot_sync(0xffffffffu, k < wn && (ent_pq[min(k, wn - 1u)].y & 0xffffu) == q);
-                    while (hits) {
-                        const uint32_t kk = k0 + (uint32_t)__ffs((int)hits) - 1u;
-                        hits &= hits - 1u;
-                        const uint2 pq = ent_pq[kk];
-                        const longlong2 as = ent_as[kk];
-                        const int64_t xfer = (int64_t)(pq.x & 0x7fffffffu);
-                        const bool op = (pq.x >> 31) != 0u;
-                        const int64_t a = as.x + (op ? xfer : 0);
-                        BT = max(a, BT) + as.y; BA = max(a, BA) + as.y;
-                        if (BT != BA && lane == 0) {          // the serve pass wrote BA + post
-                            const uint64_t i = min(tile_begin + cb + (pq.y >> 16), tile_end - 1);
-                            const int64_t done = BT + (op ? 0 : xfer);
-                            completion[i] = done; stall[i] = done - as.x;
-                            dstall += BT - BA; max_c = max(max_c, (long long)done);
-                        }
-                    }
+            fill_window(cb, wn);
+            __syncthreads();
+            // Every straggling queue has the window's records of its own in a short list (in the order the threads happened
+            // to append them): one thread per queue sorts its list by position (the window is in batch order) and re-serves
+            // them, carrying the two runs.
+            auto reserve_one = [&](uint32_t kk, int64_t &BT, int64_t &BA, bool writer) {
+                const uint2 pq = ent_pq[kk];
+                const longlong2 as = ent_as[kk];
+                const int64_t xfer = (int64_t)(pq.x & 0x7fffffffu);
+                const bool op = (pq.x >> 31) != 0u;
+                const int64_t a = as.x + (op ? xfer : 0);
+                BT = max(a, BT) + as.y; BA = max(a, BA) + as.y;
+                if (BT != BA && writer) {                     // the serve pass wrote BA + post
+                    const uint64_t i = min(tile_begin + cb + (pq.y >> 16), tile_end - 1);
+                    const int64_t done = BT + (op ? 0 : xfer);
+                    completion[i] = done; stall[i] = done - as.x;
+                    dstall += BT - BA; max_c = max(max_c, (long long)done);
                 }
-                if (lane == 0) {
+            };
+            if (!s_overflow) {
+                for (uint32_t t = (uint32_t)tid; t < stragglers; t += kInStrThreads) {
+                    const uint32_t q = oq[t];
+                    const uint32_t cnt = lcount[t];
+                    lcount[t] = 0u;
+                    if (!open[q] || cnt == 0u) continue;
+                    uint16_t *mine = lst + t * kInStrList;
+                    for (uint32_t i = 1; i < cnt; ++i) {      // a handful of entries: insertion sort
+                        const uint16_t key = mine[i];
+                        uint32_t j = i;
+                        while (j > 0u && mine[j - 1u] > key) { mine[j] = mine[j - 1u]; --j; }
+                        mine[j] = key;
+                    }
+                    int64_t BT = Bt[q], BA = Ba[q];
+                    for (uint32_t i = 0; i < cnt; ++i) reserve_one(mine[i], BT, BA, true);
                     Bt[q] = BT; Ba[q] = BA;
                     if (BT == BA) { open[q] = 0; atomicSub(&s_open, 1); }   // the runs have met: the rest of the tile was served right
                 }
+            } else {
+                // some queue has more records in this window than a list holds: one warp per straggling queue scans the
+                // window 32 records at a time and re-serves its own in order; every lane carries the two runs, lane 0 writes
+                for (uint32_t t = (uint32_t)warp; t < stragglers; t += kInStrWarps) {
+                    const uint32_t q = oq[t];
+                    if (lane == 0) lcount[t] = 0u;
+                    if (!open[q]) continue;
+                    int64_t BT = Bt[q], BA = Ba[q];
+                    for (uint32_t k0 = 0; k0 < wn; k0 += 32u) {
+                        const uint32_t k = k0 + (uint32_t)lane;
+                        unsigned hits = __ballot_sync(0xffffffffu, k < wn && (ent_pq[min(k, wn - 1u)].y & 0xffffu) == q);
+                        while (hits) {
+                            const uint32_t kk = k0 + (uint32_t)__ffs((int)hits) - 1u;
+                            hits &= hits - 1u;
+                            reserve_one(kk, BT, BA, lane == 0);
+                        }
+                    }
+                    if (lane == 0) {
+                        Bt[q] = BT; Ba[q] = BA;
+                        if (BT == BA) { open[q] = 0; atomicSub(&s_open, 1); }
+                    }
+                }
+                __syncthreads();
+                if (tid == 0) s_overflow = 0u;
             }
             __syncthreads();
         }
+#ifdef HBF_DBG_ONEITER
+        break;
+#endif
         if (*reinterpret_cast<volatile int *>(&s_open) <= 0) break;
         cb += step;
     }
@@ -954,7 +1032,9 @@ InTileMap inorder_tile_map(uint64_t n, int sm_count) {
 
 // dynamic shared memory of the serve kernel: the per-queue state and the per-die counters
 size_t inorder_serve_smem(uint32_t n_dies) { return (size_t)kInMaxQueues * 16 + (size_t)n_dies * 28; }
-static size_t inorder_straggle_smem() { return (size_t)kInMaxQueues * 16 + (size_t)kInStrKeep * 24 + (size_t)kInMaxQueues * 3; }
+static size_t inorder_straggle_smem() {
+    return (size_t)kInMaxQueues * 16 + (size_t)kInStrKeep * 24 + (size_t)kInMaxQueues * 3 + (size_t)kInStrMaxStragglers * (kInStrList * 2 + 4);
+}
 
 size_t inorder_head_bytes(uint64_t tiles, uint32_t n_queues) { return tiles * n_queues * (size_t)kInHead * sizeof(InHead); }
 
