@@ -150,6 +150,8 @@ __host__ __device__ inline uint64_t tile_last(const InTileMap &m, uint32_t t) { 
     return e < m.n ? e : m.n;
 }
 InTileMap inorder_tile_map(uint64_t n, int sm_count);
+// per-tile bookkeeping of the stall total: as-if-idle sum, fix-up corrections, and the exact sum of a re-served tile
+struct InTile { long long spec_sum, fix_delta, true_sum; uint32_t reserve; uint32_t stragglers; };
 size_t inorder_head_bytes(uint64_t tiles, uint32_t n_queues);
 size_t inorder_serve_smem(uint32_t n_dies);
 cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st);

@@ -178,8 +178,6 @@ __device__ __forceinline__ Served serve_terms_geom(const FastGeom &g, const Mode
     }
     return r;
 }
-// per-tile bookkeeping of the stall total: as-if-idle sum, fix-up corrections, and the exact sum of a re-served tile
-struct InTile { long long spec_sum, fix_delta, true_sum; uint32_t reserve; uint32_t stragglers; };
 // The first kInHead accesses of every (tile, queue), as the serve pass saw them: all the fix-up needs in the common case.
 constexpr int kInHead = 8;
 struct InHead { int64_t m, s; uint32_t xo, idx; };       // arrival + service, service, transfer | op << 31, batch index
@@ -381,7 +379,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, const __grid_c
         if (!RESERVE && turn * (uint32_t)(K * 32) < qid_stride) {   // (the stride is a multiple of a turn's records)
 #pragma unroll
             for (int u = 0; u < K; ++u)
-                if (valid[u]) qid_t[i[u]] = ready[u] ? (uint16_t)v[u].queue : (uint16_t)0xffffu;
+                if (valid[u]) qid_t[i[u]] = ready[u] ? (uint16_t)v[u].queue : (uint16_t)kInMaxQueues;   // (one past the last queue: not modeled)
         }
         if (!RESERVE) {
 #pragma unroll
@@ -617,7 +615,7 @@ __device__ __forceinline__ uint32_t fast_queue(const FastRange &f, const ModelPa
 // busy-until) and the as-if-idle run (to know what the serve pass wrote).  A queue is done when the two runs meet:
 // from there on the serve pass was right.  The block stops at the chunk in which its last queue is done.
 // What it streams: for the first kInQidPrefix records of every tile the serve pass left the queue of each record
-// as a 16-bit number (0xffff: not modeled), so the filter reads 2 bytes per record, 32 records per thread and turn;
+// as a 16-bit number (kInMaxQueues: not modeled), so the filter reads 2 bytes per record, 32 records per thread and turn;
 // past that prefix (queues that stay backlogged for very long) it decodes the queue from the records.
 // ======================================================================================================
 struct FixRun { int64_t B, Bs; long long dstall, max_c; bool settled; };
@@ -679,7 +677,7 @@ k_inorder_fixstraggle(const hbf_access_t *__restrict__ acc, uint64_t n, const __
     uint2 *ent_pq = reinterpret_cast<uint2 *>(ent_as + kInStrKeep);            //        transfer | op << 31, queue | position << 16
     uint16_t *oq = reinterpret_cast<uint16_t *>(ent_pq + kInStrKeep);          // [stragglers] their queues
     uint8_t *open = reinterpret_cast<uint8_t *>(oq + kInMaxQueues);            // [queues] 0, or 1 + the queue's place in oq while its runs have not met
-    uint16_t *lst = reinterpret_cast<uint16_t *>(open + kInMaxQueues);         // [stragglers][kInStrList] the window's records of each queue
+    uint16_t *lst = reinterpret_cast<uint16_t *>(open + kInMaxQueues + 64);    // [stragglers][kInStrList] the window's records of each queue
     uint32_t *lcount = reinterpret_cast<uint32_t *>(lst + kInStrMaxStragglers * kInStrList);   // [stragglers] how many
     __shared__ uint32_t s_overflow;
     if (tid < kInStrMaxStragglers) lcount[tid] = 0u;
@@ -706,6 +704,7 @@ k_inorder_fixstraggle(const hbf_access_t *__restrict__ acc, uint64_t n, const __
         for (int k = 0; k < kInStrQueuesPerThread; ++k) {
             const uint32_t q = (uint32_t)(k * kInStrThreads + tid);
             if (q < kInMaxQueues) { open[q] = 0; Ba[q] = kNegInf; Bt[q] = Bin[k]; }
+            if (q < 64u) open[kInMaxQueues + q] = 0;         // (the entry of records that are not modeled, and padding)
             if (c[k] == 0u) continue;
             if (Bin[k] <= e0[k].m - e0[k].s) continue;       // idle on arrival: the as-if run was right from the start
             deep[atomicAdd(&s_total, 1u)] = (uint16_t)q;
@@ -821,13 +820,22 @@ k_inorder_fixstraggle(const hbf_access_t *__restrict__ acc, uint64_t n, const __
         uint32_t keep = 0, first = 0, rk[kInStrItems];
         if (by_qid) {
             const uint32_t room = tile_len - cb;             // records of the tile from this chunk on
+            if (room >= (uint32_t)kInStrQChunk) {            // a whole chunk: every number was written by the serve pass
 #pragma unroll
-            for (int j = 0; j < kInStrQItems; ++j) {
-                const uint4 v = nx_q[j >> 3];
-                const uint32_t w = ((j >> 1) & 3) == 0 ? v.x : ((j >> 1) & 3) == 1 ? v.y : ((j >> 1) & 3) == 2 ? v.z : v.w;
-                const uint32_t q = (w >> (16 * (j & 1))) & 0xffffu;
-                const bool k = q < R && (uint32_t)(tid * kInStrQItems + j) < room && open[q] != 0;
-                keep |= k ? 1u << j : 0u;
+                for (int j = 0; j < kInStrQItems; ++j) {
+                    const uint4 v = nx_q[j >> 3];
+                    const uint32_t w = ((j >> 1) & 3) == 0 ? v.x : ((j >> 1) & 3) == 1 ? v.y : ((j >> 1) & 3) == 2 ? v.z : v.w;
+                    keep |= open[(w >> (16 * (j & 1))) & 0xffffu] != 0 ? 1u << j : 0u;
+                }
+            } else {                                         // the tile's last chunk: past its end the numbers are not defined
+#pragma unroll
+                for (int j = 0; j < kInStrQItems; ++j) {
+                    const uint4 v = nx_q[j >> 3];
+                    const uint32_t w = ((j >> 1) & 3) == 0 ? v.x : ((j >> 1) & 3) == 1 ? v.y : ((j >> 1) & 3) == 2 ? v.z : v.w;
+                    const uint32_t q = (w >> (16 * (j & 1))) & 0xffffu;
+                    const bool k = q < R && (uint32_t)(tid * kInStrQItems + j) < room && open[q] != 0;
+                    keep |= k ? 1u << j : 0u;
+                }
             }
             fetch(cb + step);
             const uint32_t cnt = (uint32_t)__popc(keep);
@@ -990,18 +998,6 @@ k_inorder_fixstraggle(const hbf_access_t *__restrict__ acc, uint64_t n, const __
     }
 }
 
-// stall total of the batch: per tile the exact sum if it was re-served, else the as-if sum plus its corrections
-__global__ void k_inorder_total(BatchCtrl *ctrl, const InTile *__restrict__ in_tile, uint32_t n_tiles) {
-    if (ctrl->skip || ctrl->run_sort || !ctrl->inorder_used) return;
-    long long tot = 0;
-    for (uint32_t t = threadIdx.x; t < n_tiles; t += blockDim.x) {
-        const InTile v = in_tile[t];
-        tot += v.reserve ? v.true_sum : v.spec_sum + v.fix_delta;
-    }
-    tot = warp_sum(tot);
-    if ((threadIdx.x & 31) == 0 && tot) atomicAdd((unsigned long long *)&ctrl->modeled_ns, (unsigned long long)tot);
-}
-
 #ifndef HBF_IN_SKEW_PERMILLE
 #define HBF_IN_SKEW_PERMILLE 60
 #endif
@@ -1033,7 +1029,7 @@ InTileMap inorder_tile_map(uint64_t n, int sm_count) {
 // dynamic shared memory of the serve kernel: the per-queue state and the per-die counters
 size_t inorder_serve_smem(uint32_t n_dies) { return (size_t)kInMaxQueues * 16 + (size_t)n_dies * 28; }
 static size_t inorder_straggle_smem() {
-    return (size_t)kInMaxQueues * 16 + (size_t)kInStrKeep * 24 + (size_t)kInMaxQueues * 3 + (size_t)kInStrMaxStragglers * (kInStrList * 2 + 4);
+    return (size_t)kInMaxQueues * 16 + (size_t)kInStrKeep * 24 + (size_t)kInMaxQueues * 3 + 64 + (size_t)kInStrMaxStragglers * (kInStrList * 2 + 4);
 }
 
 size_t inorder_head_bytes(uint64_t tiles, uint32_t n_queues) { return tiles * n_queues * (size_t)kInHead * sizeof(InHead); }
@@ -1074,8 +1070,7 @@ cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st) {
         a.acc, n, tmap, a.ranges, a.mp, a.fast, a.ctrl, a.ws.in_bin, heads, a.ws.in_headcnt, a.completion, a.stall, tiles,
         a.claim_limit, a.ws.in_qid, qid_stride);
     serve(true);
-    k_inorder_total<<<1, 256, 0, st>>>(a.ctrl, tiles, n_tiles);
-    g_kernel_launches += 5;
+    g_kernel_launches += 4;
     return cudaGetLastError();
 }
 

@@ -1014,9 +1014,9 @@ static cudaError_t launch_sort_path(const SubmitArgs &a, cudaStream_t st) {
 // ---- the sort path launched from the device -----------------------------------------------------------
 // With HBF_PATH_AUTO the host enqueues the in-order kernels only.  A batch that turns out not to be in issue
 // order (or has a service time the in-order kernels cannot hold) needs the sort path after all, and the host
-// cannot know that without waiting for the device.  So one thread looks at the batch's control block and, in
-// that case only, launches the sort path's kernels itself, in order, into the tail-launch stream: they run
-// after this one-thread kernel and before the next kernel of the host's stream (a parent grid is complete
+// cannot know that without waiting for the device.  So the kernel that follows the in-order kernels (it also sums the
+// batch's stall total when they did serve it) looks at the batch's control block and, in that case only, one thread launches the sort path's kernels itself, in order, into the tail-launch stream: they run
+// after this kernel and before the next kernel of the host's stream (a parent grid is complete
 // only when its children are), which is the batch's finish kernel.  A batch in issue order pays one empty
 // launch instead of thirteen.
 struct SortChain {
@@ -1026,14 +1026,28 @@ struct SortChain {
     const unsigned long long *claim_limit; uint32_t *die_claims;
     uint32_t n_queues, n_dies; uint64_t desc_words, scan_words;
     unsigned cls_grid, hist_grid, sort_grid, scan_grid;
+    const InTile *in_tile; uint32_t n_tiles; int may_sort;
 };
 
 __global__ void k_zero_words(uint32_t *p, uint64_t words) {
     for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < words; i += (uint64_t)gridDim.x * blockDim.x) p[i] = 0u;
 }
 
-__global__ void k_sort_fallback(const __grid_constant__ SortChain c) {
-    if (c.ctrl->skip || !c.ctrl->run_sort) return;           // served in issue order, or refused: nothing to do
+__global__ void __launch_bounds__(256) k_after_inorder(const __grid_constant__ SortChain c) {
+    if (c.ctrl->skip) return;                                // refused: nothing to do
+    if (c.ctrl->inorder_used) {
+        // served in issue order.  Stall total of the batch: per tile the exact sum if it was re-served, else the as-if
+        // sum plus its corrections
+        long long tot = 0;
+        for (uint32_t t = threadIdx.x; t < c.n_tiles; t += blockDim.x) {
+            const InTile v = c.in_tile[t];
+            tot += v.reserve ? v.true_sum : v.spec_sum + v.fix_delta;
+        }
+        tot = warp_sum(tot);
+        if ((threadIdx.x & 31) == 0 && tot) atomicAdd((unsigned long long *)&c.ctrl->modeled_ns, (unsigned long long)tot);
+        return;
+    }
+    if (!c.ctrl->run_sort || !c.may_sort || threadIdx.x != 0) return;
     cudaStream_t st = cudaStreamTailLaunch;
     k_begin<<<1, 1024, 0, st>>>(c.ctrl, c.state, c.busy, c.busy_stage, c.stats_stage, c.hist, c.n_queues, c.n_dies, 1, 1, c.die_claims);
     k_zero_words<<<(unsigned)min((unsigned long long)((c.desc_words + 1023) / 1024), 592ull), 1024, 0, st>>>(c.desc0, c.desc_words);
@@ -1048,7 +1062,7 @@ __global__ void k_sort_fallback(const __grid_constant__ SortChain c) {
                                                  c.claim_limit, c.die_claims);
 }
 
-static cudaError_t launch_sort_fallback(const SubmitArgs &a, cudaStream_t st) {
+static cudaError_t launch_after_inorder(const SubmitArgs &a, bool may_sort, cudaStream_t st) {
     const uint64_t n = a.n;
     const uint64_t sort_tiles = (n + kSortTile - 1) / kSortTile, scan_tiles = (n + kScanTile - 1) / kScanTile;
     cudaError_t e = ensure_dyn_smem((const void *)k_sort_pass, kSortSmem);   // (an attribute of the kernel: device-side launches use it too)
@@ -1065,7 +1079,9 @@ static cudaError_t launch_sort_fallback(const SubmitArgs &a, cudaStream_t st) {
     c.hist_grid = (unsigned)std::min<uint64_t>((n + kHistThreads * 8 - 1) / (kHistThreads * 8), (uint64_t)a.sm_count * 4);
     c.sort_grid = (unsigned)std::min<uint64_t>(sort_tiles, (uint64_t)a.sm_count * 3);
     c.scan_grid = (unsigned)std::min<uint64_t>(scan_tiles, (uint64_t)a.sm_count * 8);
-    k_sort_fallback<<<1, 1, 0, st>>>(c);
+    const InTileMap tmap = inorder_tile_map(n, a.sm_count);
+    c.in_tile = reinterpret_cast<const InTile *>(a.ws.in_tile); c.n_tiles = tmap.n_tiles; c.may_sort = may_sort ? 1 : 0;
+    k_after_inorder<<<1, 256, 0, st>>>(c);
     g_kernel_launches += 1;
     return cudaGetLastError();
 }
@@ -1088,10 +1104,8 @@ cudaError_t launch_submit(const SubmitArgs &a, cudaStream_t st) {
             cudaError_t e = launch_inorder(a, st);
             if (e != cudaSuccess) return e;
             mark(8);
-            if (sort_kernels) {
-                e = launch_sort_fallback(a, st);
-                if (e != cudaSuccess) return e;
-            }
+            e = launch_after_inorder(a, sort_kernels, st);
+            if (e != cudaSuccess) return e;
             mark(1); mark(2); mark(3); mark(4);
         } else {
             cudaError_t e = launch_sort_path(a, st);
