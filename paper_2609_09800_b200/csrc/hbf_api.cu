@@ -47,6 +47,7 @@ struct hbf_ctx {
     bool ret_on = false; RetDev ret{}; hbf_retention_config_t ret_cfg{};
     float *h_hot = nullptr;                      // pinned [3]
     float *h_ext = nullptr;                      // pinned [n_regions]
+    std::vector<float> last_ext;                 // the external powers the device holds (empty: none sent yet)
     bool submitted = false;
     bool profiling = false; cudaEvent_t ev[kProfEvents] = {}; cudaEvent_t ev_th[2] = {}; bool ev_made = false;
     bool prof_submit = false, prof_thermal = false, prof_inorder = false, inorder_ok = false;
@@ -673,8 +674,12 @@ int hbf_thermal_step(hbf_ctx *c, int64_t dt_ns, const float *ext_power_w, uint32
     if (!c->rom && dt_sub > c->euler_limit_s) return HBF_E_INVAL;
     if (c->bin_ns && dt_ns != c->bin_ns) return HBF_E_INVAL;
     if (c->rom && (dt_ns != c->rom_dt_ns || d_temps_out)) return HBF_E_INVAL;
-    if (n_ext)      // pageable source: the runtime stages the bytes before returning, so the caller's array is free at once
+    // pageable source: the runtime stages the bytes before returning, so the caller's array is free at once.  A loop that
+    // steps with the same powers every time (the usual case) sends them once.
+    if (n_ext && (c->last_ext.size() != n_ext || memcmp(c->last_ext.data(), ext_power_w, n_ext * sizeof(float)) != 0)) {
         CK(cudaMemcpyAsync(c->td.ext_power, ext_power_w, n_ext * sizeof(float), cudaMemcpyHostToDevice, c->stream));
+        c->last_ext.assign(ext_power_w, ext_power_w + n_ext);
+    }
     if (c->bin_ns) {                                         // the step is the bin the thermal clock stands in
         CK(launch_take_bin(c->d_ledger + (size_t)(c->cur_bin % c->n_bins) * c->mp.n_dies, c->d_pending, c->mp.n_dies, c->stream));
         c->cur_bin += 1;

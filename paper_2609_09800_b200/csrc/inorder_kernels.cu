@@ -1046,7 +1046,9 @@ cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st) {
         const void *serve_fns[4] = {(const void *)k_inorder_serve<false, false>, (const void *)k_inorder_serve<true, false>,
                                     (const void *)k_inorder_serve<false, true>, (const void *)k_inorder_serve<true, true>};
         for (const void *f : serve_fns) { cudaError_t e = ensure_dyn_smem(f, smem_serve); if (e != cudaSuccess) return e; }
-        cudaError_t e = ensure_dyn_smem((const void *)k_inorder_fixstraggle<false>, smem_str);
+        cudaError_t e = ensure_dyn_smem((const void *)k_inorder_scan, 0);
+        if (e != cudaSuccess) return e;
+        e = ensure_dyn_smem((const void *)k_inorder_fixstraggle<false>, smem_str);
         if (e != cudaSuccess) return e;
         e = ensure_dyn_smem((const void *)k_inorder_fixstraggle<true>, smem_str);
         if (e != cudaSuccess) return e;

@@ -973,7 +973,12 @@ cudaError_t ensure_dyn_smem(const void *kernel, size_t bytes) {
             if (e == cudaSuccess) en.bytes = bytes;
             return e;
         }
-    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (bytes > 48u * 1024u) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+#ifdef HBF_EXP_CARVEOUT
+    // the kernels of a step follow one another closely: the same shared-memory carve-out for all of them spares the SMs a
+    // reconfiguration at every kernel boundary
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, HBF_EXP_CARVEOUT);
+#endif
     if (e == cudaSuccess) set.push_back(Entry{dev, kernel, bytes});
     return e;
 }
@@ -1094,6 +1099,10 @@ cudaError_t launch_submit(const SubmitArgs &a, cudaStream_t st) {
     auto mark = [&](int k) { if (a.ev) cudaEventRecord(a.ev[k], st); };
     const bool try_inorder = a.inorder_ok && (a.path == HBF_PATH_AUTO || a.path == HBF_PATH_INORDER);
     const bool sort_kernels = a.path != HBF_PATH_INORDER || !a.inorder_ok;
+    {
+        const void *small[] = {(const void *)k_begin, (const void *)k_finish, (const void *)k_after_inorder};
+        for (const void *f : small) { cudaError_t e = ensure_dyn_smem(f, 0); if (e != cudaSuccess) return e; }
+    }
     mark(0);
     k_begin<<<1, 1024, 0, st>>>(a.ctrl, a.state, a.busy, a.busy_stage, a.stats_stage, a.ws.hist, a.mp.n_queues, a.mp.n_dies,
                                0, try_inorder ? 0 : 1, a.die_claims);
