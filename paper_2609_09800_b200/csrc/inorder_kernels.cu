@@ -618,6 +618,15 @@ __device__ __forceinline__ uint32_t fast_queue(const FastRange &f, const ModelPa
 // as a 16-bit number (kInMaxQueues: not modeled), so the filter reads 2 bytes per record, 32 records per thread and turn;
 // past that prefix (queues that stay backlogged for very long) it decodes the queue from the records.
 // ======================================================================================================
+// The general form of the terms (several ranges, any geometry, thermal scaling), kept out of line here: this kernel runs
+// nearly straight through once per block, so what it costs is fetching its instructions, and the common configuration
+// never takes this path.
+__device__ __noinline__ Served serve_terms_general(const RangeSnap &rs, const ModelParams &mp, uint64_t addr, int64_t issue, uint64_t bf,
+                                                   int64_t q_ppm, Div64 div_q) {
+    unsigned ignored = 0;                                    // (the serve pass has already vetted every service time)
+    return serve_terms(rs, mp, addr, issue, bf, q_ppm, div_q, ignored, 33);
+}
+
 struct FixRun { int64_t B, Bs; long long dstall, max_c; bool settled; };
 __device__ __forceinline__ void fix_entry(FixRun &f, const InHead &h, int64_t *completion, int64_t *stall) {
     if (f.settled) return;
@@ -636,15 +645,10 @@ constexpr int kInStrThreads = 512;
 constexpr int kInStrWarps = kInStrThreads / 32;
 constexpr int kInStrQItems = 32;                          // records per thread and turn inside the queue-number prefix
 constexpr int kInStrQChunk = kInStrThreads * kInStrQItems;
-constexpr int kInStrItems = 8;                            // and past it, where the queue is decoded from the record
-constexpr int kInStrChunk = kInStrThreads * kInStrItems;
 constexpr int kInStrKeep = 1024;                          // kept records served at a time (a chunk with more is served in windows)
 constexpr int kInStrMaxStragglers = 128;                   // a tile with as many is served again whole instead
 constexpr int kInStrList = 32;                            // records of one queue in a window that its list holds (more: the window is scanned)
-constexpr int kInStrCells = kInStrItems * kInStrWarps;    // (item, warp) cells of the kept-record counts, decode path
-constexpr int kInStrCellsPerLane = kInStrCells / 32;
 constexpr int kInStrQueuesPerThread = (kInMaxQueues + kInStrThreads - 1) / kInStrThreads;
-static_assert(kInStrCells % 32 == 0, "the offset scan gives every lane the same number of cells");
 static_assert(kInStrQChunk <= 65536, "a kept record's position in its chunk is stored in 16 bits");
 static_assert(kInQidPrefix % kInStrQChunk == 0 && kInStrQItems == 32, "a thread's 32 queue numbers are four 16-byte loads");
 
@@ -659,7 +663,7 @@ k_inorder_fixstraggle(const hbf_access_t *__restrict__ acc, uint64_t n, const __
     extern __shared__ __align__(16) unsigned char str_smem[];
     __shared__ ModelParams mp;
     __shared__ FastRange fast_range;
-    __shared__ uint32_t s_cells[kInStrCells];
+    __shared__ uint32_t s_cells[kInStrWarps];
     __shared__ uint32_t s_total;
     __shared__ uint32_t s_stragglers;                        // straggling queues of the tile
     __shared__ int s_open;                                   // those whose two runs have not met yet
@@ -676,8 +680,8 @@ k_inorder_fixstraggle(const hbf_access_t *__restrict__ acc, uint64_t n, const __
     longlong2 *ent_as = reinterpret_cast<longlong2 *>(Ba + kInMaxQueues);      // [keep] kept records, batch order: issue time, service time
     uint2 *ent_pq = reinterpret_cast<uint2 *>(ent_as + kInStrKeep);            //        transfer | op << 31, queue | position << 16
     uint16_t *oq = reinterpret_cast<uint16_t *>(ent_pq + kInStrKeep);          // [stragglers] their queues
-    uint8_t *open = reinterpret_cast<uint8_t *>(oq + kInMaxQueues);            // [queues] 0, or 1 + the queue's place in oq while its runs have not met
-    uint16_t *lst = reinterpret_cast<uint16_t *>(open + kInMaxQueues + 64);    // [stragglers][kInStrList] the window's records of each queue
+    uint8_t *open = reinterpret_cast<uint8_t *>(oq + kInMaxQueues);            // [2 x queues] 0, or 1 + the queue's place in oq while its runs have not met
+    uint16_t *lst = reinterpret_cast<uint16_t *>(open + 2 * kInMaxQueues);     // [stragglers][kInStrList] the window's records of each queue
     uint32_t *lcount = reinterpret_cast<uint32_t *>(lst + kInStrMaxStragglers * kInStrList);   // [stragglers] how many
     __shared__ uint32_t s_overflow;
     if (tid < kInStrMaxStragglers) lcount[tid] = 0u;
@@ -703,8 +707,7 @@ k_inorder_fixstraggle(const hbf_access_t *__restrict__ acc, uint64_t n, const __
 #pragma unroll
         for (int k = 0; k < kInStrQueuesPerThread; ++k) {
             const uint32_t q = (uint32_t)(k * kInStrThreads + tid);
-            if (q < kInMaxQueues) { open[q] = 0; Ba[q] = kNegInf; Bt[q] = Bin[k]; }
-            if (q < 64u) open[kInMaxQueues + q] = 0;         // (the entry of records that are not modeled, and padding)
+            if (q < kInMaxQueues) { open[q] = 0; open[kInMaxQueues + q] = 0; Ba[q] = kNegInf; Bt[q] = Bin[k]; }   // (upper half: not modeled, or not defined)
             if (c[k] == 0u) continue;
             if (Bin[k] <= e0[k].m - e0[k].s) continue;       // idle on arrival: the as-if run was right from the start
             deep[atomicAdd(&s_total, 1u)] = (uint16_t)q;
@@ -766,7 +769,6 @@ k_inorder_fixstraggle(const hbf_access_t *__restrict__ acc, uint64_t n, const __
     const uint32_t tile_len = (uint32_t)(tile_end - tile_begin);       // offsets inside a tile fit 32 bits
     const hbf_access_t *acc_t = acc + tile_begin;
     const uint4 *qid_t = reinterpret_cast<const uint4 *>(in_qid + (uint64_t)tile * qid_stride);
-    unsigned ignored = 0;                                    // (the serve pass has already vetted every service time)
     if (tid == 0) s_open = (int)stragglers;
 
     // the queue numbers of the next chunk are on their way while this one is filtered
@@ -797,7 +799,7 @@ k_inorder_fixstraggle(const hbf_access_t *__restrict__ acc, uint64_t n, const __
             const uint32_t slot = (uint32_t)(k * kInStrThreads + tid);
             if (slot < wn) {
                 Served v = fast_terms ? serve_terms_fast(fast_range, mp, r_addr[k], r_issue[k], r_bf[k])
-                                      : serve_terms(rs, mp, r_addr[k], r_issue[k], r_bf[k], q_ppm, div_q, ignored, 33);
+                                      : serve_terms_general(rs, mp, r_addr[k], r_issue[k], r_bf[k], q_ppm, div_q);
                 if (DEBT && tile_begin + cb + r_e[k] < claim_limit) v.s += quantum_ns;
                 ent_as[slot] = make_longlong2(r_issue[k], v.s);
                 ent_pq[slot] = make_uint2(v.xfer | (v.op << 31), v.queue | (r_e[k] << 16));
@@ -814,30 +816,45 @@ k_inorder_fixstraggle(const hbf_access_t *__restrict__ acc, uint64_t n, const __
     uint32_t cb = 0;
     while (cb < tile_len) {
         const bool by_qid = cb + kInStrQChunk <= qid_stride;  // the same for the whole block
-        const uint32_t step = by_qid ? (uint32_t)kInStrQChunk : (uint32_t)kInStrChunk;
-        // ---- keep the modeled records of the open queues, in batch order: bit j of `keep` is this thread's item j.
-        // Inside the prefix a thread's items are 32 consecutive records; past it, eight records a block width apart.
-        uint32_t keep = 0, first = 0, rk[kInStrItems];
+        // ---- keep the modeled records of the open queues, in batch order: bit j of `keep` is this thread's item j, the
+        // thread's items being 32 consecutive records
+        uint32_t keep = 0;
         if (by_qid) {
-            const uint32_t room = tile_len - cb;             // records of the tile from this chunk on
-            if (room >= (uint32_t)kInStrQChunk) {            // a whole chunk: every number was written by the serve pass
+            // (numbers past the tile's end are not defined: the table is indexed by 12 bits, twice the queues, and whatever
+            // such a number finds there is masked off by position)
 #pragma unroll
-                for (int j = 0; j < kInStrQItems; ++j) {
-                    const uint4 v = nx_q[j >> 3];
-                    const uint32_t w = ((j >> 1) & 3) == 0 ? v.x : ((j >> 1) & 3) == 1 ? v.y : ((j >> 1) & 3) == 2 ? v.z : v.w;
-                    keep |= open[(w >> (16 * (j & 1))) & 0xffffu] != 0 ? 1u << j : 0u;
-                }
-            } else {                                         // the tile's last chunk: past its end the numbers are not defined
-#pragma unroll
-                for (int j = 0; j < kInStrQItems; ++j) {
-                    const uint4 v = nx_q[j >> 3];
-                    const uint32_t w = ((j >> 1) & 3) == 0 ? v.x : ((j >> 1) & 3) == 1 ? v.y : ((j >> 1) & 3) == 2 ? v.z : v.w;
-                    const uint32_t q = (w >> (16 * (j & 1))) & 0xffffu;
-                    const bool k = q < R && (uint32_t)(tid * kInStrQItems + j) < room && open[q] != 0;
+            for (int j = 0; j < kInStrQItems; ++j) {
+                const uint4 v = nx_q[j >> 3];
+                const uint32_t w = ((j >> 1) & 3) == 0 ? v.x : ((j >> 1) & 3) == 1 ? v.y : ((j >> 1) & 3) == 2 ? v.z : v.w;
+                keep |= open[(w >> (16 * (j & 1))) & (2u * kInMaxQueues - 1u)] != 0 ? 1u << j : 0u;
+            }
+            const uint32_t room = tile_len - cb, mine = (uint32_t)(tid * kInStrQItems);   // records of the tile from this chunk on
+            const uint32_t have = room > mine ? min(room - mine, (uint32_t)kInStrQItems) : 0u;
+            keep &= have >= 32u ? 0xffffffffu : (1u << have) - 1u;
+            fetch(cb + kInStrQChunk);
+        } else {
+            // past the prefix (a rare stretch: its size matters more than its speed) the queue comes from the record
+#pragma unroll 2
+            for (int j = 0; j < kInStrQItems; ++j) {
+                const uint32_t i = cb + (uint32_t)(tid * kInStrQItems + j);
+                if (i < tile_len) {
+                    const uint64_t *rec = reinterpret_cast<const uint64_t *>(acc_t + i);
+                    const uint64_t addr = __ldg(rec);
+                    bool k;
+                    if (one_range) {
+                        const uint32_t q = fast_queue(fast_range, mp, addr);
+                        k = q != 0xffffffffu && open[q] != 0;
+                    } else {
+                        const Served v = serve_terms_general(rs, mp, addr, (int64_t)__ldg(rec + 1), __ldg(rec + 2), q_ppm, div_q);
+                        k = v.st == HBF_ST_READY && open[v.queue] != 0;
+                    }
                     keep |= k ? 1u << j : 0u;
                 }
             }
-            fetch(cb + step);
+            fetch(cb + kInStrQChunk);
+        }
+        uint32_t first;                                      // place of this thread's first kept record among the chunk's
+        {
             const uint32_t cnt = (uint32_t)__popc(keep);
             uint32_t incl = cnt;
 #pragma unroll
@@ -854,54 +871,12 @@ k_inorder_fixstraggle(const hbf_access_t *__restrict__ acc, uint64_t n, const __
             }
             __syncthreads();
             first = s_cells[warp] + incl - cnt;
-        } else {
-            uint64_t addr[kInStrItems];
-#pragma unroll
-            for (int j = 0; j < kInStrItems; ++j) {
-                const uint32_t i = cb + (uint32_t)(j * kInStrThreads + tid);
-                addr[j] = i < tile_len ? __ldg(reinterpret_cast<const uint64_t *>(acc_t + i)) : ~0ull;
-            }
-#pragma unroll
-            for (int j = 0; j < kInStrItems; ++j) {
-                const uint32_t i = cb + (uint32_t)(j * kInStrThreads + tid);
-                bool k = false;
-                if (i < tile_len) {
-                    if (one_range) {
-                        const uint32_t q = fast_queue(fast_range, mp, addr[j]);
-                        k = q != 0xffffffffu && open[q] != 0;
-                    } else {
-                        const uint64_t *rec = reinterpret_cast<const uint64_t *>(acc_t + i);
-                        const Served v = serve_terms(rs, mp, addr[j], (int64_t)__ldg(rec + 1), __ldg(rec + 2), q_ppm, div_q, ignored, 33);
-                        k = v.st == HBF_ST_READY && open[v.queue] != 0;
-                    }
-                }
-                const unsigned bal = __ballot_sync(0xffffffffu, k);
-                rk[j] = (uint32_t)__popc(bal & lanemask_lt());
-                if (lane == 0) s_cells[j * kInStrWarps + warp] = (uint32_t)__popc(bal);
-                keep |= k ? 1u << j : 0u;
-            }
-            __syncthreads();
-            if (warp == 0) {
-                uint32_t c[kInStrCellsPerLane], tot = 0;
-#pragma unroll
-                for (int b = 0; b < kInStrCellsPerLane; ++b) { c[b] = s_cells[lane * kInStrCellsPerLane + b]; tot += c[b]; }
-                uint32_t incl = tot;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += t; }
-                uint32_t run = incl - tot;
-#pragma unroll
-                for (int b = 0; b < kInStrCellsPerLane; ++b) { s_cells[lane * kInStrCellsPerLane + b] = run; run += c[b]; }
-                if (lane == 31) s_total = incl;
-            }
-            __syncthreads();
-#pragma unroll
-            for (int j = 0; j < kInStrItems; ++j) rk[j] += s_cells[j * kInStrWarps + warp];
         }
         // ---- the kept records, a window of kInStrKeep at a time (one window, nearly always)
         const uint32_t total = s_total;
         for (uint32_t wb = 0; wb < total; wb += (uint32_t)kInStrKeep) {
             const uint32_t wn = min(total - wb, (uint32_t)kInStrKeep);
-            if (by_qid) {
+            {
                 uint32_t m = keep;
                 while (m) {
                     const uint32_t j = (uint32_t)__ffs((int)m) - 1u;
@@ -909,10 +884,6 @@ k_inorder_fixstraggle(const hbf_access_t *__restrict__ acc, uint64_t n, const __
                     const uint32_t slot = first + (uint32_t)__popc(keep & ((1u << j) - 1u)) - wb;   // (wraps below the window)
                     if (slot < wn) ent_pq[slot].y = (uint32_t)(tid * kInStrQItems) + j;
                 }
-            } else {
-#pragma unroll
-                for (int j = 0; j < kInStrItems; ++j)
-                    if ((keep >> j) & 1u) { const uint32_t slot = rk[j] - wb; if (slot < wn) ent_pq[slot].y = (uint32_t)(j * kInStrThreads + tid); }
             }
             __syncthreads();
             fill_window(cb, wn);
@@ -983,7 +954,7 @@ k_inorder_fixstraggle(const hbf_access_t *__restrict__ acc, uint64_t n, const __
         break;
 #endif
         if (*reinterpret_cast<volatile int *>(&s_open) <= 0) break;
-        cb += step;
+        cb += kInStrQChunk;
     }
     }
     dstall = warp_sum(dstall); max_c = warp_max(max_c);
@@ -1029,7 +1000,7 @@ InTileMap inorder_tile_map(uint64_t n, int sm_count) {
 // dynamic shared memory of the serve kernel: the per-queue state and the per-die counters
 size_t inorder_serve_smem(uint32_t n_dies) { return (size_t)kInMaxQueues * 16 + (size_t)n_dies * 28; }
 static size_t inorder_straggle_smem() {
-    return (size_t)kInMaxQueues * 16 + (size_t)kInStrKeep * 24 + (size_t)kInMaxQueues * 3 + 64 + (size_t)kInStrMaxStragglers * (kInStrList * 2 + 4);
+    return (size_t)kInMaxQueues * 16 + (size_t)kInStrKeep * 24 + (size_t)kInMaxQueues * 4 + (size_t)kInStrMaxStragglers * (kInStrList * 2 + 4);
 }
 
 size_t inorder_head_bytes(uint64_t tiles, uint32_t n_queues) { return tiles * n_queues * (size_t)kInHead * sizeof(InHead); }
