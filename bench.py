@@ -33,12 +33,26 @@ UNIT = "accesses/s"
 ALGO_BYTES_PER_ACCESS = 41            # 24 B record in, 8 B completion + 8 B stall + 1 B status out
 # algorithmic bytes per access of each kernel group (what the kernel itself must move)
 STAGE_BYTES = {"classify": 24 + 8 + 1, "plan_hist": 8, "scan": 8 + 4 + 24 + 16, "inorder": 24 + 16 + 1}
-# DRAM bytes per access of the in-order serve kernel from one one-pass ncu capture at the full 200 M size
-# (dram__bytes_read + write of one launch, see the summary under profiles/); scaled to the batch in use
-NCU_TRAFFIC_BYTES_PER_ACCESS = {"inorder": 42.6}
-# warp instructions the in-order serve pass executes per access (smsp__inst_executed.sum of a one-pass ncu capture at
-# 200 M, profiles/inorder_path_capacity_20M.md) and the SM's issue rate: 148 SMs x 4 schedulers x one instruction per cycle
-NCU_WARP_INSTR_PER_ACCESS = {"inorder": 7.76}
+# Profiler counters of the dominant kernel (DRAM bytes and warp instructions per access) are not typed in here: they come
+# from a small tracked file that names the kernel source it was captured on; when that source has changed since, the
+# bench reports no traffic and no instruction roofline rather than stale ones.
+COUNTERS_FILE = os.path.join(ROOT, "profiles", "inorder_serve_capacity_200M.json")
+KERNEL_SOURCES = {"inorder": os.path.join(ROOT, "paper_2609_09800_b200", "csrc", "inorder_kernels.cu")}
+
+
+def profiled_counters(kernel: str):
+    """{'dram_bytes_per_access', 'warp_instr_per_access', ...} of an ncu capture of this kernel's present source, or None."""
+    import hashlib
+    try:
+        with open(COUNTERS_FILE) as f:
+            rec = json.load(f)
+        with open(KERNEL_SOURCES[kernel], "rb") as f:
+            sha = hashlib.sha256(f.read()).hexdigest()
+    except Exception:
+        return None
+    return rec if rec.get("kernel") == kernel and rec.get("source_sha256") == sha else None
+
+
 SM_COUNT, SCHEDULERS_PER_SM = 148, 4
 FALLBACK_HBM_GBS = 6650.0
 
@@ -51,11 +65,14 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--n", type=int, default=200_000_000, help="accesses per batch (default: the capacity-mode config)")
     ap.add_argument("--path", default="auto", choices=["auto", "sort", "sort_full"])
-    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--e2e-chunk", type=int, default=12_500_000, help="records per chunk of the end-to-end pipeline")
     ap.add_argument("--cpu-sample", type=int, default=20_000_000)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-configs", action="store_true", help="skip the per-configuration block (other streams, coupled run)")
+    ap.add_argument("--shuffle", action="store_true", help="submit the records in a random order: the sort path has to serve the batch")
+    ap.add_argument("--profile", default="nominal", choices=["nominal", "aggressive"], help="timing profile of the coupled_thermal run")
     ap.add_argument("--workload", default="capacity_mode", choices=["capacity_mode", "coupled_thermal", "capacity_paged", "rom", "capacity_retention"],
                     help="coupled_thermal: the prefix-KV stream in 1 ms batches, each followed by a thermal step; "
                          "capacity_paged: the capacity-mode batch through the page-granular submit; rom: fit the reduced-order "
@@ -167,6 +184,31 @@ def cpu_oracle_rate(w, sample: int, repeats: int = 1):
     return acc.shape[0] / min(times), times
 
 
+def cpu_oracle_rate_all_cores(w, sample: int):
+    """The same oracle on all host cores: queues are independent, so the sample is dealt to one oracle instance per core
+    by channel (a channel's queues stay together) and the instances run side by side (plain threads around the C call).
+    Returns (accesses/s, cores, seconds, sum of stalls) -- the sum lets the caller check the dealing against the one-core run."""
+    from concurrent.futures import ThreadPoolExecutor
+    from oracle import hbfo
+    cores = max(1, len(os.sched_getaffinity(0)))
+    acc = w.acc[:sample]
+    stripe = int(w.profile["stripe_bytes"]).bit_length() - 1
+    channel = ((acc["addr"] - np.uint64(w.ranges[0][0])) >> np.uint64(stripe)) % np.uint64(w.profile["channels"])
+    groups = min(cores, int(w.profile["channels"]))
+    subs = [np.ascontiguousarray(acc[(channel % np.uint64(groups)) == np.uint64(g)]) for g in range(groups)]
+    oracles = []
+    for _ in range(groups):
+        o = hbfo.Oracle(w.profile)
+        for r in w.ranges:
+            o.register_range(*r)
+        oracles.append(o)
+    with ThreadPoolExecutor(groups) as pool:
+        t = time.perf_counter()
+        outs = list(pool.map(lambda g: oracles[g].submit(subs[g]), range(groups)))
+        dt = time.perf_counter() - t
+    return acc.shape[0] / dt, groups, dt, int(sum(int(o[2].sum()) for o in outs))
+
+
 def run_reference(args, rank: int):
     """The CPU oracle on this machine's host cores: each step is a bounded sample of the workload."""
     if rank != 0:
@@ -195,25 +237,63 @@ def run_reference(args, rank: int):
     print(json.dumps(line), flush=True)
 
 
-def run_coupled(args):
-    """Long-run coupled mode on one GPU: 1 ms batches of the prefix-KV stream, a thermal step after each."""
+def time_one_batch(hbf, w, path, repeats: int = 3):
+    """hbf_submit_batch alone on one stream of records, device-resident, on idle queues: best of `repeats` after a warm-up."""
     import torch
-    from paper_2609_09800_b200 import build as hbf_build, hbf
-    hbf_build.build()
-    t0 = time.time()
-    w = wl.prefix_kv()
+    ctx = hbf.Context(w.profile)
+    for r in w.ranges:
+        ctx.register_range(*r)
+    ctx.set_path(path)
+    n = w.n
+    d_acc = torch.from_numpy(w.acc.view(np.int64).reshape(-1)).cuda()
+    d_comp = torch.empty(n, dtype=torch.int64, device="cuda"); d_stall = torch.empty_like(d_comp)
+    d_status = torch.empty(n, dtype=torch.uint8, device="cuda")
+    d_stats = torch.empty(ctx.n_dies * 6, dtype=torch.int64, device="cuda")
+    ws = ctx.workspace(n)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    best = None
+    for k in range(repeats + 1):
+        ctx.reset(); flush.fill_(1)
+        e0.record(); rc = ctx.submit_batch(d_acc, n, d_comp, d_stall, d_status, d_stats, ws); e1.record(); e1.synchronize()
+        assert rc == 0 and ctx.last_result()["code"] == 0
+        if k:
+            best = e0.elapsed_time(e1) if best is None else min(best, e0.elapsed_time(e1))
+    ctx.destroy()
+    del d_acc, d_comp, d_stall, d_status, d_stats, ws, flush
+    return {"accesses": n, "ms": round(best, 4), "accesses_per_s": n / (best * 1e-3)}
+
+
+def other_configs(hbf, args):
+    """The other configurations of the benchmark definition, one batch each on idle queues (in-order path as the library
+    chooses it, and the sort path forced), and the long coupled run per step.  Reported beside the headline."""
+    out = {}
+    streams = [("tiny_uniform_65k", lambda: wl.tiny_uniform()), ("decode_weights_256_tokens", lambda: wl.decode_weights(256)),
+               ("decode_weights_48_tokens", lambda: wl.decode_weights(48)), ("prefix_kv", lambda: wl.prefix_kv())]
+    kv = None
+    for name, make in streams:
+        w = make()
+        out[name] = {"auto": time_one_batch(hbf, w, hbf.PATH_AUTO), "sort_forced": time_one_batch(hbf, w, hbf.PATH_SORT)}
+        if name == "prefix_kv":
+            kv = w
+    out["coupled_thermal_10s"] = coupled_run(hbf, kv, 10_000, hbf.PATH_AUTO)
+    return out
+
+
+def coupled_run(hbf, w, n_steps: int, path, energy_bins=False, retention=False):
+    """1 ms batches of the prefix-KV stream, device-resident, a thermal step after each: device time per (submit + step)."""
+    import torch
     fp = wl.package_floorplan()
-    batches = [b for _, b in wl.timed_batches(w, args.horizon_ms * 1_000_000)]
+    batches = [b for _, b in wl.timed_batches(w, n_steps * 1_000_000)]
     sizes = [b.shape[0] for b in batches]
     allrec = np.concatenate(batches)
-    gen_s = time.time() - t0
     ctx = hbf.Context(w.profile, fp)
     for r in w.ranges:
         ctx.register_range(*r)
-    ctx.set_path(hbf.PATH_INORDER)             # the caller knows its stream is in issue order: no sort kernels are launched
-    if args.energy_bins:
+    ctx.set_path(path)
+    if energy_bins:
         ctx.enable_energy_bins(1_000_000, 64)
-    if args.retention:
+    if retention:
         ctx.enable_retention(pages_per_block=64, blocks_per_plane=64, blocks_per_zone=8, max_pec=3000, disturb_limit=0,
                              l_ref_s=3.15e7, t_ref_c=40.0, ea_ev=1.04, accel=2.0e6, lead_threshold=0.8)
     d_all = torch.from_numpy(allrec.view(np.int64).reshape(-1, 3)).cuda()
@@ -225,34 +305,54 @@ def run_coupled(args):
     ext = fp["ext_power_w"]
 
     def run():
+        refused = 0
         for k, nk in enumerate(sizes):
             rc = ctx.submit_batch(d_all[offs[k]:offs[k + 1]], nk, d_comp, d_stall, None, d_stats, ws)
-            assert rc == 0, rc
+            if rc != 0:                                      # (the controller shut the link down: later batches are refused)
+                refused += 1
             ctx.thermal_step(1_000_000, ext, None, want_hot=False)
-            if args.retention:
+            if retention:
                 ctx.retention_advance(1_000_000)
+        return refused
     ctx.reset(); run(); torch.cuda.synchronize()               # warm-up pass over the same horizon
     ctx.reset()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     l0 = hbf.kernel_launches()
     t_host = time.perf_counter()
-    e0.record(); run(); e1.record(); torch.cuda.synchronize()
+    e0.record(); refused = run(); e1.record(); torch.cuda.synchronize()
     wall = time.perf_counter() - t_host
     ms = e0.elapsed_time(e1)
     hot = ctx.thermal_step(1_000_000, ext)
     mode, q = ctx.get_mode()
-    n_acc = int(offs[-1])
-    line = {"metric": METRIC, "value": n_acc / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": len(sizes), "warmup": len(sizes),
-            "ms_per_step": ms / len(sizes), "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64",
-            "data": "synthetic",
-            "config": {"workload": "coupled_thermal", "accesses": n_acc, "mean_accesses_per_step": n_acc / len(sizes),
-                       "simulated_ms": args.horizon_ms, "geometry": "32x8x4", "path": "inorder (declared by the caller)",
+    res = {"steps": len(sizes), "accesses": int(offs[-1]), "us_per_submit_plus_step": ms * 1e3 / len(sizes), "device_ms": ms,
+           "host_wall_s": round(wall, 3), "gpu_launches": int(hbf.kernel_launches() - l0), "batches_refused_at_launch": refused,
+           "path": "auto" if path == hbf.PATH_AUTO else "inorder (declared by the caller)",
+           "final": {"hot_c": [round(float(x), 3) for x in hot], "mode": mode, "q_ppm": q}}
+    if retention:
+        res["retention"] = ctx.retention_totals()
+    ctx.destroy()
+    return res
+
+
+def run_coupled(args):
+    """Long-run coupled mode on one GPU: 1 ms batches of the prefix-KV stream, a thermal step after each."""
+    from paper_2609_09800_b200 import build as hbf_build, hbf
+    hbf_build.build()
+    t0 = time.time()
+    w = wl.prefix_kv(profile=args.profile)
+    gen_s = time.time() - t0
+    r = coupled_run(hbf, w, args.horizon_ms, hbf.PATH_INORDER, energy_bins=args.energy_bins, retention=args.retention)
+    line = {"metric": METRIC, "value": r["accesses"] / (r["device_ms"] * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": r["steps"],
+            "warmup": r["steps"], "ms_per_step": r["device_ms"] / r["steps"], "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+            "config": {"workload": "coupled_thermal", "profile": args.profile, "accesses": r["accesses"],
+                       "mean_accesses_per_step": r["accesses"] / r["steps"],
+                       "simulated_ms": args.horizon_ms, "geometry": "32x8x4", "path": r["path"],
                        "thermal_grid": "128x128", "gen_seconds": round(gen_s, 1),
                        "energy": "1 ms bins, split by time overlap" if args.energy_bins else "charged at submit"},
-            "gpu_launches": int(hbf.kernel_launches() - l0), "host_wall_s": round(wall, 3),
-            "final": {"hot_c": [round(float(x), 3) for x in hot], "mode": mode, "q_ppm": q}}
+            "gpu_launches": r["gpu_launches"], "host_wall_s": r["host_wall_s"], "final": r["final"]}
     if args.retention:
-        line["retention"] = ctx.retention_totals()
+        line["retention"] = r["retention"]
         line["config"]["retention"] = "one epoch per thermal step, region temperatures from the field, a_t = 2e6"
     print(json.dumps(line), flush=True)
 
@@ -301,7 +401,9 @@ def run_paged(args):
     launches = hbf.kernel_launches() - l0
     peak, kind = measured_peak()
     rate = n * args.steps / (ms * 1e-3)
-    # what the split path must move: the records in, the part records out and in again, their results out and in, the results out
+    # The method's bytes: 41 per queued request (a part), whatever the implementation moves.  What this implementation moves
+    # (records in, part records out and in again, their results out and in, results out) is reported beside it.
+    algo = ALGO_BYTES_PER_ACCESS * parts
     moved = 24 * n + 2 * 24 * parts + 2 * 17 * parts + 17 * n
     line = {"metric": METRIC, "value": rate, "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64",
@@ -310,10 +412,11 @@ def run_paged(args):
                        "queues": 2048, "thermal_grid": "128x128",
                        "gen_seconds": round(gen_s, 1), "state": "queues idle at the start of every step"},
             "gpu_launches": int(launches),
-            "roofline": {"bound": "hbm", "kernel": "paged submit, all kernels", "achieved": moved * args.steps / (ms * 1e-3) / 1e9,
+            "roofline": {"bound": "hbm", "kernel": "paged submit, all kernels", "achieved": algo * args.steps / (ms * 1e-3) / 1e9,
                          "peak": peak, "peak_kind": kind, "unit": "GB/s",
-                         "frac": moved * args.steps / (ms * 1e-3) / 1e9 / peak, "traffic": None,
-                         "algorithmic_bytes_per_access": moved / n},
+                         "frac": algo * args.steps / (ms * 1e-3) / 1e9 / peak, "traffic": None,
+                         "algorithmic_bytes_per_part": ALGO_BYTES_PER_ACCESS,
+                         "implementation_bytes_moved_per_step": moved},
             "batch_result": {k: res[k] for k in ("n_modeled", "n_native", "max_completion_ns")}}
     print(json.dumps(line), flush=True)
 
@@ -368,8 +471,8 @@ def run_retention(args):
     ms = float(t.sum())
     peak, kind = measured_peak()
     rate = 2 * n * args.steps / (ms * 1e-3)
-    # per batch: the records in, completion + stall + status out (41 B), the records in again for the read-disturb pass (24 B)
-    moved = 2 * (41 + 24) * n
+    # the method's bytes: 41 per access and batch (two batches per step)
+    moved = 2 * ALGO_BYTES_PER_ACCESS * n
     line = {"metric": METRIC, "value": rate, "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64",
             "data": "synthetic",
@@ -383,7 +486,7 @@ def run_retention(args):
             "roofline": {"bound": "hbm", "kernel": "submit with retention, all kernels", "achieved": moved * args.steps / (ms * 1e-3) / 1e9,
                          "peak": peak, "peak_kind": kind, "unit": "GB/s",
                          "frac": moved * args.steps / (ms * 1e-3) / 1e9 / peak, "traffic": None,
-                         "algorithmic_bytes_per_access": 65},
+                         "algorithmic_bytes_per_access": ALGO_BYTES_PER_ACCESS},
             "batch_result": {k: res[k] for k in ("n_modeled", "n_native", "max_completion_ns")}}
     print(json.dumps(line), flush=True)
 
@@ -479,6 +582,8 @@ def main():
     sampler.start()
     n = args.n
     w, gen_s = make_stream(n, seed=replicas.rank_seed(0, rank))   # every rank: an independent replica on its own stream
+    if args.shuffle:                           # the same records in a random order (seeded): nothing is in issue order any more
+        w.acc = w.acc[np.random.Generator(np.random.PCG64([7, rank])).permutation(n)]
     fp = wl.package_floorplan(channels=w.profile["channels"], dies=w.profile["dies"])
     ctx = hbf.Context(w.profile, fp)
     for r in w.ranges:
@@ -551,7 +656,7 @@ def main():
 
     # end to end through the C ABI with host buffers: H2D of the records, submit + thermal step, D2H of results
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not args.shuffle:   # (the chunked host call equals one batch only for records in issue order)
         h_in = h_acc.pin_memory()
         h_comp = torch.empty(n, dtype=torch.int64).pin_memory()
         h_stall = torch.empty(n, dtype=torch.int64).pin_memory()
@@ -561,7 +666,7 @@ def main():
 
         def e2e_step():
             # the public host-buffer call: chunks of the batch are copied in, served and read back on three streams
-            rc = ctx.submit_pinned(h_in, n, h_comp, h_stall, h_stats, chunk=e2e_chunk)
+            rc, _ = ctx.submit_pinned(h_in, n, h_comp, h_stall, h_stats, chunk=e2e_chunk)
             assert rc == 0, rc
             ctx.thermal_step(1_000_000, ext, None, want_hot=False)
         ctx.reset(); e2e_step(); sync_all()
@@ -571,7 +676,7 @@ def main():
         e2e_units, ms = replicas.combine(n * args.e2e_steps, ms, device="cuda")
         e2e = {"value": e2e_units / (ms * 1e-3), "unit": UNIT, "steps": args.e2e_steps,
                "h2d_bytes_per_step": n * 24, "d2h_bytes_per_step": n * 16 + ctx.n_dies * 48,
-               "call": "Context.submit_pinned: %d chunks, copy-in / service / read-back overlapped on three streams" % (-(-n // e2e_chunk))}
+               "call": "hbf_submit_host (C ABI, pinned host buffers): %d chunks, copy-in / service / read-back overlapped on three streams" % (-(-n // e2e_chunk))}
 
     if rank == 0:
         peak, peak_kind = measured_peak()
@@ -585,24 +690,27 @@ def main():
         else:
             dom_bytes = STAGE_BYTES[dom]; per_launch_ms = med[dom]
         achieved = dom_bytes * n / (per_launch_ms * 1e-3) / 1e9 if per_launch_ms > 0 else 0.0
-        traffic = NCU_TRAFFIC_BYTES_PER_ACCESS.get(dom)
+        counters = profiled_counters(dom) if dom in KERNEL_SOURCES else None
         roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
-                    "frac": achieved / peak, "traffic": traffic * n if traffic else None,
+                    "frac": achieved / peak, "traffic": counters["dram_bytes_per_access"] * n if counters else None,
+                    "traffic_source": (os.path.relpath(COUNTERS_FILE, ROOT) if counters else
+                                       "none: no capture of the present kernel source under profiles/"),
                     "algorithmic_bytes_per_access": dom_bytes, "ms_per_launch": per_launch_ms}
-        if dom in NCU_WARP_INSTR_PER_ACCESS and per_launch_ms > 0:
+        if counters and per_launch_ms > 0:
             # the same kernel against the issue rate at the clock sampled during the timed region: what actually binds it
             mhz = (clocks or {}).get("sm_mhz") or 1965.0
             issue_peak = SM_COUNT * SCHEDULERS_PER_SM * mhz * 1e6
-            issued = NCU_WARP_INSTR_PER_ACCESS[dom] * n / (per_launch_ms * 1e-3)
+            issued = counters["warp_instr_per_access"] * n / (per_launch_ms * 1e-3)
             roofline["alu"] = {"achieved": issued / 1e12, "peak": issue_peak / 1e12, "unit": "T warp instructions/s",
-                               "frac": issued / issue_peak, "warp_instructions_per_access": NCU_WARP_INSTR_PER_ACCESS[dom],
+                               "frac": issued / issue_peak, "warp_instructions_per_access": counters["warp_instr_per_access"],
                                "note": "instruction count from an ncu capture, time measured live"}
         path_gbs = ALGO_BYTES_PER_ACCESS * value / world / 1e9
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
                 "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": "int64", "data": "synthetic",
                 "config": {"workload": "capacity_mode", "accesses_per_step": n, "geometry": "64x8x4", "queues": 2048,
-                           "path": args.path, "channel_bus_stage": bool(args.channel_bus), "thermal_grid": "128x128", "l2": "inputs (%.1f GB) larger than L2" % (n * 24 / 1e9),
+                           "path": args.path, "input_order": "shuffled" if args.shuffle else "issue order",
+                           "channel_bus_stage": bool(args.channel_bus), "thermal_grid": "128x128", "l2": "inputs (%.1f GB) larger than L2, and a 256 MB write before every timed step" % (n * 24 / 1e9),
                            "multi_gpu": "replicas only", "gen_seconds": round(gen_s, 1),
                            "state": "queues idle at the start of every step (reset outside the timed region)"},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
@@ -614,8 +722,16 @@ def main():
         if world == 1 and not args.no_cpu_baseline:
             sample = min(n, args.cpu_sample)
             rate, times = cpu_oracle_rate(w, sample)
-            line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": 1, "kind": "oracle",
-                                    "sample": "first %d accesses of the same stream, one pass (%.1f s)" % (sample, min(times))}
+            rate_all, cores, dt_all, _ = cpu_oracle_rate_all_cores(w, sample)
+            line["cpu_baseline"] = {"value": rate_all, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                    "sample": "first %d accesses of the same stream, one pass, dealt by channel to one oracle "
+                                              "instance per core (%.1f s)" % (sample, dt_all),
+                                    "one_core": {"value": rate, "cores": 1, "seconds": round(min(times), 2)}}
+        if world == 1 and not args.no_configs:
+            del d_acc, d_comp, d_stall, d_status, ws
+            ctx.destroy()
+            torch.cuda.empty_cache()
+            line["configs"] = other_configs(hbf, args)
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.barrier()

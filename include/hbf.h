@@ -132,6 +132,22 @@ HBF_API int hbf_submit_batch(hbf_ctx *ctx, const hbf_access_t *d_acc, uint64_t n
                      int64_t *d_stall_ns, uint8_t *d_status, hbf_die_stats_t *d_die_stats,
                      void *d_workspace, size_t workspace_bytes);
 
+/* The same service for a batch that lives in HOST memory (no step of the method is defined by this call, so it cites
+ * none: it is hbf_submit_batch behind a copy pipeline).  The batch is cut into chunks of `chunk` records (0 = a default
+ * of 12.5 M); the copy-in of chunk k+1, the service of chunk k and the read-back of chunk k-1 run on three streams of
+ * the library, so both directions of the link are busy while the kernels run.  Equivalent to one hbf_submit_batch per
+ * chunk, in order: for records in issue order that is the same as one batch.
+ * h_acc [n] host, read only; h_completion_ns, h_stall_ns [n] host; h_die_stats [channels*dies] host, nullable: totals
+ * over the chunks.  Pinned host memory (cudaMallocHost / cudaHostRegister) makes the copies asynchronous and
+ * overlapped; pageable memory works, slower.  The library owns the device buffers (two chunks of records and results,
+ * one workspace), allocated at the first call and kept until hbf_destroy; a larger chunk reallocates them.
+ * The call returns when every result is in the caller's buffers.  summary_out (host, nullable) receives the chunks'
+ * summaries added up (counts and times summed, the largest completion, mode and q of the first chunk) with code =
+ * the first chunk code that is not HBF_OK; that code is also the return value.  A refused chunk (fail-closed access,
+ * throttled) leaves zeros in its part of the outputs and changes no state; later chunks are still served. */
+HBF_API int hbf_submit_host(hbf_ctx *ctx, const hbf_access_t *h_acc, uint64_t n, int64_t *h_completion_ns,
+                            int64_t *h_stall_ns, hbf_die_stats_t *h_die_stats, uint64_t chunk, hbf_batch_result_t *summary_out);
+
 /* Page-granular variant of hbf_submit_batch (an extension: the paper's back end is a page-based flash simulator,
  * Section "Design", but the text does not define the splitting; this is the library's definition).  A modeled
  * access is cut at the page boundaries of the media; every part is a request of its own: decoded by its own

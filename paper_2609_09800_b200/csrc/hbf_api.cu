@@ -54,6 +54,15 @@ struct hbf_ctx {
     // thermal
     bool thermal = false; ThermalDev td{}; int cur = 0; double euler_limit_s = 0.0; bool thermal_generic = false;
     std::vector<void *> owned;
+    // host-buffer pipeline of hbf_submit_host (allocated at its first use, sized for the largest chunk seen)
+    struct HostPipe {
+        uint64_t chunk = 0; size_t ws_bytes = 0;
+        hbf_access_t *acc[2] = {}; int64_t *comp[2] = {}, *stall[2] = {}; hbf_die_stats_t *stats = nullptr, *total = nullptr; void *ws = nullptr;
+        hbf_batch_result_t *d_sum = nullptr, *h_sum = nullptr;          // the chunks' summaries added up: device, and pinned
+        cudaStream_t s_in = nullptr, s_out = nullptr;
+        cudaEvent_t arrived[2] = {}, served[2] = {}, read[2] = {}, start = nullptr;
+        bool made = false;
+    } pipe;
 };
 
 #define CK(expr) do { cudaError_t e_ = (expr); if (e_ != cudaSuccess) return HBF_E_CUDA; } while (0)
@@ -227,6 +236,15 @@ int hbf_destroy(hbf_ctx *c) {
     if (c->d_rom_p) cudaFree(c->d_rom_p);
     if (c->h_hot) cudaFreeHost(c->h_hot);
     if (c->h_ext) cudaFreeHost(c->h_ext);
+    if (c->pipe.made) {
+        hbf_ctx::HostPipe &p = c->pipe;
+        cudaStreamSynchronize(p.s_in); cudaStreamSynchronize(p.s_out);
+        for (int k = 0; k < 2; ++k) { cudaFree(p.acc[k]); cudaFree(p.comp[k]); cudaFree(p.stall[k]); cudaEventDestroy(p.arrived[k]); cudaEventDestroy(p.served[k]); cudaEventDestroy(p.read[k]); }
+        cudaFree(p.stats); cudaFree(p.total); cudaFree(p.ws); cudaEventDestroy(p.start);
+        if (p.h_sum) cudaFreeHost(p.h_sum);
+        cudaFree(p.d_sum);
+        cudaStreamDestroy(p.s_in); cudaStreamDestroy(p.s_out);
+    }
     delete c;
     return HBF_OK;
 }
@@ -450,6 +468,86 @@ int hbf_submit_batch(hbf_ctx *c, const hbf_access_t *d_acc, uint64_t n, int64_t 
         CK(launch_bus_stage(a, c->d_bus_ctrl, c->d_bus_busy, c->stream));
     c->submitted = true;
     return HBF_OK;
+}
+
+// Host-buffer submit: the batch is cut into chunks; the copy-in of chunk k+1, the service of chunk k (hbf_submit_batch)
+// and the read-back of chunk k-1 run on three streams, so the link moves both ways while the kernels run.
+static int host_pipe_prepare(hbf_ctx *c, uint64_t chunk) {
+    hbf_ctx::HostPipe &p = c->pipe;
+    if (!p.made) {
+        CK(cudaStreamCreateWithFlags(&p.s_in, cudaStreamNonBlocking));
+        CK(cudaStreamCreateWithFlags(&p.s_out, cudaStreamNonBlocking));
+        for (int k = 0; k < 2; ++k) {
+            CK(cudaEventCreateWithFlags(&p.arrived[k], cudaEventDisableTiming));
+            CK(cudaEventCreateWithFlags(&p.served[k], cudaEventDisableTiming));
+            CK(cudaEventCreateWithFlags(&p.read[k], cudaEventDisableTiming));
+        }
+        CK(cudaEventCreateWithFlags(&p.start, cudaEventDisableTiming));
+        if (cudaMalloc(&p.stats, (size_t)c->mp.n_dies * sizeof(hbf_die_stats_t)) != cudaSuccess) return HBF_E_NOMEM;
+        if (cudaMalloc(&p.total, (size_t)c->mp.n_dies * sizeof(hbf_die_stats_t)) != cudaSuccess) return HBF_E_NOMEM;
+        if (cudaMalloc(&p.d_sum, sizeof(hbf_batch_result_t)) != cudaSuccess) return HBF_E_NOMEM;
+        if (cudaMallocHost(&p.h_sum, sizeof(hbf_batch_result_t)) != cudaSuccess) return HBF_E_NOMEM;
+        p.made = true;
+    }
+    const size_t ws_need = hbf_workspace_bytes(c, chunk);
+    if (chunk > p.chunk || ws_need > p.ws_bytes) {
+        CK(cudaStreamSynchronize(c->stream)); CK(cudaStreamSynchronize(p.s_in)); CK(cudaStreamSynchronize(p.s_out));
+        for (int k = 0; k < 2; ++k) {
+            cudaFree(p.acc[k]); cudaFree(p.comp[k]); cudaFree(p.stall[k]); p.acc[k] = nullptr; p.comp[k] = p.stall[k] = nullptr;
+            if (cudaMalloc(&p.acc[k], chunk * sizeof(hbf_access_t)) != cudaSuccess || cudaMalloc(&p.comp[k], chunk * 8) != cudaSuccess ||
+                cudaMalloc(&p.stall[k], chunk * 8) != cudaSuccess) { p.chunk = 0; return HBF_E_NOMEM; }
+        }
+        cudaFree(p.ws); p.ws = nullptr;
+        if (cudaMalloc(&p.ws, ws_need) != cudaSuccess) { p.chunk = 0; p.ws_bytes = 0; return HBF_E_NOMEM; }
+        p.chunk = chunk; p.ws_bytes = ws_need;
+    }
+    return HBF_OK;
+}
+
+int hbf_submit_host(hbf_ctx *c, const hbf_access_t *h_acc, uint64_t n, int64_t *h_completion_ns, int64_t *h_stall_ns,
+                    hbf_die_stats_t *h_die_stats, uint64_t chunk, hbf_batch_result_t *summary_out) {
+    if (!c || !on_own_device(c)) return HBF_E_INVAL;
+    if (c->terminal) return HBF_E_LINK_SHUTDOWN;
+    if (n && (!h_acc || !h_completion_ns || !h_stall_ns)) return HBF_E_INVAL;
+    if (chunk == 0) chunk = 12500000;
+    chunk = std::min<uint64_t>(std::min<uint64_t>(chunk, HBF_MAX_BATCH), std::max<uint64_t>(n, 1));
+    int rc = host_pipe_prepare(c, chunk);
+    if (rc != HBF_OK) return rc;
+    hbf_ctx::HostPipe &p = c->pipe;
+    cudaStream_t main = c->stream;
+    CK(cudaEventRecord(p.start, main));                      // the side streams begin behind what the context has enqueued so far
+    CK(cudaStreamWaitEvent(p.s_in, p.start, 0)); CK(cudaStreamWaitEvent(p.s_out, p.start, 0));
+    CK(cudaMemsetAsync(p.total, 0, (size_t)c->mp.n_dies * sizeof(hbf_die_stats_t), main));
+    bool served[2] = {false, false}, read[2] = {false, false};
+    size_t k = 0;
+    for (uint64_t lo = 0; lo < n; lo += chunk, ++k) {
+        const uint64_t m = std::min<uint64_t>(chunk, n - lo);
+        const int s = (int)(k & 1);
+        if (served[s]) CK(cudaStreamWaitEvent(p.s_in, p.served[s], 0));   // the slot's records have been read by the chunk before last
+        CK(cudaMemcpyAsync(p.acc[s], h_acc + lo, m * sizeof(hbf_access_t), cudaMemcpyHostToDevice, p.s_in));
+        CK(cudaEventRecord(p.arrived[s], p.s_in));
+        CK(cudaStreamWaitEvent(main, p.arrived[s], 0));
+        if (read[s]) CK(cudaStreamWaitEvent(main, p.read[s], 0));         // the slot's results have left
+        rc = hbf_submit_batch(c, p.acc[s], m, p.comp[s], p.stall[s], nullptr, p.stats, p.ws, p.ws_bytes);
+        if (rc != HBF_OK) break;
+        CK(launch_add_stats(p.total, p.stats, c->mp.n_dies, main));       // (a refused chunk leaves zeros)
+        CK(launch_add_result(p.d_sum, c->d_result, k == 0 ? 1 : 0, main));
+        CK(cudaEventRecord(p.served[s], main)); served[s] = true;
+        CK(cudaStreamWaitEvent(p.s_out, p.served[s], 0));
+        CK(cudaMemcpyAsync(h_completion_ns + lo, p.comp[s], m * 8, cudaMemcpyDeviceToHost, p.s_out));
+        CK(cudaMemcpyAsync(h_stall_ns + lo, p.stall[s], m * 8, cudaMemcpyDeviceToHost, p.s_out));
+        CK(cudaEventRecord(p.read[s], p.s_out)); read[s] = true;
+    }
+    for (int s = 0; s < 2; ++s) if (read[s]) CK(cudaStreamWaitEvent(main, p.read[s], 0));
+    if (rc != HBF_OK) { cudaStreamSynchronize(main); return rc; }
+    if (k) CK(cudaMemcpyAsync(p.h_sum, p.d_sum, sizeof(hbf_batch_result_t), cudaMemcpyDeviceToHost, main));
+    if (h_die_stats) CK(cudaMemcpyAsync(h_die_stats, p.total, (size_t)c->mp.n_dies * sizeof(hbf_die_stats_t), cudaMemcpyDeviceToHost, main));
+    CK(cudaStreamSynchronize(main));                         // results, totals and the chunks' summaries are on the host
+    hbf_batch_result_t sum; memset(&sum, 0, sizeof(sum));
+    if (k) sum = *p.h_sum;
+    if (sum.code == HBF_E_LINK_SHUTDOWN) c->terminal = true;
+    if (summary_out) *summary_out = sum;
+    return sum.code;
 }
 
 size_t hbf_workspace_bytes_paged(const hbf_ctx *c, uint64_t n, uint64_t parts_capacity) {

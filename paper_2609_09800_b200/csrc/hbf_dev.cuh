@@ -156,6 +156,10 @@ size_t inorder_head_bytes(uint64_t tiles, uint32_t n_queues);
 size_t inorder_serve_smem(uint32_t n_dies);
 cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st);
 cudaError_t launch_submit(const SubmitArgs &a, cudaStream_t st);
+// total[i] += part[i] over the 6 * n_dies counters of a per-die statistics array (host-buffer pipeline: totals over its chunks)
+cudaError_t launch_add_stats(hbf_die_stats_t *total, const hbf_die_stats_t *part, uint32_t n_dies, cudaStream_t st);
+// the same for batch summaries: counts and times added, the largest completion, the first code that is not HBF_OK; first != 0 starts over
+cudaError_t launch_add_result(hbf_batch_result_t *sum, const hbf_batch_result_t *part, int first, cudaStream_t st);
 cudaError_t launch_queue_order(const BatchCtrl *ctrl, const Workspace &ws, uint32_t *out, uint64_t n, cudaStream_t st);
 
 // ---- page-granular submit ---------------------------------------------------------------------------

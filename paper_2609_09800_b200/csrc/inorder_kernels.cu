@@ -646,7 +646,7 @@ constexpr int kInStrWarps = kInStrThreads / 32;
 constexpr int kInStrQItems = 32;                          // records per thread and turn inside the queue-number prefix
 constexpr int kInStrQChunk = kInStrThreads * kInStrQItems;
 constexpr int kInStrKeep = 1024;                          // kept records served at a time (a chunk with more is served in windows)
-constexpr int kInStrMaxStragglers = 128;                   // a tile with as many is served again whole instead
+constexpr int kInStrMaxStragglers = 255;                   // a tile with as many is served again whole instead (a queue's place, plus one, is a byte)
 constexpr int kInStrList = 32;                            // records of one queue in a window that its list holds (more: the window is scanned)
 constexpr int kInStrQueuesPerThread = (kInMaxQueues + kInStrThreads - 1) / kInStrThreads;
 static_assert(kInStrQChunk <= 65536, "a kept record's position in its chunk is stored in 16 bits");
@@ -749,7 +749,9 @@ k_inorder_fixstraggle(const hbf_access_t *__restrict__ acc, uint64_t n, const __
     }
     __syncthreads();
     const uint32_t stragglers = s_stragglers;
-    if (stragglers >= min(max(8u, R / 16u), (uint32_t)kInStrMaxStragglers)) {   // many queues far behind: the re-serve pass takes the whole tile
+    // many queues far behind: the re-serve pass takes the whole tile (one block serves it again from end to end, which costs
+    // as much as the serve pass itself, so the bar is as high as this loop's tables allow)
+    if (stragglers >= min(max(8u, R / 4u), (uint32_t)kInStrMaxStragglers)) {
         if (tid == 0) in_tile[tile].reserve = 1u;
         return;
     }

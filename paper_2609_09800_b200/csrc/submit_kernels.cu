@@ -1132,6 +1132,34 @@ cudaError_t launch_submit(const SubmitArgs &a, cudaStream_t st) {
     return cudaGetLastError();
 }
 
+__global__ void k_add_stats(long long *total, const long long *part, uint32_t words) {
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < words) total[i] += part[i];
+}
+cudaError_t launch_add_stats(hbf_die_stats_t *total, const hbf_die_stats_t *part, uint32_t n_dies, cudaStream_t st) {
+    const uint32_t words = n_dies * 6u;
+    k_add_stats<<<(words + 255) / 256, 256, 0, st>>>(reinterpret_cast<long long *>(total), reinterpret_cast<const long long *>(part), words);
+    g_kernel_launches += 1;
+    return cudaGetLastError();
+}
+
+__global__ void k_add_result(hbf_batch_result_t *sum, const hbf_batch_result_t *part, int first) {
+    hbf_batch_result_t s = *sum; const hbf_batch_result_t r = *part;
+    if (first) { s = r; }
+    else {
+        if (s.code == HBF_OK && r.code != HBF_OK) s.code = r.code;
+        s.n_native += r.n_native; s.n_modeled += r.n_modeled; s.n_fault += r.n_fault;
+        s.modeled_ns += r.modeled_ns; s.service_ns += r.service_ns;
+        s.max_completion_ns = max(s.max_completion_ns, r.max_completion_ns);
+    }
+    *sum = s;
+}
+cudaError_t launch_add_result(hbf_batch_result_t *sum, const hbf_batch_result_t *part, int first, cudaStream_t st) {
+    k_add_result<<<1, 1, 0, st>>>(sum, part, first);
+    g_kernel_launches += 1;
+    return cudaGetLastError();
+}
+
 cudaError_t launch_queue_order(const BatchCtrl *ctrl, const Workspace &ws, uint32_t *out, uint64_t n, cudaStream_t st) {
     if (n == 0) return cudaSuccess;
     k_queue_order<<<(unsigned)std::min<uint64_t>((n + 255) / 256, 1184), 256, 0, st>>>(ctrl, ws.idx[0], ws.idx[1], out, n);

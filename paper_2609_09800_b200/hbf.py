@@ -30,7 +30,7 @@ EXPORTS = ("hbf_create", "hbf_destroy", "hbf_register_range", "hbf_clear_ranges"
            "hbf_reset", "hbf_set_path", "hbf_get_state", "hbf_set_state", "hbf_get_busy_until",
            "hbf_get_pending_energy", "hbf_get_temps", "hbf_euler_limit_ns", "hbf_queue_order", "hbf_strerror",
            "hbf_set_profiling", "hbf_get_profile", "hbf_kernel_launches", "hbf_euler_substeps_static", "hbf_set_thermal_path",
-           "hbf_workspace_bytes_paged", "hbf_submit_batch_paged",
+           "hbf_workspace_bytes_paged", "hbf_submit_batch_paged", "hbf_submit_host",
            "hbf_enable_energy_bins", "hbf_get_energy_bins", "hbf_enable_channel_bus", "hbf_get_bus_busy_until",
            "hbf_rom_create", "hbf_rom_destroy", "hbf_rom_reset", "hbf_rom_step", "hbf_rom_get_state",
            "hbf_attach_rom", "hbf_get_rom_temps",
@@ -104,6 +104,7 @@ def lib():
         L.hbf_workspace_bytes.argtypes = [vp, u64]
         L.hbf_workspace_bytes.restype = C.c_size_t
         L.hbf_submit_batch.argtypes = [vp, vp, u64, vp, vp, vp, vp, vp, C.c_size_t]
+        L.hbf_submit_host.argtypes = [vp, vp, u64, vp, vp, vp, u64, C.POINTER(hbf_batch_result_t)]
         L.hbf_workspace_bytes_paged.argtypes = [vp, u64, u64]
         L.hbf_workspace_bytes_paged.restype = C.c_size_t
         L.hbf_submit_batch_paged.argtypes = [vp, vp, u64, u64, vp, vp, vp, vp, vp, C.c_size_t]
@@ -485,61 +486,15 @@ class Context:
         if rc != 0:
             raise HbfError(rc, "hbf_set_state")
 
-    # ---- pinned host buffers, streamed: copy-in, service and read-back of consecutive chunks overlap ----------
-    def submit_pinned(self, h_acc, n, h_completion, h_stall, h_die_stats=None, chunk=25_000_000):
-        """Serves a batch that lives in pinned host memory, chunk by chunk: while chunk k is served on the context's
-        stream, chunk k+1 is copied in and the results of chunk k-1 are copied out on two copy streams (PCIe moves
-        both ways at once).  Equivalent to one ``hbf_submit_batch`` per chunk, in order: for records in issue order
-        that is the same as one batch.  h_acc: pinned int64 tensor [3 n] (the records); h_completion, h_stall:
-        pinned int64 [n]; h_die_stats: pinned int64 [6 dies] or None (summed over the chunks).  Everything is
-        enqueued when the call returns; the context's stream has the read-backs as its last dependency."""
-        torch = self._torch
-        main = self.stream
-        chunk = max(1, min(int(chunk), n if n else 1))
-        pipe = getattr(self, "_pipe", None)
-        if pipe is None or pipe["chunk"] < chunk:
-            dev = dict(dtype=torch.int64, device="cuda")
-            pipe = dict(chunk=chunk, acc=[torch.empty(chunk * 3, **dev) for _ in range(2)],
-                        comp=[torch.empty(chunk, **dev) for _ in range(2)], stall=[torch.empty(chunk, **dev) for _ in range(2)],
-                        stats=torch.empty(self.n_dies * 6, **dev), total=torch.empty(self.n_dies * 6, **dev),
-                        ws=torch.empty(self.workspace_bytes(chunk), dtype=torch.uint8, device="cuda"),
-                        s_in=torch.cuda.Stream(), s_out=torch.cuda.Stream())
-            self._pipe = pipe
-        s_in, s_out = pipe["s_in"], pipe["s_out"]
-        start = torch.cuda.Event(); start.record(main)
-        s_in.wait_event(start); s_out.wait_event(start)
-        with torch.cuda.stream(main):
-            pipe["total"].zero_()
-        served, read = [None, None], [None, None]
-        rc = 0
-        for k, lo in enumerate(range(0, n, chunk)):
-            hi = min(n, lo + chunk); m = hi - lo; s = k & 1
-            with torch.cuda.stream(s_in):
-                if served[s] is not None:
-                    s_in.wait_event(served[s])               # the slot's records have been read by the chunk before last
-                pipe["acc"][s][:m * 3].copy_(h_acc[lo * 3:hi * 3], non_blocking=True)
-                arrived = torch.cuda.Event(); arrived.record(s_in)
-            main.wait_event(arrived)
-            if read[s] is not None:
-                main.wait_event(read[s])                     # the slot's results have left
-            with torch.cuda.stream(main):
-                rc = self.submit_batch(pipe["acc"][s], m, pipe["comp"][s], pipe["stall"][s], None, pipe["stats"], pipe["ws"])
-                if rc != 0:
-                    break
-                pipe["total"] += pipe["stats"]
-                served[s] = torch.cuda.Event(); served[s].record(main)
-            with torch.cuda.stream(s_out):
-                s_out.wait_event(served[s])
-                h_completion[lo:hi].copy_(pipe["comp"][s][:m], non_blocking=True)
-                h_stall[lo:hi].copy_(pipe["stall"][s][:m], non_blocking=True)
-                read[s] = torch.cuda.Event(); read[s].record(s_out)
-        for e in read:
-            if e is not None:
-                main.wait_event(e)
-        if h_die_stats is not None and rc == 0:
-            with torch.cuda.stream(main):
-                h_die_stats.copy_(pipe["total"], non_blocking=True)
-        return rc
+    # ---- host buffers through the library's copy pipeline --------------------------------------------------------
+    def submit_pinned(self, h_acc, n, h_completion, h_stall, h_die_stats=None, chunk=0):
+        """``hbf_submit_host``: serves a batch that lives in host memory (torch CPU tensors, pinned for overlapped copies:
+        h_acc int64 [3 n] (the records), h_completion, h_stall int64 [n], h_die_stats int64 [6 dies] or None).  The
+        library cuts it into chunks and overlaps copy-in, service and read-back; the call returns when the results are in
+        the caller's buffers.  Returns (code, summary dict)."""
+        r = hbf_batch_result_t()
+        rc = lib().hbf_submit_host(self._h, _ptr(h_acc), n, _ptr(h_completion), _ptr(h_stall), _ptr(h_die_stats), chunk, C.byref(r))
+        return rc, r.as_dict()
 
     # ---- host-buffer convenience: copies in, one submit, copies out ---------------------------------
     def submit_host(self, acc: np.ndarray, want_status=True, check=True, parts_capacity=None):

@@ -48,6 +48,7 @@ def test_host_side_argument_checks_need_no_gpu(so_path):
     assert lib.hbf_create(None, None, None) == hbf.E_INVAL
     assert lib.hbf_destroy(None) == hbf.E_INVAL
     assert lib.hbf_workspace_bytes(None, 10) == 0
+    assert lib.hbf_submit_host(None, None, 0, None, None, None, 0, None) == hbf.E_INVAL
     cfg = hbf.hbf_config_t()                       # all zero: rejected before any CUDA call
     h = ctypes.c_void_p()
     assert lib.hbf_create(ctypes.byref(cfg), None, ctypes.byref(h)) == hbf.E_INVAL

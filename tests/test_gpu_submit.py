@@ -320,8 +320,9 @@ def test_inorder_long_busy_periods(hbf, rho):
 
 
 def test_pinned_host_pipeline_equals_one_batch(hbf):
-    """Copy-in, service and read-back of consecutive chunks on three streams: for records in issue order the
-    result is that of one batch."""
+    """hbf_submit_host: copy-in, service and read-back of consecutive chunks on three streams of the library: for records
+    in issue order the result (outputs, per-die totals, summary, queue state) is that of one batch; pageable buffers
+    work too; a chunk with a fail-closed access is reported and leaves zeros."""
     import torch
     w = wl.capacity_mode(n=230_000, seed=4)
     g, o = contexts(hbf, w.profile, w.ranges)
@@ -336,10 +337,10 @@ def test_pinned_host_pipeline_equals_one_batch(hbf):
         else:
             n_use = n
         g.reset()
-        assert g.submit_pinned(h_in, n_use, h_c, h_s, h_ds, chunk=chunk) == 0
-        torch.cuda.synchronize()
-        assert g.last_result()["code"] == 0
+        rc, summary = g.submit_pinned(h_in, n_use, h_c, h_s, h_ds, chunk=chunk)     # hbf_submit_host: returns when the results are home
+        assert rc == 0 and summary["code"] == 0 and summary["n_modeled"] + summary["n_native"] == n_use
         if n_use == n:
+            assert summary == o.last_result()
             assert np.array_equal(h_c.numpy(), c_o) and np.array_equal(h_s.numpy(), s_o)
             assert np.array_equal(h_ds.numpy().view(hbfo.DIE_STATS_DTYPE)["bytes_read"], ds_o["bytes_read"])
             assert np.array_equal(g.get_busy_until(), o.busy_until())
@@ -349,3 +350,14 @@ def test_pinned_host_pipeline_equals_one_batch(hbf):
                 o2.register_range(*r)
             _, c2, s2, _, _ = o2.submit(w.acc[:n_use])
             assert np.array_equal(h_c.numpy()[:n_use], c2) and np.array_equal(h_s.numpy()[:n_use], s2)
+    # pageable buffers, and a refusal in the middle: the second chunk holds a zero-byte access
+    bad = w.acc[:30_000].copy(); bad["bytes"][17_000] = 0
+    h_bad = torch.from_numpy(bad.view(np.int64).reshape(-1))
+    c2, s2 = torch.empty(30_000, dtype=torch.int64), torch.empty(30_000, dtype=torch.int64)
+    g.reset()
+    rc, summary = g.submit_pinned(h_bad, 30_000, c2, s2, None, chunk=10_000)
+    assert rc == hbf.E_ACCESS_FAULT and summary["n_fault"] == 1
+    assert not c2[10_000:20_000].any() and c2[:10_000].all() and c2[20_000:].all()
+    o2 = hbfo.Oracle(w.profile); o2.register_range(*w.ranges[0])
+    _, c_a, *_ = o2.submit(bad[:10_000]); _, c_b, *_ = o2.submit(bad[20_000:])
+    assert np.array_equal(c2[:10_000].numpy(), c_a) and np.array_equal(c2[20_000:].numpy(), c_b)
