@@ -253,7 +253,15 @@ HBF_API int hbf_queue_order(hbf_ctx *ctx, const void *d_workspace, uint64_t n, u
 #define HBF_PROF_STAGES 8
 HBF_API int hbf_set_profiling(hbf_ctx *ctx, int on);
 HBF_API int hbf_get_profile(hbf_ctx *ctx, float *ms_out, uint32_t cap);
-/* Number of kernels this library has launched in the calling process so far. */
+/* Test support, off by default.  The sort path's kernels wait on one another's tiles (decoupled look-back); every such
+ * wait polls a bounded number of times and then gives up: the batch's result becomes HBF_E_TIMEOUT, its outputs are zeroed,
+ * no state changes, the context is poisoned (later batches return HBF_E_TIMEOUT until hbf_reset).  This call lets a test
+ * see that happen without any real stall: poll_limit replaces the bound (0 = the default, 2^24 polls), and tile `tile` of
+ * stage 1 (the first radix pass) or 2 (the scan) publishes nothing, so that every tile behind it runs out of polls and
+ * returns.  stage 0 = no tile is silenced.  Nothing here makes a kernel wait without a bound. */
+HBF_API int hbf_debug_wait_test(hbf_ctx *ctx, uint32_t poll_limit, uint32_t stage, uint32_t tile);
+/* Number of kernels this library has launched from the host in the calling process so far (kernels that the device itself
+ * launches, the sort path behind HBF_PATH_AUTO's in-order attempt, are not counted). */
 HBF_API uint64_t hbf_kernel_launches(void);
 
 /* Explicit-Euler substeps of the package RC network without any allocation.  (The paper has no

@@ -49,6 +49,7 @@ struct hbf_ctx {
     float *h_ext = nullptr;                      // pinned [n_regions]
     std::vector<float> last_ext;                 // the external powers the device holds (empty: none sent yet)
     bool submitted = false;
+    uint32_t spin_limit = kSpinLimit, test_stage = 0, test_tile = 0;   // bounded device-side waits (test support: hbf_debug_wait_test)
     bool profiling = false; cudaEvent_t ev[kProfEvents] = {}; cudaEvent_t ev_th[2] = {}; bool ev_made = false;
     bool prof_submit = false, prof_thermal = false, prof_inorder = false, inorder_ok = false;
     // thermal
@@ -307,6 +308,7 @@ int hbf_create(const hbf_config_t *cfg, void *cuda_stream, hbf_ctx **out) {
         }
     }
     DevState st0; st0.mode = HBF_MODE_NORMAL; st0.poisoned = 0; st0.q_ppm = 1000000;
+    st0.spin_limit = c->spin_limit; st0.test_stage = c->test_stage; st0.test_tile = c->test_tile; st0.pad = 0;
     if ((rc = dev_copy(c, &c->d_ranges, nullptr, 1))) return fail(rc);
     if ((rc = dev_copy(c, &c->d_mp, &mp, 1))) return fail(rc);
     if ((rc = dev_copy(c, &c->d_state, &st0, 1))) return fail(rc);
@@ -811,6 +813,18 @@ int hbf_force_mode(hbf_ctx *c, int32_t mode, int64_t q_ppm) {
     return HBF_OK;
 }
 
+int hbf_debug_wait_test(hbf_ctx *c, uint32_t poll_limit, uint32_t stage, uint32_t tile) {
+    if (!c || stage > 2u) return HBF_E_INVAL;
+    DevState s;
+    CK(cudaMemcpyAsync(&s, c->d_state, sizeof(s), cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    c->spin_limit = poll_limit ? poll_limit : kSpinLimit; c->test_stage = stage; c->test_tile = tile;
+    s.spin_limit = c->spin_limit; s.test_stage = stage; s.test_tile = tile;
+    CK(cudaMemcpyAsync(c->d_state, &s, sizeof(s), cudaMemcpyHostToDevice, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    return HBF_OK;
+}
+
 int hbf_get_mode(hbf_ctx *c, int32_t *mode, int64_t *q_ppm) {
     if (!c) return HBF_E_INVAL;
     DevState s;
@@ -824,6 +838,7 @@ int hbf_get_mode(hbf_ctx *c, int32_t *mode, int64_t *q_ppm) {
 int hbf_reset(hbf_ctx *c) {
     if (!c) return HBF_E_INVAL;
     DevState s; s.mode = HBF_MODE_NORMAL; s.poisoned = 0; s.q_ppm = 1000000;
+    s.spin_limit = c->spin_limit; s.test_stage = c->test_stage; s.test_tile = c->test_tile; s.pad = 0;
     CK(cudaStreamSynchronize(c->stream));
     CK(cudaMemcpyAsync(c->d_state, &s, sizeof(s), cudaMemcpyHostToDevice, c->stream));
     CK(cudaMemsetAsync(c->d_busy, 0, c->mp.n_queues * sizeof(int64_t), c->stream));
@@ -934,6 +949,7 @@ int hbf_set_state(hbf_ctx *c, const void *host_buf, size_t bytes) {
     if (h.magic != kStateMagic || h.version != 1u || h.n_queues != c->mp.n_queues || h.n_dies != c->mp.n_dies ||
         h.n_cells != (uint32_t)nc || h.mode < 0 || h.mode > 3 || h.q_ppm < 1 || h.q_ppm > 1000000) return HBF_E_INVAL;
     DevState s; s.mode = h.mode; s.q_ppm = h.q_ppm; s.poisoned = h.poisoned;
+    s.spin_limit = c->spin_limit; s.test_stage = c->test_stage; s.test_tile = c->test_tile; s.pad = 0;
     CK(cudaStreamSynchronize(c->stream));
     CK(cudaMemcpyAsync(c->d_state, &s, sizeof(s), cudaMemcpyHostToDevice, c->stream));
     CK(cudaMemcpyAsync(c->d_busy, p, (size_t)c->mp.n_queues * 8, cudaMemcpyHostToDevice, c->stream)); p += (size_t)c->mp.n_queues * 8;

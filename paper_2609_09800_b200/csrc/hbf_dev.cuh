@@ -78,6 +78,9 @@ struct BatchCtrl {
 struct DevState {
     int32_t mode; int32_t poisoned;
     int64_t q_ppm;
+    uint32_t spin_limit;                 // polls of one look-back slot before a waiter gives up (kSpinLimit unless a test lowers it)
+    uint32_t test_stage, test_tile;      // test support: tile `test_tile` of stage 1 (first radix pass) or 2 (scan) publishes nothing
+    uint32_t pad;
 };
 
 // Workspace carve-up for a batch of n records.

@@ -239,6 +239,8 @@ k_sort_pass(int pass, uint64_t n, BatchCtrl *ctrl, DevState *state, const uint32
     __syncthreads();
     const uint32_t tile = s_tile;
     if (tile >= n_tiles) break;
+    const uint32_t spin_limit = state->spin_limit;
+    const bool mute = state->test_stage == 1u && pass == 0 && state->test_tile == tile;   // (test support: this tile stays silent)
     const uint64_t base = (uint64_t)tile * kSortTile;
     if (tid < kRadix) desc_next[(uint64_t)tile * kRadix + tid] = 0u;     // ready for the pass after this one
 
@@ -275,7 +277,7 @@ k_sort_pass(int pass, uint64_t n, BatchCtrl *ctrl, DevState *state, const uint32
     if (tid < kRadix) {
 #pragma unroll
         for (int w = 0; w < kSortWarps; ++w) { const uint32_t c = s_cnt[w * kRadix + tid]; s_cnt[w * kRadix + tid] = tile_count; tile_count += c; }
-        st_relaxed_u32(desc + (uint64_t)tile * kRadix + tid, (tile == 0 ? kFlagPrefix : kFlagAgg) | tile_count);
+        if (!mute) st_relaxed_u32(desc + (uint64_t)tile * kRadix + tid, (tile == 0 ? kFlagPrefix : kFlagAgg) | tile_count);
         hist_mine = hist[pass * kRadix + tid];
         local_incl = tile_count; hist_incl = hist_mine;
 #pragma unroll
@@ -298,7 +300,7 @@ k_sort_pass(int pass, uint64_t n, BatchCtrl *ctrl, DevState *state, const uint32
             const uint32_t *p = desc + (uint64_t)t * kRadix + tid;
             uint32_t v = ld_relaxed_u32(p), spins = 0;
             while ((v >> 30) == 0u) {
-                if (++spins > kSpinLimit) { failed = true; break; }
+                if (++spins > spin_limit) { failed = true; break; }
                 __nanosleep(20);
                 v = ld_relaxed_u32(p);
             }
@@ -306,8 +308,9 @@ k_sort_pass(int pass, uint64_t n, BatchCtrl *ctrl, DevState *state, const uint32
             excl += v & kCountMask;
             if ((v >> 30) == 2u) break;
         }
-        if (failed) { atomicExch(&ctrl->code, (int)HBF_E_TIMEOUT); state->poisoned = 1; }
-        if (tile != 0) st_relaxed_u32(desc + (uint64_t)tile * kRadix + tid, kFlagPrefix | ((excl + tile_count) & kCountMask));
+        // a wait that ran out: the batch is given up (later kernels of it exit at once) and the context is poisoned
+        if (failed) { atomicExch(&ctrl->code, (int)HBF_E_TIMEOUT); ctrl->skip = 1; state->poisoned = 1; }
+        if (tile != 0 && !mute) st_relaxed_u32(desc + (uint64_t)tile * kRadix + tid, kFlagPrefix | ((excl + tile_count) & kCountMask));
         s_local_start[tid] = local_start;
         s_delta[tid] = gstart + excl - local_start;
     }
@@ -506,7 +509,10 @@ k_scan(const hbf_access_t *__restrict__ acc, uint64_t n, const RangeSnap *__rest
         const Map agg = compose(excl, tm);
         ScanDesc *my = desc + tile;
         int64_t tile_in = 0;
-        if (agg.f) {
+        const uint32_t spin_limit = state->spin_limit;
+        const bool mute = state->test_stage == 2u && state->test_tile == tile;        // (test support: this tile stays silent)
+        if (mute) {
+        } else if (agg.f) {
             st_relaxed_s64(&my->value, agg.M);
             st_release_u32(&my->status, 2u);
             // the tile's own first segment may still continue the previous tile's queue
@@ -522,7 +528,7 @@ k_scan(const hbf_access_t *__restrict__ acc, uint64_t n, const RangeSnap *__rest
                 const ScanDesc *p = desc + t;
                 uint32_t stt = ld_acquire_u32(&p->status), spins = 0;
                 while (stt == 0u) {
-                    if (++spins > kSpinLimit) { failed = true; break; }
+                    if (++spins > spin_limit) { failed = true; break; }
                     __nanosleep(20);
                     stt = ld_acquire_u32(&p->status);
                 }
@@ -536,9 +542,9 @@ k_scan(const hbf_access_t *__restrict__ acc, uint64_t n, const RangeSnap *__rest
                 const int64_t St = ld_relaxed_s64(&p->S), Mt = ld_relaxed_s64(&p->M);
                 M_acc = max(Mt + S_acc, M_acc); S_acc += St;
             }
-            if (failed) { atomicExch(&ctrl->code, (int)HBF_E_TIMEOUT); state->poisoned = 1; }
+            if (failed) { atomicExch(&ctrl->code, (int)HBF_E_TIMEOUT); ctrl->skip = 1; state->poisoned = 1; }
         }
-        if (!agg.f) {
+        if (!agg.f && !mute) {
             st_relaxed_s64(&my->value, max(tile_in + agg.S, agg.M));
             st_release_u32(&my->status, 2u);
         }

@@ -30,7 +30,7 @@ EXPORTS = ("hbf_create", "hbf_destroy", "hbf_register_range", "hbf_clear_ranges"
            "hbf_reset", "hbf_set_path", "hbf_get_state", "hbf_set_state", "hbf_get_busy_until",
            "hbf_get_pending_energy", "hbf_get_temps", "hbf_euler_limit_ns", "hbf_queue_order", "hbf_strerror",
            "hbf_set_profiling", "hbf_get_profile", "hbf_kernel_launches", "hbf_euler_substeps_static", "hbf_set_thermal_path",
-           "hbf_workspace_bytes_paged", "hbf_submit_batch_paged", "hbf_submit_host",
+           "hbf_workspace_bytes_paged", "hbf_submit_batch_paged", "hbf_submit_host", "hbf_debug_wait_test",
            "hbf_enable_energy_bins", "hbf_get_energy_bins", "hbf_enable_channel_bus", "hbf_get_bus_busy_until",
            "hbf_rom_create", "hbf_rom_destroy", "hbf_rom_reset", "hbf_rom_step", "hbf_rom_get_state",
            "hbf_attach_rom", "hbf_get_rom_temps",
@@ -104,6 +104,7 @@ def lib():
         L.hbf_workspace_bytes.argtypes = [vp, u64]
         L.hbf_workspace_bytes.restype = C.c_size_t
         L.hbf_submit_batch.argtypes = [vp, vp, u64, vp, vp, vp, vp, vp, C.c_size_t]
+        L.hbf_debug_wait_test.argtypes = [vp, u32, u32, u32]
         L.hbf_submit_host.argtypes = [vp, vp, u64, vp, vp, vp, u64, C.POINTER(hbf_batch_result_t)]
         L.hbf_workspace_bytes_paged.argtypes = [vp, u64, u64]
         L.hbf_workspace_bytes_paged.restype = C.c_size_t
@@ -419,6 +420,12 @@ class Context:
                 raise HbfError(rc, "hbf_thermal_step")
             return rc
         return hot
+
+    def debug_wait_test(self, poll_limit=0, stage=0, tile=0):
+        """Test support (``hbf_debug_wait_test``): a small poll budget and one silent tile make the bounded waits run out."""
+        rc = lib().hbf_debug_wait_test(self._h, poll_limit, stage, tile)
+        if rc != 0:
+            raise HbfError(rc, "hbf_debug_wait_test")
 
     def force_mode(self, mode, q_ppm):
         rc = lib().hbf_force_mode(self._h, mode, q_ppm)

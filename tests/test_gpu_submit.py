@@ -361,3 +361,25 @@ def test_pinned_host_pipeline_equals_one_batch(hbf):
     o2 = hbfo.Oracle(w.profile); o2.register_range(*w.ranges[0])
     _, c_a, *_ = o2.submit(bad[:10_000]); _, c_b, *_ = o2.submit(bad[20_000:])
     assert np.array_equal(c2[:10_000].numpy(), c_a) and np.array_equal(c2[20_000:].numpy(), c_b)
+
+
+@pytest.mark.parametrize("stage", [1, 2])
+def test_bounded_waits_run_out_and_the_batch_is_given_up(hbf, stage):
+    """The look-back waits of the sort path are bounded.  With a poll budget of a few hundred and one early tile silenced
+    (test support of the library: nothing stalls for real), every tile behind it runs out of polls and returns: the batch's
+    result is HBF_E_TIMEOUT, its outputs are zeroed, the queue state is untouched, the context is poisoned and refuses
+    later batches, and hbf_reset brings it back."""
+    w = wl.mixed_status(30_000, seed=12)                     # shuffled: several radix passes, 8 sort tiles, 15 scan tiles
+    g, o = contexts(hbf, w.profile, w.ranges, hbf.PATH_SORT_FULL)
+    compare_batch(g, o, w.acc[:5000])
+    busy0, pend0 = g.get_busy_until(), g.get_pending_energy()
+    g.debug_wait_test(poll_limit=300, stage=stage, tile=1)
+    rc, c_g, s_g, _, ds_g = g.submit_host(w.acc[5000:], check=False)
+    assert rc == hbf.E_TIMEOUT and not c_g.any() and not s_g.any() and not ds_g["n_read"].any()
+    assert np.array_equal(g.get_busy_until(), busy0) and np.array_equal(g.get_pending_energy(), pend0)
+    g.debug_wait_test()                                     # the switch is off again, but the context stays poisoned
+    rc, *_ = g.submit_host(w.acc[5000:], check=False)
+    assert rc == hbf.E_TIMEOUT
+    assert np.array_equal(g.get_busy_until(), busy0)
+    g.reset(); o.reset()
+    compare_batch(g, o, w.acc)                              # usable again, and exact
