@@ -87,6 +87,7 @@ struct DevState {
 struct Workspace {
     uint64_t *keys[2];
     uint32_t *idx[2];
+    uint64_t *terms;                     // [n] per record, in batch order: bytes | op << 32 | pages << 33 (what the scan needs of it)
     uint32_t *hist;                      // [kMaxPasses][kRadix]
     uint32_t *sort_desc[2];              // [tiles][kRadix] look-back words, ping-pong between passes
     void *scan_desc;                     // [scan tiles] ScanDesc
