@@ -28,6 +28,8 @@ def full():
     from paper_2609_09800_b200 import build, hbf
     build.build()
     w = wl.capacity_mode(n=N_FULL)
+    from paper_2609_09800_b200.config import fingerprint_streams as fps
+    assert fps.sha256_of(w.acc) == fps.recorded()["sha256"]["capacity_mode(200,000,000, seed 0)"]   # the stream every number is quoted on
     u = ((w.acc["addr"] - np.uint64(wl.RANGE_BASE)) >> np.uint64(16)).astype(np.int64)   # 64 KiB stripe units
     queue = (((u % 64) * 8 + (u // 64) % 8) * 4 + (u // 512) % 4).astype(np.int32)
     shards = shards_of(queue, host_workers())
@@ -193,6 +195,8 @@ def test_serving_configurations_at_full_size_element_by_element(which):
     from paper_2609_09800_b200 import build, hbf
     build.build()
     w = wl.decode_weights() if which == "decode_weights" else wl.prefix_kv()
+    from paper_2609_09800_b200.config import fingerprint_streams as fps
+    assert fps.sha256_of(w.acc) == fps.recorded()["sha256"]["decode_weights(256 tokens, seed 0)" if which == "decode_weights" else "prefix_kv(seed 0)"]
     g, o = hbf.Context(w.profile), hbfo.Oracle(w.profile)
     for r in w.ranges:
         g.register_range(*r); o.register_range(*r)

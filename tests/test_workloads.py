@@ -81,3 +81,15 @@ def test_floorplans():
     # unlike neighbours: series half cells
     gx = fp["cell_Gx"].reshape(128, 128)
     assert abs(gx[10, 31] - 2 * 0.03 * 0.075 / 0.105) < 1e-7
+
+
+def test_stream_fingerprints():
+    """The committed SHA-256 of every stream small enough for this box (the two largest are checked where they are used, on
+    the GPU machine): a numpy release or an edit that reshuffles a stream fails here, and the file names the numpy it was made with."""
+    from paper_2609_09800_b200.config import fingerprint_streams as fps
+    rec = fps.recorded()
+    assert set(rec["sha256"]) == set(fps.STREAMS) and rec["numpy"].split(".")[0] == np.__version__.split(".")[0]
+    got = fps.compute(cheap_only=True)
+    assert len(got) >= 5
+    for name, sha in got.items():
+        assert rec["sha256"][name] == sha, name
