@@ -179,7 +179,7 @@ HBF_API int hbf_submit_batch_paged(hbf_ctx *ctx, const hbf_access_t *d_acc, uint
  * HBF_ISSUE_LIMIT): a batch whose largest completion time would reach 2^47 ns is refused with HBF_E_INVAL before anything
  * is committed (outputs zeroed, queue, bus and energy state unchanged); the context stays usable.
  * hbf_get_bus_busy_until synchronises and copies the per-channel bus state to host_out [channels]; hbf_reset clears
- * it.  The state blob of hbf_get_state does not carry it.  hbf_submit_batch_paged is refused while the stage is on. */
+ * it.  hbf_submit_batch_paged is refused while the stage is on. */
 HBF_API int hbf_enable_channel_bus(hbf_ctx *ctx);
 HBF_API int hbf_get_bus_busy_until(hbf_ctx *ctx, int64_t *host_out, uint64_t cap);
 
@@ -192,7 +192,7 @@ HBF_API int hbf_get_bus_busy_until(hbf_ctx *ctx, int64_t *host_out, uint64_t cap
  * end into its last bin.  hbf_thermal_step must then be called with dt_ns == bin_ns (HBF_E_INVAL otherwise):
  * it consumes the clock's bin and advances the clock by one.  hbf_get_energy_bins synchronises and copies the
  * ring to host_out [n_bins][channels*dies] (row k = bin *first_bin + k).  The ledger is library-owned device
- * memory allocated by hbf_enable_energy_bins; it is not part of the hbf_get_state blob.
+ * memory allocated by hbf_enable_energy_bins.
  * hbf_submit_batch_paged is refused (HBF_E_INVAL) while the ledger is on. */
 HBF_API int hbf_enable_energy_bins(hbf_ctx *ctx, int64_t bin_ns, uint32_t n_bins);
 HBF_API int hbf_get_energy_bins(hbf_ctx *ctx, int64_t *host_out, uint64_t cap, int64_t *first_bin);
@@ -230,8 +230,12 @@ HBF_API int hbf_set_path(hbf_ctx *ctx, int32_t path);
  * Both perform the same arithmetic in the same order (Eq. 1). */
 HBF_API int hbf_set_thermal_path(hbf_ctx *ctx, int32_t generic_only);
 
-/* State snapshot (host blob): header, busy_until[queues], pending energy[dies], thermal field and
- * its compensation term.  Call with host_buf NULL to get the size. */
+/* State snapshot (host blob): header, busy_until[queues], pending energy[dies], thermal field and its compensation
+ * term; then, for whatever is switched on: the channel buses' busy-until, the energy ledger with its clock, the whole
+ * retention state (counters, per-block damage / disturb / cycles / epoch / worn flag, the plan ring).  A blob goes back
+ * only into a context with the same geometry and the same things switched on at the same sizes (HBF_E_INVAL otherwise): a
+ * long coupled run can be stopped and resumed, or two implementations re-synchronised, at any batch boundary.  Call with
+ * host_buf NULL to get the size.  A reduced-order model's state is its own (hbf_rom_get_state). */
 HBF_API int hbf_get_state(hbf_ctx *ctx, void *host_buf, size_t *bytes);
 HBF_API int hbf_set_state(hbf_ctx *ctx, const void *host_buf, size_t bytes);
 /* Individual state arrays, host outputs; each waits for pending work. */
@@ -354,7 +358,7 @@ HBF_API int hbf_get_rom_temps(hbf_ctx *ctx, double *host_out, uint64_t cap);
  * hbf_get_retention_blocks / _plan / _totals synchronise the stream and copy to host memory: per-block arrays
  *   [n_blocks] (each nullable); the outstanding quanta in plan order (quanta == NULL: count only); the counters.
  * hbf_reset returns every block to fresh and empties the plan.  The block state and the plan are library-owned
- * device memory (33 bytes per block, 4 bytes per page of the medium); they are not part of the hbf_get_state blob. */
+ * device memory (33 bytes per block, 4 bytes per page of the medium). */
 typedef struct {
     uint32_t pages_per_block, blocks_per_plane, blocks_per_zone;   /* blocks_per_plane a multiple of blocks_per_zone */
     uint32_t max_pec;                      /* a block that has committed this many cycles is worn out: no more damage, never eligible */

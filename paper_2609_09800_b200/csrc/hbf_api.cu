@@ -17,7 +17,12 @@ struct HostRange { uint64_t base, length, media_offset; uint32_t perms, kind, st
 
 struct StateHeader {            // hbf_get_state / hbf_set_state blob header
     uint32_t magic, version, n_queues, n_dies, n_cells; int32_t mode; int64_t q_ppm; int32_t poisoned, cur;
+    // version 2: what else the context has switched on, each with the sizes that fix its section's length
+    uint32_t flags, n_channels;          // kStateBus | kStateBins | kStateRetention
+    int64_t bin_ns, cur_bin; uint32_t n_bins, pad;
+    uint64_t ret_blocks, ret_plan_cap;
 };
+constexpr uint32_t kStateBus = 1u, kStateBins = 2u, kStateRetention = 4u;
 constexpr uint32_t kStateMagic = 0x48424631u;   // "HBF1"
 
 }  // namespace
@@ -916,10 +921,21 @@ uint64_t hbf_kernel_launches(void) { return g_kernel_launches.load(); }
 
 double hbf_euler_limit_ns(const hbf_ctx *c) { return c && c->thermal ? c->euler_limit_s * 1e9 : 0.0; }
 
+// Sections of the blob after the header, in order: busy_until[queues], pending energy[dies], field and compensation
+// [cells each]; then, for what is switched on: bus busy-until[channels]; ledger [n_bins][dies]; retention: the counters,
+// per block damage (f64), disturb, PEC, epoch (u32 each), worn (u8), last plan position (u64), then the plan ring.
+static size_t state_bytes(const hbf_ctx *c, size_t nc) {
+    size_t need = sizeof(StateHeader) + (size_t)c->mp.n_queues * 8 + (size_t)c->mp.n_dies * 8 + nc * 8;
+    if (c->d_bus_busy) need += (size_t)c->mp.channels * 8;
+    if (c->bin_ns) need += (size_t)c->n_bins * c->mp.n_dies * 8;
+    if (c->ret_on) need += sizeof(RetState) + (size_t)c->ret.n_blocks * (8 + 4 + 4 + 4 + 1 + 8) + (size_t)c->ret.plan_cap * 4;
+    return need;
+}
+
 int hbf_get_state(hbf_ctx *c, void *host_buf, size_t *bytes) {
     if (!c || !bytes) return HBF_E_INVAL;
     const size_t nc = c->thermal ? (size_t)c->td.H * c->td.W : 0;
-    const size_t need = sizeof(StateHeader) + (size_t)c->mp.n_queues * 8 + (size_t)c->mp.n_dies * 8 + nc * 8;
+    const size_t need = state_bytes(c, nc);
     if (!host_buf) { *bytes = need; return HBF_OK; }
     if (*bytes < need) return HBF_E_INVAL;
     *bytes = need;
@@ -927,36 +943,59 @@ int hbf_get_state(hbf_ctx *c, void *host_buf, size_t *bytes) {
     DevState s;
     CK(cudaMemcpyAsync(&s, c->d_state, sizeof(s), cudaMemcpyDeviceToHost, c->stream));
     CK(cudaStreamSynchronize(c->stream));
-    StateHeader h{kStateMagic, 1u, c->mp.n_queues, c->mp.n_dies, (uint32_t)nc, s.mode, s.q_ppm, s.poisoned, 0};
+    StateHeader h{};
+    h.magic = kStateMagic; h.version = 2u; h.n_queues = c->mp.n_queues; h.n_dies = c->mp.n_dies; h.n_cells = (uint32_t)nc;
+    h.mode = s.mode; h.q_ppm = s.q_ppm; h.poisoned = s.poisoned; h.cur = 0;
+    h.flags = (c->d_bus_busy ? kStateBus : 0u) | (c->bin_ns ? kStateBins : 0u) | (c->ret_on ? kStateRetention : 0u);
+    h.n_channels = c->mp.channels; h.bin_ns = c->bin_ns; h.cur_bin = c->cur_bin; h.n_bins = c->n_bins;
+    h.ret_blocks = c->ret_on ? c->ret.n_blocks : 0; h.ret_plan_cap = c->ret_on ? c->ret.plan_cap : 0;
     memcpy(p, &h, sizeof(h)); p += sizeof(h);
-    CK(cudaMemcpyAsync(p, c->d_busy, (size_t)c->mp.n_queues * 8, cudaMemcpyDeviceToHost, c->stream)); p += (size_t)c->mp.n_queues * 8;
-    CK(cudaMemcpyAsync(p, c->d_pending, (size_t)c->mp.n_dies * 8, cudaMemcpyDeviceToHost, c->stream)); p += (size_t)c->mp.n_dies * 8;
-    if (nc) {
-        CK(cudaMemcpyAsync(p, c->td.theta[c->cur], nc * 4, cudaMemcpyDeviceToHost, c->stream)); p += nc * 4;
-        CK(cudaMemcpyAsync(p, c->td.comp, nc * 4, cudaMemcpyDeviceToHost, c->stream));
+    auto pull = [&](const void *dev, size_t n) { cudaError_t e = cudaMemcpyAsync(p, dev, n, cudaMemcpyDeviceToHost, c->stream); p += n; return e; };
+    CK(pull(c->d_busy, (size_t)c->mp.n_queues * 8));
+    CK(pull(c->d_pending, (size_t)c->mp.n_dies * 8));
+    if (nc) { CK(pull(c->td.theta[c->cur], nc * 4)); CK(pull(c->td.comp, nc * 4)); }
+    if (c->d_bus_busy) CK(pull(c->d_bus_busy, (size_t)c->mp.channels * 8));
+    if (c->bin_ns) CK(pull(c->d_ledger, (size_t)c->n_bins * c->mp.n_dies * 8));
+    if (c->ret_on) {
+        const RetDev &r = c->ret;
+        CK(pull(r.st, sizeof(RetState)));
+        CK(pull(r.damage, r.n_blocks * 8)); CK(pull(r.disturb, r.n_blocks * 4)); CK(pull(r.pec, r.n_blocks * 4));
+        CK(pull(r.epoch_of, r.n_blocks * 4)); CK(pull(r.worn, r.n_blocks)); CK(pull(r.last_pos, r.n_blocks * 8));
+        CK(pull(r.plan, r.plan_cap * 4));
     }
     CK(cudaStreamSynchronize(c->stream));
     return HBF_OK;
 }
 
 int hbf_set_state(hbf_ctx *c, const void *host_buf, size_t bytes) {
-    if (!c || !host_buf) return HBF_E_INVAL;
+    if (!c || !host_buf || bytes < sizeof(StateHeader)) return HBF_E_INVAL;
     const size_t nc = c->thermal ? (size_t)c->td.H * c->td.W : 0;
-    const size_t need = sizeof(StateHeader) + (size_t)c->mp.n_queues * 8 + (size_t)c->mp.n_dies * 8 + nc * 8;
+    const size_t need = state_bytes(c, nc);
     if (bytes < need) return HBF_E_INVAL;
     const char *p = static_cast<const char *>(host_buf);
     StateHeader h; memcpy(&h, p, sizeof(h)); p += sizeof(h);
-    if (h.magic != kStateMagic || h.version != 1u || h.n_queues != c->mp.n_queues || h.n_dies != c->mp.n_dies ||
+    const uint32_t flags = (c->d_bus_busy ? kStateBus : 0u) | (c->bin_ns ? kStateBins : 0u) | (c->ret_on ? kStateRetention : 0u);
+    if (h.magic != kStateMagic || h.version != 2u || h.n_queues != c->mp.n_queues || h.n_dies != c->mp.n_dies ||
         h.n_cells != (uint32_t)nc || h.mode < 0 || h.mode > 3 || h.q_ppm < 1 || h.q_ppm > 1000000) return HBF_E_INVAL;
+    // the blob must come from a context with the same things switched on, at the same sizes
+    if (h.flags != flags || h.n_channels != c->mp.channels || (c->bin_ns && (h.bin_ns != c->bin_ns || h.n_bins != c->n_bins)) ||
+        (c->ret_on && (h.ret_blocks != c->ret.n_blocks || h.ret_plan_cap != c->ret.plan_cap))) return HBF_E_INVAL;
     DevState s; s.mode = h.mode; s.q_ppm = h.q_ppm; s.poisoned = h.poisoned;
     s.spin_limit = c->spin_limit; s.test_stage = c->test_stage; s.test_tile = c->test_tile; s.pad = 0;
     CK(cudaStreamSynchronize(c->stream));
     CK(cudaMemcpyAsync(c->d_state, &s, sizeof(s), cudaMemcpyHostToDevice, c->stream));
-    CK(cudaMemcpyAsync(c->d_busy, p, (size_t)c->mp.n_queues * 8, cudaMemcpyHostToDevice, c->stream)); p += (size_t)c->mp.n_queues * 8;
-    CK(cudaMemcpyAsync(c->d_pending, p, (size_t)c->mp.n_dies * 8, cudaMemcpyHostToDevice, c->stream)); p += (size_t)c->mp.n_dies * 8;
-    if (nc) {
-        CK(cudaMemcpyAsync(c->td.theta[c->cur], p, nc * 4, cudaMemcpyHostToDevice, c->stream)); p += nc * 4;
-        CK(cudaMemcpyAsync(c->td.comp, p, nc * 4, cudaMemcpyHostToDevice, c->stream));
+    auto push = [&](void *dev, size_t n) { cudaError_t e = cudaMemcpyAsync(dev, p, n, cudaMemcpyHostToDevice, c->stream); p += n; return e; };
+    CK(push(c->d_busy, (size_t)c->mp.n_queues * 8));
+    CK(push(c->d_pending, (size_t)c->mp.n_dies * 8));
+    if (nc) { CK(push(c->td.theta[c->cur], nc * 4)); CK(push(c->td.comp, nc * 4)); }
+    if (c->d_bus_busy) CK(push(c->d_bus_busy, (size_t)c->mp.channels * 8));
+    if (c->bin_ns) { CK(push(c->d_ledger, (size_t)c->n_bins * c->mp.n_dies * 8)); c->cur_bin = h.cur_bin; }
+    if (c->ret_on) {
+        const RetDev &r = c->ret;
+        CK(push(r.st, sizeof(RetState)));
+        CK(push(r.damage, r.n_blocks * 8)); CK(push(r.disturb, r.n_blocks * 4)); CK(push(r.pec, r.n_blocks * 4));
+        CK(push(r.epoch_of, r.n_blocks * 4)); CK(push(r.worn, r.n_blocks)); CK(push(r.last_pos, r.n_blocks * 8));
+        CK(push(r.plan, r.plan_cap * 4));
     }
     CK(cudaStreamSynchronize(c->stream));
     c->terminal = (h.mode == HBF_MODE_SHUTDOWN) ? c->terminal : false;

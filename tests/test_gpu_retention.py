@@ -337,3 +337,49 @@ def test_other_geometries_and_two_ranges(hbf, geom):
         compare_state(g, o)
     t = o.retention_totals()
     assert t["claimed"] > 0 and t["commits"] > 0
+
+
+def test_state_blob_carries_bus_ledger_and_retention(hbf):
+    """Checkpoint and resume in the middle of a run with everything switched on (channel bus, energy bins, retention with
+    outstanding debt): a fresh context that takes the blob serves the rest of the run exactly as the original does, which
+    in turn is checked against the oracle throughout; a blob from a context with other things switched on is refused."""
+    rng = np.random.default_rng(21)
+
+    def batch(n, t0):
+        a = np.zeros(n, hbfo.ACCESS_DTYPE)
+        a["addr"] = BASE + rng.integers(0, 1 << 24, n).astype(np.uint64)
+        a["issue_ns"] = t0 + np.sort(rng.integers(0, 3_000_000, n))
+        a["bytes"] = rng.choice([64, 4096, 16384, 40_000], n)
+        a["flags"] = rng.random(n) < 0.05
+        return a
+    ret = dict(RET, disturb_limit=3)
+
+    def fresh():
+        g, o, prof = contexts(hbf, ret)
+        g.enable_channel_bus(); o.enable_channel_bus()
+        g.enable_energy_bins(500_000, 32); o.enable_energy_bins(500_000, 32)
+        return g, o
+    g, o = fresh()
+    compare_batch(g, o, batch(4000, 0))
+    g.retention_advance(10**9, np.array([70.0])); o.retention_advance(10**9, np.array([70.0]))
+    compare_batch(g, o, batch(50, 3_000_000))                # claims part of the debt; the rest stays outstanding
+    assert g.retention_totals()["planned"] > g.retention_totals()["claimed"] > 0
+    blob = g.get_state()
+    later = [batch(3000, 6_000_000), batch(3000, 9_000_000)]
+    g2, _ = fresh()
+    g2.set_state(blob)
+    for acc in later:
+        compare_batch(g, o, acc)
+        rc2, c2, s2, st2, ds2 = g2.submit_host(acc, check=False)
+        rc1 = g.last_result()["code"]
+        assert rc2 == rc1 and g2.last_result() == g.last_result()
+        assert np.array_equal(g2.get_busy_until(), g.get_busy_until()) and np.array_equal(g2.get_bus_busy_until(), g.get_bus_busy_until())
+        (f1, b1), (f2, b2) = g.energy_bins(), g2.energy_bins()
+        assert f1 == f2 and np.array_equal(b1, b2)
+        assert g2.retention_totals() == g.retention_totals() and np.array_equal(g2.retention_plan(), g.retention_plan())
+        r1, r2 = g.retention_blocks(), g2.retention_blocks()
+        for k in r1:
+            assert np.array_equal(r1[k], r2[k]), k
+    plain, _, _ = contexts(hbf, ret)                          # retention only: the blob does not fit
+    with pytest.raises(hbf.HbfError):
+        plain.set_state(blob)
