@@ -363,7 +363,7 @@ __device__ __forceinline__ Map shfl_up_map(const Map &m, int o) {
     r.f = __shfl_up_sync(0xffffffffu, m.f, o); return r;
 }
 
-__global__ void __launch_bounds__(kScanThreads)
+__global__ void __launch_bounds__(kScanThreads, 2)
 k_scan(const uint64_t *__restrict__ terms, uint64_t n,
        const ModelParams *__restrict__ mp_g, BatchCtrl *ctrl, DevState *state,
        const uint64_t *keys0, const uint64_t *keys1, const uint32_t *idx0, const uint32_t *idx1,
