@@ -755,11 +755,7 @@ k_inorder_fixstraggle(const hbf_access_t *__restrict__ acc, uint64_t n, const __
         if (tid == 0) in_tile[tile].reserve = 1u;
         return;
     }
-#ifdef HBF_DBG_FIXONLY
-    if (false) {
-#else
     if (stragglers > 0u) {
-#endif
     const int64_t q_ppm = ctrl->q_ppm;
     const Div64 div_q = ctrl->div_q;
     const bool one_range = fast_arg.on != 0u && mp_arg.pow2_geom != 0u;
@@ -952,9 +948,6 @@ k_inorder_fixstraggle(const hbf_access_t *__restrict__ acc, uint64_t n, const __
             }
             __syncthreads();
         }
-#ifdef HBF_DBG_ONEITER
-        break;
-#endif
         if (*reinterpret_cast<volatile int *>(&s_open) <= 0) break;
         cb += kInStrQChunk;
     }

@@ -990,11 +990,6 @@ cudaError_t ensure_dyn_smem(const void *kernel, size_t bytes) {
             return e;
         }
     if (bytes > 48u * 1024u) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
-#ifdef HBF_EXP_CARVEOUT
-    // the kernels of a step follow one another closely: the same shared-memory carve-out for all of them spares the SMs a
-    // reconfiguration at every kernel boundary
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, HBF_EXP_CARVEOUT);
-#endif
     if (e == cudaSuccess) set.push_back(Entry{dev, kernel, bytes});
     return e;
 }
@@ -1048,13 +1043,16 @@ struct SortChain {
     const unsigned long long *claim_limit; uint32_t *die_claims;
     uint32_t n_queues, n_dies; uint64_t desc_words, scan_words;
     unsigned cls_grid, hist_grid, sort_grid, scan_grid, stall_grid;
-    const InTile *in_tile; uint32_t n_tiles; int may_sort;
+    const InTile *in_tile; uint32_t n_tiles;
 };
 
 __global__ void k_zero_words(uint32_t *p, uint64_t words) {
     for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < words; i += (uint64_t)gridDim.x * blockDim.x) p[i] = 0u;
 }
 
+// (MAY_SORT = false, for a context whose caller declares issue order: the same kernel without the device-side launches,
+// which cost a kernel that contains them several microseconds even when none is made)
+template <bool MAY_SORT>
 __global__ void __launch_bounds__(256) k_after_inorder(const __grid_constant__ SortChain c) {
     if (c.ctrl->skip) return;                                // refused: nothing to do
     if (c.ctrl->inorder_used) {
@@ -1069,7 +1067,8 @@ __global__ void __launch_bounds__(256) k_after_inorder(const __grid_constant__ S
         if ((threadIdx.x & 31) == 0 && tot) atomicAdd((unsigned long long *)&c.ctrl->modeled_ns, (unsigned long long)tot);
         return;
     }
-    if (!c.ctrl->run_sort || !c.may_sort || threadIdx.x != 0) return;
+    if constexpr (MAY_SORT) {
+    if (!c.ctrl->run_sort || threadIdx.x != 0) return;
     cudaStream_t st = cudaStreamTailLaunch;
     k_begin<<<1, 1024, 0, st>>>(c.ctrl, c.state, c.busy, c.busy_stage, c.stats_stage, c.hist, c.n_queues, c.n_dies, 1, 1, c.die_claims);
     k_zero_words<<<(unsigned)min((unsigned long long)((c.desc_words + 1023) / 1024), 592ull), 1024, 0, st>>>(c.desc0, c.desc_words);
@@ -1083,6 +1082,7 @@ __global__ void __launch_bounds__(256) k_after_inorder(const __grid_constant__ S
                                                  (ScanDesc *)c.scan_desc, c.busy, c.busy_stage, c.stats_stage, c.completion, c.stall,
                                                  c.claim_limit, c.die_claims);
     k_stalls<<<c.stall_grid, 256, 0, st>>>(c.acc, c.n, c.ctrl, c.completion, c.stall);
+    }
 }
 
 static cudaError_t launch_after_inorder(const SubmitArgs &a, bool may_sort, cudaStream_t st) {
@@ -1104,8 +1104,8 @@ static cudaError_t launch_after_inorder(const SubmitArgs &a, bool may_sort, cuda
     c.scan_grid = (unsigned)std::min<uint64_t>(scan_tiles, (uint64_t)a.sm_count * 8);
     c.stall_grid = (unsigned)std::max<uint64_t>(1, std::min<uint64_t>((n + 255) / 256, (uint64_t)a.sm_count * 16));
     const InTileMap tmap = inorder_tile_map(n, a.sm_count);
-    c.in_tile = reinterpret_cast<const InTile *>(a.ws.in_tile); c.n_tiles = tmap.n_tiles; c.may_sort = may_sort ? 1 : 0;
-    k_after_inorder<<<1, 256, 0, st>>>(c);
+    c.in_tile = reinterpret_cast<const InTile *>(a.ws.in_tile); c.n_tiles = tmap.n_tiles;
+    if (may_sort) k_after_inorder<true><<<1, 256, 0, st>>>(c); else k_after_inorder<false><<<1, 256, 0, st>>>(c);
     g_kernel_launches += 1;
     return cudaGetLastError();
 }
@@ -1119,7 +1119,7 @@ cudaError_t launch_submit(const SubmitArgs &a, cudaStream_t st) {
     const bool try_inorder = a.inorder_ok && (a.path == HBF_PATH_AUTO || a.path == HBF_PATH_INORDER);
     const bool sort_kernels = a.path != HBF_PATH_INORDER || !a.inorder_ok;
     {
-        const void *small[] = {(const void *)k_begin, (const void *)k_finish, (const void *)k_after_inorder};
+        const void *small[] = {(const void *)k_begin, (const void *)k_finish};
         for (const void *f : small) { cudaError_t e = ensure_dyn_smem(f, 0); if (e != cudaSuccess) return e; }
     }
     mark(0);
