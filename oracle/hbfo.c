@@ -757,31 +757,26 @@ done:
 /* ---- submit, page-granular (an extension the paper only implies: its back end is a flash simulator that
  * works in pages, Section "Design"; what follows is this build's definition) ---------------------------------
  * A modeled access is cut at page boundaries of the media into parts; part k covers the bytes of the access
- * that fall into its k-th page.  Every part is a request of its own: it is decoded by its own first byte (so
- * consecutive pages follow the stripe interleave onto other channels, dies and planes), charged one page of
- * array time and the transfer of its own bytes (whole granules), and queued on its own queue in the order
- * (issue time, access index, part index).  The access completes when its last part does.  Per-die
- * statistics count parts (page operations); the batch summary counts accesses. */
-typedef struct { int64_t issue_ns; uint32_t idx; uint32_t part; uint64_t slot; } pent_t;
-
-static int cmp_pent(const void *pa, const void *pb) {
-    const pent_t *a = (const pent_t *)pa, *b = (const pent_t *)pb;
-    if (a->issue_ns != b->issue_ns) return a->issue_ns < b->issue_ns ? -1 : 1;
-    if (a->idx != b->idx) return a->idx < b->idx ? -1 : 1;
-    if (a->part != b->part) return a->part < b->part ? -1 : 1;
-    return 0;
-}
-
+ * that fall into its k-th page.  Every part is a request of its own: the batch of parts, listed in (access
+ * index, part index) order, is served exactly as hbfo_submit_batch serves a batch of accesses.  So a part is
+ * decoded by its own first byte (consecutive pages follow the stripe interleave onto other channels, dies and
+ * planes), charged one page of array time and the transfer of its own bytes (whole granules), and queued on its
+ * own queue in the order (issue time, access index, part index); and whatever else is switched on sees parts
+ * too: a part's array interval is an event of the energy ledger on the part's die, a read part's transfer
+ * queues on the bus of the part's channel in (array-done time, position in the list of parts) order, the parts
+ * claim outstanding refresh quanta in list order, one each, and a read part disturbs the block of its own
+ * page.  The access completes when its last part does.  Per-die statistics count parts (page operations); the
+ * batch summary counts accesses.  An access that is not modeled is one part. */
 int hbfo_submit_batch_paged(hbfo_ctx *c, const hbfo_access_t *acc, uint64_t n, int64_t *completion_ns,
                             int64_t *stall_ns, uint8_t *status, hbfo_die_stats_t *die_stats) {
-    if (!c || (n && (!acc || !completion_ns || !stall_ns)) || n > 0xffffffffull || c->ret) return HBFO_E_INVAL;
+    if (!c || (n && (!acc || !completion_ns || !stall_ns)) || n > 0xffffffffull) return HBFO_E_INVAL;
     hbfo_batch_result_t res; memset(&res, 0, sizeof(res));
-    const int64_t q = c->q_ppm;
-    res.mode = c->mode; res.q_ppm = q;
+    res.mode = c->mode; res.q_ppm = c->q_ppm;
     if (c->mode == HBFO_MODE_SHUTDOWN) { res.code = HBFO_E_LINK_SHUTDOWN; c->last = res; return res.code; }
     if (c->mode == HBFO_MODE_SEVERE)   { res.code = HBFO_E_THROTTLED;     c->last = res; return res.code; }
     c->order_count = 0;
 
+    /* the accesses' own status; a fault refuses the batch before anything is split */
     uint8_t *st = (uint8_t *)malloc(n ? n : 1);
     int32_t *rg = (int32_t *)malloc((n ? n : 1) * sizeof(int32_t));
     if (!st || !rg) { free(st); free(rg); return HBFO_E_NOMEM; }
@@ -789,7 +784,7 @@ int hbfo_submit_batch_paged(hbfo_ctx *c, const hbfo_access_t *acc, uint64_t n, i
     const uint64_t pg = c->cfg.page_bytes;
     for (uint64_t i = 0; i < n; ++i) {
         st[i] = (uint8_t)hbfo_classify(c, &acc[i], &rg[i]);
-        if (st[i] == HBFO_ST_NATIVE) ++n_native;
+        if (st[i] == HBFO_ST_NATIVE) { ++n_native; ++n_parts; }
         else if (st[i] == HBFO_ST_READY) {
             const range_t *r = &c->ranges[rg[i]];
             uint64_t off = r->media_offset + (acc[i].addr - r->base);
@@ -798,101 +793,61 @@ int hbfo_submit_batch_paged(hbfo_ctx *c, const hbfo_access_t *acc, uint64_t n, i
         } else ++n_fault;
     }
     if (status) memcpy(status, st, n);
-    if (die_stats) memset(die_stats, 0, c->n_dies * sizeof(hbfo_die_stats_t));
     if (n_fault) {
+        if (die_stats) memset(die_stats, 0, c->n_dies * sizeof(hbfo_die_stats_t));
         memset(completion_ns, 0, n * sizeof(int64_t)); memset(stall_ns, 0, n * sizeof(int64_t));
         res.code = HBFO_E_ACCESS_FAULT; res.n_fault = n_fault; res.n_native = n_native;
         c->last = res; free(st); free(rg);
         return res.code;
     }
+    if (n_parts > 0xffffffffull) { free(st); free(rg); return HBFO_E_INVAL; }
 
-    /* one record per part */
+    /* the list of parts: records of their own, in (access, part) order */
     const uint64_t m = n_parts ? n_parts : 1;
-    uint32_t *queue = (uint32_t *)malloc(m * sizeof(uint32_t));
-    uint32_t *die   = (uint32_t *)malloc(m * sizeof(uint32_t));
-    int64_t *a_ns = (int64_t *)malloc(m * sizeof(int64_t));
-    int64_t *s_ns = (int64_t *)malloc(m * sizeof(int64_t));
-    int64_t *post = (int64_t *)malloc(m * sizeof(int64_t));
-    int64_t *cbs  = (int64_t *)malloc(m * sizeof(int64_t));
-    int64_t *eng  = (int64_t *)malloc(m * sizeof(int64_t));
-    uint8_t *opp  = (uint8_t *)malloc(m);
-    uint64_t *cnt = (uint64_t *)calloc((size_t)c->n_queues + 1, sizeof(uint64_t));
-    pent_t *ent = (pent_t *)malloc(m * sizeof(pent_t));
-    pent_t *byq = (pent_t *)malloc(m * sizeof(pent_t));
-    hbfo_die_stats_t *ds = (hbfo_die_stats_t *)calloc(c->n_dies, sizeof(hbfo_die_stats_t));
+    hbfo_access_t *part = (hbfo_access_t *)malloc(m * sizeof(hbfo_access_t));
+    uint64_t *first = (uint64_t *)malloc((n + 1) * sizeof(uint64_t));   /* parts of access i: first[i] .. first[i + 1] - 1 */
+    int64_t *pc = (int64_t *)malloc(m * sizeof(int64_t)), *ps = (int64_t *)malloc(m * sizeof(int64_t));
     int rc = HBFO_OK;
-    if (!queue || !die || !a_ns || !s_ns || !post || !cbs || !eng || !opp || !cnt || !ent || !byq || !ds) { rc = HBFO_E_NOMEM; goto done; }
-
+    if (!part || !first || !pc || !ps) { rc = HBFO_E_NOMEM; goto done; }
     uint64_t slot = 0;
     for (uint64_t i = 0; i < n; ++i) {
-        if (st[i] != HBFO_ST_READY) continue;
+        first[i] = slot;
+        if (st[i] != HBFO_ST_READY) { part[slot++] = acc[i]; continue; }
         const range_t *r = &c->ranges[rg[i]];
         const uint64_t off = r->media_offset + (acc[i].addr - r->base), end = off + acc[i].bytes;
-        const uint32_t op = acc[i].flags & 1u;
-        uint32_t part = 0;
-        for (uint64_t lo = off; lo < end; ++part) {
+        for (uint64_t lo = off; lo < end; ) {
             uint64_t hi = (lo / pg + 1) * pg;                 /* next page boundary */
             if (hi > end) hi = end;
-            uint32_t ch, di, pl, qu; uint64_t np;
-            hbfo_decode(c, lo, (uint32_t)(hi - lo), &ch, &di, &pl, NULL, NULL, &np, &qu);   /* np is 1: the part lies in one page */
-            int64_t cb, xfer, s, e;
-            hbfo_service_terms(c, (uint32_t)(hi - lo), np, op, q, &cb, &xfer, &s, &e);
-            queue[slot] = qu; die[slot] = ch * c->cfg.dies + di; opp[slot] = (uint8_t)op;
-            s_ns[slot] = s; cbs[slot] = cb; eng[slot] = e;
-            if (op) { a_ns[slot] = acc[i].issue_ns + xfer; post[slot] = 0; }
-            else    { a_ns[slot] = acc[i].issue_ns;        post[slot] = xfer; }
-            ent[slot].issue_ns = acc[i].issue_ns; ent[slot].idx = (uint32_t)i; ent[slot].part = part; ent[slot].slot = slot;
-            cnt[qu + 1]++;
+            part[slot] = acc[i];
+            part[slot].addr = acc[i].addr + (lo - off);
+            part[slot].bytes = (uint32_t)(hi - lo);
             ++slot;
             lo = hi;
         }
     }
-    for (uint32_t r = 0; r < c->n_queues; ++r) cnt[r + 1] += cnt[r];
-    {
-        uint64_t *fill = (uint64_t *)malloc((size_t)c->n_queues * sizeof(uint64_t));
-        if (!fill) { rc = HBFO_E_NOMEM; goto done; }
-        memcpy(fill, cnt, (size_t)c->n_queues * sizeof(uint64_t));
-        for (uint64_t k = 0; k < n_parts; ++k) byq[fill[queue[k]]++] = ent[k];
-        free(fill);
-    }
-    for (uint32_t r = 0; r < c->n_queues; ++r)
-        qsort(byq + cnt[r], (size_t)(cnt[r + 1] - cnt[r]), sizeof(pent_t), cmp_pent);
+    first[n] = slot;
 
-    for (uint64_t i = 0; i < n; ++i) {
-        if (st[i] == HBFO_ST_NATIVE) { completion_ns[i] = acc[i].issue_ns; stall_ns[i] = 0; }
-        else completion_ns[i] = INT64_MIN;                    /* the maximum over the parts is taken below */
+    rc = hbfo_submit_batch(c, part, n_parts, pc, ps, NULL, die_stats);
+    c->order_count = 0;                                       /* the served order of parts is not reported */
+    if (rc != HBFO_OK) {                                      /* refused as a whole, nothing changed */
+        memset(completion_ns, 0, n * sizeof(int64_t)); memset(stall_ns, 0, n * sizeof(int64_t));
+        goto done;
     }
-    for (uint32_t r = 0; r < c->n_queues; ++r) {
-        int64_t B = c->busy_until[r];
-        for (uint64_t k = cnt[r]; k < cnt[r + 1]; ++k) {
-            const uint64_t p = byq[k].slot;
-            const uint32_t i = byq[k].idx;
-            int64_t start = a_ns[p] > B ? a_ns[p] : B;
-            B = start + s_ns[p];
-            int64_t done_ns = B + post[p];
-            if (done_ns > completion_ns[i]) completion_ns[i] = done_ns;
-            hbfo_die_stats_t *d = &ds[die[p]];
-            d->busy_ns += s_ns[p]; d->energy_pj += eng[p];
-            if (opp[p]) { d->bytes_prog += cbs[p]; d->n_prog += 1; }
-            else        { d->bytes_read += cbs[p]; d->n_read += 1; }
-            res.service_ns += s_ns[p];
-        }
-        c->busy_until[r] = B;
-    }
+    /* join: an access ends with the last of its parts */
+    res = c->last;
+    res.n_native = n_native; res.n_modeled = n_ready; res.modeled_ns = 0;
     for (uint64_t i = 0; i < n; ++i) {
-        if (st[i] != HBFO_ST_READY) continue;
-        stall_ns[i] = completion_ns[i] - acc[i].issue_ns;
+        if (st[i] != HBFO_ST_READY) { completion_ns[i] = acc[i].issue_ns; stall_ns[i] = 0; continue; }
+        int64_t last = pc[first[i]];
+        for (uint64_t k = first[i] + 1; k < first[i + 1]; ++k) if (pc[k] > last) last = pc[k];
+        completion_ns[i] = last;
+        stall_ns[i] = last - acc[i].issue_ns;
         res.modeled_ns += stall_ns[i];
-        if (completion_ns[i] > res.max_completion_ns) res.max_completion_ns = completion_ns[i];
     }
-    for (uint32_t d = 0; d < c->n_dies; ++d) c->pending_pj[d] += ds[d].energy_pj;
-    if (die_stats) memcpy(die_stats, ds, c->n_dies * sizeof(hbfo_die_stats_t));
-    res.code = HBFO_OK; res.n_native = n_native; res.n_modeled = n_ready;
     c->last = res;
 
 done:
-    free(st); free(rg); free(queue); free(die); free(a_ns); free(s_ns); free(post); free(cbs); free(eng); free(opp);
-    free(cnt); free(ent); free(byq); free(ds);
+    free(st); free(rg); free(part); free(first); free(pc); free(ps);
     return rc;
 }
 

@@ -81,7 +81,10 @@ int  hbfo_submit_batch(hbfo_ctx *ctx, const hbfo_access_t *acc, uint64_t n, int6
                        int64_t *stall_ns, uint8_t *status, hbfo_die_stats_t *die_stats);
 /* Page-granular variant (this build's extension; the paper's back end is a page-based flash simulator but the
  * text does not spell the splitting out): every page of a modeled access is a request of its own, queued by
- * its own decode; the access completes with its last part.  Same arguments as hbfo_submit_batch. */
+ * its own decode; the access completes with its last part.  Same arguments as hbfo_submit_batch.  The parts, listed
+ * in (access, part) order, are served as hbfo_submit_batch serves a batch of accesses, so the energy bins, the
+ * channel bus and retention, when on, see parts: one ledger event, one bus transfer, one possible refresh claim and
+ * one disturbing read per part. */
 int  hbfo_submit_batch_paged(hbfo_ctx *ctx, const hbfo_access_t *acc, uint64_t n, int64_t *completion_ns,
                              int64_t *stall_ns, uint8_t *status, hbfo_die_stats_t *die_stats);
 /* Time-bin power integration (Section "Design", event-based energy model: a ledger of energy per time bin, a long

@@ -340,10 +340,39 @@ def test_refused_batch_changes_nothing():
         assert np.array_equal(before[1][k], after[1][k])
 
 
-def test_not_with_the_paged_submit():
-    o, _ = make(RET)
-    rc, *_ = o.submit(recs([(0, 0, 64, 0)]), check=False, paged=True)
-    assert rc != 0
+def test_with_the_paged_submit_every_part_claims_and_disturbs_on_its_own():
+    """A 32 KiB read is two parts on two channels (stripe = page).  With two quanta owed both parts claim: each is served
+    395,000 + 20,000 ns from 10^6 on its own queue and moves its 16 KiB in 683 ns, so the access ends at 10^6 + 415,683 (as
+    one request of two pages it claims once and ends at 10^6 + 395,000 + 40,000 + 1,366).  With one quantum owed only the
+    first part claims.  Each part disturbs the block of its own page."""
+    ret = dict(RET, disturb_limit=1, lead_threshold=1e9, pages_per_block=2)
+    o, prof = make(ret)
+    o.submit(recs([(offset_of(prof, ret, 5, 0, 0, 0), 0, 64, 0)]))
+    o.retention_advance(0, np.array([40.0]))                              # block (5, 0, 0, 0) is due: two quanta
+    row = recs([(offset_of(prof, ret, 0, 0, 0, 0), 10**6, 2 * PAGE, 0)])
+    whole, _ = make(ret)
+    whole.submit(recs([(offset_of(prof, ret, 5, 0, 0, 0), 0, 64, 0)]))
+    whole.retention_advance(0, np.array([40.0]))
+    assert whole.submit(row)[1].tolist() == [10**6 + 436_366] and whole.retention_totals()["claimed"] == 1
+    _, comp, _, _, ds = o.submit(row, paged=True)
+    assert comp.tolist() == [10**6 + 415_683]
+    t = o.retention_totals()
+    assert t["claimed"] == 2 and t["commits"] == 1
+    P = prof["planes"]
+    busy = o.busy_until()
+    assert busy[(0 * prof["dies"] + 0) * P] == 10**6 + 415_000 and busy[(1 * prof["dies"] + 0) * P] == 10**6 + 415_000
+    d = o.retention_blocks()["disturb"]
+    assert d[block_id(prof, ret, 0, 0, 0, 0)] == 1 and d[block_id(prof, ret, 1, 0, 0, 0)] == 1
+    assert int(ds["busy_ns"].sum()) == 2 * 415_000 and int(ds["n_read"].sum()) == 2
+    # one quantum owed: the first part of the list claims, the second does not
+    ret1 = dict(ret, pages_per_block=1)
+    o1, prof = make(ret1)
+    o1.submit(recs([(offset_of(prof, ret1, 5, 0, 0, 0), 0, 64, 0)]))
+    o1.retention_advance(0, np.array([40.0]))
+    _, comp, _, _, _ = o1.submit(recs([(offset_of(prof, ret1, 0, 0, 0, 0), 10**6, 2 * PAGE, 0)]), paged=True)
+    assert comp.tolist() == [10**6 + 415_683] and o1.retention_totals()["claimed"] == 1
+    busy = o1.busy_until()
+    assert busy[(0 * prof["dies"] + 0) * P] == 10**6 + 415_000 and busy[(1 * prof["dies"] + 0) * P] == 10**6 + 20_000
 
 
 def test_with_the_channel_bus_claims_lengthen_the_array_stage_only():
