@@ -155,7 +155,11 @@ HBF_API int hbf_submit_host(hbf_ctx *ctx, const hbf_access_t *h_acc, uint64_t n,
  * the transfer of its own bytes in whole granules, queued in (issue_ns, access index, part index) order.  The
  * access completes when its last part does; d_stall_ns[i] = completion - issue.  d_die_stats counts parts
  * (page operations); the batch summary read with hbf_last_result counts accesses.  An access that is not
- * modeled (native, or failing) is one part.
+ * modeled (native, or failing) is one part.  The list of parts, in (access, part) order, is served as hbf_submit_batch
+ * serves a batch of accesses, so whatever else is switched on sees parts: with the energy bins a part's array interval
+ * is a ledger event on the part's die; with the channel-bus stage a read part's transfer queues on the bus of the part's
+ * channel in (array-done time, position in the list of parts) order; with retention the parts claim outstanding
+ * refresh quanta in list order, one each, and a read part disturbs the block of its own page.
  * parts_capacity: upper bound, chosen by the caller, of the number of parts of the batch (at least n; e.g.
  * n * (largest access / page_bytes + 2)); it sizes the workspace, hbf_workspace_bytes_paged(ctx, n, capacity).
  * The call counts the parts on the device and waits for that count (one stream synchronisation) before it
@@ -179,7 +183,7 @@ HBF_API int hbf_submit_batch_paged(hbf_ctx *ctx, const hbf_access_t *d_acc, uint
  * HBF_ISSUE_LIMIT): a batch whose largest completion time would reach 2^47 ns is refused with HBF_E_INVAL before anything
  * is committed (outputs zeroed, queue, bus and energy state unchanged); the context stays usable.
  * hbf_get_bus_busy_until synchronises and copies the per-channel bus state to host_out [channels]; hbf_reset clears
- * it.  hbf_submit_batch_paged is refused while the stage is on. */
+ * it.  With hbf_submit_batch_paged the stage queues parts (see there); its workspace then holds 4 bytes per part. */
 HBF_API int hbf_enable_channel_bus(hbf_ctx *ctx);
 HBF_API int hbf_get_bus_busy_until(hbf_ctx *ctx, int64_t *host_out, uint64_t cap);
 
@@ -192,8 +196,7 @@ HBF_API int hbf_get_bus_busy_until(hbf_ctx *ctx, int64_t *host_out, uint64_t cap
  * end into its last bin.  hbf_thermal_step must then be called with dt_ns == bin_ns (HBF_E_INVAL otherwise):
  * it consumes the clock's bin and advances the clock by one.  hbf_get_energy_bins synchronises and copies the
  * ring to host_out [n_bins][channels*dies] (row k = bin *first_bin + k).  The ledger is library-owned device
- * memory allocated by hbf_enable_energy_bins.
- * hbf_submit_batch_paged is refused (HBF_E_INVAL) while the ledger is on. */
+ * memory allocated by hbf_enable_energy_bins.  With hbf_submit_batch_paged every part is an event (see there). */
 HBF_API int hbf_enable_energy_bins(hbf_ctx *ctx, int64_t bin_ns, uint32_t n_bins);
 HBF_API int hbf_get_energy_bins(hbf_ctx *ctx, int64_t *host_out, uint64_t cap, int64_t *first_bin);
 
@@ -341,7 +344,7 @@ HBF_API int hbf_get_rom_temps(hbf_ctx *ctx, double *host_out, uint64_t cap);
  * page, programs add nothing; the modeled accesses of a batch claim in index (ticket) order; commits take effect
  * when the batch, or the decay, that claimed a block's last quantum has completed.
  *
- * hbf_enable_retention: allocates the block state (all fresh).  hbf_submit_batch_paged is refused while it is on.  The
+ * hbf_enable_retention: allocates the block state (all fresh).  With hbf_submit_batch_paged the parts claim and disturb (see there).  The
  *   channel-bus stage works on top of it unchanged (claims lengthen the array stage only).  With the energy bins on, a claimed quantum is an event of its
  *   own in the ledger: its energy over the interval in which it was served, ahead of the claiming access's event.
  * hbf_retention_advance: one epoch, asynchronously on the context's stream.  Every block that is not worn out gains

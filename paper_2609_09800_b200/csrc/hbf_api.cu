@@ -434,6 +434,36 @@ int hbf_set_path(hbf_ctx *c, int32_t path) {
     return HBF_OK;
 }
 
+// Everything a batch of records goes through once its arguments are in place: the claim window (retention), the submit
+// path, the energy ledger, read disturb / commits, the channel-bus stage.  Shared by hbf_submit_batch (the caller's
+// accesses) and hbf_submit_batch_paged (the list of parts).
+static int serve_records(hbf_ctx *c, SubmitArgs &a) {
+    a.ranges = c->d_ranges; a.mp_dev = c->d_mp; a.mp = c->mp; a.state = c->d_state; a.ctrl = c->d_ctrl; a.result = c->d_result;
+    a.busy = c->d_busy; a.busy_stage = c->d_busy_stage; a.pending = c->d_pending; a.stats_stage = c->d_stats_stage;
+    a.path = c->path; a.sm_count = c->sm_count; a.inorder_ok = c->inorder_ok ? 1 : 0;
+    if (c->ranges.size() == 1) {
+        const HostRange &r = c->ranges[0];
+        a.fast.base = r.base; a.fast.length = r.length; a.fast.media_offset = r.media_offset; a.fast.perms = r.perms; a.fast.on = 1u;
+    }
+    a.binned = c->bin_ns != 0; a.bus_on = c->d_bus_busy ? 1 : 0;
+    if (c->ret_on) {                                         // how far the outstanding refresh quanta reach into this batch
+        CK(launch_ret_window(a.acc, a.n, c->d_ranges, c->ret, c->sm_count, c->stream));
+        a.claim_limit = &c->ret.st->claim_limit; a.die_claims = c->ret.die_claims; a.ret = &c->ret;
+    }
+    CK(launch_submit(a, c->stream));
+    if (a.binned) {
+        const int64_t page = (int64_t)1 << c->mp.page_shift;
+        const int64_t quantum_pj = c->mp.e_cmd_read_pj + c->mp.e_byte_read_pj * page + c->mp.e_cmd_prog_pj + c->mp.e_byte_prog_pj * page;
+        CK(launch_energy_bins(a.acc, a.n, a.completion, c->d_ranges, c->d_mp, c->d_ctrl, c->d_result, c->d_ledger, c->bin_ns,
+                              c->n_bins, c->cur_bin, c->sm_count, a.claim_limit, quantum_pj, c->stream));
+    }
+    if (c->ret_on)                                           // read disturb, commits, the claimed energy (after the ledger: it needs the claim limit)
+        CK(launch_ret_close(a.acc, a.n, c->d_ranges, c->d_mp, c->mp, c->d_result, c->d_pending, a.binned, c->ret, c->sm_count, c->stream));
+    if (c->d_bus_busy)                                       // after the ledger: its events are the array intervals
+        CK(launch_bus_stage(a, c->d_bus_ctrl, c->d_bus_busy, c->stream));
+    return HBF_OK;
+}
+
 int hbf_submit_batch(hbf_ctx *c, const hbf_access_t *d_acc, uint64_t n, int64_t *d_completion_ns,
                      int64_t *d_stall_ns, uint8_t *d_status, hbf_die_stats_t *d_die_stats,
                      void *d_workspace, size_t workspace_bytes) {
@@ -447,32 +477,11 @@ int hbf_submit_batch(hbf_ctx *c, const hbf_access_t *d_acc, uint64_t n, int64_t 
     const size_t need = workspace_layout(n, c->mp.n_queues, &a.ws, d_workspace, c->d_bus_busy ? 1 : 0);
     if (!d_workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(d_workspace) & 255u)) return HBF_E_WORKSPACE;
     a.acc = d_acc; a.n = n; a.completion = d_completion_ns; a.stall = d_stall_ns; a.status = d_status; a.die_stats = d_die_stats;
-    a.ranges = c->d_ranges; a.mp_dev = c->d_mp; a.mp = c->mp; a.state = c->d_state; a.ctrl = c->d_ctrl; a.result = c->d_result;
-    a.busy = c->d_busy; a.busy_stage = c->d_busy_stage; a.pending = c->d_pending; a.stats_stage = c->d_stats_stage;
-    a.path = c->path; a.sm_count = c->sm_count; a.inorder_ok = c->inorder_ok ? 1 : 0;
-    if (c->ranges.size() == 1) {
-        const HostRange &r = c->ranges[0];
-        a.fast.base = r.base; a.fast.length = r.length; a.fast.media_offset = r.media_offset; a.fast.perms = r.perms; a.fast.on = 1u;
-    }
     c->prof_inorder = c->profiling && n > 0 && c->inorder_ok && (c->path == HBF_PATH_AUTO || c->path == HBF_PATH_INORDER);
     a.ev = c->profiling ? c->ev : nullptr;
     c->prof_submit = c->profiling;
-    a.binned = c->bin_ns != 0; a.bus_on = c->d_bus_busy ? 1 : 0;
-    if (c->ret_on) {                                         // how far the outstanding refresh quanta reach into this batch
-        CK(launch_ret_window(d_acc, n, c->d_ranges, c->ret, c->sm_count, c->stream));
-        a.claim_limit = &c->ret.st->claim_limit; a.die_claims = c->ret.die_claims; a.ret = &c->ret;
-    }
-    CK(launch_submit(a, c->stream));
-    if (a.binned) {
-        const int64_t page = (int64_t)1 << c->mp.page_shift;
-        const int64_t quantum_pj = c->mp.e_cmd_read_pj + c->mp.e_byte_read_pj * page + c->mp.e_cmd_prog_pj + c->mp.e_byte_prog_pj * page;
-        CK(launch_energy_bins(d_acc, n, d_completion_ns, c->d_ranges, c->d_mp, c->d_ctrl, c->d_result, c->d_ledger, c->bin_ns,
-                              c->n_bins, c->cur_bin, c->sm_count, a.claim_limit, quantum_pj, c->stream));
-    }
-    if (c->ret_on)                                           // read disturb, commits, the claimed energy (after the ledger: it needs the claim limit)
-        CK(launch_ret_close(d_acc, n, c->d_ranges, c->d_mp, c->mp, c->d_result, c->d_pending, a.binned, c->ret, c->sm_count, c->stream));
-    if (c->d_bus_busy)                                       // after the ledger: its events are the array intervals
-        CK(launch_bus_stage(a, c->d_bus_ctrl, c->d_bus_busy, c->stream));
+    const int rc = serve_records(c, a);
+    if (rc != HBF_OK) return rc;
     c->submitted = true;
     return HBF_OK;
 }
@@ -559,7 +568,7 @@ int hbf_submit_host(hbf_ctx *c, const hbf_access_t *h_acc, uint64_t n, int64_t *
 
 size_t hbf_workspace_bytes_paged(const hbf_ctx *c, uint64_t n, uint64_t parts_capacity) {
     if (!c) return 0;
-    return paged_layout(n, std::max<uint64_t>(parts_capacity, n), c->mp.n_queues, nullptr, nullptr);
+    return paged_layout(n, std::max<uint64_t>(parts_capacity, n), c->mp.n_queues, nullptr, nullptr, c->d_bus_busy ? 1 : 0);
 }
 
 int hbf_submit_batch_paged(hbf_ctx *c, const hbf_access_t *d_acc, uint64_t n, uint64_t parts_capacity,
@@ -570,13 +579,14 @@ int hbf_submit_batch_paged(hbf_ctx *c, const hbf_access_t *d_acc, uint64_t n, ui
         return hbf_submit_batch(c, d_acc, 0, d_completion_ns, d_stall_ns, d_status, d_die_stats, d_workspace, workspace_bytes);
     if (!on_own_device(c)) return HBF_E_INVAL;
     if (c->terminal) return HBF_E_LINK_SHUTDOWN;
-    if (n > HBF_MAX_BATCH || c->bin_ns != 0 || c->d_bus_busy || c->ret_on) return HBF_E_INVAL;   // ledger, bus stage and retention take whole accesses only
+    if (n > HBF_MAX_BATCH) return HBF_E_INVAL;
     if (!d_acc || !d_completion_ns || !d_stall_ns) return HBF_E_INVAL;
     if ((reinterpret_cast<uintptr_t>(d_acc) & 7u) || (reinterpret_cast<uintptr_t>(d_completion_ns) & 7u) ||
         (reinterpret_cast<uintptr_t>(d_stall_ns) & 7u) || (reinterpret_cast<uintptr_t>(d_die_stats) & 7u)) return HBF_E_INVAL;
     const uint64_t capacity = std::min<uint64_t>(std::max<uint64_t>(parts_capacity, n), HBF_MAX_BATCH);
     PagedWorkspace pw{};
-    const size_t need = paged_layout(n, capacity, c->mp.n_queues, &pw, d_workspace);
+    const int with_bus = c->d_bus_busy ? 1 : 0;
+    const size_t need = paged_layout(n, capacity, c->mp.n_queues, &pw, d_workspace, with_bus);
     if (!d_workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(d_workspace) & 255u)) return HBF_E_WORKSPACE;
     // how many parts: the one point where the host waits for the device inside a submit
     CK(launch_paged_count(d_acc, n, c->d_ranges, c->d_mp, pw, c->stream));
@@ -586,20 +596,15 @@ int hbf_submit_batch_paged(hbf_ctx *c, const hbf_access_t *d_acc, uint64_t n, ui
     const uint64_t total = *h_total;
     if (total > capacity) return HBF_E_WORKSPACE;            // nothing has changed: the caller may come back with more room
     CK(launch_paged_expand(d_acc, n, c->d_ranges, c->d_mp, capacity, pw, c->stream));
+    // the list of parts is a batch of records like any other: the ledger, the bus stage and retention, when on, see parts
     SubmitArgs a{};
-    workspace_layout(total, c->mp.n_queues, &a.ws, pw.inner);
+    workspace_layout(total, c->mp.n_queues, &a.ws, pw.inner, with_bus);
     a.acc = pw.parts; a.n = total; a.completion = pw.part_completion; a.stall = pw.part_stall; a.status = pw.part_status;
     a.die_stats = d_die_stats;
-    a.ranges = c->d_ranges; a.mp_dev = c->d_mp; a.mp = c->mp; a.state = c->d_state; a.ctrl = c->d_ctrl; a.result = c->d_result;
-    a.busy = c->d_busy; a.busy_stage = c->d_busy_stage; a.pending = c->d_pending; a.stats_stage = c->d_stats_stage;
-    a.path = c->path; a.sm_count = c->sm_count; a.inorder_ok = c->inorder_ok ? 1 : 0;
-    if (c->ranges.size() == 1) {
-        const HostRange &r = c->ranges[0];
-        a.fast.base = r.base; a.fast.length = r.length; a.fast.media_offset = r.media_offset; a.fast.perms = r.perms; a.fast.on = 1u;
-    }
     c->prof_inorder = false; c->prof_submit = false;
     a.ev = nullptr;
-    CK(launch_submit(a, c->stream));
+    const int rc = serve_records(c, a);
+    if (rc != HBF_OK) return rc;
     CK(launch_paged_join(d_acc, n, pw, c->d_result, d_completion_ns, d_stall_ns, d_status, c->sm_count, c->stream));
     c->submitted = true;
     return HBF_OK;

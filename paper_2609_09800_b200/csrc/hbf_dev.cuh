@@ -177,7 +177,7 @@ struct PagedWorkspace {
     void *inner; size_t inner_bytes;     // workspace of the ordinary path for `capacity` records
     size_t bytes;
 };
-size_t paged_layout(uint64_t n, uint64_t capacity, uint32_t n_queues, PagedWorkspace *pw, void *base);
+size_t paged_layout(uint64_t n, uint64_t capacity, uint32_t n_queues, PagedWorkspace *pw, void *base, int with_bus = 0);
 cudaError_t launch_paged_count(const hbf_access_t *acc, uint64_t n, const RangeSnap *ranges, const ModelParams *mp_dev,
                                const PagedWorkspace &pw, cudaStream_t st);
 cudaError_t launch_paged_expand(const hbf_access_t *acc, uint64_t n, const RangeSnap *ranges, const ModelParams *mp_dev,

@@ -176,7 +176,7 @@ __global__ void k_paged_finish(hbf_batch_result_t *result, const PagedSums *sums
     if (result->code == HBF_OK) { result->n_modeled = sums->n_ready; result->modeled_ns = (int64_t)sums->stall_sum; }
 }
 
-size_t paged_layout(uint64_t n, uint64_t capacity, uint32_t n_queues, PagedWorkspace *pw, void *base_ptr) {
+size_t paged_layout(uint64_t n, uint64_t capacity, uint32_t n_queues, PagedWorkspace *pw, void *base_ptr, int with_bus) {
     const uint64_t nn = n ? n : 1, cap = capacity ? capacity : 1;
     const uint64_t tiles = (nn + kPgTile - 1) / kPgTile;
     size_t off = 0;
@@ -184,7 +184,7 @@ size_t paged_layout(uint64_t n, uint64_t capacity, uint32_t n_queues, PagedWorks
     auto take = [&](size_t bytes) { size_t o = off; off = (off + bytes + 255) / 256 * 256; return b ? b + o : nullptr; };
     void *ts = take(tiles * 8), *tot = take(sizeof(PagedSums) + 8), *pf = take((nn + 1) * 4);
     void *pa = take(cap * sizeof(hbf_access_t)), *pc = take(cap * 8), *ps = take(cap * 8), *pst = take(cap);
-    const size_t inner = workspace_layout(cap, n_queues, nullptr, nullptr);
+    const size_t inner = workspace_layout(cap, n_queues, nullptr, nullptr, with_bus);
     void *in = take(inner);
     if (pw) {
         pw->tile_sum = (unsigned long long *)ts; pw->total = (unsigned long long *)tot;

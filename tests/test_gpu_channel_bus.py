@@ -98,8 +98,10 @@ def test_capacity_geometry_statuses_refusal_and_reset(hbf):
     g.reset(); o.reset()
     assert not g.get_bus_busy_until().any()
     compare(g, o, wm.acc)
-    rc, *_ = g.submit_host(wm.acc, check=False, parts_capacity=100_000)
-    assert rc == hbf.E_INVAL
+    rc_o, c_o, s_o, _, _ = o.submit(wm.acc, check=False, paged=True)          # the page-granular submit queues parts on the buses
+    rc_g, c_g, s_g, _, _ = g.submit_host(wm.acc, check=False, parts_capacity=100_000)
+    assert rc_g == rc_o == 0 and np.array_equal(c_g, c_o) and np.array_equal(s_g, s_o)
+    assert np.array_equal(g.get_bus_busy_until(), o.bus_busy_until())
 
 
 def test_with_the_energy_ledger_on(hbf):

@@ -80,14 +80,14 @@ def test_mixed_stream_in_two_batches(hbf, bin_ns, path):
     assert bins.sum() > 0 and not g.get_pending_energy().any()
 
 
-def test_refused_batches_book_nothing_and_paged_is_refused(hbf):
+def test_refused_batches_book_nothing(hbf):
     wf = wl.mixed_status(5000, seed=2, faults=True)
     g, o = contexts(hbf, wf.profile, wf.ranges)
     g.enable_energy_bins(100_000, 64); o.enable_energy_bins(100_000, 64)
     rc, *_ = g.submit_host(wf.acc, check=False)
     assert rc == hbf.E_ACCESS_FAULT and not g.energy_bins()[1].any()
-    rc, *_ = g.submit_host(wf.acc, check=False, parts_capacity=100_000)
-    assert rc == hbf.E_INVAL
+    rc, *_ = g.submit_host(wf.acc, check=False, parts_capacity=100_000)     # the page-granular submit refuses it the same way
+    assert rc == hbf.E_ACCESS_FAULT and not g.energy_bins()[1].any()
 
 
 def test_thermal_steps_consume_the_bins(hbf):

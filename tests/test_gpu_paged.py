@@ -98,3 +98,78 @@ def test_empty_batch_and_too_small_a_capacity(hbf):
     rc, *_ = g.submit_host(w.acc, check=False, parts_capacity=5000)     # these 5,000 reads have about 7,000 pages
     assert rc == hbf.E_WORKSPACE and not g.get_busy_until().any()
     compare(g, o, w.acc)
+
+
+# ---- with the energy ledger, the channel bus and retention on: the list of parts is served like any batch of records ----
+
+RET = dict(pages_per_block=4, blocks_per_plane=8, blocks_per_zone=2, max_pec=3, disturb_limit=40,
+           l_ref_s=1000.0, t_ref_c=40.0, ea_ev=1.04, accel=1.0, lead_threshold=0.02)
+
+
+def same_extras(g, o, bins, bus, ret):
+    if bins:
+        fg, bg = g.energy_bins(); fo, bo = o.energy_bins()
+        assert fg == fo
+        bad = np.argwhere(bg != bo)
+        assert bad.size == 0, "bins: first difference at bin %d die %d: gpu %d oracle %d" % (bad[0][0], bad[0][1], bg[tuple(bad[0])], bo[tuple(bad[0])])
+    if bus:
+        assert np.array_equal(g.get_bus_busy_until(), o.bus_busy_until())
+    if ret:
+        bg, bo = g.retention_blocks(), o.retention_blocks()
+        for k in ("disturb", "pec", "epoch"):
+            assert np.array_equal(bg[k], bo[k]), k
+        assert np.allclose(bg["damage"], bo["damage"], rtol=1e-12, atol=0.0)
+        assert g.retention_totals() == o.retention_totals()
+        assert np.array_equal(g.retention_plan(), o.retention_plan())
+
+
+def busy_stream(rng, n, t0, gap):
+    acc = np.zeros(n, hbfo.ACCESS_DTYPE)
+    acc["addr"] = wl.RANGE_BASE + rng.integers(0, 1 << 24, n).astype(np.uint64)
+    acc["issue_ns"] = t0 + np.sort(rng.integers(0, gap * n + 1, n))
+    acc["bytes"] = rng.choice([64, 4096, 16384, 20000, 65536, 200_000], n)
+    acc["flags"] = rng.random(n) < 0.1
+    nat = rng.random(n) < 0.05
+    acc["addr"][nat] = 0x2000 + 64 * np.arange(int(nat.sum()), dtype=np.uint64)
+    return acc
+
+
+@pytest.mark.parametrize("path", ["auto", "sort"])
+@pytest.mark.parametrize("extras", ["bins", "bus", "retention", "bins+bus+retention"])
+def test_parts_with_the_ledger_the_bus_and_retention(hbf, extras, path):
+    bins, bus, ret = "bins" in extras, "bus" in extras, "retention" in extras
+    prof = wl.load_profile("nominal", **wl.GEOMETRY["tiny"])
+    g, o = contexts(hbf, prof, [(wl.RANGE_BASE, wl.GIB, 3, 0, 0, 0)], hbf.PATH_AUTO if path == "auto" else hbf.PATH_SORT)
+    for x in (g, o):
+        if bins:
+            x.enable_energy_bins(250_000, 64)
+        if bus:
+            x.enable_channel_bus()
+        if ret:
+            x.enable_retention(**RET)
+    rng = np.random.default_rng(len(extras))
+    t0 = 0
+    for n in (1, 4000, 30_000, 2049):
+        acc = busy_stream(rng, n, t0, gap=4000)
+        assert compare(g, o, acc) == 0
+        same_extras(g, o, bins, bus, ret)
+        t0 = int(acc["issue_ns"][-1]) + 1
+        if ret:                                              # an epoch: disturbed blocks come due, the next batch's parts claim
+            g.retention_advance(10**9, np.array([50.0])); o.retention_advance(10**9, np.array([50.0]))
+            same_extras(g, o, bins, bus, ret)
+    if ret:
+        assert o.retention_totals()["claimed"] > 500
+    if bus:
+        assert o.bus_busy_until().any()
+    if bins:
+        assert o.energy_bins()[1].any()
+
+
+def test_a_refused_paged_batch_changes_nothing_with_everything_on(hbf):
+    wf = wl.mixed_status(6000, seed=4, faults=True)
+    g, o = contexts(hbf, wf.profile, wf.ranges)
+    for x in (g, o):
+        x.enable_energy_bins(100_000, 64); x.enable_channel_bus(); x.enable_retention(**RET)
+    assert compare(g, o, wf.acc) == hbfo.E_ACCESS_FAULT
+    same_extras(g, o, True, True, True)
+    assert not g.energy_bins()[1].any() and not g.get_bus_busy_until().any() and not g.retention_blocks()["disturb"].any()

@@ -292,11 +292,22 @@ def test_with_the_channel_bus(hbf, path):
     assert o.retention_totals()["claimed"] > 1000
 
 
-def test_not_with_the_paged_submit(hbf):
-    g, o, prof = contexts(hbf, RET)
-    acc = recs([(0, 0, 64, 0)])
-    rc, *_ = g.submit_host(acc, check=False, parts_capacity=4)
-    assert rc == hbf.E_INVAL
+def test_with_the_paged_submit_every_part_claims_and_disturbs_on_its_own(hbf):
+    """The oracle's hand-worked case: a 32 KiB read is two parts on two channels; with two quanta owed both claim."""
+    ret = dict(RET, disturb_limit=1, lead_threshold=1e9, pages_per_block=2)
+    g, o, prof = contexts(hbf, ret)
+    first = recs([(offset_of(prof, ret, 5, 0, 0, 0), 0, 64, 0)])
+    g.submit_host(first); o.submit(first)
+    g.retention_advance(0, np.array([40.0])); o.retention_advance(0, np.array([40.0]))
+    row = recs([(offset_of(prof, ret, 0, 0, 0, 0), 10**6, 2 * PAGE, 0)])
+    _, c_g, s_g, _, ds_g = g.submit_host(row, parts_capacity=4)
+    _, c_o, s_o, _, ds_o = o.submit(row, paged=True)
+    assert c_g.tolist() == [10**6 + 415_683] and np.array_equal(c_g, c_o) and np.array_equal(s_g, s_o)
+    assert g.retention_totals()["claimed"] == 2
+    for k in hbfo.DIE_STATS_DTYPE.names:
+        assert np.array_equal(ds_g[k], ds_o[k]), k
+    assert np.array_equal(g.get_busy_until(), o.busy_until())
+    compare_state(g, o)
 
 
 def test_reset_clears_the_block_state(hbf):
