@@ -595,7 +595,12 @@ int hbf_submit_batch_paged(hbf_ctx *c, const hbf_access_t *d_acc, uint64_t n, ui
     CK(cudaStreamSynchronize(c->stream));
     const uint64_t total = *h_total;
     if (total > capacity) return HBF_E_WORKSPACE;            // nothing has changed: the caller may come back with more room
-    CK(launch_paged_expand(d_acc, n, c->d_ranges, c->d_mp, capacity, pw, c->stream));
+    FastRange fast{};
+    if (c->ranges.size() == 1) {
+        const HostRange &r = c->ranges[0];
+        fast.base = r.base; fast.length = r.length; fast.media_offset = r.media_offset; fast.perms = r.perms; fast.on = 1u;
+    }
+    CK(launch_paged_expand(d_acc, n, c->d_ranges, c->d_mp, fast, c->mp.page_shift, capacity, pw, c->sm_count, c->stream));
     // the list of parts is a batch of records like any other: the ledger, the bus stage and retention, when on, see parts
     SubmitArgs a{};
     workspace_layout(total, c->mp.n_queues, &a.ws, pw.inner, with_bus);

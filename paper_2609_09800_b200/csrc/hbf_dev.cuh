@@ -169,6 +169,7 @@ cudaError_t launch_queue_order(const BatchCtrl *ctrl, const Workspace &ws, uint3
 // ---- page-granular submit ---------------------------------------------------------------------------
 struct PagedWorkspace {
     unsigned long long *tile_sum;        // [tiles of 2,048 accesses] parts per tile, then exclusive offsets
+    uint32_t *row_off;                   // [rows of 32 accesses] parts before the row within its tile
     unsigned long long *total;           // parts of the batch
     void *sums;                          // accesses served and their stall total
     uint32_t *part_first;                // [n + 1] first part of every access
@@ -181,7 +182,8 @@ size_t paged_layout(uint64_t n, uint64_t capacity, uint32_t n_queues, PagedWorks
 cudaError_t launch_paged_count(const hbf_access_t *acc, uint64_t n, const RangeSnap *ranges, const ModelParams *mp_dev,
                                const PagedWorkspace &pw, cudaStream_t st);
 cudaError_t launch_paged_expand(const hbf_access_t *acc, uint64_t n, const RangeSnap *ranges, const ModelParams *mp_dev,
-                                uint64_t capacity, const PagedWorkspace &pw, cudaStream_t st);
+                                const FastRange &fast, uint32_t page_shift, uint64_t capacity, const PagedWorkspace &pw, int sm_count,
+                                cudaStream_t st);
 cudaError_t launch_paged_join(const hbf_access_t *acc, uint64_t n, const PagedWorkspace &pw, hbf_batch_result_t *result,
                               int64_t *completion, int64_t *stall, uint8_t *status, int sm_count, cudaStream_t st);
 

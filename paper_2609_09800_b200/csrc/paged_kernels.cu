@@ -1,9 +1,11 @@
 // Page-granular submit: every page a modeled access touches becomes a request of its own (decoded by its own
 // first byte, one page of array time, the transfer of its own bytes), and the access completes with its last
 // part.  The paper's back end is a page-based flash simulator; the splitting rule itself is this library's.
-//   count   parts per access (1 for an access that is not modeled), summed per tile of 2,048 accesses
+//   count   parts per access (1 for an access that is not modeled), summed per row of 32 accesses and per tile of 64 rows;
+//           a row's parts-before-it within its tile are kept
 //   scan    exclusive scan of the tile sums by one block; the total goes back to the host, which sizes the rest
-//   expand  every tile writes its accesses' parts, in (access, part) order, as ordinary access records
+//   expand  a warp per row, no block-wide step: the warp reads its 32 records, knows where its parts begin (tile offset
+//           + row offset), and writes them, in (access, part) order, as ordinary access records
 //   serve   the ordinary submit path runs on the part records (they keep the batch's issue order)
 //   join    completion of an access = the latest completion of its parts; the batch summary counts accesses
 #include <algorithm>
@@ -15,6 +17,7 @@ namespace hbf {
 constexpr int kPgThreads = 256;
 constexpr int kPgItems = 8;
 constexpr int kPgTile = kPgThreads * kPgItems;
+constexpr int kPgRows = kPgTile / 32;                    // rows of 32 consecutive accesses per tile
 
 // parts of one access: its pages when it is modeled, one (the record itself) otherwise
 __device__ __forceinline__ uint32_t parts_of(const RangeSnap &rs, const ModelParams &mp, const uint64_t *rec, uint64_t *first_bytes) {
@@ -30,25 +33,45 @@ __device__ __forceinline__ uint32_t parts_of(const RangeSnap &rs, const ModelPar
     return (uint32_t)((in_page + bytes + page - 1ull) >> mp.page_shift);
 }
 
+// the same with the one registered range in the kernel's arguments: nothing is read from memory to classify
+__device__ __forceinline__ uint32_t parts_of_fast(const FastRange &fr, uint32_t page_shift, uint64_t addr, int64_t issue, uint64_t bf,
+                                                  uint32_t *first_bytes) {
+    const uint32_t bytes = (uint32_t)bf, flags = (uint32_t)(bf >> 32);
+    const uint64_t rel = addr - fr.base;
+    const uint32_t need = (flags & 1u) ? (uint32_t)HBF_PERM_PROGRAM : (uint32_t)HBF_PERM_READ;
+    const bool ready = bytes != 0u && (flags & ~1u) == 0u && issue >= 0 && issue < HBF_ISSUE_LIMIT && addr >= fr.base &&
+                       rel < fr.length && (uint64_t)bytes <= fr.length - rel && (fr.perms & need) != 0u;
+    *first_bytes = bytes;
+    if (!ready) return 1u;
+    const uint32_t page = 1u << page_shift, in_page = (uint32_t)(fr.media_offset + rel) & (page - 1u);
+    *first_bytes = min(bytes, page - in_page);
+    return (uint32_t)(((uint64_t)in_page + bytes + page - 1u) >> page_shift);
+}
+
 __global__ void __launch_bounds__(kPgThreads)
 k_paged_count(const hbf_access_t *__restrict__ acc, uint64_t n, const RangeSnap *__restrict__ ranges, const ModelParams *__restrict__ mp,
-              unsigned long long *__restrict__ tile_sum) {
-    __shared__ unsigned long long s_warp[kPgThreads / 32];
+              unsigned long long *__restrict__ tile_sum, uint32_t *__restrict__ row_off) {
+    __shared__ uint32_t s_row[kPgRows];
     const uint64_t base = (uint64_t)blockIdx.x * kPgTile;
-    unsigned long long mine = 0;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 #pragma unroll
-    for (int j = 0; j < kPgItems; ++j) {
-        const uint64_t i = base + (uint64_t)(j * kPgThreads + threadIdx.x);
+    for (int j = 0; j < kPgItems; ++j) {                     // row j * 8 + warp of the tile: accesses base + 32 row .. + 31
+        const uint64_t i = base + (uint64_t)(j * kPgThreads + tid);
         uint64_t fb;
-        if (i < n) mine += parts_of(*ranges, *mp, reinterpret_cast<const uint64_t *>(acc + i), &fb);
+        uint32_t c = i < n ? parts_of(*ranges, *mp, reinterpret_cast<const uint64_t *>(acc + i), &fb) : 0u;
+        c = (uint32_t)warp_sum((long long)c);
+        if (lane == 0) s_row[j * (kPgThreads / 32) + warp] = c;
     }
-    mine = (unsigned long long)warp_sum((long long)mine);
-    if ((threadIdx.x & 31) == 0) s_warp[threadIdx.x >> 5] = mine;
     __syncthreads();
-    if (threadIdx.x == 0) {
-        unsigned long long t = 0;
-        for (int w = 0; w < kPgThreads / 32; ++w) t += s_warp[w];
-        tile_sum[blockIdx.x] = t;
+    if (warp == 0) {                                         // exclusive scan of the 64 row sums: two per lane
+        const uint32_t a = s_row[2 * lane], b = s_row[2 * lane + 1];
+        uint32_t incl = a + b;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += t; }
+        const uint32_t before = incl - (a + b);
+        uint32_t *ro = row_off + (uint64_t)blockIdx.x * kPgRows;
+        ro[2 * lane] = before; ro[2 * lane + 1] = before + a;
+        if (lane == 31) tile_sum[blockIdx.x] = incl;
     }
 }
 
@@ -78,66 +101,87 @@ k_paged_tile_scan(unsigned long long *tile_sum, uint64_t n_tiles, unsigned long 
     if (tid == 0) *total = s_carry;
 }
 
-// A tile first lays out where the parts of each of its accesses go (thread t takes kPgItems consecutive accesses,
-// block scan of the counts); then the threads walk the tile's OUTPUT slots, consecutive threads writing
-// consecutive part records: each finds its access by binary search in the tile's offsets and cuts its part out.
+// A warp per row of 32 consecutive accesses, rows dealt round-robin to the grid's warps; no block-wide step.  The warp
+// reads its 768 bytes of records, scans the part counts with shuffles, and every lane writes the parts of its access,
+// walking through the access page by page: the 32 accesses' parts are consecutive in the output, so a warp's stores of
+// one round fall into one short stretch.  An access of more than kPgWide parts (a very large access) is cut by the
+// whole warp, a part per lane.  The kernel is bound by instruction issue, not by its bytes, which is why the common
+// case (one registered range, an access inside one page) is kept short.
+constexpr uint32_t kPgWide = 8;
+constexpr int kPgUnroll = 2;                             // rows whose loads a warp has in flight together
+constexpr int kPgWaves = 4;                              // blocks of the expand grid per resident block slot
+
+template <bool FAST>
 __global__ void __launch_bounds__(kPgThreads)
 k_paged_expand(const hbf_access_t *__restrict__ acc, uint64_t n, const RangeSnap *__restrict__ ranges, const ModelParams *__restrict__ mp,
-               const unsigned long long *__restrict__ tile_off, uint64_t capacity, hbf_access_t *__restrict__ parts,
-               uint32_t *__restrict__ part_first) {
-    __shared__ unsigned long long s_warp[kPgThreads / 32];
-    __shared__ uint32_t s_first[kPgTile + 1];               // first part of every access of the tile, relative to the tile's first
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint64_t tile_base = (uint64_t)blockIdx.x * kPgTile;
-    const uint32_t in_tile = (uint32_t)min((uint64_t)kPgTile, n - tile_base);
-    const uint64_t first = tile_base + (uint64_t)tid * kPgItems;
-    uint32_t cnt[kPgItems];
-    unsigned long long mine = 0;
+               const FastRange fast, const uint32_t page_shift, const unsigned long long *__restrict__ tile_off,
+               const uint32_t *__restrict__ row_off, uint64_t capacity, hbf_access_t *__restrict__ parts, uint32_t *__restrict__ part_first) {
+    const int lane = threadIdx.x & 31;
+    const uint64_t warps = (uint64_t)gridDim.x * (kPgThreads / 32), rows = (n + 31) / 32;
+    const uint32_t page = 1u << page_shift;
+    uint64_t *out = reinterpret_cast<uint64_t *>(parts);
+    for (uint64_t row0 = (uint64_t)blockIdx.x * (kPgThreads / 32) + (threadIdx.x >> 5); row0 < rows; row0 += warps * kPgUnroll) {
+        // the loads of kPgUnroll rows go out together
+        uint64_t r_addr[kPgUnroll], r_issue[kPgUnroll], r_bf[kPgUnroll], r_at[kPgUnroll];
 #pragma unroll
-    for (int j = 0; j < kPgItems; ++j) {
-        uint64_t fb;
-        cnt[j] = first + j < n ? parts_of(*ranges, *mp, reinterpret_cast<const uint64_t *>(acc + first + j), &fb) : 0u;
-        mine += cnt[j];
-    }
-    unsigned long long incl = mine;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) { const unsigned long long t = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += t; }
-    if (lane == 31) s_warp[warp] = incl;
-    __syncthreads();
-    unsigned long long local = incl - mine;
-    for (int w = 0; w < warp; ++w) local += s_warp[w];
-    const unsigned long long off0 = tile_off[blockIdx.x];
-#pragma unroll
-    for (int j = 0; j < kPgItems; ++j) {
-        if (first + j < n) {
-            s_first[tid * kPgItems + j] = (uint32_t)local;
-            part_first[first + j] = (uint32_t)(off0 + local);
-            local += cnt[j];
+        for (int u = 0; u < kPgUnroll; ++u) {
+            const uint64_t row = row0 + (uint64_t)u * warps, i = row * 32 + (uint64_t)lane;
+            r_addr[u] = r_issue[u] = r_bf[u] = r_at[u] = 0ull;
+            if (row < rows) r_at[u] = tile_off[row / kPgRows] + row_off[row];
+            if (i < n) {
+                const uint64_t *rec = reinterpret_cast<const uint64_t *>(acc + i);
+                r_addr[u] = __ldg(rec); r_issue[u] = __ldg(rec + 1); r_bf[u] = __ldg(rec + 2);
+            }
         }
-    }
-    unsigned long long tile_total = 0;
-    for (int w = 0; w < kPgThreads / 32; ++w) tile_total += s_warp[w];
-    if (tid == 0) {
-        s_first[in_tile] = (uint32_t)tile_total;
-        if (tile_base + in_tile == n) part_first[n] = (uint32_t)(off0 + tile_total);     // the tile that holds the last access
-    }
-    __syncthreads();
-    const uint64_t page = 1ull << mp->page_shift;
-    for (unsigned long long k = (unsigned long long)tid; k < tile_total; k += kPgThreads) {
-        uint32_t lo = 0, hi = in_tile;                       // last access e with s_first[e] <= k
-        while (hi - lo > 1u) { const uint32_t mid = (lo + hi) >> 1; if ((unsigned long long)s_first[mid] <= k) lo = mid; else hi = mid; }
-        const uint32_t e = lo, part = (uint32_t)(k - s_first[e]), of = s_first[e + 1] - s_first[e];
-        hbf_access_t r = acc[tile_base + e];
-        if (of > 1u) {                                       // a modeled access of several pages
-            int g = 0;
-            classify(*ranges, r.addr, r.issue_ns, r.bytes, r.flags, &g);
-            const uint64_t off = ranges->media_offset[g] + (r.addr - ranges->base[g]);
-            const uint64_t head = page - (off & (page - 1ull));          // bytes in its first page
-            const uint64_t skip = part == 0u ? 0ull : head + (uint64_t)(part - 1u) * page;
-            const uint64_t len = part == 0u ? head : min((uint64_t)r.bytes - skip, page);
-            r.addr += skip; r.bytes = (uint32_t)len;
+#pragma unroll
+        for (int u = 0; u < kPgUnroll; ++u) {
+        const uint64_t row = row0 + (uint64_t)u * warps;
+        if (row >= rows) break;
+        const uint64_t i = row * 32 + (uint64_t)lane;
+        const bool have = i < n;
+        const uint64_t addr = r_addr[u], issue = r_issue[u], bf = r_bf[u];
+        uint32_t cnt = 0u, head = 0u;
+        const uint64_t row_at = r_at[u];
+        if (have) {
+            if (FAST) cnt = parts_of_fast(fast, page_shift, addr, (int64_t)issue, bf, &head);
+            else { uint64_t h; cnt = parts_of(*ranges, *mp, reinterpret_cast<const uint64_t *>(acc + i), &h); head = (uint32_t)h; }
         }
-        if (off0 + k < capacity) parts[off0 + k] = r;       // the host checked the total against the capacity before this launch
+        uint32_t incl = cnt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += t; }
+        const uint64_t at = row_at + (incl - cnt);
+        if (have) part_first[i] = (uint32_t)at;
+        if (i == n - 1) part_first[n] = (uint32_t)(at + cnt);
+        // the host checked the total against the capacity before this launch; the tests on it only keep a wrong call harmless
+        if (cnt == 1u) {
+            if (at < capacity) { uint64_t *o = out + at * 3ull; o[0] = addr; o[1] = issue; o[2] = bf; }
+        } else if (cnt > 1u && cnt <= kPgWide) {
+            uint64_t *o = out + at * 3ull;
+            uint64_t a = addr;
+            uint32_t left = (uint32_t)bf, len = head;
+            const uint64_t hi = bf & 0xffffffff00000000ull;
+            for (uint32_t p = 0; p < cnt; ++p) {
+                if (at + p < capacity) { o[0] = a; o[1] = issue; o[2] = hi | len; }
+                o += 3; a += len; left -= len; len = min(left, page);
+            }
+        }
+        unsigned wide = __ballot_sync(0xffffffffu, cnt > kPgWide);
+        while (wide) {
+            const int src = __ffs(wide) - 1;
+            wide &= wide - 1u;
+            const uint64_t a0 = __shfl_sync(0xffffffffu, addr, src), is = __shfl_sync(0xffffffffu, issue, src);
+            const uint64_t b = __shfl_sync(0xffffffffu, bf, src), base_at = __shfl_sync(0xffffffffu, at, src);
+            const uint32_t hd = __shfl_sync(0xffffffffu, head, src), c = __shfl_sync(0xffffffffu, cnt, src);
+            for (uint32_t p = (uint32_t)lane; p < c; p += 32u) {
+                const uint64_t skip = p == 0u ? 0ull : (uint64_t)hd + (uint64_t)(p - 1u) * page;
+                const uint64_t len = p == 0u ? (uint64_t)hd : min((uint64_t)(uint32_t)b - skip, (uint64_t)page);
+                if (base_at + p < capacity) {
+                    uint64_t *o = out + (base_at + p) * 3ull;
+                    o[0] = a0 + skip; o[1] = is; o[2] = (b & 0xffffffff00000000ull) | len;
+                }
+            }
+        }
+        }
     }
 }
 
@@ -182,12 +226,12 @@ size_t paged_layout(uint64_t n, uint64_t capacity, uint32_t n_queues, PagedWorks
     size_t off = 0;
     char *b = static_cast<char *>(base_ptr);
     auto take = [&](size_t bytes) { size_t o = off; off = (off + bytes + 255) / 256 * 256; return b ? b + o : nullptr; };
-    void *ts = take(tiles * 8), *tot = take(sizeof(PagedSums) + 8), *pf = take((nn + 1) * 4);
+    void *ts = take(tiles * 8), *ro = take(tiles * kPgRows * 4), *tot = take(sizeof(PagedSums) + 8), *pf = take((nn + 1) * 4);
     void *pa = take(cap * sizeof(hbf_access_t)), *pc = take(cap * 8), *ps = take(cap * 8), *pst = take(cap);
     const size_t inner = workspace_layout(cap, n_queues, nullptr, nullptr, with_bus);
     void *in = take(inner);
     if (pw) {
-        pw->tile_sum = (unsigned long long *)ts; pw->total = (unsigned long long *)tot;
+        pw->tile_sum = (unsigned long long *)ts; pw->row_off = (uint32_t *)ro; pw->total = (unsigned long long *)tot;
         pw->sums = (void *)((char *)tot + (tot ? 8 : 0)); pw->part_first = (uint32_t *)pf;
         pw->parts = (hbf_access_t *)pa; pw->part_completion = (int64_t *)pc; pw->part_stall = (int64_t *)ps; pw->part_status = (uint8_t *)pst;
         pw->inner = in; pw->inner_bytes = inner; pw->bytes = off;
@@ -200,16 +244,21 @@ cudaError_t launch_paged_count(const hbf_access_t *acc, uint64_t n, const RangeS
     const uint64_t tiles = (n + kPgTile - 1) / kPgTile;
     cudaError_t e = cudaMemsetAsync(pw.total, 0, sizeof(PagedSums) + 8, st);
     if (e != cudaSuccess) return e;
-    k_paged_count<<<(unsigned)tiles, kPgThreads, 0, st>>>(acc, n, ranges, mp_dev, pw.tile_sum);
+    k_paged_count<<<(unsigned)tiles, kPgThreads, 0, st>>>(acc, n, ranges, mp_dev, pw.tile_sum, pw.row_off);
     k_paged_tile_scan<<<1, 1024, 0, st>>>(pw.tile_sum, tiles, pw.total);
     g_kernel_launches += 2;
     return cudaGetLastError();
 }
 
 cudaError_t launch_paged_expand(const hbf_access_t *acc, uint64_t n, const RangeSnap *ranges, const ModelParams *mp_dev,
-                                uint64_t capacity, const PagedWorkspace &pw, cudaStream_t st) {
-    const uint64_t tiles = (n + kPgTile - 1) / kPgTile;
-    k_paged_expand<<<(unsigned)tiles, kPgThreads, 0, st>>>(acc, n, ranges, mp_dev, pw.tile_sum, capacity, pw.parts, pw.part_first);
+                                const FastRange &fast, uint32_t page_shift, uint64_t capacity, const PagedWorkspace &pw, int sm_count,
+                                cudaStream_t st) {
+    const uint64_t blocks = ((n + 31) / 32 + kPgThreads / 32 - 1) / (kPgThreads / 32);
+    const unsigned grid = (unsigned)std::min<uint64_t>(blocks, (uint64_t)std::max(1, sm_count) * 8 * kPgWaves);
+    if (fast.on)
+        k_paged_expand<true><<<grid, kPgThreads, 0, st>>>(acc, n, ranges, mp_dev, fast, page_shift, pw.tile_sum, pw.row_off, capacity, pw.parts, pw.part_first);
+    else
+        k_paged_expand<false><<<grid, kPgThreads, 0, st>>>(acc, n, ranges, mp_dev, fast, page_shift, pw.tile_sum, pw.row_off, capacity, pw.parts, pw.part_first);
     g_kernel_launches += 1;
     return cudaGetLastError();
 }
