@@ -159,6 +159,9 @@ struct InTile { long long spec_sum, fix_delta, true_sum; uint32_t reserve; uint3
 size_t inorder_head_bytes(uint64_t tiles, uint32_t n_queues);
 size_t inorder_serve_smem(uint32_t n_dies);
 cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st);
+constexpr uint32_t kInSmallMax = 8192;   // batches of at most this many records are served by one block in one launch
+bool inorder_small_batch(uint64_t n);   // whether launch_inorder takes that route
+uint32_t inorder_small_blocks(uint32_t n_queues);   // its blocks: each leaves one entry of the tile table (the slice's stall total)
 cudaError_t launch_submit(const SubmitArgs &a, cudaStream_t st);
 // total[i] += part[i] over the 6 * n_dies counters of a per-die statistics array (host-buffer pipeline: totals over its chunks)
 cudaError_t launch_add_stats(hbf_die_stats_t *total, const hbf_die_stats_t *part, uint32_t n_dies, cudaStream_t st);

@@ -967,12 +967,6 @@ k_inorder_fixstraggle(const hbf_access_t *__restrict__ acc, uint64_t n, const __
 #ifndef HBF_IN_SKEW_PERMILLE
 #define HBF_IN_SKEW_PERMILLE 60
 #endif
-// Batches of at most this many records are one tile (served from the true queue state, exact at once, no fix-up or
-// straggle launch).  Measured on 1 ms batches of 5,900 records: one block serving them all takes 65 us (about 0.3 us per
-// row of 32 when nothing else hides the latency of the row chain), six tiles with the fix-up kernel behind them 54 us;
-// the single tile wins only up to about two thousand records.
-constexpr uint64_t kInSingleTile = 2048;
-
 // One wave of resident blocks: as many tiles as the device holds serve blocks.  When the batch is large enough to fill
 // that wave, the tiles of the blocks that the hardware favours (one per SM) are larger by the skew, the others smaller,
 // so that both blocks of an SM finish together.
@@ -982,10 +976,6 @@ InTileMap inorder_tile_map(uint64_t n, int sm_count) {
     const uint64_t sms = (uint64_t)std::max(1, sm_count);
     const uint64_t want_tiles = std::min<uint64_t>(kInMaxTiles, sms * kInBlocksPerSM);
     auto round_up = [](uint64_t v) { return std::max<uint64_t>((v + kInTileQuantum - 1) / kInTileQuantum * kInTileQuantum, kInTileQuantum); };
-    if (n <= kInSingleTile) {                                // a small batch: one tile, served from the true queue state, is exact at once
-        m.n_big = 0; m.big = m.small = (uint32_t)round_up(n); m.n_tiles = 1;
-        return m;
-    }
     const uint64_t even = round_up((n + want_tiles - 1) / want_tiles);
     if (kInBlocksPerSM == 2 && want_tiles == 2 * sms && even >= 64 * kInTileQuantum && HBF_IN_SKEW_PERMILLE > 0) {
         const uint64_t big = round_up(even * (1000 + HBF_IN_SKEW_PERMILLE) / 1000);
@@ -1008,10 +998,322 @@ static size_t inorder_straggle_smem() {
     return (size_t)kInMaxQueues * 16 + (size_t)kInStrKeep * 24 + (size_t)kInMaxQueues * 4 + (size_t)kInStrMaxStragglers * (kInStrList * 2 + 4);
 }
 
+// ======================================================================================================
+// Small batches (at most kInSmallMax records, in issue order) are served exactly in one launch, instead of tiles, a scan, a
+// fix-up and a straggle pass whose fixed costs a few thousand records cannot pay for.  Queues do not interact, so the
+// queues are dealt to the blocks in slices of 64 consecutive ones, and a block serves its slice on its own; no block
+// waits for another.  Every block reads ALL the records (a few hundred KB, from the L2 after the first block):
+//   terms   every thread takes records i, i + 1024, ...: status, queue, service terms (the short form for the common
+//           configuration, else the general one).  Every block counts the statuses of the whole batch, so all blocks
+//           take the same decision about it; a record of the block's slice leaves service and transfer in shared
+//           memory by batch index and gets the sort key (queue in the slice) << 14 | index << 1 | op; the others all ones
+//   sort    one stable radix pass over the 6 queue bits of the slice, in shared memory: a warp owns consecutive keys and
+//           ranks them 32 at a time (match_any); keys of other slices go behind every queue
+//   serve   a segmented max-plus scan over the slice's sorted keys (a queue's run is a segment): every thread owns up to 8
+//           consecutive entries, composes their maps, the block scans the threads' maps, and the thread walks its
+//           entries again from the busy-until that reaches it; per-die totals are summed along the runs (a die's
+//           queues are neighbours)
+// Statuses and the results of records that are not modeled are written by the block whose turn the record's round is.
+// A batch that is not in issue order is handed to the sort path exactly as the tiled path hands it over.
+// ======================================================================================================
+constexpr int kInSmallThreads = 1024;
+constexpr int kInSmallWarps = kInSmallThreads / 32;
+constexpr uint32_t kInSmallItems = kInSmallMax / kInSmallThreads;          // sorted entries per thread, at most
+constexpr uint32_t kInSmallIdxBits = 13, kInSmallQShift = kInSmallIdxBits + 1;
+constexpr uint32_t kInSmallSlice = 64;                                     // queues per block: the bins of the radix pass, plus one for the rest
+static_assert((1u << kInSmallIdxBits) == kInSmallMax, "index << 1 | op fits below the queue bits of the key");
+static_assert(kInSmallMax % (kInSmallWarps * 32) == 0 && kInSmallWarps == 32, "a warp sorts whole rounds of 32 keys; a lane per warp in the offsets' scan");
+
+size_t inorder_small_smem() { return (size_t)kInSmallMax * (8 + 4 + 4 + 4); }
+uint32_t inorder_small_blocks(uint32_t n_queues) { return (n_queues + kInSmallSlice - 1) / kInSmallSlice; }
+
+// one stable pass: src -> dst by the queue bits of the key; keys that are all ones take the extra bin behind every queue
+__device__ __forceinline__ void small_radix_pass(const uint32_t *src, uint32_t *dst, uint32_t padded,
+                                                 uint32_t (*hist)[kInSmallSlice + 1], uint32_t *dbase) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t per_warp = padded / kInSmallWarps;                      // (padded is a multiple of 1024)
+    auto digit = [&](uint32_t key) { return key == 0xffffffffu ? kInSmallSlice : key >> kInSmallQShift; };
+    for (uint32_t e = tid; e < kInSmallWarps * (kInSmallSlice + 1); e += kInSmallThreads) (&hist[0][0])[e] = 0u;
+    __syncthreads();
+    for (uint32_t r = 0; r < per_warp; r += 32u) {                         // counts per (warp, digit)
+        const uint32_t d = digit(src[warp * per_warp + r + lane]);
+        const unsigned peers = __match_any_sync(0xffffffffu, d);
+        if (lane == __ffs(peers) - 1) hist[warp][d] += __popc(peers);
+        __syncwarp();
+    }
+    __syncthreads();
+    // where the keys of (digit, warp) begin: digits in order, within a digit the warps in order
+    for (uint32_t d = warp; d <= kInSmallSlice; d += kInSmallWarps) {      // lane = the warp whose count this is
+        const uint32_t v = hist[lane][d];
+        uint32_t inc = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += t; }
+        hist[lane][d] = inc - v;
+        if (lane == 31) dbase[d] = inc;
+    }
+    __syncthreads();
+    if (warp == 0) {                                                       // exclusive scan of the 65 digit totals: three per lane
+        uint32_t v[3], sum = 0;
+#pragma unroll
+        for (int k = 0; k < 3; ++k) { const uint32_t d = lane * 3 + k; v[k] = d <= kInSmallSlice ? dbase[d] : 0u; sum += v[k]; }
+        uint32_t inc = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += t; }
+        uint32_t run = inc - sum;
+#pragma unroll
+        for (int k = 0; k < 3; ++k) { const uint32_t d = lane * 3 + k; if (d <= kInSmallSlice) dbase[d] = run; run += v[k]; }
+    }
+    __syncthreads();
+    for (uint32_t r = 0; r < per_warp; r += 32u) {                         // scatter, 32 keys at a time, in order
+        const uint32_t key = src[warp * per_warp + r + lane], d = digit(key);
+        const unsigned peers = __match_any_sync(0xffffffffu, d);
+        const uint32_t rank = __popc(peers & ((1u << lane) - 1u));
+        dst[dbase[d] + hist[warp][d] + rank] = key;
+        __syncwarp();
+        if (lane == __ffs(peers) - 1) hist[warp][d] += __popc(peers);
+        __syncwarp();
+    }
+    __syncthreads();
+}
+
+template <bool DEBT>
+__global__ void __launch_bounds__(kInSmallThreads, 1)
+k_small_serve(const hbf_access_t *__restrict__ acc, const uint32_t n, const RangeSnap *__restrict__ ranges_g,
+              const ModelParams *__restrict__ mp_g, const __grid_constant__ FastRange fast_arg, BatchCtrl *ctrl,
+              uint8_t *__restrict__ status, int64_t *__restrict__ completion,
+              int64_t *__restrict__ stall, hbf_die_stats_t *stats_stage, const int64_t *__restrict__ busy, int64_t *busy_stage,
+              InTile *in_tile, const unsigned long long *claim_limit_p, uint32_t *die_claims, int forced) {
+    extern __shared__ __align__(16) unsigned char sm_small[];
+    __shared__ RangeSnap rs;
+    __shared__ ModelParams mp;
+    __shared__ FastRange fast_range;
+    __shared__ unsigned long long s_cnt[4];                  // of the whole batch: native, ready, failing; ready in this block's slice
+    __shared__ uint32_t s_unsorted;
+    __shared__ long long s_tot[3];                           // of the slice: stalls, services, largest completion
+    __shared__ uint32_t s_hist[kInSmallWarps][kInSmallSlice + 1];
+    __shared__ uint32_t s_dbase[kInSmallSlice + 1];
+    __shared__ int64_t w_S[kInSmallWarps], w_M[kInSmallWarps];
+    __shared__ int w_f[kInSmallWarps];
+    // (a flag another block of this launch may just have set takes the same decision this block is about to take)
+    if (ctrl->skip || ctrl->run_sort) return;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t slice = blockIdx.x, n_slices = gridDim.x, q_lo = slice * kInSmallSlice;
+    int64_t *s_s = reinterpret_cast<int64_t *>(sm_small);                     // [kInSmallMax] service time, by batch index
+    uint32_t *s_px = reinterpret_cast<uint32_t *>(s_s + kInSmallMax);        //               transfer | op << 31
+    uint32_t *s_key = s_px + kInSmallMax, *s_key2 = s_key + kInSmallMax;      //               the keys and the sort's second buffer
+    for (int i = tid; i < (int)(sizeof(RangeSnap) / 4); i += kInSmallThreads)
+        reinterpret_cast<uint32_t *>(&rs)[i] = reinterpret_cast<const uint32_t *>(ranges_g)[i];
+    for (int i = tid; i < (int)(sizeof(ModelParams) / 4); i += kInSmallThreads)
+        reinterpret_cast<uint32_t *>(&mp)[i] = reinterpret_cast<const uint32_t *>(mp_g)[i];
+    if (tid < 4) s_cnt[tid] = 0;
+    if (tid < 3) s_tot[tid] = tid == 2 ? INT64_MIN : 0;
+    if (tid == 0) { s_unsorted = 0u; fast_range = fast_arg; }
+    const uint32_t padded = (n + kInSmallThreads - 1u) / kInSmallThreads * kInSmallThreads;     // whole rounds for every warp
+    __syncthreads();
+
+    // ---- terms
+    const int64_t q_ppm = ctrl->q_ppm;
+    const Div64 div_q = ctrl->div_q;
+    const bool fast_terms = fast_arg.on != 0u && mp.pow2_geom != 0u && mp.xfer_tab_max_cb != 0u && q_ppm == 1000000;
+    const uint64_t claim_limit = DEBT ? *claim_limit_p : 0ull;
+    const int64_t quantum_ns = !DEBT ? 0 : q_ppm == 1000000 ? mp.t_read_ns + mp.t_prog_ns
+        : (int64_t)div64((uint64_t)(mp.t_read_ns + mp.t_prog_ns) * 1000000ull + (uint64_t)q_ppm - 1ull, div_q);
+    uint32_t c_native = 0, c_ready = 0, c_fault = 0, c_unsorted = 0, c_mine = 0;
+    long long sum_s = 0;
+    for (uint32_t i0 = (uint32_t)tid; i0 < padded; i0 += 4u * kInSmallThreads) {
+        uint64_t r_addr[4], r_bf[4]; int64_t r_issue[4], r_prev[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {                        // four records' loads go out together
+            const uint32_t i = i0 + (uint32_t)k * kInSmallThreads;
+            if (i < n) {
+                const uint64_t *rec = reinterpret_cast<const uint64_t *>(acc + i);
+                r_addr[k] = __ldg(rec); r_issue[k] = (int64_t)__ldg(rec + 1); r_bf[k] = __ldg(rec + 2);
+                r_prev[k] = i > 0u ? (int64_t)__ldg(rec - 2) : INT64_MIN;
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const uint32_t i = i0 + (uint32_t)k * kInSmallThreads;
+            if (i >= padded) break;
+            uint32_t key = 0xffffffffu;                      // not modeled, another block's, or padding: behind every queue
+            if (i < n) {
+                const bool writer = (i / kInSmallThreads) % n_slices == slice;       // the block that writes what is not queue work
+                if (r_issue[k] < r_prev[k]) c_unsorted = 1u;
+                const Served v = fast_terms ? serve_terms_fast(fast_range, mp, r_addr[k], r_issue[k], r_bf[k])
+                                            : serve_terms_general(rs, mp, r_addr[k], r_issue[k], r_bf[k], q_ppm, div_q);
+                if (status && writer) status[i] = (uint8_t)v.st;
+                if (v.st == HBF_ST_READY) {
+                    ++c_ready;
+                    if (v.queue - q_lo < kInSmallSlice) {    // (unsigned: queues below the slice wrap around)
+                        ++c_mine;
+                        int64_t sv = v.s;
+                        if (DEBT && (uint64_t)i < claim_limit) sv += quantum_ns;
+                        s_s[i] = sv; s_px[i] = v.xfer | (v.op << 31);
+                        key = ((v.queue - q_lo) << kInSmallQShift) | (i << 1) | v.op;
+                        sum_s += sv;
+                    }
+                } else if (v.st == HBF_ST_NATIVE) {
+                    ++c_native;
+                    if (writer) { completion[i] = r_issue[k]; stall[i] = 0; }
+                } else {
+                    ++c_fault;
+                }
+            }
+            s_key[i] = key;
+        }
+    }
+    c_native = (uint32_t)warp_sum((long long)c_native); c_ready = (uint32_t)warp_sum((long long)c_ready);
+    c_fault = (uint32_t)warp_sum((long long)c_fault); c_mine = (uint32_t)warp_sum((long long)c_mine); sum_s = warp_sum(sum_s);
+    c_unsorted = __any_sync(0xffffffffu, c_unsorted);
+    if (lane == 0) {
+        if (c_native) atomicAdd(&s_cnt[0], (unsigned long long)c_native);
+        if (c_ready) atomicAdd(&s_cnt[1], (unsigned long long)c_ready);
+        if (c_fault) atomicAdd(&s_cnt[2], (unsigned long long)c_fault);
+        if (c_mine) atomicAdd(&s_cnt[3], (unsigned long long)c_mine);
+        if (c_unsorted) atomicOr(&s_unsorted, 1u);
+        if (sum_s) atomicAdd((unsigned long long *)&s_tot[1], (unsigned long long)sum_s);
+    }
+    __syncthreads();
+    // what happens to the batch: the same decisions, in the same order, as the tiled path takes after its serve pass;
+    // every block has seen every record and decides alike, the first one records it
+    const bool fault = s_cnt[2] != 0ull, unsorted = s_unsorted != 0u;
+    if (tid == 0 && slice == 0u) {
+        ctrl->n_native = s_cnt[0]; ctrl->n_ready = s_cnt[1]; ctrl->n_fault = s_cnt[2];
+        if (unsorted) ctrl->unsorted = 1u;
+        if (fault) { ctrl->code = HBF_E_ACCESS_FAULT; ctrl->skip = 1; }                 // fail closed: refuse the batch
+        else if (unsorted && forced) { ctrl->code = HBF_E_INVAL; ctrl->skip = 1; }
+        else if (unsorted) ctrl->run_sort = 1u;                                         // hand the batch to the sort path
+        else ctrl->inorder_used = 1u;
+    }
+    if (fault || unsorted) return;                           // nothing of the batch's state has been written yet
+
+    // ---- sort the slice's keys by queue, stable (so a queue's records stay in batch order)
+    small_radix_pass(s_key, s_key2, padded, s_hist, s_dbase);
+    const uint32_t *sorted = s_key2;
+
+    // ---- serve: a segmented max-plus scan over the sorted entries.  An entry is the map B -> max(B + s, a + s); the head
+    // of a run starts from the busy-until earlier batches left on its queue, so its map no longer depends on what
+    // comes in (f).
+    const uint32_t m = (uint32_t)s_cnt[3];
+    long long sum_stall = 0, max_c = INT64_MIN;
+    {
+        struct SMap { int64_t S, M; int f; };
+        auto then = [](const SMap &x, const SMap &y) {         // x first, then y
+            if (y.f) return y;
+            SMap r; r.S = x.S + y.S; r.M = max((int64_t)(x.M + y.S), y.M); r.f = x.f; return r;
+        };
+        const uint32_t per = (m + kInSmallThreads - 1u) / kInSmallThreads;   // entries per thread (at most kInSmallItems)
+        const uint32_t p0 = (uint32_t)tid * per;
+        uint32_t key[kInSmallItems]; int64_t a[kInSmallItems], sv[kInSmallItems]; uint32_t px[kInSmallItems];
+        int64_t issue[kInSmallItems]; uint32_t bytes[kInSmallItems];
+        const uint32_t prev_q = p0 > 0u && p0 <= m ? sorted[p0 - 1u] >> kInSmallQShift : 0xffffffffu;
+#pragma unroll
+        for (uint32_t j = 0; j < kInSmallItems; ++j) {       // the issue times and sizes come from the records again, side by side
+            const uint32_t p = p0 + j;
+            key[j] = j < per && p < m ? sorted[p] : 0xffffffffu;
+            if (key[j] != 0xffffffffu) {
+                const uint64_t *rec = reinterpret_cast<const uint64_t *>(acc + ((key[j] >> 1) & (kInSmallMax - 1u)));
+                issue[j] = (int64_t)__ldg(rec + 1); bytes[j] = (uint32_t)__ldg(rec + 2);
+            }
+        }
+        // per-die totals along the thread's entries: a die's queues are neighbours in the sorted order
+        uint32_t run_die = 0xffffffffu, run_n = 0, run_np = 0, run_cl = 0;
+        unsigned long long run_busy = 0, run_br = 0, run_bp = 0;
+        auto flush = [&]() {
+            if (run_die == 0xffffffffu) return;
+            // (the staging copy was cleared by the begin kernel; a handful of adds per thread; the energy follows from the
+            // counts when the batch is committed)
+            unsigned long long *g = reinterpret_cast<unsigned long long *>(stats_stage + run_die);
+            atomicAdd(&g[0], run_busy);
+            if (run_br) atomicAdd(&g[1], run_br);
+            if (run_bp) atomicAdd(&g[2], run_bp);
+            if (run_n - run_np) atomicAdd(&g[4], (unsigned long long)(run_n - run_np));
+            if (run_np) atomicAdd(&g[5], (unsigned long long)run_np);
+            if (DEBT && run_cl) atomicAdd(&die_claims[run_die], run_cl);
+            run_busy = 0; run_br = 0; run_bp = 0; run_n = 0; run_np = 0; run_cl = 0;
+        };
+        SMap agg; agg.S = 0; agg.M = kNegInf; agg.f = 0;
+#pragma unroll
+        for (uint32_t j = 0; j < kInSmallItems; ++j) {
+            if (key[j] != 0xffffffffu) {
+                const uint32_t i = (key[j] >> 1) & (kInSmallMax - 1u), q = q_lo + (key[j] >> kInSmallQShift), op = key[j] & 1u;
+                sv[j] = s_s[i]; px[j] = s_px[i];
+                a[j] = issue[j] + (op ? (int64_t)(px[j] & 0x7fffffffu) : 0);
+                const uint32_t before = j == 0u ? prev_q : key[j - 1u] >> kInSmallQShift;
+                SMap e; e.S = sv[j]; e.f = before != (key[j] >> kInSmallQShift);
+                e.M = (e.f ? max(a[j], busy[q]) : a[j]) + sv[j];
+                agg = then(agg, e);
+                const uint32_t die = mp.queue_level == 0u ? q / mp.planes : q;
+                if (die != run_die) { flush(); run_die = die; }
+                const uint32_t gs = op ? mp.prog_gran_shift : mp.read_gran_shift;
+                const unsigned long long cb = (((unsigned long long)bytes[j] + (1ull << gs) - 1ull) >> gs) << gs;
+                run_busy += (unsigned long long)sv[j]; ++run_n;
+                if (op) { run_bp += cb; ++run_np; } else run_br += cb;
+                if (DEBT && (uint64_t)i < claim_limit) ++run_cl;
+            }
+        }
+        flush();
+        // inclusive scan of the threads' maps across the warp, then across the warps
+        SMap inc = agg;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            SMap u; u.S = __shfl_up_sync(0xffffffffu, inc.S, o); u.M = __shfl_up_sync(0xffffffffu, inc.M, o); u.f = __shfl_up_sync(0xffffffffu, inc.f, o);
+            if (lane >= o) inc = then(u, inc);
+        }
+        if (lane == 31) { w_S[warp] = inc.S; w_M[warp] = inc.M; w_f[warp] = inc.f; }
+        __syncthreads();
+        SMap ex; ex.S = 0; ex.M = kNegInf; ex.f = 0;          // everything before this thread's entries
+        for (int w = 0; w < warp; ++w) { SMap u; u.S = w_S[w]; u.M = w_M[w]; u.f = w_f[w]; ex = then(ex, u); }
+        {
+            SMap u; u.S = __shfl_up_sync(0xffffffffu, inc.S, 1); u.M = __shfl_up_sync(0xffffffffu, inc.M, 1); u.f = __shfl_up_sync(0xffffffffu, inc.f, 1);
+            if (lane > 0) ex = then(ex, u);
+        }
+        // (the first entry of the slice is a head, so a map without a head never reaches an entry that needs its input)
+        int64_t B = ex.M;
+#pragma unroll
+        for (uint32_t j = 0; j < kInSmallItems; ++j) {
+            if (key[j] != 0xffffffffu) {
+                const uint32_t i = (key[j] >> 1) & (kInSmallMax - 1u), lq = key[j] >> kInSmallQShift, op = key[j] & 1u;
+                const uint32_t before = j == 0u ? prev_q : key[j - 1u] >> kInSmallQShift;
+                if (before != lq) B = busy[q_lo + lq];
+                B = max(a[j], B) + sv[j];
+                const int64_t c = B + (op ? 0 : (int64_t)(px[j] & 0x7fffffffu)), waited = c - issue[j];
+                completion[i] = c; stall[i] = waited;
+                sum_stall += waited; max_c = max(max_c, (long long)c);
+                const uint32_t p = p0 + j;
+                const uint32_t after = p + 1u < m ? (j + 1u < per ? key[j + 1u] : sorted[p + 1u]) >> kInSmallQShift : 0xffffffffu;
+                if (after != lq) busy_stage[q_lo + lq] = B;  // last access of its queue in this batch (the other queues keep the begin kernel's copy)
+            }
+        }
+    }
+    sum_stall = warp_sum(sum_stall); max_c = warp_max(max_c);
+    if (lane == 0) { if (sum_stall) atomicAdd((unsigned long long *)&s_tot[0], (unsigned long long)sum_stall); atomicMax(&s_tot[2], max_c); }
+    __syncthreads();
+    if (tid == 0) {                                          // the slice's totals: one "tile" of the stall sum; the rest straight into the batch's
+        InTile t; t.spec_sum = s_tot[0]; t.fix_delta = 0; t.true_sum = 0; t.reserve = 0u; t.stragglers = 0u; in_tile[slice] = t;
+        if (s_tot[1]) atomicAdd((unsigned long long *)&ctrl->service_ns, (unsigned long long)s_tot[1]);
+        if (s_tot[2] != INT64_MIN) atomicMax(&ctrl->max_completion_ns, s_tot[2]);
+    }
+}
+
+bool inorder_small_batch(uint64_t n) { return n <= kInSmallMax; }
+
 size_t inorder_head_bytes(uint64_t tiles, uint32_t n_queues) { return tiles * n_queues * (size_t)kInHead * sizeof(InHead); }
 
 cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st) {
     const uint64_t n = a.n;
+    if (inorder_small_batch(n)) {                            // one launch, a block per 64 queues
+        const bool debt = a.claim_limit != nullptr;
+        const size_t smem = inorder_small_smem();
+        cudaError_t e = ensure_dyn_smem((const void *)k_small_serve<false>, smem);
+        if (e == cudaSuccess) e = ensure_dyn_smem((const void *)k_small_serve<true>, smem);
+        if (e != cudaSuccess) return e;
+        (debt ? k_small_serve<true> : k_small_serve<false>)<<<inorder_small_blocks(a.mp.n_queues), kInSmallThreads, smem, st>>>(
+            a.acc, (uint32_t)n, a.ranges, a.mp_dev, a.fast, a.ctrl, a.status, a.completion, a.stall, a.stats_stage, a.busy, a.busy_stage,
+            reinterpret_cast<InTile *>(a.ws.in_tile), a.claim_limit, a.die_claims, a.path == HBF_PATH_INORDER ? 1 : 0);
+        g_kernel_launches += 1;
+        return cudaGetLastError();
+    }
     const InTileMap tmap = inorder_tile_map(n, a.sm_count);
     const unsigned n_tiles = tmap.n_tiles;
     const uint64_t tile_records = std::max(tmap.big, tmap.small);
@@ -1044,14 +1346,11 @@ cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st) {
     serve(false);
     k_inorder_scan<<<(R + kInScanQueues - 1) / kInScanQueues, dim3(kInScanQueues, kInScanChunks), 0, st>>>(
         a.ctrl, a.mp_dev, n_tiles, a.ws.in_agg, a.ws.in_bin, a.busy, a.busy_stage, a.stats_stage, a.path == HBF_PATH_INORDER ? 1 : 0);
-    if (n_tiles > 1) {                                       // (the first tile needs no fix-up and is never served again)
-        (debt ? k_inorder_fixstraggle<true> : k_inorder_fixstraggle<false>)<<<n_tiles, kInStrThreads, smem_str, st>>>(
-            a.acc, n, tmap, a.ranges, a.mp, a.fast, a.ctrl, a.ws.in_bin, heads, a.ws.in_headcnt, a.completion, a.stall, tiles,
-            a.claim_limit, a.ws.in_qid, qid_stride);
-        serve(true);
-        g_kernel_launches += 2;
-    }
-    g_kernel_launches += 2;
+    (debt ? k_inorder_fixstraggle<true> : k_inorder_fixstraggle<false>)<<<n_tiles, kInStrThreads, smem_str, st>>>(
+        a.acc, n, tmap, a.ranges, a.mp, a.fast, a.ctrl, a.ws.in_bin, heads, a.ws.in_headcnt, a.completion, a.stall, tiles,
+        a.claim_limit, a.ws.in_qid, qid_stride);
+    serve(true);
+    g_kernel_launches += 4;
     return cudaGetLastError();
 }
 

@@ -319,6 +319,64 @@ def test_inorder_long_busy_periods(hbf, rho):
     compare_batch(g, o, w.acc)
 
 
+# ---- batches of at most 8,192 records in issue order take a route of their own (one launch, a block per 64 queues) ----
+
+@pytest.mark.parametrize("n", [8191, 8192, 8193])
+def test_small_batch_route_and_its_upper_end(hbf, n):
+    """Both sides of the size at which the tiled kernels take over, each batch on the queues the one before left."""
+    w = wl.mixed_status(3 * n, seed=n)
+    acc = issue_sorted(w.acc)
+    for path in (hbf.PATH_AUTO, hbf.PATH_INORDER):
+        g, o = contexts(hbf, w.profile, w.ranges, path)
+        for k in range(3):
+            compare_batch(g, o, acc[k * n:(k + 1) * n])
+
+
+@pytest.mark.parametrize("geo", [dict(channels=3, dies=5, planes=2, page_bytes=4096, stripe_bytes=16384),
+                                 dict(channels=8, dies=4, planes=2, page_bytes=16384, stripe_bytes=16384, queue_level=1),
+                                 dict(channels=64, dies=8, planes=4, page_bytes=16384, stripe_bytes=65536),
+                                 dict(channels=1, dies=1, planes=1, page_bytes=16384, stripe_bytes=16384)])
+def test_small_batches_other_geometries_and_thermal_scaling(hbf, geo):
+    """30 queues (a slice that is not full), one queue per die, 2,048 queues (32 slices), a single queue; then the same
+    with the service scaled (Eq. 3), which takes the general form of the terms."""
+    w = wl.mixed_status(12_000, seed=11)
+    prof = dict(w.profile); prof.update(geo)
+    acc = issue_sorted(w.acc)
+    g, o = contexts(hbf, prof, w.ranges, hbf.PATH_AUTO)
+    compare_batch(g, o, acc[:5000])
+    g.force_mode(hbf.MODE_LIGHT, 612_345); o.force_mode(hbfo.MODE_LIGHT, 612_345)
+    compare_batch(g, o, acc[5000:])
+
+
+def test_small_batch_all_on_one_queue_and_equal_issue_times(hbf):
+    rng = np.random.default_rng(21)
+    n = 8192
+    acc = np.zeros(n, hbfo.ACCESS_DTYPE)
+    acc["addr"] = wl.RANGE_BASE + rng.integers(0, 4, n).astype(np.uint64) * np.uint64(4096)      # one page: one queue
+    acc["issue_ns"] = np.sort(rng.integers(0, 50, n))
+    acc["bytes"] = rng.choice([64, 4096, 9000], n)
+    acc["flags"] = rng.random(n) < 0.3
+    prof = wl.load_profile("nominal", **wl.GEOMETRY["tiny"])
+    g, o = contexts(hbf, prof, [(wl.RANGE_BASE, wl.GIB, 3, 0, 0, 0)], hbf.PATH_AUTO)
+    compare_batch(g, o, acc)
+    compare_batch(g, o, acc[:3000])                          # again, on the backlog
+
+
+def test_small_batch_out_of_order_faults_and_natives_only(hbf):
+    w = wl.mixed_status(6000, seed=31)
+    g, o = contexts(hbf, w.profile, w.ranges, hbf.PATH_AUTO)
+    compare_batch(g, o, w.acc, check_order=True)             # shuffled: handed to the sort path from the device
+    compare_batch(g, o, issue_sorted(w.acc))                 # and the small route again on what it left
+    wf = wl.mixed_status(6000, seed=31, faults=True)
+    assert compare_batch(g, o, issue_sorted(wf.acc)) == hbfo.E_ACCESS_FAULT
+    nat = issue_sorted(w.acc).copy()
+    nat["addr"] = 0x1000 + 64 * np.arange(nat.shape[0], dtype=np.uint64)        # nothing inside a range
+    compare_batch(g, o, nat)
+    g2, _ = contexts(hbf, w.profile, w.ranges, hbf.PATH_INORDER)
+    rc, comp, stall, _, ds = g2.submit_host(w.acc, check=False)                  # declared in order, but it is not
+    assert rc == hbf.E_INVAL and not comp.any() and not g2.get_busy_until().any()
+
+
 def test_pinned_host_pipeline_equals_one_batch(hbf):
     """hbf_submit_host: copy-in, service and read-back of consecutive chunks on three streams of the library: for records
     in issue order the result (outputs, per-die totals, summary, queue state) is that of one batch; pageable buffers
