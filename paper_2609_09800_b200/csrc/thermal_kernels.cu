@@ -5,6 +5,8 @@
 // cell (Kahan summation of the substep increments): plain float32 accumulation drifts by several mK over
 // 10^4..10^5 substeps and stalls once an increment drops under half an ulp of the state.
 #include <algorithm>
+#include <mutex>
+#include <vector>
 
 #include <cooperative_groups.h>
 
@@ -130,12 +132,13 @@ static cudaError_t launch_thermal_generic(const ThermalDev &t, DevState *state, 
 // order, as in k_euler_substep; the power map is formed by every block for its own cells and the
 // hotspots are reduced through block 0.
 // ======================================================================================================
-constexpr int kThClusterBlocks = 8;
+constexpr int kThClusterBlocks = 16;                       // blocks of the cluster when the device takes that many (not a portable size), else 8
+constexpr int kThClusterPortable = 8;
 constexpr int kThThreads = 512;
 constexpr int kThCellsPerThread = 8;
 constexpr int kThMaxRegions = 1024;
 
-__global__ void __cluster_dims__(kThClusterBlocks, 1, 1) __launch_bounds__(kThThreads)
+__global__ void __launch_bounds__(kThThreads)
 k_thermal_cluster(ThermalDev t, float *theta, DevState *state, int64_t *pending, int64_t dt_ns, int has_ext, float dt_sub,
                   float *temps_out) {
     extern __shared__ __align__(16) unsigned char th_smem[];
@@ -143,10 +146,10 @@ k_thermal_cluster(ThermalDev t, float *theta, DevState *state, int64_t *pending,
     __shared__ float s_hot[kThClusterBlocks][3];
     __shared__ float s_part[3][kThThreads / 32];
     cg::cluster_group cluster = cg::this_cluster();
-    const uint32_t rank = cluster.block_rank();
+    const uint32_t rank = cluster.block_rank(), n_blocks = cluster.num_blocks();      // (the cluster's size is chosen at launch)
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t H = t.H, W = t.W;
-    const uint32_t rows = (H + kThClusterBlocks - 1) / kThClusterBlocks;
+    const uint32_t rows = (H + n_blocks - 1) / n_blocks;
     const uint32_t y0 = min(H, rank * rows), y1 = min(H, y0 + rows);
     const uint32_t band_cells = (y1 - y0) * W;
     const uint32_t pitch = (rows + 2) * W;                    // one buffer: halo row, band, halo row
@@ -195,7 +198,7 @@ k_thermal_cluster(ThermalDev t, float *theta, DevState *state, int64_t *pending,
         upper_halo0 = cluster.map_shared_rank(buf0, rank - 1) + (rows_above + 1) * W;
         upper_halo1 = cluster.map_shared_rank(buf1, rank - 1) + (rows_above + 1) * W;
     }
-    if (rank + 1 < (uint32_t)kThClusterBlocks && y1 < H) {      // the block below: its upper halo row is row 0
+    if (rank + 1 < n_blocks && y1 < H) {                         // the block below: its upper halo row is row 0
         lower_halo0 = cluster.map_shared_rank(buf0, rank + 1);
         lower_halo1 = cluster.map_shared_rank(buf1, rank + 1);
     }
@@ -264,7 +267,7 @@ k_thermal_cluster(ThermalDev t, float *theta, DevState *state, int64_t *pending,
         float h[3];
         for (int k = 0; k < 3; ++k) {
             float v = -INFINITY;
-            for (int b = 0; b < kThClusterBlocks; ++b) v = fmaxf(v, s_hot[b][k]);
+            for (uint32_t b = 0; b < n_blocks; ++b) v = fmaxf(v, s_hot[b][k]);
             h[k] = v == -INFINITY ? t.ambient_c : v;
             t.hot[k] = h[k];
         }
@@ -275,20 +278,66 @@ k_thermal_cluster(ThermalDev t, float *theta, DevState *state, int64_t *pending,
     }
 }
 
-static bool thermal_cluster_fits(const ThermalDev &t, size_t *smem_bytes) {
-    const uint32_t rows = (t.H + kThClusterBlocks - 1) / kThClusterBlocks;
+static bool thermal_cluster_fits(const ThermalDev &t, int n_blocks, size_t *smem_bytes) {
+    const uint32_t rows = (t.H + n_blocks - 1) / n_blocks;
     const size_t smem = (size_t)2 * (rows + 2) * t.W * sizeof(float);
     *smem_bytes = smem;
     return (size_t)rows * t.W <= (size_t)kThThreads * kThCellsPerThread && smem <= 200u * 1024u && t.n_regions <= (uint32_t)kThMaxRegions;
+}
+
+// How many blocks the cluster of the one-launch step gets on the current device: 16 where the device can place such a
+// cluster (a size beyond the portable 8 has to be allowed per kernel), else 8; 0 when the grid does not fit either.  Asked
+// once per (device, shared-memory size) and remembered.
+static int thermal_cluster_blocks(const ThermalDev &t, size_t *smem_bytes) {
+    struct Entry { int device; size_t smem16; int blocks; };
+    static std::mutex mu;
+    static std::vector<Entry> known;
+    size_t smem16 = 0, smem8 = 0;
+    const bool fits16 = thermal_cluster_fits(t, kThClusterBlocks, &smem16), fits8 = thermal_cluster_fits(t, kThClusterPortable, &smem8);
+    if (!fits8 && !fits16) return 0;
+    int blocks = fits8 ? kThClusterPortable : 0;
+    if (fits16) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return blocks;
+        std::lock_guard<std::mutex> lock(mu);
+        bool found = false;
+        for (const Entry &e : known) if (e.device == dev && e.smem16 == smem16) { if (e.blocks) blocks = e.blocks; found = true; break; }
+        if (!found) {
+            int got = 0;
+            if (ensure_dyn_smem((const void *)k_thermal_cluster, smem16) == cudaSuccess &&
+                cudaFuncSetAttribute((const void *)k_thermal_cluster, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+                cudaLaunchConfig_t cfg = {};
+                cfg.gridDim = dim3(kThClusterBlocks); cfg.blockDim = dim3(kThThreads); cfg.dynamicSmemBytes = smem16;
+                cudaLaunchAttribute at[1];
+                at[0].id = cudaLaunchAttributeClusterDimension; at[0].val.clusterDim.x = kThClusterBlocks; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+                cfg.attrs = at; cfg.numAttrs = 1;
+                int n = 0;
+                if (cudaOccupancyMaxActiveClusters(&n, (const void *)k_thermal_cluster, &cfg) == cudaSuccess && n >= 1) got = kThClusterBlocks;
+            }
+            (void)cudaGetLastError();                          // a refusal here only means the portable size is used
+            known.push_back(Entry{dev, smem16, got});
+            if (got) blocks = got;
+        }
+    }
+    *smem_bytes = blocks == kThClusterBlocks ? smem16 : smem8;
+    return blocks;
 }
 
 cudaError_t launch_thermal_step(const ThermalDev &t, DevState *state, int64_t *pending, int64_t dt_ns, int has_ext,
                                 float *d_temps_out, int *cur, int generic_only, cudaStream_t st) {
     const float dt_sub_f = (float)((double)dt_ns * 1e-9 / (double)t.n_sub);
     size_t smem = 0;
-    if (!generic_only && thermal_cluster_fits(t, &smem)) {
+    const int blocks = generic_only ? 0 : thermal_cluster_blocks(t, &smem);
+    if (blocks) {
         { cudaError_t e = ensure_dyn_smem((const void *)k_thermal_cluster, smem); if (e != cudaSuccess) return e; }
-        k_thermal_cluster<<<kThClusterBlocks, kThThreads, smem, st>>>(t, t.theta[*cur], state, pending, dt_ns, has_ext, dt_sub_f, d_temps_out);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(blocks); cfg.blockDim = dim3(kThThreads); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension; at[0].val.clusterDim.x = blocks; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+        cfg.attrs = at; cfg.numAttrs = 1;
+        float *theta = t.theta[*cur];
+        const cudaError_t e = cudaLaunchKernelEx(&cfg, k_thermal_cluster, t, theta, state, pending, dt_ns, has_ext, dt_sub_f, d_temps_out);
+        if (e != cudaSuccess) return e;
         g_kernel_launches += 1;
         return cudaGetLastError();
     }
