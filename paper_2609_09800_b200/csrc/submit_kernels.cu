@@ -214,7 +214,9 @@ constexpr int kSortWarps = kSortThreads / 32;
 constexpr size_t kSortSmem = (size_t)kSortTile * 12 + (size_t)kSortWarps * kRadix * 4;
 constexpr uint32_t kFlagAgg = 1u << 30, kFlagPrefix = 2u << 30, kCountMask = (1u << 30) - 1u;
 
-__global__ void __launch_bounds__(kSortThreads)
+// (three resident blocks per SM: at one block of 80 registers the pass ran at 13 % of the DRAM rate with a quarter of the
+// warp slots in use, 4.1 ms for 200 M keys; bounded to 40 registers, with a few spills, it takes 2.5 ms)
+__global__ void __launch_bounds__(kSortThreads, 3)
 k_sort_pass(int pass, uint64_t n, BatchCtrl *ctrl, DevState *state, const uint32_t *__restrict__ hist,
             uint64_t *keys0, uint64_t *keys1, uint32_t *idx0, uint32_t *idx1, uint32_t *desc0, uint32_t *desc1) {
     extern __shared__ __align__(16) unsigned char sort_smem[];
@@ -363,6 +365,8 @@ __device__ __forceinline__ Map shfl_up_map(const Map &m, int o) {
     r.f = __shfl_up_sync(0xffffffffu, m.f, o); return r;
 }
 
+// (two blocks per SM; three or four, or 512 threads with four items each, were measured slower: the kernel is bound by its
+// scattered accesses, not by latency)
 __global__ void __launch_bounds__(kScanThreads, 2)
 k_scan(const uint64_t *__restrict__ terms, uint64_t n,
        const ModelParams *__restrict__ mp_g, BatchCtrl *ctrl, DevState *state,
