@@ -168,7 +168,8 @@ __global__ void k_plan(BatchCtrl *ctrl, int force_full) {
 }
 
 // =====================================================================================================
-// histogram of every planned digit (shared-memory bins, warp-aggregated with match_any)
+// histogram of the first pass's digit (shared-memory bins).  The later passes' histograms are counted by the pass before
+// each, which has the keys in registers anyway: six shared-memory adds per key in one kernel took 1.8 ms at 200 M.
 // =====================================================================================================
 constexpr int kHistThreads = 512;
 
@@ -185,7 +186,7 @@ k_hist(const uint64_t *__restrict__ keys, uint64_t n, const BatchCtrl *ctrl, uin
     for (uint64_t i = (uint64_t)blockIdx.x * kHistThreads + threadIdx.x; i < n_round; i += stride) {
         const bool valid = i < n;
         const uint64_t ck = valid ? compact_key(keys[i], p.lo_bits, p.hi_bits) : 0ull;
-        for (uint32_t k = 0; k < p.n_passes; ++k) {
+        for (uint32_t k = 0; k < 1u; ++k) {
             const uint32_t d = valid ? (uint32_t)(ck >> p.shift[k]) & ((1u << p.bits[k]) - 1u) : 0xffffffffu;
             // the high digits of neighbouring keys are mostly equal, the low ones mostly all different: one vote tells the
             // two cases apart, and neither needs the lane-by-lane match (measured: 8.0 ms of a 58 ms sort at 200 M with it)
@@ -198,7 +199,7 @@ k_hist(const uint64_t *__restrict__ keys, uint64_t n, const BatchCtrl *ctrl, uin
         }
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < (int)p.n_passes * kRadix; i += kHistThreads)
+    for (int i = threadIdx.x; i < kRadix; i += kHistThreads)
         if (sh[i]) atomicAdd(&hist[i], sh[i]);
 }
 
@@ -218,7 +219,7 @@ constexpr uint32_t kFlagAgg = 1u << 30, kFlagPrefix = 2u << 30, kCountMask = (1u
 // (three resident blocks per SM: at one block of 80 registers the pass ran at 13 % of the DRAM rate with a quarter of the
 // warp slots in use, 4.1 ms for 200 M keys; bounded to 40 registers, with a few spills, it takes 2.5 ms)
 __global__ void __launch_bounds__(kSortThreads, 3)
-k_sort_pass(int pass, uint64_t n, BatchCtrl *ctrl, DevState *state, const uint32_t *__restrict__ hist,
+k_sort_pass(int pass, uint64_t n, BatchCtrl *ctrl, DevState *state, uint32_t *hist,
             uint64_t *keys0, uint64_t *keys1, uint32_t *idx0, uint32_t *idx1, uint32_t *desc0, uint32_t *desc1) {
     extern __shared__ __align__(16) unsigned char sort_smem[];
     uint64_t *s_keys = reinterpret_cast<uint64_t *>(sort_smem);                       // [kSortTile]
@@ -228,9 +229,13 @@ k_sort_pass(int pass, uint64_t n, BatchCtrl *ctrl, DevState *state, const uint32
     __shared__ uint32_t s_delta[kRadix];
     __shared__ uint32_t s_warp_tot[kRadix / 32], s_hist_tot[kRadix / 32];
     __shared__ uint32_t s_tile;
+    __shared__ uint32_t s_next[kRadix];                     // this block's share of the next pass's histogram
     if (ctrl->skip || !ctrl->run_sort) return;
     const SortPlan &pl = ctrl->plan;
     if (pass >= (int)pl.n_passes) return;
+    const bool count_next = pass + 1 < (int)pl.n_passes;
+    const uint32_t next_shift = count_next ? pl.shift[pass + 1] : 0u, next_mask = count_next ? (1u << pl.bits[pass + 1]) - 1u : 0u;
+    if (threadIdx.x < kRadix) s_next[threadIdx.x] = 0u;
     const uint32_t lo_bits = pl.lo_bits, hi_bits = pl.hi_bits, shift = pl.shift[pass];
     const uint32_t dmask = (1u << pl.bits[pass]) - 1u;
     const uint64_t *kin = (pass & 1) ? keys1 : keys0;
@@ -266,6 +271,18 @@ k_sort_pass(int pass, uint64_t n, BatchCtrl *ctrl, DevState *state, const uint32
             dig[j] = (uint32_t)(compact_key(key[j], lo_bits, hi_bits) >> shift) & dmask;
         } else {
             key[j] = ~0ull; val[j] = 0u; dig[j] = kRadix - 1;       // padding ranks behind every real key
+        }
+    }
+    // the next pass's digit of every key, counted now (the high digits of neighbouring keys are mostly equal, the low ones
+    // mostly all different: one vote tells the two cases apart)
+    if (count_next) {
+#pragma unroll
+        for (int j = 0; j < kSortItems; ++j) {
+            const bool valid = wbase + j * 32 + lane < n;
+            const uint32_t d2 = valid ? (uint32_t)(compact_key(key[j], lo_bits, hi_bits) >> next_shift) & next_mask : 0xffffffffu;
+            const uint32_t d0 = __shfl_sync(0xffffffffu, d2, 0);
+            if (__all_sync(0xffffffffu, d2 == d0)) { if (lane == 0 && valid) atomicAdd(&s_next[d2], 32u); }
+            else if (valid) atomicAdd(&s_next[d2], 1u);
         }
     }
     // rank inside the warp, in memory order
@@ -341,6 +358,8 @@ k_sort_pass(int pass, uint64_t n, BatchCtrl *ctrl, DevState *state, const uint32
         kout[g] = k; iout[g] = s_idx[i];
     }
   }
+    // (the loop was left behind a block-wide barrier)
+    if (count_next && tid < kRadix && s_next[tid]) atomicAdd(&hist[(pass + 1) * kRadix + tid], s_next[tid]);
 }
 
 // =====================================================================================================
