@@ -260,18 +260,14 @@ k_sort_pass(int pass, uint64_t n, BatchCtrl *ctrl, DevState *state, uint32_t *hi
     if (tid < kRadix) desc_next[(uint64_t)tile * kRadix + tid] = 0u;     // ready for the pass after this one
 
     // load, warp-striped: the warp's chunk is contiguous and item j of lane l sits at j*32 + l
-    uint64_t key[kSortItems]; uint32_t val[kSortItems]; uint32_t dig[kSortItems]; uint32_t rank[kSortItems];
+    uint64_t key[kSortItems]; uint32_t rank[kSortItems];
+    // (a key's digit is computed where it is needed: eight registers fewer than keeping it)
+    auto digit_of = [&](uint64_t k) { return k == ~0ull ? (uint32_t)(kRadix - 1) : (uint32_t)(compact_key(k, lo_bits, hi_bits) >> shift) & dmask; };
     const uint64_t wbase = base + (uint64_t)warp * (32 * kSortItems);
 #pragma unroll
     for (int j = 0; j < kSortItems; ++j) {
         const uint64_t i = wbase + j * 32 + lane;
-        if (i < n) {
-            key[j] = kin[i];
-            val[j] = pass == 0 ? (uint32_t)i : iin[i];
-            dig[j] = (uint32_t)(compact_key(key[j], lo_bits, hi_bits) >> shift) & dmask;
-        } else {
-            key[j] = ~0ull; val[j] = 0u; dig[j] = kRadix - 1;       // padding ranks behind every real key
-        }
+        key[j] = i < n ? kin[i] : ~0ull;                            // padding (no real key is all ones) ranks behind every real key
     }
     // the next pass's digit of every key, counted now (the high digits of neighbouring keys are mostly equal, the low ones
     // mostly all different: one vote tells the two cases apart)
@@ -289,11 +285,12 @@ k_sort_pass(int pass, uint64_t n, BatchCtrl *ctrl, DevState *state, uint32_t *hi
     uint32_t *wcnt = s_cnt + warp * kRadix;
 #pragma unroll
     for (int j = 0; j < kSortItems; ++j) {
-        const unsigned peers = __match_any_sync(0xffffffffu, dig[j]);
-        const uint32_t before = wcnt[dig[j]];
+        const uint32_t dg = digit_of(key[j]);
+        const unsigned peers = __match_any_sync(0xffffffffu, dg);
+        const uint32_t before = wcnt[dg];
         rank[j] = before + (uint32_t)__popc(peers & lanemask_lt());
         __syncwarp();
-        if ((peers >> lane) <= 1u) wcnt[dig[j]] = before + (uint32_t)__popc(peers);    // highest peer lane writes
+        if ((peers >> lane) <= 1u) wcnt[dg] = before + (uint32_t)__popc(peers);    // highest peer lane writes
         __syncwarp();
     }
     __syncthreads();
@@ -343,10 +340,18 @@ k_sort_pass(int pass, uint64_t n, BatchCtrl *ctrl, DevState *state, uint32_t *hi
     }
     __syncthreads();
 
-    // place keys at their position inside the tile, then write runs out
+    // place keys at their position inside the tile, then write runs out (the indices are fetched only now: eight registers
+    // fewer while the keys are ranked)
+    uint32_t val[kSortItems];
 #pragma unroll
     for (int j = 0; j < kSortItems; ++j) {
-        const uint32_t pos = s_local_start[dig[j]] + wcnt[dig[j]] + rank[j];
+        const uint64_t i = wbase + j * 32 + lane;
+        val[j] = pass == 0 ? (uint32_t)i : (i < n ? iin[i] : 0u);
+    }
+#pragma unroll
+    for (int j = 0; j < kSortItems; ++j) {
+        const uint32_t dg = digit_of(key[j]);
+        const uint32_t pos = s_local_start[dg] + wcnt[dg] + rank[j];
         s_keys[pos] = key[j]; s_idx[pos] = val[j];
     }
     __syncthreads();
