@@ -987,7 +987,9 @@ size_t workspace_layout(uint64_t n, uint32_t n_queues, Workspace *ws, void *base
     const uint64_t in_tiles = inorder_tiles_bound(nn);
     const bool inorder = n_queues <= kInMaxQueues;
     void *ia = take(inorder ? in_tiles * n_queues * 16 : 0), *ib = take(inorder ? in_tiles * n_queues * 8 : 0);
-    void *it = take(inorder ? in_tiles * 32 : 0), *ih = take(inorder ? inorder_head_bytes(in_tiles, n_queues) : 0);
+    // (the tile table also takes one entry per block of the small-batch route, which a batch of few records has more of than tiles)
+    void *it = take(inorder ? std::max<uint64_t>(in_tiles, inorder_small_blocks(n_queues)) * sizeof(InTile) : 0);
+    void *ih = take(inorder ? inorder_head_bytes(in_tiles, n_queues) : 0);
     void *ic = take(inorder ? in_tiles * n_queues : 0);
     void *iq = take(inorder ? inorder_qid_entries(nn) * 2 : 0);
     void *bx = take(with_bus ? nn * 4 : 0);
