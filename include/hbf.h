@@ -222,14 +222,17 @@ HBF_API int hbf_reset(hbf_ctx *ctx);                                            
 /* Chooses how batches are ordered: HBF_PATH_AUTO (default) serves a batch whose records arrive in
  * non-decreasing issue order without a global sort and falls back to the radix sort otherwise (also for a batch in
  * which a single access's service time reaches 2^33 ns, 2^32 ns with retention on: the in-order kernels keep
- * per-tile sums of service times in 56 bits);
+ * per-tile sums of service times in 56 bits; batches of at most 8,192 records take a route of their own that has no such
+ * limit);
  * HBF_PATH_SORT always sorts (a batch already in issue order is sorted on its queue bits only, which a
  * stable sort allows); HBF_PATH_SORT_FULL sorts on every key bit regardless; HBF_PATH_INORDER is the caller's
  * declaration that its batches are in issue order: only the in-order kernels are launched, and a batch that is not in
- * issue order, or has such a long service time, is refused with HBF_E_INVAL.  All give identical results. */
+ * issue order, or has such a long service time (and more than 8,192 records), is refused with HBF_E_INVAL.  All give
+ * identical results. */
 HBF_API int hbf_set_path(hbf_ctx *ctx, int32_t path);
 /* Thermal step implementation: 0 (default) runs the whole step in one launch of a thread-block cluster when
- * the grid fits its shared memory (up to 32,768 cells), else one launch per substep; 1 always uses the latter.
+ * the grid fits its registers and shared memory (up to 32,768 cells with the portable cluster of 8 blocks, 65,536 where
+ * the device can place a cluster of 16), else one launch per substep; 1 always uses the latter.
  * Both perform the same arithmetic in the same order (Eq. 1). */
 HBF_API int hbf_set_thermal_path(hbf_ctx *ctx, int32_t generic_only);
 
