@@ -362,6 +362,18 @@ def test_small_batch_all_on_one_queue_and_equal_issue_times(hbf):
     compare_batch(g, o, acc[:3000])                          # again, on the backlog
 
 
+def test_small_batch_with_a_very_long_service(hbf):
+    """A 512 MiB program (12.3 s of array time, beyond the 2^33 ns the tiled kernels' per-tile sums allow) among 3,000 ordinary
+    reads: the small-batch route keeps services in 64 bits, so the batch is served even with the in-order path declared."""
+    w = wl.tiny_uniform(3000, seed=14)
+    acc = w.acc.copy()
+    acc["bytes"][1234] = 512 << 20; acc["flags"][1234] = 1; acc["addr"][1234] = wl.RANGE_BASE
+    for path in (hbf.PATH_AUTO, hbf.PATH_INORDER):
+        g, o = contexts(hbf, w.profile, w.ranges, path)
+        assert compare_batch(g, o, acc) == 0
+        compare_batch(g, o, w.acc)                           # and the next batch behind it
+
+
 def test_small_batch_out_of_order_faults_and_natives_only(hbf):
     w = wl.mixed_status(6000, seed=31)
     g, o = contexts(hbf, w.profile, w.ranges, hbf.PATH_AUTO)
