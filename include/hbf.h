@@ -230,6 +230,17 @@ HBF_API int hbf_reset(hbf_ctx *ctx);                                            
  * issue order, or has such a long service time (and more than 8,192 records), is refused with HBF_E_INVAL.  All give
  * identical results. */
 HBF_API int hbf_set_path(hbf_ctx *ctx, int32_t path);
+/* Tile sizes of the in-order path from measurements, on by default: when a batch fills one wave of the device (two tiles
+ * per SM), every block of the streaming pass leaves how long its tile took, and later batches size their tiles in
+ * proportion to the rates measured at each place (the SMs of a device are not equally fast, and the pass lasts as long as
+ * its slowest block).  The record is read through an asynchronous copy that nothing waits for.  Results never depend on
+ * where tiles begin; 0 switches the measurements off (tiles in two fixed sizes), which makes run times reproducible from
+ * the first batch on.  Waits for nothing. */
+HBF_API int hbf_set_tile_balance(hbf_ctx *ctx, int32_t on);
+/* The record those sizes come from, as the last batch that filled a wave left it: for each of its tiles (a tile = a place:
+ * SM and kind of block) the records it had and the nanoseconds its block took (0: taken out of turn, not measured).
+ * Waits for the stream.  *count = number of tiles (0: no such batch yet); with records_out and ns_out (host, [cap]) the values. */
+HBF_API int hbf_get_tile_times(hbf_ctx *ctx, uint32_t *records_out, uint32_t *ns_out, uint32_t cap, uint32_t *count);
 /* Thermal step implementation: 0 (default) runs the whole step in one launch of a thread-block cluster when
  * the grid fits its registers and shared memory (up to 32,768 cells with the portable cluster of 8 blocks, 65,536 where
  * the device can place a cluster of 16), else one launch per substep; 1 always uses the latter.

@@ -42,6 +42,7 @@ struct hbf_ctx {
     BatchCtrl *d_ctrl = nullptr; hbf_batch_result_t *d_result = nullptr;
     int64_t *d_busy = nullptr, *d_busy_stage = nullptr, *d_pending = nullptr; hbf_die_stats_t *d_stats_stage = nullptr;
     hbf_batch_result_t *h_result = nullptr;      // pinned
+    TileBalanceHost bal;                         // tile sizes of the in-order path from the times earlier batches left
     // thermal steps on a reduced-order model instead of the grid (off while rom == nullptr)
     hbf_rom *rom = nullptr; int64_t rom_dt_ns = 0; int32_t *d_rom_kind = nullptr; double *d_rom_p = nullptr, *d_rom_T = nullptr;
     // channel bus as a second queued stage (off while d_bus_busy == nullptr)
@@ -235,6 +236,7 @@ int hbf_destroy(hbf_ctx *c) {
     for (void *p : c->owned) cudaFree(p);
     if (c->ev_made) { for (auto &e : c->ev) cudaEventDestroy(e); for (auto &e : c->ev_th) cudaEventDestroy(e); }
     if (c->h_result) cudaFreeHost(c->h_result);
+    if (c->bal.pinned) cudaFreeHost(c->bal.pinned);
     if (c->d_ledger) cudaFree(c->d_ledger);
     if (c->d_bus_busy) cudaFree(c->d_bus_busy);
     if (c->d_bus_ctrl) cudaFree(c->d_bus_ctrl);
@@ -326,6 +328,9 @@ int hbf_create(const hbf_config_t *cfg, void *cuda_stream, hbf_ctx **out) {
     if (cudaMallocHost(&c->h_result, sizeof(hbf_batch_result_t)) != cudaSuccess) return fail(HBF_E_NOMEM);
     memset(c->h_result, 0, sizeof(hbf_batch_result_t));
     if (cudaMallocHost(&c->h_hot, 3 * sizeof(float)) != cudaSuccess) return fail(HBF_E_NOMEM);
+    if ((rc = dev_copy(c, &c->bal.dev, nullptr, 1))) return fail(rc);
+    if (cudaMallocHost(&c->bal.pinned, sizeof(TileBalance)) != cudaSuccess) return fail(HBF_E_NOMEM);
+    memset(c->bal.pinned, 0, sizeof(TileBalance));
 
     c->thermal = cfg->cell_C != nullptr;
     if (c->thermal) {
@@ -434,6 +439,27 @@ int hbf_set_path(hbf_ctx *c, int32_t path) {
     return HBF_OK;
 }
 
+int hbf_get_tile_times(hbf_ctx *c, uint32_t *records_out, uint32_t *ns_out, uint32_t cap, uint32_t *count) {
+    if (!c || !count) return HBF_E_INVAL;
+    CK(cudaStreamSynchronize(c->stream));
+    const TileBalance &r = *c->bal.pinned;
+    uint32_t n = 0;
+    while (n < kInBalMax && r.claim[n] != 0u && r.claim[n] == r.claim[0]) ++n;
+    *count = n;
+    if (records_out && ns_out) {
+        if (cap < n) return HBF_E_INVAL;
+        for (uint32_t t = 0; t < n; ++t) { records_out[t] = r.len[t]; ns_out[t] = r.ns[t]; }
+    }
+    return HBF_OK;
+}
+
+int hbf_set_tile_balance(hbf_ctx *c, int32_t on) {
+    if (!c) return HBF_E_INVAL;
+    c->bal.on = on != 0;
+    if (c->bal.pinned) memset(c->bal.pinned, 0, sizeof(TileBalance));      // (measurements start over)
+    return HBF_OK;
+}
+
 // Everything a batch of records goes through once its arguments are in place: the claim window (retention), the submit
 // path, the energy ledger, read disturb / commits, the channel-bus stage.  Shared by hbf_submit_batch (the caller's
 // accesses) and hbf_submit_batch_paged (the list of parts).
@@ -446,6 +472,7 @@ static int serve_records(hbf_ctx *c, SubmitArgs &a) {
         a.fast.base = r.base; a.fast.length = r.length; a.fast.media_offset = r.media_offset; a.fast.perms = r.perms; a.fast.on = 1u;
     }
     a.binned = c->bin_ns != 0; a.bus_on = c->d_bus_busy ? 1 : 0;
+    a.bal = &c->bal;
     if (c->ret_on) {                                         // how far the outstanding refresh quanta reach into this batch
         CK(launch_ret_window(a.acc, a.n, c->d_ranges, c->ret, c->sm_count, c->stream));
         a.claim_limit = &c->ret.st->claim_limit; a.die_claims = c->ret.die_claims; a.ret = &c->ret;

@@ -105,6 +105,7 @@ struct Workspace {
 // a kernel argument, so that the common configuration reads nothing from memory to classify an access.
 struct FastRange { uint64_t base, length, media_offset; uint32_t perms, on; };
 
+struct TileBalanceHost;
 struct SubmitArgs {
     const hbf_access_t *acc; uint64_t n;
     int64_t *completion, *stall; uint8_t *status; hbf_die_stats_t *die_stats;
@@ -119,6 +120,7 @@ struct SubmitArgs {
     uint32_t *die_claims;                   // retention on: [dies] claims of the batch
     const struct RetDev *ret;               // retention on: the block state (host copy of the device pointers)
     cudaEvent_t *ev;                     // [kProfEvents] or null: recorded between kernel groups
+    TileBalanceHost *bal;                // tile sizes from measurements (null: off)
 };
 constexpr int kProfEvents = 10;
 extern std::atomic<unsigned long long> g_kernel_launches;
@@ -145,15 +147,31 @@ size_t workspace_layout(uint64_t n, uint32_t n_queues, Workspace *ws, void *base
 cudaError_t launch_bus_stage(const SubmitArgs &a, BatchCtrl *bc, int64_t *bus_busy, cudaStream_t st);
 // How the in-order path cuts a batch of n records into contiguous tiles: n_big tiles of `big` records, then tiles of
 // `small` records (the last one ragged).  All sizes are multiples of kInTileQuantum.  n_big == 0: one size only.
-struct InTileMap { uint64_t n; uint32_t n_tiles, n_big; uint32_t big, small; };
-__host__ __device__ inline uint64_t tile_first(const InTileMap &m, uint32_t t) {
+// With `first` set (device memory, n_tiles + 1 entries) the tiles begin where that table says instead: sizes that follow
+// from how long each tile's block took in an earlier batch (TileBalance below).  by_sm: a block takes the tile of its SM
+// and of its kind (tile = kind * n_big + SM), so that a tile's time tells how fast that place serves.
+struct InTileMap { uint64_t n; uint32_t n_tiles, n_big; uint32_t big, small; const uint32_t *first; uint32_t max_tile, by_sm; };
+__device__ inline uint64_t tile_first(const InTileMap &m, uint32_t t) {
+    if (m.first) return m.first[t];
     return t < m.n_big ? (uint64_t)t * m.big : (uint64_t)m.n_big * m.big + (uint64_t)(t - m.n_big) * m.small;
 }
-__host__ __device__ inline uint64_t tile_last(const InTileMap &m, uint32_t t) {      // one past the tile's last record
-    const uint64_t e = tile_first(m, t) + (t < m.n_big ? m.big : m.small);
+__device__ inline uint64_t tile_last(const InTileMap &m, uint32_t t) {      // one past the tile's last record
+    const uint64_t e = m.first ? (uint64_t)m.first[t + 1] : tile_first(m, t) + (t < m.n_big ? m.big : m.small);
     return e < m.n ? e : m.n;
 }
-InTileMap inorder_tile_map(uint64_t n, int sm_count);
+// Tile sizes from measurements.  The SMs of a device do not serve a tile equally fast (the same few are about 3 % slower
+// in every launch, and of the two blocks of an SM the one in the lower warp slots is faster), and the pass lasts as long
+// as its slowest block.  Every block of the streaming pass leaves how many records its tile had and how long it took;
+// the host reads that record of an earlier batch (an asynchronous copy: nothing waits for it) and sizes the next
+// batch's tiles in proportion to the measured rates.  Results do not depend on where tiles begin.
+constexpr uint32_t kInBalMax = 320;      // tiles this can describe (two per SM)
+struct TileBalance {
+    uint32_t claim[kInBalMax];           // number of the last batch in which the tile was taken (hand-out by SM and kind)
+    uint32_t len[kInBalMax], ns[kInBalMax];   // records of the tile, and how long its block took (0: taken out of turn, not measured)
+    uint32_t first[kInBalMax + 1];       // device only: where the tiles of the batch in flight begin
+};
+struct TileBalanceHost { TileBalance *dev = nullptr, *pinned = nullptr; uint32_t seq = 0; bool on = true; };
+InTileMap inorder_tile_map(uint64_t n, int sm_count, bool by_table);   // by_table: a full wave gets exactly two tiles per SM, placed by a table
 // per-tile bookkeeping of the stall total: as-if-idle sum, fix-up corrections, and the exact sum of a re-served tile
 struct InTile { long long spec_sum, fix_delta, true_sum; uint32_t reserve; uint32_t stragglers; };
 size_t inorder_head_bytes(uint64_t tiles, uint32_t n_queues);

@@ -26,6 +26,7 @@
 // warp through the hardware's named barriers.  Records of one queue that fall into the same row are chained
 // in registers with shuffles.
 #include <algorithm>
+#include <cstddef>
 #include <type_traits>
 
 #include "device_utils.cuh"
@@ -218,9 +219,11 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, const __grid_c
                 hbf_die_stats_t *stats_stage, int64_t *__restrict__ completion, int64_t *__restrict__ stall,
                 const int64_t *__restrict__ in_bin, InTile *in_tile, InHead *__restrict__ in_head, uint8_t *__restrict__ in_headcnt,
                 const int64_t *__restrict__ busy, const unsigned long long *claim_limit_p, uint32_t *die_claims,
-                const __grid_constant__ RetDev ret, uint16_t *__restrict__ in_qid, uint32_t qid_stride) {
+                const __grid_constant__ RetDev ret, uint16_t *__restrict__ in_qid, uint32_t qid_stride,
+                TileBalance *bal, uint32_t bal_seq) {
     extern __shared__ __align__(16) unsigned char in_smem[];
     __shared__ long long s_red[2];
+    __shared__ unsigned long long s_t0;                   // when this block took its tile (0: its time is not recorded)
     __shared__ uint32_t s_heads_full;                     // queues whose head entries are complete
     __shared__ ModelParams mp;                            // measured: reads from shared memory beat reads of the argument
     __shared__ FastRange fast_range;
@@ -256,16 +259,29 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, const __grid_c
     if (!RESERVE) {
         if (tid == 0) {
             uint32_t t = blockIdx.x;
+            unsigned long long t0 = 0ull;
             if (tmap.n_big != 0u) {
                 unsigned slot;
                 asm volatile("mov.u32 %0, %%warpid;" : "=r"(slot));
                 const uint32_t late = slot >= 4u ? 1u : 0u;   // warp 0 of the block that came second sits past the first four slots
-                const uint32_t have[2] = {tmap.n_big, tmap.n_tiles - tmap.n_big};
-                uint32_t k = atomicAdd(&ctrl->role_count[late], 1u);
-                if (k < have[late]) t = late ? tmap.n_big + k : k;
-                else { k = atomicAdd(&ctrl->role_count[1u - late], 1u); t = late ? k : tmap.n_big + k; }
+                if (bal) {
+                    // the tile of this SM and this kind; should it be gone (the slots did not say what they usually say),
+                    // any tile that is left: every tile is taken exactly once, marked with the batch's number
+                    unsigned sm;
+                    asm volatile("mov.u32 %0, %%smid;" : "=r"(sm));
+                    const uint32_t want = late * tmap.n_big + sm;
+                    bool mine = sm < tmap.n_big && atomicExch(&bal->claim[want], bal_seq) != bal_seq;
+                    t = want;
+                    for (uint32_t k = 0; !mine && k < tmap.n_tiles; ++k) { t = k; mine = atomicExch(&bal->claim[k], bal_seq) != bal_seq; }
+                    if (t == want) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+                } else {
+                    const uint32_t have[2] = {tmap.n_big, tmap.n_tiles - tmap.n_big};
+                    uint32_t k = atomicAdd(&ctrl->role_count[late], 1u);
+                    if (k < have[late]) t = late ? tmap.n_big + k : k;
+                    else { k = atomicAdd(&ctrl->role_count[1u - late], 1u); t = late ? k : tmap.n_big + k; }
+                }
             }
-            s_tile_id = t;
+            s_tile_id = t; s_t0 = t0;
         }
         __syncthreads();
     }
@@ -525,6 +541,12 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, const __grid_c
         if (RESERVE) in_tile[tile].true_sum = s_red[0];
         else { InTile t; t.spec_sum = s_red[0]; t.fix_delta = 0; t.true_sum = 0; t.reserve = 0u; t.stragglers = 0u; in_tile[tile] = t; }
         if (s_red[1] != INT64_MIN) atomicMax(&ctrl->max_completion_ns, s_red[1]);
+        if (!RESERVE && bal) {                               // how many records, how long: what the next batches' tile sizes follow from
+            unsigned long long now;
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+            bal->len[tile] = tile_len;
+            bal->ns[tile] = s_t0 ? (uint32_t)min(now - s_t0, 0xffffffffull) : 0u;
+        }
     }
 }
 
@@ -970,7 +992,7 @@ k_inorder_fixstraggle(const hbf_access_t *__restrict__ acc, uint64_t n, const __
 // One wave of resident blocks: as many tiles as the device holds serve blocks.  When the batch is large enough to fill
 // that wave, the tiles of the blocks that the hardware favours (one per SM) are larger by the skew, the others smaller,
 // so that both blocks of an SM finish together.
-InTileMap inorder_tile_map(uint64_t n, int sm_count) {
+InTileMap inorder_tile_map(uint64_t n, int sm_count, bool by_table) {
     InTileMap m{};
     m.n = n;
     const uint64_t sms = (uint64_t)std::max(1, sm_count);
@@ -979,17 +1001,61 @@ InTileMap inorder_tile_map(uint64_t n, int sm_count) {
     const uint64_t even = round_up((n + want_tiles - 1) / want_tiles);
     if (kInBlocksPerSM == 2 && want_tiles == 2 * sms && even >= 64 * kInTileQuantum && HBF_IN_SKEW_PERMILLE > 0) {
         const uint64_t big = round_up(even * (1000 + HBF_IN_SKEW_PERMILLE) / 1000);
+        if (by_table && 2 * sms <= kInBalMax) {
+            // exactly two tiles per SM, their places in a table (launch_inorder writes it: the two nominal sizes until
+            // measurements are at hand); big and small are the nominal sizes only
+            m.n_big = (uint32_t)sms; m.n_tiles = (uint32_t)(2 * sms); m.big = (uint32_t)big;
+            m.small = (uint32_t)round_up(even * (1000 - HBF_IN_SKEW_PERMILLE) / 1000);
+            m.max_tile = (uint32_t)round_up(even * 1200 / 1000); m.by_sm = 1u;
+            return m;
+        }
         if (big * sms < n) {
             const uint64_t rest = n - big * sms;
             const uint64_t small = round_up((rest + sms - 1) / sms);
             m.n_big = (uint32_t)sms; m.big = (uint32_t)big; m.small = (uint32_t)small;
             m.n_tiles = (uint32_t)(sms + (rest + small - 1) / small);
+            m.max_tile = (uint32_t)std::max(big, small);
             return m;
         }
     }
     m.n_big = 0; m.big = m.small = (uint32_t)even;
     m.n_tiles = (uint32_t)((n + even - 1) / even);
+    m.max_tile = (uint32_t)even;
     return m;
+}
+
+// Where n_tiles tiles begin when tile t gets the share share[t] of a batch of n records, in whole quanta (every tile at
+// least one); first[n_tiles] >= n.
+static void tiles_from_shares(const double *share, uint32_t n_tiles, uint64_t n, uint32_t *first, uint32_t *max_tile) {
+    double sum_share = 0.0;
+    for (uint32_t t = 0; t < n_tiles; ++t) sum_share += share[t];
+    const uint64_t quanta = (n + kInTileQuantum - 1) / kInTileQuantum;
+    uint64_t q[kInBalMax], used = 0;
+    for (uint32_t t = 0; t < n_tiles; ++t) { q[t] = std::max<uint64_t>(1, (uint64_t)(share[t] / sum_share * (double)quanta)); used += q[t]; }
+    for (uint32_t t = 0; used < quanta; t = (t + 1) % n_tiles) { ++q[t]; ++used; }           // what rounding down left over
+    for (uint32_t t = 0; used > quanta; t = (t + 1) % n_tiles) if (q[t] > 1) { --q[t]; --used; }
+    uint64_t at = 0, largest = 0;
+    for (uint32_t t = 0; t < n_tiles; ++t) { first[t] = (uint32_t)(at * kInTileQuantum); at += q[t]; largest = std::max(largest, q[t]); }
+    first[n_tiles] = (uint32_t)(at * kInTileQuantum);
+    *max_tile = (uint32_t)(largest * kInTileQuantum);
+}
+
+// Shares from the record an earlier batch left (see TileBalance): every tile in proportion to the rate measured at its
+// place, blended with the share it had (so that one odd measurement moves a tile by little), within 15 % of the mean.
+// False when the record is not a complete measurement of one batch with this many tiles.
+static bool measured_shares(const TileBalance &rec, uint32_t n_tiles, double *share) {
+    double rate[kInBalMax], sum_rate = 0.0, sum_len = 0.0;
+    for (uint32_t t = 0; t < n_tiles; ++t) {
+        if (rec.claim[t] != rec.claim[0] || rec.claim[t] == 0u || rec.ns[t] == 0u || rec.len[t] == 0u) return false;
+        rate[t] = (double)rec.len[t] / (double)rec.ns[t];
+        sum_rate += rate[t]; sum_len += (double)rec.len[t];
+    }
+    const double mean = 1.0 / n_tiles;
+    for (uint32_t t = 0; t < n_tiles; ++t) {
+        const double s = 0.3 * ((double)rec.len[t] / sum_len) + 0.7 * (rate[t] / sum_rate);
+        share[t] = std::min(std::max(s, 0.85 * mean), 1.15 * mean);
+    }
+    return true;
 }
 
 // dynamic shared memory of the serve kernel: the per-queue state and the per-die counters
@@ -1314,9 +1380,28 @@ cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st) {
         g_kernel_launches += 1;
         return cudaGetLastError();
     }
-    const InTileMap tmap = inorder_tile_map(n, a.sm_count);
+    const bool by_table = a.bal && a.bal->on && a.bal->dev;
+    InTileMap tmap = inorder_tile_map(n, a.sm_count, by_table);
     const unsigned n_tiles = tmap.n_tiles;
-    const uint64_t tile_records = std::max(tmap.big, tmap.small);
+    // one full wave of two tiles per SM: the blocks take their tiles by SM and kind and leave their times; the tiles' places
+    // come from a table in device memory: sized by the record of an earlier batch when there is a complete one, else in the
+    // two nominal sizes
+    TileBalanceHost *bal = tmap.by_sm ? a.bal : nullptr;
+    uint32_t bal_seq = 0;
+    if (bal) {
+        bal_seq = ++bal->seq;
+        if (bal_seq == 0u) bal_seq = ++bal->seq;             // (0 marks a tile never taken)
+        double share[kInBalMax];
+        if (!measured_shares(*bal->pinned, n_tiles, share))
+            for (uint32_t t = 0; t < n_tiles; ++t) share[t] = t < tmap.n_big ? (double)tmap.big : (double)tmap.small;
+        uint32_t first[kInBalMax + 1], max_tile = 0;
+        tiles_from_shares(share, n_tiles, n, first, &max_tile);
+        // (from pageable memory: the copy is staged before the call returns, so the array may go out of scope)
+        cudaError_t e = cudaMemcpyAsync(bal->dev->first, first, (n_tiles + 1) * sizeof(uint32_t), cudaMemcpyHostToDevice, st);
+        if (e != cudaSuccess) return e;
+        tmap.first = bal->dev->first; tmap.max_tile = max_tile;
+    }
+    const uint64_t tile_records = tmap.max_tile;
     if (n_tiles > inorder_tiles_bound(n)) return cudaErrorInvalidValue;       // the workspace is carved for that many
     const uint32_t R = a.mp.n_queues, nd = a.mp.n_dies;
     const size_t smem_serve = inorder_serve_smem(nd), smem_str = inorder_straggle_smem();
@@ -1341,9 +1426,14 @@ cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st) {
                          : (debt ? k_inorder_serve<false, true> : k_inorder_serve<false, false>);
         k<<<n_tiles, kInThreads, smem_serve, st>>>(a.acc, n, tmap, a.ranges, a.mp, a.fast, a.ctrl, a.status, a.ws.in_agg,
                                                    a.stats_stage, a.completion, a.stall, a.ws.in_bin, tiles, heads, a.ws.in_headcnt,
-                                                   a.busy, a.claim_limit, a.die_claims, debt ? *a.ret : RetDev{}, a.ws.in_qid, qid_stride);
+                                                   a.busy, a.claim_limit, a.die_claims, debt ? *a.ret : RetDev{}, a.ws.in_qid, qid_stride,
+                                                   bal ? bal->dev : nullptr, bal_seq);
     };
     serve(false);
+    if (bal) {                                               // the tiles' times, for later batches; nothing waits for this copy
+        cudaError_t e = cudaMemcpyAsync(bal->pinned, bal->dev, offsetof(TileBalance, first), cudaMemcpyDeviceToHost, st);
+        if (e != cudaSuccess) return e;
+    }
     k_inorder_scan<<<(R + kInScanQueues - 1) / kInScanQueues, dim3(kInScanQueues, kInScanChunks), 0, st>>>(
         a.ctrl, a.mp_dev, n_tiles, a.ws.in_agg, a.ws.in_bin, a.busy, a.busy_stage, a.stats_stage, a.path == HBF_PATH_INORDER ? 1 : 0);
     (debt ? k_inorder_fixstraggle<true> : k_inorder_fixstraggle<false>)<<<n_tiles, kInStrThreads, smem_str, st>>>(

@@ -1134,7 +1134,7 @@ static cudaError_t launch_after_inorder(const SubmitArgs &a, bool may_sort, cuda
     c.sort_grid = (unsigned)std::min<uint64_t>(sort_tiles, (uint64_t)a.sm_count * 3);
     c.scan_grid = (unsigned)std::min<uint64_t>(scan_tiles, (uint64_t)a.sm_count * 8);
     c.stall_grid = (unsigned)std::max<uint64_t>(1, std::min<uint64_t>((n + 255) / 256, (uint64_t)a.sm_count * 16));
-    const InTileMap tmap = inorder_tile_map(n, a.sm_count);
+    const InTileMap tmap = inorder_tile_map(n, a.sm_count, a.bal && a.bal->on && a.bal->dev);
     c.in_tile = reinterpret_cast<const InTile *>(a.ws.in_tile);
     c.n_tiles = inorder_small_batch(n) ? inorder_small_blocks(a.mp.n_queues) : tmap.n_tiles;
     if (may_sort) k_after_inorder<true><<<1, 256, 0, st>>>(c); else k_after_inorder<false><<<1, 256, 0, st>>>(c);

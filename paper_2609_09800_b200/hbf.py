@@ -27,7 +27,7 @@ DIE_STATS_DTYPE = np.dtype([(k, "<i8") for k in
 
 EXPORTS = ("hbf_create", "hbf_destroy", "hbf_register_range", "hbf_clear_ranges", "hbf_workspace_bytes",
            "hbf_submit_batch", "hbf_last_result", "hbf_thermal_step", "hbf_force_mode", "hbf_get_mode",
-           "hbf_reset", "hbf_set_path", "hbf_get_state", "hbf_set_state", "hbf_get_busy_until",
+           "hbf_reset", "hbf_set_path", "hbf_set_tile_balance", "hbf_get_tile_times", "hbf_get_state", "hbf_set_state", "hbf_get_busy_until",
            "hbf_get_pending_energy", "hbf_get_temps", "hbf_euler_limit_ns", "hbf_queue_order", "hbf_strerror",
            "hbf_set_profiling", "hbf_get_profile", "hbf_kernel_launches", "hbf_euler_substeps_static", "hbf_set_thermal_path",
            "hbf_workspace_bytes_paged", "hbf_submit_batch_paged", "hbf_submit_host", "hbf_debug_wait_test",
@@ -132,6 +132,8 @@ def lib():
         L.hbf_get_mode.argtypes = [vp, C.POINTER(i32), C.POINTER(i64)]
         L.hbf_reset.argtypes = [vp]
         L.hbf_set_path.argtypes = [vp, i32]
+        L.hbf_set_tile_balance.argtypes = [vp, i32]
+        L.hbf_get_tile_times.argtypes = [vp, vp, vp, C.c_uint32, vp]
         L.hbf_set_thermal_path.argtypes = [vp, i32]
         L.hbf_get_state.argtypes = [vp, vp, C.POINTER(C.c_size_t)]
         L.hbf_set_state.argtypes = [vp, vp, C.c_size_t]
@@ -400,6 +402,24 @@ class Context:
         rc = lib().hbf_set_path(self._h, path)
         if rc != 0:
             raise HbfError(rc, "hbf_set_path")
+
+    def tile_times(self):
+        """(records, ns) per tile of the last batch that filled a wave of the device; empty arrays when there was none."""
+        cnt = C.c_uint32()
+        rc = lib().hbf_get_tile_times(self._h, None, None, 0, C.byref(cnt))
+        if rc != 0:
+            raise HbfError(rc, "hbf_get_tile_times")
+        rec = np.zeros(cnt.value, np.uint32); ns = np.zeros(cnt.value, np.uint32)
+        if cnt.value:
+            rc = lib().hbf_get_tile_times(self._h, rec.ctypes.data, ns.ctypes.data, cnt.value, C.byref(cnt))
+            if rc != 0:
+                raise HbfError(rc, "hbf_get_tile_times")
+        return rec, ns
+
+    def set_tile_balance(self, on: bool):
+        rc = lib().hbf_set_tile_balance(self._h, 1 if on else 0)
+        if rc != 0:
+            raise HbfError(rc, "hbf_set_tile_balance")
 
     # ---- thermal ------------------------------------------------------------------------------
     def set_thermal_path(self, generic_only: bool):

@@ -183,6 +183,54 @@ def test_full_size_batch_with_refresh_claims(full):
     ctx.destroy()
 
 
+def test_tile_sizes_from_measurements_leave_every_result_as_it_was():
+    """A batch that fills one wave of the device (two tiles per SM) leaves each tile's time; the next batches cut their tiles
+    in proportion to the measured rates.  Results must not move: three batches with the measurements on (fixed sizes,
+    then sizes from one and from two measurements) against the same batch with them off, and against the oracle."""
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2609_09800_b200 import build, hbf
+    build.build()
+    n = 24_000_123
+    w = wl.capacity_mode(n=n, seed=5)
+    d_acc = torch.from_numpy(w.acc.view(np.int64).reshape(-1)).cuda()
+    d_comp = torch.empty(n, dtype=torch.int64, device="cuda"); d_stall = torch.empty_like(d_comp)
+    d_status = torch.empty(n, dtype=torch.uint8, device="cuda")
+    outs, lens = [], []
+    for on in (False, True):
+        ctx = hbf.Context(w.profile)
+        for r in w.ranges:
+            ctx.register_range(*r)
+        ctx.set_tile_balance(on)
+        d_ds = torch.empty(ctx.n_dies * 6, dtype=torch.int64, device="cuda")
+        ws = ctx.workspace(n)
+        for k in range(3 if on else 1):
+            ctx.reset()
+            assert ctx.submit_batch(d_acc, n, d_comp, d_stall, d_status, d_ds, ws) == 0 and ctx.last_result()["code"] == 0
+            outs.append((d_comp.cpu().numpy(), d_stall.cpu().numpy(), d_ds.cpu().numpy().copy(), ctx.get_busy_until(), ctx.last_result()))
+            rec, ns = ctx.tile_times()
+            if on:
+                sms = torch.cuda.get_device_properties(0).multi_processor_count
+                assert rec.size == 2 * sms and int(rec.astype(np.int64).sum()) == n and (ns > 0).sum() >= rec.size - 4
+                lens.append(rec.copy())
+            else:
+                assert rec.size == 0
+        ctx.destroy()
+    assert np.unique(lens[0]).size <= 6                       # the two nominal sizes, give or take a quantum, and the ragged last tile
+    assert np.unique(lens[2]).size > 8 and not np.array_equal(lens[1], lens[0])      # sized tile by tile
+    base = outs[0]
+    for o in outs[1:]:
+        assert np.array_equal(o[0], base[0]) and np.array_equal(o[1], base[1]) and np.array_equal(o[2], base[2])
+        assert np.array_equal(o[3], base[3]) and o[4] == base[4]
+    orc = hbfo.Oracle(w.profile)
+    for r in w.ranges:
+        orc.register_range(*r)
+    _, c_o, s_o, _, ds_o = orc.submit(w.acc)
+    assert np.array_equal(base[0], c_o) and np.array_equal(base[1], s_o)
+    assert np.array_equal(base[3], orc.busy_until())
+
+
 @pytest.mark.parametrize("which", ["decode_weights", "prefix_kv"])
 def test_serving_configurations_at_full_size_element_by_element(which):
     """The 21 M-access decode-weight stream and the 28 M-access prefix-KV stream (the two serving configurations),
