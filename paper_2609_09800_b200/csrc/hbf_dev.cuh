@@ -94,7 +94,7 @@ struct Workspace {
     int64_t *in_agg;                     // [tiles][queues][2]: per-tile, per-queue max-plus aggregate (S, M)
     int64_t *in_bin;                     // [tiles][queues]: busy-until entering each tile
     void *in_tile;                       // [tiles] stall bookkeeping of the in-order path
-    void *in_head;                       // [tiles][queues][8]: the first accesses of every (tile, queue), contiguous, for the fix-up
+    void *in_head;                       // [tiles]: the first 8 accesses of every (tile, queue) for the fix-up: a tile's first entries, then each queue's other seven
     uint8_t *in_headcnt;                 // [tiles][queues]: how many of them exist; 0xff marks a queue for the straggle pass
     uint16_t *in_qid;                    // [tiles][stride]: queue of each of the first records of every tile (0xffff: not modeled), for the straggle pass
     uint32_t *bus_xfer;                  // [n] transfer time of every read (only with the channel-bus stage on)

@@ -182,6 +182,13 @@ __device__ __forceinline__ Served serve_terms_geom(const FastGeom &g, const Mode
 // The first kInHead accesses of every (tile, queue), as the serve pass saw them: all the fix-up needs in the common case.
 constexpr int kInHead = 8;
 struct InHead { int64_t m, s; uint32_t xo, idx; };       // arrival + service, service, transfer | op << 31, batch index
+// Where entry ci of (tile, queue) sits: a tile's first entries side by side (the fix-up reads the first entry of every
+// queue: one coalesced stretch instead of a record every 192 bytes), then every queue's later entries side by side (read
+// only for the queues still behind, all seven at once).
+__device__ __forceinline__ uint64_t head_slot(uint32_t tile, uint32_t R, uint32_t q, uint32_t ci) {
+    const uint64_t base = (uint64_t)tile * R * kInHead;
+    return ci == 0u ? base + q : base + R + (uint64_t)q * (kInHead - 1) + (ci - 1u);
+}
 
 // ======================================================================================================
 // serve.  RESERVE = false: the streaming pass over every tile, every queue taken as idle at the tile's start.
@@ -489,7 +496,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, const __grid_c
                         const uint32_t ci = c0[u] + rank1[u] - 1u;
                         if (ci < (uint32_t)kInHead) {
                             InHead h; h.m = a[u] + v[u].s; h.s = v[u].s; h.xo = v[u].xfer | (v[u].op << 31); h.idx = (uint32_t)tile_begin + i[u];
-                            in_head[((uint64_t)tile * R + qi[u]) * kInHead + ci] = h;
+                            in_head[head_slot(tile, R, qi[u], ci)] = h;
                         }
                         if (last[u] && c1[u] != c0[u] && c1[u] == (uint32_t)kInHead) atomicAdd(&s_heads_full, 1u);
                     }
@@ -725,7 +732,7 @@ k_inorder_fixstraggle(const hbf_access_t *__restrict__ acc, uint64_t n, const __
         }
 #pragma unroll
         for (int k = 0; k < kInStrQueuesPerThread; ++k)
-            if (c[k] > 0u) e0[k] = in_head[((uint64_t)tile * R + (uint32_t)(k * kInStrThreads + tid)) * kInHead];
+            if (c[k] > 0u) e0[k] = in_head[head_slot(tile, R, (uint32_t)(k * kInStrThreads + tid), 0u)];
 #pragma unroll
         for (int k = 0; k < kInStrQueuesPerThread; ++k) {
             const uint32_t q = (uint32_t)(k * kInStrThreads + tid);
@@ -744,11 +751,12 @@ k_inorder_fixstraggle(const hbf_access_t *__restrict__ acc, uint64_t n, const __
             const uint32_t q = deep[d];
             const uint64_t idx = (uint64_t)tile * R + q;
             const uint32_t c = in_headcnt[idx];
-            const InHead *h = in_head + idx * kInHead;
+            const InHead *h = in_head + head_slot(tile, R, q, 1u) - 1;       // h[j], j >= 1: the queue's later entries, side by side
             FixRun f; f.B = Bt[q]; f.Bs = kNegInf; f.dstall = 0; f.max_c = INT64_MIN; f.settled = false;
             InHead g[4];
+            g[0] = in_head[head_slot(tile, R, q, 0u)];       // (listed queues have at least one entry)
 #pragma unroll
-            for (int j = 0; j < 4; ++j) if ((uint32_t)j < c) g[j] = h[j];
+            for (int j = 1; j < 4; ++j) if ((uint32_t)j < c) g[j] = h[j];
 #pragma unroll
             for (int j = 0; j < 4; ++j) if ((uint32_t)j < c) fix_entry(f, g[j], completion, stall);
             if (!f.settled && c > 4u) {
