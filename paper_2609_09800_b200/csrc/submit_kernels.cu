@@ -790,11 +790,15 @@ __global__ void k_bus_check(BatchCtrl *bc) { if (bc->code != HBF_OK) bc->skip = 
 
 // entry j of the sorted order as a map on its channel's bus
 __device__ __forceinline__ BusMap bus_entry(uint64_t j, const uint64_t *__restrict__ ks, const uint32_t *__restrict__ is, bool have_idx,
-                                            const uint32_t *__restrict__ xfer, const int64_t *__restrict__ bus_busy,
-                                            uint32_t *idx_out, uint32_t *ch_out, int64_t *plain_out) {
+                                            const uint32_t *__restrict__ xfer, const uint32_t *xs, const int64_t *__restrict__ bus_busy,
+                                            uint32_t *idx_out, uint32_t *ch_out, int64_t *plain_out, uint32_t *x_out) {
     const uint64_t key = ks[j];
     const uint32_t ch = (uint32_t)(key >> kIssueBits), idx = have_idx ? is[j] : (uint32_t)j;
-    const int64_t done = (int64_t)(key & kIssueMask), x = (int64_t)xfer[idx];
+    // the transfer time: by batch index from the array the keys kernel wrote (a gather), or in sorted order from the copy the
+    // reduce pass made of what it gathered
+    const uint32_t xr = xs ? xs[j] : xfer[idx];
+    *x_out = xr;
+    const int64_t done = (int64_t)(key & kIssueMask), x = (int64_t)xr;
     const bool head = j == 0 || (uint32_t)(ks[j - 1] >> kIssueBits) != ch;
     BusMap m; m.S = x; m.M = (head ? max(bus_busy[ch], done) : done) + x; m.f = head ? 1 : 0;
     *idx_out = idx; *ch_out = ch; *plain_out = done + x;
@@ -802,13 +806,14 @@ __device__ __forceinline__ BusMap bus_entry(uint64_t j, const uint64_t *__restri
 }
 
 __global__ void __launch_bounds__(kBusThreads)
-k_bus_reduce(const BatchCtrl *bc, const uint64_t *k0, const uint64_t *k1, const uint32_t *i0, const uint32_t *i1,
+k_bus_reduce(const BatchCtrl *bc, const uint64_t *k0, const uint64_t *k1, uint32_t *i0, uint32_t *i1,
              const uint32_t *__restrict__ xfer, const int64_t *__restrict__ bus_busy, ScanDesc *agg) {
     __shared__ BusMap s_warp[kBusThreads / 32];
     if (bc->skip) return;
     const uint64_t m = bc->n_ready;
     const uint32_t np = bc->plan.n_passes;
     const uint64_t *ks = (np & 1u) ? k1 : k0; const uint32_t *is = (np & 1u) ? i1 : i0;
+    uint32_t *xs = np != 0u ? ((np & 1u) ? i0 : i1) : nullptr;      // the index buffer the sort no longer needs (no passes: the order is the batch's)
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     for (uint64_t tile = blockIdx.x; tile * kBusTile < m; tile += gridDim.x) {
         BusMap mine = bus_identity();
@@ -816,8 +821,9 @@ k_bus_reduce(const BatchCtrl *bc, const uint64_t *k0, const uint64_t *k1, const 
         for (int u = 0; u < kBusItems; ++u) {
             const uint64_t j = first + u;
             if (j >= m) break;
-            uint32_t idx, ch; int64_t plain;
-            mine = bus_then(mine, bus_entry(j, ks, is, np != 0u, xfer, bus_busy, &idx, &ch, &plain));
+            uint32_t idx, ch, x; int64_t plain;
+            mine = bus_then(mine, bus_entry(j, ks, is, np != 0u, xfer, nullptr, bus_busy, &idx, &ch, &plain, &x));
+            if (xs) xs[j] = x;                               // for the apply pass: it reads this in order instead of gathering again
         }
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) { const BusMap p = bus_shfl_up(mine, o); if (lane >= o) mine = bus_then(p, mine); }
@@ -870,6 +876,7 @@ k_bus_apply(const hbf_access_t *__restrict__ acc, BatchCtrl *bc, const uint64_t 
     const uint64_t m = bc->n_ready;
     const uint32_t np = bc->plan.n_passes;
     const uint64_t *ks = (np & 1u) ? k1 : k0; const uint32_t *is = (np & 1u) ? i1 : i0;
+    const uint32_t *xs = np != 0u ? ((np & 1u) ? i0 : i1) : nullptr;    // the transfer times in sorted order, left by the reduce pass
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     long long moved = 0, max_c = INT64_MIN;
     for (uint64_t tile = blockIdx.x; tile * kBusTile < m; tile += gridDim.x) {
@@ -879,7 +886,8 @@ k_bus_apply(const hbf_access_t *__restrict__ acc, BatchCtrl *bc, const uint64_t 
 #pragma unroll
         for (int u = 0; u < kBusItems; ++u) {
             const uint64_t j = first + u;
-            if (j < m) { e[u] = bus_entry(j, ks, is, np != 0u, xfer, bus_busy, &idx[u], &ch[u], &plain[u]); mine = bus_then(mine, e[u]); }
+            uint32_t x;
+            if (j < m) { e[u] = bus_entry(j, ks, is, np != 0u, xfer, xs, bus_busy, &idx[u], &ch[u], &plain[u], &x); mine = bus_then(mine, e[u]); }
             else { e[u] = bus_identity(); idx[u] = 0; ch[u] = 0; plain[u] = 0; }
         }
         BusMap incl = mine;
