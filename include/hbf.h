@@ -230,7 +230,8 @@ HBF_API int hbf_reset(hbf_ctx *ctx);                                            
  * issue order, or has such a long service time (and more than 8,192 records), is refused with HBF_E_INVAL.  All give
  * identical results. */
 HBF_API int hbf_set_path(hbf_ctx *ctx, int32_t path);
-/* Tile sizes of the in-order path from measurements, on by default: when a batch fills one wave of the device (two tiles
+/* (No step of the method is defined by the next two calls: they steer how the library spreads a batch over the device.)
+ * Tile sizes of the in-order path from measurements, on by default: when a batch fills one wave of the device (two tiles
  * per SM), every block of the streaming pass leaves how long its tile took, and later batches size their tiles in
  * proportion to the rates measured at each place (the SMs of a device are not equally fast, and the pass lasts as long as
  * its slowest block).  The record is read through an asynchronous copy that nothing waits for.  Results never depend on
