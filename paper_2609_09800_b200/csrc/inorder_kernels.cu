@@ -44,6 +44,7 @@ namespace hbf {
 constexpr int kInThreads = HBF_IN_THREADS;               // threads of a serve block
 constexpr int kInBlocksPerSM = HBF_IN_BLOCKS;            // resident serve blocks per SM
 constexpr int kInWarps = kInThreads / 32;
+constexpr uint32_t kInTagStride = kInMaxQueues + 32;      // bytes of a warp's table of lane numbers: one per queue, one per lane
 #ifndef HBF_IN_ROWS
 #define HBF_IN_ROWS 2
 #endif
@@ -257,6 +258,8 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, const __grid_c
     uint32_t *st_bp_lo = st_br_hi + n_dies, *st_bp_hi = st_bp_lo + n_dies;
     uint32_t *st_nr = st_bp_hi + n_dies, *st_np = st_nr + n_dies;
     uint32_t *st_claims = st_np + n_dies;                 // refresh quanta claimed on each die (claims variant)
+    // per warp and row of a turn: a byte per queue (which lane of the row holds it) and one per lane
+    uint8_t *warp_tag = reinterpret_cast<uint8_t *>(st_claims + n_dies) + (uint32_t)(threadIdx.x >> 5) * (kInRows * kInTagStride);
 
     // Which tile this block serves.  Two blocks share an SM, and the hardware favours the one in the lower warp slots: with
     // equal tiles it finishes about 12 % earlier (measured) and the pass lasts as long as the other one.  So the tiles come in
@@ -399,6 +402,17 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, const __grid_c
                 atomicAdd(&ret.disturb[ret_block_of(mp, ret, off)], npages);
             }
         }
+        // ---- which lanes of a row hold the same queue: every lane writes its number where its queue's entry is in the
+        // warp's own table and reads the entry back (the answer is needed only further down: the latency is covered).
+        // Nothing is ever cleared: a lane reads what a lane of this row wrote.  Accesses that are not modeled have an
+        // entry per lane.  (`match_any` for every row kept the unit that executes it busy three quarters of the time.)
+        uint8_t *tag_at[K];
+        uint32_t tagged[K];
+#pragma unroll
+        for (int u = 0; u < K; ++u) { tag_at[u] = warp_tag + u * kInTagStride + (ready[u] ? v[u].queue : kInMaxQueues + (uint32_t)lane); *tag_at[u] = (uint8_t)lane; }
+        __syncwarp();
+#pragma unroll
+        for (int u = 0; u < K; ++u) tagged[u] = *reinterpret_cast<volatile uint8_t *>(tag_at[u]);
         if (!RESERVE && turn * (uint32_t)(K * 32) < qid_stride) {   // (the stride is a multiple of a turn's records)
 #pragma unroll
             for (int u = 0; u < K; ++u)
@@ -436,19 +450,32 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, const __grid_c
 #pragma unroll
         for (int u = 0; u < K; ++u) {
             a[u] = issue[u] + (int64_t)(v[u].op ? v[u].xfer : 0u);   // arrival at the queue: a program's data is transferred first
-            const uint32_t q = ready[u] ? v[u].queue : (0x10000u | (uint32_t)lane);
-            const unsigned peers = __match_any_sync(0xffffffffu, q);
-            const unsigned le = peers & le_mask;
-            rank1[u] = (uint32_t)__popc(le);               // this access is the rank1-th of its queue in the row
-            last[u] = ready[u] && (peers >> lane) == 1u;    // no later access of this queue in the row
+            rank1[u] = 1u;                                  // this access is the rank1-th of its queue in the row
+            last[u] = ready[u];                             // no later access of this queue in the row
+            pc[u] = HEADS ? 1u : 0u;                        // accesses of this queue in the row
             S[u] = v[u].s; M[u] = a[u] + v[u].s;
-            if (__any_sync(0xffffffffu, rank1[u] > 1u)) {    // one row in five: some queue occurs twice
-                if (!__any_sync(0xffffffffu, rank1[u] > 2u)) {
+            // A lane that did not read its own number back shares its queue with another lane of the row: one row in five.
+            const bool loser = tagged[u] != (uint32_t)lane;
+            if (__any_sync(0xffffffffu, loser)) {
+                // Second round: the lanes that lost write again.  In a pair the winner now reads its peer's number and the
+                // loser its own; a loser that loses again has two peers or more, and only then is the row matched in full.
+                if (loser) *tag_at[u] = (uint8_t)lane;
+                __syncwarp();
+                const uint32_t t2 = *reinterpret_cast<volatile uint8_t *>(tag_at[u]);
+                if (!__any_sync(0xffffffffu, loser && t2 != (uint32_t)lane)) {
                     // pairs only (nearly always): the second lane of a pair composes its peer's map with its own
-                    const int src = rank1[u] == 2u ? __ffs((int)(le & ~(1u << lane))) - 1 : lane;
-                    const int64_t mp_ = __shfl_sync(0xffffffffu, M[u], src), sp_ = __shfl_sync(0xffffffffu, (int64_t)v[u].s, src);
-                    if (rank1[u] == 2u) { M[u] = max(mp_, a[u]) + v[u].s; S[u] = sp_ + v[u].s; }
+                    const uint32_t peer = loser ? tagged[u] : t2;                  // the lane itself when it has none
+                    const bool second = peer < (uint32_t)lane;
+                    const int64_t mp_ = __shfl_sync(0xffffffffu, M[u], (int)peer), sp_ = __shfl_sync(0xffffffffu, (int64_t)v[u].s, (int)peer);
+                    if (second) { M[u] = max(mp_, a[u]) + v[u].s; S[u] = sp_ + v[u].s; rank1[u] = 2u; }
+                    if (peer > (uint32_t)lane) last[u] = false;
+                    if (HEADS && peer != (uint32_t)lane) pc[u] = 2u;
                 } else {
+                    const unsigned peers = __match_any_sync(0xffffffffu, ready[u] ? v[u].queue : (0x10000u | (uint32_t)lane));
+                    const unsigned le = peers & le_mask;
+                    rank1[u] = (uint32_t)__popc(le);
+                    last[u] = ready[u] && (peers >> lane) == 1u;
+                    pc[u] = HEADS ? (uint32_t)__popc(peers) : 0u;
                     const uint32_t n_it = __reduce_max_sync(0xffffffffu, rank1[u]);
                     unsigned rem = le & ~(1u << lane);       // earlier lanes of the same queue, lowest first
                     S[u] = 0; M[u] = kNegInf;
@@ -462,7 +489,6 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, const __grid_c
             }
             qi[u] = ready[u] ? v[u].queue : 0u;
             pq[u] = qst + qi[u];
-            pc[u] = HEADS ? (uint32_t)__popc(peers) : 0u;
         }
         // ---- the queue updates, in row order: everything they need is in registers before the wait ---------------
         if (turn > 0) {
@@ -1066,8 +1092,8 @@ static bool measured_shares(const TileBalance &rec, uint32_t n_tiles, double *sh
     return true;
 }
 
-// dynamic shared memory of the serve kernel: the per-queue state and the per-die counters
-size_t inorder_serve_smem(uint32_t n_dies) { return (size_t)kInMaxQueues * 16 + (size_t)n_dies * 28; }
+// dynamic shared memory of the serve kernel: the per-queue state, the per-die counters, every warp's tables of lane numbers
+size_t inorder_serve_smem(uint32_t n_dies) { return (size_t)kInMaxQueues * 16 + (size_t)n_dies * 28 + (size_t)kInWarps * kInRows * kInTagStride; }
 static size_t inorder_straggle_smem() {
     return (size_t)kInMaxQueues * 16 + (size_t)kInStrKeep * 24 + (size_t)kInMaxQueues * 4 + (size_t)kInStrMaxStragglers * (kInStrList * 2 + 4);
 }
