@@ -250,7 +250,7 @@ k_sort_pass(int pass, uint64_t n, BatchCtrl *ctrl, DevState *state, uint32_t *hi
   for (;;) {                                  // persistent: tiles are taken in order from a counter
     __syncthreads();                          // shared memory of the previous tile is no longer read
     if (tid == 0) s_tile = atomicAdd(&ctrl->tile_counter[pass], 1u);
-    for (int i = tid; i < kSortWarps * kRadix; i += kSortThreads) s_cnt[i] = 0u;
+    for (int i = tid; i < kSortWarps * kRadix; i += kSortThreads) { s_cnt[i] = 0u; reinterpret_cast<uint32_t *>(s_keys)[i] = 0u; }
     __syncthreads();
     const uint32_t tile = s_tile;
     if (tile >= n_tiles) break;
@@ -270,28 +270,52 @@ k_sort_pass(int pass, uint64_t n, BatchCtrl *ctrl, DevState *state, uint32_t *hi
         key[j] = i < n ? kin[i] : ~0ull;                            // padding (no real key is all ones) ranks behind every real key
     }
     // the next pass's digit of every key, counted now (the high digits of neighbouring keys are mostly equal, the low ones
-    // mostly all different: one vote tells the two cases apart)
+    // mostly all different: one vote over the warp's 256 keys tells the two cases apart)
     if (count_next) {
+        auto next_digit = [&](int j) {
+            return wbase + j * 32 + lane < n ? (uint32_t)(compact_key(key[j], lo_bits, hi_bits) >> next_shift) & next_mask : 0xffffffffu;
+        };
+        const uint32_t d0 = __shfl_sync(0xffffffffu, next_digit(0), 0);
+        bool one_digit = d0 != 0xffffffffu;
 #pragma unroll
-        for (int j = 0; j < kSortItems; ++j) {
-            const bool valid = wbase + j * 32 + lane < n;
-            const uint32_t d2 = valid ? (uint32_t)(compact_key(key[j], lo_bits, hi_bits) >> next_shift) & next_mask : 0xffffffffu;
-            const uint32_t d0 = __shfl_sync(0xffffffffu, d2, 0);
-            if (__all_sync(0xffffffffu, d2 == d0)) { if (lane == 0 && valid) atomicAdd(&s_next[d2], 32u); }
-            else if (valid) atomicAdd(&s_next[d2], 1u);
+        for (int j = 0; j < kSortItems; ++j) one_digit = one_digit && next_digit(j) == d0;
+        if (__all_sync(0xffffffffu, one_digit)) {
+            if (lane == 0) atomicAdd(&s_next[d0], 32u * kSortItems);
+        } else {
+#pragma unroll
+            for (int j = 0; j < kSortItems; ++j) {
+                const uint32_t d2 = next_digit(j);
+                if (d2 != 0xffffffffu) atomicAdd(&s_next[d2], 1u);
+            }
         }
     }
-    // rank inside the warp, in memory order
+    // rank inside the warp, in memory order.  Which lanes hold the same digit is found through shared memory: every lane
+    // sets its bit in the digit's word of the warp's table (which lies where the tile's keys are put later) and reads the
+    // word back; the highest of the lanes clears it and moves the warp's count on.  (`match_any` per key kept the unit that
+    // executes it busier than any other: a pass took 2.4 ms at 200 M.)  A warp whose keys all share the digit needs no table.
     uint32_t *wcnt = s_cnt + warp * kRadix;
+    uint32_t *wmask = reinterpret_cast<uint32_t *>(s_keys) + warp * kRadix;
+    const uint32_t dg0 = __shfl_sync(0xffffffffu, digit_of(key[0]), 0);
+    bool one_digit = true;
 #pragma unroll
-    for (int j = 0; j < kSortItems; ++j) {
-        const uint32_t dg = digit_of(key[j]);
-        const unsigned peers = __match_any_sync(0xffffffffu, dg);
-        const uint32_t before = wcnt[dg];
-        rank[j] = before + (uint32_t)__popc(peers & lanemask_lt());
-        __syncwarp();
-        if ((peers >> lane) <= 1u) wcnt[dg] = before + (uint32_t)__popc(peers);    // highest peer lane writes
-        __syncwarp();
+    for (int j = 0; j < kSortItems; ++j) one_digit = one_digit && digit_of(key[j]) == dg0;
+    if (__all_sync(0xffffffffu, one_digit)) {                // all 256 keys of the warp: the high digits of input in order
+#pragma unroll
+        for (int j = 0; j < kSortItems; ++j) rank[j] = (uint32_t)(j * 32 + lane);
+        if (lane == 0) wcnt[dg0] = 32u * kSortItems;
+    } else {
+#pragma unroll
+        for (int j = 0; j < kSortItems; ++j) {
+            const uint32_t dg = digit_of(key[j]);
+            const uint32_t before = wcnt[dg];
+            atomicOr(&wmask[dg], 1u << lane);
+            __syncwarp();
+            const unsigned peers = wmask[dg];
+            rank[j] = before + (uint32_t)__popc(peers & lanemask_lt());
+            __syncwarp();
+            if ((peers >> lane) <= 1u) { wcnt[dg] = before + (uint32_t)__popc(peers); wmask[dg] = 0u; }    // highest peer lane writes
+            __syncwarp();
+        }
     }
     __syncthreads();
 
