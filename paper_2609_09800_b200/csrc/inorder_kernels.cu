@@ -107,7 +107,8 @@ __device__ __forceinline__ Served serve_terms_fast(const FastRange &f, const Mod
     r.s = (int64_t)npages * (r.op ? mp.t_prog_ns : mp.t_read_ns);
     return r;
 }
-// The common configuration once more, laid out for the serve pass: seven 16-byte vectors in shared memory, every field a
+// The common configuration once more, laid out for the serve pass (a kernel argument: its fields are operands of the
+// instructions that use them, which measured 1.8 % faster than seven 16-byte vectors in shared memory), every field a
 // 32-bit operand where the values allow it (page times and the transfer table's reach below 2^32).
 struct __align__(16) FastGeom {
     uint64_t base, length;                                  // the one registered range
@@ -125,7 +126,7 @@ __device__ __forceinline__ bool fast_geom_ok(const FastRange &f, const ModelPara
     return f.on != 0u && mp.pow2_geom != 0u && mp.xfer_tab_max_cb != 0u && mp.t_read_ns < (1ll << 32) && mp.t_prog_ns < (1ll << 32) &&
            pages * (uint64_t)max(mp.t_read_ns, mp.t_prog_ns) < (1ull << 32);
 }
-__device__ __forceinline__ FastGeom make_fast_geom(const FastRange &f, const ModelParams &mp) {
+__host__ __device__ __forceinline__ FastGeom make_fast_geom(const FastRange &f, const ModelParams &mp) {
     FastGeom g;
     g.base = f.base; g.length = f.length; g.media_offset = f.media_offset; g.perms = f.perms; g.stripe_shift = mp.stripe_shift;
     g.ch_mask = mp.channels - 1u; g.ch_shift = mp.ch_shift; g.die_mask = mp.dies - 1u; g.chdie_shift = mp.ch_shift + mp.die_shift;
@@ -228,20 +229,19 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, const __grid_c
                 const int64_t *__restrict__ in_bin, InTile *in_tile, InHead *__restrict__ in_head, uint8_t *__restrict__ in_headcnt,
                 const int64_t *__restrict__ busy, const unsigned long long *claim_limit_p, uint32_t *die_claims,
                 const __grid_constant__ RetDev ret, uint16_t *__restrict__ in_qid, uint32_t qid_stride,
-                TileBalance *bal, uint32_t bal_seq) {
+                TileBalance *bal, uint32_t bal_seq, const __grid_constant__ FastGeom geom) {
     extern __shared__ __align__(16) unsigned char in_smem[];
     __shared__ long long s_red[2];
     __shared__ unsigned long long s_t0;                   // when this block took its tile (0: its time is not recorded)
     __shared__ uint32_t s_heads_full;                     // queues whose head entries are complete
     __shared__ ModelParams mp;                            // measured: reads from shared memory beat reads of the argument
     __shared__ FastRange fast_range;
-    __shared__ FastGeom geom;
 
     if (ctrl->skip || ctrl->run_sort) return;             // (run_sort set this early: the batch went to the sort path at its start)
     if (RESERVE && (!ctrl->inorder_used || !in_tile[blockIdx.x].reserve)) return;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const RangeSnap &rs = *ranges_g;                      // read through the cache; the common configuration does not touch it
-    if (tid == 0) { mp = mp_arg; fast_range = fast_arg; geom = make_fast_geom(fast_arg, mp_arg); }
+    if (tid == 0) { mp = mp_arg; fast_range = fast_arg; }
     if (DEBT && !RESERVE && tid == 0 && blockIdx.x == 0) ret.st->observed_inline = 1u;
     const uint32_t R = mp_arg.n_queues, n_dies = mp_arg.n_dies;
     const int64_t q_ppm = ctrl->q_ppm;
@@ -513,19 +513,16 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, const __grid_c
 #pragma unroll
         for (int u = 0; u < K; ++u) {
             if (valid[u]) {
-                int64_t done = issue[u], st = 0;             // not modeled: completion = issue, no stall (a refused batch is cleared at the end)
-                if (ready[u]) {
-                    done = B[u] + (int64_t)(v[u].op ? 0u : v[u].xfer); // a read's data is transferred after its service
-                    st = done - issue[u];
-                    sum_stall += st; max_c = max(max_c, (long long)done);
-                    if (HEADS) {
-                        const uint32_t ci = c0[u] + rank1[u] - 1u;
-                        if (ci < (uint32_t)kInHead) {
-                            InHead h; h.m = a[u] + v[u].s; h.s = v[u].s; h.xo = v[u].xfer | (v[u].op << 31); h.idx = (uint32_t)tile_begin + i[u];
-                            in_head[head_slot(tile, R, qi[u], ci)] = h;
-                        }
-                        if (last[u] && c1[u] != c0[u] && c1[u] == (uint32_t)kInHead) atomicAdd(&s_heads_full, 1u);
+                const int64_t done = ready[u] ? B[u] + (int64_t)(v[u].op ? 0u : v[u].xfer) : issue[u];   // a read's data is transferred after its service;
+                const int64_t st = done - issue[u];                                                    // not modeled: completion = issue, no stall
+                sum_stall += st; max_c = max(max_c, ready[u] ? (long long)done : (long long)INT64_MIN);
+                if (HEADS && ready[u]) {
+                    const uint32_t ci = c0[u] + rank1[u] - 1u;
+                    if (ci < (uint32_t)kInHead) {
+                        InHead h; h.m = a[u] + v[u].s; h.s = v[u].s; h.xo = v[u].xfer | (v[u].op << 31); h.idx = (uint32_t)tile_begin + i[u];
+                        in_head[head_slot(tile, R, qi[u], ci)] = h;
                     }
+                    if (last[u] && c1[u] != c0[u] && c1[u] == (uint32_t)kInHead) atomicAdd(&s_heads_full, 1u);
                 }
                 // results are written once and not read again by this pass: streaming stores
                 __stcs(reinterpret_cast<long long *>(completion_t + i[u]), (long long)done);
@@ -1461,7 +1458,7 @@ cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st) {
         k<<<n_tiles, kInThreads, smem_serve, st>>>(a.acc, n, tmap, a.ranges, a.mp, a.fast, a.ctrl, a.status, a.ws.in_agg,
                                                    a.stats_stage, a.completion, a.stall, a.ws.in_bin, tiles, heads, a.ws.in_headcnt,
                                                    a.busy, a.claim_limit, a.die_claims, debt ? *a.ret : RetDev{}, a.ws.in_qid, qid_stride,
-                                                   bal ? bal->dev : nullptr, bal_seq);
+                                                   bal ? bal->dev : nullptr, bal_seq, make_fast_geom(a.fast, a.mp));
     };
     serve(false);
     if (bal) {                                               // the tiles' times, for later batches; nothing waits for this copy
