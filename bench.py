@@ -66,7 +66,7 @@ def parse_args():
     ap.add_argument("--n", type=int, default=200_000_000, help="accesses per batch (default: the capacity-mode config)")
     ap.add_argument("--path", default="auto", choices=["auto", "sort", "sort_full"])
     ap.add_argument("--e2e-steps", type=int, default=5)
-    ap.add_argument("--e2e-chunk", type=int, default=12_500_000, help="records per chunk of the end-to-end pipeline")
+    ap.add_argument("--e2e-chunk", type=int, default=4_000_000, help="records per chunk of the end-to-end pipeline")
     ap.add_argument("--cpu-sample", type=int, default=20_000_000)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")

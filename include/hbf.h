@@ -134,7 +134,7 @@ HBF_API int hbf_submit_batch(hbf_ctx *ctx, const hbf_access_t *d_acc, uint64_t n
 
 /* The same service for a batch that lives in HOST memory (no step of the method is defined by this call, so it cites
  * none: it is hbf_submit_batch behind a copy pipeline).  The batch is cut into chunks of `chunk` records (0 = a default
- * of 12.5 M); the copy-in of chunk k+1, the service of chunk k and the read-back of chunk k-1 run on three streams of
+ * of 4 M); the copy-in of chunk k+1, the service of chunk k and the read-back of chunk k-1 run on three streams of
  * the library, so both directions of the link are busy while the kernels run.  Equivalent to one hbf_submit_batch per
  * chunk, in order: for records in issue order that is the same as one batch.
  * h_acc [n] host, read only; h_completion_ns, h_stall_ns [n] host; h_die_stats [channels*dies] host, nullable: totals

@@ -552,7 +552,7 @@ int hbf_submit_host(hbf_ctx *c, const hbf_access_t *h_acc, uint64_t n, int64_t *
     if (!c || !on_own_device(c)) return HBF_E_INVAL;
     if (c->terminal) return HBF_E_LINK_SHUTDOWN;
     if (n && (!h_acc || !h_completion_ns || !h_stall_ns)) return HBF_E_INVAL;
-    if (chunk == 0) chunk = 12500000;
+    if (chunk == 0) chunk = 4000000;
     chunk = std::min<uint64_t>(std::min<uint64_t>(chunk, HBF_MAX_BATCH), std::max<uint64_t>(n, 1));
     int rc = host_pipe_prepare(c, chunk);
     if (rc != HBF_OK) return rc;

@@ -274,6 +274,47 @@ def test_inorder_hot_queue_and_equal_issue(hbf):
     compare_batch(g, o, acc)
 
 
+def test_inorder_rows_with_lanes_on_one_queue(hbf):
+    """The serve pass takes a row of 32 consecutive records at a time and has a path of its own for rows in which no two
+    records share a queue, for rows with pairs only, and for rows where three or more do.  Every kind of row, built by
+    hand on the 2,048 queues of the capacity geometry: no pair, one pair (neighbours, far apart, first and last lane),
+    two and three pairs, a triple, four neighbours (the parts of a split access look like this), a triple beside a pair,
+    all 32 on one queue, a pair broken by a record that is not modeled, and rows that repeat the queues of the row
+    before."""
+    rng = np.random.default_rng(21)
+    labels = lambda pairs: [next((g for g, lanes in enumerate(pairs) if l in lanes), 100 + l) for l in range(32)]
+    patterns = [labels([]), labels([(3, 4)]), labels([(2, 29)]), labels([(0, 31)]), labels([(1, 9), (10, 30)]),
+                labels([(0, 1), (15, 16), (30, 31)]), labels([(5, 6, 20)]), labels([(8, 9, 10, 11)]),
+                labels([(4, 12, 28), (7, 8)]), [0] * 32, labels([(13, 14)]), labels([(6, 7, 8, 9), (20, 21, 22, 23)])]
+    rows, native_at = [], []
+    prev_map = None
+    for k in range(420):                                           # 13,440 records: beyond the small-batch route
+        pat = patterns[int(rng.integers(0, len(patterns)))]
+        if k % 7 == 3 and prev_map is not None:
+            m = prev_map                                           # the same queues as in the row before
+        else:
+            units = rng.permutation(2048)
+            m = {g: int(units[j]) for j, g in enumerate(sorted(set(range(200))))}
+        prev_map = m
+        rows.append([m[g] for g in pat])
+        if pat == patterns[10]:
+            native_at.append(32 * k + 13)                          # the first of the pair is outside every range
+    unit = np.array(rows, np.uint64).reshape(-1)
+    n = unit.shape[0]
+    acc = np.zeros(n, hbfo.ACCESS_DTYPE)
+    acc["addr"] = np.uint64(wl.RANGE_BASE) + unit * np.uint64(65536) + rng.integers(0, 4, n).astype(np.uint64) * np.uint64(16384)
+    acc["addr"][native_at] = 1 << 20
+    acc["issue_ns"] = np.sort(rng.integers(0, 40_000_000, n))
+    acc["issue_ns"][5000:5064] = acc["issue_ns"][5000]             # equal issue times across two rows
+    acc["bytes"] = rng.choice([128, 4096, 16384], n)
+    acc["flags"] = rng.random(n) < 0.2
+    prof = wl.load_profile("nominal", **wl.GEOMETRY["capacity"])
+    for path in (hbf.PATH_INORDER, hbf.PATH_SORT):
+        g, o = contexts(hbf, prof, [(wl.RANGE_BASE, 2048 * 65536, 3, 0, 0, 0)], path)
+        compare_batch(g, o, acc)
+        compare_batch(g, o, acc)                                   # again, on the queues the first pass filled
+
+
 @pytest.mark.parametrize("geo", [dict(channels=3, dies=5, planes=2, page_bytes=4096, stripe_bytes=16384),
                                  dict(channels=8, dies=4, planes=2, page_bytes=16384, stripe_bytes=16384, queue_level=1),
                                  dict(channels=32, dies=8, planes=8, page_bytes=16384, stripe_bytes=16384),
