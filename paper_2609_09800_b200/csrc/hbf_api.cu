@@ -675,6 +675,12 @@ int hbf_enable_retention(hbf_ctx *c, const hbf_retention_config_t *cfg) {
     r.ppb = cfg->pages_per_block; r.bpp = cfg->blocks_per_plane; r.bpz = cfg->blocks_per_zone; r.max_pec = cfg->max_pec;
     r.disturb_limit = cfg->disturb_limit; r.n_regions = c->thermal ? c->td.n_regions : 1u;
     r.div_ppb = make_div64_host(cfg->pages_per_block); r.div_bpp = make_div64_host(cfg->blocks_per_plane);
+    {
+        const uint64_t ppb = cfg->pages_per_block, bpp = cfg->blocks_per_plane;
+        r.pow2 = ((ppb & (ppb - 1)) == 0 && (bpp & (bpp - 1)) == 0 && ppb * bpp < (1ull << 32) && c->mp.pow2_geom && c->mp.stripe_shift < 32) ? 1u : 0u;
+        r.ppb_shift = 0;
+        while ((1ull << r.ppb_shift) < ppb) ++r.ppb_shift;
+    }
     r.accel = cfg->accel; r.lead = cfg->lead_threshold; r.l_ref_s = cfg->l_ref_s; r.t_ref_k = cfg->t_ref_c + 273.15;
     r.ea_over_kb = cfg->ea_ev / 8.617333262e-5;                             // Boltzmann constant in eV/K
     r.n_blocks = nb; r.plan_cap = nb * cfg->pages_per_block;

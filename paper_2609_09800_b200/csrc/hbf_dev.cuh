@@ -234,6 +234,7 @@ struct RetState {
 struct RetDev {
     uint32_t ppb, bpp, bpz, max_pec, disturb_limit, n_regions;
     Div64 div_ppb, div_bpp;              // exact division by pages_per_block and by blocks_per_plane
+    uint32_t pow2, ppb_shift;            // pages_per_block and blocks_per_plane are powers of two (and a plane has fewer than 2^32 pages): shifts do
     double accel, lead, l_ref_s, t_ref_k, ea_over_kb;
     uint64_t n_blocks, plan_cap;
     double *damage; uint32_t *disturb, *pec, *epoch_of; uint8_t *worn;
