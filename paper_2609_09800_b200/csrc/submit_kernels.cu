@@ -206,7 +206,7 @@ k_hist(const uint64_t *__restrict__ keys, uint64_t n, const BatchCtrl *ctrl, uin
 // =====================================================================================================
 // one onesweep pass: stable partition of (key, index) by one digit, in a single sweep.  Tiles take
 // their number from a counter (so every predecessor of a running tile has started), rank their keys
-// per warp with match_any, publish the tile's digit counts and look back over earlier tiles for the
+// per warp (equal digits are found through bit masks in shared memory), publish the tile's digit counts and look back over earlier tiles for the
 // running totals.  Look-back words carry flag and count in one 32-bit word.
 // =====================================================================================================
 constexpr int kSortThreads = 512;
