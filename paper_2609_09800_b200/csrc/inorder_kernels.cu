@@ -489,14 +489,19 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, const __grid_c
                     rank1[u] = (uint32_t)__popc(le);
                     last[u] = ready[u] && (peers >> lane) == 1u;
                     pc[u] = HEADS ? (uint32_t)__popc(peers) : 0u;
-                    const uint32_t n_it = __reduce_max_sync(0xffffffffu, rank1[u]);
-                    unsigned rem = le & ~(1u << lane);       // earlier lanes of the same queue, lowest first
-                    S[u] = 0; M[u] = kNegInf;
-                    for (uint32_t it = 0; it < n_it; ++it) {
-                        const int src = rem ? __ffs((int)rem) - 1 : lane;
-                        const int64_t ab = __shfl_sync(0xffffffffu, a[u], src), sb = __shfl_sync(0xffffffffu, (int64_t)v[u].s, src);
-                        if (rem || it + 1u == rank1[u]) { M[u] = max(M[u], ab) + sb; S[u] += sb; }   // its peers first, then the lane's own
-                        rem &= rem - 1u;
+                    // Every lane composes the maps of the lanes of its queue up to its own by doubling: it holds the map of a
+                    // stretch of them that ends with itself and the lane before that stretch, takes that lane's stretch in front
+                    // of its own, and goes on from the lane before that one; ceil(log2(most lanes on one queue)) rounds.
+                    // (One lane after the other took as many rounds as lanes: 12.7 warp instructions per part where the parts
+                    // of a split access, neighbours on one queue, fill the rows, against 9 per access unsplit.)
+                    const unsigned before = le & ~(1u << lane);
+                    int prev = before ? 31 - __clz((int)before) : -1;
+                    const uint32_t n_max = __reduce_max_sync(0xffffffffu, rank1[u]);
+                    for (uint32_t span = 1; span < n_max; span <<= 1) {
+                        const int src = prev >= 0 ? prev : lane;
+                        const int64_t Se = __shfl_sync(0xffffffffu, S[u], src), Me = __shfl_sync(0xffffffffu, M[u], src);
+                        const int pe = __shfl_sync(0xffffffffu, prev, src);
+                        if (prev >= 0) { M[u] = max((int64_t)(Me + S[u]), M[u]); S[u] = Se + S[u]; prev = pe; }
                     }
                 }
             }
