@@ -148,6 +148,23 @@ __device__ __forceinline__ uint64_t compact_key(uint64_t key, uint32_t lo_bits, 
     return lo | (hi << lo_bits);
 }
 
+// The digit of one pass straight from the key: the digit's bits lie in the issue field, in the queue field, or (one pass
+// at most) in both; two shifts and two masks instead of compacting the whole key first.
+struct DigitSel { uint32_t sh_lo, m_lo, sh_hi, m_hi, up; uint64_t raw; };      // raw: the digit's bits where they lie in the key
+__device__ __forceinline__ DigitSel digit_sel(const SortPlan &p, int pass) {
+    const uint32_t shift = p.shift[pass], bits = p.bits[pass];
+    const uint32_t n_lo = shift < p.lo_bits ? min(bits, p.lo_bits - shift) : 0u, n_hi = bits - n_lo;
+    DigitSel d;
+    d.sh_lo = n_lo ? shift : 0u; d.m_lo = (1u << n_lo) - 1u;
+    d.sh_hi = n_hi ? (max(shift, p.lo_bits) - p.lo_bits) + (uint32_t)kIssueBits : 0u; d.m_hi = (1u << n_hi) - 1u;
+    d.up = n_lo;
+    d.raw = ((uint64_t)d.m_lo << d.sh_lo) | ((uint64_t)d.m_hi << d.sh_hi);
+    return d;
+}
+__device__ __forceinline__ uint32_t digit_at(uint64_t key, const DigitSel &d) {
+    return ((uint32_t)(key >> d.sh_lo) & d.m_lo) | (((uint32_t)(key >> d.sh_hi) & d.m_hi) << d.up);
+}
+
 __global__ void k_plan(BatchCtrl *ctrl, int force_full) {
     if (threadIdx.x != 0 || ctrl->skip || !ctrl->run_sort) return;
     if (ctrl->n_fault) { ctrl->code = HBF_E_ACCESS_FAULT; ctrl->skip = 1; return; }
@@ -179,15 +196,16 @@ k_hist(const uint64_t *__restrict__ keys, uint64_t n, const BatchCtrl *ctrl, uin
     if (ctrl->skip || !ctrl->run_sort) return;
     const SortPlan p = ctrl->plan;
     if (p.n_passes == 0) return;
+    const DigitSel sel0 = digit_sel(p, 0);
     for (int i = threadIdx.x; i < kMaxPasses * kRadix; i += kHistThreads) sh[i] = 0u;
     __syncthreads();
     const uint64_t stride = (uint64_t)gridDim.x * kHistThreads;
     const uint64_t n_round = (n + 31ull) & ~31ull;         // whole warps stay in the loop together
     for (uint64_t i = (uint64_t)blockIdx.x * kHistThreads + threadIdx.x; i < n_round; i += stride) {
         const bool valid = i < n;
-        const uint64_t ck = valid ? compact_key(keys[i], p.lo_bits, p.hi_bits) : 0ull;
+        const uint64_t ck = valid ? keys[i] : 0ull;
         for (uint32_t k = 0; k < 1u; ++k) {
-            const uint32_t d = valid ? (uint32_t)(ck >> p.shift[k]) & ((1u << p.bits[k]) - 1u) : 0xffffffffu;
+            const uint32_t d = valid ? digit_at(ck, sel0) : 0xffffffffu;
             // the high digits of neighbouring keys are mostly equal, the low ones mostly all different: one vote tells the
             // two cases apart, and neither needs the lane-by-lane match (measured: 8.0 ms of a 58 ms sort at 200 M with it)
             const uint32_t d0 = __shfl_sync(0xffffffffu, d, 0);
@@ -234,10 +252,8 @@ k_sort_pass(int pass, uint64_t n, BatchCtrl *ctrl, DevState *state, uint32_t *hi
     const SortPlan &pl = ctrl->plan;
     if (pass >= (int)pl.n_passes) return;
     const bool count_next = pass + 1 < (int)pl.n_passes;
-    const uint32_t next_shift = count_next ? pl.shift[pass + 1] : 0u, next_mask = count_next ? (1u << pl.bits[pass + 1]) - 1u : 0u;
+    const DigitSel sel = digit_sel(pl, pass), sel_next = digit_sel(pl, count_next ? pass + 1 : pass);
     if (threadIdx.x < kRadix) s_next[threadIdx.x] = 0u;
-    const uint32_t lo_bits = pl.lo_bits, hi_bits = pl.hi_bits, shift = pl.shift[pass];
-    const uint32_t dmask = (1u << pl.bits[pass]) - 1u;
     const uint64_t *kin = (pass & 1) ? keys1 : keys0;
     uint64_t *kout = (pass & 1) ? keys0 : keys1;
     const uint32_t *iin = (pass & 1) ? idx1 : idx0;
@@ -259,10 +275,11 @@ k_sort_pass(int pass, uint64_t n, BatchCtrl *ctrl, DevState *state, uint32_t *hi
     const uint64_t base = (uint64_t)tile * kSortTile;
     if (tid < kRadix) desc_next[(uint64_t)tile * kRadix + tid] = 0u;     // ready for the pass after this one
 
+    const bool has_pad = base + kSortTile > n;                        // only the last tile holds padding
     // load, warp-striped: the warp's chunk is contiguous and item j of lane l sits at j*32 + l
     uint64_t key[kSortItems]; uint32_t rank[kSortItems];
     // (a key's digit is computed where it is needed: eight registers fewer than keeping it)
-    auto digit_of = [&](uint64_t k) { return k == ~0ull ? (uint32_t)(kRadix - 1) : (uint32_t)(compact_key(k, lo_bits, hi_bits) >> shift) & dmask; };
+    auto digit_of = [&](uint64_t k) { return (has_pad && k == ~0ull) ? (uint32_t)(kRadix - 1) : digit_at(k, sel); };
     const uint64_t wbase = base + (uint64_t)warp * (32 * kSortItems);
 #pragma unroll
     for (int j = 0; j < kSortItems; ++j) {
@@ -273,14 +290,15 @@ k_sort_pass(int pass, uint64_t n, BatchCtrl *ctrl, DevState *state, uint32_t *hi
     // mostly all different: one vote over the warp's 256 keys tells the two cases apart)
     if (count_next) {
         auto next_digit = [&](int j) {
-            return wbase + j * 32 + lane < n ? (uint32_t)(compact_key(key[j], lo_bits, hi_bits) >> next_shift) & next_mask : 0xffffffffu;
+            return wbase + j * 32 + lane < n ? digit_at(key[j], sel_next) : 0xffffffffu;
         };
-        const uint32_t d0 = __shfl_sync(0xffffffffu, next_digit(0), 0);
-        bool one_digit = d0 != 0xffffffffu;
+        // (equal digits: the keys agree on the digit's bits; a tile with padding takes the other branch)
+        const uint64_t k0 = __shfl_sync(0xffffffffu, key[0], 0);
+        uint64_t differ = has_pad ? ~0ull : 0ull;
 #pragma unroll
-        for (int j = 0; j < kSortItems; ++j) one_digit = one_digit && next_digit(j) == d0;
-        if (__all_sync(0xffffffffu, one_digit)) {
-            if (lane == 0) atomicAdd(&s_next[d0], 32u * kSortItems);
+        for (int j = 0; j < kSortItems; ++j) differ |= (key[j] ^ k0) & sel_next.raw;
+        if (__all_sync(0xffffffffu, differ == 0ull)) {
+            if (lane == 0) atomicAdd(&s_next[digit_at(k0, sel_next)], 32u * kSortItems);
         } else {
 #pragma unroll
             for (int j = 0; j < kSortItems; ++j) {
@@ -295,11 +313,12 @@ k_sort_pass(int pass, uint64_t n, BatchCtrl *ctrl, DevState *state, uint32_t *hi
     // executes it busier than any other: a pass took 2.4 ms at 200 M.)  A warp whose keys all share the digit needs no table.
     uint32_t *wcnt = s_cnt + warp * kRadix;
     uint32_t *wmask = reinterpret_cast<uint32_t *>(s_keys) + warp * kRadix;
-    const uint32_t dg0 = __shfl_sync(0xffffffffu, digit_of(key[0]), 0);
-    bool one_digit = true;
+    const uint64_t key0 = __shfl_sync(0xffffffffu, key[0], 0);
+    uint64_t differ = has_pad ? ~0ull : 0ull;
 #pragma unroll
-    for (int j = 0; j < kSortItems; ++j) one_digit = one_digit && digit_of(key[j]) == dg0;
-    if (__all_sync(0xffffffffu, one_digit)) {                // all 256 keys of the warp: the high digits of input in order
+    for (int j = 0; j < kSortItems; ++j) differ |= (key[j] ^ key0) & sel.raw;
+    const uint32_t dg0 = digit_at(key0, sel);
+    if (__all_sync(0xffffffffu, differ == 0ull)) {           // all 256 keys of the warp: the high digits of input in order
 #pragma unroll
         for (int j = 0; j < kSortItems; ++j) rank[j] = (uint32_t)(j * 32 + lane);
         if (lane == 0) wcnt[dg0] = 32u * kSortItems;
@@ -382,7 +401,7 @@ k_sort_pass(int pass, uint64_t n, BatchCtrl *ctrl, DevState *state, uint32_t *hi
     const int cnt = (int)min((uint64_t)kSortTile, n - base);
     for (int i = tid; i < cnt; i += kSortThreads) {
         const uint64_t k = s_keys[i];
-        const uint32_t d = (uint32_t)(compact_key(k, lo_bits, hi_bits) >> shift) & dmask;
+        const uint32_t d = digit_at(k, sel);
         const uint32_t g = (uint32_t)i + s_delta[d];
         kout[g] = k; iout[g] = s_idx[i];
     }
