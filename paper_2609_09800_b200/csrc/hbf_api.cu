@@ -695,6 +695,11 @@ int hbf_enable_retention(hbf_ctx *c, const hbf_retention_config_t *cfg) {
     if ((rc = dev_copy<uint32_t>(c, &r.rank, nullptr, nb)) != HBF_OK) return rc;
     if ((rc = dev_copy<unsigned long long>(c, &r.die_len, nullptr, c->mp.n_dies)) != HBF_OK) return rc;
     if ((rc = dev_copy<unsigned long long>(c, &r.chan_len, nullptr, c->mp.channels)) != HBF_OK) return rc;
+    r.chan_tab = nullptr;
+    if (c->mp.channels <= kRetTabChannels) {
+        const size_t C = c->mp.channels;
+        if ((rc = dev_copy<uint32_t>(c, &r.chan_tab, nullptr, 2 * C + 1 + C * C)) != HBF_OK) return rc;
+    }
     if ((rc = dev_copy<uint32_t>(c, &r.die_claims, nullptr, c->mp.n_dies)) != HBF_OK) return rc;
     if ((rc = dev_copy<uint32_t>(c, &r.tile_count, nullptr, (HBF_MAX_BATCH + 1023) / 1024 + 1)) != HBF_OK) return rc;
     if ((rc = dev_copy<double>(c, &r.rate, nullptr, r.n_regions)) != HBF_OK) return rc;

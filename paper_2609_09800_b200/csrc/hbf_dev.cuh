@@ -231,6 +231,7 @@ struct RetState {
     uint32_t epoch;
     uint32_t observed_inline;            // the in-order serve pass has counted this batch's reads into the disturb counters
 };
+constexpr uint32_t kRetTabChannels = 128;
 struct RetDev {
     uint32_t ppb, bpp, bpz, max_pec, disturb_limit, n_regions;
     Div64 div_ppb, div_bpp;              // exact division by pages_per_block and by blocks_per_plane
@@ -242,6 +243,7 @@ struct RetDev {
     uint32_t *plan;                      // [plan_cap] ring of quanta (block * ppb + page), position modulo plan_cap
     uint32_t *rank;                      // [blocks] rank of a newly eligible block in its die's (zone, plane, block) order
     unsigned long long *die_len, *chan_len;   // quanta the epoch in progress adds per die, per channel
+    uint32_t *chan_tab;                  // the channels' lengths sorted, their running sums, and per channel the sorted lengths of the channels before it (null: more than kRetTabChannels channels)
     uint32_t *die_claims;                // [dies] quanta claimed on each die by the batch in progress
     uint32_t *tile_count;                // [tiles of 1,024 records] modeled accesses, claim window
     double *rate, *region_temp;          // [regions] damage per block of this epoch; temperatures

@@ -300,6 +300,43 @@ __global__ void k_ret_chan(RetDev r, uint32_t channels, uint32_t dies) {
     }
     __syncthreads();
     if (threadIdx.x == 0) r.st->epoch_total = s_total;
+    // For the plan kernel: the lengths in ascending order with their running sums, and for every channel the lengths of
+    // the channels before it in ascending order.  With them the place of a quantum among the channels, a sum of
+    // min(length, x) over all channels and a count of longer channels before its own, takes two binary searches
+    // instead of a pass over the channels.  (Every length, and their sum, is below 2^32.)
+    if (r.chan_tab) {
+        uint32_t *sorted = r.chan_tab, *run = r.chan_tab + channels, *before = r.chan_tab + 2 * channels + 1;
+        for (uint32_t c = threadIdx.x; c < channels; c += blockDim.x) {
+            const unsigned long long lc = r.chan_len[c];
+            uint32_t at = 0;
+            for (uint32_t j = 0; j < channels; ++j) { const unsigned long long lj = r.chan_len[j]; at += (lj < lc || (lj == lc && j < c)) ? 1u : 0u; }
+            sorted[at] = (uint32_t)lc;
+        }
+        for (uint32_t k = threadIdx.x; k < channels * channels; k += blockDim.x) {
+            const uint32_t ch = k / channels, c = k % channels;      // channel c among the channels before ch
+            if (c >= ch) continue;
+            const unsigned long long lc = r.chan_len[c];
+            uint32_t at = 0;
+            for (uint32_t j = 0; j < ch; ++j) { const unsigned long long lj = r.chan_len[j]; at += (lj < lc || (lj == lc && j < c)) ? 1u : 0u; }
+            before[(size_t)ch * channels + at] = (uint32_t)lc;
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            uint32_t sum = 0;
+            for (uint32_t k = 0; k < channels; ++k) { run[k] = sum; sum += sorted[k]; }
+            run[channels] = sum;
+        }
+    }
+}
+
+// how many of the n ascending values at tab are at most x
+__device__ __forceinline__ uint32_t count_at_most(const uint32_t *__restrict__ tab, uint32_t n, uint32_t x) {
+    uint32_t lo = 0, len = n;
+    while (len > 0u) {
+        const uint32_t half = len >> 1;
+        if (__ldg(tab + lo + half) <= x) { lo += half + 1u; len -= half + 1u; } else len = half;
+    }
+    return lo;
 }
 
 // one warp per block, its lanes over the block's pages.  Every length and rank of an epoch is below 2^32 (a quantum id
@@ -326,9 +363,15 @@ k_ret_emit(RetDev r, uint32_t channels, uint32_t dies, uint32_t planes) {
                 r_ch += min(len, r_die) + ((d < di && len > r_die) ? 1u : 0u);
             }
             uint32_t pos = 0;
-            for (uint32_t c = 0; c < channels; ++c) {
-                const uint32_t len = (uint32_t)__ldg(r.chan_len + c);
-                pos += min(len, r_ch) + ((c < ch && len > r_ch) ? 1u : 0u);
+            if (r.chan_tab) {
+                const uint32_t k = count_at_most(r.chan_tab, channels, r_ch);                       // channels no longer than r_ch: all of theirs
+                pos = __ldg(r.chan_tab + channels + k) + r_ch * (channels - k);                       // the others: r_ch each
+                pos += ch - count_at_most(r.chan_tab + 2 * channels + 1 + (size_t)ch * channels, ch, r_ch);   // and one more of every longer channel before this one
+            } else {
+                for (uint32_t c = 0; c < channels; ++c) {
+                    const uint32_t len = (uint32_t)__ldg(r.chan_len + c);
+                    pos += min(len, r_ch) + ((c < ch && len > r_ch) ? 1u : 0u);
+                }
             }
             uint64_t slot = base_mod + pos;
             if (slot >= r.plan_cap) slot -= r.plan_cap;
