@@ -182,11 +182,14 @@ __device__ __forceinline__ Served serve_terms_geom(const FastGeom &g, const Mode
     return r;
 }
 // The first kInHead accesses of every (tile, queue), as the serve pass saw them: all the fix-up needs in the common case.
-constexpr int kInHead = 8;
+// (Six, measured on the capacity stream at loads 0.3 to 0.9: eight cost 2.5 % more at every load for the table's traffic
+// and bookkeeping and fell back to a second pass at the same load, between 0.6 and 0.7; five or fewer are faster still
+// at low load but need the second pass from 0.6 on.)
+constexpr int kInHead = 6;
 struct InHead { int64_t m, s; uint32_t xo, idx; };       // arrival + service, service, transfer | op << 31, batch index
 // Where entry ci of (tile, queue) sits: a tile's first entries side by side (the fix-up reads the first entry of every
 // queue: one coalesced stretch instead of a record every 192 bytes), then every queue's later entries side by side (read
-// only for the queues still behind, all seven at once).
+// only for the queues still behind, all of them at once).
 __device__ __forceinline__ uint64_t head_slot(uint32_t tile, uint32_t R, uint32_t q, uint32_t ci) {
     const uint64_t base = (uint64_t)tile * R * kInHead;
     return ci == 0u ? base + q : base + R + (uint64_t)q * (kInHead - 1) + (ci - 1u);
