@@ -230,7 +230,7 @@ HBF_API int hbf_reset(hbf_ctx *ctx);                                            
  * issue order, or has such a long service time (and more than 8,192 records), is refused with HBF_E_INVAL.  All give
  * identical results. */
 HBF_API int hbf_set_path(hbf_ctx *ctx, int32_t path);
-/* (No step of the method is defined by the next two calls: they steer how the library spreads a batch over the device.)
+/* (No step of the method is defined by the next three calls: they steer how the library spreads a batch over the device.)
  * Tile sizes of the in-order path from measurements, on by default: when a batch fills one wave of the device (two tiles
  * per SM), every block of the streaming pass leaves how long its tile took, and later batches size their tiles in
  * proportion to the rates measured at each place (the SMs of a device are not equally fast, and the pass lasts as long as
@@ -242,6 +242,11 @@ HBF_API int hbf_set_tile_balance(hbf_ctx *ctx, int32_t on);
  * SM and kind of block) the records it had and the nanoseconds its block took (0: taken out of turn, not measured).
  * Waits for the stream.  *count = number of tiles (0: no such batch yet); with records_out and ns_out (host, [cap]) the values. */
 HBF_API int hbf_get_tile_times(hbf_ctx *ctx, uint32_t *records_out, uint32_t *ns_out, uint32_t cap, uint32_t *count);
+/* Head entries of the in-order path: how many of the first accesses of every (tile, queue) the streaming pass keeps for the
+ * pass that corrects the results of queues that were busy when their tile began.  0 (the default): from measurements, as
+ * the tile sizes (the number follows how many queues the last batch that filled a wave left to the slower correction:
+ * 3 to 6); 1 to 6: fixed.  Results never depend on it.  HBF_E_INVAL above 6.  Waits for nothing. */
+HBF_API int hbf_set_head_entries(hbf_ctx *ctx, uint32_t entries);
 /* Thermal step implementation: 0 (default) runs the whole step in one launch of a thread-block cluster when
  * the grid fits its registers and shared memory (up to 32,768 cells with the portable cluster of 8 blocks, 65,536 where
  * the device can place a cluster of 16), else one launch per substep; 1 always uses the latter.

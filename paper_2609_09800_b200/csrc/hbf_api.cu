@@ -457,6 +457,13 @@ int hbf_set_tile_balance(hbf_ctx *c, int32_t on) {
     if (!c) return HBF_E_INVAL;
     c->bal.on = on != 0;
     if (c->bal.pinned) memset(c->bal.pinned, 0, sizeof(TileBalance));      // (measurements start over)
+    c->bal.depth = 0; c->bal.depth_seen = 0;
+    return HBF_OK;
+}
+
+int hbf_set_head_entries(hbf_ctx *c, uint32_t entries) {
+    if (!c || entries > 6u) return HBF_E_INVAL;
+    c->bal.depth_fixed = entries;
     return HBF_OK;
 }
 

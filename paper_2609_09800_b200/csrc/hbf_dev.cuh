@@ -168,9 +168,10 @@ constexpr uint32_t kInBalMax = 320;      // tiles this can describe (two per SM)
 struct TileBalance {
     uint32_t claim[kInBalMax];           // number of the last batch in which the tile was taken (hand-out by SM and kind)
     uint32_t len[kInBalMax], ns[kInBalMax];   // records of the tile, and how long its block took (0: taken out of turn, not measured)
+    uint32_t strag_seq, strag_max, strag_flagged, strag_depth;   // of batch strag_seq: most straggling queues in a tile, tiles served a second time, head entries kept
     uint32_t first[kInBalMax + 1];       // device only: where the tiles of the batch in flight begin
 };
-struct TileBalanceHost { TileBalance *dev = nullptr, *pinned = nullptr; uint32_t seq = 0; bool on = true; };
+struct TileBalanceHost { TileBalance *dev = nullptr, *pinned = nullptr; uint32_t seq = 0; bool on = true; uint32_t depth = 0, depth_fixed = 0, depth_seen = 0; };   // depth: head entries per (tile, queue) of the next batch (0: the most); depth_fixed != 0: set by the caller; depth_seen: batch whose record was read last
 InTileMap inorder_tile_map(uint64_t n, int sm_count, bool by_table);   // by_table: a full wave gets exactly two tiles per SM, placed by a table
 // per-tile bookkeeping of the stall total: as-if-idle sum, fix-up corrections, and the exact sum of a re-served tile
 struct InTile { long long spec_sum, fix_delta, true_sum; uint32_t reserve; uint32_t stragglers; };

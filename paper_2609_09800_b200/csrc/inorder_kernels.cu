@@ -232,7 +232,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, const __grid_c
                 const int64_t *__restrict__ in_bin, InTile *in_tile, InHead *__restrict__ in_head, uint8_t *__restrict__ in_headcnt,
                 const int64_t *__restrict__ busy, const unsigned long long *claim_limit_p, uint32_t *die_claims,
                 const __grid_constant__ RetDev ret, uint16_t *__restrict__ in_qid, uint32_t qid_stride,
-                TileBalance *bal, uint32_t bal_seq, const __grid_constant__ FastGeom geom) {
+                TileBalance *bal, uint32_t bal_seq, const __grid_constant__ FastGeom geom, const uint32_t head_depth) {
     extern __shared__ __align__(16) unsigned char in_smem[];
     __shared__ long long s_red[2];
     __shared__ unsigned long long s_t0;                   // when this block took its tile (0: its time is not recorded)
@@ -246,6 +246,7 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, const __grid_c
     const RangeSnap &rs = *ranges_g;                      // read through the cache; the common configuration does not touch it
     if (tid == 0) { mp = mp_arg; fast_range = fast_arg; }
     if (DEBT && !RESERVE && tid == 0 && blockIdx.x == 0) ret.st->observed_inline = 1u;
+    if (!RESERVE && bal && tid == 0 && blockIdx.x == 0) { bal->strag_seq = bal_seq; bal->strag_max = 0u; bal->strag_flagged = 0u; bal->strag_depth = head_depth; }
     const uint32_t R = mp_arg.n_queues, n_dies = mp_arg.n_dies;
     const int64_t q_ppm = ctrl->q_ppm;
     const Div64 div_q = ctrl->div_q;
@@ -522,8 +523,8 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, const __grid_c
             B[u] = max((int64_t)(state.x + S[u]), M[u]);
             uint32_t inc = 0u;
             if (HEADS) {
-                c0[u] = min((uint32_t)state.y & 0xffu, (uint32_t)kInHead);
-                inc = min(pc[u], (uint32_t)kInHead - c0[u]);
+                c0[u] = min((uint32_t)state.y & 0xffu, head_depth);
+                inc = min(pc[u], head_depth - c0[u]);
                 c1[u] = c0[u] + inc;
             }
             if (last[u]) *pq[u] = make_longlong2(B[u], state.y + (S[u] << 8) + (long long)inc);
@@ -539,11 +540,11 @@ k_inorder_serve(const hbf_access_t *__restrict__ acc, uint64_t n, const __grid_c
                 sum_stall += st; max_c = max(max_c, ready[u] ? (long long)done : (long long)INT64_MIN);
                 if (HEADS && ready[u]) {
                     const uint32_t ci = c0[u] + rank1[u] - 1u;
-                    if (ci < (uint32_t)kInHead) {
+                    if (ci < head_depth) {
                         InHead h; h.m = a[u] + v[u].s; h.s = v[u].s; h.xo = v[u].xfer | (v[u].op << 31); h.idx = (uint32_t)tile_begin + i[u];
                         in_head[head_slot(tile, R, qi[u], ci)] = h;
                     }
-                    if (last[u] && c1[u] != c0[u] && c1[u] == (uint32_t)kInHead) atomicAdd(&s_heads_full, 1u);
+                    if (last[u] && c1[u] != c0[u] && c1[u] == head_depth) atomicAdd(&s_heads_full, 1u);
                 }
                 // results are written once and not read again by this pass: streaming stores
                 __stcs(reinterpret_cast<long long *>(completion_t + i[u]), (long long)done);
@@ -732,7 +733,8 @@ k_inorder_fixstraggle(const hbf_access_t *__restrict__ acc, uint64_t n, const __
                       const __grid_constant__ FastRange fast_arg, BatchCtrl *ctrl,
                       const int64_t *__restrict__ in_bin, const InHead *__restrict__ in_head,
                       const uint8_t *__restrict__ in_headcnt, int64_t *completion, int64_t *stall, InTile *in_tile,
-                      const unsigned long long *claim_limit_p, const uint16_t *__restrict__ in_qid, uint32_t qid_stride) {
+                      const unsigned long long *claim_limit_p, const uint16_t *__restrict__ in_qid, uint32_t qid_stride,
+                      const uint32_t head_depth, TileBalance *bal) {
     extern __shared__ __align__(16) unsigned char str_smem[];
     __shared__ ModelParams mp;
     __shared__ FastRange fast_range;
@@ -810,7 +812,7 @@ k_inorder_fixstraggle(const hbf_access_t *__restrict__ acc, uint64_t n, const __
                 for (int j = 4; j < kInHead; ++j) if ((uint32_t)j < c) fix_entry(f, g[j - 4], completion, stall);
             }
             max_c = max(max_c, f.max_c);                     // (true completions: valid whoever writes them last)
-            if (!f.settled && c == (uint32_t)kInHead) {
+            if (!f.settled && c == head_depth) {
                 // still backlogged after its head entries: the loop below serves this queue again from the tile's
                 // start (Bt[q] still holds the entering value) and accounts for all of its corrections
                 const uint32_t place = atomicAdd(&s_stragglers, 1u);
@@ -823,6 +825,10 @@ k_inorder_fixstraggle(const hbf_access_t *__restrict__ acc, uint64_t n, const __
     }
     __syncthreads();
     const uint32_t stragglers = s_stragglers;
+    if (bal && tid == 0) {                                   // what the number of head entries of later batches follows from
+        atomicMax(&bal->strag_max, stragglers);
+        if (stragglers >= min(max(8u, R / 4u), (uint32_t)kInStrMaxStragglers)) atomicAdd(&bal->strag_flagged, 1u);
+    }
     // many queues far behind: the re-serve pass takes the whole tile (one block serves it again from end to end, which costs
     // as much as the serve pass itself, so the bar is as high as this loop's tables allow)
     if (stragglers >= min(max(8u, R / 4u), (uint32_t)kInStrMaxStragglers)) {
@@ -1453,6 +1459,26 @@ cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st) {
         if (e != cudaSuccess) return e;
         tmap.first = bal->dev->first; tmap.max_tile = max_tile;
     }
+    // Head entries per (tile, queue).  Fewer cost the serve pass less (a shorter stretch of every tile with the head
+    // bookkeeping, a smaller table) and leave more queues to the straggle pass; past 254 of those in a tile the tile is
+    // served a second time.  So the number follows what the last batch needed: one fewer while no tile had 148 straggling
+    // queues (an entry fewer leaves about 1.3 times as many: 100, 130, 164, 224 per tile with 6, 5, 4, 3 entries on the
+    // capacity stream at half load, so 148 become about 200), one more above 200, all of them after a tile was served twice.  Results do not
+    // depend on it.
+    uint32_t depth = (uint32_t)kInHead;
+    if (bal) {
+        if (bal->depth == 0u || bal->depth > (uint32_t)kInHead) bal->depth = (uint32_t)kInHead;
+        const TileBalance &rec = *bal->pinned;
+        if (rec.strag_seq != 0u && rec.strag_seq != bal->depth_seen && rec.strag_depth == bal->depth) {
+            bal->depth_seen = rec.strag_seq;
+            if (rec.strag_flagged != 0u) bal->depth = (uint32_t)kInHead;
+            else if (rec.strag_max > 200u && bal->depth < (uint32_t)kInHead) ++bal->depth;
+            else if (rec.strag_max < 148u && bal->depth > 3u) --bal->depth;
+        }
+        depth = bal->depth_fixed != 0u ? std::min<uint32_t>(bal->depth_fixed, (uint32_t)kInHead) : bal->depth;
+    } else if (a.bal && a.bal->depth_fixed != 0u) {
+        depth = std::min<uint32_t>(a.bal->depth_fixed, (uint32_t)kInHead);
+    }
     const uint64_t tile_records = tmap.max_tile;
     if (n_tiles > inorder_tiles_bound(n)) return cudaErrorInvalidValue;       // the workspace is carved for that many
     const uint32_t R = a.mp.n_queues, nd = a.mp.n_dies;
@@ -1479,19 +1505,19 @@ cudaError_t launch_inorder(const SubmitArgs &a, cudaStream_t st) {
         k<<<n_tiles, kInThreads, smem_serve, st>>>(a.acc, n, tmap, a.ranges, a.mp, a.fast, a.ctrl, a.status, a.ws.in_agg,
                                                    a.stats_stage, a.completion, a.stall, a.ws.in_bin, tiles, heads, a.ws.in_headcnt,
                                                    a.busy, a.claim_limit, a.die_claims, debt ? *a.ret : RetDev{}, a.ws.in_qid, qid_stride,
-                                                   bal ? bal->dev : nullptr, bal_seq, make_fast_geom(a.fast, a.mp));
+                                                   bal ? bal->dev : nullptr, bal_seq, make_fast_geom(a.fast, a.mp), depth);
     };
     serve(false);
-    if (bal) {                                               // the tiles' times, for later batches; nothing waits for this copy
-        cudaError_t e = cudaMemcpyAsync(bal->pinned, bal->dev, offsetof(TileBalance, first), cudaMemcpyDeviceToHost, st);
-        if (e != cudaSuccess) return e;
-    }
     k_inorder_scan<<<(R + kInScanQueues - 1) / kInScanQueues, dim3(kInScanQueues, kInScanChunks), 0, st>>>(
         a.ctrl, a.mp_dev, n_tiles, a.ws.in_agg, a.ws.in_bin, a.busy, a.busy_stage, a.stats_stage, a.path == HBF_PATH_INORDER ? 1 : 0);
     (debt ? k_inorder_fixstraggle<true> : k_inorder_fixstraggle<false>)<<<n_tiles, kInStrThreads, smem_str, st>>>(
         a.acc, n, tmap, a.ranges, a.mp, a.fast, a.ctrl, a.ws.in_bin, heads, a.ws.in_headcnt, a.completion, a.stall, tiles,
-        a.claim_limit, a.ws.in_qid, qid_stride);
+        a.claim_limit, a.ws.in_qid, qid_stride, depth, bal ? bal->dev : nullptr);
     serve(true);
+    if (bal) {                                               // the tiles' times and straggler counts, for later batches; nothing waits for this copy
+        cudaError_t e = cudaMemcpyAsync(bal->pinned, bal->dev, offsetof(TileBalance, first), cudaMemcpyDeviceToHost, st);
+        if (e != cudaSuccess) return e;
+    }
     g_kernel_launches += 4;
     return cudaGetLastError();
 }

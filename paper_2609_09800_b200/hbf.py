@@ -27,7 +27,7 @@ DIE_STATS_DTYPE = np.dtype([(k, "<i8") for k in
 
 EXPORTS = ("hbf_create", "hbf_destroy", "hbf_register_range", "hbf_clear_ranges", "hbf_workspace_bytes",
            "hbf_submit_batch", "hbf_last_result", "hbf_thermal_step", "hbf_force_mode", "hbf_get_mode",
-           "hbf_reset", "hbf_set_path", "hbf_set_tile_balance", "hbf_get_tile_times", "hbf_get_state", "hbf_set_state", "hbf_get_busy_until",
+           "hbf_reset", "hbf_set_path", "hbf_set_tile_balance", "hbf_get_tile_times", "hbf_set_head_entries", "hbf_get_state", "hbf_set_state", "hbf_get_busy_until",
            "hbf_get_pending_energy", "hbf_get_temps", "hbf_euler_limit_ns", "hbf_queue_order", "hbf_strerror",
            "hbf_set_profiling", "hbf_get_profile", "hbf_kernel_launches", "hbf_euler_substeps_static", "hbf_set_thermal_path",
            "hbf_workspace_bytes_paged", "hbf_submit_batch_paged", "hbf_submit_host", "hbf_debug_wait_test",
@@ -133,6 +133,7 @@ def lib():
         L.hbf_reset.argtypes = [vp]
         L.hbf_set_path.argtypes = [vp, i32]
         L.hbf_set_tile_balance.argtypes = [vp, i32]
+        L.hbf_set_head_entries.argtypes = [vp, u32]
         L.hbf_get_tile_times.argtypes = [vp, vp, vp, C.c_uint32, vp]
         L.hbf_set_thermal_path.argtypes = [vp, i32]
         L.hbf_get_state.argtypes = [vp, vp, C.POINTER(C.c_size_t)]
@@ -415,6 +416,11 @@ class Context:
             if rc != 0:
                 raise HbfError(rc, "hbf_get_tile_times")
         return rec, ns
+
+    def set_head_entries(self, entries: int):
+        rc = lib().hbf_set_head_entries(self._h, int(entries))
+        if rc != 0:
+            raise HbfError(rc, "hbf_set_head_entries")
 
     def set_tile_balance(self, on: bool):
         rc = lib().hbf_set_tile_balance(self._h, 1 if on else 0)

@@ -360,6 +360,21 @@ def test_inorder_long_busy_periods(hbf, rho):
     compare_batch(g, o, w.acc)
 
 
+@pytest.mark.parametrize("entries", [1, 2, 3, 4, 5, 6])
+def test_inorder_head_entries_do_not_change_results(hbf, entries):
+    """How many of a (tile, queue)'s first accesses the streaming pass keeps for the correction pass is a matter of speed
+    only (by default the library sets it from what earlier batches needed): with every fixed number the results are the
+    oracle's, on lightly and on heavily loaded queues, twice in a row (the second batch finds every queue busy)."""
+    for w in (wl.capacity_mode(n=600_000, seed=9, rho=0.5), wl.capacity_mode(n=600_000, seed=9, rho=0.85), wl.tiny_uniform(150_000, seed=2, rho=0.9)):
+        g, o = contexts(hbf, w.profile, w.ranges, hbf.PATH_INORDER)
+        g.set_head_entries(entries)
+        compare_batch(g, o, w.acc)
+        compare_batch(g, o, w.acc)
+    g = hbf.Context(w.profile)
+    with pytest.raises(hbf.HbfError):
+        g.set_head_entries(7)
+
+
 # ---- batches of at most 8,192 records in issue order take a route of their own (one launch, a block per 64 queues) ----
 
 @pytest.mark.parametrize("n", [8191, 8192, 8193])
